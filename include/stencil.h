@@ -1,0 +1,159 @@
+/*
+ * stencil.h — C ABI of the sm_100a stencil-sweep library (libstencil_b200.so).
+ *
+ * The operation is the one the paper's case-study protocol defines: a stencil
+ * of radius R is the single-channel (2R+1)^d cross-correlation with zero
+ * padding R and stride 1,
+ *
+ *     out[p] = sum_o  w[o] * in[p + o]        for every grid point p,
+ *
+ * applied once or iterated over time steps (the protocol repeats the sweep and
+ * reports the amortised per-step latency).  This library generalises the
+ * paper's 2D box to 2D/3D, star or box neighbourhoods, fp32 grids.
+ *
+ * Conventions for every call
+ *   - returns a status (STENCIL_OK or a negative STENCIL_ERR_*); never throws,
+ *     aborts or prints; results come back through pointers.
+ *   - dims are slowest axis first: (ny, nx) or (nz, ny, nx); x is contiguous,
+ *     rows are not padded.
+ *   - "HOST" / "DEVICE" beside a pointer says where the memory must live.
+ *   - there is no CPU fallback: without a CUDA device every compute call
+ *     returns STENCIL_ERR_CUDA.
+ */
+#ifndef STENCIL_B200_H
+#define STENCIL_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define STENCIL_API __attribute__((visibility("default")))
+#else
+#define STENCIL_API
+#endif
+
+typedef struct stencil_plan_s* stencil_plan_t;   /* opaque, owned by the library */
+
+enum { STENCIL_STAR = 0, STENCIL_BOX = 1 };      /* shape    */
+enum { STENCIL_ZERO = 0, STENCIL_PERIODIC = 1 }; /* boundary */
+
+enum {
+    STENCIL_OK              =  0,
+    STENCIL_ERR_INVALID     = -1,  /* bad argument (NULL, size, enum, alignment, aliasing)      */
+    STENCIL_ERR_UNSUPPORTED = -2,  /* valid request outside what the kernels cover               */
+    STENCIL_ERR_CUDA        = -3,  /* a CUDA runtime/driver call failed (or no device)           */
+    STENCIL_ERR_ALLOC       = -4,  /* host or device allocation failed                           */
+    STENCIL_ERR_TIMEOUT     = -5   /* a bounded device-side wait gave up (see query_status)      */
+};
+
+/* Kernel families a plan can run.  AUTO lets the plan choose. */
+enum {
+    STENCIL_VARIANT_AUTO    = 0,
+    STENCIL_VARIANT_GENERIC = 1,   /* one thread per point, global-memory gather; any request    */
+    STENCIL_VARIANT_STREAM  = 2,   /* TMA-staged x-y tiles streamed along the slowest axis       */
+    STENCIL_VARIANT_FUSED   = 3    /* STREAM with several time steps fused per pass              */
+};
+
+/* Keys of stencil_plan_set / stencil_plan_get. */
+enum {
+    STENCIL_KEY_VARIANT      = 0,  /* set/get: STENCIL_VARIANT_*                                 */
+    STENCIL_KEY_TILE_X       = 1,  /* set/get: tile width in points (0 = default)                */
+    STENCIL_KEY_TILE_Y       = 2,  /* set/get: tile height in rows   (0 = default)               */
+    STENCIL_KEY_FUSE_STEPS   = 3,  /* set/get: time steps fused per pass (0 = default, 1 = off)  */
+    STENCIL_KEY_LAUNCHES     = 4,  /* get: kernels launched by this plan so far                  */
+    STENCIL_KEY_SCRATCH_BYTES= 5,  /* get: device bytes the plan currently owns as scratch       */
+    STENCIL_KEY_CHUNK_Z      = 6,  /* set/get: planes per CTA along the streamed axis (0 = auto) */
+    STENCIL_KEY_STAGES       = 7,  /* set/get: depth of the shared-memory plane ring (0 = auto)  */
+    STENCIL_KEY_STREAMING_STORE = 8, /* set/get: 1 = write results with evict-first stores       */
+    STENCIL_KEY_ROWS_PER_THREAD = 9  /* set/get: tile rows each thread computes (0 = default)    */
+};
+
+/*
+ * stencil_plan — validate a stencil and prepare to run it.
+ * Paper: "Case-study protocol" (radius R, (2R+1)^d neighbourhood, zero padding
+ * R, stride 1, cross-correlation orientation).
+ *
+ *   plan_out  HOST, receives the handle; set to NULL on any error.
+ *   ndim      2 or 3.
+ *   dims      HOST, ndim entries, slowest axis first, each >= 1.
+ *   radius    R >= 1; R <= 8 (larger: STENCIL_ERR_UNSUPPORTED).
+ *   shape     STENCIL_STAR or STENCIL_BOX.
+ *   weights   HOST, dense (2R+1)^ndim floats in C order, same axis order as
+ *             dims: entry [dz+R][dy+R][dx+R] multiplies in[p+(dz,dy,dx)]
+ *             (byte-for-byte the weight of a 1-channel conv2d/conv3d).  Copied;
+ *             the caller keeps ownership.  STAR is a promise that every
+ *             off-axis entry is exactly zero, and is checked
+ *             (STENCIL_ERR_INVALID otherwise).  Zero entries cost nothing.
+ *   boundary  STENCIL_ZERO (taps outside the grid contribute 0; every grid
+ *             point is an output) or STENCIL_PERIODIC (indices wrap).
+ *
+ * Needs no device memory until the first apply.  Errors: INVALID, UNSUPPORTED,
+ * ALLOC.
+ */
+STENCIL_API int stencil_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radius,
+                 int shape, const float* weights, int boundary);
+
+/*
+ * stencil_apply — enqueue `steps` sweeps on `stream`:  out = S^steps(in).
+ * Paper: "Case-study protocol" (the sweep, and its repetition over time steps
+ * with each step consuming the previous result).
+ *
+ *   in, out   DEVICE, N = prod(dims) floats each, 16-byte aligned, must not
+ *             overlap; caller-owned.  `in` is never written.
+ *   steps     >= 0.  0 copies in to out.  k > 1 iterates; every intermediate
+ *             field is an fp32 grid (ping-pong between `out` and one
+ *             plan-owned scratch grid of N floats, allocated on first need).
+ *   stream    a cudaStream_t (NULL = the legacy default stream).
+ *
+ * Enqueue only: returns without waiting for the GPU.  A plan must not be used
+ * by two applies that overlap in time (they would share the scratch grid).
+ * Errors: INVALID (NULL plan/pointers, misaligned, overlapping, steps < 0),
+ * ALLOC (scratch), CUDA (launch or tensor-map encode failed).
+ */
+STENCIL_API int stencil_apply(stencil_plan_t plan, const float* in, float* out, int steps, void* stream);
+
+/*
+ * stencil_apply_host — the same operation on HOST buffers: copies `in_host`
+ * to a plan-owned device grid, runs stencil_apply, copies the result back to
+ * `out_host` and waits for it.  Pinned host memory makes the copies
+ * asynchronous up to the final wait; pageable memory works but is slower.
+ * `in_host` and `out_host` may be the same buffer.  Allocates two plan-owned
+ * device grids of N floats on first use.
+ */
+STENCIL_API int stencil_apply_host(stencil_plan_t plan, const float* in_host, float* out_host, int steps,
+                       void* stream);
+
+/* stencil_destroy — free the plan and everything it owns.  NULL is a no-op. */
+STENCIL_API int stencil_destroy(stencil_plan_t plan);
+
+/* Static, NUL-terminated description of a status code. */
+STENCIL_API const char* stencil_status_string(int status);
+
+/* Static name of a STENCIL_VARIANT_* value ("generic", "stream", ...). */
+STENCIL_API const char* stencil_variant_name(int variant);
+
+/*
+ * stencil_query_status — wait for the stream of the plan's last apply and
+ * return the device status word: STENCIL_OK, or STENCIL_ERR_TIMEOUT if a
+ * bounded wait inside a kernel expired (the kernel then returned early and
+ * `out` is not valid).  The word is cleared by the query.
+ */
+STENCIL_API int stencil_query_status(stencil_plan_t plan);
+
+/*
+ * stencil_plan_set / stencil_plan_get — tuning knobs and counters
+ * (STENCIL_KEY_*).  Setting a variant the plan cannot run for its
+ * dims/radius/boundary returns STENCIL_ERR_UNSUPPORTED and leaves the plan
+ * unchanged.  `value` of get is HOST.
+ */
+STENCIL_API int stencil_plan_set(stencil_plan_t plan, int key, int64_t value);
+STENCIL_API int stencil_plan_get(stencil_plan_t plan, int key, int64_t* value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STENCIL_B200_H */

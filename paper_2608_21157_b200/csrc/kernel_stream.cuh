@@ -1,0 +1,310 @@
+// STREAM kernels: 3D sweep with a zero boundary, x-y tiles staged by TMA into a
+// shared-memory ring and streamed along the slowest axis (z).
+//
+// One CTA owns a TX x TY tile of the x-y plane and a contiguous range of z.
+// A producer warp issues one TMA tile load per input plane (tile plus halo;
+// everything outside the grid arrives as zero, so the zero boundary costs no
+// branches).  NW consumer warps each own K rows of the tile, one float4 of x
+// per lane.  Every arriving plane is used once, at arrival:
+//
+//   star  - the in-plane taps (x through warp shuffles / the smem halo, y from
+//           smem rows) start the output of that plane; the +-z taps are
+//           applied by forward accumulation: the plane's own-column values
+//           are added into the R outputs still pending, and the last R
+//           own-column values (a register queue) feed the new output.
+//   box   - the plane's (2R+1)^2 in-plane sums for each dz are added into the
+//           2R+1 outputs it touches; the oldest is complete and is stored.
+//
+// Finished outputs go to global memory as 128-bit coalesced stores straight
+// from registers.  Every intermediate stays in registers; shared memory only
+// holds the ring of input planes.
+#pragma once
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace stencil {
+
+constexpr int kStreamTX = 128;            // tile width (points); one warp spans a row
+constexpr int kStreamPX = kStreamTX + 8;  // smem row pitch: 4-float halo each side keeps
+                                          // TMA x-coordinates and LDS.128 16-byte aligned
+constexpr int kMaxStages = 8;
+
+template <int R>
+struct StarWeights {            // taps of a star stencil, index d + R along each axis
+    float c;
+    float x[2 * R + 1], y[2 * R + 1], z[2 * R + 1];   // entry [R] unused
+};
+
+template <int R>
+struct BoxWeights {             // dense cube, [dz+R][dy+R][dx+R]
+    float w[2 * R + 1][2 * R + 1][2 * R + 1];
+};
+
+struct StreamGeom {
+    int nz, ny, nx;
+    int tiles_x, tiles_y;
+    int chunk_z;                // planes of output per CTA
+    int stages;                 // depth of the plane ring
+    int streaming_store;        // 1: st.global.cs
+};
+
+template <int R, int K, int NW>
+struct StreamShape {
+    static constexpr int TY = NW * K;
+    static constexpr int ROWS = TY + 2 * R;
+    static constexpr int PLANE_FLOATS = ROWS * kStreamPX;
+    static constexpr int BOX_BYTES = PLANE_FLOATS * 4;
+    static constexpr int PLANE_BYTES = (BOX_BYTES + 127) / 128 * 128;
+    static constexpr int THREADS = (NW + 1) * 32;
+    static size_t smem_bytes(int stages) { return (size_t)stages * PLANE_BYTES + 128 + 128; }
+};
+
+__device__ __forceinline__ float f4get(const float4& v, int m) {
+    return m == 0 ? v.x : (m == 1 ? v.y : (m == 2 ? v.z : v.w));
+}
+
+__device__ __forceinline__ void store_f4(float* p, const float4& v, int streaming) {
+    if (streaming) __stcs(reinterpret_cast<float4*>(p), v);
+    else *reinterpret_cast<float4*>(p) = v;
+}
+
+// Fills v[0 .. 4+2R) with the R values left of the lane's float4, the float4
+// itself, and the R values right of it, for one smem row.  `rowp` points at the
+// lane's float4 inside the row; `rowbase` at the row's first float (x = -4).
+template <int R>
+__device__ __forceinline__ void gather_row(const float* rowp, const float* rowbase, int lane,
+                                           const float4& ctr, float (&v)[4 + 2 * R]) {
+    v[R + 0] = ctr.x; v[R + 1] = ctr.y; v[R + 2] = ctr.z; v[R + 3] = ctr.w;
+    if constexpr (R <= 2) {
+        // neighbours' registers through shuffles; the row's two end lanes read the smem halo
+        const float c4[4] = {ctr.x, ctr.y, ctr.z, ctr.w};
+#pragma unroll
+        for (int t = 0; t < R; ++t) {
+            float l = __shfl_up_sync(0xffffffffu, c4[4 - R + t], 1);
+            float r = __shfl_down_sync(0xffffffffu, c4[t], 1);
+            if (lane == 0) l = rowbase[4 - R + t];
+            if (lane == 31) r = rowbase[4 + kStreamTX + t];
+            v[t] = l;
+            v[R + 4 + t] = r;
+        }
+    } else {
+        const float4 l = *reinterpret_cast<const float4*>(rowp - 4);
+        const float4 r = *reinterpret_cast<const float4*>(rowp + 4);
+        const float l4[4] = {l.x, l.y, l.z, l.w};
+        const float r4[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int t = 0; t < R; ++t) {
+            v[t] = l4[4 - R + t];
+            v[R + 4 + t] = r4[t];
+        }
+    }
+}
+
+template <int R, bool BOX, int K, int NW, int MINB>
+__global__ void __launch_bounds__((NW + 1) * 32, MINB)
+stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restrict__ out,
+                      const StreamGeom g,
+                      const __grid_constant__ StarWeights<R> sw,
+                      const __grid_constant__ BoxWeights<BOX ? R : 0> bw,
+                      int* __restrict__ status) {
+    using S = StreamShape<R, K, NW>;
+    constexpr int PX = kStreamPX;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    // ring of planes first (128-byte aligned slots), then the barriers
+    unsigned char* ring = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)g.stages * S::PLANE_BYTES);
+    const uint32_t full0 = smem_addr(bars);
+    const uint32_t empty0 = smem_addr(bars + kMaxStages);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int nstage = g.stages;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < nstage; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, NW);
+        }
+        fence_barrier_init();
+    }
+    __syncthreads();
+
+    // tile and z range of this CTA; x-y tiles vary fastest so that neighbours
+    // (which share halo rows) are resident together and hit in L2
+    const int bid = blockIdx.x;
+    const int tile_x = bid % g.tiles_x;
+    const int tile_y = (bid / g.tiles_x) % g.tiles_y;
+    const int chunk = bid / (g.tiles_x * g.tiles_y);
+    const int x0 = tile_x * kStreamTX;
+    const int y0 = tile_y * S::TY;
+    const int z0 = chunk * g.chunk_z;
+    const int z1 = min(z0 + g.chunk_z, g.nz);
+    const int nplanes = (z1 - z0) + 2 * R;      // input planes z0-R .. z1-1+R
+    const int pstart = z0 - R;
+
+    if (warp == NW) {
+        // ---------------- producer: one lane drives the TMA ring ----------------
+        if (lane == 0) {
+            prefetch_tensormap(&tmap_in);
+            bool ok = true;
+            int issued = 0;
+            for (int i = 0; i < nplanes; ++i) {
+                const int s = i % nstage;
+                const int n = i / nstage;
+                if (n > 0 && !mbar_wait_bounded(empty0 + 8 * s, (n - 1) & 1)) { ok = false; break; }
+                mbar_arrive_expect_tx(full0 + 8 * s, S::BOX_BYTES);
+                tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_BYTES), &tmap_in, full0 + 8 * s,
+                            x0 - 4, y0 - R, pstart + i);
+                issued = i + 1;
+            }
+            if (!ok) {
+                atomicExch(status, kStatusTimeout);
+                // let copies already in flight land before the CTA's smem goes away
+                for (int i = max(0, issued - nstage); i < issued; ++i)
+                    mbar_wait_bounded(full0 + 8 * (i % nstage), (i / nstage) & 1);
+            }
+        }
+        return;
+    }
+
+    // ------------------------------- consumers --------------------------------
+    const int row0 = warp * K;                         // first tile row of this warp
+    const int xg = x0 + 4 * lane;                      // global x of the lane's float4
+    const bool x_in = xg < g.nx;
+    const size_t plane_stride = (size_t)g.ny * g.nx;
+
+    if constexpr (!BOX) {
+        float4 q[K][R], pend[K][R];
+#pragma unroll
+        for (int k = 0; k < K; ++k)
+#pragma unroll
+            for (int j = 0; j < R; ++j) {
+                q[k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                pend[k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+
+        for (int i0 = 0; i0 < nplanes; i0 += R) {
+#pragma unroll
+            for (int u = 0; u < R; ++u) {
+                const int i = i0 + u;
+                if (i >= nplanes) break;
+                const int s = i % nstage;
+                if (!mbar_wait_bounded(full0 + 8 * s, (i / nstage) & 1)) {
+                    atomicExch(status, kStatusTimeout);
+                    return;
+                }
+                const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
+                const float* colp = pl + row0 * PX + 4 + 4 * lane;
+                float4 c[K + 2 * R];
+#pragma unroll
+                for (int kk = 0; kk < K + 2 * R; ++kk)
+                    c[kk] = *reinterpret_cast<const float4*>(colp + kk * PX);
+
+                float4 done[K];
+#pragma unroll
+                for (int k = 0; k < K; ++k) {
+                    const float4 ctr = c[k + R];
+                    float v[4 + 2 * R];
+                    gather_row<R>(colp + (k + R) * PX, pl + (row0 + k + R) * PX, lane, ctr, v);
+                    float acc[4];
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) {
+                        float a = sw.c * v[R + m];
+#pragma unroll
+                        for (int d = 1; d <= R; ++d) {
+                            a = fmaf(sw.x[R - d], v[R + m - d], a);
+                            a = fmaf(sw.x[R + d], v[R + m + d], a);
+                        }
+#pragma unroll
+                        for (int d = 1; d <= R; ++d) {
+                            a = fmaf(sw.y[R - d], f4get(c[k + R - d], m), a);
+                            a = fmaf(sw.y[R + d], f4get(c[k + R + d], m), a);
+                        }
+#pragma unroll
+                        for (int j = 1; j <= R; ++j)      // taps at dz = -j: plane i-j
+                            a = fmaf(sw.z[R - j], f4get(q[k][(u - j + R) % R], m), a);
+                        acc[m] = a;
+                    }
+#pragma unroll
+                    for (int j = 1; j <= R; ++j) {        // this plane is dz = +j of output i-j
+                        float4& p = pend[k][(u - j + R) % R];
+                        p.x = fmaf(sw.z[R + j], ctr.x, p.x);
+                        p.y = fmaf(sw.z[R + j], ctr.y, p.y);
+                        p.z = fmaf(sw.z[R + j], ctr.z, p.z);
+                        p.w = fmaf(sw.z[R + j], ctr.w, p.w);
+                    }
+                    done[k] = pend[k][u];                 // output plane i-R is complete
+                    pend[k][u] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                    q[k][u] = ctr;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8 * s);
+
+                if (i >= 2 * R && x_in) {
+                    const int zo = z0 + i - 2 * R;
+                    float* op = out + (size_t)zo * plane_stride + (size_t)(y0 + row0) * g.nx + xg;
+#pragma unroll
+                    for (int k = 0; k < K; ++k)
+                        if (y0 + row0 + k < g.ny) store_f4(op + (size_t)k * g.nx, done[k], g.streaming_store);
+                }
+            }
+        }
+    } else {
+        // acc[k][j]: partial output of plane (i-1-j)+... carried between planes;
+        // at step i, T[d] (d = 0..2R) is the output plane i - (d - R).
+        float4 T[K][2 * R + 1];
+#pragma unroll
+        for (int k = 0; k < K; ++k)
+#pragma unroll
+            for (int d = 0; d <= 2 * R; ++d) T[k][d] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+        for (int i = 0; i < nplanes; ++i) {
+            const int s = i % nstage;
+            if (!mbar_wait_bounded(full0 + 8 * s, (i / nstage) & 1)) {
+                atomicExch(status, kStatusTimeout);
+                return;
+            }
+            const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
+            const float* colp = pl + row0 * PX + 4 + 4 * lane;
+            float v[K + 2 * R][4 + 2 * R];
+#pragma unroll
+            for (int kk = 0; kk < K + 2 * R; ++kk) {
+                const float4 ctr = *reinterpret_cast<const float4*>(colp + kk * PX);
+                gather_row<R>(colp + kk * PX, pl + (row0 + kk) * PX, lane, ctr, v[kk]);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8 * s);
+
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+                // shift: the accumulator of output plane z moves one slot per input plane
+#pragma unroll
+                for (int d = 2 * R; d > 0; --d) T[k][d] = T[k][d - 1];
+                T[k][0] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int d = 0; d <= 2 * R; ++d) {        // T[k][d]: this plane is its tap dz = d - R
+                    float a[4] = {T[k][d].x, T[k][d].y, T[k][d].z, T[k][d].w};
+#pragma unroll
+                    for (int dy = 0; dy <= 2 * R; ++dy)
+#pragma unroll
+                        for (int dx = 0; dx <= 2 * R; ++dx) {
+                            const float wv = bw.w[d][dy][dx];
+#pragma unroll
+                            for (int m = 0; m < 4; ++m) a[m] = fmaf(wv, v[k + dy][m + dx], a[m]);
+                        }
+                    T[k][d] = make_float4(a[0], a[1], a[2], a[3]);
+                }
+            }
+            if (i >= 2 * R && x_in) {
+                const int zo = z0 + i - 2 * R;
+                float* op = out + (size_t)zo * plane_stride + (size_t)(y0 + row0) * g.nx + xg;
+#pragma unroll
+                for (int k = 0; k < K; ++k)
+                    if (y0 + row0 + k < g.ny) store_f4(op + (size_t)k * g.nx, T[k][2 * R], g.streaming_store);
+            }
+        }
+    }
+}
+
+}  // namespace stencil

@@ -1,0 +1,552 @@
+// Host side of the stencil library: plan validation, kernel selection, tensor
+// maps, launches, and the extern "C" boundary declared in include/stencil.h.
+// No CPU compute path exists here: every sweep runs in the CUDA kernels.
+#include "../../include/stencil.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "kernel_generic.cuh"
+#include "kernel_stream.cuh"
+
+using namespace stencil;
+
+namespace {
+
+constexpr uint32_t kPlanMagic = 0x5354434cu;   // "STCL"
+constexpr int kMaxRadius = 8;
+
+// ---------------------------------------------------------------------------
+// driver entry point for tensor-map encoding, fetched at run time so that the
+// library loads on machines without a driver
+// ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+// ---------------------------------------------------------------------------
+// STREAM kernel configurations
+// ---------------------------------------------------------------------------
+struct StreamConfig {
+    int radius;
+    bool box;
+    int K, NW;            // rows per thread, consumer warps
+    int tile_y;           // K * NW
+    int plane_bytes, box_rows, threads;
+    const void* kernel;
+    cudaError_t (*launch)(const struct stencil_plan_s*, const StreamConfig&, const CUtensorMap&,
+                          float*, const StreamGeom&, int grid, size_t smem, cudaStream_t);
+};
+
+}  // namespace
+
+struct stencil_plan_s {
+    uint32_t magic;
+    int ndim;
+    int nz, ny, nx;
+    int64_t npoints;
+    int radius, shape, boundary;
+    std::vector<float> w;          // dense (2R+1)^ndim, as given
+    std::vector<Tap> taps;         // non-zero taps, dense C order
+    // device state (created lazily, on the device current at first apply)
+    int device;
+    Tap* d_taps;
+    int* d_status;
+    float* scratch;                // N floats, iteration ping-pong
+    float* host_in;                // N floats each, apply_host staging
+    float* host_out;
+    // selection and tuning
+    int variant;                   // resolved STENCIL_VARIANT_*
+    int tile_y, rows_per_thread, chunk_z, stages, fuse_steps, streaming_store;
+    const StreamConfig* stream_cfg;
+    // bookkeeping
+    int64_t launches;
+    cudaStream_t last_stream;
+    bool used;
+    // tensor-map cache: one entry per source pointer
+    struct MapEntry { const float* ptr; const StreamConfig* cfg; CUtensorMap map; };
+    std::vector<MapEntry> maps;
+};
+
+namespace {
+
+// ---------------------------------------------------------------------------
+// weight packing for the tiled kernels
+// ---------------------------------------------------------------------------
+inline float dense_w(const stencil_plan_s* p, int dz, int dy, int dx) {
+    const int R = p->radius, side = 2 * R + 1;
+    if (p->ndim == 3) return p->w[((size_t)(dz + R) * side + (dy + R)) * side + (dx + R)];
+    return dz == 0 ? p->w[(size_t)(dy + R) * side + (dx + R)] : 0.0f;
+}
+
+template <int R, bool BOX, int K, int NW, int MINB>
+cudaError_t launch_stream_t(const stencil_plan_s* p, const StreamConfig&, const CUtensorMap& map,
+                            float* out, const StreamGeom& g, int grid, size_t smem, cudaStream_t st) {
+    StarWeights<R> sw;
+    BoxWeights<BOX ? R : 0> bw;
+    std::memset(&sw, 0, sizeof(sw));
+    std::memset(&bw, 0, sizeof(bw));
+    if (!BOX) {
+        sw.c = dense_w(p, 0, 0, 0);
+        for (int d = -R; d <= R; ++d) {
+            if (d == 0) continue;
+            sw.x[d + R] = dense_w(p, 0, 0, d);
+            sw.y[d + R] = dense_w(p, 0, d, 0);
+            sw.z[d + R] = dense_w(p, d, 0, 0);
+        }
+    } else {
+        constexpr int RB = BOX ? R : 0;
+        for (int a = -RB; a <= RB; ++a)
+            for (int b = -RB; b <= RB; ++b)
+                for (int c = -RB; c <= RB; ++c) bw.w[a + RB][b + RB][c + RB] = dense_w(p, a, b, c);
+    }
+    stencil_stream_kernel<R, BOX, K, NW, MINB>
+        <<<grid, StreamShape<R, K, NW>::THREADS, smem, st>>>(map, out, g, sw, bw, p->d_status);
+    return cudaGetLastError();
+}
+
+template <int R, bool BOX, int K, int NW, int MINB>
+StreamConfig make_cfg() {
+    using S = StreamShape<R, K, NW>;
+    StreamConfig c;
+    c.radius = R; c.box = BOX; c.K = K; c.NW = NW; c.tile_y = S::TY;
+    c.plane_bytes = S::PLANE_BYTES; c.box_rows = S::ROWS; c.threads = S::THREADS;
+    c.kernel = reinterpret_cast<const void*>(&stencil_stream_kernel<R, BOX, K, NW, MINB>);
+    c.launch = &launch_stream_t<R, BOX, K, NW, MINB>;
+    return c;
+}
+
+// First entry of a (radius, box) group is the default; the others are reachable
+// through STENCIL_KEY_TILE_Y / STENCIL_KEY_ROWS_PER_THREAD.
+const std::vector<StreamConfig>& stream_configs() {
+    static const std::vector<StreamConfig> v = {
+        make_cfg<1, false, 2, 8, 1>(),  make_cfg<1, false, 4, 8, 1>(),  make_cfg<1, false, 1, 8, 1>(),
+        make_cfg<2, false, 2, 8, 1>(),  make_cfg<2, false, 4, 8, 1>(),
+        make_cfg<3, false, 2, 8, 1>(),  make_cfg<3, false, 4, 8, 1>(),
+        make_cfg<4, false, 2, 8, 1>(),  make_cfg<4, false, 4, 8, 1>(),  make_cfg<4, false, 2, 16, 1>(),
+        make_cfg<1, true, 2, 8, 1>(),   make_cfg<1, true, 4, 8, 1>(),   make_cfg<1, true, 1, 8, 1>(),
+    };
+    return v;
+}
+
+const StreamConfig* find_stream_cfg(int radius, bool box, int tile_y, int rows_per_thread) {
+    for (const StreamConfig& c : stream_configs())
+        if (c.radius == radius && c.box == box && (tile_y == 0 || c.tile_y == tile_y) &&
+            (rows_per_thread == 0 || c.K == rows_per_thread))
+            return &c;
+    return nullptr;
+}
+
+bool stream_supported(const stencil_plan_s* p) {
+    if (p->ndim != 3 || p->boundary != STENCIL_ZERO) return false;
+    if (p->nx % 4 != 0) return false;              // TMA global strides must be 16-byte multiples
+    const bool box = p->shape == STENCIL_BOX;
+    return find_stream_cfg(p->radius, box, 0, 0) != nullptr;
+}
+
+int resolve_variant(stencil_plan_s* p, int want) {
+    if (want == STENCIL_VARIANT_AUTO) want = stream_supported(p) ? STENCIL_VARIANT_STREAM : STENCIL_VARIANT_GENERIC;
+    if (want == STENCIL_VARIANT_GENERIC) { p->variant = want; return STENCIL_OK; }
+    if (want == STENCIL_VARIANT_STREAM) {
+        if (!stream_supported(p)) return STENCIL_ERR_UNSUPPORTED;
+        const StreamConfig* c = find_stream_cfg(p->radius, p->shape == STENCIL_BOX, p->tile_y, p->rows_per_thread);
+        if (!c) return STENCIL_ERR_UNSUPPORTED;
+        p->stream_cfg = c;
+        p->variant = want;
+        return STENCIL_OK;
+    }
+    return STENCIL_ERR_UNSUPPORTED;
+}
+
+// ---------------------------------------------------------------------------
+// device state
+// ---------------------------------------------------------------------------
+int ensure_device_state(stencil_plan_s* p) {
+    if (p->d_status) return STENCIL_OK;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    p->device = dev;
+    if (cudaMalloc(&p->d_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    if (cudaMemset(p->d_status, 0, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    const size_t bytes = p->taps.size() * sizeof(Tap);
+    if (bytes) {
+        if (cudaMalloc(&p->d_taps, bytes) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_ALLOC; }
+        if (cudaMemcpy(p->d_taps, p->taps.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaGetLastError();
+            return STENCIL_ERR_CUDA;
+        }
+    }
+    return STENCIL_OK;
+}
+
+int ensure_grid(float** slot, int64_t npoints) {
+    if (*slot) return STENCIL_OK;
+    if (cudaMalloc(slot, (size_t)npoints * sizeof(float)) != cudaSuccess) {
+        cudaGetLastError();
+        *slot = nullptr;
+        return STENCIL_ERR_ALLOC;
+    }
+    return STENCIL_OK;
+}
+
+// ---------------------------------------------------------------------------
+// launches
+// ---------------------------------------------------------------------------
+int launch_generic(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
+    Grid g{p->nz, p->ny, p->nx};
+    const int64_t blocks_needed = (p->npoints + kGenericThreads - 1) / kGenericThreads;
+    const int grid = (int)std::min<int64_t>(blocks_needed, 148 * 16);
+    const int ntaps = (int)p->taps.size();
+    if (p->boundary == STENCIL_PERIODIC)
+        stencil_generic_kernel<true><<<grid, kGenericThreads, 0, st>>>(src, dst, g, p->d_taps, ntaps);
+    else
+        stencil_generic_kernel<false><<<grid, kGenericThreads, 0, st>>>(src, dst, g, p->d_taps, ntaps);
+    if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
+    p->launches++;
+    return STENCIL_OK;
+}
+
+int get_tensor_map(stencil_plan_s* p, const StreamConfig* cfg, const float* src, const CUtensorMap** out) {
+    for (auto& e : p->maps)
+        if (e.ptr == src && e.cfg == cfg) { *out = &e.map; return STENCIL_OK; }
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) return STENCIL_ERR_CUDA;
+    stencil_plan_s::MapEntry e;
+    e.ptr = src; e.cfg = cfg;
+    const cuuint64_t dims[3] = {(cuuint64_t)p->nx, (cuuint64_t)p->ny, (cuuint64_t)p->nz};
+    const cuuint64_t strides[2] = {(cuuint64_t)p->nx * 4, (cuuint64_t)p->nx * (cuuint64_t)p->ny * 4};
+    const cuuint32_t box[3] = {(cuuint32_t)kStreamPX, (cuuint32_t)cfg->box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(&e.map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(src), dims, strides,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return STENCIL_ERR_CUDA;
+    if (p->maps.size() >= 8) p->maps.erase(p->maps.begin());
+    p->maps.push_back(e);
+    *out = &p->maps.back().map;
+    return STENCIL_OK;
+}
+
+int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
+    const StreamConfig* cfg = p->stream_cfg;
+    const CUtensorMap* map = nullptr;
+    int rc = get_tensor_map(p, cfg, src, &map);
+    if (rc != STENCIL_OK) return rc;
+
+    StreamGeom g;
+    g.nz = p->nz; g.ny = p->ny; g.nx = p->nx;
+    g.tiles_x = (p->nx + kStreamTX - 1) / kStreamTX;
+    g.tiles_y = (p->ny + cfg->tile_y - 1) / cfg->tile_y;
+    g.stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 4;
+    g.streaming_store = p->streaming_store;
+    const int tiles = g.tiles_x * g.tiles_y;
+    int chunk = p->chunk_z;
+    if (chunk <= 0) {
+        // enough CTAs for several waves of the 148 SMs, but chunks long enough
+        // that the 2R halo planes per chunk stay a small fraction
+        const int want_ctas = 148 * 8;
+        int nchunks = std::max(1, std::min((want_ctas + tiles - 1) / tiles, p->nz / std::max(16 * p->radius, 32)));
+        chunk = (p->nz + nchunks - 1) / nchunks;
+    }
+    chunk = std::max(1, std::min(chunk, p->nz));
+    g.chunk_z = chunk;
+    const int nchunks = (p->nz + chunk - 1) / chunk;
+    const int64_t grid64 = (int64_t)tiles * nchunks;
+    if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)g.stages * cfg->plane_bytes + 128 + 2 * kMaxStages * sizeof(uint64_t);
+    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
+    if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        cudaGetLastError();
+        return STENCIL_ERR_CUDA;
+    }
+    if (cfg->launch(p, *cfg, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
+    p->launches++;
+    return STENCIL_OK;
+}
+
+int launch_sweep(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
+    switch (p->variant) {
+        case STENCIL_VARIANT_STREAM: return launch_stream(p, src, dst, st);
+        default: return launch_generic(p, src, dst, st);
+    }
+}
+
+bool valid_plan(const stencil_plan_s* p) { return p && p->magic == kPlanMagic; }
+
+}  // namespace
+
+// ===========================================================================
+// C ABI
+// ===========================================================================
+extern "C" {
+
+int stencil_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radius, int shape,
+                 const float* weights, int boundary) {
+    if (!plan_out) return STENCIL_ERR_INVALID;
+    *plan_out = nullptr;
+    if ((ndim != 2 && ndim != 3) || !dims || !weights) return STENCIL_ERR_INVALID;
+    if (shape != STENCIL_STAR && shape != STENCIL_BOX) return STENCIL_ERR_INVALID;
+    if (boundary != STENCIL_ZERO && boundary != STENCIL_PERIODIC) return STENCIL_ERR_INVALID;
+    if (radius < 1) return STENCIL_ERR_INVALID;
+    if (radius > kMaxRadius) return STENCIL_ERR_UNSUPPORTED;
+    int64_t n = 1;
+    for (int i = 0; i < ndim; ++i) {
+        if (dims[i] < 1) return STENCIL_ERR_INVALID;
+        if (dims[i] > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
+        if (n > (int64_t)1 << 40) return STENCIL_ERR_UNSUPPORTED;
+        n *= dims[i];
+    }
+
+    stencil_plan_s* p = new (std::nothrow) stencil_plan_s();
+    if (!p) return STENCIL_ERR_ALLOC;
+    p->magic = kPlanMagic;
+    p->ndim = ndim;
+    p->nz = ndim == 3 ? (int)dims[0] : 1;
+    p->ny = ndim == 3 ? (int)dims[1] : (int)dims[0];
+    p->nx = ndim == 3 ? (int)dims[2] : (int)dims[1];
+    p->npoints = n;
+    p->radius = radius; p->shape = shape; p->boundary = boundary;
+    p->device = -1;
+    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr;
+    p->host_in = nullptr; p->host_out = nullptr;
+    p->variant = STENCIL_VARIANT_GENERIC;
+    p->tile_y = 0; p->rows_per_thread = 0; p->chunk_z = 0; p->stages = 0; p->fuse_steps = 0; p->streaming_store = 0;
+    p->stream_cfg = nullptr;
+    p->launches = 0; p->last_stream = nullptr; p->used = false;
+
+    const int side = 2 * radius + 1;
+    size_t count = 1;
+    for (int i = 0; i < ndim; ++i) count *= (size_t)side;
+    try {
+        p->w.assign(weights, weights + count);
+        for (size_t f = 0; f < count; ++f) {
+            const float wv = p->w[f];
+            int dx = (int)(f % side) - radius;
+            int dy = (int)((f / side) % side) - radius;
+            int dz = ndim == 3 ? (int)(f / ((size_t)side * side)) - radius : 0;
+            const int nonzero_axes = (dx != 0) + (dy != 0) + (dz != 0);
+            if (shape == STENCIL_STAR && nonzero_axes > 1 && wv != 0.0f) {
+                delete p;
+                return STENCIL_ERR_INVALID;       // STAR promises zero off-axis weights
+            }
+            if (wv != 0.0f) p->taps.push_back(Tap{dz, dy, dx, wv});
+        }
+    } catch (...) {
+        delete p;
+        return STENCIL_ERR_ALLOC;
+    }
+    resolve_variant(p, STENCIL_VARIANT_AUTO);
+    *plan_out = p;
+    return STENCIL_OK;
+}
+
+int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void* stream) {
+    if (!valid_plan(p) || !in || !out || steps < 0) return STENCIL_ERR_INVALID;
+    const uintptr_t a = reinterpret_cast<uintptr_t>(in), b = reinterpret_cast<uintptr_t>(out);
+    if ((a | b) & 15u) return STENCIL_ERR_INVALID;
+    const uintptr_t bytes = (uintptr_t)p->npoints * sizeof(float);
+    if (a < b + bytes && b < a + bytes) return STENCIL_ERR_INVALID;      // overlap (covers in == out)
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+
+    int rc = ensure_device_state(p);
+    if (rc != STENCIL_OK) return rc;
+    p->last_stream = st;
+    p->used = true;
+
+    if (steps == 0) {
+        if (cudaMemcpyAsync(out, in, bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+            cudaGetLastError();
+            return STENCIL_ERR_CUDA;
+        }
+        return STENCIL_OK;
+    }
+    if (steps > 1) {
+        rc = ensure_grid(&p->scratch, p->npoints);
+        if (rc != STENCIL_OK) return rc;
+    }
+    // ping-pong so that the last sweep writes `out` and `in` stays intact
+    const float* src = in;
+    for (int k = 0; k < steps; ++k) {
+        const int remaining = steps - 1 - k;
+        float* dst = (remaining % 2 == 0) ? out : p->scratch;
+        rc = launch_sweep(p, src, dst, st);
+        if (rc != STENCIL_OK) return rc;
+        src = dst;
+    }
+    return STENCIL_OK;
+}
+
+int stencil_apply_host(stencil_plan_t p, const float* in_host, float* out_host, int steps, void* stream) {
+    if (!valid_plan(p) || !in_host || !out_host || steps < 0) return STENCIL_ERR_INVALID;
+    int rc = ensure_device_state(p);
+    if (rc != STENCIL_OK) return rc;
+    if ((rc = ensure_grid(&p->host_in, p->npoints)) != STENCIL_OK) return rc;
+    if ((rc = ensure_grid(&p->host_out, p->npoints)) != STENCIL_OK) return rc;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const size_t bytes = (size_t)p->npoints * sizeof(float);
+    if (cudaMemcpyAsync(p->host_in, in_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return STENCIL_ERR_CUDA;
+    }
+    rc = stencil_apply(p, p->host_in, p->host_out, steps, stream);
+    if (rc != STENCIL_OK) return rc;
+    if (cudaMemcpyAsync(out_host, p->host_out, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return STENCIL_ERR_CUDA;
+    }
+    return STENCIL_OK;
+}
+
+int stencil_destroy(stencil_plan_t p) {
+    if (!p) return STENCIL_OK;
+    if (!valid_plan(p)) return STENCIL_ERR_INVALID;
+    int rc = STENCIL_OK;
+    if (p->d_status || p->scratch || p->host_in || p->host_out || p->d_taps) {
+        int cur = -1;
+        cudaGetDevice(&cur);
+        if (p->device >= 0 && cur != p->device) cudaSetDevice(p->device);
+        if (p->used) cudaStreamSynchronize(p->last_stream);
+        void* ptrs[] = {p->d_status, p->scratch, p->host_in, p->host_out, p->d_taps};
+        for (void* q : ptrs)
+            if (q && cudaFree(q) != cudaSuccess) rc = STENCIL_ERR_CUDA;
+        if (p->device >= 0 && cur >= 0 && cur != p->device) cudaSetDevice(cur);
+        cudaGetLastError();
+    }
+    p->magic = 0;
+    delete p;
+    return rc;
+}
+
+const char* stencil_status_string(int status) {
+    switch (status) {
+        case STENCIL_OK: return "ok";
+        case STENCIL_ERR_INVALID: return "invalid argument";
+        case STENCIL_ERR_UNSUPPORTED: return "unsupported request";
+        case STENCIL_ERR_CUDA: return "CUDA call failed or no device";
+        case STENCIL_ERR_ALLOC: return "allocation failed";
+        case STENCIL_ERR_TIMEOUT: return "bounded device wait expired";
+        default: return "unknown status";
+    }
+}
+
+const char* stencil_variant_name(int variant) {
+    switch (variant) {
+        case STENCIL_VARIANT_AUTO: return "auto";
+        case STENCIL_VARIANT_GENERIC: return "generic";
+        case STENCIL_VARIANT_STREAM: return "stream";
+        case STENCIL_VARIANT_FUSED: return "fused";
+        default: return "unknown";
+    }
+}
+
+int stencil_query_status(stencil_plan_t p) {
+    if (!valid_plan(p)) return STENCIL_ERR_INVALID;
+    if (!p->d_status) return STENCIL_OK;               // nothing has run yet
+    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    int word = 0;
+    if (cudaMemcpy(&word, p->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemset(p->d_status, 0, sizeof(int)) != cudaSuccess) {
+        cudaGetLastError();
+        return STENCIL_ERR_CUDA;
+    }
+    return word == 0 ? STENCIL_OK : STENCIL_ERR_TIMEOUT;
+}
+
+int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
+    if (!valid_plan(p)) return STENCIL_ERR_INVALID;
+    switch (key) {
+        case STENCIL_KEY_VARIANT: {
+            const int old_variant = p->variant;
+            const StreamConfig* old_cfg = p->stream_cfg;
+            int rc = resolve_variant(p, (int)value);
+            if (rc != STENCIL_OK) { p->variant = old_variant; p->stream_cfg = old_cfg; }
+            return rc;
+        }
+        case STENCIL_KEY_TILE_X:
+            return (value == 0 || value == kStreamTX) ? STENCIL_OK : STENCIL_ERR_UNSUPPORTED;
+        case STENCIL_KEY_TILE_Y:
+        case STENCIL_KEY_ROWS_PER_THREAD: {
+            if (value < 0) return STENCIL_ERR_INVALID;
+            int ty = key == STENCIL_KEY_TILE_Y ? (int)value : p->tile_y;
+            int k = key == STENCIL_KEY_ROWS_PER_THREAD ? (int)value : p->rows_per_thread;
+            if (p->variant == STENCIL_VARIANT_STREAM) {
+                const StreamConfig* c = find_stream_cfg(p->radius, p->shape == STENCIL_BOX, ty, k);
+                if (!c) return STENCIL_ERR_UNSUPPORTED;
+                p->stream_cfg = c;
+            }
+            p->tile_y = ty;
+            p->rows_per_thread = k;
+            return STENCIL_OK;
+        }
+        case STENCIL_KEY_FUSE_STEPS:
+            if (value < 0) return STENCIL_ERR_INVALID;
+            p->fuse_steps = (int)value;
+            return STENCIL_OK;
+        case STENCIL_KEY_CHUNK_Z:
+            if (value < 0) return STENCIL_ERR_INVALID;
+            p->chunk_z = (int)std::min<int64_t>(value, 0x7fffffff);
+            return STENCIL_OK;
+        case STENCIL_KEY_STAGES:
+            if (value < 0 || value > kMaxStages || value == 1) return STENCIL_ERR_INVALID;
+            p->stages = (int)value;
+            return STENCIL_OK;
+        case STENCIL_KEY_STREAMING_STORE:
+            p->streaming_store = value ? 1 : 0;
+            return STENCIL_OK;
+        default:
+            return STENCIL_ERR_INVALID;
+    }
+}
+
+int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
+    if (!valid_plan(p) || !value) return STENCIL_ERR_INVALID;
+    switch (key) {
+        case STENCIL_KEY_VARIANT: *value = p->variant; return STENCIL_OK;
+        case STENCIL_KEY_TILE_X: *value = p->variant == STENCIL_VARIANT_STREAM ? kStreamTX : 0; return STENCIL_OK;
+        case STENCIL_KEY_TILE_Y:
+            *value = (p->variant == STENCIL_VARIANT_STREAM && p->stream_cfg) ? p->stream_cfg->tile_y : 0;
+            return STENCIL_OK;
+        case STENCIL_KEY_ROWS_PER_THREAD:
+            *value = (p->variant == STENCIL_VARIANT_STREAM && p->stream_cfg) ? p->stream_cfg->K : 0;
+            return STENCIL_OK;
+        case STENCIL_KEY_FUSE_STEPS: *value = p->fuse_steps; return STENCIL_OK;
+        case STENCIL_KEY_LAUNCHES: *value = p->launches; return STENCIL_OK;
+        case STENCIL_KEY_SCRATCH_BYTES: {
+            int64_t grids = (p->scratch != nullptr) + (p->host_in != nullptr) + (p->host_out != nullptr);
+            *value = grids * p->npoints * (int64_t)sizeof(float);
+            return STENCIL_OK;
+        }
+        case STENCIL_KEY_CHUNK_Z: *value = p->chunk_z; return STENCIL_OK;
+        case STENCIL_KEY_STAGES: *value = p->stages; return STENCIL_OK;
+        case STENCIL_KEY_STREAMING_STORE: *value = p->streaming_store; return STENCIL_OK;
+        default: return STENCIL_ERR_INVALID;
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,161 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports
+every symbol the header declares, validates arguments, and refuses to compute
+without a device instead of falling back to anything."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2608_21157_b200 import binding as b
+from paper_2608_21157_b200 import build as build_mod
+from paper_2608_21157_b200 import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_mod.build()
+    b.load()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "stencil.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"STENCIL_API\s+[\w\s\*]+?\b(stencil_\w+)\s*\(", text)))
+
+
+def test_header_and_binding_list_the_same_symbols():
+    assert _declared_symbols() == sorted(b.EXPORTS)
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(b.LIB_PATH)
+    for name in _declared_symbols():
+        assert getattr(lib, name) is not None
+
+
+def test_binding_does_not_import_the_oracle():
+    import paper_2608_21157_b200
+    pkg_dir = os.path.dirname(paper_2608_21157_b200.__file__)
+    for dirpath, _, files in os.walk(pkg_dir):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                src = open(os.path.join(dirpath, f)).read()
+                assert "import oracle" not in src and "from oracle" not in src
+                assert "stencil_oracle" not in src
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith((".py", ".c")):
+            src = open(os.path.join(ROOT, "oracle", f)).read()
+            assert "paper_2608_21157_b200" not in src and "stencil.h" not in src
+
+
+def test_status_and_variant_strings():
+    assert b.status_string(b.OK) == "ok"
+    for code in (b.ERR_INVALID, b.ERR_UNSUPPORTED, b.ERR_CUDA, b.ERR_ALLOC, b.ERR_TIMEOUT, 12345):
+        assert isinstance(b.status_string(code), str) and b.status_string(code)
+    assert b.variant_name(b.VARIANT_GENERIC) == "generic"
+    assert b.variant_name(b.VARIANT_STREAM) == "stream"
+
+
+def _w(ndim, R):
+    return wl.random_box_weights(ndim, R, 1)
+
+
+@pytest.mark.parametrize("dims,R,shape,boundary,want", [
+    ((8, 8), 0, b.BOX, b.ZERO, b.ERR_INVALID),
+    ((8, 8), 9, b.BOX, b.ZERO, b.ERR_UNSUPPORTED),
+    ((8, 0), 1, b.BOX, b.ZERO, b.ERR_INVALID),
+    ((8, -3, 4), 1, b.BOX, b.ZERO, b.ERR_INVALID),
+    ((8, 8), 1, 7, b.ZERO, b.ERR_INVALID),
+    ((8, 8), 1, b.BOX, 5, b.ERR_INVALID),
+    ((8,), 1, b.BOX, b.ZERO, b.ERR_INVALID),
+    ((4, 4, 4, 4), 1, b.BOX, b.ZERO, b.ERR_INVALID),
+])
+def test_plan_rejects_bad_arguments(dims, R, shape, boundary, want):
+    ndim = min(max(len(dims), 2), 3)
+    rc, h = b.stencil_plan(dims, R, shape, _w(ndim, max(R, 1)), boundary)
+    assert rc == want
+    assert not h.value
+
+
+def test_plan_null_pointers():
+    lib = b.load()
+    h = ctypes.c_void_p()
+    d = (ctypes.c_int64 * 2)(4, 4)
+    w = _w(2, 1)
+    wp = w.ctypes.data_as(ctypes.POINTER(ctypes.c_float))
+    assert lib.stencil_plan(None, 2, d, 1, b.BOX, wp, b.ZERO) == b.ERR_INVALID
+    assert lib.stencil_plan(ctypes.byref(h), 2, None, 1, b.BOX, wp, b.ZERO) == b.ERR_INVALID
+    assert lib.stencil_plan(ctypes.byref(h), 2, d, 1, b.BOX, None, b.ZERO) == b.ERR_INVALID
+
+
+def test_star_promise_is_checked():
+    w = _w(3, 1)                                   # dense box weights are not a star
+    rc, h = b.stencil_plan((8, 8, 8), 1, b.STAR, w, b.ZERO)
+    assert rc == b.ERR_INVALID and not h.value
+    rc, h = b.stencil_plan((8, 8, 8), 1, b.STAR, wl.star_weights(3, 1, -6.0, [1.0]), b.ZERO)
+    assert rc == b.OK
+    assert b.stencil_destroy(h) == b.OK
+
+
+def test_variant_selection_rules():
+    star = wl.star_weights(3, 1, -6.0, [1.0])
+    with b.Plan((64, 64, 64), 1, b.STAR, star, b.ZERO) as p:
+        assert p.variant == "stream"
+        p.set(b.KEY_VARIANT, b.VARIANT_GENERIC)
+        assert p.variant == "generic"
+    with b.Plan((64, 64, 66), 1, b.STAR, star, b.ZERO) as p:       # nx % 4 != 0
+        assert p.variant == "generic"
+        with pytest.raises(b.StencilError) as e:
+            p.set(b.KEY_VARIANT, b.VARIANT_STREAM)
+        assert e.value.status == b.ERR_UNSUPPORTED
+        assert p.variant == "generic"
+    with b.Plan((64, 64, 64), 1, b.STAR, star, b.PERIODIC) as p:
+        assert p.variant == "generic"
+    with b.Plan((64, 64), 1, b.STAR, wl.star_weights(2, 1, -4.0, [1.0]), b.ZERO) as p:
+        assert p.variant in ("generic", "stream")
+    with b.Plan((64, 64, 64), 1, b.STAR, star, b.ZERO) as p:
+        with pytest.raises(b.StencilError):
+            p.set(b.KEY_TILE_Y, 7)
+        with pytest.raises(b.StencilError):
+            p.set(b.KEY_STAGES, 99)
+        with pytest.raises(b.StencilError):
+            p.set(12345, 1)
+
+
+def test_apply_argument_checks_and_no_cpu_fallback():
+    with b.Plan((8, 8, 8), 1, b.BOX, _w(3, 1), b.ZERO) as p:
+        n = 8 * 8 * 8 * 4
+        base = 1 << 30
+        assert b.stencil_apply(p._h, 0, base, 1) == b.ERR_INVALID            # NULL in
+        assert b.stencil_apply(p._h, base, 0, 1) == b.ERR_INVALID            # NULL out
+        assert b.stencil_apply(p._h, base, base, 1) == b.ERR_INVALID         # in == out
+        assert b.stencil_apply(p._h, base, base + n - 16, 1) == b.ERR_INVALID  # overlap
+        assert b.stencil_apply(p._h, base + 4, base + 2 * n, 1) == b.ERR_INVALID  # misaligned
+        assert b.stencil_apply(p._h, base, base + 2 * n, -1) == b.ERR_INVALID
+        assert b.stencil_apply(None, base, base + 2 * n, 1) == b.ERR_INVALID
+        import torch
+        if not torch.cuda.is_available():
+            # valid arguments but no device: the library must refuse, not compute on the CPU
+            assert b.stencil_apply(p._h, base, base + 2 * n, 1) == b.ERR_CUDA
+            a = np.zeros((8, 8, 8), np.float32)
+            o = np.zeros_like(a)
+            assert b.stencil_apply_host(p._h, a.ctypes.data, o.ctypes.data, 1) == b.ERR_CUDA
+
+
+def test_destroy_null_is_ok_and_get_counters():
+    assert b.stencil_destroy(None) == b.OK
+    with b.Plan((8, 8, 8), 1, b.BOX, _w(3, 1), b.ZERO) as p:
+        assert p.launches == 0
+        assert p.get(b.KEY_SCRATCH_BYTES) == 0
+        assert p.query_status() == b.OK
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(b, "_lib", None)
+    monkeypatch.setattr(b, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        b.load()

@@ -1,0 +1,204 @@
+"""CUDA path vs CPU oracle, element by element, through the C ABI.
+
+Acceptance: max|gpu - oracle| <= 1e-5 * sum|w| * max|in| * steps + 1e-6.
+Every output buffer is poisoned with NaN and fenced by guard bands first, so a
+point that was never written or a store outside the grid fails the test.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_21157_b200 import binding as b
+from paper_2608_21157_b200 import build as build_mod
+from paper_2608_21157_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+GUARD = 4096          # floats of guard band on each side of the output
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_mod.build()
+    b.load()
+
+
+def gpu_sweep(dims, R, shape, weights, boundary, a, steps=1, variant=None, repeat=1, **knobs):
+    """Runs the library on `a`; returns the result as numpy after checking guards."""
+    dev = torch.device("cuda:0")
+    n = int(np.prod(dims))
+    src = torch.from_numpy(a).to(dev)
+    src_copy = src.clone()
+    buf = torch.full((n + 2 * GUARD,), float("nan"), dtype=torch.float32, device=dev)
+    buf[:GUARD] = 12345.0
+    buf[GUARD + n:] = 12345.0
+    dst = buf[GUARD:GUARD + n]
+    stream = torch.cuda.current_stream().cuda_stream
+    with b.Plan(dims, R, shape, weights, boundary, variant=variant, **knobs) as p:
+        for _ in range(repeat):
+            p.apply(src, dst, steps, stream)
+        assert p.query_status() == b.OK
+        used = p.variant
+    torch.cuda.synchronize()
+    assert torch.equal(src, src_copy), "input was modified"
+    assert bool((buf[:GUARD] == 12345.0).all()) and bool((buf[GUARD + n:] == 12345.0).all()), \
+        "store outside the output grid"
+    out = dst.cpu().numpy().reshape(dims)
+    assert not np.isnan(out).any(), "some output points were never written"
+    return out, used
+
+
+def check(dims, R, shape, weights, boundary, a, steps=1, **kw):
+    got, used = gpu_sweep(dims, R, shape, weights, boundary, a, steps, **kw)
+    want = oracle.apply(a, weights, boundary, steps)
+    tol = wl.tolerance(weights, float(np.abs(a).max()), steps)
+    err = float(np.max(np.abs(got.astype(np.float64) - want.astype(np.float64)))) if got.size else 0.0
+    assert err <= tol, f"{used}: max err {err:.3e} > tol {tol:.3e} for dims={dims} R={R} steps={steps} {kw}"
+    return used
+
+
+# ------------------------------------------------------------------ generic --
+GENERIC_CASES = [
+    # dims, R, star?, boundary
+    ((256, 256), 1, True, b.ZERO),
+    ((5, 7), 1, False, b.ZERO), ((5, 7), 2, False, b.PERIODIC), ((33, 47), 3, False, b.ZERO),
+    ((2, 3), 3, False, b.ZERO), ((2, 3), 3, False, b.PERIODIC), ((1, 9), 1, True, b.ZERO),
+    ((1, 1), 2, False, b.PERIODIC), ((61, 130), 4, True, b.PERIODIC), ((40, 64), 8, False, b.ZERO),
+    ((5, 7, 11), 1, False, b.ZERO), ((5, 7, 11), 2, False, b.PERIODIC), ((3, 2, 4), 4, True, b.ZERO),
+    ((19, 23, 30), 1, True, b.PERIODIC), ((17, 33, 66), 2, True, b.ZERO), ((9, 12, 20), 3, False, b.ZERO),
+    ((1, 1, 5), 1, False, b.ZERO), ((12, 10, 36), 4, False, b.ZERO),
+]
+
+
+@pytest.mark.parametrize("dims,R,star,boundary", GENERIC_CASES)
+def test_generic_kernel_small_and_odd_shapes(dims, R, star, boundary):
+    ndim = len(dims)
+    w = wl.random_star_weights(ndim, R, 7) if star else wl.random_box_weights(ndim, R, 7)
+    a = wl.normal_field(dims, 8)
+    used = check(dims, R, b.STAR if star else b.BOX, w, boundary, a, variant=b.VARIANT_GENERIC)
+    assert used == "generic"
+
+
+@pytest.mark.parametrize("steps", [0, 1, 2, 3, 6])
+@pytest.mark.parametrize("boundary", [b.ZERO, b.PERIODIC])
+def test_generic_iteration_and_ping_pong(steps, boundary):
+    dims = (9, 14, 22)
+    w = wl.random_box_weights(3, 1, 11)              # sum|w| = 1: iterates stay bounded
+    a = wl.normal_field(dims, 12)
+    check(dims, 1, b.BOX, w, boundary, a, steps=steps, variant=b.VARIANT_GENERIC)
+
+
+# ------------------------------------------------------------------- stream --
+def _stream_knob_sets(R, box):
+    if box:
+        return [dict(), dict(rows_per_thread=4), dict(rows_per_thread=1)]
+    if R == 1:
+        return [dict(), dict(rows_per_thread=4), dict(rows_per_thread=1)]
+    if R == 4:
+        return [dict(), dict(rows_per_thread=4), dict(tile_y=32, rows_per_thread=2)]
+    return [dict(), dict(rows_per_thread=4)]
+
+
+STREAM_OPS = [(1, False), (2, False), (3, False), (4, False), (1, True)]
+
+
+@pytest.mark.parametrize("R,box", STREAM_OPS)
+@pytest.mark.parametrize("dims,chunk_z,stages", [
+    ((37, 45, 132), 10, 3),      # ragged in x, y and z; several chunks; 2 x-tiles
+    ((8, 16, 128), 0, 0),        # exactly one tile, default knobs
+    ((3, 5, 4), 0, 2),           # smaller than one tile and than the stencil reach
+    ((70, 33, 260), 32, 0),      # three x-tiles, last one 4 points wide
+])
+def test_stream_kernel_matches_oracle(R, box, dims, chunk_z, stages):
+    w = wl.random_box_weights(3, R, 21) if box else wl.random_star_weights(3, R, 21)
+    a = wl.normal_field(dims, 22)
+    for knobs in _stream_knob_sets(R, box):
+        used = check(dims, R, b.BOX if box else b.STAR, w, b.ZERO, a, variant=b.VARIANT_STREAM,
+                     chunk_z=chunk_z or None, stages=stages or None, **knobs)
+        assert used == "stream"
+
+
+@pytest.mark.parametrize("R,box", STREAM_OPS)
+@pytest.mark.parametrize("steps", [2, 5])
+def test_stream_iteration(R, box, steps):
+    dims = (21, 40, 136)
+    w = wl.random_box_weights(3, R, 31) if box else wl.random_star_weights(3, R, 31)
+    a = wl.normal_field(dims, 32)
+    check(dims, R, b.BOX if box else b.STAR, w, b.ZERO, a, steps=steps, variant=b.VARIANT_STREAM)
+
+
+def test_stream_streaming_store_and_determinism():
+    dims = (40, 50, 256)
+    w = wl.fd8_laplacian_weights(3)
+    a = wl.smooth_sine_field(dims, 4)
+    one, _ = gpu_sweep(dims, 4, b.STAR, w, b.ZERO, a, variant=b.VARIANT_STREAM, streaming_store=1)
+    two, _ = gpu_sweep(dims, 4, b.STAR, w, b.ZERO, a, variant=b.VARIANT_STREAM, repeat=3)
+    assert np.array_equal(one, two)                 # same summation order, bitwise repeatable
+    want = oracle.apply(a, w, b.ZERO, 1)
+    assert np.max(np.abs(one - want)) <= wl.tolerance(w, float(np.abs(a).max()), 1)
+
+
+def test_time_composition_on_gpu():
+    dims = (24, 32, 64)
+    w = wl.star_weights(3, 1, 0.4, [0.1])
+    a = wl.uniform_field(dims, 0.0, 1.0, 41)
+    full, _ = gpu_sweep(dims, 1, b.STAR, w, b.ZERO, a, steps=7)
+    half, _ = gpu_sweep(dims, 1, b.STAR, w, b.ZERO, a, steps=3)
+    rest, _ = gpu_sweep(dims, 1, b.STAR, w, b.ZERO, half, steps=4)
+    assert np.max(np.abs(full - rest)) <= wl.tolerance(w, 1.0, 7)
+
+
+def test_apply_host_round_trip():
+    wk = wl.get("cfg2").scaled((40, 48, 128))
+    a = wk.input()
+    w = wk.weights()
+    src = torch.from_numpy(a).pin_memory()
+    dst = torch.empty_like(src).pin_memory()
+    with b.Plan.for_workload(wk) as p:
+        p.apply_host(src, dst, 1, torch.cuda.current_stream().cuda_stream)
+        assert p.launches == 1
+        assert p.get(b.KEY_SCRATCH_BYTES) == 2 * a.nbytes
+    want = oracle.apply(a, w, b.ZERO, 1)
+    assert np.max(np.abs(dst.numpy() - want)) <= wl.tolerance(w, float(np.abs(a).max()), 1)
+
+
+def test_non_default_stream():
+    dims = (16, 32, 128)
+    w = wl.random_box_weights(3, 1, 51)
+    a = wl.normal_field(dims, 52)
+    s = torch.cuda.Stream()
+    src = torch.from_numpy(a).cuda()
+    dst = torch.empty_like(src)
+    torch.cuda.synchronize()
+    with b.Plan(dims, 1, b.BOX, w, b.ZERO) as p:
+        with torch.cuda.stream(s):
+            p.apply(src, dst, 3, s.cuda_stream)
+        s.synchronize()
+        assert p.launches == 3
+    want = oracle.apply(a, w, b.ZERO, 3)
+    assert np.max(np.abs(dst.cpu().numpy() - want)) <= wl.tolerance(w, float(np.abs(a).max()), 3)
+
+
+# ----------------------------------------------------- the five full configs --
+@pytest.mark.parametrize("name", wl.BASELINE_CONFIGS)
+def test_baseline_config_full_size(name):
+    """Full-size grids, default plan (the launch configuration the benchmark
+    times), every point compared with the oracle."""
+    wk = wl.get(name)
+    a = wk.input()
+    w = wk.weights()
+    got, used = gpu_sweep(wk.dims, wk.radius, wk.shape, w, wk.boundary, a, wk.steps)
+    want = oracle.apply(a, w, wk.boundary, wk.steps)
+    tol = wl.tolerance(w, float(np.abs(a).max()), wk.steps)
+    err = float(np.max(np.abs(got - want)))
+    assert err <= tol, f"{name} ({used}): max err {err:.3e} > tol {tol:.3e}"
+    if name == "cfg5":
+        # max principle of the heat update: 0 <= u <= max u0
+        assert got.min() >= 0.0 and got.max() <= a.max()
+
+
+def test_generic_kernel_on_a_full_3d_config():
+    wk = wl.get("cfg2").scaled((128, 128, 128))
+    a, w = wk.input(), wk.weights()
+    check(wk.dims, wk.radius, wk.shape, w, wk.boundary, a, variant=b.VARIANT_GENERIC)
