@@ -154,6 +154,13 @@ def config_summary(wk, total_ms, steps, peak):
             "taps": wk.taps()}
 
 
+def pick_workload(args):
+    wk = wl.get(args.workload)
+    if args.dims:
+        wk = wk.scaled(tuple(int(v) for v in args.dims.split(",")), name=wk.name)
+    return wk
+
+
 def run_gpu(args):
     import torch
     from paper_2608_21157_b200 import binding as b
@@ -177,7 +184,7 @@ def run_gpu(args):
     b.load()
 
     peak, peak_kind = measured_hbm_peak()
-    wk = wl.get(args.workload)
+    wk = pick_workload(args)
     knobs = dict(tile_y=args.tile_y, chunk_z=args.chunk_z, stages=args.stages,
                  rows_per_thread=args.rows_per_thread, streaming_store=args.streaming_store,
                  fuse_steps=args.fuse_steps)
@@ -407,7 +414,7 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    wk = wl.get(args.workload)
+    wk = pick_workload(args)
     a_host = wk.input()
     w = wk.weights()
     cores = oracle.num_threads()
@@ -451,6 +458,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--dims", default=None, help="override the grid, e.g. 256,512,512 (profiling on smaller cases)")
     ap.add_argument("--variant", default="auto", choices=["auto", "generic", "stream", "fused"])
     ap.add_argument("--tile-y", dest="tile_y", type=int, default=None)
     ap.add_argument("--rows-per-thread", dest="rows_per_thread", type=int, default=None)
