@@ -55,15 +55,18 @@ enum {
     STENCIL_VARIANT_AUTO    = 0,
     STENCIL_VARIANT_GENERIC = 1,   /* one thread per point, global-memory gather; any request    */
     STENCIL_VARIANT_STREAM  = 2,   /* TMA-staged x-y tiles streamed along the slowest axis       */
-    STENCIL_VARIANT_FUSED   = 3    /* STREAM with several time steps fused per pass              */
+    STENCIL_VARIANT_FUSED   = 3    /* set only: STREAM, and fail unless iterated applies can fuse
+                                      several time steps per pass; reads back as STREAM with
+                                      STENCIL_KEY_FUSE_STEPS >= 2                                */
 };
 
 /* Keys of stencil_plan_set / stencil_plan_get. */
 enum {
     STENCIL_KEY_VARIANT      = 0,  /* set/get: STENCIL_VARIANT_*                                 */
-    STENCIL_KEY_TILE_X       = 1,  /* set/get: tile width in points (0 = default)                */
+    STENCIL_KEY_TILE_X       = 1,  /* set/get: region width of fused passes, 128 or 256 (0 = auto) */
     STENCIL_KEY_TILE_Y       = 2,  /* set/get: tile height in rows   (0 = default)               */
-    STENCIL_KEY_FUSE_STEPS   = 3,  /* set/get: time steps fused per pass (0 = default, 1 = off)  */
+    STENCIL_KEY_FUSE_STEPS   = 3,  /* set: time steps fused per pass (0 = auto, 1 = off);
+                                      get: the number iterated applies will use (1 = none)       */
     STENCIL_KEY_LAUNCHES     = 4,  /* get: kernels launched by this plan so far                  */
     STENCIL_KEY_SCRATCH_BYTES= 5,  /* get: device bytes the plan currently owns as scratch       */
     STENCIL_KEY_CHUNK_Z      = 6,  /* set/get: planes per CTA along the streamed axis (0 = auto) */

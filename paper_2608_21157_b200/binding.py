@@ -146,7 +146,7 @@ class Plan:
         if variant is not None:
             self.set(KEY_VARIANT, variant)
         keys = {"tile_y": KEY_TILE_Y, "chunk_z": KEY_CHUNK_Z, "stages": KEY_STAGES,
-                "fuse_steps": KEY_FUSE_STEPS, "streaming_store": KEY_STREAMING_STORE,
+                "fuse_steps": KEY_FUSE_STEPS, "tile_x": KEY_TILE_X, "streaming_store": KEY_STREAMING_STORE,
                 "rows_per_thread": KEY_ROWS_PER_THREAD}
         for name, value in knobs.items():
             if value is not None:

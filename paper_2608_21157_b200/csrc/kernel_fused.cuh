@@ -1,0 +1,268 @@
+// FUSED kernel: temporal blocking for the iterated 3D star sweep with a zero
+// boundary.  One pass over the grid advances it by up to T time steps while
+// reading the input once and writing the result once.
+//
+// A CTA owns a TXE x TYE region of the x-y plane (its output tile plus a halo
+// of T*R cells that is recomputed redundantly) and a range of z.  Input planes
+// arrive through a TMA ring exactly as in the single-step kernel.  Time level
+// l (1..T) is computed from level l-1 one plane at a time:
+//
+//   - each thread owns the same K rows x one float4 column at every level, so
+//     the centre values of level l-1 are already in its registers;
+//   - the rows above/below its block and the cells left/right of a warp come
+//     from the level's plane in shared memory (double-buffered; one CTA
+//     barrier per level per plane);
+//   - the +-z taps never touch shared memory: forward accumulation with a
+//     register queue, as in the single-step kernel.
+//
+// Level l lags level l-1 by R planes.  Cells outside the grid are forced back
+// to zero at every level (the zero boundary holds at every time step), and
+// every intermediate level is an fp32 value, so the result equals T separate
+// sweeps up to summation order.  The last level goes straight to global
+// memory; only the tile interior is stored.
+#pragma once
+#include "common.cuh"
+#include "kernel_stream.cuh"
+#include "ptx.cuh"
+
+namespace stencil {
+
+struct FusedGeom {
+    int nz, ny, nx;
+    int tiles_x, tiles_y;
+    int tile_x, tile_y;        // output tile (interior) size
+    int halo_x, halo_y;        // region = tile + 2*halo; halo_x is a multiple of 4
+    int chunk_z;
+    int stages;
+    int nlev;                  // time steps advanced by this pass, 1..T
+};
+
+template <int R, int K, int XW, int NWY>
+struct FusedShape {
+    static constexpr int TXE = 128 * XW;
+    static constexpr int TYE = NWY * K;
+    static constexpr int THREADS = XW * NWY * 32;
+    static constexpr int SLOT_FLOATS = (TYE + 2 * R) * TXE;     // R pad rows above and below
+    static constexpr int SLOT_BYTES = SLOT_FLOATS * 4;          // multiple of 512
+    static constexpr int BOX_BYTES = TYE * TXE * 4;
+    static size_t smem_bytes(int stages, int T) {
+        return (size_t)(stages + 2 * (T - 1)) * SLOT_BYTES + 128 + kMaxStages * 8;
+    }
+};
+
+__device__ __forceinline__ void consumer_barrier(int nthreads) {
+    asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+}
+
+template <int R, int T, int K, int XW, int NWY>
+__global__ void __launch_bounds__(XW * NWY * 32, 1)
+stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restrict__ out,
+                     const FusedGeom g, const __grid_constant__ StarWeights<R> sw,
+                     int* __restrict__ status) {
+    using S = FusedShape<R, K, XW, NWY>;
+    constexpr int TXE = S::TXE;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    unsigned char* base = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    const int nstage = g.stages;
+    float* ring = reinterpret_cast<float*>(base);                                   // nstage slots
+    float* lvl = ring + (size_t)nstage * S::SLOT_FLOATS;                            // (T-1) x 2 slots
+    uint64_t* bars = reinterpret_cast<uint64_t*>(lvl + (size_t)2 * (T - 1) * S::SLOT_FLOATS);
+    const uint32_t full0 = smem_addr(bars);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int wx = warp % XW, wy = warp / XW;
+    const int col = 4 * (wx * 32 + lane);          // x offset inside the region
+    const int row0 = wy * K;                       // first region row of this thread
+
+    // zero the pad rows of every slot once; TMA and the level stores never touch them
+    {
+        const int nslots = nstage + 2 * (T - 1);
+        for (int s = 0; s < nslots; ++s) {
+            float* slot = ring + (size_t)s * S::SLOT_FLOATS;
+            for (int e = tid; e < R * TXE; e += S::THREADS) {
+                slot[e] = 0.0f;
+                slot[(S::TYE + R) * TXE + e] = 0.0f;
+            }
+        }
+    }
+    if (tid == 0) {
+        for (int s = 0; s < nstage; ++s) mbar_init(full0 + 8 * s, 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+
+    const int bid = blockIdx.x;
+    const int tix = bid % g.tiles_x;
+    const int tiy = (bid / g.tiles_x) % g.tiles_y;
+    const int chunk = bid / (g.tiles_x * g.tiles_y);
+    const int x0e = tix * g.tile_x - g.halo_x;     // region origin (may be negative)
+    const int y0e = tiy * g.tile_y - g.halo_y;
+    const int z0 = chunk * g.chunk_z;
+    const int z1 = min(z0 + g.chunk_z, g.nz);
+    const int nlev = g.nlev;
+    const int pstart = z0 - nlev * R;
+    const int nsteps = (z1 - z0) + 2 * nlev * R;
+
+    const int xg = x0e + col;
+    const bool x_in = xg >= 0 && xg < g.nx;
+    const bool x_store = x_in && col >= g.halo_x && col < g.halo_x + g.tile_x;
+    bool cell_in[K], row_store[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const int yg = y0e + row0 + k;
+        const bool y_in = yg >= 0 && yg < g.ny;
+        cell_in[k] = y_in && x_in;
+        row_store[k] = y_in && x_store && (row0 + k) >= g.halo_y && (row0 + k) < g.halo_y + g.tile_y;
+    }
+    const size_t plane_stride = (size_t)g.ny * g.nx;
+
+    int issued = 0;                                // planes requested so far (thread 0 only)
+    if (tid == 0) {
+        prefetch_tensormap(&tmap_in);
+        const int pre = min(nstage, nsteps);
+        issued = pre;
+        for (int i = 0; i < pre; ++i) {
+            mbar_arrive_expect_tx(full0 + 8 * i, S::BOX_BYTES);
+            tma_load_3d(smem_addr(ring + (size_t)i * S::SLOT_FLOATS + R * TXE), &tmap_in, full0 + 8 * i,
+                        x0e, y0e, pstart + i);
+        }
+    }
+
+    float4 q[T][K][R], pend[T][K][R];
+#pragma unroll
+    for (int l = 0; l < T; ++l)
+#pragma unroll
+        for (int k = 0; k < K; ++k)
+#pragma unroll
+            for (int j = 0; j < R; ++j) {
+                q[l][k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                pend[l][k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+
+    bool dead = false;
+    for (int i0 = 0; i0 < nsteps; i0 += R) {
+#pragma unroll
+        for (int u = 0; u < R; ++u) {
+            const int i = i0 + u;
+            if (i >= nsteps) break;
+            const int s = i % nstage;
+            if (!dead && !mbar_wait_bounded(full0 + 8 * s, (i / nstage) & 1)) {
+                dead = true;
+                atomicExch(status, kStatusTimeout);
+            }
+            const float* src = ring + (size_t)s * S::SLOT_FLOATS + R * TXE;     // region row 0
+            float4 cin[K + 2 * R];
+#pragma unroll
+            for (int kk = 0; kk < K + 2 * R; ++kk)
+                cin[kk] = *reinterpret_cast<const float4*>(src + (row0 + kk - R) * TXE + col);
+
+#pragma unroll
+            for (int l = 1; l <= T; ++l) {
+                if (l <= nlev) {
+                    const int zl = pstart + i - l * R;          // plane this level completes now
+                    const bool z_in = zl >= 0 && zl < g.nz;
+                    float4 e[K];
+#pragma unroll
+                    for (int k = 0; k < K; ++k) {
+                        const float4 ctr = cin[k + R];
+                        float v[4 + 2 * R];
+                        v[R + 0] = ctr.x; v[R + 1] = ctr.y; v[R + 2] = ctr.z; v[R + 3] = ctr.w;
+                        {
+                            const float c4[4] = {ctr.x, ctr.y, ctr.z, ctr.w};
+                            const float* rowp = src + (row0 + k) * TXE + col;
+#pragma unroll
+                            for (int t = 0; t < R; ++t) {
+                                float lft = __shfl_up_sync(0xffffffffu, c4[4 - R + t], 1);
+                                float rgt = __shfl_down_sync(0xffffffffu, c4[t], 1);
+                                if (lane == 0) lft = (wx > 0) ? rowp[t - R] : 0.0f;
+                                if (lane == 31) rgt = (wx < XW - 1) ? rowp[4 + t] : 0.0f;
+                                v[t] = lft;
+                                v[R + 4 + t] = rgt;
+                            }
+                        }
+                        float acc[4];
+#pragma unroll
+                        for (int m = 0; m < 4; ++m) {
+                            float a = sw.c * v[R + m];
+#pragma unroll
+                            for (int d = 1; d <= R; ++d) {
+                                a = fmaf(sw.x[R - d], v[R + m - d], a);
+                                a = fmaf(sw.x[R + d], v[R + m + d], a);
+                            }
+#pragma unroll
+                            for (int d = 1; d <= R; ++d) {
+                                a = fmaf(sw.y[R - d], f4get(cin[k + R - d], m), a);
+                                a = fmaf(sw.y[R + d], f4get(cin[k + R + d], m), a);
+                            }
+#pragma unroll
+                            for (int j = 1; j <= R; ++j)
+                                a = fmaf(sw.z[R - j], f4get(q[l - 1][k][(u - j + R) % R], m), a);
+                            acc[m] = a;
+                        }
+#pragma unroll
+                        for (int j = 1; j <= R; ++j) {
+                            float4& p = pend[l - 1][k][(u - j + R) % R];
+                            p.x = fmaf(sw.z[R + j], ctr.x, p.x);
+                            p.y = fmaf(sw.z[R + j], ctr.y, p.y);
+                            p.z = fmaf(sw.z[R + j], ctr.z, p.z);
+                            p.w = fmaf(sw.z[R + j], ctr.w, p.w);
+                        }
+                        float4 done = pend[l - 1][k][u];
+                        pend[l - 1][k][u] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                        q[l - 1][k][u] = ctr;
+                        // the zero boundary holds at every time level
+                        if (!(cell_in[k] && z_in)) done = make_float4(0.f, 0.f, 0.f, 0.f);
+                        e[k] = done;
+                    }
+
+                    if (l == nlev) {
+                        // last level of this pass: interior of the tile goes to global memory
+                        const int zo = zl;
+                        if (!dead && zo >= z0 && zo < z1) {
+                            float* op = out + (size_t)zo * plane_stride + (size_t)(y0e + row0) * g.nx + xg;
+#pragma unroll
+                            for (int k = 0; k < K; ++k)
+                                if (row_store[k]) *reinterpret_cast<float4*>(op + (size_t)k * g.nx) = e[k];
+                        }
+                    } else {
+                        float* buf = lvl + (size_t)(2 * (l - 1) + (i & 1)) * S::SLOT_FLOATS + R * TXE;
+#pragma unroll
+                        for (int k = 0; k < K; ++k)
+                            *reinterpret_cast<float4*>(buf + (row0 + k) * TXE + col) = e[k];
+                    }
+                    if (l < nlev || l == 1) {
+                        // everyone has finished with level l-1's plane and has published level l
+                        consumer_barrier(S::THREADS);
+                        if (l == 1 && tid == 0 && i + nstage < nsteps) {
+                            // the input slot is free: refill it with the plane nstage steps ahead
+                            mbar_arrive_expect_tx(full0 + 8 * s, S::BOX_BYTES);
+                            tma_load_3d(smem_addr(ring + (size_t)s * S::SLOT_FLOATS + R * TXE), &tmap_in,
+                                        full0 + 8 * s, x0e, y0e, pstart + i + nstage);
+                            issued = i + nstage + 1;
+                        }
+                    }
+                    if (l < nlev) {
+                        const float* buf = lvl + (size_t)(2 * (l - 1) + (i & 1)) * S::SLOT_FLOATS + R * TXE;
+                        src = buf;
+#pragma unroll
+                        for (int k = 0; k < K; ++k) cin[k + R] = e[k];
+#pragma unroll
+                        for (int kk = 0; kk < R; ++kk) {
+                            cin[kk] = *reinterpret_cast<const float4*>(buf + (row0 - R + kk) * TXE + col);
+                            cin[K + R + kk] = *reinterpret_cast<const float4*>(buf + (row0 + K + kk) * TXE + col);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    if (dead && tid == 0) {
+        // let copies that may still be in flight land before shared memory is released
+        for (int i = max(0, issued - nstage); i < issued; ++i)
+            mbar_wait_bounded(full0 + 8 * (i % nstage), (i / nstage) & 1);
+    }
+}
+
+}  // namespace stencil

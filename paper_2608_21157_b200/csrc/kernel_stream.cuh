@@ -149,14 +149,15 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
             prefetch_tensormap(&tmap_in);
             bool ok = true;
             int issued = 0;
+            int s = 0;
+            uint32_t ph = 1;                       // parity of the previous use of the slot
             for (int i = 0; i < nplanes; ++i) {
-                const int s = i % nstage;
-                const int n = i / nstage;
-                if (n > 0 && !mbar_wait_bounded(empty0 + 8 * s, (n - 1) & 1)) { ok = false; break; }
+                if (i >= nstage && !mbar_wait_bounded(empty0 + 8 * s, ph)) { ok = false; break; }
                 mbar_arrive_expect_tx(full0 + 8 * s, S::BOX_BYTES);
                 tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_BYTES), &tmap_in, full0 + 8 * s,
                             x0 - 4, y0 - R, pstart + i);
                 issued = i + 1;
+                if (++s == nstage) { s = 0; ph ^= 1; }
             }
             if (!ok) {
                 atomicExch(status, kStatusTimeout);
@@ -173,6 +174,14 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
     const int xg = x0 + 4 * lane;                      // global x of the lane's float4
     const bool x_in = xg < g.nx;
     const size_t plane_stride = (size_t)g.ny * g.nx;
+    bool row_ok[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) row_ok[k] = x_in && (y0 + row0 + k) < g.ny;
+    // next output plane of this thread (advanced after every stored plane)
+    float* op = out + (size_t)z0 * plane_stride + (size_t)(y0 + row0) * g.nx + xg;
+    const int streaming = g.streaming_store;
+    int s = 0;                                      // ring slot and its phase parity
+    uint32_t ph = 0;
 
     if constexpr (!BOX) {
         float4 q[K][R], pend[K][R];
@@ -189,8 +198,7 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
             for (int u = 0; u < R; ++u) {
                 const int i = i0 + u;
                 if (i >= nplanes) break;
-                const int s = i % nstage;
-                if (!mbar_wait_bounded(full0 + 8 * s, (i / nstage) & 1)) {
+                if (!mbar_wait_bounded(full0 + 8 * s, ph)) {
                     atomicExch(status, kStatusTimeout);
                     return;
                 }
@@ -240,13 +248,13 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8 * s);
+                if (++s == nstage) { s = 0; ph ^= 1; }
 
-                if (i >= 2 * R && x_in) {
-                    const int zo = z0 + i - 2 * R;
-                    float* op = out + (size_t)zo * plane_stride + (size_t)(y0 + row0) * g.nx + xg;
+                if (i >= 2 * R) {
 #pragma unroll
                     for (int k = 0; k < K; ++k)
-                        if (y0 + row0 + k < g.ny) store_f4(op + (size_t)k * g.nx, done[k], g.streaming_store);
+                        if (row_ok[k]) store_f4(op + (size_t)k * g.nx, done[k], streaming);
+                    op += plane_stride;
                 }
             }
         }
@@ -260,8 +268,7 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
             for (int d = 0; d <= 2 * R; ++d) T[k][d] = make_float4(0.f, 0.f, 0.f, 0.f);
 
         for (int i = 0; i < nplanes; ++i) {
-            const int s = i % nstage;
-            if (!mbar_wait_bounded(full0 + 8 * s, (i / nstage) & 1)) {
+            if (!mbar_wait_bounded(full0 + 8 * s, ph)) {
                 atomicExch(status, kStatusTimeout);
                 return;
             }
@@ -275,6 +282,7 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + 8 * s);
+            if (++s == nstage) { s = 0; ph ^= 1; }
 
 #pragma unroll
             for (int k = 0; k < K; ++k) {
@@ -296,12 +304,11 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                     T[k][d] = make_float4(a[0], a[1], a[2], a[3]);
                 }
             }
-            if (i >= 2 * R && x_in) {
-                const int zo = z0 + i - 2 * R;
-                float* op = out + (size_t)zo * plane_stride + (size_t)(y0 + row0) * g.nx + xg;
+            if (i >= 2 * R) {
 #pragma unroll
                 for (int k = 0; k < K; ++k)
-                    if (y0 + row0 + k < g.ny) store_f4(op + (size_t)k * g.nx, T[k][2 * R], g.streaming_store);
+                    if (row_ok[k]) store_f4(op + (size_t)k * g.nx, T[k][2 * R], streaming);
+                op += plane_stride;
             }
         }
     }

@@ -16,6 +16,7 @@
 #include "common.cuh"
 #include "kernel_generic.cuh"
 #include "kernel_stream.cuh"
+#include "kernel_fused.cuh"
 
 using namespace stencil;
 
@@ -63,6 +64,17 @@ struct StreamConfig {
                           float*, const StreamGeom&, int grid, size_t smem, cudaStream_t);
 };
 
+// ---------------------------------------------------------------------------
+// FUSED kernel configurations (temporal blocking, 3D star)
+// ---------------------------------------------------------------------------
+struct FusedConfig {
+    int radius, T, K, XW, NWY;
+    int txe, tye, threads, slot_bytes;
+    const void* kernel;
+    cudaError_t (*launch)(const struct stencil_plan_s*, const CUtensorMap&, float*, const FusedGeom&,
+                          int grid, size_t smem, cudaStream_t);
+};
+
 }  // namespace
 
 struct stencil_plan_s {
@@ -84,12 +96,14 @@ struct stencil_plan_s {
     int variant;                   // resolved STENCIL_VARIANT_*
     int tile_y, rows_per_thread, chunk_z, stages, fuse_steps, streaming_store;
     const StreamConfig* stream_cfg;
+    const FusedConfig* fused_cfg;  // non-null: iterated applies run fused passes
+    int tile_x;                    // requested region width for fused passes (0 = auto)
     // bookkeeping
     int64_t launches;
     cudaStream_t last_stream;
     bool used;
     // tensor-map cache: one entry per source pointer
-    struct MapEntry { const float* ptr; const StreamConfig* cfg; CUtensorMap map; };
+    struct MapEntry { const float* ptr; const void* cfg; CUtensorMap map; };
     std::vector<MapEntry> maps;
 };
 
@@ -162,6 +176,55 @@ const StreamConfig* find_stream_cfg(int radius, bool box, int tile_y, int rows_p
     return nullptr;
 }
 
+template <int R>
+void pack_star(const stencil_plan_s* p, StarWeights<R>& sw) {
+    std::memset(&sw, 0, sizeof(sw));
+    sw.c = dense_w(p, 0, 0, 0);
+    for (int d = -R; d <= R; ++d) {
+        if (d == 0) continue;
+        sw.x[d + R] = dense_w(p, 0, 0, d);
+        sw.y[d + R] = dense_w(p, 0, d, 0);
+        sw.z[d + R] = dense_w(p, d, 0, 0);
+    }
+}
+
+template <int R, int T, int K, int XW, int NWY>
+cudaError_t launch_fused_t(const stencil_plan_s* p, const CUtensorMap& map, float* out, const FusedGeom& g,
+                           int grid, size_t smem, cudaStream_t st) {
+    StarWeights<R> sw;
+    pack_star<R>(p, sw);
+    stencil_fused_kernel<R, T, K, XW, NWY>
+        <<<grid, FusedShape<R, K, XW, NWY>::THREADS, smem, st>>>(map, out, g, sw, p->d_status);
+    return cudaGetLastError();
+}
+
+template <int R, int T, int K, int XW, int NWY>
+FusedConfig make_fused() {
+    using S = FusedShape<R, K, XW, NWY>;
+    FusedConfig c;
+    c.radius = R; c.T = T; c.K = K; c.XW = XW; c.NWY = NWY;
+    c.txe = S::TXE; c.tye = S::TYE; c.threads = S::THREADS; c.slot_bytes = S::SLOT_BYTES;
+    c.kernel = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY>);
+    c.launch = &launch_fused_t<R, T, K, XW, NWY>;
+    return c;
+}
+
+// First match of (radius, T, region width) wins; T == 0 / width == 0 match anything.
+const std::vector<FusedConfig>& fused_configs() {
+    static const std::vector<FusedConfig> v = {
+        make_fused<1, 2, 4, 2, 8>(),  make_fused<1, 3, 4, 2, 8>(),
+        make_fused<1, 4, 2, 1, 16>(), make_fused<1, 2, 2, 1, 16>(), make_fused<1, 3, 2, 1, 16>(),
+        make_fused<2, 2, 2, 1, 16>(),
+    };
+    return v;
+}
+
+const FusedConfig* find_fused_cfg(int radius, int T, int txe) {
+    for (const FusedConfig& c : fused_configs())
+        if (c.radius == radius && (T == 0 || c.T == T) && (txe == 0 || c.txe == txe)) return &c;
+    return nullptr;
+}
+
 bool stream_supported(const stencil_plan_s* p) {
     if (p->ndim != 3 || p->boundary != STENCIL_ZERO) return false;
     if (p->nx % 4 != 0) return false;              // TMA global strides must be 16-byte multiples
@@ -169,15 +232,32 @@ bool stream_supported(const stencil_plan_s* p) {
     return find_stream_cfg(p->radius, box, 0, 0) != nullptr;
 }
 
+// Temporal blocking covers what the STREAM kernels cover, restricted to star stencils.
+const FusedConfig* pick_fused(const stencil_plan_s* p) {
+    if (!stream_supported(p) || p->shape != STENCIL_STAR) return nullptr;
+    if (p->fuse_steps == 1) return nullptr;
+    int txe = p->tile_x;
+    if (p->fuse_steps == 0 && txe == 0) {
+        // default: two steps per pass on a 256-wide region when that covers a whole row
+        // (no redundant columns), otherwise four steps on 128-wide regions
+        const FusedConfig* c = p->nx <= 256 ? find_fused_cfg(p->radius, 2, 256) : find_fused_cfg(p->radius, 4, 128);
+        return c ? c : find_fused_cfg(p->radius, 0, 0);
+    }
+    return find_fused_cfg(p->radius, p->fuse_steps, txe);
+}
+
 int resolve_variant(stencil_plan_s* p, int want) {
     if (want == STENCIL_VARIANT_AUTO) want = stream_supported(p) ? STENCIL_VARIANT_STREAM : STENCIL_VARIANT_GENERIC;
-    if (want == STENCIL_VARIANT_GENERIC) { p->variant = want; return STENCIL_OK; }
-    if (want == STENCIL_VARIANT_STREAM) {
+    if (want == STENCIL_VARIANT_GENERIC) { p->variant = want; p->fused_cfg = nullptr; return STENCIL_OK; }
+    if (want == STENCIL_VARIANT_STREAM || want == STENCIL_VARIANT_FUSED) {
         if (!stream_supported(p)) return STENCIL_ERR_UNSUPPORTED;
         const StreamConfig* c = find_stream_cfg(p->radius, p->shape == STENCIL_BOX, p->tile_y, p->rows_per_thread);
         if (!c) return STENCIL_ERR_UNSUPPORTED;
+        const FusedConfig* f = pick_fused(p);
+        if (want == STENCIL_VARIANT_FUSED && !f) return STENCIL_ERR_UNSUPPORTED;
         p->stream_cfg = c;
-        p->variant = want;
+        p->fused_cfg = f;
+        p->variant = STENCIL_VARIANT_STREAM;
         return STENCIL_OK;
     }
     return STENCIL_ERR_UNSUPPORTED;
@@ -231,7 +311,8 @@ int launch_generic(stencil_plan_s* p, const float* src, float* dst, cudaStream_t
     return STENCIL_OK;
 }
 
-int get_tensor_map(stencil_plan_s* p, const StreamConfig* cfg, const float* src, const CUtensorMap** out) {
+int get_tensor_map(stencil_plan_s* p, const void* cfg, int box_x, int box_y, const float* src,
+                   const CUtensorMap** out) {
     for (auto& e : p->maps)
         if (e.ptr == src && e.cfg == cfg) { *out = &e.map; return STENCIL_OK; }
     EncodeTiledFn enc = get_encode_fn();
@@ -240,7 +321,7 @@ int get_tensor_map(stencil_plan_s* p, const StreamConfig* cfg, const float* src,
     e.ptr = src; e.cfg = cfg;
     const cuuint64_t dims[3] = {(cuuint64_t)p->nx, (cuuint64_t)p->ny, (cuuint64_t)p->nz};
     const cuuint64_t strides[2] = {(cuuint64_t)p->nx * 4, (cuuint64_t)p->nx * (cuuint64_t)p->ny * 4};
-    const cuuint32_t box[3] = {(cuuint32_t)kStreamPX, (cuuint32_t)cfg->box_rows, 1};
+    const cuuint32_t box[3] = {(cuuint32_t)box_x, (cuuint32_t)box_y, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = enc(&e.map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(src), dims, strides,
                      box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
@@ -255,7 +336,7 @@ int get_tensor_map(stencil_plan_s* p, const StreamConfig* cfg, const float* src,
 int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
     const StreamConfig* cfg = p->stream_cfg;
     const CUtensorMap* map = nullptr;
-    int rc = get_tensor_map(p, cfg, src, &map);
+    int rc = get_tensor_map(p, cfg, kStreamPX, cfg->box_rows, src, &map);
     if (rc != STENCIL_OK) return rc;
 
     StreamGeom g;
@@ -285,6 +366,56 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
         return STENCIL_ERR_CUDA;
     }
     if (cfg->launch(p, *cfg, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
+    p->launches++;
+    return STENCIL_OK;
+}
+
+// One fused pass: dst = S^nlev(src), nlev <= cfg->T.
+int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cudaStream_t st) {
+    const FusedConfig* cfg = p->fused_cfg;
+    const CUtensorMap* map = nullptr;
+    int rc = get_tensor_map(p, cfg, cfg->txe, cfg->tye, src, &map);
+    if (rc != STENCIL_OK) return rc;
+    const int R = p->radius, T = cfg->T;
+    FusedGeom g;
+    g.nz = p->nz; g.ny = p->ny; g.nx = p->nx;
+    g.nlev = nlev;
+    if (p->nx <= cfg->txe) {                     // one region spans the row: the x halo is the zero boundary
+        g.halo_x = 0; g.tile_x = cfg->txe; g.tiles_x = 1;
+    } else {
+        g.halo_x = (T * R + 3) / 4 * 4;
+        g.tile_x = cfg->txe - 2 * g.halo_x;
+        g.tiles_x = (p->nx + g.tile_x - 1) / g.tile_x;
+    }
+    g.halo_y = T * R;
+    g.tile_y = cfg->tye - 2 * g.halo_y;
+    if (g.tile_x < 4 || g.tile_y < 1) return STENCIL_ERR_UNSUPPORTED;
+    g.tiles_y = (p->ny + g.tile_y - 1) / g.tile_y;
+    // shared memory: input ring + two planes per intermediate level
+    int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
+    auto smem_for = [&](int s) { return (size_t)(s + 2 * (T - 1)) * cfg->slot_bytes + 128 + kMaxStages * sizeof(uint64_t); };
+    while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;
+    const size_t smem = smem_for(stages);
+    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
+    g.stages = stages;
+    const int tiles = g.tiles_x * g.tiles_y;
+    int chunk = p->chunk_z;
+    if (chunk <= 0) {
+        // one CTA per SM: as many z chunks as fill the 148 SMs once, but not so short that
+        // the 2*T*R extra input planes per chunk dominate
+        int nchunks = std::max(1, 148 / std::max(tiles, 1));
+        nchunks = std::min(nchunks, std::max(1, p->nz / (4 * T * R)));
+        chunk = (p->nz + nchunks - 1) / nchunks;
+    }
+    chunk = std::max(1, std::min(chunk, p->nz));
+    g.chunk_z = chunk;
+    const int64_t grid64 = (int64_t)tiles * ((p->nz + chunk - 1) / chunk);
+    if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
+    if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        cudaGetLastError();
+        return STENCIL_ERR_CUDA;
+    }
+    if (cfg->launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
     p->launches++;
     return STENCIL_OK;
 }
@@ -336,7 +467,7 @@ int stencil_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int ra
     p->host_in = nullptr; p->host_out = nullptr;
     p->variant = STENCIL_VARIANT_GENERIC;
     p->tile_y = 0; p->rows_per_thread = 0; p->chunk_z = 0; p->stages = 0; p->fuse_steps = 0; p->streaming_store = 0;
-    p->stream_cfg = nullptr;
+    p->stream_cfg = nullptr; p->fused_cfg = nullptr; p->tile_x = 0;
     p->launches = 0; p->last_stream = nullptr; p->used = false;
 
     const int side = 2 * radius + 1;
@@ -389,13 +520,21 @@ int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void
         rc = ensure_grid(&p->scratch, p->npoints);
         if (rc != STENCIL_OK) return rc;
     }
-    // ping-pong so that the last sweep writes `out` and `in` stays intact
+    // A pass advances the field by T time steps (T = 1 without temporal blocking).
+    // Ping-pong between `out` and the scratch grid so that the last pass writes
+    // `out` and `in` stays intact.
+    const bool fuse = p->variant == STENCIL_VARIANT_STREAM && p->fused_cfg != nullptr && steps > 1;
+    const int T = fuse ? p->fused_cfg->T : 1;
+    const int passes = (steps + T - 1) / T;
     const float* src = in;
-    for (int k = 0; k < steps; ++k) {
-        const int remaining = steps - 1 - k;
+    int done = 0;
+    for (int k = 0; k < passes; ++k) {
+        const int remaining = passes - 1 - k;
         float* dst = (remaining % 2 == 0) ? out : p->scratch;
-        rc = launch_sweep(p, src, dst, st);
+        const int nlev = std::min(T, steps - done);
+        rc = (fuse && nlev > 1) ? launch_fused(p, src, dst, nlev, st) : launch_sweep(p, src, dst, st);
         if (rc != STENCIL_OK) return rc;
+        done += nlev;
         src = dst;
     }
     return STENCIL_OK;
@@ -484,12 +623,28 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
         case STENCIL_KEY_VARIANT: {
             const int old_variant = p->variant;
             const StreamConfig* old_cfg = p->stream_cfg;
+            const FusedConfig* old_fused = p->fused_cfg;
             int rc = resolve_variant(p, (int)value);
-            if (rc != STENCIL_OK) { p->variant = old_variant; p->stream_cfg = old_cfg; }
+            if (rc != STENCIL_OK) { p->variant = old_variant; p->stream_cfg = old_cfg; p->fused_cfg = old_fused; }
             return rc;
         }
         case STENCIL_KEY_TILE_X:
-            return (value == 0 || value == kStreamTX) ? STENCIL_OK : STENCIL_ERR_UNSUPPORTED;
+        case STENCIL_KEY_FUSE_STEPS: {
+            // region width (128 or 256) and time steps per pass of the fused kernel
+            if (value < 0) return STENCIL_ERR_INVALID;
+            const int old_fuse = p->fuse_steps, old_tx = p->tile_x;
+            if (key == STENCIL_KEY_TILE_X) p->tile_x = (int)value; else p->fuse_steps = (int)value;
+            if (p->variant == STENCIL_VARIANT_STREAM) {
+                const FusedConfig* f = pick_fused(p);
+                const bool wants_fusion = p->fuse_steps > 1 || (key == STENCIL_KEY_TILE_X && value != 0 && p->fuse_steps != 1);
+                if (!f && wants_fusion) { p->fuse_steps = old_fuse; p->tile_x = old_tx; return STENCIL_ERR_UNSUPPORTED; }
+                p->fused_cfg = f;
+            } else if (p->fuse_steps > 1) {
+                p->fuse_steps = old_fuse; p->tile_x = old_tx;
+                return STENCIL_ERR_UNSUPPORTED;
+            }
+            return STENCIL_OK;
+        }
         case STENCIL_KEY_TILE_Y:
         case STENCIL_KEY_ROWS_PER_THREAD: {
             if (value < 0) return STENCIL_ERR_INVALID;
@@ -504,10 +659,6 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
             p->rows_per_thread = k;
             return STENCIL_OK;
         }
-        case STENCIL_KEY_FUSE_STEPS:
-            if (value < 0) return STENCIL_ERR_INVALID;
-            p->fuse_steps = (int)value;
-            return STENCIL_OK;
         case STENCIL_KEY_CHUNK_Z:
             if (value < 0) return STENCIL_ERR_INVALID;
             p->chunk_z = (int)std::min<int64_t>(value, 0x7fffffff);
@@ -528,14 +679,18 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
     if (!valid_plan(p) || !value) return STENCIL_ERR_INVALID;
     switch (key) {
         case STENCIL_KEY_VARIANT: *value = p->variant; return STENCIL_OK;
-        case STENCIL_KEY_TILE_X: *value = p->variant == STENCIL_VARIANT_STREAM ? kStreamTX : 0; return STENCIL_OK;
+        case STENCIL_KEY_TILE_X:
+            *value = p->variant != STENCIL_VARIANT_STREAM ? 0 : (p->fused_cfg ? p->fused_cfg->txe : kStreamTX);
+            return STENCIL_OK;
         case STENCIL_KEY_TILE_Y:
             *value = (p->variant == STENCIL_VARIANT_STREAM && p->stream_cfg) ? p->stream_cfg->tile_y : 0;
             return STENCIL_OK;
         case STENCIL_KEY_ROWS_PER_THREAD:
             *value = (p->variant == STENCIL_VARIANT_STREAM && p->stream_cfg) ? p->stream_cfg->K : 0;
             return STENCIL_OK;
-        case STENCIL_KEY_FUSE_STEPS: *value = p->fuse_steps; return STENCIL_OK;
+        case STENCIL_KEY_FUSE_STEPS:
+            *value = (p->variant == STENCIL_VARIANT_STREAM && p->fused_cfg) ? p->fused_cfg->T : 1;
+            return STENCIL_OK;
         case STENCIL_KEY_LAUNCHES: *value = p->launches; return STENCIL_OK;
         case STENCIL_KEY_SCRATCH_BYTES: {
             int64_t grids = (p->scratch != nullptr) + (p->host_in != nullptr) + (p->host_out != nullptr);

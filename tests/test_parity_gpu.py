@@ -180,6 +180,65 @@ def test_non_default_stream():
     assert np.max(np.abs(dst.cpu().numpy() - want)) <= wl.tolerance(w, float(np.abs(a).max()), 3)
 
 
+# -------------------------------------------------------------------- fused --
+FUSED_CONFIGS = [   # (radius, fuse_steps, region width)
+    (1, 2, 256), (1, 3, 256), (1, 4, 128), (1, 2, 128), (1, 3, 128), (2, 2, 128),
+]
+
+
+@pytest.mark.parametrize("R,T,width", FUSED_CONFIGS)
+@pytest.mark.parametrize("dims,chunk_z", [
+    ((29, 70, 300), 11),        # several regions in x and y, ragged everywhere, several z chunks
+    ((40, 64, 256), 0),         # a 256-wide region spans the whole row
+    ((5, 9, 12), 0),            # much smaller than one region
+])
+def test_fused_passes_match_oracle(R, T, width, dims, chunk_z):
+    w = wl.random_star_weights(3, R, 61)            # asymmetric taps, sum|w| = 1
+    a = wl.normal_field(dims, 62)
+    for steps in (T, T + 1, 2 * T + 1):
+        dev = torch.device("cuda:0")
+        src = torch.from_numpy(a).to(dev)
+        dst = torch.full_like(src, float("nan"))
+        with b.Plan(dims, R, b.STAR, w, b.ZERO, fuse_steps=T, tile_x=width, chunk_z=chunk_z or None) as p:
+            assert p.get(b.KEY_FUSE_STEPS) == T
+            p.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
+            assert p.query_status() == b.OK
+            assert p.launches == -(-steps // T)
+        got = dst.cpu().numpy()
+        want = oracle.apply(a, w, b.ZERO, steps)
+        tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+        err = float(np.max(np.abs(got - want)))
+        assert err <= tol, f"R={R} T={T} width={width} dims={dims} steps={steps}: {err:.3e} > {tol:.3e}"
+
+
+def test_fused_equals_unfused_within_tolerance_and_keeps_zero_boundary():
+    """A field that would leak through the boundary if out-of-grid cells were
+    allowed to evolve inside a fused pass: constant ones, heat weights."""
+    dims = (20, 30, 64)
+    w = wl.star_weights(3, 1, 0.4, [0.1])
+    a = np.ones(dims, dtype=np.float32)
+    fused, _ = gpu_sweep(dims, 1, b.STAR, w, b.ZERO, a, steps=8, fuse_steps=4, tile_x=128)
+    plain, _ = gpu_sweep(dims, 1, b.STAR, w, b.ZERO, a, steps=8, fuse_steps=1)
+    want = oracle.apply(a, w, b.ZERO, 8)
+    tol = wl.tolerance(w, 1.0, 8)
+    assert np.max(np.abs(fused - want)) <= tol and np.max(np.abs(plain - want)) <= tol
+    assert fused[0, 0, 0] < 0.5                     # the corner has lost heat to the zero exterior
+
+
+def test_fuse_knob_rules():
+    star = wl.star_weights(3, 1, 0.4, [0.1])
+    with b.Plan((64, 64, 64), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) >= 2         # iterated applies fuse by default
+        p.set(b.KEY_FUSE_STEPS, 1)
+        assert p.get(b.KEY_FUSE_STEPS) == 1
+        with pytest.raises(b.StencilError):
+            p.set(b.KEY_FUSE_STEPS, 7)
+    with b.Plan((64, 64, 64), 1, b.BOX, wl.random_box_weights(3, 1, 3), b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # no fused kernel for box stencils
+        with pytest.raises(b.StencilError):
+            p.set(b.KEY_VARIANT, b.VARIANT_FUSED)
+
+
 # ----------------------------------------------------- the five full configs --
 @pytest.mark.parametrize("name", wl.BASELINE_CONFIGS)
 def test_baseline_config_full_size(name):
