@@ -47,8 +47,12 @@ enum {
     STENCIL_ERR_UNSUPPORTED = -2,  /* valid request outside what the kernels cover               */
     STENCIL_ERR_CUDA        = -3,  /* a CUDA runtime/driver call failed (or no device)           */
     STENCIL_ERR_ALLOC       = -4,  /* host or device allocation failed                           */
-    STENCIL_ERR_TIMEOUT     = -5   /* a bounded device-side wait gave up (see query_status)      */
+    STENCIL_ERR_TIMEOUT     = -5,  /* a bounded device-side wait gave up (see query_status)      */
+    STENCIL_ERR_TOO_LARGE   = -6   /* grid larger than stencil_apply_static's fixed scratch      */
 };
+
+/* Largest grid, in points, that stencil_apply_static accepts (8 MiB of fp32). */
+#define STENCIL_STATIC_MAX_POINTS (1 << 21)
 
 /* Kernel families a plan can run.  AUTO lets the plan choose. */
 enum {
@@ -129,6 +133,38 @@ STENCIL_API int stencil_apply(stencil_plan_t plan, const float* in, float* out, 
  */
 STENCIL_API int stencil_apply_host(stencil_plan_t plan, const float* in_host, float* out_host, int steps,
                        void* stream);
+
+/*
+ * stencil_apply_static — stencil_apply for callers that must not allocate
+ * device memory.  (An addition of this library; the paper has no counterpart.)
+ *
+ * Some programs cannot call cudaMalloc where they run the sweep: a solver or
+ * server that has already handed all device memory to its own pool, or a
+ * time-stepping loop that cannot afford the device-wide stall cudaMalloc and
+ * cudaFree bring.  stencil_apply allocates on first use (a status word, the tap
+ * list, and for steps > 1 a scratch grid).  This entry point allocates nothing,
+ * neither through the CUDA runtime nor through any library: its ping-pong grid
+ * and tap list sit in one fixed array inside the library, 8 MiB + 79 KiB of
+ * device memory that every GPU which loads the library holds until the process
+ * ends.
+ *
+ *   in, out, steps, stream   exactly as for stencil_apply; the result is the
+ *                            same up to fp32 summation order (it runs the
+ *                            one-thread-per-point kernel, whatever the plan's
+ *                            variant).
+ *   limit                    prod(dims) <= STENCIL_STATIC_MAX_POINTS, else
+ *                            STENCIL_ERR_TOO_LARGE and nothing is enqueued.
+ *
+ * The first call on each device also looks up the array's device address (the
+ * name of the array is not an address on the host); make that first call with
+ * the device current and before starting any stream capture.  All calls, from
+ * all plans, share the one array: two calls whose GPU work overlaps (different
+ * streams, or different host threads) race on it and on the tap list, so
+ * serialise them.  Nothing has to be cleared between calls: each call rewrites
+ * the taps and writes every scratch cell before reading it.
+ */
+STENCIL_API int stencil_apply_static(stencil_plan_t plan, const float* in, float* out, int steps,
+                                     void* stream);
 
 /* stencil_destroy — free the plan and everything it owns.  NULL is a no-op. */
 STENCIL_API int stencil_destroy(stencil_plan_t plan);

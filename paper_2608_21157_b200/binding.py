@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libstencil_b200.so")
 STAR, BOX = 0, 1
 ZERO, PERIODIC = 0, 1
 
-OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_ALLOC, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_ALLOC, ERR_TIMEOUT, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6
+STATIC_MAX_POINTS = 1 << 21
 
 VARIANT_AUTO, VARIANT_GENERIC, VARIANT_STREAM, VARIANT_FUSED = 0, 1, 2, 3
 
@@ -28,7 +29,7 @@ VARIANT_AUTO, VARIANT_GENERIC, VARIANT_STREAM, VARIANT_FUSED = 0, 1, 2, 3
 
 #: every symbol include/stencil.h declares
 EXPORTS = (
-    "stencil_plan", "stencil_apply", "stencil_apply_host", "stencil_destroy",
+    "stencil_plan", "stencil_apply", "stencil_apply_host", "stencil_apply_static", "stencil_destroy",
     "stencil_status_string", "stencil_variant_name", "stencil_query_status",
     "stencil_plan_set", "stencil_plan_get",
 )
@@ -60,6 +61,8 @@ def load() -> ctypes.CDLL:
     lib.stencil_apply.argtypes = [vp, vp, vp, ctypes.c_int, vp]
     lib.stencil_apply_host.restype = ctypes.c_int
     lib.stencil_apply_host.argtypes = [vp, vp, vp, ctypes.c_int, vp]
+    lib.stencil_apply_static.restype = ctypes.c_int
+    lib.stencil_apply_static.argtypes = [vp, vp, vp, ctypes.c_int, vp]
     lib.stencil_destroy.restype = ctypes.c_int
     lib.stencil_destroy.argtypes = [vp]
     lib.stencil_status_string.restype = ctypes.c_char_p
@@ -108,6 +111,17 @@ def stencil_apply_host(plan, in_ptr: int, out_ptr: int, steps: int, stream: int 
     """``in_ptr`` / ``out_ptr``: host addresses (pinned memory recommended)."""
     return load().stencil_apply_host(plan, ctypes.c_void_p(in_ptr), ctypes.c_void_p(out_ptr),
                                      int(steps), ctypes.c_void_p(stream))
+
+
+def stencil_apply_static(plan, in_ptr: int, out_ptr: int, steps: int, stream: int = 0) -> int:
+    """Like ``stencil_apply`` but never allocates device memory: the scratch is
+    a fixed array inside the library, so grids above ``STATIC_MAX_POINTS`` are
+    refused with ``ERR_TOO_LARGE``.  For callers that cannot call cudaMalloc
+    where they run the sweep (all memory already in their own pool, or no room
+    for the stall an allocation causes).  Calls share that one array: do not let
+    two of them overlap on the GPU."""
+    return load().stencil_apply_static(plan, ctypes.c_void_p(in_ptr), ctypes.c_void_p(out_ptr), int(steps),
+                                       ctypes.c_void_p(stream))
 
 
 def stencil_destroy(plan) -> int:
@@ -183,6 +197,11 @@ class Plan:
         rc = stencil_apply(self._h, self._ptr(src), self._ptr(dst), steps, stream)
         if rc != OK:
             raise StencilError(rc, "stencil_apply")
+
+    def apply_static(self, src, dst, steps: int = 1, stream: int = 0) -> None:
+        rc = stencil_apply_static(self._h, self._ptr(src), self._ptr(dst), steps, stream)
+        if rc != OK:
+            raise StencilError(rc, "stencil_apply_static")
 
     def apply_host(self, src, dst, steps: int = 1, stream: int = 0) -> None:
         rc = stencil_apply_host(self._h, self._ptr(src), self._ptr(dst), steps, stream)

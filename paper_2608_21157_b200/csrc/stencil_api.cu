@@ -10,6 +10,7 @@
 #include <cstdint>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -429,6 +430,41 @@ int launch_sweep(stencil_plan_s* p, const float* src, float* dst, cudaStream_t s
 
 bool valid_plan(const stencil_plan_s* p) { return p && p->magic == kPlanMagic; }
 
+// ---------------------------------------------------------------------------
+// Fixed scratch for stencil_apply_static: the ping-pong grid and the tap list
+// live in one file-scope device array, so that entry point never allocates.
+// Every GPU that loads the library holds these bytes until the process exits.
+// ---------------------------------------------------------------------------
+constexpr int64_t kStaticMaxPoints = STENCIL_STATIC_MAX_POINTS;
+constexpr int kStaticMaxTaps = (2 * kMaxRadius + 1) * (2 * kMaxRadius + 1) * (2 * kMaxRadius + 1);
+constexpr size_t kStaticGridBytes = (size_t)kStaticMaxPoints * sizeof(float);
+constexpr size_t kStaticTapBytes = ((size_t)kStaticMaxTaps * sizeof(Tap) + 255) / 256 * 256;
+constexpr int kStaticMaxDevices = 64;
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticGridBytes + kStaticTapBytes];
+
+// In host code `g_static_scratch` is only a handle; the device address has to be
+// asked for, once per device, while that device is current.
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[kStaticMaxDevices] = {nullptr};
+
+int static_scratch_address(unsigned char** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    if (dev < 0 || dev >= kStaticMaxDevices) return STENCIL_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return STENCIL_ERR_CUDA;
+        }
+        g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
+    }
+    *out = g_static_ptr[dev];
+    return STENCIL_OK;
+}
+
 }  // namespace
 
 // ===========================================================================
@@ -562,6 +598,55 @@ int stencil_apply_host(stencil_plan_t p, const float* in_host, float* out_host, 
     return STENCIL_OK;
 }
 
+int stencil_apply_static(stencil_plan_t p, const float* in, float* out, int steps, void* stream) {
+    if (!valid_plan(p) || !in || !out || steps < 0) return STENCIL_ERR_INVALID;
+    const uintptr_t a = reinterpret_cast<uintptr_t>(in), b = reinterpret_cast<uintptr_t>(out);
+    if ((a | b) & 15u) return STENCIL_ERR_INVALID;
+    const uintptr_t bytes = (uintptr_t)p->npoints * sizeof(float);
+    if (a < b + bytes && b < a + bytes) return STENCIL_ERR_INVALID;
+    if (p->npoints > kStaticMaxPoints || (int64_t)p->taps.size() > kStaticMaxTaps) return STENCIL_ERR_TOO_LARGE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+
+    unsigned char* base = nullptr;                 // first call on a device also looks the array up
+    int rc = static_scratch_address(&base);
+    if (rc != STENCIL_OK) return rc;
+    float* grid = reinterpret_cast<float*>(base);
+    Tap* taps = reinterpret_cast<Tap*>(base + kStaticGridBytes);
+
+    if (steps == 0) {
+        if (cudaMemcpyAsync(out, in, bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+            cudaGetLastError();
+            return STENCIL_ERR_CUDA;
+        }
+        return STENCIL_OK;
+    }
+    const int ntaps = (int)p->taps.size();
+    if (ntaps > 0 && cudaMemcpyAsync(taps, p->taps.data(), (size_t)ntaps * sizeof(Tap), cudaMemcpyHostToDevice,
+                                     st) != cudaSuccess) {
+        cudaGetLastError();
+        return STENCIL_ERR_CUDA;
+    }
+    // Same ping-pong as stencil_apply, with the fixed array in place of the plan's
+    // scratch grid.  Every cell of it is written before it is read, so nothing of
+    // an earlier call's contents has to be cleared.
+    Grid g{p->nz, p->ny, p->nx};
+    const int64_t blocks_needed = (p->npoints + kGenericThreads - 1) / kGenericThreads;
+    const int nblocks = (int)std::min<int64_t>(blocks_needed, 148 * 16);
+    const float* src = in;
+    for (int k = 0; k < steps; ++k) {
+        const int remaining = steps - 1 - k;
+        float* dst = (remaining % 2 == 0) ? out : grid;
+        if (p->boundary == STENCIL_PERIODIC)
+            stencil_generic_kernel<true><<<nblocks, kGenericThreads, 0, st>>>(src, dst, g, taps, ntaps);
+        else
+            stencil_generic_kernel<false><<<nblocks, kGenericThreads, 0, st>>>(src, dst, g, taps, ntaps);
+        if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
+        p->launches++;
+        src = dst;
+    }
+    return STENCIL_OK;
+}
+
 int stencil_destroy(stencil_plan_t p) {
     if (!p) return STENCIL_OK;
     if (!valid_plan(p)) return STENCIL_ERR_INVALID;
@@ -590,6 +675,7 @@ const char* stencil_status_string(int status) {
         case STENCIL_ERR_CUDA: return "CUDA call failed or no device";
         case STENCIL_ERR_ALLOC: return "allocation failed";
         case STENCIL_ERR_TIMEOUT: return "bounded device wait expired";
+        case STENCIL_ERR_TOO_LARGE: return "grid exceeds the fixed scratch of stencil_apply_static";
         default: return "unknown status";
     }
 }
