@@ -62,8 +62,8 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
     using S = FusedShape<R, K, XW, NWY>;
     constexpr int TXE = S::TXE;
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    unsigned char* base = reinterpret_cast<unsigned char*>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    // indexing the shared array keeps every derived pointer in the shared address space
+    unsigned char* base = smem_raw + ((128u - (smem_addr(smem_raw) & 127u)) & 127u);
     const int nstage = g.stages;
     float* ring = reinterpret_cast<float*>(base);                                   // nstage slots
     float* lvl = ring + (size_t)nstage * S::SLOT_FLOATS;                            // (T-1) x 2 slots
@@ -176,8 +176,14 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                             for (int t = 0; t < R; ++t) {
                                 float lft = __shfl_up_sync(0xffffffffu, c4[4 - R + t], 1);
                                 float rgt = __shfl_down_sync(0xffffffffu, c4[t], 1);
-                                if (lane == 0) lft = (wx > 0) ? rowp[t - R] : 0.0f;
-                                if (lane == 31) rgt = (wx < XW - 1) ? rowp[4 + t] : 0.0f;
+                                // warp-edge lanes: the neighbour warp's value from the plane in
+                                // shared memory, or zero at the edge of the region
+                                if (lane == 0) lft = 0.0f;
+                                if (lane == 31) rgt = 0.0f;
+                                if (XW > 1) {
+                                    lft = lds_if(lane == 0 && wx > 0, rowp + t - R, lft);
+                                    rgt = lds_if(lane == 31 && wx < XW - 1, rowp + 4 + t, rgt);
+                                }
                                 v[t] = lft;
                                 v[R + 4 + t] = rgt;
                             }

@@ -19,6 +19,9 @@
 // from registers.  Every intermediate stays in registers; shared memory only
 // holds the ring of input planes.
 #pragma once
+#include <type_traits>
+#include <utility>
+
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -59,6 +62,18 @@ struct StreamShape {
     static size_t smem_bytes(int stages) { return (size_t)stages * PLANE_BYTES + 128 + 128; }
 };
 
+// Calls f(integral_constant<int, 0>) ... f(integral_constant<int, N-1>) in order and
+// stops at the first call that returns false.  The index is a compile-time constant
+// inside f, which keeps register arrays indexed by it in registers.
+template <class F, int... Is>
+__device__ __forceinline__ bool static_for_impl(F&& f, std::integer_sequence<int, Is...>) {
+    return (f(std::integral_constant<int, Is>{}) && ...);
+}
+template <int N, class F>
+__device__ __forceinline__ bool static_for(F&& f) {
+    return static_for_impl(f, std::make_integer_sequence<int, N>{});
+}
+
 __device__ __forceinline__ float f4get(const float4& v, int m) {
     return m == 0 ? v.x : (m == 1 ? v.y : (m == 2 ? v.z : v.w));
 }
@@ -66,6 +81,19 @@ __device__ __forceinline__ float f4get(const float4& v, int m) {
 __device__ __forceinline__ void store_f4(float* p, const float4& v, int streaming) {
     if (streaming) __stcs(reinterpret_cast<float4*>(p), v);
     else *reinterpret_cast<float4*>(p) = v;
+}
+
+// Predicated shared-memory load: returns *p where `take` holds, `keep` elsewhere,
+// without a divergent branch.
+__device__ __forceinline__ float lds_if(bool take, const float* p, float keep) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "setp.ne.u32 q, %2, 0;\n\t"
+        "@q ld.shared.f32 %0, [%1];\n\t}"
+        : "+f"(keep)
+        : "r"(smem_addr(p)), "r"((uint32_t)take)
+        : "memory");
+    return keep;
 }
 
 // Fills v[0 .. 4+2R) with the R values left of the lane's float4, the float4
@@ -80,12 +108,14 @@ __device__ __forceinline__ void gather_row(const float* rowp, const float* rowba
         const float c4[4] = {ctr.x, ctr.y, ctr.z, ctr.w};
 #pragma unroll
         for (int t = 0; t < R; ++t) {
-            float l = __shfl_up_sync(0xffffffffu, c4[4 - R + t], 1);
-            float r = __shfl_down_sync(0xffffffffu, c4[t], 1);
-            if (lane == 0) l = rowbase[4 - R + t];
-            if (lane == 31) r = rowbase[4 + kStreamTX + t];
-            v[t] = l;
-            v[R + 4 + t] = r;
+            // every lane reads the two halo words (a broadcast, one wavefront each, no
+            // branch); only the end lanes keep them
+            const float hl = rowbase[4 - R + t];
+            const float hr = rowbase[4 + kStreamTX + t];
+            const float l = __shfl_up_sync(0xffffffffu, c4[4 - R + t], 1);
+            const float r = __shfl_down_sync(0xffffffffu, c4[t], 1);
+            v[t] = lane == 0 ? hl : l;
+            v[R + 4 + t] = lane == 31 ? hr : r;
         }
     } else {
         const float4 l = *reinterpret_cast<const float4*>(rowp - 4);
@@ -110,9 +140,10 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
     using S = StreamShape<R, K, NW>;
     constexpr int PX = kStreamPX;
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    // ring of planes first (128-byte aligned slots), then the barriers
-    unsigned char* ring = reinterpret_cast<unsigned char*>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    // ring of planes first (128-byte aligned slots), then the barriers.  The pointer is
+    // formed by indexing the shared array (no integer round trip), so the compiler
+    // keeps it in the shared address space and emits ld.shared for the plane reads.
+    unsigned char* ring = smem_raw + ((128u - (smem_addr(smem_raw) & 127u)) & 127u);
     uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)g.stages * S::PLANE_BYTES);
     const uint32_t full0 = smem_addr(bars);
     const uint32_t empty0 = smem_addr(bars + kMaxStages);
@@ -193,15 +224,14 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                 pend[k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
 
+        // R planes per trip; the slot of the register queues that a plane uses is a
+        // compile-time constant inside each of the R copies of the body
         for (int i0 = 0; i0 < nplanes; i0 += R) {
-#pragma unroll
-            for (int u = 0; u < R; ++u) {
+            const bool ok = static_for<R>([&](auto uc) -> bool {
+                constexpr int u = decltype(uc)::value;
                 const int i = i0 + u;
-                if (i >= nplanes) break;
-                if (!mbar_wait_bounded(full0 + 8 * s, ph)) {
-                    atomicExch(status, kStatusTimeout);
-                    return;
-                }
+                if (i >= nplanes) return true;
+                if (!mbar_wait_bounded(full0 + 8 * s, ph)) return false;
                 const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
                 const float* colp = pl + row0 * PX + 4 + 4 * lane;
                 float4 c[K + 2 * R];
@@ -247,7 +277,7 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                     q[k][u] = ctr;
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8 * s);
+                mbar_arrive_if(lane == 0, empty0 + 8 * s);
                 if (++s == nstage) { s = 0; ph ^= 1; }
 
                 if (i >= 2 * R) {
@@ -256,59 +286,76 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                         if (row_ok[k]) store_f4(op + (size_t)k * g.nx, done[k], streaming);
                     op += plane_stride;
                 }
-            }
-        }
-    } else {
-        // acc[k][j]: partial output of plane (i-1-j)+... carried between planes;
-        // at step i, T[d] (d = 0..2R) is the output plane i - (d - R).
-        float4 T[K][2 * R + 1];
-#pragma unroll
-        for (int k = 0; k < K; ++k)
-#pragma unroll
-            for (int d = 0; d <= 2 * R; ++d) T[k][d] = make_float4(0.f, 0.f, 0.f, 0.f);
-
-        for (int i = 0; i < nplanes; ++i) {
-            if (!mbar_wait_bounded(full0 + 8 * s, ph)) {
+                return true;
+            });
+            if (!ok) {
                 atomicExch(status, kStatusTimeout);
                 return;
             }
-            const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
-            const float* colp = pl + row0 * PX + 4 + 4 * lane;
-            float v[K + 2 * R][4 + 2 * R];
+        }
+    } else {
+        // M = 2R+1 accumulators per row; the accumulator of output plane z lives in slot
+        // z mod M, so nothing is shifted: M planes per trip, slots known at compile time.
+        constexpr int M = 2 * R + 1;
+        float4 T[K][M];
 #pragma unroll
-            for (int kk = 0; kk < K + 2 * R; ++kk) {
-                const float4 ctr = *reinterpret_cast<const float4*>(colp + kk * PX);
-                gather_row<R>(colp + kk * PX, pl + (row0 + kk) * PX, lane, ctr, v[kk]);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty0 + 8 * s);
-            if (++s == nstage) { s = 0; ph ^= 1; }
+        for (int k = 0; k < K; ++k)
+#pragma unroll
+            for (int d = 0; d < M; ++d) T[k][d] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+        for (int i0 = 0; i0 < nplanes; i0 += M) {
+            const bool ok = static_for<M>([&](auto uc) -> bool {
+                constexpr int u = decltype(uc)::value;
+                const int i = i0 + u;
+                if (i >= nplanes) return true;
+                if (!mbar_wait_bounded(full0 + 8 * s, ph)) return false;
+                const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
+                const float* colp = pl + row0 * PX + 4 + 4 * lane;
+                float v[K + 2 * R][4 + 2 * R];
+#pragma unroll
+                for (int kk = 0; kk < K + 2 * R; ++kk) {
+                    const float4 ctr = *reinterpret_cast<const float4*>(colp + kk * PX);
+                    gather_row<R>(colp + kk * PX, pl + (row0 + kk) * PX, lane, ctr, v[kk]);
+                }
+                __syncwarp();
+                mbar_arrive_if(lane == 0, empty0 + 8 * s);
+                if (++s == nstage) { s = 0; ph ^= 1; }
 
 #pragma unroll
-            for (int k = 0; k < K; ++k) {
-                // shift: the accumulator of output plane z moves one slot per input plane
+                for (int k = 0; k < K; ++k) {
 #pragma unroll
-                for (int d = 2 * R; d > 0; --d) T[k][d] = T[k][d - 1];
-                T[k][0] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int d = 0; d < M; ++d) {         // this plane is tap dz = d - R of output i-(d-R)
+                        float4& t = T[k][(u - d + R + 2 * M) % M];
+                        float a[4];
+                        if (d == 0) {                     // first contribution: starts the accumulator
 #pragma unroll
-                for (int d = 0; d <= 2 * R; ++d) {        // T[k][d]: this plane is its tap dz = d - R
-                    float a[4] = {T[k][d].x, T[k][d].y, T[k][d].z, T[k][d].w};
-#pragma unroll
-                    for (int dy = 0; dy <= 2 * R; ++dy)
-#pragma unroll
-                        for (int dx = 0; dx <= 2 * R; ++dx) {
-                            const float wv = bw.w[d][dy][dx];
-#pragma unroll
-                            for (int m = 0; m < 4; ++m) a[m] = fmaf(wv, v[k + dy][m + dx], a[m]);
+                            for (int m = 0; m < 4; ++m) a[m] = bw.w[0][0][0] * v[k][m];
+                        } else {
+                            a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
                         }
-                    T[k][d] = make_float4(a[0], a[1], a[2], a[3]);
-                }
-            }
-            if (i >= 2 * R) {
 #pragma unroll
-                for (int k = 0; k < K; ++k)
-                    if (row_ok[k]) store_f4(op + (size_t)k * g.nx, T[k][2 * R], streaming);
-                op += plane_stride;
+                        for (int dy = 0; dy < M; ++dy)
+#pragma unroll
+                            for (int dx = 0; dx < M; ++dx) {
+                                if (d == 0 && dy == 0 && dx == 0) continue;
+                                const float wv = bw.w[d][dy][dx];
+#pragma unroll
+                                for (int m = 0; m < 4; ++m) a[m] = fmaf(wv, v[k + dy][m + dx], a[m]);
+                            }
+                        t = make_float4(a[0], a[1], a[2], a[3]);
+                    }
+                }
+                if (i >= 2 * R) {
+#pragma unroll
+                    for (int k = 0; k < K; ++k)           // tap dz = +R was the last one of plane i-R
+                        if (row_ok[k]) store_f4(op + (size_t)k * g.nx, T[k][(u + R + 1) % M], streaming);
+                    op += plane_stride;
+                }
+                return true;
+            });
+            if (!ok) {
+                atomicExch(status, kStatusTimeout);
+                return;
             }
         }
     }

@@ -29,24 +29,40 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
+// Arrival by the lanes where `take` holds, as a predicated instruction (no branch).
+__device__ __forceinline__ void mbar_arrive_if(bool take, uint32_t bar) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "@q mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}"
+        ::"r"(bar), "r"((uint32_t)take)
+        : "memory");
+}
+
+// One poll; the thread may sleep inside it for up to kWaitHintNs nanoseconds
+// (a hint to the hardware), which keeps waiting warps out of the issue slots.
+constexpr uint32_t kWaitHintNs = 20000;
+
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.b32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kWaitHintNs)
         : "memory");
     return ok != 0;
 }
 
-// Every wait in the library is bounded: after kWaitPolls unsuccessful polls the
-// caller records a timeout in the plan's status word and leaves the kernel.
-constexpr uint32_t kWaitPolls = 1u << 22;
+// Every wait in the library is bounded: after kWaitPolls unsuccessful polls
+// (each at most kWaitHintNs long, so some seconds in total at worst) the caller
+// records a timeout in the plan's status word and leaves the kernel.
+constexpr uint32_t kWaitPolls = 1u << 20;
 
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    for (uint32_t it = 0; it < kWaitPolls; ++it)
+    if (mbar_try_wait(bar, parity)) return true;          // the usual case: already complete
+    for (uint32_t it = 1; it < kWaitPolls; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

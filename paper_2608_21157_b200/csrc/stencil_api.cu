@@ -60,6 +60,9 @@ struct StreamConfig {
     int K, NW;            // rows per thread, consumer warps
     int tile_y;           // K * NW
     int plane_bytes, box_rows, threads;
+    mutable int occupancy[kMaxStages + 1];   // resident CTAs per SM by ring depth; 0 = not asked yet
+    mutable size_t smem_allowed;             // dynamic shared memory the kernel is currently allowed
+    mutable int cache_device;                // device the two caches above were filled on
     const void* kernel;
     cudaError_t (*launch)(const struct stencil_plan_s*, const StreamConfig&, const CUtensorMap&,
                           float*, const StreamGeom&, int grid, size_t smem, cudaStream_t);
@@ -97,6 +100,8 @@ struct stencil_plan_s {
     int variant;                   // resolved STENCIL_VARIANT_*
     int tile_y, rows_per_thread, chunk_z, stages, fuse_steps, streaming_store;
     const StreamConfig* stream_cfg;
+    bool stream_cfg_fixed;         // the caller chose the tile shape
+    bool stream_cfg_tuned;         // the library has chosen it for this grid
     const FusedConfig* fused_cfg;  // non-null: iterated applies run fused passes
     int tile_x;                    // requested region width for fused passes (0 = auto)
     // bookkeeping
@@ -151,6 +156,9 @@ StreamConfig make_cfg() {
     StreamConfig c;
     c.radius = R; c.box = BOX; c.K = K; c.NW = NW; c.tile_y = S::TY;
     c.plane_bytes = S::PLANE_BYTES; c.box_rows = S::ROWS; c.threads = S::THREADS;
+    for (int& o : c.occupancy) o = 0;
+    c.smem_allowed = 0;
+    c.cache_device = -1;
     c.kernel = reinterpret_cast<const void*>(&stencil_stream_kernel<R, BOX, K, NW, MINB>);
     c.launch = &launch_stream_t<R, BOX, K, NW, MINB>;
     return c;
@@ -159,12 +167,17 @@ StreamConfig make_cfg() {
 // First entry of a (radius, box) group is the default; the others are reachable
 // through STENCIL_KEY_TILE_Y / STENCIL_KEY_ROWS_PER_THREAD.
 const std::vector<StreamConfig>& stream_configs() {
+    // tile heights 14 and 28 (7 consumer warps + the producer = 256 threads) exist
+    // because 4 x 37 tiles of 128 x 14 cover a 512 x 512 plane with one tile per SM
     static const std::vector<StreamConfig> v = {
-        make_cfg<1, false, 2, 8, 1>(),  make_cfg<1, false, 4, 8, 1>(),  make_cfg<1, false, 1, 8, 1>(),
-        make_cfg<2, false, 2, 8, 1>(),  make_cfg<2, false, 4, 8, 1>(),
-        make_cfg<3, false, 2, 8, 1>(),  make_cfg<3, false, 4, 8, 1>(),
-        make_cfg<4, false, 2, 8, 1>(),  make_cfg<4, false, 4, 8, 1>(),  make_cfg<4, false, 2, 16, 1>(),
-        make_cfg<1, true, 2, 8, 1>(),   make_cfg<1, true, 4, 8, 1>(),   make_cfg<1, true, 1, 8, 1>(),
+        make_cfg<1, false, 2, 8, 1>(),  make_cfg<1, false, 2, 7, 4>(),  make_cfg<1, false, 4, 8, 1>(),
+        make_cfg<1, false, 4, 7, 1>(),  make_cfg<1, false, 1, 8, 1>(),
+        make_cfg<2, false, 2, 8, 1>(),  make_cfg<2, false, 2, 7, 1>(),  make_cfg<2, false, 4, 8, 1>(),
+        make_cfg<3, false, 2, 8, 1>(),  make_cfg<3, false, 2, 7, 2>(),  make_cfg<3, false, 4, 8, 1>(),
+        make_cfg<4, false, 2, 8, 1>(),  make_cfg<4, false, 2, 7, 2>(),  make_cfg<4, false, 4, 8, 1>(),
+        make_cfg<4, false, 2, 16, 1>(),
+        make_cfg<1, true, 2, 8, 1>(),   make_cfg<1, true, 2, 7, 4>(),   make_cfg<1, true, 4, 8, 1>(),
+        make_cfg<1, true, 4, 7, 1>(),   make_cfg<1, true, 1, 8, 1>(),
     };
     return v;
 }
@@ -334,7 +347,106 @@ int get_tensor_map(stencil_plan_s* p, const void* cfg, int box_x, int box_y, con
     return STENCIL_OK;
 }
 
+int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n = v;
+        else { cudaGetLastError(); n = 148; }
+    }
+    return n;
+}
+
+size_t stream_smem_bytes(const StreamConfig* cfg, int stages) {
+    return (size_t)stages * cfg->plane_bytes + 128 + 2 * kMaxStages * sizeof(uint64_t);
+}
+
+// Resident CTAs per SM of a configuration at a given ring depth (asked once).
+int stream_occupancy(const StreamConfig* cfg, int stages) {
+    const size_t smem = stream_smem_bytes(cfg, stages);
+    if (smem > 227 * 1024) return -1;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return -1; }
+    if (dev != cfg->cache_device) {                // function attributes are per device
+        for (int& o : cfg->occupancy) o = 0;
+        cfg->smem_allowed = 0;
+        cfg->cache_device = dev;
+    }
+    if (smem > cfg->smem_allowed) {                // the limit only ever grows
+        if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+            cudaGetLastError();
+            return -1;
+        }
+        cfg->smem_allowed = smem;
+    }
+    if (cfg->occupancy[stages] != 0) return cfg->occupancy[stages];
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, cfg->kernel, cfg->threads, smem) != cudaSuccess) {
+        cudaGetLastError();
+        occ = 0;
+    }
+    cfg->occupancy[stages] = occ > 0 ? occ : -1;
+    return cfg->occupancy[stages];
+}
+
+// The sweeps with few FMAs per point are bound by HBM: there many short CTAs work
+// best (the hardware scheduler balances them, and CTAs that outlive the others
+// simply get more bandwidth).  The others are bound by instruction issue: there
+// every SM must get the same amount of work, so the grid is cut into whole waves.
+bool issue_bound(const stencil_plan_s* p) {
+    return p->shape == STENCIL_STAR && p->radius >= 3;
+}
+
+// Planes of output per CTA, and the relative cost of the launch, for one configuration.
+int choose_chunk(const stencil_plan_s* p, const StreamConfig* cfg, int stages, double* cost_out) {
+    const int R = p->radius;
+    const int tiles = ((p->nx + kStreamTX - 1) / kStreamTX) * ((p->ny + cfg->tile_y - 1) / cfg->tile_y);
+    const int occ = std::max(1, stream_occupancy(cfg, stages));
+    const int slots = occ * sm_count();
+    if (!issue_bound(p)) {
+        // measured on 512^3: 32-plane chunks (several thousand short CTAs) beat every longer chunk
+        const int chunk = p->nz >= 64 ? 32 : p->nz;
+        if (cost_out) {
+            const int64_t ctas = (int64_t)tiles * ((p->nz + chunk - 1) / chunk);
+            *cost_out = ((double)ctas / slots + 0.5) * occ * (chunk + 2 * R) * cfg->tile_y;
+        }
+        return chunk;
+    }
+    const double fill = 4.0;                       // pipeline start-up, in planes
+    int best_chunk = p->nz;
+    double best = 1e300;
+    const int max_chunks = std::max(1, p->nz / std::max(8 * R, 16));
+    for (int nch = 1; nch <= max_chunks; ++nch) {
+        const int chunk = (p->nz + nch - 1) / nch;
+        const int real_nch = (p->nz + chunk - 1) / chunk;
+        const int64_t ctas = (int64_t)tiles * real_nch;
+        const double waves = (double)((ctas + slots - 1) / slots);
+        // CTAs resident together share the SM, so a wave of `occ` CTAs per SM costs occ units
+        const double cost = waves * occ * (chunk + 2 * R + fill) * cfg->tile_y;
+        if (cost < best * 0.999) { best = cost; best_chunk = chunk; }
+    }
+    if (cost_out) *cost_out = best;
+    return best_chunk;
+}
+
 int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
+    const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 4;
+    if (!p->stream_cfg_fixed && !p->stream_cfg_tuned) {
+        // pick the tile height that balances this grid best (same rows per thread)
+        const StreamConfig* best_cfg = p->stream_cfg;
+        double best = 1e300;
+        for (const StreamConfig& c : stream_configs()) {
+            if (c.radius != p->radius || c.box != (p->shape == STENCIL_BOX) || c.K != p->stream_cfg->K) continue;
+            if (stream_occupancy(&c, stages) <= 0) continue;
+            double cost = 0;
+            choose_chunk(p, &c, stages, &cost);
+            if (cost < best * 0.98) { best = cost; best_cfg = &c; }
+        }
+        p->stream_cfg = best_cfg;
+        p->stream_cfg_tuned = true;
+    }
     const StreamConfig* cfg = p->stream_cfg;
     const CUtensorMap* map = nullptr;
     int rc = get_tensor_map(p, cfg, kStreamPX, cfg->box_rows, src, &map);
@@ -344,28 +456,17 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     g.nz = p->nz; g.ny = p->ny; g.nx = p->nx;
     g.tiles_x = (p->nx + kStreamTX - 1) / kStreamTX;
     g.tiles_y = (p->ny + cfg->tile_y - 1) / cfg->tile_y;
-    g.stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 4;
+    g.stages = stages;
     g.streaming_store = p->streaming_store;
     const int tiles = g.tiles_x * g.tiles_y;
-    int chunk = p->chunk_z;
-    if (chunk <= 0) {
-        // enough CTAs for several waves of the 148 SMs, but chunks long enough
-        // that the 2R halo planes per chunk stay a small fraction
-        const int want_ctas = 148 * 8;
-        int nchunks = std::max(1, std::min((want_ctas + tiles - 1) / tiles, p->nz / std::max(16 * p->radius, 32)));
-        chunk = (p->nz + nchunks - 1) / nchunks;
-    }
+    if (stream_occupancy(cfg, stages) <= 0) return STENCIL_ERR_UNSUPPORTED;
+    int chunk = p->chunk_z > 0 ? p->chunk_z : choose_chunk(p, cfg, stages, nullptr);
     chunk = std::max(1, std::min(chunk, p->nz));
     g.chunk_z = chunk;
     const int nchunks = (p->nz + chunk - 1) / chunk;
     const int64_t grid64 = (int64_t)tiles * nchunks;
     if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
-    const size_t smem = (size_t)g.stages * cfg->plane_bytes + 128 + 2 * kMaxStages * sizeof(uint64_t);
-    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
-        cudaGetLastError();
-        return STENCIL_ERR_CUDA;
-    }
+    const size_t smem = stream_smem_bytes(cfg, stages);
     if (cfg->launch(p, *cfg, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
     p->launches++;
     return STENCIL_OK;
@@ -504,6 +605,7 @@ int stencil_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int ra
     p->variant = STENCIL_VARIANT_GENERIC;
     p->tile_y = 0; p->rows_per_thread = 0; p->chunk_z = 0; p->stages = 0; p->fuse_steps = 0; p->streaming_store = 0;
     p->stream_cfg = nullptr; p->fused_cfg = nullptr; p->tile_x = 0;
+    p->stream_cfg_fixed = false; p->stream_cfg_tuned = false;
     p->launches = 0; p->last_stream = nullptr; p->used = false;
 
     const int side = 2 * radius + 1;
@@ -743,6 +845,8 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
             }
             p->tile_y = ty;
             p->rows_per_thread = k;
+            p->stream_cfg_fixed = ty != 0;
+            p->stream_cfg_tuned = false;
             return STENCIL_OK;
         }
         case STENCIL_KEY_CHUNK_Z:

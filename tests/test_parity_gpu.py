@@ -91,13 +91,15 @@ def test_generic_iteration_and_ping_pong(steps, boundary):
 
 # ------------------------------------------------------------------- stream --
 def _stream_knob_sets(R, box):
-    if box:
-        return [dict(), dict(rows_per_thread=4), dict(rows_per_thread=1)]
-    if R == 1:
-        return [dict(), dict(rows_per_thread=4), dict(rows_per_thread=1)]
+    """Every compiled tile shape of the operator (tile_y = rows per thread x consumer warps)."""
+    if box or R == 1:
+        return [dict(), dict(tile_y=16), dict(tile_y=14), dict(tile_y=32), dict(tile_y=28), dict(tile_y=8)]
     if R == 4:
-        return [dict(), dict(rows_per_thread=4), dict(tile_y=32, rows_per_thread=2)]
-    return [dict(), dict(rows_per_thread=4)]
+        return [dict(), dict(tile_y=16), dict(tile_y=14), dict(tile_y=32, rows_per_thread=4),
+                dict(tile_y=32, rows_per_thread=2)]
+    if R == 3:
+        return [dict(), dict(tile_y=16), dict(tile_y=14), dict(tile_y=32)]
+    return [dict(), dict(tile_y=16), dict(tile_y=14), dict(tile_y=32)]
 
 
 STREAM_OPS = [(1, False), (2, False), (3, False), (4, False), (1, True)]
