@@ -234,47 +234,59 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                 if (!mbar_wait_bounded(full0 + 8 * s, ph)) return false;
                 const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
                 const float* colp = pl + row0 * PX + 4 + 4 * lane;
-                float4 c[K + 2 * R];
+                // Rows are visited once, top to bottom.  A row is a y-neighbour of up to 2R
+                // output rows and the centre row of at most one; it is consumed at once, so
+                // only one loaded row is live at a time (the register budget goes to the z
+                // queues instead).
+                float acc[K][4];
 #pragma unroll
-                for (int kk = 0; kk < K + 2 * R; ++kk)
-                    c[kk] = *reinterpret_cast<const float4*>(colp + kk * PX);
-
+                for (int k = 0; k < K; ++k)
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) acc[k][m] = 0.0f;
+#pragma unroll
+                for (int kk = 0; kk < K + 2 * R; ++kk) {
+                    const float4 c = *reinterpret_cast<const float4*>(colp + kk * PX);
+#pragma unroll
+                    for (int k = 0; k < K; ++k) {
+                        const int d = kk - k - R;          // row kk is tap dy = d of output row k
+                        if (d != 0 && d >= -R && d <= R) {
+#pragma unroll
+                            for (int m = 0; m < 4; ++m) acc[k][m] = fmaf(sw.y[d + R], f4get(c, m), acc[k][m]);
+                        }
+                    }
+                    if (kk >= R && kk < K + R) {
+                        const int k = kk - R;              // centre row of output row k
+                        float v[4 + 2 * R];
+                        gather_row<R>(colp + kk * PX, pl + (row0 + kk) * PX, lane, c, v);
+#pragma unroll
+                        for (int m = 0; m < 4; ++m) {
+                            float a = fmaf(sw.c, v[R + m], acc[k][m]);
+#pragma unroll
+                            for (int d = 1; d <= R; ++d) {
+                                a = fmaf(sw.x[R - d], v[R + m - d], a);
+                                a = fmaf(sw.x[R + d], v[R + m + d], a);
+                            }
+#pragma unroll
+                            for (int j = 1; j <= R; ++j)  // taps at dz = -j: plane i-j
+                                a = fmaf(sw.z[R - j], f4get(q[k][(u - j + R) % R], m), a);
+                            acc[k][m] = a;
+                        }
+#pragma unroll
+                        for (int j = 1; j <= R; ++j) {    // this plane is dz = +j of output i-j
+                            float4& p = pend[k][(u - j + R) % R];
+                            p.x = fmaf(sw.z[R + j], c.x, p.x);
+                            p.y = fmaf(sw.z[R + j], c.y, p.y);
+                            p.z = fmaf(sw.z[R + j], c.z, p.z);
+                            p.w = fmaf(sw.z[R + j], c.w, p.w);
+                        }
+                        q[k][u] = c;
+                    }
+                }
                 float4 done[K];
 #pragma unroll
                 for (int k = 0; k < K; ++k) {
-                    const float4 ctr = c[k + R];
-                    float v[4 + 2 * R];
-                    gather_row<R>(colp + (k + R) * PX, pl + (row0 + k + R) * PX, lane, ctr, v);
-                    float acc[4];
-#pragma unroll
-                    for (int m = 0; m < 4; ++m) {
-                        float a = sw.c * v[R + m];
-#pragma unroll
-                        for (int d = 1; d <= R; ++d) {
-                            a = fmaf(sw.x[R - d], v[R + m - d], a);
-                            a = fmaf(sw.x[R + d], v[R + m + d], a);
-                        }
-#pragma unroll
-                        for (int d = 1; d <= R; ++d) {
-                            a = fmaf(sw.y[R - d], f4get(c[k + R - d], m), a);
-                            a = fmaf(sw.y[R + d], f4get(c[k + R + d], m), a);
-                        }
-#pragma unroll
-                        for (int j = 1; j <= R; ++j)      // taps at dz = -j: plane i-j
-                            a = fmaf(sw.z[R - j], f4get(q[k][(u - j + R) % R], m), a);
-                        acc[m] = a;
-                    }
-#pragma unroll
-                    for (int j = 1; j <= R; ++j) {        // this plane is dz = +j of output i-j
-                        float4& p = pend[k][(u - j + R) % R];
-                        p.x = fmaf(sw.z[R + j], ctr.x, p.x);
-                        p.y = fmaf(sw.z[R + j], ctr.y, p.y);
-                        p.z = fmaf(sw.z[R + j], ctr.z, p.z);
-                        p.w = fmaf(sw.z[R + j], ctr.w, p.w);
-                    }
                     done[k] = pend[k][u];                 // output plane i-R is complete
-                    pend[k][u] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-                    q[k][u] = ctr;
+                    pend[k][u] = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
                 }
                 __syncwarp();
                 mbar_arrive_if(lane == 0, empty0 + 8 * s);

@@ -174,7 +174,7 @@ const std::vector<StreamConfig>& stream_configs() {
         make_cfg<1, false, 4, 7, 1>(),  make_cfg<1, false, 1, 8, 1>(),
         make_cfg<2, false, 2, 8, 1>(),  make_cfg<2, false, 2, 7, 1>(),  make_cfg<2, false, 4, 8, 1>(),
         make_cfg<3, false, 2, 8, 1>(),  make_cfg<3, false, 2, 7, 2>(),  make_cfg<3, false, 4, 8, 1>(),
-        make_cfg<4, false, 2, 8, 1>(),  make_cfg<4, false, 2, 7, 2>(),  make_cfg<4, false, 4, 8, 1>(),
+        make_cfg<4, false, 2, 8, 2>(),  make_cfg<4, false, 2, 7, 2>(),  make_cfg<4, false, 4, 8, 1>(),
         make_cfg<4, false, 2, 16, 1>(),
         make_cfg<1, true, 2, 8, 1>(),   make_cfg<1, true, 2, 7, 4>(),   make_cfg<1, true, 4, 8, 1>(),
         make_cfg<1, true, 4, 7, 1>(),   make_cfg<1, true, 1, 8, 1>(),
