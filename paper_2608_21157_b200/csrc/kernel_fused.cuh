@@ -108,15 +108,20 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
     const int xg = x0e + col;
     const bool x_in = xg >= 0 && xg < g.nx;
     const bool x_store = x_in && col >= g.halo_x && col < g.halo_x + g.tile_x;
-    bool cell_in[K], row_store[K];
+    // per-row flags packed into bit masks; the common case (every row inside the grid,
+    // every row stored) is tested once per plane instead of once per row
+    uint32_t in_mask = 0, store_mask = 0;
 #pragma unroll
     for (int k = 0; k < K; ++k) {
         const int yg = y0e + row0 + k;
         const bool y_in = yg >= 0 && yg < g.ny;
-        cell_in[k] = y_in && x_in;
-        row_store[k] = y_in && x_store && (row0 + k) >= g.halo_y && (row0 + k) < g.halo_y + g.tile_y;
+        if (y_in && x_in) in_mask |= 1u << k;
+        if (y_in && x_store && (row0 + k) >= g.halo_y && (row0 + k) < g.halo_y + g.tile_y) store_mask |= 1u << k;
     }
+    constexpr uint32_t kAllRows = (1u << K) - 1u;
     const size_t plane_stride = (size_t)g.ny * g.nx;
+    float* const out_col = out + (size_t)(y0e + row0) * g.nx + xg;     // this thread's column of rows
+    const int toff = row0 * TXE + col;                                  // its offset inside a plane
 
     int issued = 0;                                // planes requested so far (thread 0 only)
     if (tid == 0) {
@@ -130,25 +135,27 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
         }
     }
 
-    float4 q[T][K][R], pend[T][K][R];
+    // A[l][k][j]: level l+1's partial sums, oldest incomplete output plane first (see the
+    // single-step kernel: arriving planes update them in place, nothing is copied)
+    float4 A[T][K][2 * R];
 #pragma unroll
     for (int l = 0; l < T; ++l)
 #pragma unroll
         for (int k = 0; k < K; ++k)
 #pragma unroll
-            for (int j = 0; j < R; ++j) {
-                q[l][k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                pend[l][k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
+            for (int j = 0; j < 2 * R; ++j) A[l][k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
 
     bool dead = false;
-    for (int i0 = 0; i0 < nsteps; i0 += R) {
-#pragma unroll
-        for (int u = 0; u < R; ++u) {
-            const int i = i0 + u;
-            if (i >= nsteps) break;
-            const int s = i % nstage;
-            if (!dead && !mbar_wait_bounded(full0 + 8 * s, (i / nstage) & 1)) {
+    int s = 0;                                     // input ring slot and its phase parity
+    uint32_t ph = 0;
+    // two planes per trip, so that the parity of the level buffers is a compile-time
+    // constant in each copy of the body
+    for (int i0 = 0; i0 < nsteps; i0 += 2) {
+        static_for<2>([&](auto uc) -> bool {
+            constexpr int par = decltype(uc)::value & 1;
+            const int i = i0 + decltype(uc)::value;
+            if (i >= nsteps) return true;
+            if (!dead && !mbar_wait_bounded(full0 + 8 * s, ph)) {
                 dead = true;
                 atomicExch(status, kStatusTimeout);
             }
@@ -156,87 +163,103 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
             float4 cin[K + 2 * R];
 #pragma unroll
             for (int kk = 0; kk < K + 2 * R; ++kk)
-                cin[kk] = *reinterpret_cast<const float4*>(src + (row0 + kk - R) * TXE + col);
+                cin[kk] = *reinterpret_cast<const float4*>(src + toff + (kk - R) * TXE);
 
 #pragma unroll
             for (int l = 1; l <= T; ++l) {
                 if (l <= nlev) {
                     const int zl = pstart + i - l * R;          // plane this level completes now
-                    const bool z_in = zl >= 0 && zl < g.nz;
                     float4 e[K];
+                    {
 #pragma unroll
-                    for (int k = 0; k < K; ++k) {
-                        const float4 ctr = cin[k + R];
-                        float v[4 + 2 * R];
-                        v[R + 0] = ctr.x; v[R + 1] = ctr.y; v[R + 2] = ctr.z; v[R + 3] = ctr.w;
-                        {
-                            const float c4[4] = {ctr.x, ctr.y, ctr.z, ctr.w};
-                            const float* rowp = src + (row0 + k) * TXE + col;
+                        for (int k = 0; k < K; ++k) {
+                            const float4 ctr = cin[k + R];
+                            float v[4 + 2 * R];
+                            v[R + 0] = ctr.x; v[R + 1] = ctr.y; v[R + 2] = ctr.z; v[R + 3] = ctr.w;
+                            {
+                                const float c4[4] = {ctr.x, ctr.y, ctr.z, ctr.w};
+                                const float* rowb = src + (row0 + k) * TXE;   // first cell of the region row
 #pragma unroll
-                            for (int t = 0; t < R; ++t) {
-                                float lft = __shfl_up_sync(0xffffffffu, c4[4 - R + t], 1);
-                                float rgt = __shfl_down_sync(0xffffffffu, c4[t], 1);
-                                // warp-edge lanes: the neighbour warp's value from the plane in
-                                // shared memory, or zero at the edge of the region
-                                if (lane == 0) lft = 0.0f;
-                                if (lane == 31) rgt = 0.0f;
-                                if (XW > 1) {
-                                    lft = lds_if(lane == 0 && wx > 0, rowp + t - R, lft);
-                                    rgt = lds_if(lane == 31 && wx < XW - 1, rowp + 4 + t, rgt);
+                                for (int t = 0; t < R; ++t) {
+                                    // cells across the warp boundary: one broadcast read per side from the
+                                    // level's plane (wx is warp-uniform); zero at the region's edge
+                                    float xl = 0.0f, xr = 0.0f;
+                                    if (XW > 1) {
+                                        if (wx > 0) xl = rowb[wx * 128 - R + t];
+                                        if (wx < XW - 1) xr = rowb[(wx + 1) * 128 + t];
+                                    }
+                                    const float lft = __shfl_up_sync(0xffffffffu, c4[4 - R + t], 1);
+                                    const float rgt = __shfl_down_sync(0xffffffffu, c4[t], 1);
+                                    v[t] = lane == 0 ? xl : lft;
+                                    v[R + 4 + t] = lane == 31 ? xr : rgt;
                                 }
-                                v[t] = lft;
-                                v[R + 4 + t] = rgt;
                             }
-                        }
-                        float acc[4];
+                            float4 (&Al)[2 * R] = A[l - 1][k];
+                            // the output whose centre plane this is continues from Al[R]
+                            float acc[4] = {Al[R].x, Al[R].y, Al[R].z, Al[R].w};
 #pragma unroll
-                        for (int m = 0; m < 4; ++m) {
-                            float a = sw.c * v[R + m];
+                            for (int m = 0; m < 4; ++m) {
+                                float a = fmaf(sw.c, v[R + m], acc[m]);
 #pragma unroll
-                            for (int d = 1; d <= R; ++d) {
-                                a = fmaf(sw.x[R - d], v[R + m - d], a);
-                                a = fmaf(sw.x[R + d], v[R + m + d], a);
+                                for (int d = 1; d <= R; ++d) {
+                                    a = fmaf(sw.x[R - d], v[R + m - d], a);
+                                    a = fmaf(sw.x[R + d], v[R + m + d], a);
+                                }
+#pragma unroll
+                                for (int d = 1; d <= R; ++d) {
+                                    a = fmaf(sw.y[R - d], f4get(cin[k + R - d], m), a);
+                                    a = fmaf(sw.y[R + d], f4get(cin[k + R + d], m), a);
+                                }
+                                acc[m] = a;
                             }
+                            // z taps: oldest output complete; the others slide down inside their FMA
+                            e[k].x = fmaf(sw.z[2 * R], ctr.x, Al[0].x);
+                            e[k].y = fmaf(sw.z[2 * R], ctr.y, Al[0].y);
+                            e[k].z = fmaf(sw.z[2 * R], ctr.z, Al[0].z);
+                            e[k].w = fmaf(sw.z[2 * R], ctr.w, Al[0].w);
 #pragma unroll
-                            for (int d = 1; d <= R; ++d) {
-                                a = fmaf(sw.y[R - d], f4get(cin[k + R - d], m), a);
-                                a = fmaf(sw.y[R + d], f4get(cin[k + R + d], m), a);
+                            for (int j = 0; j < 2 * R - 1; ++j) {
+                                if (j == R - 1) continue;
+                                const float wz = sw.z[2 * R - 1 - j];
+                                Al[j].x = fmaf(wz, ctr.x, Al[j + 1].x);
+                                Al[j].y = fmaf(wz, ctr.y, Al[j + 1].y);
+                                Al[j].z = fmaf(wz, ctr.z, Al[j + 1].z);
+                                Al[j].w = fmaf(wz, ctr.w, Al[j + 1].w);
                             }
-#pragma unroll
-                            for (int j = 1; j <= R; ++j)
-                                a = fmaf(sw.z[R - j], f4get(q[l - 1][k][(u - j + R) % R], m), a);
-                            acc[m] = a;
+                            Al[2 * R - 1] = make_float4(sw.z[0] * ctr.x, sw.z[0] * ctr.y, sw.z[0] * ctr.z,
+                                                        sw.z[0] * ctr.w);
+                            Al[R - 1] = make_float4(acc[0], acc[1], acc[2], acc[3]);
                         }
-#pragma unroll
-                        for (int j = 1; j <= R; ++j) {
-                            float4& p = pend[l - 1][k][(u - j + R) % R];
-                            p.x = fmaf(sw.z[R + j], ctr.x, p.x);
-                            p.y = fmaf(sw.z[R + j], ctr.y, p.y);
-                            p.z = fmaf(sw.z[R + j], ctr.z, p.z);
-                            p.w = fmaf(sw.z[R + j], ctr.w, p.w);
-                        }
-                        float4 done = pend[l - 1][k][u];
-                        pend[l - 1][k][u] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-                        q[l - 1][k][u] = ctr;
-                        // the zero boundary holds at every time level
-                        if (!(cell_in[k] && z_in)) done = make_float4(0.f, 0.f, 0.f, 0.f);
-                        e[k] = done;
-                    }
-
-                    if (l == nlev) {
-                        // last level of this pass: interior of the tile goes to global memory
-                        const int zo = zl;
-                        if (!dead && zo >= z0 && zo < z1) {
-                            float* op = out + (size_t)zo * plane_stride + (size_t)(y0e + row0) * g.nx + xg;
+                        // the zero boundary holds at every time level: cells outside the grid go
+                        // back to zero (nothing to do for regions and planes inside the grid)
+                        if (in_mask != kAllRows || zl < 0 || zl >= g.nz) {
+                            const bool z_in = zl >= 0 && zl < g.nz;
 #pragma unroll
                             for (int k = 0; k < K; ++k)
-                                if (row_store[k]) *reinterpret_cast<float4*>(op + (size_t)k * g.nx) = e[k];
+                                if (!(z_in && ((in_mask >> k) & 1u))) e[k] = make_float4(0.f, 0.f, 0.f, 0.f);
                         }
-                    } else {
-                        float* buf = lvl + (size_t)(2 * (l - 1) + (i & 1)) * S::SLOT_FLOATS + R * TXE;
+
+                        if (l == nlev) {
+                            // last level of this pass: interior of the tile goes to global memory
+                            if (!dead && zl >= z0 && zl < z1) {
+                                float* op = out_col + (size_t)zl * plane_stride;
+                                if (store_mask == kAllRows) {
 #pragma unroll
-                        for (int k = 0; k < K; ++k)
-                            *reinterpret_cast<float4*>(buf + (row0 + k) * TXE + col) = e[k];
+                                    for (int k = 0; k < K; ++k)
+                                        *reinterpret_cast<float4*>(op + (size_t)k * g.nx) = e[k];
+                                } else {
+#pragma unroll
+                                    for (int k = 0; k < K; ++k)
+                                        if ((store_mask >> k) & 1u)
+                                            *reinterpret_cast<float4*>(op + (size_t)k * g.nx) = e[k];
+                                }
+                            }
+                        } else {
+                            float* buf = lvl + (size_t)(2 * (l - 1) + par) * S::SLOT_FLOATS + R * TXE;
+#pragma unroll
+                            for (int k = 0; k < K; ++k)
+                                *reinterpret_cast<float4*>(buf + toff + k * TXE) = e[k];
+                        }
                     }
                     if (l < nlev || l == 1) {
                         // everyone has finished with level l-1's plane and has published level l
@@ -250,19 +273,21 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                         }
                     }
                     if (l < nlev) {
-                        const float* buf = lvl + (size_t)(2 * (l - 1) + (i & 1)) * S::SLOT_FLOATS + R * TXE;
+                        const float* buf = lvl + (size_t)(2 * (l - 1) + par) * S::SLOT_FLOATS + R * TXE;
                         src = buf;
 #pragma unroll
                         for (int k = 0; k < K; ++k) cin[k + R] = e[k];
 #pragma unroll
                         for (int kk = 0; kk < R; ++kk) {
-                            cin[kk] = *reinterpret_cast<const float4*>(buf + (row0 - R + kk) * TXE + col);
-                            cin[K + R + kk] = *reinterpret_cast<const float4*>(buf + (row0 + K + kk) * TXE + col);
+                            cin[kk] = *reinterpret_cast<const float4*>(buf + toff + (kk - R) * TXE);
+                            cin[K + R + kk] = *reinterpret_cast<const float4*>(buf + toff + (K + kk) * TXE);
                         }
                     }
                 }
             }
-        }
+            if (++s == nstage) { s = 0; ph ^= 1; }
+            return true;
+        });
     }
     if (dead && tid == 0) {
         // let copies that may still be in flight land before shared memory is released

@@ -215,94 +215,88 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
     uint32_t ph = 0;
 
     if constexpr (!BOX) {
-        float4 q[K][R], pend[K][R];
+        // A[k][j]: partial sum of the output 1+j planes above the oldest incomplete one.
+        // An arriving plane adds its tap to each of the 2R+1 outputs it reaches: the oldest
+        // is then complete, the others move down one slot as part of the FMA that updates
+        // them (no register copies), and a new one starts at the top.
+        float4 A[K][2 * R];
 #pragma unroll
         for (int k = 0; k < K; ++k)
 #pragma unroll
-            for (int j = 0; j < R; ++j) {
-                q[k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                pend[k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
+            for (int j = 0; j < 2 * R; ++j) A[k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
 
-        // R planes per trip; the slot of the register queues that a plane uses is a
-        // compile-time constant inside each of the R copies of the body
-        for (int i0 = 0; i0 < nplanes; i0 += R) {
-            const bool ok = static_for<R>([&](auto uc) -> bool {
-                constexpr int u = decltype(uc)::value;
-                const int i = i0 + u;
-                if (i >= nplanes) return true;
-                if (!mbar_wait_bounded(full0 + 8 * s, ph)) return false;
-                const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
-                const float* colp = pl + row0 * PX + 4 + 4 * lane;
-                // Rows are visited once, top to bottom.  A row is a y-neighbour of up to 2R
-                // output rows and the centre row of at most one; it is consumed at once, so
-                // only one loaded row is live at a time (the register budget goes to the z
-                // queues instead).
-                float acc[K][4];
-#pragma unroll
-                for (int k = 0; k < K; ++k)
-#pragma unroll
-                    for (int m = 0; m < 4; ++m) acc[k][m] = 0.0f;
-#pragma unroll
-                for (int kk = 0; kk < K + 2 * R; ++kk) {
-                    const float4 c = *reinterpret_cast<const float4*>(colp + kk * PX);
-#pragma unroll
-                    for (int k = 0; k < K; ++k) {
-                        const int d = kk - k - R;          // row kk is tap dy = d of output row k
-                        if (d != 0 && d >= -R && d <= R) {
-#pragma unroll
-                            for (int m = 0; m < 4; ++m) acc[k][m] = fmaf(sw.y[d + R], f4get(c, m), acc[k][m]);
-                        }
-                    }
-                    if (kk >= R && kk < K + R) {
-                        const int k = kk - R;              // centre row of output row k
-                        float v[4 + 2 * R];
-                        gather_row<R>(colp + kk * PX, pl + (row0 + kk) * PX, lane, c, v);
-#pragma unroll
-                        for (int m = 0; m < 4; ++m) {
-                            float a = fmaf(sw.c, v[R + m], acc[k][m]);
-#pragma unroll
-                            for (int d = 1; d <= R; ++d) {
-                                a = fmaf(sw.x[R - d], v[R + m - d], a);
-                                a = fmaf(sw.x[R + d], v[R + m + d], a);
-                            }
-#pragma unroll
-                            for (int j = 1; j <= R; ++j)  // taps at dz = -j: plane i-j
-                                a = fmaf(sw.z[R - j], f4get(q[k][(u - j + R) % R], m), a);
-                            acc[k][m] = a;
-                        }
-#pragma unroll
-                        for (int j = 1; j <= R; ++j) {    // this plane is dz = +j of output i-j
-                            float4& p = pend[k][(u - j + R) % R];
-                            p.x = fmaf(sw.z[R + j], c.x, p.x);
-                            p.y = fmaf(sw.z[R + j], c.y, p.y);
-                            p.z = fmaf(sw.z[R + j], c.z, p.z);
-                            p.w = fmaf(sw.z[R + j], c.w, p.w);
-                        }
-                        q[k][u] = c;
-                    }
-                }
-                float4 done[K];
-#pragma unroll
-                for (int k = 0; k < K; ++k) {
-                    done[k] = pend[k][u];                 // output plane i-R is complete
-                    pend[k][u] = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
-                }
-                __syncwarp();
-                mbar_arrive_if(lane == 0, empty0 + 8 * s);
-                if (++s == nstage) { s = 0; ph ^= 1; }
-
-                if (i >= 2 * R) {
-#pragma unroll
-                    for (int k = 0; k < K; ++k)
-                        if (row_ok[k]) store_f4(op + (size_t)k * g.nx, done[k], streaming);
-                    op += plane_stride;
-                }
-                return true;
-            });
-            if (!ok) {
+        for (int i = 0; i < nplanes; ++i) {
+            if (!mbar_wait_bounded(full0 + 8 * s, ph)) {
                 atomicExch(status, kStatusTimeout);
                 return;
+            }
+            const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
+            const float* colp = pl + row0 * PX + 4 + 4 * lane;
+            // Rows are visited once, top to bottom.  A row is a y-neighbour of up to 2R output
+            // rows and the centre row of at most one; it is consumed at once, so only one
+            // loaded row is live at a time.  acc[k] is the output whose centre plane this is:
+            // it continues from the partial sum A[k][R] that the planes below have built.
+            float acc[K][4];
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+                acc[k][0] = A[k][R].x; acc[k][1] = A[k][R].y; acc[k][2] = A[k][R].z; acc[k][3] = A[k][R].w;
+            }
+            float4 done[K];
+#pragma unroll
+            for (int kk = 0; kk < K + 2 * R; ++kk) {
+                const float4 c = *reinterpret_cast<const float4*>(colp + kk * PX);
+#pragma unroll
+                for (int k = 0; k < K; ++k) {
+                    const int d = kk - k - R;              // row kk is tap dy = d of output row k
+                    if (d != 0 && d >= -R && d <= R) {
+#pragma unroll
+                        for (int m = 0; m < 4; ++m) acc[k][m] = fmaf(sw.y[d + R], f4get(c, m), acc[k][m]);
+                    }
+                }
+                if (kk >= R && kk < K + R) {
+                    const int k = kk - R;                  // centre row of output row k
+                    float v[4 + 2 * R];
+                    gather_row<R>(colp + kk * PX, pl + (row0 + kk) * PX, lane, c, v);
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) {
+                        float a = fmaf(sw.c, v[R + m], acc[k][m]);
+#pragma unroll
+                        for (int d = 1; d <= R; ++d) {
+                            a = fmaf(sw.x[R - d], v[R + m - d], a);
+                            a = fmaf(sw.x[R + d], v[R + m + d], a);
+                        }
+                        acc[k][m] = a;
+                    }
+                    // z taps: this plane is tap dz = +R of the oldest output (now complete),
+                    // dz = R-1-j of the one moving into slot j, dz = -R of the new one
+                    done[k].x = fmaf(sw.z[2 * R], c.x, A[k][0].x);
+                    done[k].y = fmaf(sw.z[2 * R], c.y, A[k][0].y);
+                    done[k].z = fmaf(sw.z[2 * R], c.z, A[k][0].z);
+                    done[k].w = fmaf(sw.z[2 * R], c.w, A[k][0].w);
+#pragma unroll
+                    for (int j = 0; j < 2 * R - 1; ++j) {
+                        if (j == R - 1) continue;          // that slot receives acc[k] below
+                        const float wz = sw.z[2 * R - 1 - j];
+                        A[k][j].x = fmaf(wz, c.x, A[k][j + 1].x);
+                        A[k][j].y = fmaf(wz, c.y, A[k][j + 1].y);
+                        A[k][j].z = fmaf(wz, c.z, A[k][j + 1].z);
+                        A[k][j].w = fmaf(wz, c.w, A[k][j + 1].w);
+                    }
+                    A[k][2 * R - 1] = make_float4(sw.z[0] * c.x, sw.z[0] * c.y, sw.z[0] * c.z, sw.z[0] * c.w);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < K; ++k)
+                A[k][R - 1] = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
+            __syncwarp();
+            mbar_arrive_if(lane == 0, empty0 + 8 * s);
+            if (++s == nstage) { s = 0; ph ^= 1; }
+
+            if (i >= 2 * R) {
+#pragma unroll
+                for (int k = 0; k < K; ++k)
+                    if (row_ok[k]) store_f4(op + (size_t)k * g.nx, done[k], streaming);
+                op += plane_stride;
             }
         }
     } else {
