@@ -432,7 +432,7 @@ int choose_chunk(const stencil_plan_s* p, const StreamConfig* cfg, int stages, d
 }
 
 int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
-    const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 4;
+    const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : (issue_bound(p) ? 5 : 4);
     if (!p->stream_cfg_fixed && !p->stream_cfg_tuned) {
         // pick the tile height that balances this grid best (same rows per thread)
         const StreamConfig* best_cfg = p->stream_cfg;
@@ -494,7 +494,7 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
     if (g.tile_x < 4 || g.tile_y < 1) return STENCIL_ERR_UNSUPPORTED;
     g.tiles_y = (p->ny + g.tile_y - 1) / g.tile_y;
     // shared memory: input ring + two planes per intermediate level
-    int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
+    int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 2;   // measured: 2 beats 3 and 4
     auto smem_for = [&](int s) { return (size_t)(s + 2 * (T - 1)) * cfg->slot_bytes + 128 + kMaxStages * sizeof(uint64_t); };
     while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;
     const size_t smem = smem_for(stages);
