@@ -18,6 +18,7 @@
 #include "kernel_generic.cuh"
 #include "kernel_stream.cuh"
 #include "kernel_fused.cuh"
+#include "kernel_rows2d.cuh"
 
 using namespace stencil;
 
@@ -79,6 +80,20 @@ struct FusedConfig {
                           int grid, size_t smem, cudaStream_t);
 };
 
+// ---------------------------------------------------------------------------
+// ROWS2D kernel configurations (2D grids)
+// ---------------------------------------------------------------------------
+struct Rows2DConfig {
+    int radius;
+    bool box;
+    int YB, NW, batch_bytes;
+    const void* kernel;
+    mutable size_t smem_allowed;
+    mutable int cache_device;
+    cudaError_t (*launch)(const struct stencil_plan_s*, const CUtensorMap&, float*, const Rows2DGeom&,
+                          int grid, size_t smem, cudaStream_t);
+};
+
 }  // namespace
 
 struct stencil_plan_s {
@@ -103,6 +118,7 @@ struct stencil_plan_s {
     bool stream_cfg_fixed;         // the caller chose the tile shape
     bool stream_cfg_tuned;         // the library has chosen it for this grid
     const FusedConfig* fused_cfg;  // non-null: iterated applies run fused passes
+    const Rows2DConfig* rows2d_cfg; // non-null: 2D grid on the row-streaming kernel
     int tile_x;                    // requested region width for fused passes (0 = auto)
     // bookkeeping
     int64_t launches;
@@ -239,23 +255,61 @@ const FusedConfig* find_fused_cfg(int radius, int T, int txe) {
     return nullptr;
 }
 
+template <int R, bool BOX, int YB, int NW>
+cudaError_t launch_rows2d_t(const stencil_plan_s* p, const CUtensorMap& map, float* out, const Rows2DGeom& g,
+                            int grid, size_t smem, cudaStream_t st) {
+    Weights2D<R> wt;
+    for (int a = -R; a <= R; ++a)
+        for (int b = -R; b <= R; ++b) wt.w[a + R][b + R] = dense_w(p, 0, a, b);
+    stencil_rows2d_kernel<R, BOX, YB, NW><<<grid, NW * 32, smem, st>>>(map, out, g, wt, p->d_status);
+    return cudaGetLastError();
+}
+
+template <int R, bool BOX, int YB, int NW>
+Rows2DConfig make_rows2d() {
+    Rows2DConfig c;
+    c.radius = R; c.box = BOX; c.YB = YB; c.NW = NW; c.batch_bytes = Rows2DShape<YB>::BATCH_BYTES;
+    c.kernel = reinterpret_cast<const void*>(&stencil_rows2d_kernel<R, BOX, YB, NW>);
+    c.smem_allowed = 0; c.cache_device = -1;
+    c.launch = &launch_rows2d_t<R, BOX, YB, NW>;
+    return c;
+}
+
+const std::vector<Rows2DConfig>& rows2d_configs() {
+    static const std::vector<Rows2DConfig> v = {
+        make_rows2d<1, false, 8, 8>(), make_rows2d<2, false, 8, 8>(), make_rows2d<3, false, 8, 8>(),
+        make_rows2d<4, false, 8, 8>(),
+        make_rows2d<1, true, 8, 8>(),  make_rows2d<2, true, 8, 8>(),  make_rows2d<3, true, 8, 8>(),
+    };
+    return v;
+}
+
+const Rows2DConfig* find_rows2d_cfg(int radius, bool box) {
+    for (const Rows2DConfig& c : rows2d_configs())
+        if (c.radius == radius && c.box == box) return &c;
+    return nullptr;
+}
+
+// The tiled kernels need a zero boundary (TMA fills out-of-grid cells with zero) and rows
+// whose byte length is a multiple of 16 (a TMA stride rule).
 bool stream_supported(const stencil_plan_s* p) {
-    if (p->ndim != 3 || p->boundary != STENCIL_ZERO) return false;
-    if (p->nx % 4 != 0) return false;              // TMA global strides must be 16-byte multiples
+    if (p->boundary != STENCIL_ZERO || p->nx % 4 != 0) return false;
     const bool box = p->shape == STENCIL_BOX;
+    if (p->ndim == 2) return find_rows2d_cfg(p->radius, box) != nullptr;
     return find_stream_cfg(p->radius, box, 0, 0) != nullptr;
 }
 
 // Temporal blocking covers what the STREAM kernels cover, restricted to star stencils.
 const FusedConfig* pick_fused(const stencil_plan_s* p) {
-    if (!stream_supported(p) || p->shape != STENCIL_STAR) return nullptr;
+    if (!stream_supported(p) || p->shape != STENCIL_STAR || p->ndim != 3) return nullptr;
     if (p->fuse_steps == 1) return nullptr;
     int txe = p->tile_x;
     if (p->fuse_steps == 0 && txe == 0) {
-        // default: two steps per pass on a 256-wide region when that covers a whole row
-        // (no redundant columns), otherwise four steps on 128-wide regions
-        const FusedConfig* c = p->nx <= 256 ? find_fused_cfg(p->radius, 2, 256) : find_fused_cfg(p->radius, 4, 128);
-        return c ? c : find_fused_cfg(p->radius, 0, 0);
+        // Default: fuse two steps per pass when one 256-wide region spans a whole row (no
+        // redundant columns).  On wider grids the halo recomputation of several regions per
+        // row costs more than the saved traffic (measured on 512^3), so those stay unfused
+        // unless the caller asks for fusion.
+        return p->nx <= 256 ? find_fused_cfg(p->radius, 2, 256) : nullptr;
     }
     return find_fused_cfg(p->radius, p->fuse_steps, txe);
 }
@@ -265,6 +319,13 @@ int resolve_variant(stencil_plan_s* p, int want) {
     if (want == STENCIL_VARIANT_GENERIC) { p->variant = want; p->fused_cfg = nullptr; return STENCIL_OK; }
     if (want == STENCIL_VARIANT_STREAM || want == STENCIL_VARIANT_FUSED) {
         if (!stream_supported(p)) return STENCIL_ERR_UNSUPPORTED;
+        if (p->ndim == 2) {
+            if (want == STENCIL_VARIANT_FUSED) return STENCIL_ERR_UNSUPPORTED;
+            p->rows2d_cfg = find_rows2d_cfg(p->radius, p->shape == STENCIL_BOX);
+            p->stream_cfg = nullptr; p->fused_cfg = nullptr;
+            p->variant = STENCIL_VARIANT_STREAM;
+            return STENCIL_OK;
+        }
         const StreamConfig* c = find_stream_cfg(p->radius, p->shape == STENCIL_BOX, p->tile_y, p->rows_per_thread);
         if (!c) return STENCIL_ERR_UNSUPPORTED;
         const FusedConfig* f = pick_fused(p);
@@ -472,6 +533,54 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     return STENCIL_OK;
 }
 
+// 2D grids: one warp per (128-column strip, chunk of rows).
+int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
+    const Rows2DConfig* cfg = p->rows2d_cfg;
+    const CUtensorMap* map = nullptr;
+    int rc = get_tensor_map(p, cfg, kStreamPX, cfg->YB, src, &map);
+    if (rc != STENCIL_OK) return rc;
+    const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
+    const size_t smem = (size_t)cfg->NW * stages * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8;
+    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->cache_device = dev; }
+    if (smem > cfg->smem_allowed) {
+        if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+            cudaGetLastError();
+            return STENCIL_ERR_CUDA;
+        }
+        cfg->smem_allowed = smem;
+    }
+    Rows2DGeom g;
+    g.ny = p->ny; g.nx = p->nx;
+    g.strips = (p->nx + kStreamTX - 1) / kStreamTX;
+    g.stages = stages;
+    int chunk = p->chunk_z;                          // the streamed axis of a 2D grid is y
+    if (chunk <= 0) {
+        // As many (strip, chunk) units as fill the machine's warp slots once (two CTAs per SM),
+        // never more: a second, partial wave of long units would double the run time.  A unit
+        // reads chunk + 2R rows in batches of YB, so chunk + 2R is made a whole number of
+        // batches; small grids end up with one batch per warp and as many warps as rows allow.
+        const int R = p->radius;
+        const int slots = 2 * sm_count() * cfg->NW;
+        const int nch_max = std::max(1, slots / g.strips);
+        const int chunk_min = (p->ny + nch_max - 1) / nch_max;
+        int nbatch = std::max(1, (chunk_min + 2 * R + cfg->YB - 1) / cfg->YB);
+        while (nbatch * cfg->YB - 2 * R < 1) ++nbatch;
+        chunk = nbatch * cfg->YB - 2 * R;
+    }
+    chunk = std::max(1, std::min(chunk, p->ny));
+    g.chunk_y = chunk;
+    g.nchunks = (p->ny + chunk - 1) / chunk;
+    const int64_t units = (int64_t)g.strips * g.nchunks;
+    const int64_t grid64 = (units + cfg->NW - 1) / cfg->NW;
+    if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
+    if (cfg->launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
+    p->launches++;
+    return STENCIL_OK;
+}
+
 // One fused pass: dst = S^nlev(src), nlev <= cfg->T.
 int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cudaStream_t st) {
     const FusedConfig* cfg = p->fused_cfg;
@@ -524,7 +633,8 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
 
 int launch_sweep(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
     switch (p->variant) {
-        case STENCIL_VARIANT_STREAM: return launch_stream(p, src, dst, st);
+        case STENCIL_VARIANT_STREAM:
+            return p->ndim == 2 ? launch_rows2d(p, src, dst, st) : launch_stream(p, src, dst, st);
         default: return launch_generic(p, src, dst, st);
     }
 }
@@ -604,7 +714,7 @@ int stencil_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int ra
     p->host_in = nullptr; p->host_out = nullptr;
     p->variant = STENCIL_VARIANT_GENERIC;
     p->tile_y = 0; p->rows_per_thread = 0; p->chunk_z = 0; p->stages = 0; p->fuse_steps = 0; p->streaming_store = 0;
-    p->stream_cfg = nullptr; p->fused_cfg = nullptr; p->tile_x = 0;
+    p->stream_cfg = nullptr; p->fused_cfg = nullptr; p->rows2d_cfg = nullptr; p->tile_x = 0;
     p->stream_cfg_fixed = false; p->stream_cfg_tuned = false;
     p->launches = 0; p->last_stream = nullptr; p->used = false;
 
@@ -838,6 +948,7 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
             if (value < 0) return STENCIL_ERR_INVALID;
             int ty = key == STENCIL_KEY_TILE_Y ? (int)value : p->tile_y;
             int k = key == STENCIL_KEY_ROWS_PER_THREAD ? (int)value : p->rows_per_thread;
+            if (p->variant == STENCIL_VARIANT_STREAM && p->ndim == 2) return value == 0 ? STENCIL_OK : STENCIL_ERR_UNSUPPORTED;
             if (p->variant == STENCIL_VARIANT_STREAM) {
                 const StreamConfig* c = find_stream_cfg(p->radius, p->shape == STENCIL_BOX, ty, k);
                 if (!c) return STENCIL_ERR_UNSUPPORTED;
@@ -871,6 +982,7 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
         case STENCIL_KEY_VARIANT: *value = p->variant; return STENCIL_OK;
         case STENCIL_KEY_TILE_X:
             *value = p->variant != STENCIL_VARIANT_STREAM ? 0 : (p->fused_cfg ? p->fused_cfg->txe : kStreamTX);
+            if (p->ndim == 2 && p->variant == STENCIL_VARIANT_STREAM) *value = kStreamTX;
             return STENCIL_OK;
         case STENCIL_KEY_TILE_Y:
             *value = (p->variant == STENCIL_VARIANT_STREAM && p->stream_cfg) ? p->stream_cfg->tile_y : 0;

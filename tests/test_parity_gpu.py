@@ -182,6 +182,45 @@ def test_non_default_stream():
     assert np.max(np.abs(dst.cpu().numpy() - want)) <= wl.tolerance(w, float(np.abs(a).max()), 3)
 
 
+# ------------------------------------------------------------- 2D row streaming --
+ROWS2D_OPS = [(1, False), (2, False), (3, False), (4, False), (1, True), (2, True), (3, True)]
+
+
+@pytest.mark.parametrize("R,box", ROWS2D_OPS)
+@pytest.mark.parametrize("dims,chunk,stages", [
+    ((67, 132), 0, 0),           # two strips, the second 4 columns wide; ragged rows
+    ((200, 260), 37, 2),         # several chunks of rows per strip, chunk not a multiple of the batch
+    ((3, 8), 0, 0),              # smaller than the stencil reach and than one batch
+    ((129, 1024), 16, 4),        # many strips, short chunks
+])
+def test_rows2d_kernel_matches_oracle(R, box, dims, chunk, stages):
+    w = wl.random_box_weights(2, R, 71) if box else wl.random_star_weights(2, R, 71)
+    a = wl.normal_field(dims, 72)
+    used = check(dims, R, b.BOX if box else b.STAR, w, b.ZERO, a, variant=b.VARIANT_STREAM,
+                 chunk_z=chunk or None, stages=stages or None)
+    assert used == "stream"
+
+
+@pytest.mark.parametrize("R,box", [(1, False), (3, True)])
+def test_rows2d_iteration(R, box):
+    dims = (150, 384)
+    w = wl.random_box_weights(2, R, 73) if box else wl.random_star_weights(2, R, 73)
+    a = wl.normal_field(dims, 74)
+    for steps in (2, 5):
+        check(dims, R, b.BOX if box else b.STAR, w, b.ZERO, a, steps=steps)
+
+
+def test_paper_shaped_2d_box_radius3():
+    """The paper's operator (2D box, radius 3, 49 points) on a grid that spans many
+    strips and chunks, iterated like its protocol."""
+    wk = wl.get("paper2d").scaled((1536, 2048), steps=3)
+    a, w = wk.input(), wk.weights()
+    got, used = gpu_sweep(wk.dims, wk.radius, wk.shape, w, wk.boundary, a, wk.steps)
+    assert used == "stream"
+    want = oracle.apply(a, w, wk.boundary, wk.steps)
+    assert np.max(np.abs(got - want)) <= wl.tolerance(w, float(np.abs(a).max()), wk.steps)
+
+
 # -------------------------------------------------------------------- fused --
 FUSED_CONFIGS = [   # (radius, fuse_steps, region width)
     (1, 2, 256), (1, 3, 256), (1, 4, 128), (1, 2, 128), (1, 3, 128), (2, 2, 128),
@@ -229,6 +268,10 @@ def test_fused_equals_unfused_within_tolerance_and_keeps_zero_boundary():
 
 def test_fuse_knob_rules():
     star = wl.star_weights(3, 1, 0.4, [0.1])
+    with b.Plan((64, 64, 512), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # rows wider than one region: unfused by default
+        p.set(b.KEY_FUSE_STEPS, 4)
+        assert p.get(b.KEY_FUSE_STEPS) == 4
     with b.Plan((64, 64, 64), 1, b.STAR, star, b.ZERO) as p:
         assert p.get(b.KEY_FUSE_STEPS) >= 2         # iterated applies fuse by default
         p.set(b.KEY_FUSE_STEPS, 1)
