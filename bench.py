@@ -181,6 +181,22 @@ def config_summary(wk, total_ms, steps, peak):
             "taps": wk.taps()}
 
 
+def max_over_ranks(value, dist, device):
+    """Largest `value` over all ranks (timings of a multi-rank run are the slowest rank's)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gpoints(world, point_updates_per_apply, applies, total_ms):
+    """Replicas only: every rank sweeps its own full grid, so the job's point count is
+    world x one rank's, over the slowest rank's time."""
+    return world * point_updates_per_apply * applies / (total_ms / 1e3) / 1e9
+
+
 def pick_workload(args):
     wk = wl.get(args.workload)
     if args.dims:
@@ -262,12 +278,7 @@ def run_gpu(args):
         torch.cuda.synchronize()
     t_load1 = time.time()
 
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms_max = float(t.item())
-    else:
-        total_ms_max = total_ms
+    total_ms_max = max_over_ranks(total_ms, dist, dev)
 
     # ---- end to end: host buffers through the C ABI, copies inside the timing --
     e2e = None
@@ -284,12 +295,8 @@ def run_gpu(args):
             plan.apply_host(hsrc, hdst, wk.steps, stream.cuda_stream)
         e1.record(stream)
         barrier()
-        e2e_ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e = {"value": round(world * wk.point_updates * e2e_steps / (e2e_ms / 1e3) / 1e9, 4),
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
+        e2e = {"value": round(whole_job_gpoints(world, wk.point_updates, e2e_steps, e2e_ms), 4),
                "unit": UNIT, "h2d_bytes_per_step": int(a_host.nbytes), "d2h_bytes_per_step": int(a_host.nbytes),
                "steps": e2e_steps, "ms_per_step": round(e2e_ms / e2e_steps, 4),
                "api": "stencil_apply_host (pinned host buffers)"}
@@ -355,7 +362,7 @@ def run_gpu(args):
 
     if rank == 0:
         pts = world * wk.point_updates * args.steps
-        value = pts / (total_ms_max / 1e3) / 1e9
+        value = whole_job_gpoints(world, wk.point_updates, args.steps, total_ms_max)
         line = {
             "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(total_ms_max / args.steps, 5),

@@ -129,7 +129,11 @@ STENCIL_API int stencil_apply(stencil_plan_t plan, const float* in, float* out, 
  * `out_host` and waits for it.  Pinned host memory makes the copies
  * asynchronous up to the final wait; pageable memory works but is slower.
  * `in_host` and `out_host` may be the same buffer.  Allocates two plan-owned
- * device grids of N floats on first use.
+ * device grids of N floats on first use.  A single sweep (steps == 1) of a 3D
+ * grid on the tiled kernel is pipelined: the grid is cut into 8 or 16 slabs of planes
+ * and the upload of one slab, the sweep of the previous one and the download
+ * of the one before overlap on two plan-owned copy streams (ordered after the
+ * work already queued on `stream`), which needs pinned host memory to pay off.
  */
 STENCIL_API int stencil_apply_host(stencil_plan_t plan, const float* in_host, float* out_host, int steps,
                        void* stream);

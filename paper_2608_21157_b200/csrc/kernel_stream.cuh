@@ -46,6 +46,7 @@ struct BoxWeights {             // dense cube, [dz+R][dy+R][dx+R]
 struct StreamGeom {
     int nz, ny, nx;
     int tiles_x, tiles_y;
+    int z_begin, z_end;         // output planes of this launch: [z_begin, z_end), normally [0, nz)
     int chunk_z;                // planes of output per CTA
     int stages;                 // depth of the plane ring
     int streaming_store;        // 1: st.global.cs
@@ -169,8 +170,8 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
     const int chunk = bid / (g.tiles_x * g.tiles_y);
     const int x0 = tile_x * kStreamTX;
     const int y0 = tile_y * S::TY;
-    const int z0 = chunk * g.chunk_z;
-    const int z1 = min(z0 + g.chunk_z, g.nz);
+    const int z0 = g.z_begin + chunk * g.chunk_z;
+    const int z1 = min(z0 + g.chunk_z, g.z_end);
     const int nplanes = (z1 - z0) + 2 * R;      // input planes z0-R .. z1-1+R
     const int pstart = z0 - R;
 

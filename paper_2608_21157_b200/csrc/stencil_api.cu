@@ -111,6 +111,8 @@ struct stencil_plan_s {
     float* scratch;                // N floats, iteration ping-pong
     float* host_in;                // N floats each, apply_host staging
     float* host_out;
+    cudaStream_t copy_in, copy_out; // apply_host: upload / download streams (created on first use)
+    std::vector<cudaEvent_t> events; // apply_host: slab hand-over events
     // selection and tuning
     int variant;                   // resolved STENCIL_VARIANT_*
     int tile_y, rows_per_thread, chunk_z, stages, fuse_steps, streaming_store;
@@ -461,27 +463,29 @@ bool issue_bound(const stencil_plan_s* p) {
 }
 
 // Planes of output per CTA, and the relative cost of the launch, for one configuration.
-int choose_chunk(const stencil_plan_s* p, const StreamConfig* cfg, int stages, double* cost_out) {
+int choose_chunk(const stencil_plan_s* p, const StreamConfig* cfg, int stages, double* cost_out,
+                 int span = 0) {
     const int R = p->radius;
+    const int nz = span > 0 ? span : p->nz;      // planes this launch covers
     const int tiles = ((p->nx + kStreamTX - 1) / kStreamTX) * ((p->ny + cfg->tile_y - 1) / cfg->tile_y);
     const int occ = std::max(1, stream_occupancy(cfg, stages));
     const int slots = occ * sm_count();
     if (!issue_bound(p)) {
         // measured on 512^3: 32-plane chunks (several thousand short CTAs) beat every longer chunk
-        const int chunk = p->nz >= 64 ? 32 : p->nz;
+        const int chunk = nz >= 64 ? 32 : nz;
         if (cost_out) {
-            const int64_t ctas = (int64_t)tiles * ((p->nz + chunk - 1) / chunk);
+            const int64_t ctas = (int64_t)tiles * ((nz + chunk - 1) / chunk);
             *cost_out = ((double)ctas / slots + 0.5) * occ * (chunk + 2 * R) * cfg->tile_y;
         }
         return chunk;
     }
     const double fill = 4.0;                       // pipeline start-up, in planes
-    int best_chunk = p->nz;
+    int best_chunk = nz;
     double best = 1e300;
-    const int max_chunks = std::max(1, p->nz / std::max(8 * R, 16));
+    const int max_chunks = std::max(1, nz / std::max(8 * R, 16));
     for (int nch = 1; nch <= max_chunks; ++nch) {
-        const int chunk = (p->nz + nch - 1) / nch;
-        const int real_nch = (p->nz + chunk - 1) / chunk;
+        const int chunk = (nz + nch - 1) / nch;
+        const int real_nch = (nz + chunk - 1) / chunk;
         const int64_t ctas = (int64_t)tiles * real_nch;
         const double waves = (double)((ctas + slots - 1) / slots);
         // CTAs resident together share the SM, so a wave of `occ` CTAs per SM costs occ units
@@ -492,7 +496,11 @@ int choose_chunk(const stencil_plan_s* p, const StreamConfig* cfg, int stages, d
     return best_chunk;
 }
 
-int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
+// dst[z_begin, z_end) = one sweep of src; the whole grid when z_end <= z_begin.
+int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st, int z_begin = 0,
+                  int z_end = 0) {
+    if (z_end <= z_begin) { z_begin = 0; z_end = p->nz; }
+    const int span = z_end - z_begin;
     const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : (issue_bound(p) ? 5 : 4);
     if (!p->stream_cfg_fixed && !p->stream_cfg_tuned) {
         // pick the tile height that balances this grid best (same rows per thread)
@@ -521,10 +529,11 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     g.streaming_store = p->streaming_store;
     const int tiles = g.tiles_x * g.tiles_y;
     if (stream_occupancy(cfg, stages) <= 0) return STENCIL_ERR_UNSUPPORTED;
-    int chunk = p->chunk_z > 0 ? p->chunk_z : choose_chunk(p, cfg, stages, nullptr);
-    chunk = std::max(1, std::min(chunk, p->nz));
+    int chunk = p->chunk_z > 0 ? p->chunk_z : choose_chunk(p, cfg, stages, nullptr, span);
+    chunk = std::max(1, std::min(chunk, span));
     g.chunk_z = chunk;
-    const int nchunks = (p->nz + chunk - 1) / chunk;
+    g.z_begin = z_begin; g.z_end = z_end;
+    const int nchunks = (span + chunk - 1) / chunk;
     const int64_t grid64 = (int64_t)tiles * nchunks;
     if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
     const size_t smem = stream_smem_bytes(cfg, stages);
@@ -712,6 +721,7 @@ int stencil_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int ra
     p->device = -1;
     p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr;
     p->host_in = nullptr; p->host_out = nullptr;
+    p->copy_in = nullptr; p->copy_out = nullptr;
     p->variant = STENCIL_VARIANT_GENERIC;
     p->tile_y = 0; p->rows_per_thread = 0; p->chunk_z = 0; p->stages = 0; p->fuse_steps = 0; p->streaming_store = 0;
     p->stream_cfg = nullptr; p->fused_cfg = nullptr; p->rows2d_cfg = nullptr; p->tile_x = 0;
@@ -796,17 +806,69 @@ int stencil_apply_host(stencil_plan_t p, const float* in_host, float* out_host, 
     if ((rc = ensure_grid(&p->host_out, p->npoints)) != STENCIL_OK) return rc;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const size_t bytes = (size_t)p->npoints * sizeof(float);
-    if (cudaMemcpyAsync(p->host_in, in_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
-        cudaGetLastError();
-        return STENCIL_ERR_CUDA;
+
+    // A single 3D sweep on the tiled kernel is cut into slabs of planes so that the upload
+    // of slab s+1, the sweep of slab s and the download of slab s-1 overlap (the copies are
+    // what costs time: the sweep itself is ~1 % of a PCIe round trip).
+    constexpr int kMaxSlabs = 16;
+    const int min_planes = std::max(2 * p->radius, 8);           // per slab
+    const int kSlabs = p->nz >= kMaxSlabs * 2 * min_planes ? kMaxSlabs : kMaxSlabs / 2;
+    const bool pipelined = steps == 1 && p->variant == STENCIL_VARIANT_STREAM && p->ndim == 3 &&
+                           p->nz >= kSlabs * min_planes;
+    if (!pipelined) {
+        if (cudaMemcpyAsync(p->host_in, in_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+            cudaGetLastError();
+            return STENCIL_ERR_CUDA;
+        }
+        rc = stencil_apply(p, p->host_in, p->host_out, steps, stream);
+        if (rc != STENCIL_OK) return rc;
+        if (cudaMemcpyAsync(out_host, p->host_out, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess) {
+            cudaGetLastError();
+            return STENCIL_ERR_CUDA;
+        }
+        return STENCIL_OK;
     }
-    rc = stencil_apply(p, p->host_in, p->host_out, steps, stream);
-    if (rc != STENCIL_OK) return rc;
-    if (cudaMemcpyAsync(out_host, p->host_out, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaStreamSynchronize(st) != cudaSuccess) {
-        cudaGetLastError();
-        return STENCIL_ERR_CUDA;
+
+    auto fail = [&]() { cudaGetLastError(); return STENCIL_ERR_CUDA; };
+    if (!p->copy_in && cudaStreamCreateWithFlags(&p->copy_in, cudaStreamNonBlocking) != cudaSuccess) return fail();
+    if (!p->copy_out && cudaStreamCreateWithFlags(&p->copy_out, cudaStreamNonBlocking) != cudaSuccess) return fail();
+    while ((int)p->events.size() < 2 * kMaxSlabs + 2) {
+        cudaEvent_t e;
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return fail();
+        p->events.push_back(e);
     }
+    cudaEvent_t* up = p->events.data();              // up[s]: slab s is on the device
+    cudaEvent_t* swept = p->events.data() + kMaxSlabs;  // swept[s]: slab s of the result is ready
+    cudaEvent_t start = p->events[2 * kMaxSlabs], finished = p->events[2 * kMaxSlabs + 1];
+    p->last_stream = st;
+    p->used = true;
+
+    const size_t plane = (size_t)p->ny * p->nx;
+    auto slab_begin = [&](int s) { return (int)((int64_t)p->nz * s / kSlabs); };
+    if (cudaEventRecord(start, st) != cudaSuccess) return fail();
+    if (cudaStreamWaitEvent(p->copy_in, start, 0) != cudaSuccess) return fail();
+    if (cudaStreamWaitEvent(p->copy_out, start, 0) != cudaSuccess) return fail();
+    for (int s = 0; s < kSlabs; ++s) {
+        const int z0 = slab_begin(s), z1 = slab_begin(s + 1);
+        if (cudaMemcpyAsync(p->host_in + z0 * plane, in_host + z0 * plane, (z1 - z0) * plane * sizeof(float),
+                            cudaMemcpyHostToDevice, p->copy_in) != cudaSuccess) return fail();
+        if (cudaEventRecord(up[s], p->copy_in) != cudaSuccess) return fail();
+    }
+    for (int s = 0; s < kSlabs; ++s) {
+        const int z0 = slab_begin(s), z1 = slab_begin(s + 1);
+        // the sweep of slab s reads R planes of slab s+1 as well
+        if (cudaStreamWaitEvent(st, up[std::min(s + 1, kSlabs - 1)], 0) != cudaSuccess) return fail();
+        rc = launch_stream(p, p->host_in, p->host_out, st, z0, z1);
+        if (rc != STENCIL_OK) return rc;
+        if (cudaEventRecord(swept[s], st) != cudaSuccess) return fail();
+        if (cudaStreamWaitEvent(p->copy_out, swept[s], 0) != cudaSuccess) return fail();
+        if (cudaMemcpyAsync(out_host + z0 * plane, p->host_out + z0 * plane, (z1 - z0) * plane * sizeof(float),
+                            cudaMemcpyDeviceToHost, p->copy_out) != cudaSuccess) return fail();
+    }
+    if (cudaEventRecord(finished, p->copy_out) != cudaSuccess) return fail();
+    if (cudaStreamWaitEvent(st, finished, 0) != cudaSuccess) return fail();
+    if (cudaStreamSynchronize(st) != cudaSuccess) return fail();
     return STENCIL_OK;
 }
 
@@ -871,6 +933,9 @@ int stencil_destroy(stencil_plan_t p) {
         void* ptrs[] = {p->d_status, p->scratch, p->host_in, p->host_out, p->d_taps};
         for (void* q : ptrs)
             if (q && cudaFree(q) != cudaSuccess) rc = STENCIL_ERR_CUDA;
+        for (cudaEvent_t e : p->events) cudaEventDestroy(e);
+        if (p->copy_in) cudaStreamDestroy(p->copy_in);
+        if (p->copy_out) cudaStreamDestroy(p->copy_out);
         if (p->device >= 0 && cur >= 0 && cur != p->device) cudaSetDevice(cur);
         cudaGetLastError();
     }

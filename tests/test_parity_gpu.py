@@ -152,7 +152,7 @@ def test_time_composition_on_gpu():
 
 
 def test_apply_host_round_trip():
-    wk = wl.get("cfg2").scaled((40, 48, 128))
+    wk = wl.get("cfg2").scaled((40, 48, 128))       # too few planes for slabs: one upload, one sweep
     a = wk.input()
     w = wk.weights()
     src = torch.from_numpy(a).pin_memory()
@@ -162,6 +162,30 @@ def test_apply_host_round_trip():
         assert p.launches == 1
         assert p.get(b.KEY_SCRATCH_BYTES) == 2 * a.nbytes
     want = oracle.apply(a, w, b.ZERO, 1)
+    assert np.max(np.abs(dst.numpy() - want)) <= wl.tolerance(w, float(np.abs(a).max()), 1)
+
+
+@pytest.mark.parametrize("name,dims", [("cfg2", (100, 48, 128)), ("cfg4", (75, 40, 132)), ("cfg3", (64, 33, 128))])
+@pytest.mark.parametrize("pinned,in_place", [(True, False), (False, False), (True, True)])
+def test_apply_host_pipelined_slabs(name, dims, pinned, in_place):
+    """Enough planes for the slab pipeline (upload / sweep / download overlapped): slab seams
+    need the halo planes of the next slab, and an in-place host buffer must survive."""
+    wk = wl.get(name).scaled(dims)
+    a, w = wk.input(), wk.weights()
+    want = oracle.apply(a, w, b.ZERO, 1)
+    src = torch.from_numpy(a.copy())
+    if pinned:
+        src = src.pin_memory()
+    dst = src if in_place else torch.full_like(src, float("nan"))
+    if pinned and not in_place:
+        dst = dst.pin_memory()
+    with b.Plan.for_workload(wk) as p:
+        for _ in range(2):                           # second call reuses streams, events, grids
+            if in_place:
+                src.copy_(torch.from_numpy(a))
+            p.apply_host(src, dst, 1, torch.cuda.current_stream().cuda_stream)
+        assert p.launches == 16                      # 8 slabs per call
+        assert p.query_status() == b.OK
     assert np.max(np.abs(dst.numpy() - want)) <= wl.tolerance(w, float(np.abs(a).max()), 1)
 
 
