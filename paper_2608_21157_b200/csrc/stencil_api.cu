@@ -196,6 +196,7 @@ const std::vector<StreamConfig>& stream_configs() {
         make_cfg<4, false, 2, 16, 1>(),
         make_cfg<1, true, 2, 8, 1>(),   make_cfg<1, true, 2, 7, 4>(),   make_cfg<1, true, 4, 8, 1>(),
         make_cfg<1, true, 4, 7, 1>(),   make_cfg<1, true, 1, 8, 1>(),
+        make_cfg<2, true, 2, 8, 1>(),   make_cfg<2, true, 2, 7, 1>(),   make_cfg<2, true, 1, 8, 1>(),
     };
     return v;
 }
@@ -282,6 +283,7 @@ const std::vector<Rows2DConfig>& rows2d_configs() {
         make_rows2d<1, false, 8, 8>(), make_rows2d<2, false, 8, 8>(), make_rows2d<3, false, 8, 8>(),
         make_rows2d<4, false, 8, 8>(),
         make_rows2d<1, true, 8, 8>(),  make_rows2d<2, true, 8, 8>(),  make_rows2d<3, true, 8, 8>(),
+        make_rows2d<4, true, 8, 8>(),
     };
     return v;
 }
@@ -459,7 +461,7 @@ int stream_occupancy(const StreamConfig* cfg, int stages) {
 // simply get more bandwidth).  The others are bound by instruction issue: there
 // every SM must get the same amount of work, so the grid is cut into whole waves.
 bool issue_bound(const stencil_plan_s* p) {
-    return p->shape == STENCIL_STAR && p->radius >= 3;
+    return (p->shape == STENCIL_STAR && p->radius >= 3) || (p->shape == STENCIL_BOX && p->radius >= 2);
 }
 
 // Planes of output per CTA, and the relative cost of the launch, for one configuration.

@@ -92,6 +92,8 @@ def test_generic_iteration_and_ping_pong(steps, boundary):
 # ------------------------------------------------------------------- stream --
 def _stream_knob_sets(R, box):
     """Every compiled tile shape of the operator (tile_y = rows per thread x consumer warps)."""
+    if box and R == 2:
+        return [dict(), dict(tile_y=16), dict(tile_y=14), dict(tile_y=8)]
     if box or R == 1:
         return [dict(), dict(tile_y=16), dict(tile_y=14), dict(tile_y=32), dict(tile_y=28), dict(tile_y=8)]
     if R == 4:
@@ -102,7 +104,7 @@ def _stream_knob_sets(R, box):
     return [dict(), dict(tile_y=16), dict(tile_y=14), dict(tile_y=32)]
 
 
-STREAM_OPS = [(1, False), (2, False), (3, False), (4, False), (1, True)]
+STREAM_OPS = [(1, False), (2, False), (3, False), (4, False), (1, True), (2, True)]
 
 
 @pytest.mark.parametrize("R,box", STREAM_OPS)
@@ -207,7 +209,7 @@ def test_non_default_stream():
 
 
 # ------------------------------------------------------------- 2D row streaming --
-ROWS2D_OPS = [(1, False), (2, False), (3, False), (4, False), (1, True), (2, True), (3, True)]
+ROWS2D_OPS = [(1, False), (2, False), (3, False), (4, False), (1, True), (2, True), (3, True), (4, True)]
 
 
 @pytest.mark.parametrize("R,box", ROWS2D_OPS)
