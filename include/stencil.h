@@ -76,7 +76,13 @@ enum {
     STENCIL_KEY_CHUNK_Z      = 6,  /* set/get: planes per CTA along the streamed axis (0 = auto) */
     STENCIL_KEY_STAGES       = 7,  /* set/get: depth of the shared-memory plane ring (0 = auto)  */
     STENCIL_KEY_STREAMING_STORE = 8, /* set/get: 1 = write results with evict-first stores       */
-    STENCIL_KEY_ROWS_PER_THREAD = 9  /* set/get: tile rows each thread computes (0 = default)    */
+    STENCIL_KEY_ROWS_PER_THREAD = 9, /* set/get: tile rows each thread computes (0 = default)    */
+    STENCIL_KEY_WAIT_POLLS   = 10, /* set/get: polls after which a device-side wait of the 3D
+                                      single-step kernel gives up (each poll sleeps <= 20 us)    */
+    STENCIL_KEY_TEST_DROP_PLANE = 11 /* set/get, test hook: every CTA of the 3D single-step kernel
+                                      never loads its input plane of this index, so the bounded
+                                      wait for it expires and stencil_query_status reports
+                                      STENCIL_ERR_TIMEOUT (-1 = off, the default)                */
 };
 
 /*

@@ -50,6 +50,8 @@ struct StreamGeom {
     int chunk_z;                // planes of output per CTA
     int stages;                 // depth of the plane ring
     int streaming_store;        // 1: st.global.cs
+    unsigned wait_polls;        // cap of every bounded wait
+    int drop_plane;             // test hook: the producer never loads this plane of a CTA (-1: none)
 };
 
 template <int R, int K, int NW>
@@ -184,10 +186,12 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
             int s = 0;
             uint32_t ph = 1;                       // parity of the previous use of the slot
             for (int i = 0; i < nplanes; ++i) {
-                if (i >= nstage && !mbar_wait_bounded(empty0 + 8 * s, ph)) { ok = false; break; }
-                mbar_arrive_expect_tx(full0 + 8 * s, S::BOX_BYTES);
-                tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_BYTES), &tmap_in, full0 + 8 * s,
-                            x0 - 4, y0 - R, pstart + i);
+                if (i >= nstage && !mbar_wait_bounded(empty0 + 8 * s, ph, g.wait_polls)) { ok = false; break; }
+                if (i != g.drop_plane) {
+                    mbar_arrive_expect_tx(full0 + 8 * s, S::BOX_BYTES);
+                    tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_BYTES), &tmap_in, full0 + 8 * s,
+                                x0 - 4, y0 - R, pstart + i);
+                }
                 issued = i + 1;
                 if (++s == nstage) { s = 0; ph ^= 1; }
             }
@@ -195,7 +199,7 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                 atomicExch(status, kStatusTimeout);
                 // let copies already in flight land before the CTA's smem goes away
                 for (int i = max(0, issued - nstage); i < issued; ++i)
-                    mbar_wait_bounded(full0 + 8 * (i % nstage), (i / nstage) & 1);
+                    mbar_wait_bounded(full0 + 8 * (i % nstage), (i / nstage) & 1, g.wait_polls);
             }
         }
         return;
@@ -227,7 +231,7 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
             for (int j = 0; j < 2 * R; ++j) A[k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
 
         for (int i = 0; i < nplanes; ++i) {
-            if (!mbar_wait_bounded(full0 + 8 * s, ph)) {
+            if (!mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) {
                 atomicExch(status, kStatusTimeout);
                 return;
             }
@@ -315,7 +319,7 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                 constexpr int u = decltype(uc)::value;
                 const int i = i0 + u;
                 if (i >= nplanes) return true;
-                if (!mbar_wait_bounded(full0 + 8 * s, ph)) return false;
+                if (!mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) return false;
                 const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
                 const float* colp = pl + row0 * PX + 4 + 4 * lane;
                 float v[K + 2 * R][4 + 2 * R];

@@ -60,9 +60,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // records a timeout in the plan's status word and leaves the kernel.
 constexpr uint32_t kWaitPolls = 1u << 20;
 
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t polls = kWaitPolls) {
     if (mbar_try_wait(bar, parity)) return true;          // the usual case: already complete
-    for (uint32_t it = 1; it < kWaitPolls; ++it)
+    for (uint32_t it = 1; it < polls; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

@@ -116,6 +116,8 @@ struct stencil_plan_s {
     // selection and tuning
     int variant;                   // resolved STENCIL_VARIANT_*
     int tile_y, rows_per_thread, chunk_z, stages, fuse_steps, streaming_store;
+    unsigned wait_polls;           // cap of the bounded device waits (single-step 3D kernel)
+    int drop_plane;                // test hook, -1 = off
     const StreamConfig* stream_cfg;
     bool stream_cfg_fixed;         // the caller chose the tile shape
     bool stream_cfg_tuned;         // the library has chosen it for this grid
@@ -535,6 +537,7 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     chunk = std::max(1, std::min(chunk, span));
     g.chunk_z = chunk;
     g.z_begin = z_begin; g.z_end = z_end;
+    g.wait_polls = p->wait_polls; g.drop_plane = p->drop_plane;
     const int nchunks = (span + chunk - 1) / chunk;
     const int64_t grid64 = (int64_t)tiles * nchunks;
     if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
@@ -728,6 +731,7 @@ int stencil_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int ra
     p->tile_y = 0; p->rows_per_thread = 0; p->chunk_z = 0; p->stages = 0; p->fuse_steps = 0; p->streaming_store = 0;
     p->stream_cfg = nullptr; p->fused_cfg = nullptr; p->rows2d_cfg = nullptr; p->tile_x = 0;
     p->stream_cfg_fixed = false; p->stream_cfg_tuned = false;
+    p->wait_polls = kWaitPolls; p->drop_plane = -1;
     p->launches = 0; p->last_stream = nullptr; p->used = false;
 
     const int side = 2 * radius + 1;
@@ -1038,6 +1042,14 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
         case STENCIL_KEY_STREAMING_STORE:
             p->streaming_store = value ? 1 : 0;
             return STENCIL_OK;
+        case STENCIL_KEY_WAIT_POLLS:
+            if (value < 1 || value > (int64_t)kWaitPolls) return STENCIL_ERR_INVALID;
+            p->wait_polls = (unsigned)value;
+            return STENCIL_OK;
+        case STENCIL_KEY_TEST_DROP_PLANE:
+            if (value < -1 || value > 0x7fffffff) return STENCIL_ERR_INVALID;
+            p->drop_plane = (int)value;
+            return STENCIL_OK;
         default:
             return STENCIL_ERR_INVALID;
     }
@@ -1069,6 +1081,8 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
         case STENCIL_KEY_CHUNK_Z: *value = p->chunk_z; return STENCIL_OK;
         case STENCIL_KEY_STAGES: *value = p->stages; return STENCIL_OK;
         case STENCIL_KEY_STREAMING_STORE: *value = p->streaming_store; return STENCIL_OK;
+        case STENCIL_KEY_WAIT_POLLS: *value = p->wait_polls; return STENCIL_OK;
+        case STENCIL_KEY_TEST_DROP_PLANE: *value = p->drop_plane; return STENCIL_OK;
         default: return STENCIL_ERR_INVALID;
     }
 }

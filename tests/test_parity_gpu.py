@@ -310,6 +310,33 @@ def test_fuse_knob_rules():
             p.set(b.KEY_VARIANT, b.VARIANT_FUSED)
 
 
+# ------------------------------------------------------------ bounded waits --
+def test_expired_device_wait_is_reported_and_the_context_stays_usable():
+    """Failure detection without a fault: the producer is told never to load one input
+    plane, so the consumers' bounded wait for it runs out (64 polls of at most 20 us), the
+    kernel returns early, and the host reads STENCIL_ERR_TIMEOUT from the status word.
+    Nothing traps or spins forever; the next apply on the same plan is correct again."""
+    dims = (8, 16, 128)                              # one CTA
+    w = wl.star_weights(3, 1, -6.0, [1.0])
+    a = wl.uniform_field(dims, -1.0, 1.0, 91)
+    src = torch.from_numpy(a).cuda()
+    dst = torch.zeros_like(src)
+    stream = torch.cuda.current_stream().cuda_stream
+    with b.Plan(dims, 1, b.STAR, w, b.ZERO, variant=b.VARIANT_STREAM) as p:
+        p.set(b.KEY_WAIT_POLLS, 64)
+        p.set(b.KEY_TEST_DROP_PLANE, 2)
+        p.apply(src, dst, 1, stream)
+        assert p.query_status() == b.ERR_TIMEOUT
+        assert p.query_status() == b.OK              # the word is cleared by the query
+        p.set(b.KEY_TEST_DROP_PLANE, -1)
+        p.set(b.KEY_WAIT_POLLS, 1 << 20)
+        p.apply(src, dst, 1, stream)
+        assert p.query_status() == b.OK
+    torch.cuda.synchronize()
+    want = oracle.apply(a, w, b.ZERO, 1)
+    assert np.max(np.abs(dst.cpu().numpy() - want)) <= wl.tolerance(w, 1.0, 1)
+
+
 # ----------------------------------------------------- the five full configs --
 @pytest.mark.parametrize("name", wl.BASELINE_CONFIGS)
 def test_baseline_config_full_size(name):
