@@ -174,11 +174,12 @@ def config_summary(wk, total_ms, steps, peak):
     pts = wk.point_updates * steps
     sec = total_ms / 1e3
     gp = pts / sec / 1e9
-    gbs = 8.0 * pts / sec / 1e9
+    gbs = 2.0 * wk.itemsize * pts / sec / 1e9      # one read + one write of the grid's element type
     return {"gpoints_per_s": round(gp, 2), "effective_gbs": round(gbs, 1),
             "frac_of_measured_hbm": round(gbs / peak, 4), "frac_of_nominal_8tbs": round(gbs / NOMINAL_HBM_GBS, 4),
             "ms_per_apply": round(total_ms / steps, 5), "time_steps_per_apply": wk.steps,
-            "taps": wk.taps()}
+            "ms_per_time_step": round(total_ms / steps / max(wk.steps, 1), 5),
+            "taps": wk.taps(), "dtype": "f64" if wk.itemsize == 8 else "f32"}
 
 
 def max_over_ranks(value, dist, device):
@@ -308,7 +309,7 @@ def run_gpu(args):
     # algorithmic bytes: 8 B (one fp32 read + one write) per point per time step; a launch
     # advances N points by (time steps per apply / launches per apply) steps
     steps_per_launch = max(wk.steps, 1) / launches_per_apply
-    algo_bytes = 8.0 * wk.npoints * steps_per_launch
+    algo_bytes = 2.0 * wk.itemsize * wk.npoints * steps_per_launch
     achieved = algo_bytes / (kernel_ms / 1e3) / 1e9
     fuse = plan.get(b.KEY_FUSE_STEPS) if wk.steps > 1 else 1
     kernel_name = "stencil_generic_kernel" if plan.variant == "generic" else (
@@ -366,7 +367,8 @@ def run_gpu(args):
         line = {
             "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(total_ms_max / args.steps, 5),
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64" if wk.itemsize == 8 else "f32",
             "data": "synthetic (seeded numpy default_rng fields; see config.workload)",
             "config": {"workload": f"{wk.name}: {wk.description}", "dims": list(wk.dims), "radius": wk.radius,
                        "taps": wk.taps(), "time_steps_per_apply": wk.steps,
@@ -374,7 +376,7 @@ def run_gpu(args):
                              if 2 * a_host.nbytes > 126e6 else "working set fits L2; warm-L2 figure",
                        "parallelism": "replicas only (one full grid per GPU, no exchange)" if world > 1 else "1 GPU",
                        **info},
-            "effective_gbs": round(8.0 * pts / (total_ms_max / 1e3) / 1e9 / world, 1),
+            "effective_gbs": round(2.0 * wk.itemsize * pts / (total_ms_max / 1e3) / 1e9 / world, 1),
             "gpu_launches": int(launches),
             "clocks": clocks,
             "e2e": e2e,
@@ -518,7 +520,7 @@ def main():
     ap.add_argument("--stages", type=int, default=None)
     ap.add_argument("--fuse-steps", dest="fuse_steps", type=int, default=None)
     ap.add_argument("--streaming-store", dest="streaming_store", type=int, default=None)
-    ap.add_argument("--also", default="cfg1,cfg3,cfg4,cfg5,cfg5L,paper2d", help="other workloads summarised in all_configs")
+    ap.add_argument("--also", default="cfg1,cfg3,cfg4,cfg5,cfg5L,paper2d,paper2d_f64", help="other workloads summarised in all_configs")
     ap.add_argument("--also-steps", dest="also_steps", type=int, default=20)
     ap.add_argument("--no-all-configs", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

@@ -130,6 +130,22 @@ STENCIL_API int stencil_plan(stencil_plan_t* plan_out, int ndim, const int64_t* 
 STENCIL_API int stencil_apply(stencil_plan_t plan, const float* in, float* out, int steps, void* stream);
 
 /*
+ * stencil_plan_f64 / stencil_apply_f64 — the same operation on FP64 grids, the
+ * precision of the paper's own case study ("Case-study protocol": FP64).
+ * Arguments, layout, ownership and errors are those of stencil_plan and
+ * stencil_apply with double in place of float (rows must still be 16-byte
+ * multiples for the tiled kernel: nx even).  A plan made by one of the two
+ * plan calls is only accepted by the matching apply call (STENCIL_ERR_INVALID
+ * otherwise); stencil_destroy, stencil_query_status and the knobs serve both.
+ * 2D grids with a zero boundary and radius <= 4 (box: <= 3) run on a TMA
+ * row-streaming kernel; everything else on the one-thread-per-point kernel.
+ */
+STENCIL_API int stencil_plan_f64(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radius,
+                                 int shape, const double* weights, int boundary);
+STENCIL_API int stencil_apply_f64(stencil_plan_t plan, const double* in, double* out, int steps,
+                                  void* stream);
+
+/*
  * stencil_apply_host — the same operation on HOST buffers: copies `in_host`
  * to a plan-owned device grid, runs stencil_apply, copies the result back to
  * `out_host` and waits for it.  Pinned host memory makes the copies

@@ -18,7 +18,9 @@
  * Precision: the sum is accumulated in double over the float32 weights and
  * float32 inputs, in dense C order of the offsets, and rounded to float32
  * once per point per step.  Weights that are exactly zero are skipped (a star
- * stencil is a dense cube with zeros off the axes).
+ * stencil is a dense cube with zeros off the axes).  The paper's own case
+ * study runs in FP64; the *_f64 entry points take double weights and fields,
+ * accumulate in long double and round to double once per point per step.
  *
  * Every part of this file is pinned by the CPU test-suite against closed
  * forms, invariants, brute force and library routines; nothing here is
@@ -188,6 +190,98 @@ int oracle_stencil_points(int ndim, const int64_t *dims, int radius, const float
         int64_t x = f % nx, y = (f / nx) % ny, z = f / (nx * ny);
         out_values[i] = point_value(in, nz, ny, nx, z, y, x, taps, ntaps, boundary);
     }
+    free(taps);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* FP64 fields (the precision of the paper's case study): same definition,    */
+/* long double accumulation, one rounding to double per point per step.       */
+/* ------------------------------------------------------------------------ */
+typedef struct {
+    int dz, dy, dx;
+    long double w;
+} tapl_t;
+
+static int build_taps_f64(int ndim, int R, const double *weights, tapl_t **taps_out)
+{
+    int side = 2 * R + 1;
+    int total = (ndim == 3) ? side * side * side : side * side;
+    tapl_t *taps = (tapl_t *)malloc(sizeof(tapl_t) * (size_t)total);
+    int n = 0;
+    if (!taps) return -1;
+    for (int f = 0; f < total; ++f) {
+        double w = weights[f];
+        if (w == 0.0) continue;
+        int c = f % side, b = (f / side) % side, a = (ndim == 3) ? f / (side * side) : R;
+        taps[n].dz = a - R; taps[n].dy = b - R; taps[n].dx = c - R;
+        taps[n].w = (long double)w;
+        ++n;
+    }
+    *taps_out = taps;
+    return n;
+}
+
+static inline double point_value_f64(const double *a, int64_t nz, int64_t ny, int64_t nx,
+                                     int64_t z, int64_t y, int64_t x,
+                                     const tapl_t *taps, int ntaps, int boundary)
+{
+    long double acc = 0.0L;
+    for (int t = 0; t < ntaps; ++t) {
+        int64_t qz = z + taps[t].dz, qy = y + taps[t].dy, qx = x + taps[t].dx;
+        if (boundary == ORACLE_PERIODIC) {
+            qz = wrap(qz, nz); qy = wrap(qy, ny); qx = wrap(qx, nx);
+        } else if (qz < 0 || qz >= nz || qy < 0 || qy >= ny || qx < 0 || qx >= nx) {
+            continue;
+        }
+        acc += taps[t].w * (long double)a[(qz * ny + qy) * nx + qx];
+    }
+    return (double)acc;
+}
+
+int oracle_stencil_apply_f64(int ndim, const int64_t *dims, int radius, const double *weights,
+                             int boundary, int steps, const double *in, double *out)
+{
+    if ((ndim != 2 && ndim != 3) || !dims || radius < 1 || !weights || !in || !out || steps < 0)
+        return -1;
+    if (boundary != ORACLE_ZERO && boundary != ORACLE_PERIODIC) return -1;
+    int64_t nz = (ndim == 3) ? dims[0] : 1;
+    int64_t ny = (ndim == 3) ? dims[1] : dims[0];
+    int64_t nx = (ndim == 3) ? dims[2] : dims[1];
+    if (nz < 1 || ny < 1 || nx < 1) return -1;
+    size_t N = (size_t)nz * (size_t)ny * (size_t)nx;
+    if (steps == 0) {
+        memcpy(out, in, N * sizeof(double));
+        return 0;
+    }
+    tapl_t *taps = NULL;
+    int ntaps = build_taps_f64(ndim, radius, weights, &taps);
+    if (ntaps < 0) return -1;
+    double *tmp = NULL;
+    if (steps > 1) {
+        tmp = (double *)malloc(N * sizeof(double));
+        if (!tmp) { free(taps); return -1; }
+    }
+    const double *cur = in;
+    for (int k = 0; k < steps; ++k) {
+        int remaining = steps - 1 - k;
+        double *nxt = (remaining % 2 == 0) ? out : tmp;
+        if (nz > 1) {
+#pragma omp parallel for schedule(static)
+            for (int64_t z = 0; z < nz; ++z)
+                for (int64_t y = 0; y < ny; ++y)
+                    for (int64_t x = 0; x < nx; ++x)
+                        nxt[(z * ny + y) * nx + x] =
+                            point_value_f64(cur, nz, ny, nx, z, y, x, taps, ntaps, boundary);
+        } else {
+#pragma omp parallel for schedule(static)
+            for (int64_t y = 0; y < ny; ++y)
+                for (int64_t x = 0; x < nx; ++x)
+                    nxt[y * nx + x] = point_value_f64(cur, 1, ny, nx, 0, y, x, taps, ntaps, boundary);
+        }
+        cur = nxt;
+    }
+    free(tmp);
     free(taps);
     return 0;
 }

@@ -50,6 +50,10 @@ def _load():
         lib.oracle_stencil_points.restype = ctypes.c_int
         lib.oracle_stencil_points.argtypes = [ctypes.c_int, i64p, ctypes.c_int, f32p,
                                               ctypes.c_int, f32p, ctypes.c_int64, i64p, f32p]
+        f64p = ctypes.POINTER(ctypes.c_double)
+        lib.oracle_stencil_apply_f64.restype = ctypes.c_int
+        lib.oracle_stencil_apply_f64.argtypes = [ctypes.c_int, i64p, ctypes.c_int, f64p,
+                                                 ctypes.c_int, ctypes.c_int, f64p, f64p]
         lib.oracle_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -60,8 +64,8 @@ def num_threads() -> int:
 
 
 def _check(weights: np.ndarray, field: np.ndarray):
-    if field.dtype != np.float32 or weights.dtype != np.float32:
-        raise TypeError("oracle takes float32 weights and float32 fields")
+    if field.dtype != weights.dtype or field.dtype not in (np.float32, np.float64):
+        raise TypeError("oracle takes float32 weights with float32 fields, or float64 with float64")
     ndim = field.ndim
     if ndim not in (2, 3) or weights.ndim != ndim:
         raise ValueError("field and weights must both be 2D or both 3D")
@@ -75,13 +79,24 @@ def _f32p(a: np.ndarray):
     return a.ctypes.data_as(ctypes.POINTER(ctypes.c_float))
 
 
+def _f64p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
 def apply(field: np.ndarray, weights: np.ndarray, boundary: int = ZERO, steps: int = 1) -> np.ndarray:
-    """``steps``-fold sweep of ``field`` with dense ``weights``; returns a new array."""
+    """``steps``-fold sweep of ``field`` with dense ``weights``; returns a new array.
+    float32 arrays use the double-accumulating oracle, float64 arrays the long-double one."""
     field = np.ascontiguousarray(field)
     weights = np.ascontiguousarray(weights)
     ndim, R = _check(weights, field)
     dims = (ctypes.c_int64 * ndim)(*field.shape)
     out = np.empty_like(field)
+    if field.dtype == np.float64:
+        rc = _load().oracle_stencil_apply_f64(ndim, dims, R, _f64p(weights), int(boundary), int(steps),
+                                              _f64p(field), _f64p(out))
+        if rc != 0:
+            raise RuntimeError(f"oracle_stencil_apply_f64 failed ({rc})")
+        return out
     rc = _load().oracle_stencil_apply(ndim, dims, R, _f32p(weights), int(boundary), int(steps),
                                       _f32p(field), _f32p(out))
     if rc != 0:
@@ -95,6 +110,8 @@ def apply_points(field: np.ndarray, weights: np.ndarray, flat_index: np.ndarray,
     field = np.ascontiguousarray(field)
     weights = np.ascontiguousarray(weights)
     ndim, R = _check(weights, field)
+    if field.dtype != np.float32:
+        raise TypeError("apply_points is float32 only")
     idx = np.ascontiguousarray(flat_index, dtype=np.int64)
     dims = (ctypes.c_int64 * ndim)(*field.shape)
     out = np.empty(idx.shape, dtype=np.float32)

@@ -30,7 +30,8 @@ VARIANT_AUTO, VARIANT_GENERIC, VARIANT_STREAM, VARIANT_FUSED = 0, 1, 2, 3
 
 #: every symbol include/stencil.h declares
 EXPORTS = (
-    "stencil_plan", "stencil_apply", "stencil_apply_host", "stencil_apply_static", "stencil_destroy",
+    "stencil_plan", "stencil_apply", "stencil_plan_f64", "stencil_apply_f64",
+    "stencil_apply_host", "stencil_apply_static", "stencil_destroy",
     "stencil_status_string", "stencil_variant_name", "stencil_query_status",
     "stencil_plan_set", "stencil_plan_get",
 )
@@ -60,6 +61,11 @@ def load() -> ctypes.CDLL:
                                  f32p, ctypes.c_int]
     lib.stencil_apply.restype = ctypes.c_int
     lib.stencil_apply.argtypes = [vp, vp, vp, ctypes.c_int, vp]
+    lib.stencil_plan_f64.restype = ctypes.c_int
+    lib.stencil_plan_f64.argtypes = [ctypes.POINTER(vp), ctypes.c_int, i64p, ctypes.c_int, ctypes.c_int,
+                                     ctypes.POINTER(ctypes.c_double), ctypes.c_int]
+    lib.stencil_apply_f64.restype = ctypes.c_int
+    lib.stencil_apply_f64.argtypes = [vp, vp, vp, ctypes.c_int, vp]
     lib.stencil_apply_host.restype = ctypes.c_int
     lib.stencil_apply_host.argtypes = [vp, vp, vp, ctypes.c_int, vp]
     lib.stencil_apply_static.restype = ctypes.c_int
@@ -100,6 +106,23 @@ def stencil_plan(dims: Sequence[int], radius: int, shape: int, weights: np.ndarr
     rc = lib.stencil_plan(ctypes.byref(h), len(dims), d, int(radius), int(shape),
                           w.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), int(boundary))
     return rc, h
+
+
+def stencil_plan_f64(dims: Sequence[int], radius: int, shape: int, weights: np.ndarray, boundary: int):
+    """-> (status, handle) of an FP64 plan.  ``weights``: dense float64 (2R+1)^ndim host array."""
+    lib = load()
+    w = np.ascontiguousarray(weights, dtype=np.float64)
+    d = (ctypes.c_int64 * len(dims))(*[int(v) for v in dims])
+    h = ctypes.c_void_p()
+    rc = lib.stencil_plan_f64(ctypes.byref(h), len(dims), d, int(radius), int(shape),
+                              w.ctypes.data_as(ctypes.POINTER(ctypes.c_double)), int(boundary))
+    return rc, h
+
+
+def stencil_apply_f64(plan, in_ptr: int, out_ptr: int, steps: int, stream: int = 0) -> int:
+    """``in_ptr`` / ``out_ptr``: device addresses of float64 grids."""
+    return load().stencil_apply_f64(plan, ctypes.c_void_p(in_ptr), ctypes.c_void_p(out_ptr), int(steps),
+                                    ctypes.c_void_p(stream))
 
 
 def stencil_apply(plan, in_ptr: int, out_ptr: int, steps: int, stream: int = 0) -> int:
@@ -152,9 +175,10 @@ class Plan:
 
     def __init__(self, dims, radius: int, shape: int, weights: np.ndarray, boundary: int = ZERO,
                  variant: Optional[int] = None, **knobs):
-        rc, h = stencil_plan(dims, radius, shape, weights, boundary)
+        self.f64 = np.asarray(weights).dtype == np.float64     # float64 weights make an FP64 plan
+        rc, h = (stencil_plan_f64 if self.f64 else stencil_plan)(dims, radius, shape, weights, boundary)
         if rc != OK:
-            raise StencilError(rc, "stencil_plan")
+            raise StencilError(rc, "stencil_plan_f64" if self.f64 else "stencil_plan")
         self._h = h
         self.dims = tuple(int(d) for d in dims)
         self.npoints = int(np.prod(self.dims))
@@ -195,9 +219,10 @@ class Plan:
         return int(x.data_ptr()) if hasattr(x, "data_ptr") else int(x)
 
     def apply(self, src, dst, steps: int = 1, stream: int = 0) -> None:
-        rc = stencil_apply(self._h, self._ptr(src), self._ptr(dst), steps, stream)
+        fn = stencil_apply_f64 if self.f64 else stencil_apply
+        rc = fn(self._h, self._ptr(src), self._ptr(dst), steps, stream)
         if rc != OK:
-            raise StencilError(rc, "stencil_apply")
+            raise StencilError(rc, "stencil_apply_f64" if self.f64 else "stencil_apply")
 
     def apply_static(self, src, dst, steps: int = 1, stream: int = 0) -> None:
         rc = stencil_apply_static(self._h, self._ptr(src), self._ptr(dst), steps, stream)

@@ -6,10 +6,15 @@
 namespace stencil {
 
 // One non-zero tap: in[p + (dz,dy,dx)] * w.
-struct Tap {
+template <typename T>
+struct TapT {
     int dz, dy, dx;
-    float w;
+    T w;
 };
+using Tap = TapT<float>;
+
+__device__ __forceinline__ float fma_t(float a, float b, float c) { return fmaf(a, b, c); }
+__device__ __forceinline__ double fma_t(double a, double b, double c) { return fma(a, b, c); }
 
 // Grid extents as the kernels see them; 2D grids have nz == 1.
 struct Grid {

@@ -20,17 +20,18 @@ __device__ __forceinline__ int wrap_index(int q, int n) {
     return q < 0 ? q + n : q;
 }
 
-template <bool kPeriodic>
+// T = float, or double for FP64 plans (the precision of the paper's case study).
+template <bool kPeriodic, typename T = float>
 __global__ void __launch_bounds__(kGenericThreads)
-stencil_generic_kernel(const float* __restrict__ in, float* __restrict__ out, Grid g,
-                       const Tap* __restrict__ taps, int ntaps) {
-    __shared__ Tap s_taps[kGenericSmemTaps];
+stencil_generic_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g,
+                       const TapT<T>* __restrict__ taps, int ntaps) {
+    __shared__ TapT<T> s_taps[kGenericSmemTaps];
     const bool staged = ntaps <= kGenericSmemTaps;
     if (staged) {
         for (int t = threadIdx.x; t < ntaps; t += blockDim.x) s_taps[t] = taps[t];
         __syncthreads();
     }
-    const Tap* tp = staged ? s_taps : taps;
+    const TapT<T>* tp = staged ? s_taps : taps;
 
     const int64_t plane = (int64_t)g.ny * g.nx;
     const int64_t N = plane * g.nz;
@@ -40,9 +41,9 @@ stencil_generic_kernel(const float* __restrict__ in, float* __restrict__ out, Gr
         const int64_t r = i / g.nx;
         const int y = (int)(r % g.ny);
         const int z = (int)(r / g.ny);
-        float acc = 0.0f;
+        T acc = T(0);
         for (int t = 0; t < ntaps; ++t) {
-            const Tap tap = tp[t];
+            const TapT<T> tap = tp[t];
             int qz = z + tap.dz, qy = y + tap.dy, qx = x + tap.dx;
             if (kPeriodic) {
                 qz = wrap_index(qz, g.nz);
@@ -52,7 +53,7 @@ stencil_generic_kernel(const float* __restrict__ in, float* __restrict__ out, Gr
                        (unsigned)qx >= (unsigned)g.nx) {
                 continue;
             }
-            acc = fmaf(tap.w, __ldg(in + (int64_t)qz * plane + (int64_t)qy * g.nx + qx), acc);
+            acc = fma_t(tap.w, __ldg(in + (int64_t)qz * plane + (int64_t)qy * g.nx + qx), acc);
         }
         out[i] = acc;
     }

@@ -19,6 +19,7 @@
 #include "kernel_stream.cuh"
 #include "kernel_fused.cuh"
 #include "kernel_rows2d.cuh"
+#include "kernel_rows2d_f64.cuh"
 
 using namespace stencil;
 
@@ -96,14 +97,31 @@ struct Rows2DConfig {
 
 }  // namespace
 
+struct Rows2D64Config {
+    int radius;
+    bool box;
+    int YB, NW, batch_bytes;
+    const void* kernel;
+    mutable size_t smem_allowed;
+    mutable int cache_device;
+    cudaError_t (*launch)(const struct stencil_plan_s*, const CUtensorMap&, double*, const Rows2DGeom&,
+                          int grid, size_t smem, cudaStream_t);
+};
+
 struct stencil_plan_s {
     uint32_t magic;
     int ndim;
     int nz, ny, nx;
     int64_t npoints;
     int radius, shape, boundary;
+    bool f64;                      // FP64 plan (stencil_plan_f64): only the *_f64 calls accept it
     std::vector<float> w;          // dense (2R+1)^ndim, as given
     std::vector<Tap> taps;         // non-zero taps, dense C order
+    std::vector<double> w64;       // the same for FP64 plans
+    std::vector<TapT<double>> taps64;
+    TapT<double>* d_taps64;
+    double* scratch64;             // N doubles, iteration ping-pong of FP64 plans
+    const struct Rows2D64Config* rows2d64_cfg;
     // device state (created lazily, on the device current at first apply)
     int device;
     Tap* d_taps;
@@ -354,6 +372,14 @@ int ensure_device_state(stencil_plan_s* p) {
     p->device = dev;
     if (cudaMalloc(&p->d_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
     if (cudaMemset(p->d_status, 0, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    const size_t bytes64 = p->taps64.size() * sizeof(TapT<double>);
+    if (bytes64) {
+        if (cudaMalloc(&p->d_taps64, bytes64) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_ALLOC; }
+        if (cudaMemcpy(p->d_taps64, p->taps64.data(), bytes64, cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaGetLastError();
+            return STENCIL_ERR_CUDA;
+        }
+    }
     const size_t bytes = p->taps.size() * sizeof(Tap);
     if (bytes) {
         if (cudaMalloc(&p->d_taps, bytes) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_ALLOC; }
@@ -653,7 +679,217 @@ int launch_sweep(stencil_plan_s* p, const float* src, float* dst, cudaStream_t s
     }
 }
 
+
+// ---------------------------------------------------------------------------
+// FP64 plans: the generic kernel for everything, the row-streaming kernel for
+// 2D grids with a zero boundary (the paper's own case)
+// ---------------------------------------------------------------------------
+inline double dense_w64(const stencil_plan_s* p, int dy, int dx) {
+    const int R = p->radius, side = 2 * R + 1;
+    return p->w64[(size_t)(dy + R) * side + (dx + R)];
+}
+
+template <int R, bool BOX, int YB, int NW>
+cudaError_t launch_rows2d64_t(const stencil_plan_s* p, const CUtensorMap& map, double* out, const Rows2DGeom& g,
+                              int grid, size_t smem, cudaStream_t st) {
+    Weights2D64<R> wt;
+    for (int a = -R; a <= R; ++a)
+        for (int b = -R; b <= R; ++b) wt.w[a + R][b + R] = dense_w64(p, a, b);
+    stencil_rows2d_f64_kernel<R, BOX, YB, NW><<<grid, NW * 32, smem, st>>>(map, out, g, wt, p->d_status);
+    return cudaGetLastError();
+}
+
+template <int R, bool BOX, int YB, int NW>
+Rows2D64Config make_rows2d64() {
+    Rows2D64Config c;
+    c.radius = R; c.box = BOX; c.YB = YB; c.NW = NW; c.batch_bytes = Rows2D64Shape<YB>::BATCH_BYTES;
+    c.kernel = reinterpret_cast<const void*>(&stencil_rows2d_f64_kernel<R, BOX, YB, NW>);
+    c.smem_allowed = 0; c.cache_device = -1;
+    c.launch = &launch_rows2d64_t<R, BOX, YB, NW>;
+    return c;
+}
+
+const std::vector<Rows2D64Config>& rows2d64_configs() {
+    static const std::vector<Rows2D64Config> v = {
+        make_rows2d64<1, false, 8, 8>(), make_rows2d64<2, false, 8, 8>(), make_rows2d64<3, false, 8, 8>(),
+        make_rows2d64<4, false, 8, 8>(),
+        make_rows2d64<1, true, 8, 8>(),  make_rows2d64<2, true, 8, 8>(),  make_rows2d64<3, true, 8, 8>(),
+    };
+    return v;
+}
+
+const Rows2D64Config* find_rows2d64_cfg(const stencil_plan_s* p) {
+    if (p->ndim != 2 || p->boundary != STENCIL_ZERO || p->nx % 2 != 0) return nullptr;   // 16-byte rows
+    for (const Rows2D64Config& c : rows2d64_configs())
+        if (c.radius == p->radius && c.box == (p->shape == STENCIL_BOX)) return &c;
+    return nullptr;
+}
+
+int resolve_variant_f64(stencil_plan_s* p, int want) {
+    const Rows2D64Config* c = find_rows2d64_cfg(p);
+    if (want == STENCIL_VARIANT_AUTO) want = c ? STENCIL_VARIANT_STREAM : STENCIL_VARIANT_GENERIC;
+    if (want == STENCIL_VARIANT_GENERIC) { p->variant = want; p->rows2d64_cfg = nullptr; return STENCIL_OK; }
+    if (want == STENCIL_VARIANT_STREAM && c) { p->variant = want; p->rows2d64_cfg = c; return STENCIL_OK; }
+    return STENCIL_ERR_UNSUPPORTED;
+}
+
+int get_tensor_map_f64(stencil_plan_s* p, const void* cfg, int box_x, int box_y, const double* src,
+                       const CUtensorMap** out) {
+    const float* key = reinterpret_cast<const float*>(src);
+    for (auto& e : p->maps)
+        if (e.ptr == key && e.cfg == cfg) { *out = &e.map; return STENCIL_OK; }
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) return STENCIL_ERR_CUDA;
+    stencil_plan_s::MapEntry e;
+    e.ptr = key; e.cfg = cfg;
+    const cuuint64_t dims[3] = {(cuuint64_t)p->nx, (cuuint64_t)p->ny, (cuuint64_t)p->nz};
+    const cuuint64_t strides[2] = {(cuuint64_t)p->nx * 8, (cuuint64_t)p->nx * (cuuint64_t)p->ny * 8};
+    const cuuint32_t box[3] = {(cuuint32_t)box_x, (cuuint32_t)box_y, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(&e.map, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, 3, const_cast<double*>(src), dims, strides, box,
+                     estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return STENCIL_ERR_CUDA;
+    if (p->maps.size() >= 8) p->maps.erase(p->maps.begin());
+    p->maps.push_back(e);
+    *out = &p->maps.back().map;
+    return STENCIL_OK;
+}
+
+int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStream_t st) {
+    if (p->variant == STENCIL_VARIANT_STREAM && p->rows2d64_cfg) {
+        const Rows2D64Config* cfg = p->rows2d64_cfg;
+        const CUtensorMap* map = nullptr;
+        int rc = get_tensor_map_f64(p, cfg, kPX64, cfg->YB, src, &map);
+        if (rc != STENCIL_OK) return rc;
+        const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
+        const size_t smem = (size_t)cfg->NW * stages * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8;
+        if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+        if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->cache_device = dev; }
+        if (smem > cfg->smem_allowed) {
+            if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess) {
+                cudaGetLastError();
+                return STENCIL_ERR_CUDA;
+            }
+            cfg->smem_allowed = smem;
+        }
+        Rows2DGeom g;
+        g.ny = p->ny; g.nx = p->nx;
+        g.strips = (p->nx + kStrip64 - 1) / kStrip64;
+        g.stages = stages;
+        int chunk = p->chunk_z;
+        if (chunk <= 0) {                             // same sizing rule as the fp32 kernel
+            const int R = p->radius;
+            const int slots = 2 * sm_count() * cfg->NW;
+            const int nch_max = std::max(1, slots / g.strips);
+            const int chunk_min = (p->ny + nch_max - 1) / nch_max;
+            int nbatch = std::max(1, (chunk_min + 2 * R + cfg->YB - 1) / cfg->YB);
+            while (nbatch * cfg->YB - 2 * R < 1) ++nbatch;
+            chunk = nbatch * cfg->YB - 2 * R;
+        }
+        chunk = std::max(1, std::min(chunk, p->ny));
+        g.chunk_y = chunk;
+        g.nchunks = (p->ny + chunk - 1) / chunk;
+        const int64_t units = (int64_t)g.strips * g.nchunks;
+        const int64_t grid64 = (units + cfg->NW - 1) / cfg->NW;
+        if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
+        if (cfg->launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
+        p->launches++;
+        return STENCIL_OK;
+    }
+    Grid g{p->nz, p->ny, p->nx};
+    const int64_t blocks_needed = (p->npoints + kGenericThreads - 1) / kGenericThreads;
+    const int grid = (int)std::min<int64_t>(blocks_needed, 148 * 16);
+    const int ntaps = (int)p->taps64.size();
+    if (p->boundary == STENCIL_PERIODIC)
+        stencil_generic_kernel<true, double><<<grid, kGenericThreads, 0, st>>>(src, dst, g, p->d_taps64, ntaps);
+    else
+        stencil_generic_kernel<false, double><<<grid, kGenericThreads, 0, st>>>(src, dst, g, p->d_taps64, ntaps);
+    if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
+    p->launches++;
+    return STENCIL_OK;
+}
+
 bool valid_plan(const stencil_plan_s* p) { return p && p->magic == kPlanMagic; }
+
+// ---------------------------------------------------------------------------
+// plan construction, shared by the fp32 and the FP64 entry point
+// ---------------------------------------------------------------------------
+template <typename T>
+int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radius, int shape,
+              const T* weights, int boundary) {
+    constexpr bool kF64 = sizeof(T) == 8;
+    if (!plan_out) return STENCIL_ERR_INVALID;
+    *plan_out = nullptr;
+    if ((ndim != 2 && ndim != 3) || !dims || !weights) return STENCIL_ERR_INVALID;
+    if (shape != STENCIL_STAR && shape != STENCIL_BOX) return STENCIL_ERR_INVALID;
+    if (boundary != STENCIL_ZERO && boundary != STENCIL_PERIODIC) return STENCIL_ERR_INVALID;
+    if (radius < 1) return STENCIL_ERR_INVALID;
+    if (radius > kMaxRadius) return STENCIL_ERR_UNSUPPORTED;
+    int64_t n = 1;
+    for (int i = 0; i < ndim; ++i) {
+        if (dims[i] < 1) return STENCIL_ERR_INVALID;
+        if (dims[i] > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
+        if (n > (int64_t)1 << 40) return STENCIL_ERR_UNSUPPORTED;
+        n *= dims[i];
+    }
+
+    stencil_plan_s* p = new (std::nothrow) stencil_plan_s();
+    if (!p) return STENCIL_ERR_ALLOC;
+    p->magic = kPlanMagic;
+    p->f64 = kF64;
+    p->ndim = ndim;
+    p->nz = ndim == 3 ? (int)dims[0] : 1;
+    p->ny = ndim == 3 ? (int)dims[1] : (int)dims[0];
+    p->nx = ndim == 3 ? (int)dims[2] : (int)dims[1];
+    p->npoints = n;
+    p->radius = radius; p->shape = shape; p->boundary = boundary;
+    p->device = -1;
+    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr;
+    p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr;
+    p->host_in = nullptr; p->host_out = nullptr;
+    p->copy_in = nullptr; p->copy_out = nullptr;
+    p->variant = STENCIL_VARIANT_GENERIC;
+    p->tile_y = 0; p->rows_per_thread = 0; p->chunk_z = 0; p->stages = 0; p->fuse_steps = 0; p->streaming_store = 0;
+    p->stream_cfg = nullptr; p->fused_cfg = nullptr; p->rows2d_cfg = nullptr; p->tile_x = 0;
+    p->stream_cfg_fixed = false; p->stream_cfg_tuned = false;
+    p->wait_polls = kWaitPolls; p->drop_plane = -1;
+    p->launches = 0; p->last_stream = nullptr; p->used = false;
+
+    const int side = 2 * radius + 1;
+    size_t count = 1;
+    for (int i = 0; i < ndim; ++i) count *= (size_t)side;
+    try {
+        if constexpr (kF64) p->w64.assign(weights, weights + count);
+        else p->w.assign(weights, weights + count);
+        for (size_t f = 0; f < count; ++f) {
+            const T wv = weights[f];
+            int dx = (int)(f % side) - radius;
+            int dy = (int)((f / side) % side) - radius;
+            int dz = ndim == 3 ? (int)(f / ((size_t)side * side)) - radius : 0;
+            const int nonzero_axes = (dx != 0) + (dy != 0) + (dz != 0);
+            if (shape == STENCIL_STAR && nonzero_axes > 1 && wv != T(0)) {
+                delete p;
+                return STENCIL_ERR_INVALID;       // STAR promises zero off-axis weights
+            }
+            if (wv != T(0)) {
+                if constexpr (kF64) p->taps64.push_back(TapT<double>{dz, dy, dx, wv});
+                else p->taps.push_back(Tap{dz, dy, dx, wv});
+            }
+        }
+    } catch (...) {
+        delete p;
+        return STENCIL_ERR_ALLOC;
+    }
+    if (kF64) resolve_variant_f64(p, STENCIL_VARIANT_AUTO);
+    else resolve_variant(p, STENCIL_VARIANT_AUTO);
+    *plan_out = p;
+    return STENCIL_OK;
+}
+
 
 // ---------------------------------------------------------------------------
 // Fixed scratch for stencil_apply_static: the ping-pong grid and the tap list
@@ -699,69 +935,16 @@ extern "C" {
 
 int stencil_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radius, int shape,
                  const float* weights, int boundary) {
-    if (!plan_out) return STENCIL_ERR_INVALID;
-    *plan_out = nullptr;
-    if ((ndim != 2 && ndim != 3) || !dims || !weights) return STENCIL_ERR_INVALID;
-    if (shape != STENCIL_STAR && shape != STENCIL_BOX) return STENCIL_ERR_INVALID;
-    if (boundary != STENCIL_ZERO && boundary != STENCIL_PERIODIC) return STENCIL_ERR_INVALID;
-    if (radius < 1) return STENCIL_ERR_INVALID;
-    if (radius > kMaxRadius) return STENCIL_ERR_UNSUPPORTED;
-    int64_t n = 1;
-    for (int i = 0; i < ndim; ++i) {
-        if (dims[i] < 1) return STENCIL_ERR_INVALID;
-        if (dims[i] > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
-        if (n > (int64_t)1 << 40) return STENCIL_ERR_UNSUPPORTED;
-        n *= dims[i];
-    }
+    return make_plan<float>(plan_out, ndim, dims, radius, shape, weights, boundary);
+}
 
-    stencil_plan_s* p = new (std::nothrow) stencil_plan_s();
-    if (!p) return STENCIL_ERR_ALLOC;
-    p->magic = kPlanMagic;
-    p->ndim = ndim;
-    p->nz = ndim == 3 ? (int)dims[0] : 1;
-    p->ny = ndim == 3 ? (int)dims[1] : (int)dims[0];
-    p->nx = ndim == 3 ? (int)dims[2] : (int)dims[1];
-    p->npoints = n;
-    p->radius = radius; p->shape = shape; p->boundary = boundary;
-    p->device = -1;
-    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr;
-    p->host_in = nullptr; p->host_out = nullptr;
-    p->copy_in = nullptr; p->copy_out = nullptr;
-    p->variant = STENCIL_VARIANT_GENERIC;
-    p->tile_y = 0; p->rows_per_thread = 0; p->chunk_z = 0; p->stages = 0; p->fuse_steps = 0; p->streaming_store = 0;
-    p->stream_cfg = nullptr; p->fused_cfg = nullptr; p->rows2d_cfg = nullptr; p->tile_x = 0;
-    p->stream_cfg_fixed = false; p->stream_cfg_tuned = false;
-    p->wait_polls = kWaitPolls; p->drop_plane = -1;
-    p->launches = 0; p->last_stream = nullptr; p->used = false;
-
-    const int side = 2 * radius + 1;
-    size_t count = 1;
-    for (int i = 0; i < ndim; ++i) count *= (size_t)side;
-    try {
-        p->w.assign(weights, weights + count);
-        for (size_t f = 0; f < count; ++f) {
-            const float wv = p->w[f];
-            int dx = (int)(f % side) - radius;
-            int dy = (int)((f / side) % side) - radius;
-            int dz = ndim == 3 ? (int)(f / ((size_t)side * side)) - radius : 0;
-            const int nonzero_axes = (dx != 0) + (dy != 0) + (dz != 0);
-            if (shape == STENCIL_STAR && nonzero_axes > 1 && wv != 0.0f) {
-                delete p;
-                return STENCIL_ERR_INVALID;       // STAR promises zero off-axis weights
-            }
-            if (wv != 0.0f) p->taps.push_back(Tap{dz, dy, dx, wv});
-        }
-    } catch (...) {
-        delete p;
-        return STENCIL_ERR_ALLOC;
-    }
-    resolve_variant(p, STENCIL_VARIANT_AUTO);
-    *plan_out = p;
-    return STENCIL_OK;
+int stencil_plan_f64(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radius, int shape,
+                     const double* weights, int boundary) {
+    return make_plan<double>(plan_out, ndim, dims, radius, shape, weights, boundary);
 }
 
 int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void* stream) {
-    if (!valid_plan(p) || !in || !out || steps < 0) return STENCIL_ERR_INVALID;
+    if (!valid_plan(p) || p->f64 || !in || !out || steps < 0) return STENCIL_ERR_INVALID;
     const uintptr_t a = reinterpret_cast<uintptr_t>(in), b = reinterpret_cast<uintptr_t>(out);
     if ((a | b) & 15u) return STENCIL_ERR_INVALID;
     const uintptr_t bytes = (uintptr_t)p->npoints * sizeof(float);
@@ -804,8 +987,44 @@ int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void
     return STENCIL_OK;
 }
 
+int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps, void* stream) {
+    if (!valid_plan(p) || !p->f64 || !in || !out || steps < 0) return STENCIL_ERR_INVALID;
+    const uintptr_t a = reinterpret_cast<uintptr_t>(in), b = reinterpret_cast<uintptr_t>(out);
+    if ((a | b) & 15u) return STENCIL_ERR_INVALID;
+    const uintptr_t bytes = (uintptr_t)p->npoints * sizeof(double);
+    if (a < b + bytes && b < a + bytes) return STENCIL_ERR_INVALID;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int rc = ensure_device_state(p);
+    if (rc != STENCIL_OK) return rc;
+    p->last_stream = st;
+    p->used = true;
+    if (steps == 0) {
+        if (cudaMemcpyAsync(out, in, bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+            cudaGetLastError();
+            return STENCIL_ERR_CUDA;
+        }
+        return STENCIL_OK;
+    }
+    if (steps > 1 && !p->scratch64) {
+        if (cudaMalloc(&p->scratch64, bytes) != cudaSuccess) {
+            cudaGetLastError();
+            p->scratch64 = nullptr;
+            return STENCIL_ERR_ALLOC;
+        }
+    }
+    const double* src = in;
+    for (int k = 0; k < steps; ++k) {
+        const int remaining = steps - 1 - k;
+        double* dst = (remaining % 2 == 0) ? out : p->scratch64;
+        rc = launch_sweep_f64(p, src, dst, st);
+        if (rc != STENCIL_OK) return rc;
+        src = dst;
+    }
+    return STENCIL_OK;
+}
+
 int stencil_apply_host(stencil_plan_t p, const float* in_host, float* out_host, int steps, void* stream) {
-    if (!valid_plan(p) || !in_host || !out_host || steps < 0) return STENCIL_ERR_INVALID;
+    if (!valid_plan(p) || p->f64 || !in_host || !out_host || steps < 0) return STENCIL_ERR_INVALID;
     int rc = ensure_device_state(p);
     if (rc != STENCIL_OK) return rc;
     if ((rc = ensure_grid(&p->host_in, p->npoints)) != STENCIL_OK) return rc;
@@ -879,7 +1098,7 @@ int stencil_apply_host(stencil_plan_t p, const float* in_host, float* out_host, 
 }
 
 int stencil_apply_static(stencil_plan_t p, const float* in, float* out, int steps, void* stream) {
-    if (!valid_plan(p) || !in || !out || steps < 0) return STENCIL_ERR_INVALID;
+    if (!valid_plan(p) || p->f64 || !in || !out || steps < 0) return STENCIL_ERR_INVALID;
     const uintptr_t a = reinterpret_cast<uintptr_t>(in), b = reinterpret_cast<uintptr_t>(out);
     if ((a | b) & 15u) return STENCIL_ERR_INVALID;
     const uintptr_t bytes = (uintptr_t)p->npoints * sizeof(float);
@@ -931,12 +1150,12 @@ int stencil_destroy(stencil_plan_t p) {
     if (!p) return STENCIL_OK;
     if (!valid_plan(p)) return STENCIL_ERR_INVALID;
     int rc = STENCIL_OK;
-    if (p->d_status || p->scratch || p->host_in || p->host_out || p->d_taps) {
+    if (p->d_status || p->scratch || p->host_in || p->host_out || p->d_taps || p->d_taps64 || p->scratch64) {
         int cur = -1;
         cudaGetDevice(&cur);
         if (p->device >= 0 && cur != p->device) cudaSetDevice(p->device);
         if (p->used) cudaStreamSynchronize(p->last_stream);
-        void* ptrs[] = {p->d_status, p->scratch, p->host_in, p->host_out, p->d_taps};
+        void* ptrs[] = {p->d_status, p->scratch, p->host_in, p->host_out, p->d_taps, p->d_taps64, p->scratch64};
         for (void* q : ptrs)
             if (q && cudaFree(q) != cudaSuccess) rc = STENCIL_ERR_CUDA;
         for (cudaEvent_t e : p->events) cudaEventDestroy(e);
@@ -990,6 +1209,7 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
     if (!valid_plan(p)) return STENCIL_ERR_INVALID;
     switch (key) {
         case STENCIL_KEY_VARIANT: {
+            if (p->f64) return resolve_variant_f64(p, (int)value);
             const int old_variant = p->variant;
             const StreamConfig* old_cfg = p->stream_cfg;
             const FusedConfig* old_fused = p->fused_cfg;
@@ -999,6 +1219,7 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
         }
         case STENCIL_KEY_TILE_X:
         case STENCIL_KEY_FUSE_STEPS: {
+            if (p->f64) return value <= 1 ? STENCIL_OK : STENCIL_ERR_UNSUPPORTED;
             // region width (128 or 256) and time steps per pass of the fused kernel
             if (value < 0) return STENCIL_ERR_INVALID;
             const int old_fuse = p->fuse_steps, old_tx = p->tile_x;
@@ -1017,6 +1238,7 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
         case STENCIL_KEY_TILE_Y:
         case STENCIL_KEY_ROWS_PER_THREAD: {
             if (value < 0) return STENCIL_ERR_INVALID;
+            if (p->f64) return value == 0 ? STENCIL_OK : STENCIL_ERR_UNSUPPORTED;
             int ty = key == STENCIL_KEY_TILE_Y ? (int)value : p->tile_y;
             int k = key == STENCIL_KEY_ROWS_PER_THREAD ? (int)value : p->rows_per_thread;
             if (p->variant == STENCIL_VARIANT_STREAM && p->ndim == 2) return value == 0 ? STENCIL_OK : STENCIL_ERR_UNSUPPORTED;
@@ -1075,7 +1297,8 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
         case STENCIL_KEY_LAUNCHES: *value = p->launches; return STENCIL_OK;
         case STENCIL_KEY_SCRATCH_BYTES: {
             int64_t grids = (p->scratch != nullptr) + (p->host_in != nullptr) + (p->host_out != nullptr);
-            *value = grids * p->npoints * (int64_t)sizeof(float);
+            *value = grids * p->npoints * (int64_t)sizeof(float) +
+                     (p->scratch64 ? p->npoints * (int64_t)sizeof(double) : 0);
             return STENCIL_OK;
         }
         case STENCIL_KEY_CHUNK_Z: *value = p->chunk_z; return STENCIL_OK;

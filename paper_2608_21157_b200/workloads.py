@@ -54,16 +54,16 @@ def star_weights(ndim: int, radius: int, center: float, axis_coeffs) -> np.ndarr
     return w.astype(np.float32)
 
 
-def random_box_weights(ndim: int, radius: int, seed: int) -> np.ndarray:
+def random_box_weights(ndim: int, radius: int, seed: int, dtype=np.float32) -> np.ndarray:
     """(2R+1)^ndim weights uniform[-1,1) in dense C order, scaled so that the
-    absolute values sum to one (in float64), then cast to float32."""
+    absolute values sum to one (in float64), then cast to ``dtype``."""
     rng = np.random.default_rng(seed)
     w = rng.uniform(-1.0, 1.0, size=(2 * radius + 1,) * ndim)
     w = w / np.abs(w).sum()
-    return w.astype(np.float32)
+    return w.astype(dtype)
 
 
-def random_star_weights(ndim: int, radius: int, seed: int) -> np.ndarray:
+def random_star_weights(ndim: int, radius: int, seed: int, dtype=np.float32) -> np.ndarray:
     """Asymmetric star: every on-axis tap gets its own uniform[-1,1) value."""
     rng = np.random.default_rng(seed)
     R = radius
@@ -78,7 +78,7 @@ def random_star_weights(ndim: int, radius: int, seed: int) -> np.ndarray:
             idx[ax] += k
             w[tuple(idx)] = rng.uniform(-1.0, 1.0)
     w = w / np.abs(w).sum()
-    return w.astype(np.float32)
+    return w.astype(dtype)
 
 
 #: per-axis coefficients of the 8th-order central second difference
@@ -97,14 +97,14 @@ def fd8_laplacian_weights(ndim: int = 3) -> np.ndarray:
 # --------------------------------------------------------------------------
 # input fields
 # --------------------------------------------------------------------------
-def uniform_field(dims, lo: float, hi: float, seed: int) -> np.ndarray:
+def uniform_field(dims, lo: float, hi: float, seed: int, dtype=np.float32) -> np.ndarray:
     rng = np.random.default_rng(seed)
-    return rng.uniform(lo, hi, size=tuple(dims)).astype(np.float32)
+    return rng.uniform(lo, hi, size=tuple(dims)).astype(dtype)
 
 
-def normal_field(dims, seed: int) -> np.ndarray:
+def normal_field(dims, seed: int, dtype=np.float32) -> np.ndarray:
     rng = np.random.default_rng(seed)
-    return rng.standard_normal(size=tuple(dims)).astype(np.float32)
+    return rng.standard_normal(size=tuple(dims)).astype(dtype)
 
 
 def smooth_sine_field(dims, seed: int, noise: float = 1e-3) -> np.ndarray:
@@ -135,6 +135,11 @@ class Workload:
     steps: int
     make_weights: Callable[[], np.ndarray] = field(repr=False)
     make_input: Callable[[], np.ndarray] = field(repr=False)
+    dtype: type = np.float32          # float32, or float64 (the paper's own precision)
+
+    @property
+    def itemsize(self) -> int:
+        return int(np.dtype(self.dtype).itemsize)
 
     @property
     def ndim(self) -> int:
@@ -152,12 +157,12 @@ class Workload:
         return self.npoints * max(self.steps, 1)
 
     def weights(self) -> np.ndarray:
-        w = np.ascontiguousarray(self.make_weights(), dtype=np.float32)
+        w = np.ascontiguousarray(self.make_weights(), dtype=self.dtype)
         assert w.shape == (2 * self.radius + 1,) * self.ndim
         return w
 
     def input(self) -> np.ndarray:
-        a = np.ascontiguousarray(self.make_input(), dtype=np.float32)
+        a = np.ascontiguousarray(self.make_input(), dtype=self.dtype)
         assert a.shape == tuple(self.dims)
         return a
 
@@ -183,6 +188,7 @@ class Workload:
             steps=self.steps if steps is None else int(steps),
             make_weights=self.make_weights,
             make_input=maker(dims),
+            dtype=self.dtype,
         )
 
 
@@ -235,6 +241,14 @@ def _build_table() -> Dict[str, Workload]:
         lambda: random_box_weights(2, 3, 7),
         _resizable(lambda d: uniform_field(d, -1.0, 1.0, 6), (10240, 10240)))
 
+    # the same in the paper's own precision: FP64 fields and weights (800 MiB per grid)
+    t["paper2d_f64"] = Workload(
+        "paper2d_f64", "2D 49-point box R=3 10240^2 in FP64, random weights sum|w|=1, zero boundary, 16 steps",
+        (10240, 10240), 3, BOX, ZERO, 16,
+        lambda: random_box_weights(2, 3, 7, np.float64),
+        _resizable(lambda d: uniform_field(d, -1.0, 1.0, 6, np.float64), (10240, 10240)),
+        dtype=np.float64)
+
     # supplementary: the iterated heat operator on a grid that does not fit L2
     t["cfg5L"] = Workload(
         "cfg5L", "3D 7-point heat diffusion 512^3, 16 steps (working set exceeds L2)",
@@ -258,6 +272,13 @@ def sha256(a: np.ndarray) -> str:
 
 def tolerance(weights: np.ndarray, max_abs_in: float, steps: int) -> float:
     """Acceptance bound max|gpu - oracle| <= 1e-5 * sum|w| * max|in| * steps + 1e-6
-    (sum in float64 over the float32 weights; steps counted as at least 1)."""
+    (sum in float64 over the float32 weights; steps counted as at least 1).
+
+    For float64 weights (FP64 sweeps) the same form with the constants scaled by the ratio of
+    the unit roundoffs, 2^-53 / 2^-24: 2e-14 * sum|w| * max|in| * steps + 2e-15.  A K-term
+    FMA chain errs by at most about K * 2^-53 * sum|w| * max|in| (5.4e-15 relative for the
+    49-point box), which leaves the same margin as the float32 bound does."""
     sw = float(np.abs(weights.astype(np.float64)).sum())
+    if weights.dtype == np.float64:
+        return 2e-14 * sw * float(max_abs_in) * max(int(steps), 1) + 2e-15
     return 1e-5 * sw * float(max_abs_in) * max(int(steps), 1) + 1e-6

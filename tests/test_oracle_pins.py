@@ -379,3 +379,80 @@ def test_grids_smaller_than_the_stencil():
     cnt_x = [sum(1 for d in range(-3, 4) if (0 + d) % 3 == xx) for xx in range(3)]
     want = sum(a[yy, xx] * cnt_y[yy] * cnt_x[xx] for yy in range(2) for xx in range(3))
     assert oracle.apply(a, w, PERIODIC, 1)[0, 0] == want
+
+
+# ------------------------------------------------ FP64 entry point (long double sums) --
+@pytest.mark.parametrize("name", ["laplace5_3x3", "shift_dx_plus1_3x3", "shift_dz_minus1_2x2x2"])
+def test_f64_hand_worked_examples(name):
+    with open(os.path.join(GOLDEN, name + ".json")) as f:
+        g = json.load(f)
+    got = oracle.apply(np.array(g["in"], dtype=np.float64), np.array(g["weights"], dtype=np.float64), ZERO, 1)
+    assert got.dtype == np.float64
+    assert np.array_equal(got, np.array(g["out"], dtype=np.float64))
+
+
+@pytest.mark.parametrize("ndim,R,boundary", [(2, 3, ZERO), (3, 1, ZERO), (3, 2, PERIODIC)])
+def test_f64_impulse_response(ndim, R, boundary):
+    w = wl.random_box_weights(ndim, R, 21, np.float64)
+    dims = (4 * R + 3, 4 * R + 2, 4 * R + 5)[:ndim]
+    p0 = tuple(d // 2 for d in dims)
+    a = np.zeros(dims)
+    a[p0] = 1.0
+    got = oracle.apply(a, w, boundary, 1)
+    want = np.zeros(dims)
+    for o in np.ndindex(*w.shape):
+        want[tuple(p0[k] - (int(o[k]) - R) for k in range(ndim))] = w[o]
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("dims,R,star,boundary", [
+    ((5, 7), 3, False, ZERO), ((6, 5), 2, False, PERIODIC), ((2, 3), 3, False, ZERO),
+    ((3, 4, 5), 1, False, ZERO), ((4, 3, 6), 2, True, PERIODIC)])
+def test_f64_brute_force_dense_matrix(dims, R, star, boundary):
+    ndim = len(dims)
+    w = (wl.random_star_weights if star else wl.random_box_weights)(ndim, R, 41 + R, np.float64)
+    a = wl.normal_field(dims, 42, np.float64)
+    A = _dense_operator(dims, w, boundary).astype(np.longdouble)
+    want = (A @ a.astype(np.longdouble).ravel()).reshape(dims)
+    got = oracle.apply(a, w, boundary, 1)
+    # long double sums in another order: after the cast to double at most one unit in the last place apart
+    assert np.max(np.abs(got - want.astype(np.float64))) <= np.spacing(np.abs(want).max().astype(np.float64))
+
+
+@pytest.mark.parametrize("dims,R", [((33, 47), 3), ((13, 17, 19), 2)])
+def test_f64_matches_torch_conv_and_scipy(dims, R):
+    import torch
+    import torch.nn.functional as F
+    from scipy import ndimage
+    ndim = len(dims)
+    w = wl.random_box_weights(ndim, R, 51, np.float64)
+    a = wl.normal_field(dims, 52, np.float64)
+    conv = F.conv2d if ndim == 2 else F.conv3d
+    want = conv(torch.from_numpy(a)[None, None], torch.from_numpy(w)[None, None], padding=R)[0, 0].numpy()
+    got = oracle.apply(a, w, ZERO, 1)
+    # the library sums in double: its own rounding error bounds the distance
+    bound = (2 * R + 1) ** ndim * 2.0 ** -52 * np.abs(w).sum() * np.abs(a).max()
+    assert np.max(np.abs(got - want)) <= bound
+    wrap = ndimage.correlate(a, w, mode="wrap")
+    assert np.max(np.abs(oracle.apply(a, w, PERIODIC, 1) - wrap)) <= bound
+
+
+def test_f64_laplacian_quadratic_composition_and_rounding_point():
+    ny, nx = 16, 18
+    y, x = np.meshgrid(np.arange(ny), np.arange(nx), indexing="ij")
+    f = (3 * x * x + 2 * y * y + 5 * x - 7 * y + 11).astype(np.float64)
+    got = oracle.apply(f, wl.star_weights(2, 1, -4.0, [1.0]).astype(np.float64), ZERO, 1)
+    assert np.all(got[1:-1, 1:-1] == 10.0)
+    w = wl.random_box_weights(2, 3, 5, np.float64)
+    a = wl.uniform_field((20, 24), -1.0, 1.0, 6, np.float64)
+    assert np.array_equal(oracle.apply(a, w, ZERO, 5), oracle.apply(oracle.apply(a, w, ZERO, 2), w, ZERO, 3))
+    # 1 + 2^-53 is a tie in double and rounds to 1; the long double sum must round once, at the end
+    w2 = np.zeros((3, 3)); w2[1, 1] = 1.0; w2[1, 2] = 2.0 ** -53
+    b2 = np.zeros((1, 3)); b2[0, 0] = 1.0; b2[0, 1] = 1.0
+    assert oracle.apply(b2, w2, ZERO, 1)[0, 0] == 1.0
+    w2[1, 2] = 2.0 ** -52
+    assert oracle.apply(b2, w2, ZERO, 1)[0, 0] == 1.0 + 2.0 ** -52
+    # and it really carries more than double inside: (1 + 2^-53) + 2^-53 = 1 + 2^-52 exactly
+    w3 = np.zeros((3, 3)); w3[1, 0] = 2.0 ** -53; w3[1, 1] = 1.0; w3[1, 2] = 2.0 ** -53
+    b3 = np.ones((1, 3))
+    assert oracle.apply(b3, w3, ZERO, 1)[0, 1] == 1.0 + 2.0 ** -52

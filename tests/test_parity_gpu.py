@@ -30,7 +30,7 @@ def gpu_sweep(dims, R, shape, weights, boundary, a, steps=1, variant=None, repea
     n = int(np.prod(dims))
     src = torch.from_numpy(a).to(dev)
     src_copy = src.clone()
-    buf = torch.full((n + 2 * GUARD,), float("nan"), dtype=torch.float32, device=dev)
+    buf = torch.full((n + 2 * GUARD,), float("nan"), dtype=src.dtype, device=dev)
     buf[:GUARD] = 12345.0
     buf[GUARD + n:] = 12345.0
     dst = buf[GUARD:GUARD + n]
@@ -308,6 +308,59 @@ def test_fuse_knob_rules():
         assert p.get(b.KEY_FUSE_STEPS) == 1         # no fused kernel for box stencils
         with pytest.raises(b.StencilError):
             p.set(b.KEY_VARIANT, b.VARIANT_FUSED)
+
+
+# --------------------------------------------------------------------- FP64 --
+def check_f64(dims, R, shape, w, boundary, a, steps=1, **kw):
+    assert a.dtype == np.float64 and w.dtype == np.float64
+    got, used = gpu_sweep(dims, R, shape, w, boundary, a, steps, **kw)
+    assert got.dtype == np.float64
+    want = oracle.apply(a, w, boundary, steps)
+    tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+    err = float(np.max(np.abs(got - want)))
+    assert err <= tol, f"{used}: max err {err:.3e} > tol {tol:.3e} for dims={dims} R={R} steps={steps}"
+    return used
+
+
+@pytest.mark.parametrize("R,box", [(1, False), (2, False), (3, False), (4, False), (1, True), (2, True), (3, True)])
+@pytest.mark.parametrize("dims,chunk,stages", [
+    ((67, 66), 0, 0),            # two 64-column strips, the second 2 columns wide
+    ((200, 258), 37, 2),         # several chunks of rows, chunk not a multiple of the batch
+    ((3, 8), 0, 0),              # smaller than the stencil reach
+    ((129, 512), 16, 4),
+])
+def test_f64_rows2d_kernel_matches_oracle(R, box, dims, chunk, stages):
+    mk = wl.random_box_weights if box else wl.random_star_weights
+    w = mk(2, R, 81, np.float64)
+    a = wl.normal_field(dims, 82, np.float64)
+    used = check_f64(dims, R, b.BOX if box else b.STAR, w, b.ZERO, a, chunk_z=chunk or None, stages=stages or None)
+    assert used == "stream"
+
+
+@pytest.mark.parametrize("dims,R,box,boundary", [
+    ((33, 47), 3, True, b.ZERO), ((20, 30), 2, True, b.PERIODIC), ((9, 12, 20), 1, True, b.ZERO),
+    ((7, 10, 14), 2, False, b.PERIODIC), ((40, 64), 5, True, b.ZERO)])
+def test_f64_generic_kernel(dims, R, box, boundary):
+    ndim = len(dims)
+    w = (wl.random_box_weights if box else wl.random_star_weights)(ndim, R, 83, np.float64)
+    a = wl.normal_field(dims, 84, np.float64)
+    used = check_f64(dims, R, b.BOX if box else b.STAR, w, boundary, a, steps=3)
+    assert used == "generic"
+
+
+def test_f64_paper_shaped_box_iterated_and_type_checks():
+    """The paper's operator in its own precision: 2D box radius 3, FP64, iterated."""
+    wk = wl.get("paper2d_f64").scaled((768, 1024), steps=3)
+    a, w = wk.input(), wk.weights()
+    assert check_f64(wk.dims, wk.radius, wk.shape, w, wk.boundary, a, wk.steps) == "stream"
+    # a plan only serves the apply call of its own precision
+    src = torch.zeros(64, 64, dtype=torch.float64, device="cuda")
+    dst = torch.zeros_like(src)
+    with b.Plan((64, 64), 3, b.BOX, wl.random_box_weights(2, 3, 1, np.float64), b.ZERO) as p:
+        assert b.stencil_apply(p._h, src.data_ptr(), dst.data_ptr(), 1, 0) == b.ERR_INVALID
+        assert b.stencil_apply_host(p._h, src.data_ptr(), dst.data_ptr(), 1, 0) == b.ERR_INVALID
+    with b.Plan((64, 64), 3, b.BOX, wl.random_box_weights(2, 3, 1), b.ZERO) as p:
+        assert b.stencil_apply_f64(p._h, src.data_ptr(), dst.data_ptr(), 1, 0) == b.ERR_INVALID
 
 
 # ------------------------------------------------------------ bounded waits --
