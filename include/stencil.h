@@ -79,6 +79,10 @@ enum {
     STENCIL_KEY_ROWS_PER_THREAD = 9, /* set/get: tile rows each thread computes (0 = default)    */
     STENCIL_KEY_WAIT_POLLS   = 10, /* set/get: polls after which a device-side wait of the 3D
                                       single-step kernel gives up (each poll sleeps <= 20 us)    */
+    STENCIL_KEY_CHAIN_LAUNCHES = 12, /* set/get: 1 (default) = launches 2..n of an iterated apply are
+                                      programmatic dependent launches: each begins its preamble
+                                      while its predecessor drains and waits for it before it
+                                      touches global memory; 0 = ordinary launches             */
     STENCIL_KEY_TEST_DROP_PLANE = 11 /* set/get, test hook: every CTA of the 3D single-step kernel
                                       never loads its input plane of this index, so the bounded
                                       wait for it expires and stencil_query_status reports

@@ -92,6 +92,8 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
         fence_barrier_init();
     }
     __syncthreads();
+    allow_dependents();
+    dependency_wait();           // the input is the output of the previous pass
 
     const int bid = blockIdx.x;
     const int tix = bid % g.tiles_x;

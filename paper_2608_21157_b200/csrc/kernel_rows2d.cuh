@@ -61,6 +61,8 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
         fence_barrier_init();
     }
     __syncwarp();
+    allow_dependents();
+    dependency_wait();           // the input may be the output of the previous launch of an iteration
 
     const int unit = blockIdx.x * NW + warp;
     if (unit >= g.strips * g.nchunks) return;           // warps are independent: no barrier follows

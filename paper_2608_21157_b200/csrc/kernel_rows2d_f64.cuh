@@ -51,6 +51,8 @@ stencil_rows2d_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
         fence_barrier_init();
     }
     __syncwarp();
+    allow_dependents();
+    dependency_wait();           // the input may be the output of the previous launch of an iteration
 
     const int unit = blockIdx.x * NW + warp;
     if (unit >= g.strips * g.nchunks) return;

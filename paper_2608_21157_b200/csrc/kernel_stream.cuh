@@ -163,6 +163,8 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
         fence_barrier_init();
     }
     __syncthreads();
+    allow_dependents();
+    dependency_wait();           // the input may be the output of the previous launch of an iteration
 
     // tile and z range of this CTA; x-y tiles vary fastest so that neighbours
     // (which share halo rows) are resident together and hit in L2

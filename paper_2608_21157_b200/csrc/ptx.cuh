@@ -79,6 +79,19 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// Programmatic dependent launch.  A kernel launched with the "programmatic stream
+// serialization" attribute may start while the previous kernel of the stream is still
+// draining; dependency_wait() then blocks until that kernel has completed and its writes
+// are visible.  Everything a kernel reads from or writes to global memory must come after
+// it.  allow_dependents() lets the next kernel of the stream begin its own preamble early.
+// Both are no-ops in a kernel launched the ordinary way.
+__device__ __forceinline__ void dependency_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void allow_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }

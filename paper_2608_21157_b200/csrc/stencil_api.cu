@@ -12,6 +12,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "common.cuh"
@@ -51,6 +52,28 @@ EncodeTiledFn get_encode_fn() {
             cudaGetLastError();
     }
     return fn;
+}
+
+// Kernel launch; `chained` marks a launch that follows another launch of this library on
+// the same stream inside one iterated apply: it may then begin its preamble while the
+// previous kernel drains (programmatic dependent launch; the kernels wait for their
+// predecessor before they touch global memory).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t st,
+                          bool chained, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (chained) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 // ---------------------------------------------------------------------------
@@ -134,6 +157,8 @@ struct stencil_plan_s {
     // selection and tuning
     int variant;                   // resolved STENCIL_VARIANT_*
     int tile_y, rows_per_thread, chunk_z, stages, fuse_steps, streaming_store;
+    bool chain_launches;           // knob: launches 2..n of an iterated apply start early (see launch_kernel)
+    bool chained;                  // set by the apply loop for those launches
     unsigned wait_polls;           // cap of the bounded device waits (single-step 3D kernel)
     int drop_plane;                // test hook, -1 = off
     const StreamConfig* stream_cfg;
@@ -183,9 +208,8 @@ cudaError_t launch_stream_t(const stencil_plan_s* p, const StreamConfig&, const 
             for (int b = -RB; b <= RB; ++b)
                 for (int c = -RB; c <= RB; ++c) bw.w[a + RB][b + RB][c + RB] = dense_w(p, a, b, c);
     }
-    stencil_stream_kernel<R, BOX, K, NW, MINB>
-        <<<grid, StreamShape<R, K, NW>::THREADS, smem, st>>>(map, out, g, sw, bw, p->d_status);
-    return cudaGetLastError();
+    return launch_kernel(&stencil_stream_kernel<R, BOX, K, NW, MINB>, grid, StreamShape<R, K, NW>::THREADS, smem,
+                         st, p->chained, map, out, g, sw, bw, p->d_status);
 }
 
 template <int R, bool BOX, int K, int NW, int MINB>
@@ -246,9 +270,8 @@ cudaError_t launch_fused_t(const stencil_plan_s* p, const CUtensorMap& map, floa
                            int grid, size_t smem, cudaStream_t st) {
     StarWeights<R> sw;
     pack_star<R>(p, sw);
-    stencil_fused_kernel<R, T, K, XW, NWY>
-        <<<grid, FusedShape<R, K, XW, NWY>::THREADS, smem, st>>>(map, out, g, sw, p->d_status);
-    return cudaGetLastError();
+    return launch_kernel(&stencil_fused_kernel<R, T, K, XW, NWY>, grid, FusedShape<R, K, XW, NWY>::THREADS, smem,
+                         st, p->chained, map, out, g, sw, p->d_status);
 }
 
 template <int R, int T, int K, int XW, int NWY>
@@ -284,8 +307,8 @@ cudaError_t launch_rows2d_t(const stencil_plan_s* p, const CUtensorMap& map, flo
     Weights2D<R> wt;
     for (int a = -R; a <= R; ++a)
         for (int b = -R; b <= R; ++b) wt.w[a + R][b + R] = dense_w(p, 0, a, b);
-    stencil_rows2d_kernel<R, BOX, YB, NW><<<grid, NW * 32, smem, st>>>(map, out, g, wt, p->d_status);
-    return cudaGetLastError();
+    return launch_kernel(&stencil_rows2d_kernel<R, BOX, YB, NW>, grid, NW * 32, smem, st, p->chained, map, out, g,
+                         wt, p->d_status);
 }
 
 template <int R, bool BOX, int YB, int NW>
@@ -695,8 +718,8 @@ cudaError_t launch_rows2d64_t(const stencil_plan_s* p, const CUtensorMap& map, d
     Weights2D64<R> wt;
     for (int a = -R; a <= R; ++a)
         for (int b = -R; b <= R; ++b) wt.w[a + R][b + R] = dense_w64(p, a, b);
-    stencil_rows2d_f64_kernel<R, BOX, YB, NW><<<grid, NW * 32, smem, st>>>(map, out, g, wt, p->d_status);
-    return cudaGetLastError();
+    return launch_kernel(&stencil_rows2d_f64_kernel<R, BOX, YB, NW>, grid, NW * 32, smem, st, p->chained, map, out,
+                         g, wt, p->d_status);
 }
 
 template <int R, bool BOX, int YB, int NW>
@@ -857,6 +880,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->stream_cfg = nullptr; p->fused_cfg = nullptr; p->rows2d_cfg = nullptr; p->tile_x = 0;
     p->stream_cfg_fixed = false; p->stream_cfg_tuned = false;
     p->wait_polls = kWaitPolls; p->drop_plane = -1;
+    p->chain_launches = true; p->chained = false;
     p->launches = 0; p->last_stream = nullptr; p->used = false;
 
     const int side = 2 * radius + 1;
@@ -979,7 +1003,9 @@ int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void
         const int remaining = passes - 1 - k;
         float* dst = (remaining % 2 == 0) ? out : p->scratch;
         const int nlev = std::min(T, steps - done);
+        p->chained = p->chain_launches && k > 0;
         rc = (fuse && nlev > 1) ? launch_fused(p, src, dst, nlev, st) : launch_sweep(p, src, dst, st);
+        p->chained = false;
         if (rc != STENCIL_OK) return rc;
         done += nlev;
         src = dst;
@@ -1016,7 +1042,9 @@ int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps
     for (int k = 0; k < steps; ++k) {
         const int remaining = steps - 1 - k;
         double* dst = (remaining % 2 == 0) ? out : p->scratch64;
+        p->chained = p->chain_launches && k > 0;
         rc = launch_sweep_f64(p, src, dst, st);
+        p->chained = false;
         if (rc != STENCIL_OK) return rc;
         src = dst;
     }
@@ -1264,6 +1292,9 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
         case STENCIL_KEY_STREAMING_STORE:
             p->streaming_store = value ? 1 : 0;
             return STENCIL_OK;
+        case STENCIL_KEY_CHAIN_LAUNCHES:
+            p->chain_launches = value != 0;
+            return STENCIL_OK;
         case STENCIL_KEY_WAIT_POLLS:
             if (value < 1 || value > (int64_t)kWaitPolls) return STENCIL_ERR_INVALID;
             p->wait_polls = (unsigned)value;
@@ -1304,6 +1335,7 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
         case STENCIL_KEY_CHUNK_Z: *value = p->chunk_z; return STENCIL_OK;
         case STENCIL_KEY_STAGES: *value = p->stages; return STENCIL_OK;
         case STENCIL_KEY_STREAMING_STORE: *value = p->streaming_store; return STENCIL_OK;
+        case STENCIL_KEY_CHAIN_LAUNCHES: *value = p->chain_launches ? 1 : 0; return STENCIL_OK;
         case STENCIL_KEY_WAIT_POLLS: *value = p->wait_polls; return STENCIL_OK;
         case STENCIL_KEY_TEST_DROP_PLANE: *value = p->drop_plane; return STENCIL_OK;
         default: return STENCIL_ERR_INVALID;
