@@ -73,8 +73,15 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), int grid, int block, size_t 
         cfg.attrs = attr;
         cfg.numAttrs = 1;
     }
-    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+    if (err != cudaSuccess) cudaGetLastError();      // leave no stale error behind for the caller
+    return err;
 }
+
+// The configuration tables below are shared by all plans and cache per-device facts
+// (occupancy, the shared-memory limit already granted to a kernel); this lock makes those
+// caches safe when several host threads drive their own plans.
+std::mutex g_config_mutex;
 
 // ---------------------------------------------------------------------------
 // STREAM kernel configurations
@@ -483,6 +490,7 @@ size_t stream_smem_bytes(const StreamConfig* cfg, int stages) {
 int stream_occupancy(const StreamConfig* cfg, int stages) {
     const size_t smem = stream_smem_bytes(cfg, stages);
     if (smem > 227 * 1024) return -1;
+    std::lock_guard<std::mutex> lock(g_config_mutex);
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return -1; }
     if (dev != cfg->cache_device) {                // function attributes are per device
@@ -607,13 +615,17 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
-    if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->cache_device = dev; }
-    if (smem > cfg->smem_allowed) {
-        if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
-            cudaGetLastError();
-            return STENCIL_ERR_CUDA;
+    {
+        std::lock_guard<std::mutex> lock(g_config_mutex);
+        if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->cache_device = dev; }
+        if (smem > cfg->smem_allowed) {
+            if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess) {
+                cudaGetLastError();
+                return STENCIL_ERR_CUDA;
+            }
+            cfg->smem_allowed = smem;
         }
-        cfg->smem_allowed = smem;
     }
     Rows2DGeom g;
     g.ny = p->ny; g.nx = p->nx;
@@ -790,14 +802,17 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
         int dev = -1;
         if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
-        if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->cache_device = dev; }
-        if (smem > cfg->smem_allowed) {
-            if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess) {
-                cudaGetLastError();
-                return STENCIL_ERR_CUDA;
+        {
+            std::lock_guard<std::mutex> lock(g_config_mutex);
+            if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->cache_device = dev; }
+            if (smem > cfg->smem_allowed) {
+                if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                    cudaSuccess) {
+                    cudaGetLastError();
+                    return STENCIL_ERR_CUDA;
+                }
+                cfg->smem_allowed = smem;
             }
-            cfg->smem_allowed = smem;
         }
         Rows2DGeom g;
         g.ny = p->ny; g.nx = p->nx;

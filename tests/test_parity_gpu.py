@@ -310,6 +310,26 @@ def test_fuse_knob_rules():
             p.set(b.KEY_VARIANT, b.VARIANT_FUSED)
 
 
+# ------------------------------------------------------ sharded sweep, one rank --
+def test_sharded_sweep_single_rank_on_gpu():
+    """World size 1 of the slab decomposition runs the real kernels: ghost planes stay zero
+    and the result is the plain iterated sweep."""
+    from paper_2608_21157_b200.sharded import ShardedSweep
+    dims = (40, 48, 128)
+    w = wl.star_weights(3, 1, 0.4, [0.1])
+    a = wl.uniform_field(dims, 0.0, 1.0, 95)
+    sw = ShardedSweep(dims, 1, b.STAR, w, rank=0, world=1)
+    try:
+        ext = sw.scatter(torch.from_numpy(a).cuda())
+        res = sw.apply(ext, 5)
+        torch.cuda.synchronize()
+        got = sw.interior(res).cpu().numpy()
+    finally:
+        sw.close()
+    want = oracle.apply(a, w, b.ZERO, 5)
+    assert np.max(np.abs(got - want)) <= wl.tolerance(w, 1.0, 5)
+
+
 # --------------------------------------------------------------------- FP64 --
 def check_f64(dims, R, shape, w, boundary, a, steps=1, **kw):
     assert a.dtype == np.float64 and w.dtype == np.float64
