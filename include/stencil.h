@@ -83,6 +83,7 @@ enum {
                                       programmatic dependent launches: each begins its preamble
                                       while its predecessor drains and waits for it before it
                                       touches global memory; 0 = ordinary launches             */
+    STENCIL_KEY_FUSED_TILE_Y = 13,   /* set/get: region height of fused passes, 16 or 32 (0 = auto) */
     STENCIL_KEY_TEST_DROP_PLANE = 11 /* set/get, test hook: every CTA of the 3D single-step kernel
                                       never loads its input plane of this index, so the bounded
                                       wait for it expires and stencil_query_status reports

@@ -248,26 +248,28 @@ def test_paper_shaped_2d_box_radius3():
 
 
 # -------------------------------------------------------------------- fused --
-FUSED_CONFIGS = [   # (radius, fuse_steps, region width)
-    (1, 2, 256), (1, 3, 256), (1, 4, 128), (1, 2, 128), (1, 3, 128), (2, 2, 128),
+FUSED_CONFIGS = [   # (radius, fuse_steps, region width, region height)
+    (1, 2, 256, 32), (1, 2, 256, 16), (1, 3, 256, 32), (1, 4, 128, 32), (1, 2, 128, 32), (1, 3, 128, 32),
+    (2, 2, 128, 32),
 ]
 
 
-@pytest.mark.parametrize("R,T,width", FUSED_CONFIGS)
+@pytest.mark.parametrize("R,T,width,height", FUSED_CONFIGS)
 @pytest.mark.parametrize("dims,chunk_z", [
     ((29, 70, 300), 11),        # several regions in x and y, ragged everywhere, several z chunks
     ((40, 64, 256), 0),         # a 256-wide region spans the whole row
     ((5, 9, 12), 0),            # much smaller than one region
 ])
-def test_fused_passes_match_oracle(R, T, width, dims, chunk_z):
+def test_fused_passes_match_oracle(R, T, width, height, dims, chunk_z):
     w = wl.random_star_weights(3, R, 61)            # asymmetric taps, sum|w| = 1
     a = wl.normal_field(dims, 62)
     for steps in (T, T + 1, 2 * T + 1):
         dev = torch.device("cuda:0")
         src = torch.from_numpy(a).to(dev)
         dst = torch.full_like(src, float("nan"))
-        with b.Plan(dims, R, b.STAR, w, b.ZERO, fuse_steps=T, tile_x=width, chunk_z=chunk_z or None) as p:
-            assert p.get(b.KEY_FUSE_STEPS) == T
+        with b.Plan(dims, R, b.STAR, w, b.ZERO, fuse_steps=T, tile_x=width, fused_tile_y=height,
+                    chunk_z=chunk_z or None) as p:
+            assert p.get(b.KEY_FUSE_STEPS) == T and p.get(b.KEY_FUSED_TILE_Y) == height
             p.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
             assert p.query_status() == b.OK
             assert p.launches == -(-steps // T)
