@@ -107,6 +107,10 @@ struct FusedConfig {
     int radius, T, K, XW, NWY;
     int txe, tye, threads, slot_bytes;
     const void* kernel;
+    mutable size_t smem_allowed;             // dynamic shared memory already granted to the kernel
+    mutable size_t occ_smem;                 // ... and the occupancy measured at this size
+    mutable int occ;
+    mutable int cache_device;
     cudaError_t (*launch)(const struct stencil_plan_s*, const CUtensorMap&, float*, const FusedGeom&,
                           int grid, size_t smem, cudaStream_t);
 };
@@ -180,7 +184,7 @@ struct stencil_plan_s {
     cudaStream_t last_stream;
     bool used;
     // tensor-map cache: one entry per source pointer
-    struct MapEntry { const float* ptr; const void* cfg; CUtensorMap map; };
+    struct MapEntry { const void* ptr; const void* cfg; CUtensorMap map; };
     std::vector<MapEntry> maps;
 };
 
@@ -289,6 +293,7 @@ FusedConfig make_fused() {
     c.radius = R; c.T = T; c.K = K; c.XW = XW; c.NWY = NWY;
     c.txe = S::TXE; c.tye = S::TYE; c.threads = S::THREADS; c.slot_bytes = S::SLOT_BYTES;
     c.kernel = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY>);
+    c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
     c.launch = &launch_fused_t<R, T, K, XW, NWY>;
     return c;
 }
@@ -406,25 +411,34 @@ int ensure_device_state(stencil_plan_s* p) {
     if (p->d_status) return STENCIL_OK;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
-    p->device = dev;
-    if (cudaMalloc(&p->d_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
-    if (cudaMemset(p->d_status, 0, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
-    const size_t bytes64 = p->taps64.size() * sizeof(TapT<double>);
-    if (bytes64) {
-        if (cudaMalloc(&p->d_taps64, bytes64) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_ALLOC; }
-        if (cudaMemcpy(p->d_taps64, p->taps64.data(), bytes64, cudaMemcpyHostToDevice) != cudaSuccess) {
-            cudaGetLastError();
-            return STENCIL_ERR_CUDA;
-        }
-    }
+    int* status = nullptr;
+    Tap* taps = nullptr;
+    TapT<double>* taps64 = nullptr;
     const size_t bytes = p->taps.size() * sizeof(Tap);
-    if (bytes) {
-        if (cudaMalloc(&p->d_taps, bytes) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_ALLOC; }
-        if (cudaMemcpy(p->d_taps, p->taps.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
-            cudaGetLastError();
-            return STENCIL_ERR_CUDA;
-        }
+    const size_t bytes64 = p->taps64.size() * sizeof(TapT<double>);
+    int rc = STENCIL_OK;
+    if (cudaMalloc(&status, sizeof(int)) != cudaSuccess) rc = STENCIL_ERR_ALLOC;
+    if (rc == STENCIL_OK && cudaMemset(status, 0, sizeof(int)) != cudaSuccess) rc = STENCIL_ERR_CUDA;
+    if (rc == STENCIL_OK && bytes && cudaMalloc(&taps, bytes) != cudaSuccess) rc = STENCIL_ERR_ALLOC;
+    if (rc == STENCIL_OK && bytes &&
+        cudaMemcpy(taps, p->taps.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess)
+        rc = STENCIL_ERR_CUDA;
+    if (rc == STENCIL_OK && bytes64 && cudaMalloc(&taps64, bytes64) != cudaSuccess) rc = STENCIL_ERR_ALLOC;
+    if (rc == STENCIL_OK && bytes64 &&
+        cudaMemcpy(taps64, p->taps64.data(), bytes64, cudaMemcpyHostToDevice) != cudaSuccess)
+        rc = STENCIL_ERR_CUDA;
+    if (rc != STENCIL_OK) {                         // all or nothing: a later call starts afresh
+        cudaGetLastError();
+        if (status) cudaFree(status);
+        if (taps) cudaFree(taps);
+        if (taps64) cudaFree(taps64);
+        cudaGetLastError();
+        return rc;
     }
+    p->device = dev;
+    p->d_status = status;
+    p->d_taps = taps;
+    p->d_taps64 = taps64;
     return STENCIL_OK;
 }
 
@@ -441,10 +455,12 @@ int ensure_grid(float** slot, int64_t npoints) {
 // ---------------------------------------------------------------------------
 // launches
 // ---------------------------------------------------------------------------
+int sm_count();
+
 int launch_generic(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
     Grid g{p->nz, p->ny, p->nx};
     const int64_t blocks_needed = (p->npoints + kGenericThreads - 1) / kGenericThreads;
-    const int grid = (int)std::min<int64_t>(blocks_needed, 148 * 16);
+    const int grid = (int)std::min<int64_t>(blocks_needed, (int64_t)sm_count() * 16);
     const int ntaps = (int)p->taps.size();
     if (p->boundary == STENCIL_PERIODIC)
         stencil_generic_kernel<true><<<grid, kGenericThreads, 0, st>>>(src, dst, g, p->d_taps, ntaps);
@@ -692,17 +708,36 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
     if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
     g.stages = stages;
     const int tiles = g.tiles_x * g.tiles_y;
+    int occ = 1;
+    {
+        // shared-memory limit and occupancy of the kernel, asked once per device and size
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+        std::lock_guard<std::mutex> lock(g_config_mutex);
+        if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->occ_smem = 0; cfg->cache_device = dev; }
+        if (smem > cfg->smem_allowed) {
+            if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess) {
+                cudaGetLastError();
+                return STENCIL_ERR_CUDA;
+            }
+            cfg->smem_allowed = smem;
+        }
+        if (cfg->occ_smem != smem) {
+            int o = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, cfg->kernel, cfg->threads, smem) != cudaSuccess) {
+                cudaGetLastError();
+                o = 0;
+            }
+            cfg->occ = std::max(o, 1);
+            cfg->occ_smem = smem;
+        }
+        occ = cfg->occ;
+    }
     int chunk = p->chunk_z;
     if (chunk <= 0) {
         // as many z chunks as fill the resident-CTA slots of the machine once, but not so short
         // that the 2*T*R extra input planes per chunk dominate
-        int occ = 1;
-        if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, cfg->kernel, cfg->threads, smem) != cudaSuccess ||
-            occ < 1) {
-            cudaGetLastError();
-            occ = 1;
-        }
         int nchunks = std::max(1, occ * sm_count() / std::max(tiles, 1));
         nchunks = std::min(nchunks, std::max(1, p->nz / (4 * T * R)));
         chunk = (p->nz + nchunks - 1) / nchunks;
@@ -711,10 +746,6 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
     g.chunk_z = chunk;
     const int64_t grid64 = (int64_t)tiles * ((p->nz + chunk - 1) / chunk);
     if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
-        cudaGetLastError();
-        return STENCIL_ERR_CUDA;
-    }
     if (cfg->launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
     p->launches++;
     return STENCIL_OK;
@@ -784,7 +815,7 @@ int resolve_variant_f64(stencil_plan_s* p, int want) {
 
 int get_tensor_map_f64(stencil_plan_s* p, const void* cfg, int box_x, int box_y, const double* src,
                        const CUtensorMap** out) {
-    const float* key = reinterpret_cast<const float*>(src);
+    const void* key = src;
     for (auto& e : p->maps)
         if (e.ptr == key && e.cfg == cfg) { *out = &e.map; return STENCIL_OK; }
     EncodeTiledFn enc = get_encode_fn();
