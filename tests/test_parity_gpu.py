@@ -430,6 +430,17 @@ def test_baseline_config_full_size(name):
         assert got.min() >= 0.0 and got.max() <= a.max()
 
 
+def test_paper_workload_full_grid_one_step():
+    """The paper's grid at full size (10240 x 10240, 49-point box), one time step, every
+    point against the oracle, in the launch configuration the benchmark times."""
+    wk = wl.get("paper2d")
+    a, w = wk.input(), wk.weights()
+    got, used = gpu_sweep(wk.dims, wk.radius, wk.shape, w, wk.boundary, a, 1)
+    assert used == "stream"
+    want = oracle.apply(a, w, wk.boundary, 1)
+    assert float(np.max(np.abs(got - want))) <= wl.tolerance(w, float(np.abs(a).max()), 1)
+
+
 def test_generic_kernel_on_a_full_3d_config():
     wk = wl.get("cfg2").scaled((128, 128, 128))
     a, w = wk.input(), wk.weights()
