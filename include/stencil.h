@@ -142,8 +142,9 @@ STENCIL_API int stencil_apply(stencil_plan_t plan, const float* in, float* out, 
  * multiples for the tiled kernel: nx even).  A plan made by one of the two
  * plan calls is only accepted by the matching apply call (STENCIL_ERR_INVALID
  * otherwise); stencil_destroy, stencil_query_status and the knobs serve both.
- * 2D grids with a zero boundary and radius <= 4 (box: <= 3) run on a TMA
- * row-streaming kernel; everything else on the one-thread-per-point kernel.
+ * Grids with a zero boundary and an even nx run on TMA-staged kernels (2D:
+ * star radius <= 4, box <= 3; 3D: star radius <= 4, box radius 1); everything
+ * else on the one-thread-per-point kernel.
  */
 STENCIL_API int stencil_plan_f64(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radius,
                                  int shape, const double* weights, int boundary);

@@ -1,0 +1,263 @@
+// STREAM kernel for FP64 grids: 3D sweep with a zero boundary, the double-precision twin
+// of the fp32 plane-streaming kernel (same CTA layout, same TMA ring with a producer warp,
+// same in-place register accumulators along z).
+//
+// Differences: a lane owns one double2 (two points), so a tile is 64 columns wide; the x
+// neighbourhood of a lane is read from shared memory as aligned double2 loads instead of
+// being exchanged by shuffles.  At 16 B per point the sweep is bound by HBM for every
+// stencil the kernel covers (star radius <= 4: 25 DFMA per point at most; box radius 1:
+// 27), since the FP64 pipe sustains 64 DFMA per clock per SM.
+#pragma once
+#include "common.cuh"
+#include "kernel_stream.cuh"
+#include "ptx.cuh"
+
+namespace stencil {
+
+constexpr int kStream64TX = 64;                  // tile width in points
+constexpr int kStream64PX = kStream64TX + 8;     // + 4 doubles of halo on both sides
+
+template <int R>
+struct StarWeights64 {
+    double c;
+    double x[2 * R + 1], y[2 * R + 1], z[2 * R + 1];   // entry [R] unused
+};
+
+template <int R>
+struct BoxWeights64 {
+    double w[2 * R + 1][2 * R + 1][2 * R + 1];         // [dz+R][dy+R][dx+R]
+};
+
+template <int R, int K, int NW>
+struct Stream64Shape {
+    static constexpr int TY = NW * K;
+    static constexpr int ROWS = TY + 2 * R;             // even, so a plane is a multiple of 128 bytes
+    static constexpr int PLANE_DOUBLES = ROWS * kStream64PX;
+    static constexpr int PLANE_BYTES = PLANE_DOUBLES * 8;
+    static constexpr int THREADS = (NW + 1) * 32;
+};
+
+__device__ __forceinline__ double d2get(const double2& v, int m) { return m == 0 ? v.x : v.y; }
+
+template <int R, bool BOX, int K, int NW, int MINB>
+__global__ void __launch_bounds__((NW + 1) * 32, MINB)
+stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* __restrict__ out,
+                          const StreamGeom g,
+                          const __grid_constant__ StarWeights64<R> sw,
+                          const __grid_constant__ BoxWeights64<BOX ? R : 0> bw,
+                          int* __restrict__ status) {
+    using S = Stream64Shape<R, K, NW>;
+    constexpr int PX = kStream64PX;
+    constexpr int HW = (R + 1) / 2 * 2;              // halo doubles read per side (a whole double2)
+    constexpr int NV = 2 * HW + 2;                   // x window of a lane
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    unsigned char* base = smem_raw + ((128u - (smem_addr(smem_raw) & 127u)) & 127u);
+    double* ring = reinterpret_cast<double*>(base);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)g.stages * S::PLANE_BYTES);
+    const uint32_t full0 = smem_addr(bars);
+    const uint32_t empty0 = smem_addr(bars + kMaxStages);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int nstage = g.stages;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < nstage; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, NW);
+        }
+        fence_barrier_init();
+    }
+    __syncthreads();
+    allow_dependents();
+    dependency_wait();
+
+    const int bid = blockIdx.x;
+    const int tile_x = bid % g.tiles_x;
+    const int tile_y = (bid / g.tiles_x) % g.tiles_y;
+    const int chunk = bid / (g.tiles_x * g.tiles_y);
+    const int x0 = tile_x * kStream64TX;
+    const int y0 = tile_y * S::TY;
+    const int z0 = g.z_begin + chunk * g.chunk_z;
+    const int z1 = min(z0 + g.chunk_z, g.z_end);
+    const int nplanes = (z1 - z0) + 2 * R;
+    const int pstart = z0 - R;
+
+    if (warp == NW) {
+        if (lane == 0) {
+            prefetch_tensormap(&tmap_in);
+            bool ok = true;
+            int issued = 0;
+            int s = 0;
+            uint32_t ph = 1;
+            for (int i = 0; i < nplanes; ++i) {
+                if (i >= nstage && !mbar_wait_bounded(empty0 + 8 * s, ph, g.wait_polls)) { ok = false; break; }
+                mbar_arrive_expect_tx(full0 + 8 * s, S::PLANE_BYTES);
+                tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_DOUBLES), &tmap_in, full0 + 8 * s,
+                            x0 - 4, y0 - R, pstart + i);
+                issued = i + 1;
+                if (++s == nstage) { s = 0; ph ^= 1; }
+            }
+            if (!ok) {
+                atomicExch(status, kStatusTimeout);
+                for (int i = max(0, issued - nstage); i < issued; ++i)
+                    mbar_wait_bounded(full0 + 8 * (i % nstage), (i / nstage) & 1, g.wait_polls);
+            }
+        }
+        return;
+    }
+
+    const int row0 = warp * K;
+    const int xg = x0 + 2 * lane;
+    const bool x_in = xg < g.nx;                     // nx is even
+    const size_t plane_stride = (size_t)g.ny * g.nx;
+    bool row_ok[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) row_ok[k] = x_in && (y0 + row0 + k) < g.ny;
+    double* op = out + (size_t)z0 * plane_stride + (size_t)(y0 + row0) * g.nx + xg;
+    int s = 0;
+    uint32_t ph = 0;
+
+    if constexpr (!BOX) {
+        double2 A[K][2 * R];                         // partial sums, oldest incomplete output plane first
+#pragma unroll
+        for (int k = 0; k < K; ++k)
+#pragma unroll
+            for (int j = 0; j < 2 * R; ++j) A[k][j] = make_double2(0.0, 0.0);
+
+        for (int i = 0; i < nplanes; ++i) {
+            if (!mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) {
+                atomicExch(status, kStatusTimeout);
+                return;
+            }
+            const double* pl = ring + (size_t)s * S::PLANE_DOUBLES;
+            const double* colp = pl + row0 * PX + 4 + 2 * lane;
+            double acc[K][2];
+#pragma unroll
+            for (int k = 0; k < K; ++k) { acc[k][0] = A[k][R].x; acc[k][1] = A[k][R].y; }
+            double2 done[K];
+#pragma unroll
+            for (int kk = 0; kk < K + 2 * R; ++kk) {
+                const double2 c = *reinterpret_cast<const double2*>(colp + kk * PX);
+#pragma unroll
+                for (int k = 0; k < K; ++k) {
+                    const int d = kk - k - R;
+                    if (d != 0 && d >= -R && d <= R) {
+                        acc[k][0] = fma(sw.y[d + R], c.x, acc[k][0]);
+                        acc[k][1] = fma(sw.y[d + R], c.y, acc[k][1]);
+                    }
+                }
+                if (kk >= R && kk < K + R) {
+                    const int k = kk - R;
+                    double v[NV];                     // v[HW + m + dx]: the input at column m + dx of the pair
+#pragma unroll
+                    for (int t = 0; t < NV / 2; ++t) {
+                        const double2 dd = *reinterpret_cast<const double2*>(colp + kk * PX - HW + 2 * t);
+                        v[2 * t] = dd.x;
+                        v[2 * t + 1] = dd.y;
+                    }
+#pragma unroll
+                    for (int m = 0; m < 2; ++m) {
+                        double a = fma(sw.c, v[HW + m], acc[k][m]);
+#pragma unroll
+                        for (int d = 1; d <= R; ++d) {
+                            a = fma(sw.x[R - d], v[HW + m - d], a);
+                            a = fma(sw.x[R + d], v[HW + m + d], a);
+                        }
+                        acc[k][m] = a;
+                    }
+                    done[k].x = fma(sw.z[2 * R], c.x, A[k][0].x);
+                    done[k].y = fma(sw.z[2 * R], c.y, A[k][0].y);
+#pragma unroll
+                    for (int j = 0; j < 2 * R - 1; ++j) {
+                        if (j == R - 1) continue;
+                        const double wz = sw.z[2 * R - 1 - j];
+                        A[k][j].x = fma(wz, c.x, A[k][j + 1].x);
+                        A[k][j].y = fma(wz, c.y, A[k][j + 1].y);
+                    }
+                    A[k][2 * R - 1] = make_double2(sw.z[0] * c.x, sw.z[0] * c.y);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < K; ++k) A[k][R - 1] = make_double2(acc[k][0], acc[k][1]);
+            __syncwarp();
+            mbar_arrive_if(lane == 0, empty0 + 8 * s);
+            if (++s == nstage) { s = 0; ph ^= 1; }
+
+            if (i >= 2 * R) {
+#pragma unroll
+                for (int k = 0; k < K; ++k)
+                    if (row_ok[k]) *reinterpret_cast<double2*>(op + (size_t)k * g.nx) = done[k];
+                op += plane_stride;
+            }
+        }
+    } else {
+        constexpr int M = 2 * R + 1;
+        double2 T[K][M];                              // accumulator of output plane z lives in slot z mod M
+#pragma unroll
+        for (int k = 0; k < K; ++k)
+#pragma unroll
+            for (int d = 0; d < M; ++d) T[k][d] = make_double2(0.0, 0.0);
+
+        for (int i0 = 0; i0 < nplanes; i0 += M) {
+            const bool ok = static_for<M>([&](auto uc) -> bool {
+                constexpr int u = decltype(uc)::value;
+                const int i = i0 + u;
+                if (i >= nplanes) return true;
+                if (!mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) return false;
+                const double* pl = ring + (size_t)s * S::PLANE_DOUBLES;
+                const double* colp = pl + row0 * PX + 4 + 2 * lane;
+                double v[K + 2 * R][NV];
+#pragma unroll
+                for (int kk = 0; kk < K + 2 * R; ++kk)
+#pragma unroll
+                    for (int t = 0; t < NV / 2; ++t) {
+                        const double2 dd = *reinterpret_cast<const double2*>(colp + kk * PX - HW + 2 * t);
+                        v[kk][2 * t] = dd.x;
+                        v[kk][2 * t + 1] = dd.y;
+                    }
+                __syncwarp();
+                mbar_arrive_if(lane == 0, empty0 + 8 * s);
+                if (++s == nstage) { s = 0; ph ^= 1; }
+
+#pragma unroll
+                for (int k = 0; k < K; ++k) {
+#pragma unroll
+                    for (int d = 0; d < M; ++d) {     // this plane is tap dz = d - R of output i-(d-R)
+                        double2& t = T[k][(u - d + R + 2 * M) % M];
+                        double a[2];
+                        if (d == 0) {
+                            a[0] = bw.w[0][0][0] * v[k][HW - R];
+                            a[1] = bw.w[0][0][0] * v[k][HW - R + 1];
+                        } else {
+                            a[0] = t.x; a[1] = t.y;
+                        }
+#pragma unroll
+                        for (int dy = 0; dy < M; ++dy)
+#pragma unroll
+                            for (int dx = 0; dx < M; ++dx) {
+                                if (d == 0 && dy == 0 && dx == 0) continue;
+                                const double wv = bw.w[d][dy][dx];
+                                a[0] = fma(wv, v[k + dy][HW - R + dx], a[0]);
+                                a[1] = fma(wv, v[k + dy][HW - R + 1 + dx], a[1]);
+                            }
+                        t = make_double2(a[0], a[1]);
+                    }
+                }
+                if (i >= 2 * R) {
+#pragma unroll
+                    for (int k = 0; k < K; ++k)
+                        if (row_ok[k]) *reinterpret_cast<double2*>(op + (size_t)k * g.nx) = T[k][(u + R + 1) % M];
+                    op += plane_stride;
+                }
+                return true;
+            });
+            if (!ok) {
+                atomicExch(status, kStatusTimeout);
+                return;
+            }
+        }
+    }
+}
+
+}  // namespace stencil

@@ -21,6 +21,7 @@
 #include "kernel_fused.cuh"
 #include "kernel_rows2d.cuh"
 #include "kernel_rows2d_f64.cuh"
+#include "kernel_stream_f64.cuh"
 
 using namespace stencil;
 
@@ -142,6 +143,17 @@ struct Rows2D64Config {
                           int grid, size_t smem, cudaStream_t);
 };
 
+struct Stream64Config {
+    int radius;
+    bool box;
+    int tile_y, plane_bytes, box_rows, threads;
+    const void* kernel;
+    mutable size_t smem_allowed;
+    mutable int cache_device;
+    cudaError_t (*launch)(const struct stencil_plan_s*, const CUtensorMap&, double*, const StreamGeom&,
+                          int grid, size_t smem, cudaStream_t);
+};
+
 struct stencil_plan_s {
     uint32_t magic;
     int ndim;
@@ -156,6 +168,7 @@ struct stencil_plan_s {
     TapT<double>* d_taps64;
     double* scratch64;             // N doubles, iteration ping-pong of FP64 plans
     const struct Rows2D64Config* rows2d64_cfg;
+    const struct Stream64Config* stream64_cfg;
     // device state (created lazily, on the device current at first apply)
     int device;
     Tap* d_taps;
@@ -805,11 +818,75 @@ const Rows2D64Config* find_rows2d64_cfg(const stencil_plan_s* p) {
     return nullptr;
 }
 
+inline double dense_w64_3d(const stencil_plan_s* p, int dz, int dy, int dx) {
+    const int R = p->radius, side = 2 * R + 1;
+    return p->w64[((size_t)(dz + R) * side + (dy + R)) * side + (dx + R)];
+}
+
+template <int R, bool BOX, int K, int NW, int MINB>
+cudaError_t launch_stream64_t(const stencil_plan_s* p, const CUtensorMap& map, double* out, const StreamGeom& g,
+                              int grid, size_t smem, cudaStream_t st) {
+    StarWeights64<R> sw;
+    BoxWeights64<BOX ? R : 0> bw;
+    std::memset(&sw, 0, sizeof(sw));
+    std::memset(&bw, 0, sizeof(bw));
+    if (!BOX) {
+        sw.c = dense_w64_3d(p, 0, 0, 0);
+        for (int d = -R; d <= R; ++d) {
+            if (d == 0) continue;
+            sw.x[d + R] = dense_w64_3d(p, 0, 0, d);
+            sw.y[d + R] = dense_w64_3d(p, 0, d, 0);
+            sw.z[d + R] = dense_w64_3d(p, d, 0, 0);
+        }
+    } else {
+        constexpr int RB = BOX ? R : 0;
+        for (int a = -RB; a <= RB; ++a)
+            for (int b = -RB; b <= RB; ++b)
+                for (int c = -RB; c <= RB; ++c) bw.w[a + RB][b + RB][c + RB] = dense_w64_3d(p, a, b, c);
+    }
+    return launch_kernel(&stencil_stream_f64_kernel<R, BOX, K, NW, MINB>, grid, Stream64Shape<R, K, NW>::THREADS,
+                         smem, st, p->chained, map, out, g, sw, bw, p->d_status);
+}
+
+template <int R, bool BOX, int K, int NW, int MINB>
+Stream64Config make_stream64() {
+    using S = Stream64Shape<R, K, NW>;
+    Stream64Config c;
+    c.radius = R; c.box = BOX; c.tile_y = S::TY; c.plane_bytes = S::PLANE_BYTES; c.box_rows = S::ROWS;
+    c.threads = S::THREADS;
+    c.kernel = reinterpret_cast<const void*>(&stencil_stream_f64_kernel<R, BOX, K, NW, MINB>);
+    c.smem_allowed = 0; c.cache_device = -1;
+    c.launch = &launch_stream64_t<R, BOX, K, NW, MINB>;
+    return c;
+}
+
+const std::vector<Stream64Config>& stream64_configs() {
+    static const std::vector<Stream64Config> v = {
+        make_stream64<1, false, 2, 8, 1>(), make_stream64<2, false, 2, 8, 1>(), make_stream64<3, false, 2, 8, 1>(),
+        make_stream64<4, false, 2, 8, 1>(), make_stream64<1, true, 2, 8, 1>(),
+    };
+    return v;
+}
+
+const Stream64Config* find_stream64_cfg(const stencil_plan_s* p) {
+    if (p->ndim != 3 || p->boundary != STENCIL_ZERO || p->nx % 2 != 0) return nullptr;   // 16-byte rows
+    for (const Stream64Config& c : stream64_configs())
+        if (c.radius == p->radius && c.box == (p->shape == STENCIL_BOX)) return &c;
+    return nullptr;
+}
+
 int resolve_variant_f64(stencil_plan_s* p, int want) {
-    const Rows2D64Config* c = find_rows2d64_cfg(p);
-    if (want == STENCIL_VARIANT_AUTO) want = c ? STENCIL_VARIANT_STREAM : STENCIL_VARIANT_GENERIC;
-    if (want == STENCIL_VARIANT_GENERIC) { p->variant = want; p->rows2d64_cfg = nullptr; return STENCIL_OK; }
-    if (want == STENCIL_VARIANT_STREAM && c) { p->variant = want; p->rows2d64_cfg = c; return STENCIL_OK; }
+    const Rows2D64Config* c2 = find_rows2d64_cfg(p);
+    const Stream64Config* c3 = find_stream64_cfg(p);
+    if (want == STENCIL_VARIANT_AUTO) want = (c2 || c3) ? STENCIL_VARIANT_STREAM : STENCIL_VARIANT_GENERIC;
+    if (want == STENCIL_VARIANT_GENERIC) {
+        p->variant = want; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr;
+        return STENCIL_OK;
+    }
+    if (want == STENCIL_VARIANT_STREAM && (c2 || c3)) {
+        p->variant = want; p->rows2d64_cfg = c2; p->stream64_cfg = c3;
+        return STENCIL_OK;
+    }
     return STENCIL_ERR_UNSUPPORTED;
 }
 
@@ -837,6 +914,48 @@ int get_tensor_map_f64(stencil_plan_s* p, const void* cfg, int box_x, int box_y,
 }
 
 int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStream_t st) {
+    if (p->variant == STENCIL_VARIANT_STREAM && p->stream64_cfg) {
+        const Stream64Config* cfg = p->stream64_cfg;
+        const CUtensorMap* map = nullptr;
+        int rc = get_tensor_map_f64(p, cfg, kStream64PX, cfg->box_rows, src, &map);
+        if (rc != STENCIL_OK) return rc;
+        const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 4;
+        const size_t smem = (size_t)stages * cfg->plane_bytes + 128 + 2 * kMaxStages * sizeof(uint64_t);
+        if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+        {
+            std::lock_guard<std::mutex> lock(g_config_mutex);
+            if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->cache_device = dev; }
+            if (smem > cfg->smem_allowed) {
+                if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                    cudaSuccess) {
+                    cudaGetLastError();
+                    return STENCIL_ERR_CUDA;
+                }
+                cfg->smem_allowed = smem;
+            }
+        }
+        StreamGeom g;
+        g.nz = p->nz; g.ny = p->ny; g.nx = p->nx;
+        g.tiles_x = (p->nx + kStream64TX - 1) / kStream64TX;
+        g.tiles_y = (p->ny + cfg->tile_y - 1) / cfg->tile_y;
+        g.stages = stages;
+        g.streaming_store = 0;
+        g.z_begin = 0; g.z_end = p->nz;
+        g.wait_polls = p->wait_polls; g.drop_plane = -1;
+        // many short CTAs, as for the bandwidth-bound fp32 sweeps; the wide stars re-read 2R halo
+        // planes per chunk, so they get longer chunks (measured on 512^3)
+        const int want_chunk = p->radius >= 3 ? 64 : 32;
+        int chunk = p->chunk_z > 0 ? p->chunk_z : (p->nz >= 2 * want_chunk ? want_chunk : p->nz);
+        chunk = std::max(1, std::min(chunk, p->nz));
+        g.chunk_z = chunk;
+        const int64_t grid64 = (int64_t)g.tiles_x * g.tiles_y * ((p->nz + chunk - 1) / chunk);
+        if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
+        if (cfg->launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
+        p->launches++;
+        return STENCIL_OK;
+    }
     if (p->variant == STENCIL_VARIANT_STREAM && p->rows2d64_cfg) {
         const Rows2D64Config* cfg = p->rows2d64_cfg;
         const CUtensorMap* map = nullptr;
@@ -932,7 +1051,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->radius = radius; p->shape = shape; p->boundary = boundary;
     p->device = -1;
     p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr;
-    p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr;
+    p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr;
     p->host_in = nullptr; p->host_out = nullptr;
     p->copy_in = nullptr; p->copy_out = nullptr;
     p->variant = STENCIL_VARIANT_GENERIC;

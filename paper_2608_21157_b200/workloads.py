@@ -249,6 +249,20 @@ def _build_table() -> Dict[str, Workload]:
         _resizable(lambda d: uniform_field(d, -1.0, 1.0, 6, np.float64), (10240, 10240)),
         dtype=np.float64)
 
+    # supplementary: two of the 3D configs in FP64 (1 GiB per grid)
+    t["cfg2_f64"] = Workload(
+        "cfg2_f64", "3D 7-point star R=1 512^3 in FP64 (centre -6, neighbours +1), zero boundary, 1 step",
+        (512, 512, 512), 1, STAR, ZERO, 1,
+        lambda: star_weights(3, 1, -6.0, [1.0]).astype(np.float64),
+        _resizable(lambda d: uniform_field(d, -1.0, 1.0, 1, np.float64), (512, 512, 512)),
+        dtype=np.float64)
+    t["cfg4_f64"] = Workload(
+        "cfg4_f64", "3D 25-point star R=4 512^3 in FP64 (8th-order FD Laplacian), zero boundary, 1 step",
+        (512, 512, 512), 4, STAR, ZERO, 1,
+        lambda: star_weights(3, 4, float(FD8_CENTER_1D * 3), [float(c) for c in FD8_AXIS]).astype(np.float64),
+        _resizable(lambda d: uniform_field(d, -1.0, 1.0, 4, np.float64), (512, 512, 512)),
+        dtype=np.float64)
+
     # supplementary: the iterated heat operator on a grid that does not fit L2
     t["cfg5L"] = Workload(
         "cfg5L", "3D 7-point heat diffusion 512^3, 16 steps (working set exceeds L2)",

@@ -359,9 +359,25 @@ def test_f64_rows2d_kernel_matches_oracle(R, box, dims, chunk, stages):
     assert used == "stream"
 
 
+@pytest.mark.parametrize("R,box", [(1, False), (2, False), (3, False), (4, False), (1, True)])
+@pytest.mark.parametrize("dims,chunk_z,stages", [
+    ((37, 45, 66), 10, 3),       # two 64-column tiles, ragged in x, y and z
+    ((8, 16, 64), 0, 0),         # exactly one tile
+    ((3, 5, 4), 0, 2),           # smaller than the stencil reach
+    ((70, 33, 130), 32, 0),      # three x tiles, the last 2 points wide
+])
+def test_f64_stream_kernel_matches_oracle(R, box, dims, chunk_z, stages):
+    w = (wl.random_box_weights if box else wl.random_star_weights)(3, R, 85, np.float64)
+    a = wl.normal_field(dims, 86, np.float64)
+    for steps in (1, 3):
+        used = check_f64(dims, R, b.BOX if box else b.STAR, w, b.ZERO, a, steps=steps,
+                         chunk_z=chunk_z or None, stages=stages or None)
+        assert used == "stream"
+
+
 @pytest.mark.parametrize("dims,R,box,boundary", [
-    ((33, 47), 3, True, b.ZERO), ((20, 30), 2, True, b.PERIODIC), ((9, 12, 20), 1, True, b.ZERO),
-    ((7, 10, 14), 2, False, b.PERIODIC), ((40, 64), 5, True, b.ZERO)])
+    ((33, 47), 3, True, b.ZERO), ((20, 30), 2, True, b.PERIODIC), ((9, 12, 21), 1, True, b.ZERO),
+    ((7, 10, 14), 2, False, b.PERIODIC), ((40, 64), 5, True, b.ZERO), ((9, 12, 20), 2, True, b.ZERO)])
 def test_f64_generic_kernel(dims, R, box, boundary):
     ndim = len(dims)
     w = (wl.random_box_weights if box else wl.random_star_weights)(ndim, R, 83, np.float64)
