@@ -215,6 +215,14 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
     bool row_ok[K];
 #pragma unroll
     for (int k = 0; k < K; ++k) row_ok[k] = x_in && (y0 + row0 + k) < g.ny;
+    // Interior warps (every lane stores every row) can take a branch-free store path.  It pays
+    // for the sweeps that are bound by instruction issue (+3 % measured on the 27-point box and
+    // the radius-4 star) and costs 3 % on the bandwidth-bound 7-point star, hence the switch.
+    constexpr bool kUniformStores = BOX || R >= 3;
+    bool mine_ok = kUniformStores;
+#pragma unroll
+    for (int k = 0; k < K; ++k) mine_ok = mine_ok && row_ok[k];
+    const bool all_ok = kUniformStores && __all_sync(0xffffffffu, mine_ok);
     // next output plane of this thread (advanced after every stored plane)
     float* op = out + (size_t)z0 * plane_stride + (size_t)(y0 + row0) * g.nx + xg;
     const int streaming = g.streaming_store;
@@ -300,9 +308,14 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
             if (++s == nstage) { s = 0; ph ^= 1; }
 
             if (i >= 2 * R) {
+                if (all_ok) {
 #pragma unroll
-                for (int k = 0; k < K; ++k)
-                    if (row_ok[k]) store_f4(op + (size_t)k * g.nx, done[k], streaming);
+                    for (int k = 0; k < K; ++k) store_f4(op + (size_t)k * g.nx, done[k], streaming);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < K; ++k)
+                        if (row_ok[k]) store_f4(op + (size_t)k * g.nx, done[k], streaming);
+                }
                 op += plane_stride;
             }
         }
@@ -358,10 +371,16 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                         t = make_float4(a[0], a[1], a[2], a[3]);
                     }
                 }
-                if (i >= 2 * R) {
+                if (i >= 2 * R) {                         // tap dz = +R was the last one of plane i-R
+                    if (all_ok) {
 #pragma unroll
-                    for (int k = 0; k < K; ++k)           // tap dz = +R was the last one of plane i-R
-                        if (row_ok[k]) store_f4(op + (size_t)k * g.nx, T[k][(u + R + 1) % M], streaming);
+                        for (int k = 0; k < K; ++k)
+                            store_f4(op + (size_t)k * g.nx, T[k][(u + R + 1) % M], streaming);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < K; ++k)
+                            if (row_ok[k]) store_f4(op + (size_t)k * g.nx, T[k][(u + R + 1) % M], streaming);
+                    }
                     op += plane_stride;
                 }
                 return true;
