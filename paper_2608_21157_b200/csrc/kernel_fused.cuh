@@ -121,6 +121,9 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
         if (y_in && x_store && (row0 + k) >= g.halo_y && (row0 + k) < g.halo_y + g.tile_y) store_mask |= 1u << k;
     }
     constexpr uint32_t kAllRows = (1u << K) - 1u;
+    // the same flags for the whole warp, so that the common case is a uniform branch
+    const bool warp_all_in = __all_sync(0xffffffffu, in_mask == kAllRows);
+    const bool warp_all_store = __all_sync(0xffffffffu, store_mask == kAllRows);
     const size_t plane_stride = (size_t)g.ny * g.nx;
     float* const out_col = out + (size_t)(y0e + row0) * g.nx + xg;     // this thread's column of rows
     const int toff = row0 * TXE + col;                                  // its offset inside a plane
@@ -234,7 +237,7 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                         }
                         // the zero boundary holds at every time level: cells outside the grid go
                         // back to zero (nothing to do for regions and planes inside the grid)
-                        if (in_mask != kAllRows || zl < 0 || zl >= g.nz) {
+                        if (!warp_all_in || zl < 0 || zl >= g.nz) {
                             const bool z_in = zl >= 0 && zl < g.nz;
 #pragma unroll
                             for (int k = 0; k < K; ++k)
@@ -245,7 +248,7 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                             // last level of this pass: interior of the tile goes to global memory
                             if (!dead && zl >= z0 && zl < z1) {
                                 float* op = out_col + (size_t)zl * plane_stride;
-                                if (store_mask == kAllRows) {
+                                if (warp_all_store) {
 #pragma unroll
                                     for (int k = 0; k < K; ++k)
                                         *reinterpret_cast<float4*>(op + (size_t)k * g.nx) = e[k];
