@@ -40,8 +40,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_write.sum from an ncu capture; see profiles/).  None = not captured.
 NCU_TRAFFIC_BYTES = {
     "cfg2": 1003.8e6,   # stream kernel, star R=1: 2 x (279.4 MB read + 222.5 MB written) on the half grid
-    "cfg3": 1004.0e6,   # stream kernel, box R=1
-    "cfg4": 994.9e6,    # stream kernel, star R=4
+    "cfg3": 1004.6e6,   # stream kernel, box R=1
+    "cfg4": 995.7e6,    # stream kernel, star R=4
     "cfg5": 101.5e6,    # one fused pass (2 time steps of 256^3): 78.2 MB read + 23.3 MB written
 }
 
