@@ -457,6 +457,79 @@ def test_paper_workload_full_grid_one_step():
     assert float(np.max(np.abs(got - want))) <= wl.tolerance(w, float(np.abs(a).max()), 1)
 
 
+def test_grid_with_more_than_2_to_the_31_points():
+    """Maximum-size case: 2100 x 1024 x 1024 = 2.2e9 points (8.8 GB per grid), beyond 32-bit
+    element offsets.  The field is a formula of the indices, built on the device; sampled
+    output planes (first, middle, last) are compared with the oracle run on the 2R+1 input
+    planes around them, built from the same formula on the host."""
+    nz, ny, nx = 2100, 1024, 1024
+    R = 1
+    w = wl.random_star_weights(3, R, 97)
+
+    def field(z_lo, z_hi, xp):
+        z = xp.arange(z_lo, z_hi).reshape(-1, 1, 1)
+        y = xp.arange(ny).reshape(1, -1, 1)
+        x = xp.arange(nx).reshape(1, 1, -1)
+        return (((x * 3 + y * 5 + z * 7) % 17) - 8)
+
+    dev = torch.device("cuda:0")
+    src = torch.empty((nz, ny, nx), dtype=torch.float32, device=dev)
+    for z0 in range(0, nz, 100):
+        z1 = min(z0 + 100, nz)
+        src[z0:z1] = field(z0, z1, torch).to(dev).float() / 8.0
+    dst = torch.empty_like(src)
+    with b.Plan((nz, ny, nx), R, b.STAR, w, b.ZERO) as p:
+        assert p.variant == "stream"
+        p.apply(src, dst, 1, torch.cuda.current_stream().cuda_stream)
+        assert p.query_status() == b.OK
+    torch.cuda.synchronize()
+    tol = wl.tolerance(w, 1.0, 1)
+    for zc in (0, 1049, nz - 1):
+        lo, hi = max(zc - R, 0), min(zc + R + 1, nz)
+        # planes outside the grid are zero: pad so that the oracle's own boundary is never the answer
+        sub = np.zeros((2 * R + 1, ny, nx), dtype=np.float32)
+        sub[lo - (zc - R):hi - (zc - R)] = (field(lo, hi, np) / 8.0).astype(np.float32)
+        want = oracle.apply(sub, w, b.ZERO, 1)[R]
+        got = dst[zc].cpu().numpy()
+        assert float(np.max(np.abs(got - want))) <= tol, f"plane {zc}"
+    del src, dst
+    torch.cuda.empty_cache()
+
+
+def test_2d_grid_with_more_than_2_to_the_31_points():
+    """The same for the 2D row-streaming kernel: 46400 x 46400 = 2.15e9 points."""
+    ny = nx = 46400
+    R = 2
+    w = wl.random_box_weights(2, R, 98)
+
+    def field(y_lo, y_hi, xp):
+        y = xp.arange(y_lo, y_hi).reshape(-1, 1)
+        x = xp.arange(nx).reshape(1, -1)
+        return (((x * 3 + y * 5) % 17) - 8)
+
+    dev = torch.device("cuda:0")
+    src = torch.empty((ny, nx), dtype=torch.float32, device=dev)
+    for y0 in range(0, ny, 4000):
+        y1 = min(y0 + 4000, ny)
+        src[y0:y1] = field(y0, y1, torch).to(dev).float() / 8.0
+    dst = torch.empty_like(src)
+    with b.Plan((ny, nx), R, b.BOX, w, b.ZERO) as p:
+        assert p.variant == "stream"
+        p.apply(src, dst, 1, torch.cuda.current_stream().cuda_stream)
+        assert p.query_status() == b.OK
+    torch.cuda.synchronize()
+    tol = wl.tolerance(w, 1.0, 1)
+    for yc in (0, 23111, ny - 1):
+        lo, hi = max(yc - R, 0), min(yc + R + 1, ny)
+        sub = np.zeros((2 * R + 1, nx), dtype=np.float32)
+        sub[lo - (yc - R):hi - (yc - R)] = (field(lo, hi, np) / 8.0).astype(np.float32)
+        want = oracle.apply(sub, w, b.ZERO, 1)[R]
+        got = dst[yc].cpu().numpy()
+        assert float(np.max(np.abs(got - want))) <= tol, f"row {yc}"
+    del src, dst
+    torch.cuda.empty_cache()
+
+
 def test_generic_kernel_on_a_full_3d_config():
     wk = wl.get("cfg2").scaled((128, 128, 128))
     a, w = wk.input(), wk.weights()
