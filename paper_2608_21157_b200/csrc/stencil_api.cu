@@ -472,8 +472,7 @@ int sm_count();
 
 int launch_generic(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
     Grid g{p->nz, p->ny, p->nx};
-    const int64_t blocks_needed = (p->npoints + kGenericThreads - 1) / kGenericThreads;
-    const int grid = (int)std::min<int64_t>(blocks_needed, (int64_t)sm_count() * 16);
+    const int grid = generic_grid_size(g, sm_count());
     const int ntaps = (int)p->taps.size();
     if (p->boundary == STENCIL_PERIODIC)
         stencil_generic_kernel<true><<<grid, kGenericThreads, 0, st>>>(src, dst, g, p->d_taps, ntaps);
@@ -1003,8 +1002,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         return STENCIL_OK;
     }
     Grid g{p->nz, p->ny, p->nx};
-    const int64_t blocks_needed = (p->npoints + kGenericThreads - 1) / kGenericThreads;
-    const int grid = (int)std::min<int64_t>(blocks_needed, 148 * 16);
+    const int grid = generic_grid_size(g, sm_count());
     const int ntaps = (int)p->taps64.size();
     if (p->boundary == STENCIL_PERIODIC)
         stencil_generic_kernel<true, double><<<grid, kGenericThreads, 0, st>>>(src, dst, g, p->d_taps64, ntaps);
@@ -1336,8 +1334,7 @@ int stencil_apply_static(stencil_plan_t p, const float* in, float* out, int step
     // scratch grid.  Every cell of it is written before it is read, so nothing of
     // an earlier call's contents has to be cleared.
     Grid g{p->nz, p->ny, p->nx};
-    const int64_t blocks_needed = (p->npoints + kGenericThreads - 1) / kGenericThreads;
-    const int nblocks = (int)std::min<int64_t>(blocks_needed, 148 * 16);
+    const int nblocks = generic_grid_size(g, sm_count());
     const float* src = in;
     for (int k = 0; k < steps; ++k) {
         const int remaining = steps - 1 - k;

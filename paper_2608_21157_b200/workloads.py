@@ -249,6 +249,13 @@ def _build_table() -> Dict[str, Workload]:
         _resizable(lambda d: uniform_field(d, -1.0, 1.0, 6, np.float64), (10240, 10240)),
         dtype=np.float64)
 
+    # supplementary: cfg2's operator with a periodic boundary
+    t["cfg2_periodic"] = Workload(
+        "cfg2_periodic", "3D 7-point star R=1 512^3, periodic boundary, 1 step",
+        (512, 512, 512), 1, STAR, PERIODIC, 1,
+        lambda: star_weights(3, 1, -6.0, [1.0]),
+        _resizable(lambda d: uniform_field(d, -1.0, 1.0, 1), (512, 512, 512)))
+
     # supplementary: two of the 3D configs in FP64 (1 GiB per grid)
     t["cfg2_f64"] = Workload(
         "cfg2_f64", "3D 7-point star R=1 512^3 in FP64 (centre -6, neighbours +1), zero boundary, 1 step",
