@@ -107,7 +107,9 @@ enum {
  *             off-axis entry is exactly zero, and is checked
  *             (STENCIL_ERR_INVALID otherwise).  Zero entries cost nothing.
  *   boundary  STENCIL_ZERO (taps outside the grid contribute 0; every grid
- *             point is an output) or STENCIL_PERIODIC (indices wrap).
+ *             point is an output) or STENCIL_PERIODIC (indices wrap; on the
+ *             tiled kernels the plan then also owns a padded copy of the grid,
+ *             allocated at the first apply).
  *
  * Needs no device memory until the first apply.  Errors: INVALID, UNSUPPORTED,
  * ALLOC.

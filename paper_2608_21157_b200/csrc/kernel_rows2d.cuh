@@ -29,6 +29,7 @@ struct Rows2DGeom {
     int chunk_y;                // output rows per warp
     int nchunks;
     int stages;                 // batches in a warp's ring
+    int in_off_x, in_off_y;     // added to the TMA coordinates (padded input of a periodic grid), else 0
 };
 
 template <int YB>
@@ -83,7 +84,7 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
         for (int b = 0; b < pre; ++b) {
             mbar_arrive_expect_tx(full0 + 8 * b, S::BATCH_BYTES);
             tma_load_3d(smem_addr(ring + (size_t)b * S::BATCH_FLOATS), &tmap_in, full0 + 8 * b,
-                        x0 - 4, ystart + b * YB, 0);
+                        x0 - 4 + g.in_off_x, ystart + b * YB + g.in_off_y, 0);
         }
     }
 
@@ -180,7 +181,7 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
         if (lane == 0 && b + nstage < nbatches) {
             mbar_arrive_expect_tx(full0 + 8 * s, S::BATCH_BYTES);
             tma_load_3d(smem_addr(ring + (size_t)s * S::BATCH_FLOATS), &tmap_in, full0 + 8 * s,
-                        x0 - 4, ystart + (b + nstage) * YB, 0);
+                        x0 - 4 + g.in_off_x, ystart + (b + nstage) * YB + g.in_off_y, 0);
             issued = b + nstage + 1;
         }
         if (++s == nstage) { s = 0; ph ^= 1; }

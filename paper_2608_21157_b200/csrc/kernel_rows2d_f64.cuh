@@ -73,7 +73,7 @@ stencil_rows2d_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
         for (int b = 0; b < pre; ++b) {
             mbar_arrive_expect_tx(full0 + 8 * b, S::BATCH_BYTES);
             tma_load_3d(smem_addr(ring + (size_t)b * S::BATCH_DOUBLES), &tmap_in, full0 + 8 * b,
-                        x0 - 4, ystart + b * YB, 0);
+                        x0 - 4 + g.in_off_x, ystart + b * YB + g.in_off_y, 0);
         }
     }
 
@@ -166,7 +166,7 @@ stencil_rows2d_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
         if (lane == 0 && b + nstage < nbatches) {
             mbar_arrive_expect_tx(full0 + 8 * s, S::BATCH_BYTES);
             tma_load_3d(smem_addr(ring + (size_t)s * S::BATCH_DOUBLES), &tmap_in, full0 + 8 * s,
-                        x0 - 4, ystart + (b + nstage) * YB, 0);
+                        x0 - 4 + g.in_off_x, ystart + (b + nstage) * YB + g.in_off_y, 0);
             issued = b + nstage + 1;
         }
         if (++s == nstage) { s = 0; ph ^= 1; }

@@ -50,6 +50,8 @@ struct StreamGeom {
     int chunk_z;                // planes of output per CTA
     int stages;                 // depth of the plane ring
     int streaming_store;        // 1: st.global.cs
+    int in_off_x, in_off_y, in_off_z;   // added to every TMA coordinate: non-zero when the input is a
+                                // padded copy of the grid (periodic boundary), else 0
     unsigned wait_polls;        // cap of every bounded wait
     int drop_plane;             // test hook: the producer never loads this plane of a CTA (-1: none)
 };
@@ -192,7 +194,7 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                 if (i != g.drop_plane) {
                     mbar_arrive_expect_tx(full0 + 8 * s, S::BOX_BYTES);
                     tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_BYTES), &tmap_in, full0 + 8 * s,
-                                x0 - 4, y0 - R, pstart + i);
+                                x0 - 4 + g.in_off_x, y0 - R + g.in_off_y, pstart + i + g.in_off_z);
                 }
                 issued = i + 1;
                 if (++s == nstage) { s = 0; ph ^= 1; }

@@ -94,7 +94,7 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
                 if (i >= nstage && !mbar_wait_bounded(empty0 + 8 * s, ph, g.wait_polls)) { ok = false; break; }
                 mbar_arrive_expect_tx(full0 + 8 * s, S::PLANE_BYTES);
                 tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_DOUBLES), &tmap_in, full0 + 8 * s,
-                            x0 - 4, y0 - R, pstart + i);
+                            x0 - 4 + g.in_off_x, y0 - R + g.in_off_y, pstart + i + g.in_off_z);
                 issued = i + 1;
                 if (++s == nstage) { s = 0; ph ^= 1; }
             }

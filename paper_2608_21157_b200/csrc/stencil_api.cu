@@ -17,6 +17,7 @@
 
 #include "common.cuh"
 #include "kernel_generic.cuh"
+#include "kernel_pad.cuh"
 #include "kernel_stream.cuh"
 #include "kernel_fused.cuh"
 #include "kernel_rows2d.cuh"
@@ -174,6 +175,7 @@ struct stencil_plan_s {
     Tap* d_taps;
     int* d_status;
     float* scratch;                // N floats, iteration ping-pong
+    float* pad;                    // padded copy of the input (periodic boundary on the tiled kernels)
     float* host_in;                // N floats each, apply_host staging
     float* host_out;
     cudaStream_t copy_in, copy_out; // apply_host: upload / download streams (created on first use)
@@ -365,10 +367,11 @@ const Rows2DConfig* find_rows2d_cfg(int radius, bool box) {
     return nullptr;
 }
 
-// The tiled kernels need a zero boundary (TMA fills out-of-grid cells with zero) and rows
-// whose byte length is a multiple of 16 (a TMA stride rule).
+// The tiled kernels need rows whose byte length is a multiple of 16 (a TMA stride rule).
+// The zero boundary comes from TMA's zero fill of out-of-grid cells; a periodic grid is first
+// copied into a padded grid with wrapped halos (kernel_pad.cuh) and swept from there.
 bool stream_supported(const stencil_plan_s* p) {
-    if (p->boundary != STENCIL_ZERO || p->nx % 4 != 0) return false;
+    if (p->nx % 4 != 0) return false;
     const bool box = p->shape == STENCIL_BOX;
     if (p->ndim == 2) return find_rows2d_cfg(p->radius, box) != nullptr;
     return find_stream_cfg(p->radius, box, 0, 0) != nullptr;
@@ -377,6 +380,7 @@ bool stream_supported(const stencil_plan_s* p) {
 // Temporal blocking covers what the STREAM kernels cover, restricted to star stencils.
 const FusedConfig* pick_fused(const stencil_plan_s* p) {
     if (!stream_supported(p) || p->shape != STENCIL_STAR || p->ndim != 3) return nullptr;
+    if (p->boundary != STENCIL_ZERO) return nullptr;      // fused passes re-impose a ZERO exterior
     if (p->fuse_steps == 1) return nullptr;
     int txe = p->tile_x;
     if (p->fuse_steps == 0 && txe == 0 && p->fused_tile_y == 0) {
@@ -484,15 +488,16 @@ int launch_generic(stencil_plan_s* p, const float* src, float* dst, cudaStream_t
 }
 
 int get_tensor_map(stencil_plan_s* p, const void* cfg, int box_x, int box_y, const float* src,
-                   const CUtensorMap** out) {
+                   const CUtensorMap** out, int tnx = 0, int tny = 0, int tnz = 0) {
+    if (tnx == 0) { tnx = p->nx; tny = p->ny; tnz = p->nz; }     // extents of the tensor `src` points at
     for (auto& e : p->maps)
         if (e.ptr == src && e.cfg == cfg) { *out = &e.map; return STENCIL_OK; }
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return STENCIL_ERR_CUDA;
     stencil_plan_s::MapEntry e;
     e.ptr = src; e.cfg = cfg;
-    const cuuint64_t dims[3] = {(cuuint64_t)p->nx, (cuuint64_t)p->ny, (cuuint64_t)p->nz};
-    const cuuint64_t strides[2] = {(cuuint64_t)p->nx * 4, (cuuint64_t)p->nx * (cuuint64_t)p->ny * 4};
+    const cuuint64_t dims[3] = {(cuuint64_t)tnx, (cuuint64_t)tny, (cuuint64_t)tnz};
+    const cuuint64_t strides[2] = {(cuuint64_t)tnx * 4, (cuuint64_t)tnx * (cuuint64_t)tny * 4};
     const cuuint32_t box[3] = {(cuuint32_t)box_x, (cuuint32_t)box_y, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = enc(&e.map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(src), dims, strides,
@@ -592,6 +597,29 @@ int choose_chunk(const stencil_plan_s* p, const StreamConfig* cfg, int stages, d
     return best_chunk;
 }
 
+// Periodic boundary: copy `src` into the plan's padded grid (wrapped halos) on `st`.
+// Extents of the padded grid come back through pnx/pny/pnz.
+int pad_periodic(stencil_plan_s* p, const float* src, cudaStream_t st, int* pnx, int* pny, int* pnz) {
+    const int R = p->radius;
+    const int rz = p->ndim == 3 ? R : 0;
+    *pnx = p->nx + 2 * kPadX; *pny = p->ny + 2 * R; *pnz = p->nz + 2 * rz;
+    if (!p->pad) {
+        const size_t bytes = (size_t)*pnx * *pny * *pnz * sizeof(float);
+        if (cudaMalloc(&p->pad, bytes) != cudaSuccess) {
+            cudaGetLastError();
+            p->pad = nullptr;
+            return STENCIL_ERR_ALLOC;
+        }
+    }
+    Grid g{p->nz, p->ny, p->nx};
+    const int64_t cells = (int64_t)(*pnx / 4) * *pny * *pnz;
+    const int grid = (int)std::min<int64_t>((cells + 255) / 256, (int64_t)sm_count() * 32);
+    stencil_pad_periodic_kernel<<<grid, 256, 0, st>>>(src, p->pad, g, R, rz);
+    if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
+    p->launches++;
+    return STENCIL_OK;
+}
+
 // dst[z_begin, z_end) = one sweep of src; the whole grid when z_end <= z_begin.
 int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st, int z_begin = 0,
                   int z_end = 0) {
@@ -614,10 +642,21 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     }
     const StreamConfig* cfg = p->stream_cfg;
     const CUtensorMap* map = nullptr;
-    int rc = get_tensor_map(p, cfg, kStreamPX, cfg->box_rows, src, &map);
+    const bool periodic = p->boundary == STENCIL_PERIODIC;
+    int rc;
+    if (periodic) {
+        int pnx, pny, pnz;
+        if ((rc = pad_periodic(p, src, st, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
+        rc = get_tensor_map(p, cfg, kStreamPX, cfg->box_rows, p->pad, &map, pnx, pny, pnz);
+    } else {
+        rc = get_tensor_map(p, cfg, kStreamPX, cfg->box_rows, src, &map);
+    }
     if (rc != STENCIL_OK) return rc;
 
     StreamGeom g;
+    g.in_off_x = periodic ? kPadX : 0;
+    g.in_off_y = periodic ? p->radius : 0;
+    g.in_off_z = periodic ? p->radius : 0;
     g.nz = p->nz; g.ny = p->ny; g.nx = p->nx;
     g.tiles_x = (p->nx + kStreamTX - 1) / kStreamTX;
     g.tiles_y = (p->ny + cfg->tile_y - 1) / cfg->tile_y;
@@ -643,7 +682,15 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
 int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
     const Rows2DConfig* cfg = p->rows2d_cfg;
     const CUtensorMap* map = nullptr;
-    int rc = get_tensor_map(p, cfg, kStreamPX, cfg->YB, src, &map);
+    const bool periodic = p->boundary == STENCIL_PERIODIC;
+    int rc;
+    if (periodic) {
+        int pnx, pny, pnz;
+        if ((rc = pad_periodic(p, src, st, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
+        rc = get_tensor_map(p, cfg, kStreamPX, cfg->YB, p->pad, &map, pnx, pny, pnz);
+    } else {
+        rc = get_tensor_map(p, cfg, kStreamPX, cfg->YB, src, &map);
+    }
     if (rc != STENCIL_OK) return rc;
     const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
     const size_t smem = (size_t)cfg->NW * stages * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8;
@@ -666,6 +713,8 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     g.ny = p->ny; g.nx = p->nx;
     g.strips = (p->nx + kStreamTX - 1) / kStreamTX;
     g.stages = stages;
+    g.in_off_x = periodic ? kPadX : 0;
+    g.in_off_y = periodic ? p->radius : 0;
     int chunk = p->chunk_z;                          // the streamed axis of a 2D grid is y
     if (chunk <= 0) {
         // As many (strip, chunk) units as fill the machine's warp slots once (two CTAs per SM),
@@ -942,6 +991,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         g.stages = stages;
         g.streaming_store = 0;
         g.z_begin = 0; g.z_end = p->nz;
+        g.in_off_x = 0; g.in_off_y = 0; g.in_off_z = 0;
         g.wait_polls = p->wait_polls; g.drop_plane = -1;
         // many short CTAs, as for the bandwidth-bound fp32 sweeps; the wide stars re-read 2R halo
         // planes per chunk, so they get longer chunks (measured on 512^3)
@@ -981,6 +1031,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         g.ny = p->ny; g.nx = p->nx;
         g.strips = (p->nx + kStrip64 - 1) / kStrip64;
         g.stages = stages;
+        g.in_off_x = 0; g.in_off_y = 0;
         int chunk = p->chunk_z;
         if (chunk <= 0) {                             // same sizing rule as the fp32 kernel
             const int R = p->radius;
@@ -1048,7 +1099,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->npoints = n;
     p->radius = radius; p->shape = shape; p->boundary = boundary;
     p->device = -1;
-    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr;
+    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr;
     p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr;
     p->host_in = nullptr; p->host_out = nullptr;
     p->copy_in = nullptr; p->copy_out = nullptr;
@@ -1244,6 +1295,7 @@ int stencil_apply_host(stencil_plan_t p, const float* in_host, float* out_host, 
     const int min_planes = std::max(2 * p->radius, 8);           // per slab
     const int kSlabs = p->nz >= kMaxSlabs * 2 * min_planes ? kMaxSlabs : kMaxSlabs / 2;
     const bool pipelined = steps == 1 && p->variant == STENCIL_VARIANT_STREAM && p->ndim == 3 &&
+                           p->boundary == STENCIL_ZERO &&
                            p->nz >= kSlabs * min_planes;
     if (!pipelined) {
         if (cudaMemcpyAsync(p->host_in, in_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
@@ -1354,12 +1406,14 @@ int stencil_destroy(stencil_plan_t p) {
     if (!p) return STENCIL_OK;
     if (!valid_plan(p)) return STENCIL_ERR_INVALID;
     int rc = STENCIL_OK;
-    if (p->d_status || p->scratch || p->host_in || p->host_out || p->d_taps || p->d_taps64 || p->scratch64) {
+    if (p->d_status || p->scratch || p->host_in || p->host_out || p->d_taps || p->d_taps64 || p->scratch64 ||
+        p->pad) {
         int cur = -1;
         cudaGetDevice(&cur);
         if (p->device >= 0 && cur != p->device) cudaSetDevice(p->device);
         if (p->used) cudaStreamSynchronize(p->last_stream);
-        void* ptrs[] = {p->d_status, p->scratch, p->host_in, p->host_out, p->d_taps, p->d_taps64, p->scratch64};
+        void* ptrs[] = {p->d_status, p->scratch, p->host_in, p->host_out, p->d_taps, p->d_taps64, p->scratch64,
+                        p->pad};
         for (void* q : ptrs)
             if (q && cudaFree(q) != cudaSuccess) rc = STENCIL_ERR_CUDA;
         for (cudaEvent_t e : p->events) cudaEventDestroy(e);
@@ -1516,7 +1570,10 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
         case STENCIL_KEY_SCRATCH_BYTES: {
             int64_t grids = (p->scratch != nullptr) + (p->host_in != nullptr) + (p->host_out != nullptr);
             *value = grids * p->npoints * (int64_t)sizeof(float) +
-                     (p->scratch64 ? p->npoints * (int64_t)sizeof(double) : 0);
+                     (p->scratch64 ? p->npoints * (int64_t)sizeof(double) : 0) +
+                     (p->pad ? (int64_t)(p->nx + 2 * kPadX) * (p->ny + 2 * p->radius) *
+                                   (p->nz + (p->ndim == 3 ? 2 * p->radius : 0)) * (int64_t)sizeof(float)
+                             : 0);
             return STENCIL_OK;
         }
         case STENCIL_KEY_CHUNK_Z: *value = p->chunk_z; return STENCIL_OK;

@@ -114,6 +114,9 @@ def test_variant_selection_rules():
         assert e.value.status == b.ERR_UNSUPPORTED
         assert p.variant == "generic"
     with b.Plan((64, 64, 64), 1, b.STAR, star, b.PERIODIC) as p:
+        assert p.variant == "stream"                # swept from a padded copy with wrapped halos
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # no temporal blocking under a periodic boundary
+    with b.Plan((64, 64, 62), 1, b.STAR, star, b.PERIODIC) as p:
         assert p.variant == "generic"
     with b.Plan((64, 64), 1, b.STAR, wl.star_weights(2, 1, -4.0, [1.0]), b.ZERO) as p:
         assert p.variant in ("generic", "stream")

@@ -208,6 +208,38 @@ def test_non_default_stream():
     assert np.max(np.abs(dst.cpu().numpy() - want)) <= wl.tolerance(w, float(np.abs(a).max()), 3)
 
 
+# ------------------------------------------------- periodic boundary, tiled path --
+@pytest.mark.parametrize("R,box", STREAM_OPS)
+@pytest.mark.parametrize("dims,chunk_z", [((37, 45, 132), 10), ((8, 16, 128), 0), ((2, 3, 4), 0), ((70, 33, 260), 32)])
+def test_periodic_3d_on_the_tiled_kernel(R, box, dims, chunk_z):
+    w = wl.random_box_weights(3, R, 101) if box else wl.random_star_weights(3, R, 101)
+    a = wl.normal_field(dims, 102)
+    for steps in (1, 3):
+        used = check(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps, chunk_z=chunk_z or None)
+        assert used == "stream"
+
+
+@pytest.mark.parametrize("R,box", [(1, False), (4, False), (2, True), (3, True)])
+@pytest.mark.parametrize("dims", [(67, 132), (3, 8), (200, 260)])
+def test_periodic_2d_on_the_tiled_kernel(R, box, dims):
+    w = wl.random_box_weights(2, R, 103) if box else wl.random_star_weights(2, R, 103)
+    a = wl.normal_field(dims, 104)
+    for steps in (1, 4):
+        used = check(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps)
+        assert used == "stream"
+
+
+def test_periodic_sum_rule_on_gpu():
+    """Under a periodic boundary the total is multiplied by sum(w) every step."""
+    dims = (48, 40, 64)
+    w = wl.star_weights(3, 1, 0.4, [0.1])
+    a = wl.uniform_field(dims, 0.0, 1.0, 105)
+    got, used = gpu_sweep(dims, 1, b.STAR, w, b.PERIODIC, a, steps=6)
+    assert used == "stream"
+    s0, s1 = a.astype(np.float64).sum(), got.astype(np.float64).sum()
+    assert abs(s1 - s0) < 1e-5 * s0
+
+
 # ------------------------------------------------------------- 2D row streaming --
 ROWS2D_OPS = [(1, False), (2, False), (3, False), (4, False), (1, True), (2, True), (3, True), (4, True)]
 
