@@ -6,70 +6,104 @@
 // out[p] = sum_t w_t * in[p + o_t]   (cross-correlation, stride 1; taps that leave the
 // grid contribute 0 under the zero boundary and wrap under the periodic one).
 //
-// A CTA owns a segment of one grid row, so y and z (and with them the row a tap reads, and
-// whether that row exists or where it wraps to) are the same for the whole CTA: the only
-// per-thread boundary work is in x.  Reads along x are coalesced; the (2R+1) rows a CTA
-// touches are shared with its neighbours through L1/L2.
+// A CTA works on one segment of one grid row at a time, so y and z are the same for all of
+// its threads.  For every segment the threads first resolve each tap once for the whole
+// CTA: which input row it reads (after the bounds test or the wrap in y and z) as a flat
+// offset, kept in shared memory.  The per-point loop is then one shared-memory read, the
+// x test or wrap, one coalesced global read and one FMA per tap.
 #pragma once
 #include "common.cuh"
 
 namespace stencil {
 
 constexpr int kGenericThreads = 256;
-constexpr int kGenericSmemTaps = 1024;   // taps staged in shared memory when they fit
+constexpr int kGenericSmemTaps = 1024;   // taps resolved per round (more taps: several rounds)
 
 __device__ __forceinline__ int wrap_index(int q, int n) {
     q %= n;
     return q < 0 ? q + n : q;
 }
 
+template <typename T>
+struct ResolvedTap {
+    long long row;      // flat offset of the input row this tap reads; -1: the row is outside the grid
+    int dx;
+    T w;
+};
+
 // T = float, or double for FP64 plans (the precision of the paper's case study).
 template <bool kPeriodic, typename T = float>
 __global__ void __launch_bounds__(kGenericThreads)
 stencil_generic_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g,
                        const TapT<T>* __restrict__ taps, int ntaps) {
-    __shared__ TapT<T> s_taps[kGenericSmemTaps];
-    const bool staged = ntaps <= kGenericSmemTaps;
-    if (staged) {
-        for (int t = threadIdx.x; t < ntaps; t += blockDim.x) s_taps[t] = taps[t];
-        __syncthreads();
-    }
-    const TapT<T>* tp = staged ? s_taps : taps;
+    constexpr int kRound = sizeof(T) == 8 ? kGenericSmemTaps / 2 : kGenericSmemTaps;   // taps per round
+    __shared__ TapT<T> s_raw[kRound];            // the taps as given (staged once when they fit)
+    __shared__ ResolvedTap<T> s_tap[kRound];     // ... resolved for the current row
 
+    const bool staged = ntaps <= kRound;
+    if (staged) {
+        for (int t = threadIdx.x; t < ntaps; t += kGenericThreads) s_raw[t] = taps[t];
+    }
     const int xblocks = (g.nx + kGenericThreads - 1) / kGenericThreads;
-    const int64_t nsegments = (int64_t)xblocks * g.ny * g.nz;
-    for (int64_t seg = blockIdx.x; seg < nsegments; seg += gridDim.x) {
+    const long long nsegments = (long long)xblocks * g.ny * g.nz;
+    // every CTA takes a contiguous run of segments (x fastest, then y): the rows above and below
+    // a row are then read by the same CTA one step earlier or later and hit in L1
+    const long long per_cta = (nsegments + gridDim.x - 1) / gridDim.x;
+    const long long seg_end = min(nsegments, (long long)(blockIdx.x + 1) * per_cta);
+    for (long long seg = (long long)blockIdx.x * per_cta; seg < seg_end; ++seg) {
         const int xb = (int)(seg % xblocks);
-        const int64_t row = seg / xblocks;                 // = z * ny + y
+        const long long row = seg / xblocks;                 // = z * ny + y
         const int y = (int)(row % g.ny);
         const int z = (int)(row / g.ny);
-        const int x = xb * kGenericThreads + threadIdx.x;
-        if (x < g.nx) {
-            T acc = T(0);
-            for (int t = 0; t < ntaps; ++t) {
-                const TapT<T> tap = tp[t];
-                int qz = z + tap.dz, qy = y + tap.dy, qx = x + tap.dx;
+        const int x = min(xb * kGenericThreads + (int)threadIdx.x, g.nx - 1);   // idle lanes shadow the last point
+        const long long self = row * g.nx + x;
+        T acc = T(0);
+        for (int t0 = 0; t0 < ntaps; t0 += kRound) {
+            const int nt = min(kRound, ntaps - t0);
+            __syncthreads();                                 // taps staged / previous round no longer read
+            for (int t = threadIdx.x; t < nt; t += kGenericThreads) {
+                const TapT<T> tap = staged ? s_raw[t] : taps[t0 + t];
+                int qz = z + tap.dz, qy = y + tap.dy;
+                bool inside = true;
                 if (kPeriodic) {
-                    qz = wrap_index(qz, g.nz);             // the same for the whole CTA
+                    qz = wrap_index(qz, g.nz);
                     qy = wrap_index(qy, g.ny);
+                } else {
+                    inside = (unsigned)qz < (unsigned)g.nz && (unsigned)qy < (unsigned)g.ny;
+                }
+                ResolvedTap<T> r;
+                r.row = inside ? ((long long)qz * g.ny + qy) * g.nx : -1;
+                r.dx = tap.dx;
+                r.w = tap.w;
+                s_tap[t] = r;
+            }
+            __syncthreads();
+            // Branch-free inner loop so that several loads are in flight per thread: a tap that
+            // leaves the grid reads the thread's own point with weight zero.
+#pragma unroll 4
+            for (int t = 0; t < nt; ++t) {
+                const ResolvedTap<T> r = s_tap[t];
+                int qx = x + r.dx;
+                bool ok = r.row >= 0;
+                if (kPeriodic) {
                     if (qx < 0 || qx >= g.nx) qx = wrap_index(qx, g.nx);
                 } else {
-                    if ((unsigned)qz >= (unsigned)g.nz || (unsigned)qy >= (unsigned)g.ny) continue;
-                    if ((unsigned)qx >= (unsigned)g.nx) continue;
+                    ok = ok && (unsigned)qx < (unsigned)g.nx;
                 }
-                acc = fma_t(tap.w, __ldg(in + ((int64_t)qz * g.ny + qy) * g.nx + qx), acc);
+                const T v = __ldg(in + (ok ? r.row + qx : self));
+                acc = fma_t(ok ? r.w : T(0), v, acc);
             }
-            out[row * g.nx + x] = acc;
         }
+        if (xb * kGenericThreads + (int)threadIdx.x < g.nx) out[self] = acc;
     }
 }
 
 // Grid size for a launch of the kernel above: a few resident waves of CTAs that loop over the
-// row segments (one CTA per segment would spend its time on CTA turnover and tap staging).
+// row segments.
 inline int generic_grid_size(const Grid& g, int sm_count) {
-    const int64_t xblocks = (g.nx + kGenericThreads - 1) / kGenericThreads;
-    const int64_t nsegments = xblocks * g.ny * g.nz;
-    const int64_t cap = (int64_t)sm_count * 8 * 4;
+    const long long xblocks = (g.nx + kGenericThreads - 1) / kGenericThreads;
+    const long long nsegments = xblocks * g.ny * g.nz;
+    const long long cap = (long long)sm_count * 8 * 4;
     return (int)(nsegments < cap ? nsegments : cap);
 }
 
