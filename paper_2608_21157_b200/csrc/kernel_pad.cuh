@@ -32,4 +32,38 @@ stencil_pad_periodic_kernel(const float* __restrict__ in, float* __restrict__ pa
     }
 }
 
+// Rows whose length is not a multiple of 16 bytes (4 floats, 2 doubles): the tiled kernels need a 16-byte row pitch
+// (a TMA stride rule, and their 128-bit stores), so such a grid is swept between two grids
+// with padded rows.  This kernel copies into and out of that layout (rows of `nx` values from
+// one pitch to another); `lanes` (a power of two, at most the CTA size) threads share a row, the CTA's other threads take further rows.
+// The tail columns of a padded row are never read as grid cells (the tensor map ends at nx),
+// so they are left as they are.
+template <typename T>
+__global__ void __launch_bounds__(256)
+stencil_repitch_rows_kernel(const T* __restrict__ src, T* __restrict__ dst, int64_t rows, int nx,
+                            int src_pitch, int dst_pitch, int lanes_log2) {
+    const int lanes = 1 << lanes_log2;
+    const int lx = threadIdx.x & (lanes - 1);
+    const int sub = threadIdx.x >> lanes_log2;
+    const int rows_per_cta = blockDim.x >> lanes_log2;
+    const int64_t group = (int64_t)gridDim.x * rows_per_cta;       // rows the grid takes per round
+    constexpr int kRows = 4;                                       // rows per thread and round: loads in flight
+    for (int64_t row = (int64_t)blockIdx.x * rows_per_cta + sub; row < rows; row += kRows * group) {
+#pragma unroll 2
+        for (int x = lx; x < nx; x += lanes) {
+            T v[kRows];
+#pragma unroll
+            for (int j = 0; j < kRows; ++j) {
+                const int64_t r = row + j * group;
+                v[j] = r < rows ? src[r * src_pitch + x] : T(0);
+            }
+#pragma unroll
+            for (int j = 0; j < kRows; ++j) {
+                const int64_t r = row + j * group;
+                if (r < rows) dst[r * dst_pitch + x] = v[j];
+            }
+        }
+    }
+}
+
 }  // namespace stencil

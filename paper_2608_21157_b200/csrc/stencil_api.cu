@@ -175,7 +175,10 @@ struct stencil_plan_s {
     Tap* d_taps;
     int* d_status;
     float* scratch;                // N floats, iteration ping-pong
-    float* pad;                    // padded copy of the input (periodic boundary on the tiled kernels)
+    float* pad;                    // padded copy of the input (periodic boundary on the tiled kernels;
+                                   // first of the two padded-row grids when nx is not a multiple of 4)
+    float* pad2;                   // second padded-row grid
+    int tmap_nx;                   // non-zero while a padded-row sweep runs: the true row length
     float* host_in;                // N floats each, apply_host staging
     float* host_out;
     cudaStream_t copy_in, copy_out; // apply_host: upload / download streams (created on first use)
@@ -369,9 +372,11 @@ const Rows2DConfig* find_rows2d_cfg(int radius, bool box) {
 
 // The tiled kernels need rows whose byte length is a multiple of 16 (a TMA stride rule).
 // The zero boundary comes from TMA's zero fill of out-of-grid cells; a periodic grid is first
-// copied into a padded grid with wrapped halos (kernel_pad.cuh) and swept from there.
+// copied into a padded grid with wrapped halos (kernel_pad.cuh) and swept from there.  A
+// zero-boundary grid with other row lengths is swept between two grids with padded rows
+// (apply_row_padded).
 bool stream_supported(const stencil_plan_s* p) {
-    if (p->nx % 4 != 0) return false;
+    if (p->nx % 4 != 0 && p->boundary != STENCIL_ZERO) return false;
     const bool box = p->shape == STENCIL_BOX;
     if (p->ndim == 2) return find_rows2d_cfg(p->radius, box) != nullptr;
     return find_stream_cfg(p->radius, box, 0, 0) != nullptr;
@@ -381,6 +386,7 @@ bool stream_supported(const stencil_plan_s* p) {
 const FusedConfig* pick_fused(const stencil_plan_s* p) {
     if (!stream_supported(p) || p->shape != STENCIL_STAR || p->ndim != 3) return nullptr;
     if (p->boundary != STENCIL_ZERO) return nullptr;      // fused passes re-impose a ZERO exterior
+    if (p->nx % 4 != 0) return nullptr;                   // ... over the row pitch, which padded rows exceed
     if (p->fuse_steps == 1) return nullptr;
     int txe = p->tile_x;
     if (p->fuse_steps == 0 && txe == 0 && p->fused_tile_y == 0) {
@@ -490,13 +496,15 @@ int launch_generic(stencil_plan_s* p, const float* src, float* dst, cudaStream_t
 int get_tensor_map(stencil_plan_s* p, const void* cfg, int box_x, int box_y, const float* src,
                    const CUtensorMap** out, int tnx = 0, int tny = 0, int tnz = 0) {
     if (tnx == 0) { tnx = p->nx; tny = p->ny; tnz = p->nz; }     // extents of the tensor `src` points at
+    // padded rows: the pitch is tnx, the cells past the true row length read as out of grid (zero)
+    const int row_cells = p->tmap_nx > 0 ? p->tmap_nx : tnx;
     for (auto& e : p->maps)
         if (e.ptr == src && e.cfg == cfg) { *out = &e.map; return STENCIL_OK; }
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return STENCIL_ERR_CUDA;
     stencil_plan_s::MapEntry e;
     e.ptr = src; e.cfg = cfg;
-    const cuuint64_t dims[3] = {(cuuint64_t)tnx, (cuuint64_t)tny, (cuuint64_t)tnz};
+    const cuuint64_t dims[3] = {(cuuint64_t)row_cells, (cuuint64_t)tny, (cuuint64_t)tnz};
     const cuuint64_t strides[2] = {(cuuint64_t)tnx * 4, (cuuint64_t)tnx * (cuuint64_t)tny * 4};
     const cuuint32_t box[3] = {(cuuint32_t)box_x, (cuuint32_t)box_y, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
@@ -820,6 +828,49 @@ int launch_sweep(stencil_plan_s* p, const float* src, float* dst, cudaStream_t s
     }
 }
 
+template <typename T>
+int repitch_rows(stencil_plan_s* p, const T* src, T* dst, int nx, int src_pitch, int dst_pitch,
+                 cudaStream_t st) {
+    const int64_t rows = (int64_t)p->nz * p->ny;
+    int lanes_log2 = 0;
+    while ((1 << lanes_log2) < nx && lanes_log2 < 8) ++lanes_log2;
+    const int rows_per_cta = 256 >> lanes_log2;
+    const int64_t ctas = (rows + 4 * rows_per_cta - 1) / (4 * rows_per_cta);      // a thread takes 4 rows per round
+    const int grid = (int)std::min<int64_t>(ctas, (int64_t)sm_count() * 16);
+    stencil_repitch_rows_kernel<T><<<grid, 256, 0, st>>>(src, dst, rows, nx, src_pitch, dst_pitch, lanes_log2);
+    if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
+    p->launches++;
+    return STENCIL_OK;
+}
+
+// Zero-boundary grid whose rows are not a multiple of 4 floats, on the tiled kernels: copy `in`
+// into a grid with padded rows, sweep `steps` times between that grid and a second one, copy
+// the result into `out`.  While the sweeps run the plan's row length is the padded one (pitch
+// of both grids, tile counts, store bounds) and the tensor maps end every row at the true
+// length, so the cells the kernels write into the padding never enter a later sweep.
+int apply_row_padded(stencil_plan_s* p, const float* in, float* out, int steps, cudaStream_t st) {
+    const int nx = p->nx, pitch = (nx + 3) & ~3;
+    const int64_t cells = (int64_t)p->nz * p->ny * pitch;
+    int rc;
+    if ((rc = ensure_grid(&p->pad, cells)) != STENCIL_OK) return rc;
+    if ((rc = ensure_grid(&p->pad2, cells)) != STENCIL_OK) return rc;
+    if ((rc = repitch_rows(p, in, p->pad, nx, nx, pitch, st)) != STENCIL_OK) return rc;
+    float* src = p->pad;
+    float* dst = p->pad2;
+    p->nx = pitch;
+    p->tmap_nx = nx;
+    for (int k = 0; k < steps && rc == STENCIL_OK; ++k) {
+        p->chained = p->chain_launches && k > 0;
+        rc = launch_sweep(p, src, dst, st);
+        std::swap(src, dst);
+    }
+    p->chained = false;
+    p->nx = nx;
+    p->tmap_nx = 0;
+    if (rc != STENCIL_OK) return rc;
+    return repitch_rows(p, src, out, nx, pitch, nx, st);
+}
+
 
 // ---------------------------------------------------------------------------
 // FP64 plans: the generic kernel for everything, the row-streaming kernel for
@@ -860,7 +911,7 @@ const std::vector<Rows2D64Config>& rows2d64_configs() {
 }
 
 const Rows2D64Config* find_rows2d64_cfg(const stencil_plan_s* p) {
-    if (p->ndim != 2 || p->boundary != STENCIL_ZERO || p->nx % 2 != 0) return nullptr;   // 16-byte rows
+    if (p->ndim != 2 || p->boundary != STENCIL_ZERO) return nullptr;   // odd rows: apply_row_padded_f64
     for (const Rows2D64Config& c : rows2d64_configs())
         if (c.radius == p->radius && c.box == (p->shape == STENCIL_BOX)) return &c;
     return nullptr;
@@ -917,7 +968,7 @@ const std::vector<Stream64Config>& stream64_configs() {
 }
 
 const Stream64Config* find_stream64_cfg(const stencil_plan_s* p) {
-    if (p->ndim != 3 || p->boundary != STENCIL_ZERO || p->nx % 2 != 0) return nullptr;   // 16-byte rows
+    if (p->ndim != 3 || p->boundary != STENCIL_ZERO) return nullptr;   // odd rows: apply_row_padded_f64
     for (const Stream64Config& c : stream64_configs())
         if (c.radius == p->radius && c.box == (p->shape == STENCIL_BOX)) return &c;
     return nullptr;
@@ -947,7 +998,9 @@ int get_tensor_map_f64(stencil_plan_s* p, const void* cfg, int box_x, int box_y,
     if (!enc) return STENCIL_ERR_CUDA;
     stencil_plan_s::MapEntry e;
     e.ptr = key; e.cfg = cfg;
-    const cuuint64_t dims[3] = {(cuuint64_t)p->nx, (cuuint64_t)p->ny, (cuuint64_t)p->nz};
+    // padded rows: the pitch is p->nx, the cell past the true row length reads as out of grid (zero)
+    const cuuint64_t dims[3] = {(cuuint64_t)(p->tmap_nx > 0 ? p->tmap_nx : p->nx), (cuuint64_t)p->ny,
+                                (cuuint64_t)p->nz};
     const cuuint64_t strides[2] = {(cuuint64_t)p->nx * 8, (cuuint64_t)p->nx * (cuuint64_t)p->ny * 8};
     const cuuint32_t box[3] = {(cuuint32_t)box_x, (cuuint32_t)box_y, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
@@ -1064,6 +1117,31 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
     return STENCIL_OK;
 }
 
+// FP64 twin of apply_row_padded: rows of an odd number of doubles, pitch rounded up to even.
+// The two padded grids live in the same plan slots, sized in doubles.
+int apply_row_padded_f64(stencil_plan_s* p, const double* in, double* out, int steps, cudaStream_t st) {
+    const int nx = p->nx, pitch = nx + 1;
+    const int64_t cells = (int64_t)p->nz * p->ny * pitch;
+    int rc;
+    if ((rc = ensure_grid(&p->pad, 2 * cells)) != STENCIL_OK) return rc;
+    if ((rc = ensure_grid(&p->pad2, 2 * cells)) != STENCIL_OK) return rc;
+    double* src = reinterpret_cast<double*>(p->pad);
+    double* dst = reinterpret_cast<double*>(p->pad2);
+    if ((rc = repitch_rows(p, in, src, nx, nx, pitch, st)) != STENCIL_OK) return rc;
+    p->nx = pitch;
+    p->tmap_nx = nx;
+    for (int k = 0; k < steps && rc == STENCIL_OK; ++k) {
+        p->chained = p->chain_launches && k > 0;
+        rc = launch_sweep_f64(p, src, dst, st);
+        std::swap(src, dst);
+    }
+    p->chained = false;
+    p->nx = nx;
+    p->tmap_nx = 0;
+    if (rc != STENCIL_OK) return rc;
+    return repitch_rows(p, static_cast<const double*>(src), out, nx, pitch, nx, st);
+}
+
 bool valid_plan(const stencil_plan_s* p) { return p && p->magic == kPlanMagic; }
 
 // ---------------------------------------------------------------------------
@@ -1099,7 +1177,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->npoints = n;
     p->radius = radius; p->shape = shape; p->boundary = boundary;
     p->device = -1;
-    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr;
+    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0;
     p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr;
     p->host_in = nullptr; p->host_out = nullptr;
     p->copy_in = nullptr; p->copy_out = nullptr;
@@ -1215,6 +1293,7 @@ int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void
         }
         return STENCIL_OK;
     }
+    if (p->variant == STENCIL_VARIANT_STREAM && p->nx % 4 != 0) return apply_row_padded(p, in, out, steps, st);
     if (steps > 1) {
         rc = ensure_grid(&p->scratch, p->npoints);
         if (rc != STENCIL_OK) return rc;
@@ -1259,6 +1338,7 @@ int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps
         }
         return STENCIL_OK;
     }
+    if (p->variant == STENCIL_VARIANT_STREAM && p->nx % 2 != 0) return apply_row_padded_f64(p, in, out, steps, st);
     if (steps > 1 && !p->scratch64) {
         if (cudaMalloc(&p->scratch64, bytes) != cudaSuccess) {
             cudaGetLastError();
@@ -1295,7 +1375,7 @@ int stencil_apply_host(stencil_plan_t p, const float* in_host, float* out_host, 
     const int min_planes = std::max(2 * p->radius, 8);           // per slab
     const int kSlabs = p->nz >= kMaxSlabs * 2 * min_planes ? kMaxSlabs : kMaxSlabs / 2;
     const bool pipelined = steps == 1 && p->variant == STENCIL_VARIANT_STREAM && p->ndim == 3 &&
-                           p->boundary == STENCIL_ZERO &&
+                           p->boundary == STENCIL_ZERO && p->nx % 4 == 0 &&
                            p->nz >= kSlabs * min_planes;
     if (!pipelined) {
         if (cudaMemcpyAsync(p->host_in, in_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
@@ -1407,13 +1487,13 @@ int stencil_destroy(stencil_plan_t p) {
     if (!valid_plan(p)) return STENCIL_ERR_INVALID;
     int rc = STENCIL_OK;
     if (p->d_status || p->scratch || p->host_in || p->host_out || p->d_taps || p->d_taps64 || p->scratch64 ||
-        p->pad) {
+        p->pad || p->pad2) {
         int cur = -1;
         cudaGetDevice(&cur);
         if (p->device >= 0 && cur != p->device) cudaSetDevice(p->device);
         if (p->used) cudaStreamSynchronize(p->last_stream);
         void* ptrs[] = {p->d_status, p->scratch, p->host_in, p->host_out, p->d_taps, p->d_taps64, p->scratch64,
-                        p->pad};
+                        p->pad, p->pad2};
         for (void* q : ptrs)
             if (q && cudaFree(q) != cudaSuccess) rc = STENCIL_ERR_CUDA;
         for (cudaEvent_t e : p->events) cudaEventDestroy(e);
@@ -1571,9 +1651,14 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
             int64_t grids = (p->scratch != nullptr) + (p->host_in != nullptr) + (p->host_out != nullptr);
             *value = grids * p->npoints * (int64_t)sizeof(float) +
                      (p->scratch64 ? p->npoints * (int64_t)sizeof(double) : 0) +
-                     (p->pad ? (int64_t)(p->nx + 2 * kPadX) * (p->ny + 2 * p->radius) *
-                                   (p->nz + (p->ndim == 3 ? 2 * p->radius : 0)) * (int64_t)sizeof(float)
-                             : 0);
+                     (p->pad && p->boundary == STENCIL_PERIODIC
+                          ? (int64_t)(p->nx + 2 * kPadX) * (p->ny + 2 * p->radius) *
+                                (p->nz + (p->ndim == 3 ? 2 * p->radius : 0)) * (int64_t)sizeof(float)
+                          : 0) +
+                     ((p->pad != nullptr && p->boundary == STENCIL_ZERO) + (p->pad2 != nullptr)) *
+                         (int64_t)p->nz * p->ny *
+                         (p->f64 ? (int64_t)(p->nx + 1) * (int64_t)sizeof(double)
+                                 : (int64_t)((p->nx + 3) & ~3) * (int64_t)sizeof(float));
             return STENCIL_OK;
         }
         case STENCIL_KEY_CHUNK_Z: *value = p->chunk_z; return STENCIL_OK;

@@ -107,8 +107,11 @@ def test_variant_selection_rules():
         assert p.variant == "stream"
         p.set(b.KEY_VARIANT, b.VARIANT_GENERIC)
         assert p.variant == "generic"
-    with b.Plan((64, 64, 66), 1, b.STAR, star, b.ZERO) as p:       # nx % 4 != 0
-        assert p.variant == "generic"
+    with b.Plan((64, 64, 66), 1, b.STAR, star, b.ZERO) as p:       # nx % 4 != 0: swept between grids with padded rows
+        assert p.variant == "stream"
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # no temporal blocking over padded rows
+    with b.Plan((64, 64, 66), 5, b.STAR, wl.star_weights(3, 5, -6.0, [1.0] * 5), b.ZERO) as p:
+        assert p.variant == "generic"               # radius beyond the tiled kernels
         with pytest.raises(b.StencilError) as e:
             p.set(b.KEY_VARIANT, b.VARIANT_STREAM)
         assert e.value.status == b.ERR_UNSUPPORTED
@@ -118,6 +121,9 @@ def test_variant_selection_rules():
         assert p.get(b.KEY_FUSE_STEPS) == 1         # no temporal blocking under a periodic boundary
     with b.Plan((64, 64, 62), 1, b.STAR, star, b.PERIODIC) as p:
         assert p.variant == "generic"
+        with pytest.raises(b.StencilError) as e:
+            p.set(b.KEY_VARIANT, b.VARIANT_STREAM)
+        assert e.value.status == b.ERR_UNSUPPORTED
     with b.Plan((64, 64), 1, b.STAR, wl.star_weights(2, 1, -4.0, [1.0]), b.ZERO) as p:
         assert p.variant in ("generic", "stream")
     with b.Plan((64, 64, 64), 1, b.STAR, star, b.ZERO) as p:
