@@ -10,25 +10,33 @@ namespace stencil {
 
 constexpr int kPadX = 4;            // halo columns per side of the padded copy
 
-// pad[z'][y'][x'] = in[(z' - rz) mod nz][(y' - ry) mod ny][(x' - 4) mod nx], one float4 per thread.
-// rz = 0 for 2D grids (nz = 1).  nx is a multiple of 4, so every float4 wraps as a whole.
+template <typename T> struct Vec16;                          // the 16-byte vector of a grid's value type
+template <> struct Vec16<float>  { using type = float4;  static constexpr int n = 4; };
+template <> struct Vec16<double> { using type = double2; static constexpr int n = 2; };
+
+// pad[z'][y'][x'] = in[(z' - rz) mod nz][(y' - ry) mod ny][(x' - 4) mod nx], one 16-byte vector per
+// thread.  rz = 0 for 2D grids (nz = 1).  A row is a whole number of vectors (nx a multiple of 4 for
+// fp32, of 2 for FP64), so every vector wraps as a whole.
+template <typename T>
 __global__ void __launch_bounds__(256)
-stencil_pad_periodic_kernel(const float* __restrict__ in, float* __restrict__ pad, Grid g, int ry, int rz) {
-    const int px4 = (g.nx + 2 * kPadX) / 4;
-    const int nx4 = g.nx / 4;
+stencil_pad_periodic_kernel(const T* __restrict__ in, T* __restrict__ pad, Grid g, int ry, int rz) {
+    using V = typename Vec16<T>::type;
+    constexpr int n = Vec16<T>::n;
+    const int pxv = (g.nx + 2 * kPadX) / n;
+    const int nxv = g.nx / n;
     const int py = g.ny + 2 * ry, pz = g.nz + 2 * rz;
-    const int64_t total = (int64_t)px4 * py * pz;          // float4 cells of the padded grid
+    const int64_t total = (int64_t)pxv * py * pz;          // vectors of the padded grid
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    const float4* src = reinterpret_cast<const float4*>(in);
-    float4* dst = reinterpret_cast<float4*>(pad);
+    const V* src = reinterpret_cast<const V*>(in);
+    V* dst = reinterpret_cast<V*>(pad);
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
-        const int x4 = (int)(i % px4);
-        const int64_t row = i / px4;
+        const int xv = (int)(i % pxv);
+        const int64_t row = i / pxv;
         const int yp = (int)(row % py), zp = (int)(row / py);
         int y = (yp - ry) % g.ny; if (y < 0) y += g.ny;
         int z = (zp - rz) % g.nz; if (z < 0) z += g.nz;
-        int s4 = (x4 - kPadX / 4) % nx4; if (s4 < 0) s4 += nx4;
-        dst[i] = src[((int64_t)z * g.ny + y) * nx4 + s4];
+        int sv = (xv - kPadX / n) % nxv; if (sv < 0) sv += nxv;
+        dst[i] = src[((int64_t)z * g.ny + y) * nxv + sv];
     }
 }
 

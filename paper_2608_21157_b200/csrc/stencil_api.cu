@@ -607,12 +607,13 @@ int choose_chunk(const stencil_plan_s* p, const StreamConfig* cfg, int stages, d
 
 // Periodic boundary: copy `src` into the plan's padded grid (wrapped halos) on `st`.
 // Extents of the padded grid come back through pnx/pny/pnz.
-int pad_periodic(stencil_plan_s* p, const float* src, cudaStream_t st, int* pnx, int* pny, int* pnz) {
+template <typename T>
+int pad_periodic(stencil_plan_s* p, const T* src, cudaStream_t st, int* pnx, int* pny, int* pnz) {
     const int R = p->radius;
     const int rz = p->ndim == 3 ? R : 0;
     *pnx = p->nx + 2 * kPadX; *pny = p->ny + 2 * R; *pnz = p->nz + 2 * rz;
     if (!p->pad) {
-        const size_t bytes = (size_t)*pnx * *pny * *pnz * sizeof(float);
+        const size_t bytes = (size_t)*pnx * *pny * *pnz * sizeof(T);
         if (cudaMalloc(&p->pad, bytes) != cudaSuccess) {
             cudaGetLastError();
             p->pad = nullptr;
@@ -620,9 +621,9 @@ int pad_periodic(stencil_plan_s* p, const float* src, cudaStream_t st, int* pnx,
         }
     }
     Grid g{p->nz, p->ny, p->nx};
-    const int64_t cells = (int64_t)(*pnx / 4) * *pny * *pnz;
+    const int64_t cells = (int64_t)(*pnx / Vec16<T>::n) * *pny * *pnz;
     const int grid = (int)std::min<int64_t>((cells + 255) / 256, (int64_t)sm_count() * 32);
-    stencil_pad_periodic_kernel<<<grid, 256, 0, st>>>(src, p->pad, g, R, rz);
+    stencil_pad_periodic_kernel<T><<<grid, 256, 0, st>>>(src, reinterpret_cast<T*>(p->pad), g, R, rz);
     if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
     p->launches++;
     return STENCIL_OK;
@@ -911,7 +912,7 @@ const std::vector<Rows2D64Config>& rows2d64_configs() {
 }
 
 const Rows2D64Config* find_rows2d64_cfg(const stencil_plan_s* p) {
-    if (p->ndim != 2 || p->boundary != STENCIL_ZERO) return nullptr;   // odd rows: apply_row_padded_f64
+    if (p->ndim != 2 || (p->boundary != STENCIL_ZERO && p->nx % 2 != 0)) return nullptr;   // odd rows: apply_row_padded_f64
     for (const Rows2D64Config& c : rows2d64_configs())
         if (c.radius == p->radius && c.box == (p->shape == STENCIL_BOX)) return &c;
     return nullptr;
@@ -968,7 +969,7 @@ const std::vector<Stream64Config>& stream64_configs() {
 }
 
 const Stream64Config* find_stream64_cfg(const stencil_plan_s* p) {
-    if (p->ndim != 3 || p->boundary != STENCIL_ZERO) return nullptr;   // odd rows: apply_row_padded_f64
+    if (p->ndim != 3 || (p->boundary != STENCIL_ZERO && p->nx % 2 != 0)) return nullptr;   // odd rows: apply_row_padded_f64
     for (const Stream64Config& c : stream64_configs())
         if (c.radius == p->radius && c.box == (p->shape == STENCIL_BOX)) return &c;
     return nullptr;
@@ -990,7 +991,8 @@ int resolve_variant_f64(stencil_plan_s* p, int want) {
 }
 
 int get_tensor_map_f64(stencil_plan_s* p, const void* cfg, int box_x, int box_y, const double* src,
-                       const CUtensorMap** out) {
+                       const CUtensorMap** out, int tnx = 0, int tny = 0, int tnz = 0) {
+    if (tnx == 0) { tnx = p->nx; tny = p->ny; tnz = p->nz; }     // extents of the tensor `src` points at
     const void* key = src;
     for (auto& e : p->maps)
         if (e.ptr == key && e.cfg == cfg) { *out = &e.map; return STENCIL_OK; }
@@ -999,9 +1001,9 @@ int get_tensor_map_f64(stencil_plan_s* p, const void* cfg, int box_x, int box_y,
     stencil_plan_s::MapEntry e;
     e.ptr = key; e.cfg = cfg;
     // padded rows: the pitch is p->nx, the cell past the true row length reads as out of grid (zero)
-    const cuuint64_t dims[3] = {(cuuint64_t)(p->tmap_nx > 0 ? p->tmap_nx : p->nx), (cuuint64_t)p->ny,
-                                (cuuint64_t)p->nz};
-    const cuuint64_t strides[2] = {(cuuint64_t)p->nx * 8, (cuuint64_t)p->nx * (cuuint64_t)p->ny * 8};
+    const cuuint64_t dims[3] = {(cuuint64_t)(p->tmap_nx > 0 ? p->tmap_nx : tnx), (cuuint64_t)tny,
+                                (cuuint64_t)tnz};
+    const cuuint64_t strides[2] = {(cuuint64_t)tnx * 8, (cuuint64_t)tnx * (cuuint64_t)tny * 8};
     const cuuint32_t box[3] = {(cuuint32_t)box_x, (cuuint32_t)box_y, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = enc(&e.map, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, 3, const_cast<double*>(src), dims, strides, box,
@@ -1018,7 +1020,16 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
     if (p->variant == STENCIL_VARIANT_STREAM && p->stream64_cfg) {
         const Stream64Config* cfg = p->stream64_cfg;
         const CUtensorMap* map = nullptr;
-        int rc = get_tensor_map_f64(p, cfg, kStream64PX, cfg->box_rows, src, &map);
+        const bool periodic = p->boundary == STENCIL_PERIODIC;      // swept from a padded copy, as in fp32
+        int rc;
+        if (periodic) {
+            int pnx, pny, pnz;
+            if ((rc = pad_periodic(p, src, st, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
+            rc = get_tensor_map_f64(p, cfg, kStream64PX, cfg->box_rows, reinterpret_cast<const double*>(p->pad),
+                                    &map, pnx, pny, pnz);
+        } else {
+            rc = get_tensor_map_f64(p, cfg, kStream64PX, cfg->box_rows, src, &map);
+        }
         if (rc != STENCIL_OK) return rc;
         const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 4;
         const size_t smem = (size_t)stages * cfg->plane_bytes + 128 + 2 * kMaxStages * sizeof(uint64_t);
@@ -1044,7 +1055,9 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         g.stages = stages;
         g.streaming_store = 0;
         g.z_begin = 0; g.z_end = p->nz;
-        g.in_off_x = 0; g.in_off_y = 0; g.in_off_z = 0;
+        g.in_off_x = periodic ? kPadX : 0;
+        g.in_off_y = periodic ? p->radius : 0;
+        g.in_off_z = periodic ? p->radius : 0;
         g.wait_polls = p->wait_polls; g.drop_plane = -1;
         // many short CTAs, as for the bandwidth-bound fp32 sweeps; the wide stars re-read 2R halo
         // planes per chunk, so they get longer chunks (measured on 512^3)
@@ -1061,7 +1074,16 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
     if (p->variant == STENCIL_VARIANT_STREAM && p->rows2d64_cfg) {
         const Rows2D64Config* cfg = p->rows2d64_cfg;
         const CUtensorMap* map = nullptr;
-        int rc = get_tensor_map_f64(p, cfg, kPX64, cfg->YB, src, &map);
+        const bool periodic = p->boundary == STENCIL_PERIODIC;
+        int rc;
+        if (periodic) {
+            int pnx, pny, pnz;
+            if ((rc = pad_periodic(p, src, st, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
+            rc = get_tensor_map_f64(p, cfg, kPX64, cfg->YB, reinterpret_cast<const double*>(p->pad), &map,
+                                    pnx, pny, pnz);
+        } else {
+            rc = get_tensor_map_f64(p, cfg, kPX64, cfg->YB, src, &map);
+        }
         if (rc != STENCIL_OK) return rc;
         const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
         const size_t smem = (size_t)cfg->NW * stages * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8;
@@ -1084,7 +1106,8 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         g.ny = p->ny; g.nx = p->nx;
         g.strips = (p->nx + kStrip64 - 1) / kStrip64;
         g.stages = stages;
-        g.in_off_x = 0; g.in_off_y = 0;
+        g.in_off_x = periodic ? kPadX : 0;
+        g.in_off_y = periodic ? p->radius : 0;
         int chunk = p->chunk_z;
         if (chunk <= 0) {                             // same sizing rule as the fp32 kernel
             const int R = p->radius;
@@ -1653,7 +1676,8 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
                      (p->scratch64 ? p->npoints * (int64_t)sizeof(double) : 0) +
                      (p->pad && p->boundary == STENCIL_PERIODIC
                           ? (int64_t)(p->nx + 2 * kPadX) * (p->ny + 2 * p->radius) *
-                                (p->nz + (p->ndim == 3 ? 2 * p->radius : 0)) * (int64_t)sizeof(float)
+                                (p->nz + (p->ndim == 3 ? 2 * p->radius : 0)) *
+                                (int64_t)(p->f64 ? sizeof(double) : sizeof(float))
                           : 0) +
                      ((p->pad != nullptr && p->boundary == STENCIL_ZERO) + (p->pad2 != nullptr)) *
                          (int64_t)p->nz * p->ny *

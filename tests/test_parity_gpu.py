@@ -484,6 +484,19 @@ def test_f64_padded_row_sweep(dims, R, box, steps):
     assert used == "stream"
 
 
+@pytest.mark.parametrize("dims,R,box", [
+    ((37, 45, 66), 1, False), ((37, 45, 66), 4, False), ((8, 16, 64), 1, True), ((2, 3, 2), 2, False),
+    ((70, 33, 130), 3, False),
+    ((67, 66), 3, True), ((3, 8), 4, False), ((200, 258), 1, False), ((64, 2), 2, True)])
+def test_f64_periodic_on_the_tiled_kernels(dims, R, box):
+    ndim = len(dims)
+    w = (wl.random_box_weights if box else wl.random_star_weights)(ndim, R, 89, np.float64)
+    a = wl.normal_field(dims, 90, np.float64)
+    for steps in (1, 3):
+        used = check_f64(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps)
+        assert used == "stream"
+
+
 def test_f64_paper_shaped_box_iterated_and_type_checks():
     """The paper's operator in its own precision: 2D box radius 3, FP64, iterated."""
     wk = wl.get("paper2d_f64").scaled((768, 1024), steps=3)
