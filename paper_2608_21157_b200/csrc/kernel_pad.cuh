@@ -40,6 +40,60 @@ stencil_pad_periodic_kernel(const T* __restrict__ in, T* __restrict__ pad, Grid 
     }
 }
 
+// Iterated periodic sweeps stay in the padded layout: a sweep over the whole padded grid
+// (as if it were a zero-boundary grid) leaves correct values in the interior and rubbish in
+// the halo cells, and this kernel rewrites the halo cells from the interior cells they
+// wrap to.  It reads interior cells only and writes halo cells only.  The shell is walked
+// in three parts: whole halo planes, halo rows of the interior planes, halo vectors of the
+// interior rows.
+template <typename T>
+__global__ void __launch_bounds__(256)
+stencil_refresh_halo_kernel(T* __restrict__ pad, Grid g, int ry, int rz) {
+    using V = typename Vec16<T>::type;
+    constexpr int n = Vec16<T>::n;
+    constexpr int hx = kPadX / n;                          // halo vectors per side of a row
+    const int pxv = (g.nx + 2 * kPadX) / n;
+    const int nxv = g.nx / n;
+    const int py = g.ny + 2 * ry;
+    const int64_t part1 = (int64_t)2 * rz * py * pxv;
+    const int64_t part2 = (int64_t)g.nz * 2 * ry * pxv;
+    const int64_t part3 = (int64_t)g.nz * g.ny * 2 * hx;
+    const int64_t total = part1 + part2 + part3;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    V* cells = reinterpret_cast<V*>(pad);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        int zp, yp, xv;                                    // the halo cell, in padded coordinates
+        if (i < part1) {
+            const int64_t plane = (int64_t)py * pxv;
+            const int zi = (int)(i / plane);
+            const int r = (int)(i % plane);
+            zp = zi < rz ? zi : g.nz + zi;
+            yp = r / pxv;
+            xv = r % pxv;
+        } else if (i < part1 + part2) {
+            const int64_t j = i - part1;
+            const int per_z = 2 * ry * pxv;
+            const int r = (int)(j % per_z);
+            const int yi = r / pxv;
+            zp = (int)(j / per_z) + rz;
+            yp = yi < ry ? yi : g.ny + yi;
+            xv = r % pxv;
+        } else {
+            const int64_t j = i - part1 - part2;
+            const int per_z = g.ny * 2 * hx;
+            const int r = (int)(j % per_z);
+            const int c = r % (2 * hx);
+            zp = (int)(j / per_z) + rz;
+            yp = r / (2 * hx) + ry;
+            xv = c < hx ? c : nxv + c;
+        }
+        int z = (zp - rz) % g.nz; if (z < 0) z += g.nz;
+        int y = (yp - ry) % g.ny; if (y < 0) y += g.ny;
+        int sv = (xv - hx) % nxv; if (sv < 0) sv += nxv;
+        cells[((int64_t)zp * py + yp) * pxv + xv] = cells[((int64_t)(z + rz) * py + (y + ry)) * pxv + sv + hx];
+    }
+}
+
 // Rows whose length is not a multiple of 16 bytes (4 floats, 2 doubles): the tiled kernels need a 16-byte row pitch
 // (a TMA stride rule, and their 128-bit stores), so such a grid is swept between two grids
 // with padded rows.  This kernel copies into and out of that layout (rows of `nx` values from

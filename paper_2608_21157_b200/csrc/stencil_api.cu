@@ -179,6 +179,8 @@ struct stencil_plan_s {
                                    // first of the two padded-row grids when nx is not a multiple of 4)
     float* pad2;                   // second padded-row grid
     int tmap_nx;                   // non-zero while a padded-row sweep runs: the true row length
+    bool src_padded;               // set while an iterated periodic apply runs: the source of a sweep is
+                                   // a padded grid with current halos
     float* host_in;                // N floats each, apply_host staging
     float* host_out;
     cudaStream_t copy_in, copy_out; // apply_host: upload / download streams (created on first use)
@@ -606,12 +608,16 @@ int choose_chunk(const stencil_plan_s* p, const StreamConfig* cfg, int stages, d
 }
 
 // Periodic boundary: copy `src` into the plan's padded grid (wrapped halos) on `st`.
-// Extents of the padded grid come back through pnx/pny/pnz.
+// The padded grid and its extents come back through padded and pnx/pny/pnz.  Inside an
+// iterated apply `src` already is a padded grid with current halos (apply_periodic) and
+// comes back as it is.
 template <typename T>
-int pad_periodic(stencil_plan_s* p, const T* src, cudaStream_t st, int* pnx, int* pny, int* pnz) {
+int pad_periodic(stencil_plan_s* p, const T* src, cudaStream_t st, const T** padded, int* pnx, int* pny,
+                 int* pnz) {
     const int R = p->radius;
     const int rz = p->ndim == 3 ? R : 0;
     *pnx = p->nx + 2 * kPadX; *pny = p->ny + 2 * R; *pnz = p->nz + 2 * rz;
+    if (p->src_padded) { *padded = src; return STENCIL_OK; }
     if (!p->pad) {
         const size_t bytes = (size_t)*pnx * *pny * *pnz * sizeof(T);
         if (cudaMalloc(&p->pad, bytes) != cudaSuccess) {
@@ -626,6 +632,7 @@ int pad_periodic(stencil_plan_s* p, const T* src, cudaStream_t st, int* pnx, int
     stencil_pad_periodic_kernel<T><<<grid, 256, 0, st>>>(src, reinterpret_cast<T*>(p->pad), g, R, rz);
     if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
     p->launches++;
+    *padded = reinterpret_cast<const T*>(p->pad);
     return STENCIL_OK;
 }
 
@@ -655,8 +662,9 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     int rc;
     if (periodic) {
         int pnx, pny, pnz;
-        if ((rc = pad_periodic(p, src, st, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
-        rc = get_tensor_map(p, cfg, kStreamPX, cfg->box_rows, p->pad, &map, pnx, pny, pnz);
+        const float* padded = nullptr;
+        if ((rc = pad_periodic(p, src, st, &padded, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
+        rc = get_tensor_map(p, cfg, kStreamPX, cfg->box_rows, padded, &map, pnx, pny, pnz);
     } else {
         rc = get_tensor_map(p, cfg, kStreamPX, cfg->box_rows, src, &map);
     }
@@ -695,8 +703,9 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     int rc;
     if (periodic) {
         int pnx, pny, pnz;
-        if ((rc = pad_periodic(p, src, st, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
-        rc = get_tensor_map(p, cfg, kStreamPX, cfg->YB, p->pad, &map, pnx, pny, pnz);
+        const float* padded = nullptr;
+        if ((rc = pad_periodic(p, src, st, &padded, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
+        rc = get_tensor_map(p, cfg, kStreamPX, cfg->YB, padded, &map, pnx, pny, pnz);
     } else {
         rc = get_tensor_map(p, cfg, kStreamPX, cfg->YB, src, &map);
     }
@@ -1024,9 +1033,9 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         int rc;
         if (periodic) {
             int pnx, pny, pnz;
-            if ((rc = pad_periodic(p, src, st, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
-            rc = get_tensor_map_f64(p, cfg, kStream64PX, cfg->box_rows, reinterpret_cast<const double*>(p->pad),
-                                    &map, pnx, pny, pnz);
+            const double* padded = nullptr;
+            if ((rc = pad_periodic(p, src, st, &padded, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
+            rc = get_tensor_map_f64(p, cfg, kStream64PX, cfg->box_rows, padded, &map, pnx, pny, pnz);
         } else {
             rc = get_tensor_map_f64(p, cfg, kStream64PX, cfg->box_rows, src, &map);
         }
@@ -1078,9 +1087,9 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         int rc;
         if (periodic) {
             int pnx, pny, pnz;
-            if ((rc = pad_periodic(p, src, st, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
-            rc = get_tensor_map_f64(p, cfg, kPX64, cfg->YB, reinterpret_cast<const double*>(p->pad), &map,
-                                    pnx, pny, pnz);
+            const double* padded = nullptr;
+            if ((rc = pad_periodic(p, src, st, &padded, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
+            rc = get_tensor_map_f64(p, cfg, kPX64, cfg->YB, padded, &map, pnx, pny, pnz);
         } else {
             rc = get_tensor_map_f64(p, cfg, kPX64, cfg->YB, src, &map);
         }
@@ -1138,6 +1147,48 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
     if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
     p->launches++;
     return STENCIL_OK;
+}
+
+int sweep_any(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) { return launch_sweep(p, src, dst, st); }
+int sweep_any(stencil_plan_s* p, const double* src, double* dst, cudaStream_t st) {
+    return launch_sweep_f64(p, src, dst, st);
+}
+
+// Iterated periodic apply on the tiled kernels.  `in` is copied once into a padded grid with
+// wrapped halos.  Every step but the last sweeps the whole padded grid as if it were a grid
+// with a zero boundary (the interior comes out right, the halo cells do not) into a second
+// padded grid and then rewrites that grid's halo cells from its interior; the last step reads
+// the padded grid with shifted coordinates and writes `out`.  Per step: one sweep over a
+// slightly larger grid and a copy of the halo shell, instead of a padded copy of everything.
+template <typename T>
+int apply_periodic(stencil_plan_s* p, const T* in, T* out, int steps, cudaStream_t st) {
+    const int R = p->radius, rz = p->ndim == 3 ? R : 0;
+    int pnx, pny, pnz, rc;
+    const T* padded = nullptr;
+    if ((rc = pad_periodic(p, in, st, &padded, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
+    const int64_t cells = (int64_t)pnx * pny * pnz;
+    if ((rc = ensure_grid(&p->pad2, cells * (int64_t)(sizeof(T) / sizeof(float)))) != STENCIL_OK) return rc;
+    T* a = reinterpret_cast<T*>(p->pad);
+    T* b = reinterpret_cast<T*>(p->pad2);
+    const Grid g{p->nz, p->ny, p->nx};
+    const int nz = p->nz, ny = p->ny, nx = p->nx;
+    const int64_t shell = cells / Vec16<T>::n - (int64_t)nz * ny * (nx / Vec16<T>::n);
+    const int shell_grid = (int)std::max<int64_t>(1, std::min<int64_t>((shell + 255) / 256, (int64_t)sm_count() * 16));
+    for (int k = 0; k + 1 < steps && rc == STENCIL_OK; ++k) {
+        p->nz = pnz; p->ny = pny; p->nx = pnx; p->boundary = STENCIL_ZERO;
+        rc = sweep_any(p, static_cast<const T*>(a), b, st);
+        p->nz = nz; p->ny = ny; p->nx = nx; p->boundary = STENCIL_PERIODIC;
+        if (rc != STENCIL_OK) break;
+        stencil_refresh_halo_kernel<T><<<shell_grid, 256, 0, st>>>(b, g, R, rz);
+        if (cudaGetLastError() != cudaSuccess) rc = STENCIL_ERR_CUDA;
+        p->launches++;
+        std::swap(a, b);
+    }
+    if (rc != STENCIL_OK) return rc;
+    p->src_padded = true;
+    rc = sweep_any(p, static_cast<const T*>(a), out, st);
+    p->src_padded = false;
+    return rc;
 }
 
 // FP64 twin of apply_row_padded: rows of an odd number of doubles, pitch rounded up to even.
@@ -1200,7 +1251,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->npoints = n;
     p->radius = radius; p->shape = shape; p->boundary = boundary;
     p->device = -1;
-    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0;
+    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0; p->src_padded = false;
     p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr;
     p->host_in = nullptr; p->host_out = nullptr;
     p->copy_in = nullptr; p->copy_out = nullptr;
@@ -1317,6 +1368,8 @@ int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void
         return STENCIL_OK;
     }
     if (p->variant == STENCIL_VARIANT_STREAM && p->nx % 4 != 0) return apply_row_padded(p, in, out, steps, st);
+    if (p->variant == STENCIL_VARIANT_STREAM && p->boundary == STENCIL_PERIODIC && steps > 1)
+        return apply_periodic(p, in, out, steps, st);
     if (steps > 1) {
         rc = ensure_grid(&p->scratch, p->npoints);
         if (rc != STENCIL_OK) return rc;
@@ -1362,6 +1415,8 @@ int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps
         return STENCIL_OK;
     }
     if (p->variant == STENCIL_VARIANT_STREAM && p->nx % 2 != 0) return apply_row_padded_f64(p, in, out, steps, st);
+    if (p->variant == STENCIL_VARIANT_STREAM && p->boundary == STENCIL_PERIODIC && steps > 1)
+        return apply_periodic(p, in, out, steps, st);
     if (steps > 1 && !p->scratch64) {
         if (cudaMalloc(&p->scratch64, bytes) != cudaSuccess) {
             cudaGetLastError();
@@ -1671,18 +1726,17 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
             return STENCIL_OK;
         case STENCIL_KEY_LAUNCHES: *value = p->launches; return STENCIL_OK;
         case STENCIL_KEY_SCRATCH_BYTES: {
-            int64_t grids = (p->scratch != nullptr) + (p->host_in != nullptr) + (p->host_out != nullptr);
+            const int64_t grids = (p->scratch != nullptr) + (p->host_in != nullptr) + (p->host_out != nullptr);
+            const int64_t elem = p->f64 ? sizeof(double) : sizeof(float);
+            // the padded grids: wrapped halos (periodic) or rows rounded up to 16 bytes (zero boundary)
+            const int64_t padded_grid =
+                p->boundary == STENCIL_PERIODIC
+                    ? (int64_t)(p->nx + 2 * kPadX) * (p->ny + 2 * p->radius) *
+                          (p->nz + (p->ndim == 3 ? 2 * p->radius : 0)) * elem
+                    : (int64_t)p->nz * p->ny * (p->f64 ? (int64_t)(p->nx + 1) : (int64_t)((p->nx + 3) & ~3)) * elem;
             *value = grids * p->npoints * (int64_t)sizeof(float) +
                      (p->scratch64 ? p->npoints * (int64_t)sizeof(double) : 0) +
-                     (p->pad && p->boundary == STENCIL_PERIODIC
-                          ? (int64_t)(p->nx + 2 * kPadX) * (p->ny + 2 * p->radius) *
-                                (p->nz + (p->ndim == 3 ? 2 * p->radius : 0)) *
-                                (int64_t)(p->f64 ? sizeof(double) : sizeof(float))
-                          : 0) +
-                     ((p->pad != nullptr && p->boundary == STENCIL_ZERO) + (p->pad2 != nullptr)) *
-                         (int64_t)p->nz * p->ny *
-                         (p->f64 ? (int64_t)(p->nx + 1) * (int64_t)sizeof(double)
-                                 : (int64_t)((p->nx + 3) & ~3) * (int64_t)sizeof(float));
+                     ((p->pad != nullptr) + (p->pad2 != nullptr)) * padded_grid;
             return STENCIL_OK;
         }
         case STENCIL_KEY_CHUNK_Z: *value = p->chunk_z; return STENCIL_OK;

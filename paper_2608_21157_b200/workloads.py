@@ -256,6 +256,13 @@ def _build_table() -> Dict[str, Workload]:
         lambda: star_weights(3, 1, -6.0, [1.0]),
         _resizable(lambda d: uniform_field(d, -1.0, 1.0, 1), (512, 512, 512)))
 
+    # supplementary: the iterated heat update on a periodic 512^3 grid (stable weights)
+    t["cfg5L_periodic"] = Workload(
+        "cfg5L_periodic", "3D 7-point heat update R=1 512^3, periodic boundary, 16 steps",
+        (512, 512, 512), 1, STAR, PERIODIC, 16,
+        lambda: star_weights(3, 1, 0.4, [0.1]),
+        _resizable(lambda d: uniform_field(d, 0.0, 1.0, 5), (512, 512, 512)))
+
     # supplementary: two of the 3D configs in FP64 (1 GiB per grid)
     t["cfg2_f64"] = Workload(
         "cfg2_f64", "3D 7-point star R=1 512^3 in FP64 (centre -6, neighbours +1), zero boundary, 1 step",

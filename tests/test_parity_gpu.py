@@ -214,8 +214,9 @@ def test_non_default_stream():
 def test_periodic_3d_on_the_tiled_kernel(R, box, dims, chunk_z):
     w = wl.random_box_weights(3, R, 101) if box else wl.random_star_weights(3, R, 101)
     a = wl.normal_field(dims, 102)
-    for steps in (1, 3):
-        used = check(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps, chunk_z=chunk_z or None)
+    for steps in (1, 2, 3, 6):                       # from 2 steps on the sweeps stay in the padded layout
+        used = check(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps, chunk_z=chunk_z or None,
+                     repeat=2 if steps == 3 else 1)
         assert used == "stream"
 
 
@@ -224,8 +225,8 @@ def test_periodic_3d_on_the_tiled_kernel(R, box, dims, chunk_z):
 def test_periodic_2d_on_the_tiled_kernel(R, box, dims):
     w = wl.random_box_weights(2, R, 103) if box else wl.random_star_weights(2, R, 103)
     a = wl.normal_field(dims, 104)
-    for steps in (1, 4):
-        used = check(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps)
+    for steps in (1, 2, 5):
+        used = check(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps, repeat=2 if steps == 5 else 1)
         assert used == "stream"
 
 
@@ -492,7 +493,7 @@ def test_f64_periodic_on_the_tiled_kernels(dims, R, box):
     ndim = len(dims)
     w = (wl.random_box_weights if box else wl.random_star_weights)(ndim, R, 89, np.float64)
     a = wl.normal_field(dims, 90, np.float64)
-    for steps in (1, 3):
+    for steps in (1, 2, 5):
         used = check_f64(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps)
         assert used == "stream"
 
