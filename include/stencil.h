@@ -84,6 +84,11 @@ enum {
                                       while its predecessor drains and waits for it before it
                                       touches global memory; 0 = ordinary launches             */
     STENCIL_KEY_FUSED_TILE_Y = 13,   /* set/get: region height of fused passes, 16 or 32 (0 = auto) */
+    STENCIL_KEY_PERIODIC_ROUTE = 14, /* set/get: how the tiled kernels handle a periodic boundary.
+                                      1 = sweep from a padded copy with wrapped halos; 2 = zero-
+                                      boundary sweep plus a correction of the points within R of
+                                      a face (needs every extent >= 2R, else as 1); 0 (default)
+                                      = whichever of the two is cheaper for the operator          */
     STENCIL_KEY_TEST_DROP_PLANE = 11 /* set/get, test hook: every CTA of the 3D single-step kernel
                                       never loads its input plane of this index, so the bounded
                                       wait for it expires and stencil_query_status reports

@@ -26,7 +26,7 @@ VARIANT_AUTO, VARIANT_GENERIC, VARIANT_STREAM, VARIANT_FUSED = 0, 1, 2, 3
 
 (KEY_VARIANT, KEY_TILE_X, KEY_TILE_Y, KEY_FUSE_STEPS, KEY_LAUNCHES, KEY_SCRATCH_BYTES,
  KEY_CHUNK_Z, KEY_STAGES, KEY_STREAMING_STORE, KEY_ROWS_PER_THREAD, KEY_WAIT_POLLS,
- KEY_TEST_DROP_PLANE, KEY_CHAIN_LAUNCHES, KEY_FUSED_TILE_Y) = range(14)
+ KEY_TEST_DROP_PLANE, KEY_CHAIN_LAUNCHES, KEY_FUSED_TILE_Y, KEY_PERIODIC_ROUTE) = range(15)
 
 #: every symbol include/stencil.h declares
 EXPORTS = (
@@ -186,7 +186,8 @@ class Plan:
             self.set(KEY_VARIANT, variant)
         keys = {"tile_y": KEY_TILE_Y, "chunk_z": KEY_CHUNK_Z, "stages": KEY_STAGES,
                 "fuse_steps": KEY_FUSE_STEPS, "tile_x": KEY_TILE_X, "streaming_store": KEY_STREAMING_STORE,
-                "rows_per_thread": KEY_ROWS_PER_THREAD, "chain_launches": KEY_CHAIN_LAUNCHES, "fused_tile_y": KEY_FUSED_TILE_Y}
+                "rows_per_thread": KEY_ROWS_PER_THREAD, "chain_launches": KEY_CHAIN_LAUNCHES, "fused_tile_y": KEY_FUSED_TILE_Y,
+                "periodic_route": KEY_PERIODIC_ROUTE}
         for name, value in knobs.items():
             if value is not None:
                 self.set(keys[name], value)

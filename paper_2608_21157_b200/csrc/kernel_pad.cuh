@@ -94,6 +94,73 @@ stencil_refresh_halo_kernel(T* __restrict__ pad, Grid g, int ry, int rz) {
     }
 }
 
+// Periodic boundary without a padded copy: a zero-boundary sweep already holds, at every
+// point, the taps that stay inside the grid.  What is missing are the taps that leave it,
+// and only points within R of a face have any.  This kernel walks that shell (whole planes
+// near the z faces, whole rows near the y faces of the other planes, the first and last R
+// points of the other rows) and adds, to each point, its wrapped taps.  Needs every extent
+// of the grid to be at least 2R, so that the three parts are disjoint.
+constexpr int kWrapSmemTaps = 128;
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+stencil_wrap_correction_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g, int R, int rz,
+                               const TapT<T>* __restrict__ taps, int ntaps) {
+    __shared__ TapT<T> s_taps[kWrapSmemTaps];
+    const bool staged = ntaps <= kWrapSmemTaps;
+    if (staged)
+        for (int t = threadIdx.x; t < ntaps; t += blockDim.x) s_taps[t] = taps[t];
+    __syncthreads();
+    const int inner_z = g.nz - 2 * rz, inner_y = g.ny - 2 * R;
+    const int64_t part1 = (int64_t)2 * rz * g.ny * g.nx;
+    const int64_t part2 = (int64_t)inner_z * 2 * R * g.nx;
+    const int64_t part3 = (int64_t)inner_z * inner_y * 2 * R;
+    const int64_t total = part1 + part2 + part3;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        int z, y, x;
+        if (i < part1) {
+            const int64_t plane = (int64_t)g.ny * g.nx;
+            const int zi = (int)(i / plane);
+            const int r = (int)(i % plane);
+            z = zi < rz ? zi : g.nz - 2 * rz + zi;
+            y = r / g.nx;
+            x = r % g.nx;
+        } else if (i < part1 + part2) {
+            const int64_t j = i - part1;
+            const int per_z = 2 * R * g.nx;
+            const int r = (int)(j % per_z);
+            const int yi = r / g.nx;
+            z = (int)(j / per_z) + rz;
+            y = yi < R ? yi : g.ny - 2 * R + yi;
+            x = r % g.nx;
+        } else {
+            const int64_t j = i - part1 - part2;
+            const int64_t per_z = (int64_t)inner_y * 2 * R;
+            const int r = (int)(j % per_z);
+            const int c = r % (2 * R);
+            z = (int)(j / per_z) + rz;
+            y = r / (2 * R) + R;
+            x = c < R ? c : g.nx - 2 * R + c;
+        }
+        T acc = T(0);
+        for (int t = 0; t < ntaps; ++t) {
+            const TapT<T> tap = staged ? s_taps[t] : taps[t];
+            int qz = z + tap.dz, qy = y + tap.dy, qx = x + tap.dx;
+            const bool inside = (unsigned)qz < (unsigned)g.nz && (unsigned)qy < (unsigned)g.ny &&
+                                (unsigned)qx < (unsigned)g.nx;
+            if (inside) continue;                          // the sweep has this tap already
+            // every extent is at least 2R >= |offset|: one step brings the index back
+            qz = qz < 0 ? qz + g.nz : (qz >= g.nz ? qz - g.nz : qz);
+            qy = qy < 0 ? qy + g.ny : (qy >= g.ny ? qy - g.ny : qy);
+            qx = qx < 0 ? qx + g.nx : (qx >= g.nx ? qx - g.nx : qx);
+            acc = fma_t(tap.w, in[((int64_t)qz * g.ny + qy) * g.nx + qx], acc);
+        }
+        const int64_t self = ((int64_t)z * g.ny + y) * g.nx + x;
+        out[self] += acc;
+    }
+}
+
 // Rows whose length is not a multiple of 16 bytes (4 floats, 2 doubles): the tiled kernels need a 16-byte row pitch
 // (a TMA stride rule, and their 128-bit stores), so such a grid is swept between two grids
 // with padded rows.  This kernel copies into and out of that layout (rows of `nx` values from

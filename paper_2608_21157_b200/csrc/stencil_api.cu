@@ -179,6 +179,7 @@ struct stencil_plan_s {
                                    // first of the two padded-row grids when nx is not a multiple of 4)
     float* pad2;                   // second padded-row grid
     int tmap_nx;                   // non-zero while a padded-row sweep runs: the true row length
+    int periodic_route;            // knob: 0 = by measured cost, 1 = padded copy, 2 = wrap correction where it fits
     bool src_padded;               // set while an iterated periodic apply runs: the source of a sweep is
                                    // a padded grid with current halos
     float* host_in;                // N floats each, apply_host staging
@@ -1191,6 +1192,58 @@ int apply_periodic(stencil_plan_s* p, const T* in, T* out, int steps, cudaStream
     return rc;
 }
 
+inline const Tap* device_taps(const stencil_plan_s* p, const float*) { return p->d_taps; }
+inline const TapT<double>* device_taps(const stencil_plan_s* p, const double*) { return p->d_taps64; }
+inline int tap_count(const stencil_plan_s* p, const float*) { return (int)p->taps.size(); }
+inline int tap_count(const stencil_plan_s* p, const double*) { return (int)p->taps64.size(); }
+
+// The wrap-correction route needs the three parts of the boundary shell to be disjoint.
+bool wrap_correction_fits(const stencil_plan_s* p) {
+    const int R = p->radius;
+    return p->nx >= 2 * R && p->ny >= 2 * R && (p->ndim == 2 || p->nz >= 2 * R);
+}
+
+// Which periodic route an apply of `steps` steps takes: true = zero-boundary sweep plus wrap
+// correction, false = padded copy.  The correction costs one pass over the taps of every
+// shell point, the padded route one copy of the grid per apply (plus a shell copy per step):
+// measured on 512^3, the correction wins except for the 125-tap box and, when the copy is
+// spread over several steps, for the wide 3D stars.
+bool use_wrap_correction(const stencil_plan_s* p, int steps) {
+    if (p->periodic_route == 1 || !wrap_correction_fits(p)) return false;
+    if (p->periodic_route == 2) return true;
+    if (p->ndim == 3 && p->shape == STENCIL_BOX && p->radius >= 2) return false;
+    if (p->ndim == 3 && p->shape == STENCIL_STAR && p->radius >= 3 && steps > 1) return false;
+    return true;
+}
+
+// Periodic apply on the tiled kernels without a padded copy: every step is a zero-boundary
+// sweep followed by stencil_wrap_correction_kernel, which adds the wrapped taps to the points
+// within R of a face.  `other` is the plan's ping-pong grid (used when steps > 1).
+template <typename T>
+int apply_periodic_corrected(stencil_plan_s* p, const T* in, T* out, T* other, int steps, cudaStream_t st) {
+    const int R = p->radius, rz = p->ndim == 3 ? R : 0;
+    const Grid g{p->nz, p->ny, p->nx};
+    const int64_t shell = (int64_t)2 * rz * g.ny * g.nx + (int64_t)(g.nz - 2 * rz) * 2 * R * g.nx +
+                          (int64_t)(g.nz - 2 * rz) * (g.ny - 2 * R) * 2 * R;
+    const int shell_grid = (int)std::max<int64_t>(1, std::min<int64_t>((shell + 255) / 256, (int64_t)sm_count() * 16));
+    const T* src = in;
+    for (int k = 0; k < steps; ++k) {
+        T* dst = ((steps - 1 - k) % 2 == 0) ? out : other;
+        p->boundary = STENCIL_ZERO;
+        const int rc = sweep_any(p, src, dst, st);
+        p->boundary = STENCIL_PERIODIC;
+        if (rc != STENCIL_OK) return rc;
+        if (shell > 0) {
+            stencil_wrap_correction_kernel<T><<<shell_grid, 256, 0, st>>>(src, dst, g, R, rz, device_taps(p, src),
+                                                                           tap_count(p, src));
+            if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
+            p->launches++;
+        }
+        src = dst;
+    }
+    return STENCIL_OK;
+}
+
 // FP64 twin of apply_row_padded: rows of an odd number of doubles, pitch rounded up to even.
 // The two padded grids live in the same plan slots, sized in doubles.
 int apply_row_padded_f64(stencil_plan_s* p, const double* in, double* out, int steps, cudaStream_t st) {
@@ -1251,7 +1304,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->npoints = n;
     p->radius = radius; p->shape = shape; p->boundary = boundary;
     p->device = -1;
-    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0; p->src_padded = false;
+    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0; p->src_padded = false; p->periodic_route = 0;
     p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr;
     p->host_in = nullptr; p->host_out = nullptr;
     p->copy_in = nullptr; p->copy_out = nullptr;
@@ -1368,11 +1421,13 @@ int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void
         return STENCIL_OK;
     }
     if (p->variant == STENCIL_VARIANT_STREAM && p->nx % 4 != 0) return apply_row_padded(p, in, out, steps, st);
-    if (p->variant == STENCIL_VARIANT_STREAM && p->boundary == STENCIL_PERIODIC && steps > 1)
-        return apply_periodic(p, in, out, steps, st);
     if (steps > 1) {
         rc = ensure_grid(&p->scratch, p->npoints);
         if (rc != STENCIL_OK) return rc;
+    }
+    if (p->variant == STENCIL_VARIANT_STREAM && p->boundary == STENCIL_PERIODIC) {
+        if (use_wrap_correction(p, steps)) return apply_periodic_corrected(p, in, out, p->scratch, steps, st);
+        if (steps > 1) return apply_periodic(p, in, out, steps, st);
     }
     // A pass advances the field by T time steps (T = 1 without temporal blocking).
     // Ping-pong between `out` and the scratch grid so that the last pass writes
@@ -1415,14 +1470,16 @@ int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps
         return STENCIL_OK;
     }
     if (p->variant == STENCIL_VARIANT_STREAM && p->nx % 2 != 0) return apply_row_padded_f64(p, in, out, steps, st);
-    if (p->variant == STENCIL_VARIANT_STREAM && p->boundary == STENCIL_PERIODIC && steps > 1)
-        return apply_periodic(p, in, out, steps, st);
     if (steps > 1 && !p->scratch64) {
         if (cudaMalloc(&p->scratch64, bytes) != cudaSuccess) {
             cudaGetLastError();
             p->scratch64 = nullptr;
             return STENCIL_ERR_ALLOC;
         }
+    }
+    if (p->variant == STENCIL_VARIANT_STREAM && p->boundary == STENCIL_PERIODIC) {
+        if (use_wrap_correction(p, steps)) return apply_periodic_corrected(p, in, out, p->scratch64, steps, st);
+        if (steps > 1) return apply_periodic(p, in, out, steps, st);
     }
     const double* src = in;
     for (int k = 0; k < steps; ++k) {
@@ -1683,6 +1740,10 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
         case STENCIL_KEY_CHAIN_LAUNCHES:
             p->chain_launches = value != 0;
             return STENCIL_OK;
+        case STENCIL_KEY_PERIODIC_ROUTE:
+            if (value < 0 || value > 2) return STENCIL_ERR_INVALID;
+            p->periodic_route = (int)value;
+            return STENCIL_OK;
         case STENCIL_KEY_FUSED_TILE_Y: {
             if (value < 0) return STENCIL_ERR_INVALID;
             const int old = p->fused_tile_y;
@@ -1743,6 +1804,7 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
         case STENCIL_KEY_STAGES: *value = p->stages; return STENCIL_OK;
         case STENCIL_KEY_STREAMING_STORE: *value = p->streaming_store; return STENCIL_OK;
         case STENCIL_KEY_CHAIN_LAUNCHES: *value = p->chain_launches ? 1 : 0; return STENCIL_OK;
+        case STENCIL_KEY_PERIODIC_ROUTE: *value = p->periodic_route; return STENCIL_OK;
         case STENCIL_KEY_FUSED_TILE_Y:
             *value = (p->variant == STENCIL_VARIANT_STREAM && p->fused_cfg) ? p->fused_cfg->tye : 0;
             return STENCIL_OK;

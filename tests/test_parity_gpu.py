@@ -209,24 +209,30 @@ def test_non_default_stream():
 
 
 # ------------------------------------------------- periodic boundary, tiled path --
+# periodic_route: None = chosen by the library, 2 = wrap correction after a zero-boundary sweep (extents >= 2R),
+# 1 = sweep from a padded copy with wrapped halos
+@pytest.mark.parametrize("route", [None, 1, 2])
 @pytest.mark.parametrize("R,box", STREAM_OPS)
-@pytest.mark.parametrize("dims,chunk_z", [((37, 45, 132), 10), ((8, 16, 128), 0), ((2, 3, 4), 0), ((70, 33, 260), 32)])
-def test_periodic_3d_on_the_tiled_kernel(R, box, dims, chunk_z):
+@pytest.mark.parametrize("dims,chunk_z", [((37, 45, 132), 10), ((8, 16, 128), 0), ((2, 3, 4), 0), ((70, 33, 260), 32),
+                                          ((8, 8, 8), 0)])
+def test_periodic_3d_on_the_tiled_kernel(R, box, dims, chunk_z, route):
     w = wl.random_box_weights(3, R, 101) if box else wl.random_star_weights(3, R, 101)
     a = wl.normal_field(dims, 102)
     for steps in (1, 2, 3, 6):                       # from 2 steps on the sweeps stay in the padded layout
         used = check(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps, chunk_z=chunk_z or None,
-                     repeat=2 if steps == 3 else 1)
+                     repeat=2 if steps == 3 else 1, periodic_route=route)
         assert used == "stream"
 
 
-@pytest.mark.parametrize("R,box", [(1, False), (4, False), (2, True), (3, True)])
-@pytest.mark.parametrize("dims", [(67, 132), (3, 8), (200, 260)])
-def test_periodic_2d_on_the_tiled_kernel(R, box, dims):
+@pytest.mark.parametrize("route", [None, 1, 2])
+@pytest.mark.parametrize("R,box", [(1, False), (4, False), (2, True), (3, True), (4, True)])
+@pytest.mark.parametrize("dims", [(67, 132), (3, 8), (200, 260), (8, 8)])
+def test_periodic_2d_on_the_tiled_kernel(R, box, dims, route):
     w = wl.random_box_weights(2, R, 103) if box else wl.random_star_weights(2, R, 103)
     a = wl.normal_field(dims, 104)
     for steps in (1, 2, 5):
-        used = check(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps, repeat=2 if steps == 5 else 1)
+        used = check(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps, repeat=2 if steps == 5 else 1,
+                     periodic_route=route)
         assert used == "stream"
 
 
@@ -489,12 +495,13 @@ def test_f64_padded_row_sweep(dims, R, box, steps):
     ((37, 45, 66), 1, False), ((37, 45, 66), 4, False), ((8, 16, 64), 1, True), ((2, 3, 2), 2, False),
     ((70, 33, 130), 3, False),
     ((67, 66), 3, True), ((3, 8), 4, False), ((200, 258), 1, False), ((64, 2), 2, True)])
-def test_f64_periodic_on_the_tiled_kernels(dims, R, box):
+@pytest.mark.parametrize("route", [None, 1, 2])
+def test_f64_periodic_on_the_tiled_kernels(dims, R, box, route):
     ndim = len(dims)
     w = (wl.random_box_weights if box else wl.random_star_weights)(ndim, R, 89, np.float64)
     a = wl.normal_field(dims, 90, np.float64)
     for steps in (1, 2, 5):
-        used = check_f64(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps)
+        used = check_f64(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps=steps, periodic_route=route)
         assert used == "stream"
 
 
