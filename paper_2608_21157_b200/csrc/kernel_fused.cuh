@@ -54,8 +54,11 @@ __device__ __forceinline__ void consumer_barrier(int nthreads) {
     asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
 }
 
-template <int R, int T, int K, int XW, int NWY>
-__global__ void __launch_bounds__(XW * NWY * 32, 1)
+// SPEC: the launch advances exactly T levels and one region spans a whole row of exactly
+// 128*XW points.  The level count, the row pitch and the x bounds are then compile-time
+// constants (the common case of the iterated apply on a 256-wide grid).
+template <int R, int T, int K, int XW, int NWY, bool SPEC = false>
+__global__ void __launch_bounds__(XW * NWY * 32, (XW * NWY * 32 <= 256 ? 2 : 1))
 stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restrict__ out,
                      const FusedGeom g, const __grid_constant__ StarWeights<R> sw,
                      int* __restrict__ status) {
@@ -99,17 +102,18 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
     const int tix = bid % g.tiles_x;
     const int tiy = (bid / g.tiles_x) % g.tiles_y;
     const int chunk = bid / (g.tiles_x * g.tiles_y);
-    const int x0e = tix * g.tile_x - g.halo_x;     // region origin (may be negative)
+    const int x0e = SPEC ? 0 : tix * g.tile_x - g.halo_x;     // region origin (may be negative)
     const int y0e = tiy * g.tile_y - g.halo_y;
     const int z0 = chunk * g.chunk_z;
     const int z1 = min(z0 + g.chunk_z, g.nz);
-    const int nlev = g.nlev;
+    const int nlev = SPEC ? T : g.nlev;
+    const int nx = SPEC ? TXE : g.nx;
     const int pstart = z0 - nlev * R;
     const int nsteps = (z1 - z0) + 2 * nlev * R;
 
     const int xg = x0e + col;
-    const bool x_in = xg >= 0 && xg < g.nx;
-    const bool x_store = x_in && col >= g.halo_x && col < g.halo_x + g.tile_x;
+    const bool x_in = SPEC || (xg >= 0 && xg < nx);
+    const bool x_store = SPEC || (x_in && col >= g.halo_x && col < g.halo_x + g.tile_x);
     // per-row flags packed into bit masks; the common case (every row inside the grid,
     // every row stored) is tested once per plane instead of once per row
     uint32_t in_mask = 0, store_mask = 0;
@@ -124,8 +128,8 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
     // the same flags for the whole warp, so that the common case is a uniform branch
     const bool warp_all_in = __all_sync(0xffffffffu, in_mask == kAllRows);
     const bool warp_all_store = __all_sync(0xffffffffu, store_mask == kAllRows);
-    const size_t plane_stride = (size_t)g.ny * g.nx;
-    float* const out_col = out + (size_t)(y0e + row0) * g.nx + xg;     // this thread's column of rows
+    const size_t plane_stride = (size_t)g.ny * nx;
+    float* const out_col = out + (size_t)(y0e + row0) * nx + xg;       // this thread's column of rows
     const int toff = row0 * TXE + col;                                  // its offset inside a plane
 
     int issued = 0;                                // planes requested so far (thread 0 only)
@@ -251,12 +255,12 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                                 if (warp_all_store) {
 #pragma unroll
                                     for (int k = 0; k < K; ++k)
-                                        *reinterpret_cast<float4*>(op + (size_t)k * g.nx) = e[k];
+                                        *reinterpret_cast<float4*>(op + (size_t)k * nx) = e[k];
                                 } else {
 #pragma unroll
                                     for (int k = 0; k < K; ++k)
                                         if ((store_mask >> k) & 1u)
-                                            *reinterpret_cast<float4*>(op + (size_t)k * g.nx) = e[k];
+                                            *reinterpret_cast<float4*>(op + (size_t)k * nx) = e[k];
                                 }
                             }
                         } else {

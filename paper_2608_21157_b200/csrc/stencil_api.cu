@@ -109,12 +109,15 @@ struct FusedConfig {
     int radius, T, K, XW, NWY;
     int txe, tye, threads, slot_bytes;
     const void* kernel;
-    mutable size_t smem_allowed;             // dynamic shared memory already granted to the kernel
+    const void* kernel_spec;                 // the instantiation for full passes over rows of exactly txe points
+    mutable size_t smem_allowed;             // dynamic shared memory already granted to both kernels
     mutable size_t occ_smem;                 // ... and the occupancy measured at this size
     mutable int occ;
     mutable int cache_device;
     cudaError_t (*launch)(const struct stencil_plan_s*, const CUtensorMap&, float*, const FusedGeom&,
                           int grid, size_t smem, cudaStream_t);
+    cudaError_t (*launch_spec)(const struct stencil_plan_s*, const CUtensorMap&, float*, const FusedGeom&,
+                               int grid, size_t smem, cudaStream_t);
 };
 
 // ---------------------------------------------------------------------------
@@ -298,13 +301,13 @@ void pack_star(const stencil_plan_s* p, StarWeights<R>& sw) {
     }
 }
 
-template <int R, int T, int K, int XW, int NWY>
+template <int R, int T, int K, int XW, int NWY, bool SPEC>
 cudaError_t launch_fused_t(const stencil_plan_s* p, const CUtensorMap& map, float* out, const FusedGeom& g,
                            int grid, size_t smem, cudaStream_t st) {
     StarWeights<R> sw;
     pack_star<R>(p, sw);
-    return launch_kernel(&stencil_fused_kernel<R, T, K, XW, NWY>, grid, FusedShape<R, K, XW, NWY>::THREADS, smem,
-                         st, p->chained, map, out, g, sw, p->d_status);
+    return launch_kernel(&stencil_fused_kernel<R, T, K, XW, NWY, SPEC>, grid, FusedShape<R, K, XW, NWY>::THREADS,
+                         smem, st, p->chained, map, out, g, sw, p->d_status);
 }
 
 template <int R, int T, int K, int XW, int NWY>
@@ -313,9 +316,11 @@ FusedConfig make_fused() {
     FusedConfig c;
     c.radius = R; c.T = T; c.K = K; c.XW = XW; c.NWY = NWY;
     c.txe = S::TXE; c.tye = S::TYE; c.threads = S::THREADS; c.slot_bytes = S::SLOT_BYTES;
-    c.kernel = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY>);
+    c.kernel = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, false>);
+    c.kernel_spec = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, true>);
     c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
-    c.launch = &launch_fused_t<R, T, K, XW, NWY>;
+    c.launch = &launch_fused_t<R, T, K, XW, NWY, false>;
+    c.launch_spec = &launch_fused_t<R, T, K, XW, NWY, true>;
     return c;
 }
 
@@ -797,7 +802,9 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
         if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->occ_smem = 0; cfg->cache_device = dev; }
         if (smem > cfg->smem_allowed) {
             if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess) {
+                    cudaSuccess ||
+                cudaFuncSetAttribute(cfg->kernel_spec, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                    cudaSuccess) {
                 cudaGetLastError();
                 return STENCIL_ERR_CUDA;
             }
@@ -826,7 +833,10 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
     g.chunk_z = chunk;
     const int64_t grid64 = (int64_t)tiles * ((p->nz + chunk - 1) / chunk);
     if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
-    if (cfg->launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
+    // full passes over rows of exactly one region take the instantiation with those facts compiled in
+    const bool spec = nlev == T && p->nx == cfg->txe;
+    if ((spec ? cfg->launch_spec : cfg->launch)(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess)
+        return STENCIL_ERR_CUDA;
     p->launches++;
     return STENCIL_OK;
 }
@@ -838,6 +848,27 @@ int launch_sweep(stencil_plan_s* p, const float* src, float* dst, cudaStream_t s
         default: return launch_generic(p, src, dst, st);
     }
 }
+
+// The sweep launchers read the grid they work on from the plan.  Some applies sweep a plan-owned
+// stand-in for the caller's grid (padded rows, a padded periodic copy); this guard swaps the
+// stand-in's extents, row length for the tensor maps and boundary into the plan for the
+// duration of those launches and puts the plan's own back on every path out.
+class ScopedGridView {
+public:
+    ScopedGridView(stencil_plan_s* p, int nz, int ny, int nx, int tmap_nx, int boundary)
+        : p_(p), nz_(p->nz), ny_(p->ny), nx_(p->nx), tmap_nx_(p->tmap_nx), boundary_(p->boundary) {
+        p->nz = nz; p->ny = ny; p->nx = nx; p->tmap_nx = tmap_nx; p->boundary = boundary;
+    }
+    ~ScopedGridView() {
+        p_->nz = nz_; p_->ny = ny_; p_->nx = nx_; p_->tmap_nx = tmap_nx_; p_->boundary = boundary_;
+        p_->chained = false;
+    }
+    ScopedGridView(const ScopedGridView&) = delete;
+    ScopedGridView& operator=(const ScopedGridView&) = delete;
+private:
+    stencil_plan_s* p_;
+    int nz_, ny_, nx_, tmap_nx_, boundary_;
+};
 
 template <typename T>
 int repitch_rows(stencil_plan_s* p, const T* src, T* dst, int nx, int src_pitch, int dst_pitch,
@@ -868,16 +899,14 @@ int apply_row_padded(stencil_plan_s* p, const float* in, float* out, int steps, 
     if ((rc = repitch_rows(p, in, p->pad, nx, nx, pitch, st)) != STENCIL_OK) return rc;
     float* src = p->pad;
     float* dst = p->pad2;
-    p->nx = pitch;
-    p->tmap_nx = nx;
-    for (int k = 0; k < steps && rc == STENCIL_OK; ++k) {
-        p->chained = p->chain_launches && k > 0;
-        rc = launch_sweep(p, src, dst, st);
-        std::swap(src, dst);
+    {
+        ScopedGridView view(p, p->nz, p->ny, pitch, nx, STENCIL_ZERO);
+        for (int k = 0; k < steps && rc == STENCIL_OK; ++k) {
+            p->chained = p->chain_launches && k > 0;
+            rc = launch_sweep(p, src, dst, st);
+            std::swap(src, dst);
+        }
     }
-    p->chained = false;
-    p->nx = nx;
-    p->tmap_nx = 0;
     if (rc != STENCIL_OK) return rc;
     return repitch_rows(p, src, out, nx, pitch, nx, st);
 }
@@ -1176,9 +1205,10 @@ int apply_periodic(stencil_plan_s* p, const T* in, T* out, int steps, cudaStream
     const int64_t shell = cells / Vec16<T>::n - (int64_t)nz * ny * (nx / Vec16<T>::n);
     const int shell_grid = (int)std::max<int64_t>(1, std::min<int64_t>((shell + 255) / 256, (int64_t)sm_count() * 16));
     for (int k = 0; k + 1 < steps && rc == STENCIL_OK; ++k) {
-        p->nz = pnz; p->ny = pny; p->nx = pnx; p->boundary = STENCIL_ZERO;
-        rc = sweep_any(p, static_cast<const T*>(a), b, st);
-        p->nz = nz; p->ny = ny; p->nx = nx; p->boundary = STENCIL_PERIODIC;
+        {
+            ScopedGridView view(p, pnz, pny, pnx, 0, STENCIL_ZERO);
+            rc = sweep_any(p, static_cast<const T*>(a), b, st);
+        }
         if (rc != STENCIL_OK) break;
         stencil_refresh_halo_kernel<T><<<shell_grid, 256, 0, st>>>(b, g, R, rz);
         if (cudaGetLastError() != cudaSuccess) rc = STENCIL_ERR_CUDA;
@@ -1229,9 +1259,11 @@ int apply_periodic_corrected(stencil_plan_s* p, const T* in, T* out, T* other, i
     const T* src = in;
     for (int k = 0; k < steps; ++k) {
         T* dst = ((steps - 1 - k) % 2 == 0) ? out : other;
-        p->boundary = STENCIL_ZERO;
-        const int rc = sweep_any(p, src, dst, st);
-        p->boundary = STENCIL_PERIODIC;
+        int rc;
+        {
+            ScopedGridView view(p, p->nz, p->ny, p->nx, 0, STENCIL_ZERO);
+            rc = sweep_any(p, src, dst, st);
+        }
         if (rc != STENCIL_OK) return rc;
         if (shell > 0) {
             stencil_wrap_correction_kernel<T><<<shell_grid, 256, 0, st>>>(src, dst, g, R, rz, device_taps(p, src),
@@ -1255,16 +1287,14 @@ int apply_row_padded_f64(stencil_plan_s* p, const double* in, double* out, int s
     double* src = reinterpret_cast<double*>(p->pad);
     double* dst = reinterpret_cast<double*>(p->pad2);
     if ((rc = repitch_rows(p, in, src, nx, nx, pitch, st)) != STENCIL_OK) return rc;
-    p->nx = pitch;
-    p->tmap_nx = nx;
-    for (int k = 0; k < steps && rc == STENCIL_OK; ++k) {
-        p->chained = p->chain_launches && k > 0;
-        rc = launch_sweep_f64(p, src, dst, st);
-        std::swap(src, dst);
+    {
+        ScopedGridView view(p, p->nz, p->ny, pitch, nx, STENCIL_ZERO);
+        for (int k = 0; k < steps && rc == STENCIL_OK; ++k) {
+            p->chained = p->chain_launches && k > 0;
+            rc = launch_sweep_f64(p, src, dst, st);
+            std::swap(src, dst);
+        }
     }
-    p->chained = false;
-    p->nx = nx;
-    p->tmap_nx = 0;
     if (rc != STENCIL_OK) return rc;
     return repitch_rows(p, static_cast<const double*>(src), out, nx, pitch, nx, st);
 }

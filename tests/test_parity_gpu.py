@@ -349,7 +349,8 @@ FUSED_CONFIGS = [   # (radius, fuse_steps, region width, region height)
 @pytest.mark.parametrize("R,T,width,height", FUSED_CONFIGS)
 @pytest.mark.parametrize("dims,chunk_z", [
     ((29, 70, 300), 11),        # several regions in x and y, ragged everywhere, several z chunks
-    ((40, 64, 256), 0),         # a 256-wide region spans the whole row
+    ((40, 64, 256), 0),         # a 256-wide region spans the whole row (the specialised instantiation)
+    ((33, 50, 128), 9),         # the same for the 128-wide regions; ragged in y, several z chunks
     ((5, 9, 12), 0),            # much smaller than one region
 ])
 def test_fused_passes_match_oracle(R, T, width, height, dims, chunk_z):
