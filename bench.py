@@ -42,7 +42,7 @@ NCU_TRAFFIC_BYTES = {
     "cfg2": 1003.8e6,   # stream kernel, star R=1: 2 x (279.4 MB read + 222.5 MB written) on the half grid
     "cfg3": 1004.6e6,   # stream kernel, box R=1
     "cfg4": 995.7e6,    # stream kernel, star R=4
-    "cfg5": 101.5e6,    # one fused pass (2 time steps of 256^3): 78.2 MB read + 23.3 MB written
+    "cfg5": 99.9e6,     # one fused pass (2 time steps of 256^3): 77.7 MB read + 22.2 MB written
 }
 
 
