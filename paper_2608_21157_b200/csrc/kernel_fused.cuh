@@ -42,9 +42,15 @@ struct FusedShape {
     static constexpr int TXE = 128 * XW;
     static constexpr int TYE = NWY * K;
     static constexpr int THREADS = XW * NWY * 32;
-    static constexpr int SLOT_FLOATS = (TYE + 2 * R) * TXE;     // R pad rows above and below
+    // A TMA box is at most 256 elements wide, so a wider plane lies in shared memory as NP parts
+    // of PW columns, each loaded by its own copy and each with its own pad rows:
+    // cell (row r, column x) of a plane is at  (x / PW) * PART_FLOATS + r * PW + x % PW.
+    static constexpr int PW = TXE > 256 ? 256 : TXE;
+    static constexpr int NP = TXE / PW;
+    static constexpr int PART_FLOATS = (TYE + 2 * R) * PW;      // R pad rows above and below
+    static constexpr int SLOT_FLOATS = NP * PART_FLOATS;
     static constexpr int SLOT_BYTES = SLOT_FLOATS * 4;          // multiple of 512
-    static constexpr int BOX_BYTES = TYE * TXE * 4;
+    static constexpr int BOX_BYTES = TYE * TXE * 4;             // bytes of all parts of one plane
     static size_t smem_bytes(int stages, int T) {
         return (size_t)(stages + 2 * (T - 1)) * SLOT_BYTES + 128 + kMaxStages * 8;
     }
@@ -64,6 +70,7 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                      int* __restrict__ status) {
     using S = FusedShape<R, K, XW, NWY>;
     constexpr int TXE = S::TXE;
+    constexpr int PW = S::PW;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     // indexing the shared array keeps every derived pointer in the shared address space
     unsigned char* base = smem_raw + ((128u - (smem_addr(smem_raw) & 127u)) & 127u);
@@ -85,8 +92,9 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
         for (int s = 0; s < nslots; ++s) {
             float* slot = ring + (size_t)s * S::SLOT_FLOATS;
             for (int e = tid; e < R * TXE; e += S::THREADS) {
-                slot[e] = 0.0f;
-                slot[(S::TYE + R) * TXE + e] = 0.0f;
+                float* part = slot + (e / (R * PW)) * S::PART_FLOATS;
+                part[e % (R * PW)] = 0.0f;
+                part[(S::TYE + R) * PW + e % (R * PW)] = 0.0f;
             }
         }
     }
@@ -130,7 +138,10 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
     const bool warp_all_store = __all_sync(0xffffffffu, store_mask == kAllRows);
     const size_t plane_stride = (size_t)g.ny * nx;
     float* const out_col = out + (size_t)(y0e + row0) * nx + xg;       // this thread's column of rows
-    const int toff = row0 * TXE + col;                                  // its offset inside a plane
+    const int toff = (col / PW) * S::PART_FLOATS + row0 * PW + col % PW;   // its offset inside a plane
+    // the cells just left and right of the warp's 128 columns (they may lie in another part)
+    const int hl_off = wx > 0 ? ((wx * 128 - 1) / PW) * S::PART_FLOATS + (wx * 128 - R) - ((wx * 128 - 1) / PW) * PW : 0;
+    const int hr_off = wx < XW - 1 ? (((wx + 1) * 128) / PW) * S::PART_FLOATS + (wx + 1) * 128 - (((wx + 1) * 128) / PW) * PW : 0;
 
     int issued = 0;                                // planes requested so far (thread 0 only)
     if (tid == 0) {
@@ -139,8 +150,10 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
         issued = pre;
         for (int i = 0; i < pre; ++i) {
             mbar_arrive_expect_tx(full0 + 8 * i, S::BOX_BYTES);
-            tma_load_3d(smem_addr(ring + (size_t)i * S::SLOT_FLOATS + R * TXE), &tmap_in, full0 + 8 * i,
-                        x0e, y0e, pstart + i);
+#pragma unroll
+            for (int part = 0; part < S::NP; ++part)
+                tma_load_3d(smem_addr(ring + (size_t)i * S::SLOT_FLOATS + part * S::PART_FLOATS + R * PW), &tmap_in,
+                            full0 + 8 * i, x0e + part * PW, y0e, pstart + i);
         }
     }
 
@@ -168,11 +181,11 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                 dead = true;
                 atomicExch(status, kStatusTimeout);
             }
-            const float* src = ring + (size_t)s * S::SLOT_FLOATS + R * TXE;     // region row 0
+            const float* src = ring + (size_t)s * S::SLOT_FLOATS + R * PW;      // region row 0 (of part 0)
             float4 cin[K + 2 * R];
 #pragma unroll
             for (int kk = 0; kk < K + 2 * R; ++kk)
-                cin[kk] = *reinterpret_cast<const float4*>(src + toff + (kk - R) * TXE);
+                cin[kk] = *reinterpret_cast<const float4*>(src + toff + (kk - R) * PW);
 
 #pragma unroll
             for (int l = 1; l <= T; ++l) {
@@ -187,15 +200,15 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                             v[R + 0] = ctr.x; v[R + 1] = ctr.y; v[R + 2] = ctr.z; v[R + 3] = ctr.w;
                             {
                                 const float c4[4] = {ctr.x, ctr.y, ctr.z, ctr.w};
-                                const float* rowb = src + (row0 + k) * TXE;   // first cell of the region row
+                                const float* rowb = src + (row0 + k) * PW;    // first cell of the region row (part 0)
 #pragma unroll
                                 for (int t = 0; t < R; ++t) {
                                     // cells across the warp boundary: one broadcast read per side from the
                                     // level's plane (wx is warp-uniform); zero at the region's edge
                                     float xl = 0.0f, xr = 0.0f;
                                     if (XW > 1) {
-                                        if (wx > 0) xl = rowb[wx * 128 - R + t];
-                                        if (wx < XW - 1) xr = rowb[(wx + 1) * 128 + t];
+                                        if (wx > 0) xl = rowb[hl_off + t];
+                                        if (wx < XW - 1) xr = rowb[hr_off + t];
                                     }
                                     const float lft = __shfl_up_sync(0xffffffffu, c4[4 - R + t], 1);
                                     const float rgt = __shfl_down_sync(0xffffffffu, c4[t], 1);
@@ -264,10 +277,10 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                                 }
                             }
                         } else {
-                            float* buf = lvl + (size_t)(2 * (l - 1) + par) * S::SLOT_FLOATS + R * TXE;
+                            float* buf = lvl + (size_t)(2 * (l - 1) + par) * S::SLOT_FLOATS + R * PW;
 #pragma unroll
                             for (int k = 0; k < K; ++k)
-                                *reinterpret_cast<float4*>(buf + toff + k * TXE) = e[k];
+                                *reinterpret_cast<float4*>(buf + toff + k * PW) = e[k];
                         }
                     }
                     if (l < nlev || l == 1) {
@@ -276,20 +289,22 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                         if (l == 1 && tid == 0 && i + nstage < nsteps) {
                             // the input slot is free: refill it with the plane nstage steps ahead
                             mbar_arrive_expect_tx(full0 + 8 * s, S::BOX_BYTES);
-                            tma_load_3d(smem_addr(ring + (size_t)s * S::SLOT_FLOATS + R * TXE), &tmap_in,
-                                        full0 + 8 * s, x0e, y0e, pstart + i + nstage);
+#pragma unroll
+                            for (int part = 0; part < S::NP; ++part)
+                                tma_load_3d(smem_addr(ring + (size_t)s * S::SLOT_FLOATS + part * S::PART_FLOATS + R * PW),
+                                            &tmap_in, full0 + 8 * s, x0e + part * PW, y0e, pstart + i + nstage);
                             issued = i + nstage + 1;
                         }
                     }
                     if (l < nlev) {
-                        const float* buf = lvl + (size_t)(2 * (l - 1) + par) * S::SLOT_FLOATS + R * TXE;
+                        const float* buf = lvl + (size_t)(2 * (l - 1) + par) * S::SLOT_FLOATS + R * PW;
                         src = buf;
 #pragma unroll
                         for (int k = 0; k < K; ++k) cin[k + R] = e[k];
 #pragma unroll
                         for (int kk = 0; kk < R; ++kk) {
-                            cin[kk] = *reinterpret_cast<const float4*>(buf + toff + (kk - R) * TXE);
-                            cin[K + R + kk] = *reinterpret_cast<const float4*>(buf + toff + (K + kk) * TXE);
+                            cin[kk] = *reinterpret_cast<const float4*>(buf + toff + (kk - R) * PW);
+                            cin[K + R + kk] = *reinterpret_cast<const float4*>(buf + toff + (K + kk) * PW);
                         }
                     }
                 }

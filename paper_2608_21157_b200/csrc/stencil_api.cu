@@ -328,7 +328,7 @@ FusedConfig make_fused() {
 const std::vector<FusedConfig>& fused_configs() {
     static const std::vector<FusedConfig> v = {
         make_fused<1, 2, 4, 2, 8>(),  make_fused<1, 3, 4, 2, 8>(),  make_fused<1, 2, 4, 2, 4>(),
-        make_fused<1, 2, 2, 2, 8>(),
+        make_fused<1, 2, 2, 2, 8>(),  make_fused<1, 2, 4, 4, 4>(),
         make_fused<1, 4, 2, 1, 16>(), make_fused<1, 2, 2, 1, 16>(), make_fused<1, 3, 2, 1, 16>(),
         make_fused<2, 2, 2, 1, 16>(),
     };
@@ -397,16 +397,26 @@ const FusedConfig* pick_fused(const stencil_plan_s* p) {
     if (p->nx % 4 != 0) return nullptr;                   // ... over the row pitch, which padded rows exceed
     if (p->fuse_steps == 1) return nullptr;
     int txe = p->tile_x;
-    if (p->fuse_steps == 0 && txe == 0 && p->fused_tile_y == 0) {
-        // Default: fuse two steps per pass when one 256-wide region spans a whole row (no
-        // redundant columns).  On wider grids the halo recomputation of several regions per
-        // row costs more than the saved traffic (measured on 512^3), so those stay unfused
-        // unless the caller asks for fusion.
-        // 16-row regions: two CTAs fit an SM and cover each other's barrier stalls, which
-        // outweighs their larger halo share (measured on 256^3: 922 vs 846 G updates/s)
-        if (p->nx > 256) return nullptr;
-        const FusedConfig* c = find_fused_cfg(p->radius, 2, 256, 16);
-        return c ? c : find_fused_cfg(p->radius, 2, 256);
+    // no preference for the region: the default below, also when the caller asks for its step count
+    if ((p->fuse_steps == 0 || p->fuse_steps == 2) && txe == 0 && p->fused_tile_y == 0) {
+        // Default: fuse two steps per pass when one region spans a whole row (no redundant
+        // columns): 256 wide, or 512 wide (one CTA per SM, each plane loaded as two TMA boxes).
+        // With several regions per row the halo recomputation costs more than the saved
+        // traffic (measured on 512^3 with 128-wide regions), and a 512-wide region on a much
+        // narrower row idles too many lanes, so those grids stay unfused unless the caller
+        // asks for fusion.
+        // 16-row regions: at 256 columns two CTAs fit an SM and cover each other's barrier
+        // stalls, which outweighs their larger halo share (measured on 256^3: 922 vs 846 G
+        // updates/s)
+        const FusedConfig* c = nullptr;
+        if (p->nx <= 256) {
+            c = find_fused_cfg(p->radius, 2, 256, 16);
+            if (!c) c = find_fused_cfg(p->radius, 2, 256);
+        } else if (p->nx > 416 && p->nx <= 512) {
+            // measured on 512 x 512 x nx: 448 columns 851 vs 788 G updates/s unfused, 400 columns 761 vs 776
+            c = find_fused_cfg(p->radius, 2, 512, 16);
+        }
+        if (c || p->fuse_steps == 0) return c;
     }
     return find_fused_cfg(p->radius, p->fuse_steps, txe, p->fused_tile_y);
 }
@@ -768,7 +778,7 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
 int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cudaStream_t st) {
     const FusedConfig* cfg = p->fused_cfg;
     const CUtensorMap* map = nullptr;
-    int rc = get_tensor_map(p, cfg, cfg->txe, cfg->tye, src, &map);
+    int rc = get_tensor_map(p, cfg, std::min(cfg->txe, 256), cfg->tye, src, &map);   // a box is at most 256 wide
     if (rc != STENCIL_OK) return rc;
     const int R = p->radius, T = cfg->T;
     FusedGeom g;
@@ -823,11 +833,24 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
     }
     int chunk = p->chunk_z;
     if (chunk <= 0) {
-        // as many z chunks as fill the resident-CTA slots of the machine once, but not so short
-        // that the 2*T*R extra input planes per chunk dominate
-        int nchunks = std::max(1, occ * sm_count() / std::max(tiles, 1));
-        nchunks = std::min(nchunks, std::max(1, p->nz / (4 * T * R)));
-        chunk = (p->nz + nchunks - 1) / nchunks;
+        // The kernel is bound by instruction issue, so every SM should get the same number of
+        // planes: cut z into the number of chunks whose CTAs fill whole waves of the machine's
+        // resident-CTA slots at the least total cost, a chunk costing its planes plus the
+        // 2*T*R extra input planes and the start-up of its pipeline.
+        const int slots = occ * sm_count();
+        const int max_chunks = std::max(1, p->nz / (4 * T * R));
+        const double fill = 4.0;
+        double best = 1e300;
+        int best_n = 1;
+        for (int n = 1; n <= max_chunks; ++n) {
+            const int c = (p->nz + n - 1) / n;
+            const int real_n = (p->nz + c - 1) / c;
+            const int64_t ctas = (int64_t)tiles * real_n;
+            const double waves = (double)((ctas + slots - 1) / slots);
+            const double cost = waves * (c + 2 * T * R + fill);
+            if (cost < best * 0.999) { best = cost; best_n = real_n; }
+        }
+        chunk = (p->nz + best_n - 1) / best_n;
     }
     chunk = std::max(1, std::min(chunk, p->nz));
     g.chunk_z = chunk;

@@ -342,7 +342,7 @@ def test_paper_shaped_2d_box_radius3():
 # -------------------------------------------------------------------- fused --
 FUSED_CONFIGS = [   # (radius, fuse_steps, region width, region height)
     (1, 2, 256, 32), (1, 2, 256, 16), (1, 3, 256, 32), (1, 4, 128, 32), (1, 2, 128, 32), (1, 3, 128, 32),
-    (2, 2, 128, 32),
+    (2, 2, 128, 32), (1, 2, 512, 16),
 ]
 
 
@@ -351,6 +351,8 @@ FUSED_CONFIGS = [   # (radius, fuse_steps, region width, region height)
     ((29, 70, 300), 11),        # several regions in x and y, ragged everywhere, several z chunks
     ((40, 64, 256), 0),         # a 256-wide region spans the whole row (the specialised instantiation)
     ((33, 50, 128), 9),         # the same for the 128-wide regions; ragged in y, several z chunks
+    ((21, 37, 512), 8),         # ... and for the 512-wide region, which is loaded as two TMA boxes
+    ((19, 30, 452), 0),         # a row that ends inside the second box of a 512-wide region
     ((5, 9, 12), 0),            # much smaller than one region
 ])
 def test_fused_passes_match_oracle(R, T, width, height, dims, chunk_z):
@@ -389,10 +391,16 @@ def test_fused_equals_unfused_within_tolerance_and_keeps_zero_boundary():
 
 def test_fuse_knob_rules():
     star = wl.star_weights(3, 1, 0.4, [0.1])
-    with b.Plan((64, 64, 512), 1, b.STAR, star, b.ZERO) as p:
+    with b.Plan((64, 64, 1024), 1, b.STAR, star, b.ZERO) as p:
         assert p.get(b.KEY_FUSE_STEPS) == 1         # rows wider than one region: unfused by default
         p.set(b.KEY_FUSE_STEPS, 4)
         assert p.get(b.KEY_FUSE_STEPS) == 4
+    with b.Plan((64, 64, 320), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # a 512-wide region would idle too many lanes
+    with b.Plan((64, 64, 512), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_FUSED_TILE_Y) == 16   # one 512-wide region per row
+    with b.Plan((64, 64, 448), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2
     with b.Plan((64, 64, 64), 1, b.STAR, star, b.ZERO) as p:
         assert p.get(b.KEY_FUSE_STEPS) >= 2         # iterated applies fuse by default
         p.set(b.KEY_FUSE_STEPS, 1)
