@@ -43,6 +43,7 @@ NCU_TRAFFIC_BYTES = {
     "cfg3": 1004.6e6,   # stream kernel, box R=1
     "cfg4": 995.7e6,    # stream kernel, star R=4
     "cfg5": 99.9e6,     # one fused pass (2 time steps of 256^3): 77.7 MB read + 22.2 MB written
+    "cfg5L": 1035.1e6,  # one fused pass (2 time steps of 512^3): 545.4 MB read + 489.7 MB written
 }
 
 
