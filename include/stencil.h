@@ -67,7 +67,7 @@ enum {
 /* Keys of stencil_plan_set / stencil_plan_get. */
 enum {
     STENCIL_KEY_VARIANT      = 0,  /* set/get: STENCIL_VARIANT_*                                 */
-    STENCIL_KEY_TILE_X       = 1,  /* set/get: region width of fused passes, 128 or 256 (0 = auto) */
+    STENCIL_KEY_TILE_X       = 1,  /* set/get: region width of fused passes, 128, 256 or 512 (0 = auto) */
     STENCIL_KEY_TILE_Y       = 2,  /* set/get: tile height in rows   (0 = default)               */
     STENCIL_KEY_FUSE_STEPS   = 3,  /* set: time steps fused per pass (0 = auto, 1 = off);
                                       get: the number iterated applies will use (1 = none)       */

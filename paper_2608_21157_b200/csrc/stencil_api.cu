@@ -400,21 +400,19 @@ const FusedConfig* pick_fused(const stencil_plan_s* p) {
     // no preference for the region: the default below, also when the caller asks for its step count
     if ((p->fuse_steps == 0 || p->fuse_steps == 2) && txe == 0 && p->fused_tile_y == 0) {
         // Default: fuse two steps per pass when one region spans a whole row (no redundant
-        // columns): 256 wide, or 512 wide (one CTA per SM, each plane loaded as two TMA boxes).
-        // With several regions per row the halo recomputation costs more than the saved
-        // traffic (measured on 512^3 with 128-wide regions), and a 512-wide region on a much
-        // narrower row idles too many lanes, so those grids stay unfused unless the caller
-        // asks for fusion.
-        // 16-row regions: at 256 columns two CTAs fit an SM and cover each other's barrier
-        // stalls, which outweighs their larger halo share (measured on 256^3: 922 vs 846 G
-        // updates/s)
+        // columns) and the row fills at least 80 % of the region's lanes.  Regions are 128, 256
+        // (two CTAs per SM, which cover each other's barrier stalls: 16-row regions beat 32-row
+        // ones, 922 vs 846 G updates/s on 256^3) or 512 columns wide (one CTA per SM, each plane
+        // loaded as two TMA boxes).  With several regions per row the halo recomputation costs
+        // more than the saved traffic, and idle lanes cost what they would compute, so other
+        // grids stay unfused unless the caller asks for fusion.  Measured (G updates/s, fused
+        // vs unfused, 512 x 512 x nx): nx = 128: 1083 vs 644 (256-wide region: 499); 192: 744 vs
+        // 709; 400: 761 vs 776; 448: 851 vs 788; 512: 1257 vs 781.
         const FusedConfig* c = nullptr;
-        if (p->nx <= 256) {
-            c = find_fused_cfg(p->radius, 2, 256, 16);
-            if (!c) c = find_fused_cfg(p->radius, 2, 256);
-        } else if (p->nx > 416 && p->nx <= 512) {
-            // measured on 512 x 512 x nx: 448 columns 851 vs 788 G updates/s unfused, 400 columns 761 vs 776
-            c = find_fused_cfg(p->radius, 2, 512, 16);
+        const int width = p->nx <= 128 ? 128 : p->nx <= 256 ? 256 : 512;
+        if (p->nx <= 512 && p->nx * 5 >= width * 4) {
+            c = find_fused_cfg(p->radius, 2, width, width == 128 ? 0 : 16);
+            if (!c && width == 256) c = find_fused_cfg(p->radius, 2, 256);
         }
         if (c || p->fuse_steps == 0) return c;
     }
@@ -1746,7 +1744,7 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
         case STENCIL_KEY_TILE_X:
         case STENCIL_KEY_FUSE_STEPS: {
             if (p->f64) return value <= 1 ? STENCIL_OK : STENCIL_ERR_UNSUPPORTED;
-            // region width (128 or 256) and time steps per pass of the fused kernel
+            // region width (128, 256 or 512) and time steps per pass of the fused kernel
             if (value < 0) return STENCIL_ERR_INVALID;
             const int old_fuse = p->fuse_steps, old_tx = p->tile_x;
             if (key == STENCIL_KEY_TILE_X) p->tile_x = (int)value; else p->fuse_steps = (int)value;

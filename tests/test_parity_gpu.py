@@ -402,7 +402,14 @@ def test_fuse_knob_rules():
     with b.Plan((64, 64, 448), 1, b.STAR, star, b.ZERO) as p:
         assert p.get(b.KEY_FUSE_STEPS) == 2
     with b.Plan((64, 64, 64), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # half of a 128-wide region's lanes would idle
+    with b.Plan((64, 64, 200), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # 78 % of a 256-wide region
+    with b.Plan((64, 64, 128), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 128
+    with b.Plan((64, 64, 256), 1, b.STAR, star, b.ZERO) as p:
         assert p.get(b.KEY_FUSE_STEPS) >= 2         # iterated applies fuse by default
+        assert p.get(b.KEY_TILE_X) == 256 and p.get(b.KEY_FUSED_TILE_Y) == 16
         p.set(b.KEY_FUSE_STEPS, 1)
         assert p.get(b.KEY_FUSE_STEPS) == 1
         with pytest.raises(b.StencilError):
