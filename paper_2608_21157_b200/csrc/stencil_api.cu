@@ -408,9 +408,15 @@ const FusedConfig* pick_fused(const stencil_plan_s* p) {
         // grids stay unfused unless the caller asks for fusion.  Measured (G updates/s, fused
         // vs unfused, 512 x 512 x nx): nx = 128: 1083 vs 644 (256-wide region: 499); 192: 744 vs
         // 709; 400: 761 vs 776; 448: 851 vs 788; 512: 1257 vs 781.
+        // Rows wider than 512 points take several 512-wide regions, each with 4 halo columns
+        // per side for every 2 levels of radius 1, under the same 80 % rule (256 x 512 x nx:
+        // nx = 1000, two regions: 977 vs 782; 1024, three regions: 629 vs 786; 2048, five: 812
+        // vs 775; 4096, nine: 848 vs 761).
         const FusedConfig* c = nullptr;
         const int width = p->nx <= 128 ? 128 : p->nx <= 256 ? 256 : 512;
-        if (p->nx <= 512 && p->nx * 5 >= width * 4) {
+        const int tile = width - 2 * ((2 * p->radius + 3) / 4 * 4);          // columns a region stores
+        const int64_t regions = p->nx <= width ? 1 : (p->nx + tile - 1) / tile;
+        if ((int64_t)p->nx * 5 >= regions * width * 4) {
             c = find_fused_cfg(p->radius, 2, width, width == 128 ? 0 : 16);
             if (!c && width == 256) c = find_fused_cfg(p->radius, 2, 256);
         }

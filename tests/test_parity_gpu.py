@@ -353,6 +353,7 @@ FUSED_CONFIGS = [   # (radius, fuse_steps, region width, region height)
     ((33, 50, 128), 9),         # the same for the 128-wide regions; ragged in y, several z chunks
     ((21, 37, 512), 8),         # ... and for the 512-wide region, which is loaded as two TMA boxes
     ((19, 30, 452), 0),         # a row that ends inside the second box of a 512-wide region
+    ((9, 20, 1000), 0),         # two 512-wide regions per row
     ((5, 9, 12), 0),            # much smaller than one region
 ])
 def test_fused_passes_match_oracle(R, T, width, height, dims, chunk_z):
@@ -391,8 +392,10 @@ def test_fused_equals_unfused_within_tolerance_and_keeps_zero_boundary():
 
 def test_fuse_knob_rules():
     star = wl.star_weights(3, 1, 0.4, [0.1])
+    with b.Plan((64, 64, 1000), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 512      # two regions, 98 % of their lanes
     with b.Plan((64, 64, 1024), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 1         # rows wider than one region: unfused by default
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # would take three regions (two store 504 columns each): 67 %
         p.set(b.KEY_FUSE_STEPS, 4)
         assert p.get(b.KEY_FUSE_STEPS) == 4
     with b.Plan((64, 64, 320), 1, b.STAR, star, b.ZERO) as p:
