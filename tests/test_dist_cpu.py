@@ -63,7 +63,7 @@ def test_slab_ranges_cover_the_axis_once():
         assert max(sizes) - min(sizes) <= 1
 
 
-def _sharded_worker(rank, world, port, dims, R, steps, out):
+def _sharded_worker(rank, world, port, dims, R, steps, halo_steps, out):
     import numpy as np
     import oracle
     from paper_2608_21157_b200 import workloads as wl
@@ -76,36 +76,49 @@ def _sharded_worker(rank, world, port, dims, R, steps, out):
         w = wl.random_box_weights(ndim, R, 5)
         a = wl.normal_field(dims, 6)                    # every rank builds the same global field
 
-        def local_apply(src, dst):                      # one sweep of the local slab, on the CPU
-            dst.copy_(torch.from_numpy(oracle.apply(src.numpy(), w, oracle.ZERO, 1)))
+        calls = []
 
-        sw = ShardedSweep(dims, R, 1, w, rank=rank, world=world, dist=dist, local_apply=local_apply)
+        def local_apply(src, dst, nsteps):              # sweeps of the local slab, on the CPU
+            calls.append(nsteps)
+            dst.copy_(torch.from_numpy(oracle.apply(src.numpy(), w, oracle.ZERO, nsteps)))
+
+        sw = ShardedSweep(dims, R, 1, w, rank=rank, world=world, dist=dist, halo_steps=halo_steps,
+                          local_apply=local_apply)
+        expected_ghosts = halo_steps * R * ((rank > 0) + (rank < world - 1))
+        assert sw.local_dims[0] == (sw.z1 - sw.z0) + expected_ghosts
         ext = sw.scatter(torch.from_numpy(a))
         res = sw.apply(ext, steps)
-        out[rank] = (sw.z0, sw.z1, sw.interior(res).numpy().copy())
+        out[rank] = (sw.z0, sw.z1, sw.interior(res).numpy().copy(), list(calls))
         dist.barrier()
     finally:
         dist.destroy_process_group()
 
 
 @pytest.mark.timeout(180)
-@pytest.mark.parametrize("world,dims,R,steps", [(2, (11, 9, 12), 1, 3), (3, (13, 10), 2, 4), (2, (4, 6, 8), 2, 2)])
-def test_sharded_sweep_equals_the_single_grid_sweep(world, dims, R, steps):
+@pytest.mark.parametrize("world,dims,R,steps,halo_steps", [
+    (2, (11, 9, 12), 1, 3, 1), (3, (13, 10), 2, 4, 1), (2, (4, 6, 8), 2, 2, 1),
+    (2, (11, 9, 12), 1, 5, 2),      # two steps per exchange, the last round one step
+    (3, (19, 10), 2, 6, 3),         # three ranks, ghost zones of 6 rows, two rounds
+    (2, (12, 6, 8), 1, 4, 4),       # one exchange for the whole run
+])
+def test_sharded_sweep_equals_the_single_grid_sweep(world, dims, R, steps, halo_steps):
     """Halo exchange + local sweeps on 2-3 gloo ranks reproduce the sweep of the whole grid
-    bit for bit (every point sees the same neighbours in the same order)."""
+    bit for bit (every point sees the same neighbours in the same order), also when the
+    ghost zones are deep enough for several steps between two exchanges."""
     import numpy as np
     import oracle
     from paper_2608_21157_b200 import workloads as wl
     port = _free_port()
     with mp.Manager() as mgr:
         out = mgr.dict()
-        mp.spawn(_sharded_worker, args=(world, port, dims, R, steps, out), nprocs=world, join=True)
+        mp.spawn(_sharded_worker, args=(world, port, dims, R, steps, halo_steps, out), nprocs=world, join=True)
         parts = dict(out)
     w = wl.random_box_weights(len(dims), R, 5)
     a = wl.normal_field(dims, 6)
     want = oracle.apply(a, w, oracle.ZERO, steps)
     got = np.empty_like(want)
     for r in range(world):
-        z0, z1, block = parts[r]
+        z0, z1, block, calls = parts[r]
         got[z0:z1] = block
+        assert sum(calls) == steps and len(calls) == -(-steps // halo_steps) and max(calls) <= halo_steps
     assert np.array_equal(got, want)

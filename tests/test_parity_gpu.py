@@ -424,14 +424,15 @@ def test_fuse_knob_rules():
 
 
 # ------------------------------------------------------ sharded sweep, one rank --
-def test_sharded_sweep_single_rank_on_gpu():
-    """World size 1 of the slab decomposition runs the real kernels: ghost planes stay zero
-    and the result is the plain iterated sweep."""
+@pytest.mark.parametrize("halo_steps", [1, 2])
+def test_sharded_sweep_single_rank_on_gpu(halo_steps):
+    """World size 1 of the slab decomposition runs the real kernels (two steps per round:
+    the fused passes) and the result is the plain iterated sweep."""
     from paper_2608_21157_b200.sharded import ShardedSweep
     dims = (40, 48, 128)
     w = wl.star_weights(3, 1, 0.4, [0.1])
     a = wl.uniform_field(dims, 0.0, 1.0, 95)
-    sw = ShardedSweep(dims, 1, b.STAR, w, rank=0, world=1)
+    sw = ShardedSweep(dims, 1, b.STAR, w, rank=0, world=1, halo_steps=halo_steps)
     try:
         ext = sw.scatter(torch.from_numpy(a).cuda())
         res = sw.apply(ext, 5)
@@ -441,6 +442,47 @@ def test_sharded_sweep_single_rank_on_gpu():
         sw.close()
     want = oracle.apply(a, w, b.ZERO, 5)
     assert np.max(np.abs(got - want)) <= wl.tolerance(w, 1.0, 5)
+
+
+@pytest.mark.parametrize("world,halo_steps,steps", [(2, 1, 3), (3, 2, 5), (4, 2, 4), (2, 3, 6)])
+def test_sharded_slabs_with_real_kernels_ranks_emulated_in_one_process(world, halo_steps, steps):
+    """The slabs of 2-4 ranks swept by the real kernels on one GPU, one after the other, with
+    the halo exchange done by direct copies between the slabs (no process group, nothing
+    waits on anything): ghost depth, edge ranks without outer ghosts and several steps per
+    exchange give the sweep of the whole grid."""
+    from paper_2608_21157_b200.sharded import ShardedSweep
+    dims = (45, 40, 128)
+    R = 1
+    w = wl.star_weights(3, R, 0.4, [0.1])
+    a = wl.uniform_field(dims, 0.0, 1.0, 96)
+    g = torch.from_numpy(a).cuda()
+    sws = [ShardedSweep(dims, R, b.STAR, w, rank=r, world=world, dist=object(), halo_steps=halo_steps)
+           for r in range(world)]
+    try:
+        cur = [sw.scatter(g) for sw in sws]
+        other = [torch.empty_like(c) for c in cur]
+        D = halo_steps * R
+        done = 0
+        while done < steps:
+            n = min(halo_steps, steps - done)
+            own = [sw.interior(c) for sw, c in zip(sws, cur)]
+            for r, sw in enumerate(sws):
+                if r > 0:
+                    cur[r][:sw.lo].copy_(own[r - 1][-D:])
+                if r < world - 1:
+                    cur[r][sw.lo + sw.nlocal:].copy_(own[r + 1][:D])
+            for r, sw in enumerate(sws):
+                sw._local_apply(cur[r], other[r], n)
+            cur, other = other, cur
+            done += n
+        torch.cuda.synchronize()
+        got = torch.cat([sw.interior(c) for sw, c in zip(sws, cur)]).cpu().numpy()
+    finally:
+        for sw in sws:
+            sw.close()
+    want = oracle.apply(a, w, b.ZERO, steps)
+    assert got.shape == want.shape
+    assert np.max(np.abs(got - want)) <= wl.tolerance(w, 1.0, steps)
 
 
 # --------------------------------------------------------------------- FP64 --
