@@ -112,9 +112,14 @@ enum {
  *             off-axis entry is exactly zero, and is checked
  *             (STENCIL_ERR_INVALID otherwise).  Zero entries cost nothing.
  *   boundary  STENCIL_ZERO (taps outside the grid contribute 0; every grid
- *             point is an output) or STENCIL_PERIODIC (indices wrap; on the
- *             tiled kernels the plan then also owns a padded copy of the grid,
- *             allocated at the first apply).
+ *             point is an output) or STENCIL_PERIODIC (indices wrap).
+ *
+ * Plan-owned device memory, all allocated at first need by an apply: one
+ * scratch grid of N floats for steps > 1; two grids with rows padded to 16
+ * bytes when nx is not a multiple of 4 (zero boundary); one or two padded
+ * copies of the grid with wrapped halos when a periodic apply takes the
+ * padded-copy route (STENCIL_KEY_PERIODIC_ROUTE).  STENCIL_KEY_SCRATCH_BYTES
+ * reports the total.
  *
  * Needs no device memory until the first apply.  Errors: INVALID, UNSUPPORTED,
  * ALLOC.
@@ -145,18 +150,36 @@ STENCIL_API int stencil_apply(stencil_plan_t plan, const float* in, float* out, 
  * stencil_plan_f64 / stencil_apply_f64 — the same operation on FP64 grids, the
  * precision of the paper's own case study ("Case-study protocol": FP64).
  * Arguments, layout, ownership and errors are those of stencil_plan and
- * stencil_apply with double in place of float (rows must still be 16-byte
- * multiples for the tiled kernel: nx even).  A plan made by one of the two
+ * stencil_apply with double in place of float.  A plan made by one of the two
  * plan calls is only accepted by the matching apply call (STENCIL_ERR_INVALID
  * otherwise); stencil_destroy, stencil_query_status and the knobs serve both.
- * Grids with a zero boundary and an even nx run on TMA-staged kernels (2D:
- * star radius <= 4, box <= 3; 3D: star radius <= 4, box radius 1); everything
- * else on the one-thread-per-point kernel.
+ * TMA-staged kernels cover 2D star radius <= 4 and box radius <= 3, 3D star
+ * radius <= 4 and box radius 1, with a zero boundary (rows of an odd number of
+ * doubles through grids with padded rows) or a periodic one (even nx);
+ * everything else runs on the one-thread-per-point kernel.  No temporal
+ * blocking in FP64.
  */
 STENCIL_API int stencil_plan_f64(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radius,
                                  int shape, const double* weights, int boundary);
 STENCIL_API int stencil_apply_f64(stencil_plan_t plan, const double* in, double* out, int steps,
                                   void* stream);
+
+/*
+ * stencil_apply_planes — one sweep restricted to the output planes
+ * [z_begin, z_end) of a 3D grid:  out[z] = S(in)[z] for those planes, the rest
+ * of `out` is left untouched.  All of `in` the planes depend on (R planes on
+ * either side, inside the grid) must be valid.  Lets a caller that owns a slab
+ * of a larger grid sweep the planes that do not depend on its neighbours'
+ * data while that data is still on its way, and the others afterwards.  The
+ * paper has no counterpart (it runs on one GPU).
+ *
+ * fp32 plans on the tiled 3D kernel with a zero boundary and nx a multiple of 4
+ * only; STENCIL_ERR_UNSUPPORTED otherwise (2D, FP64, periodic, generic
+ * variant).  Pointers and errors as for stencil_apply; INVALID also for
+ * z_begin < 0, z_end > nz or z_begin >= z_end.  Enqueue only.
+ */
+STENCIL_API int stencil_apply_planes(stencil_plan_t plan, const float* in, float* out, int64_t z_begin,
+                                     int64_t z_end, void* stream);
 
 /*
  * stencil_apply_host — the same operation on HOST buffers: copies `in_host`

@@ -1508,6 +1508,24 @@ int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void
     return STENCIL_OK;
 }
 
+int stencil_apply_planes(stencil_plan_t p, const float* in, float* out, int64_t z_begin, int64_t z_end,
+                         void* stream) {
+    if (!valid_plan(p) || p->f64 || !in || !out) return STENCIL_ERR_INVALID;
+    const uintptr_t a = reinterpret_cast<uintptr_t>(in), b = reinterpret_cast<uintptr_t>(out);
+    if ((a | b) & 15u) return STENCIL_ERR_INVALID;
+    const uintptr_t bytes = (uintptr_t)p->npoints * sizeof(float);
+    if (a < b + bytes && b < a + bytes) return STENCIL_ERR_INVALID;
+    if (z_begin < 0 || z_end > p->nz || z_begin >= z_end) return STENCIL_ERR_INVALID;
+    if (p->variant != STENCIL_VARIANT_STREAM || p->ndim != 3 || p->boundary != STENCIL_ZERO || p->nx % 4 != 0)
+        return STENCIL_ERR_UNSUPPORTED;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int rc = ensure_device_state(p);
+    if (rc != STENCIL_OK) return rc;
+    p->last_stream = st;
+    p->used = true;
+    return launch_stream(p, in, out, st, (int)z_begin, (int)z_end);
+}
+
 int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps, void* stream) {
     if (!valid_plan(p) || !p->f64 || !in || !out || steps < 0) return STENCIL_ERR_INVALID;
     const uintptr_t a = reinterpret_cast<uintptr_t>(in), b = reinterpret_cast<uintptr_t>(out);

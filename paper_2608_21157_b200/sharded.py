@@ -13,14 +13,21 @@ rank's own planes, which are exact.  ``G = 1`` exchanges before every step;
 ``G = 2`` sends half as many messages (the same bytes) and lets the local sweep
 run its two-step fused passes.
 
+With ``G = 1`` a round also overlaps the exchange with compute where the local
+sweep can be restricted to a range of planes (``stencil_apply_planes``: 3D fp32,
+zero boundary): the sends and receives are started, the planes that read no
+ghost plane are swept meanwhile, and the R planes next to each neighbour follow
+once the ghost planes have arrived.
+
 The first rank has no ghost planes below and the last none above: their slabs
 end at the grid's own zero boundary, which the local plan imposes at every
 step.  There is no all-reduce or all-gather on the data path.
 
 The paper runs every task on a single GPU and leaves multi-GPU execution open;
 this module is the natural sharding of the sweep, kept outside the three-call C
-ABI.  It has only been exercised with several ranks on CPU (gloo) and with one
-rank on a GPU.
+ABI.  It has been exercised with several ranks on CPU (gloo), with one rank on a
+GPU, and with the slabs of several ranks swept one after the other on one GPU
+(exchange by direct copies), never yet on several GPUs.
 
 Zero boundary only: a periodic grid would also wrap the first rank's planes
 around to the last rank.
@@ -52,13 +59,16 @@ class ShardedSweep:
     ``local_apply(src, dst, steps)`` advances the local extended slab (own planes plus
     the ghost planes this rank has, zero boundary at its ends) by ``steps`` time steps
     from tensor ``src`` to tensor ``dst``; by default it is a ``binding.Plan`` on the
-    current CUDA stream.  Tests pass their own callable to drive the exchange logic
-    without a GPU.
+    current CUDA stream.  ``local_apply_planes(src, dst, z_begin, z_end)``, if given (or
+    if the default plan supports it), does one sweep for the output planes
+    [z_begin, z_end) of the extended slab only and enables the overlap of exchange and
+    compute.  Tests pass their own callables to drive the exchange logic without a GPU.
     """
 
     def __init__(self, dims: Sequence[int], radius: int, shape: int, weights: np.ndarray,
                  boundary: int = ZERO, *, rank: int, world: int, dist=None, group=None,
-                 halo_steps: int = 1, local_apply: Optional[Callable] = None):
+                 halo_steps: int = 1, local_apply: Optional[Callable] = None,
+                 local_apply_planes: Optional[Callable] = None, overlap: bool = True):
         if boundary != ZERO:
             raise ValueError("sharded sweeps support the zero boundary only")
         if halo_steps < 1:
@@ -85,7 +95,17 @@ class ShardedSweep:
 
             def local_apply(src, dst, steps):
                 self._plan.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
+
+            ranged = (len(self.dims) == 3 and self._plan.variant == "stream" and not self._plan.f64
+                      and self.dims[-1] % 4 == 0)
+            if ranged and local_apply_planes is None:
+                def local_apply_planes(src, dst, z_begin, z_end):
+                    self._plan.apply_planes(src, dst, z_begin, z_end, torch.cuda.current_stream().cuda_stream)
         self._local_apply = local_apply
+        self._local_apply_planes = local_apply_planes
+        # overlap needs one step per exchange, a ranged sweep and own planes that read no ghost plane
+        self.overlap = bool(overlap and self.G == 1 and self.world > 1 and local_apply_planes is not None
+                            and self.nlocal > 2 * self.R)
 
     # ---- layout helpers ---------------------------------------------------
     def scatter(self, global_field):
@@ -100,29 +120,30 @@ class ShardedSweep:
         return ext[self.lo:self.lo + self.nlocal]
 
     # ---- halo exchange ----------------------------------------------------
-    def exchange(self, ext) -> None:
-        """Fill the ghost planes of ``ext`` with the neighbours' outermost own planes."""
+    def start_exchange(self, ext):
+        """Start the sends of the outermost own planes and the receives into the ghost planes
+        of ``ext`` (slices along the slowest axis are contiguous, so both go straight from and
+        to the slab).  Returns the pending requests."""
         if self.world == 1:
-            return
+            return []
         d, D, n, lo = self.dist, self.depth, self.nlocal, self.lo
         ops = []
-        recv_lo = recv_hi = None
-        if self.rank > 0:
-            send_lo = ext[lo:lo + D].contiguous()            # my lowest planes -> lower neighbour's upper ghosts
-            recv_lo = ext.new_empty((D,) + tuple(ext.shape[1:]))
-            ops.append(d.P2POp(d.isend, send_lo, self.rank - 1, self.group))
-            ops.append(d.P2POp(d.irecv, recv_lo, self.rank - 1, self.group))
-        if self.rank < self.world - 1:
-            send_hi = ext[lo + n - D:lo + n].contiguous()    # my highest planes -> upper neighbour's lower ghosts
-            recv_hi = ext.new_empty((D,) + tuple(ext.shape[1:]))
-            ops.append(d.P2POp(d.isend, send_hi, self.rank + 1, self.group))
-            ops.append(d.P2POp(d.irecv, recv_hi, self.rank + 1, self.group))
-        for req in d.batch_isend_irecv(ops):
+        if self.rank > 0:                                    # my lowest planes <-> lower neighbour
+            ops.append(d.P2POp(d.isend, ext[lo:lo + D], self.rank - 1, self.group))
+            ops.append(d.P2POp(d.irecv, ext[:lo], self.rank - 1, self.group))
+        if self.rank < self.world - 1:                       # my highest planes <-> upper neighbour
+            ops.append(d.P2POp(d.isend, ext[lo + n - D:lo + n], self.rank + 1, self.group))
+            ops.append(d.P2POp(d.irecv, ext[lo + n:], self.rank + 1, self.group))
+        return d.batch_isend_irecv(ops)
+
+    @staticmethod
+    def finish_exchange(reqs) -> None:
+        for req in reqs:
             req.wait()
-        if recv_lo is not None:
-            ext[:lo].copy_(recv_lo)
-        if recv_hi is not None:
-            ext[lo + n:].copy_(recv_hi)
+
+    def exchange(self, ext) -> None:
+        """Fill the ghost planes of ``ext`` with the neighbours' outermost own planes."""
+        self.finish_exchange(self.start_exchange(ext))
 
     # ---- iteration ----------------------------------------------------------
     def apply(self, ext, steps: int = 1):
@@ -135,8 +156,23 @@ class ShardedSweep:
         done = 0
         while done < steps:
             r = min(self.G, steps - done)
-            self.exchange(cur)
-            self._local_apply(cur, other, r)
+            if self.overlap:
+                # own planes [lo + R, lo + n - R) read own planes only: sweep them while the ghost
+                # planes travel, then the R planes next to each neighbour (an edge rank's outer
+                # side has no ghosts: its planes belong to the first range)
+                R, lo, n = self.R, self.lo, self.nlocal
+                inner0 = lo + (R if self.rank > 0 else 0)
+                inner1 = lo + n - (R if self.rank < self.world - 1 else 0)
+                reqs = self.start_exchange(cur)
+                self._local_apply_planes(cur, other, inner0, inner1)
+                self.finish_exchange(reqs)
+                if inner0 > lo:
+                    self._local_apply_planes(cur, other, lo, inner0)
+                if inner1 < lo + n:
+                    self._local_apply_planes(cur, other, inner1, lo + n)
+            else:
+                self.exchange(cur)
+                self._local_apply(cur, other, r)
             cur, other = other, cur
             done += r
         return cur

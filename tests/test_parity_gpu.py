@@ -472,7 +472,17 @@ def test_sharded_slabs_with_real_kernels_ranks_emulated_in_one_process(world, ha
                 if r < world - 1:
                     cur[r][sw.lo + sw.nlocal:].copy_(own[r + 1][:D])
             for r, sw in enumerate(sws):
-                sw._local_apply(cur[r], other[r], n)
+                if sw.overlap:                          # one step per exchange: inner planes, then the edges
+                    lo, nl = sw.lo, sw.nlocal
+                    inner0 = lo + (R if r > 0 else 0)
+                    inner1 = lo + nl - (R if r < world - 1 else 0)
+                    sw._local_apply_planes(cur[r], other[r], inner0, inner1)
+                    if inner0 > lo:
+                        sw._local_apply_planes(cur[r], other[r], lo, inner0)
+                    if inner1 < lo + nl:
+                        sw._local_apply_planes(cur[r], other[r], inner1, lo + nl)
+                else:
+                    sw._local_apply(cur[r], other[r], n)
             cur, other = other, cur
             done += n
         torch.cuda.synchronize()
@@ -483,6 +493,44 @@ def test_sharded_slabs_with_real_kernels_ranks_emulated_in_one_process(world, ha
     want = oracle.apply(a, w, b.ZERO, steps)
     assert got.shape == want.shape
     assert np.max(np.abs(got - want)) <= wl.tolerance(w, 1.0, steps)
+
+
+@pytest.mark.parametrize("R,box", [(1, False), (4, False), (1, True), (2, True)])
+def test_apply_planes_sweeps_exactly_the_requested_planes(R, box):
+    dims = (37, 45, 132)
+    w = wl.random_box_weights(3, R, 97) if box else wl.random_star_weights(3, R, 97)
+    a = wl.normal_field(dims, 98)
+    want = oracle.apply(a, w, b.ZERO, 1)
+    tol = wl.tolerance(w, float(np.abs(a).max()), 1)
+    src = torch.from_numpy(a).cuda()
+    st = torch.cuda.current_stream().cuda_stream
+    with b.Plan(dims, R, b.BOX if box else b.STAR, w, b.ZERO) as p:
+        dst = torch.full_like(src, float("nan"))
+        p.apply_planes(src, dst, 5, 19, st)
+        torch.cuda.synchronize()
+        got = dst.cpu().numpy()
+        assert np.isnan(got[:5]).all() and np.isnan(got[19:]).all()         # nothing else was written
+        assert np.max(np.abs(got[5:19] - want[5:19])) <= tol
+        for z0, z1 in ((0, 5), (19, 36), (36, 37)):                          # the rest, in three more ranges
+            p.apply_planes(src, dst, z0, z1, st)
+        torch.cuda.synchronize()
+        assert p.query_status() == b.OK
+        assert np.max(np.abs(dst.cpu().numpy() - want)) <= tol
+        for z0, z1 in ((-1, 4), (3, 38), (7, 7), (9, 2)):
+            with pytest.raises(b.StencilError) as e:
+                p.apply_planes(src, dst, z0, z1, st)
+            assert e.value.status == b.ERR_INVALID
+    with b.Plan(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC) as p:
+        with pytest.raises(b.StencilError) as e:
+            p.apply_planes(src, torch.empty_like(src), 0, 4, st)
+        assert e.value.status == b.ERR_UNSUPPORTED
+    a2 = wl.normal_field((40, 64), 99)
+    w2 = wl.random_star_weights(2, 1, 97)
+    with b.Plan((40, 64), 1, b.STAR, w2, b.ZERO) as p:
+        s2 = torch.from_numpy(a2).cuda()
+        with pytest.raises(b.StencilError) as e:
+            p.apply_planes(s2, torch.empty_like(s2), 0, 1, st)
+        assert e.value.status == b.ERR_UNSUPPORTED
 
 
 # --------------------------------------------------------------------- FP64 --
