@@ -417,7 +417,21 @@ const FusedConfig* pick_fused(const stencil_plan_s* p) {
         const int tile = width - 2 * ((2 * p->radius + 3) / 4 * 4);          // columns a region stores
         const int64_t regions = p->nx <= width ? 1 : (p->nx + tile - 1) / tile;
         if ((int64_t)p->nx * 5 >= regions * width * 4) {
-            c = find_fused_cfg(p->radius, 2, width, width == 128 ? 0 : 16);
+            // 128-wide regions leave registers for a third level (512 x 512 x 128: 1224 G updates/s
+            // with three steps per pass, 1083 with two, 1108 with four); at 256 columns three
+            // levels spill (256^3: 820 against 1056)
+            // ... provided the grid still cuts into a machine's worth of CTAs (a B200 has 148
+            // SMs; 128^3 x 64 steps: 302 with three levels, 393 with two)
+            if (width == 128 && p->fuse_steps == 0) {
+                const FusedConfig* c3 = find_fused_cfg(p->radius, 3, 128);
+                if (c3) {
+                    const int tile_y = c3->tye - 2 * 3 * p->radius;
+                    const int64_t ctas = tile_y < 1 ? 0 : (int64_t)((p->ny + tile_y - 1) / tile_y) *
+                                                              std::max(1, p->nz / (4 * 3 * p->radius));
+                    if (ctas >= 148) c = c3;
+                }
+            }
+            if (!c) c = find_fused_cfg(p->radius, 2, width, width == 128 ? 0 : 16);
             if (!c && width == 256) c = find_fused_cfg(p->radius, 2, 256);
         }
         if (c || p->fuse_steps == 0) return c;

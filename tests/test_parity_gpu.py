@@ -409,6 +409,10 @@ def test_fuse_knob_rules():
     with b.Plan((64, 64, 200), 1, b.STAR, star, b.ZERO) as p:
         assert p.get(b.KEY_FUSE_STEPS) == 1         # 78 % of a 256-wide region
     with b.Plan((64, 64, 128), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 128     # too few CTAs for three levels
+    with b.Plan((512, 512, 128), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 3 and p.get(b.KEY_TILE_X) == 128     # narrow regions: three levels fit
+        p.set(b.KEY_FUSE_STEPS, 2)
         assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 128
     with b.Plan((64, 64, 256), 1, b.STAR, star, b.ZERO) as p:
         assert p.get(b.KEY_FUSE_STEPS) >= 2         # iterated applies fuse by default
