@@ -256,6 +256,13 @@ def _build_table() -> Dict[str, Workload]:
         lambda: star_weights(3, 1, -6.0, [1.0]),
         _resizable(lambda d: uniform_field(d, -1.0, 1.0, 1), (512, 512, 512)))
 
+    # supplementary: the widest box the tiled 3D kernel covers (125 taps: bound by the FMA pipe)
+    t["box3d_r2"] = Workload(
+        "box3d_r2", "3D 125-point box R=2 512^3, random weights with sum|w|=1, zero boundary, 1 step",
+        (512, 512, 512), 2, BOX, ZERO, 1,
+        lambda: random_box_weights(3, 2, 8),
+        _resizable(lambda d: normal_field(d, 9), (512, 512, 512)))
+
     # supplementary: the iterated heat update on a periodic 512^3 grid (stable weights)
     t["cfg5L_periodic"] = Workload(
         "cfg5L_periodic", "3D 7-point heat update R=1 512^3, periodic boundary, 16 steps",

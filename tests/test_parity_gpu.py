@@ -93,7 +93,8 @@ def test_generic_iteration_and_ping_pong(steps, boundary):
 def _stream_knob_sets(R, box):
     """Every compiled tile shape of the operator (tile_y = rows per thread x consumer warps)."""
     if box and R == 2:
-        return [dict(), dict(tile_y=16), dict(tile_y=14), dict(tile_y=8)]
+        return [dict(), dict(tile_y=16), dict(tile_y=14), dict(tile_y=8),
+                dict(tile_y=16, rows_per_thread=2)]
     if box or R == 1:
         return [dict(), dict(tile_y=16), dict(tile_y=14), dict(tile_y=32), dict(tile_y=28), dict(tile_y=8)]
     if R == 4:
