@@ -1046,8 +1046,13 @@ Stream64Config make_stream64() {
 
 const std::vector<Stream64Config>& stream64_configs() {
     static const std::vector<Stream64Config> v = {
-        make_stream64<1, false, 2, 8, 1>(), make_stream64<2, false, 2, 8, 1>(), make_stream64<3, false, 2, 8, 1>(),
-        make_stream64<4, false, 2, 8, 1>(), make_stream64<1, true, 2, 8, 1>(),
+        // The wide stars need their register count capped at two CTAs per SM (the last template
+        // argument): left alone the compiler takes 104 (R = 3) and 124 (R = 4) registers and a single
+        // 288-thread CTA fits.  Measured on 512^3 (GPoints/s), rows per thread x consumer warps:
+        // R = 3: 2 x 8 uncapped 285, capped 366, 4 x 4 capped 379; R = 4: 2 x 8 uncapped 273,
+        // capped 313, 2 x 7 capped 323.
+        make_stream64<1, false, 2, 8, 1>(), make_stream64<2, false, 2, 8, 1>(), make_stream64<3, false, 4, 4, 2>(),
+        make_stream64<4, false, 2, 7, 2>(), make_stream64<1, true, 2, 8, 1>(),
     };
     return v;
 }
@@ -1115,7 +1120,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
             rc = get_tensor_map_f64(p, cfg, kStream64PX, cfg->box_rows, src, &map);
         }
         if (rc != STENCIL_OK) return rc;
-        const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 4;
+        const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : (p->radius >= 3 ? 5 : 4);
         const size_t smem = (size_t)stages * cfg->plane_bytes + 128 + 2 * kMaxStages * sizeof(uint64_t);
         if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
         int dev = -1;
@@ -1147,6 +1152,22 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         // planes per chunk, so they get longer chunks (measured on 512^3)
         const int want_chunk = p->radius >= 3 ? 64 : 32;
         int chunk = p->chunk_z > 0 ? p->chunk_z : (p->nz >= 2 * want_chunk ? want_chunk : p->nz);
+        if (p->chunk_z <= 0 && p->radius >= 4) {
+            // The radius-4 star is no longer bound by memory alone (25 DFMA and 15 shared-memory
+            // loads per pair of points): every SM should get the same number of planes and as
+            // few re-read halo planes as possible, so z is cut into the number of chunks whose
+            // CTAs fill whole waves of the two-per-SM slots at the least cost (512^3: one chunk,
+            // 296 CTAs, 356 against 313 GPoints/s with 64-plane chunks).
+            const int64_t tiles = (int64_t)g.tiles_x * g.tiles_y;
+            const int64_t slots = 2 * (int64_t)sm_count();
+            double best = 1e300;
+            for (int n = 1; n <= std::max(1, p->nz / (4 * p->radius)); ++n) {
+                const int c = (p->nz + n - 1) / n;
+                const int64_t ctas = tiles * ((p->nz + c - 1) / c);
+                const double cost = (double)((ctas + slots - 1) / slots) * (c + 2 * p->radius + 4.0);
+                if (cost < best * 0.999) { best = cost; chunk = c; }
+            }
+        }
         chunk = std::max(1, std::min(chunk, p->nz));
         g.chunk_z = chunk;
         const int64_t grid64 = (int64_t)g.tiles_x * g.tiles_y * ((p->nz + chunk - 1) / chunk);
