@@ -271,7 +271,9 @@ const std::vector<StreamConfig>& stream_configs() {
         make_cfg<1, false, 2, 8, 1>(),  make_cfg<1, false, 2, 7, 4>(),  make_cfg<1, false, 4, 8, 1>(),
         make_cfg<1, false, 4, 7, 1>(),  make_cfg<1, false, 1, 8, 1>(),
         make_cfg<2, false, 2, 8, 1>(),  make_cfg<2, false, 2, 7, 1>(),  make_cfg<2, false, 4, 8, 1>(),
-        make_cfg<3, false, 2, 8, 1>(),  make_cfg<3, false, 2, 7, 2>(),  make_cfg<3, false, 4, 8, 1>(),
+        // radius 3: four rows per thread (32-row tiles: the 6 halo rows are 19 % of a plane instead
+        // of 43 % with 14-row tiles) measured 799 against 667 GPoints/s on 512^3
+        make_cfg<3, false, 4, 8, 1>(),  make_cfg<3, false, 2, 8, 2>(),  make_cfg<3, false, 2, 7, 2>(),
         make_cfg<4, false, 2, 8, 2>(),  make_cfg<4, false, 2, 7, 2>(),  make_cfg<4, false, 4, 8, 1>(),
         make_cfg<4, false, 2, 16, 1>(),
         make_cfg<1, true, 2, 8, 1>(),   make_cfg<1, true, 2, 7, 4>(),   make_cfg<1, true, 4, 8, 1>(),
@@ -679,7 +681,19 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
                   int z_end = 0) {
     if (z_end <= z_begin) { z_begin = 0; z_end = p->nz; }
     const int span = z_end - z_begin;
-    const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : (issue_bound(p) ? 5 : 4);
+    // ring depth: 5 for the issue-bound sweeps and the radius-2 star (750 against 732 GPoints/s), else 4
+    const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages)
+                                     : (issue_bound(p) || (p->shape == STENCIL_STAR && p->radius == 2) ? 5 : 4);
+    if (!p->stream_cfg_fixed && !p->stream_cfg_tuned && p->rows_per_thread == 0 && p->shape == STENCIL_STAR &&
+        p->radius == 3) {
+        // Radius 3: four rows per thread (128 x 32 tiles, little halo) win where the grid cuts into a
+        // machine's worth of such tiles with chunks of 64 planes or more; smaller grids balance better on
+        // two rows per thread (GPoints/s, four rows vs two: 512^3 797 vs 667; 300^3 440 vs 511; 128^3 91 vs
+        // 140; 64 x 1024^2 697 vs 716).
+        const int64_t big_tiles = (int64_t)((p->nx + kStreamTX - 1) / kStreamTX) * ((p->ny + 31) / 32);
+        const bool plentiful = big_tiles * (span / 64) >= 2 * (int64_t)sm_count();
+        if (const StreamConfig* c = find_stream_cfg(3, false, 0, plentiful ? 4 : 2)) p->stream_cfg = c;
+    }
     if (!p->stream_cfg_fixed && !p->stream_cfg_tuned) {
         // pick the tile height that balances this grid best (same rows per thread)
         const StreamConfig* best_cfg = p->stream_cfg;
