@@ -747,6 +747,20 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     return STENCIL_OK;
 }
 
+// Upper limit of the rows per (strip, chunk) unit of a 2D sweep.  The sweeps that are bound by
+// memory (stars, the 9-point box) run best as many short units that the hardware scheduler
+// balances, like the 3D ones: about 32 rows, more for wide stars whose 2R halo rows are re-read
+// by every unit (10240^2, GPoints/s, short vs one wave of long units: 5-point 791 vs 700,
+// 17-point star 667 vs 545, FP64 5-point 410 vs 361).  The boxes from 25 taps on are bound by
+// the FMA pipe and keep the one-wave rule (49-point: 526 vs 488).
+int short_chunk_2d(const stencil_plan_s* p, int YB) {
+    const int R = p->radius;
+    if (p->shape == STENCIL_BOX && R >= 2) return 0x7fffffff;
+    const int target = std::max(32, 16 * R);
+    const int nbatch = std::max(1, (target + 2 * R + YB / 2) / YB);
+    return std::max(1, nbatch * YB - 2 * R);
+}
+
 // 2D grids: one warp per (128-column strip, chunk of rows).
 int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
     const Rows2DConfig* cfg = p->rows2d_cfg;
@@ -798,6 +812,7 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
         int nbatch = std::max(1, (chunk_min + 2 * R + cfg->YB - 1) / cfg->YB);
         while (nbatch * cfg->YB - 2 * R < 1) ++nbatch;
         chunk = nbatch * cfg->YB - 2 * R;
+        chunk = std::min(chunk, short_chunk_2d(p, cfg->YB));
     }
     chunk = std::max(1, std::min(chunk, p->ny));
     g.chunk_y = chunk;
@@ -1236,6 +1251,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
             int nbatch = std::max(1, (chunk_min + 2 * R + cfg->YB - 1) / cfg->YB);
             while (nbatch * cfg->YB - 2 * R < 1) ++nbatch;
             chunk = nbatch * cfg->YB - 2 * R;
+            chunk = std::min(chunk, short_chunk_2d(p, cfg->YB));
         }
         chunk = std::max(1, std::min(chunk, p->ny));
         g.chunk_y = chunk;
