@@ -153,8 +153,8 @@ STENCIL_API int stencil_apply(stencil_plan_t plan, const float* in, float* out, 
  * stencil_apply with double in place of float.  A plan made by one of the two
  * plan calls is only accepted by the matching apply call (STENCIL_ERR_INVALID
  * otherwise); stencil_destroy, stencil_query_status and the knobs serve both.
- * TMA-staged kernels cover 2D star radius <= 4 and box radius <= 3, 3D star
- * radius <= 4 and box radius 1, with a zero boundary (rows of an odd number of
+ * TMA-staged kernels cover 2D star and box radius <= 4, 3D star radius <= 4
+ * and box radius <= 2, with a zero boundary (rows of an odd number of
  * doubles through grids with padded rows) or a periodic one (even nx);
  * everything else runs on the one-thread-per-point kernel.  No temporal
  * blocking in FP64.

@@ -4,9 +4,9 @@
 //
 // Differences: a lane owns one double2 (two points), so a tile is 64 columns wide; the x
 // neighbourhood of a lane is read from shared memory as aligned double2 loads instead of
-// being exchanged by shuffles.  At 16 B per point the sweep is bound by HBM for every
-// stencil the kernel covers (star radius <= 4: 25 DFMA per point at most; box radius 1:
-// 27), since the FP64 pipe sustains 64 DFMA per clock per SM.
+// being exchanged by shuffles.  At 16 B per point the sweep is bound by HBM for the stars
+// (radius <= 4: 25 DFMA per point at most) and the 27-point box, since the FP64 pipe
+// sustains 64 DFMA per clock per SM; the 125-point box is bound by that pipe.
 #pragma once
 #include "common.cuh"
 #include "kernel_stream.cuh"

@@ -1026,6 +1026,7 @@ const std::vector<Rows2D64Config>& rows2d64_configs() {
         // per SM (batches of 4 rows, 16 warps per CTA): 10240^2, 49 taps 291 against 265 GPoints/s, 25
         // taps 337 against 318
         make_rows2d64<1, true, 8, 8>(),  make_rows2d64<2, true, 4, 16>(),  make_rows2d64<3, true, 4, 16>(),
+        make_rows2d64<4, true, 4, 8>(),
     };
     return v;
 }
@@ -1087,7 +1088,7 @@ const std::vector<Stream64Config>& stream64_configs() {
         // R = 3: 2 x 8 uncapped 285, capped 366, 4 x 4 capped 379; R = 4: 2 x 8 uncapped 273,
         // capped 313, 2 x 7 capped 323.
         make_stream64<1, false, 2, 8, 1>(), make_stream64<2, false, 2, 8, 1>(), make_stream64<3, false, 4, 4, 2>(),
-        make_stream64<4, false, 2, 7, 2>(), make_stream64<1, true, 2, 8, 1>(),
+        make_stream64<4, false, 2, 7, 2>(), make_stream64<1, true, 2, 8, 1>(), make_stream64<2, true, 1, 8, 1>(),
     };
     return v;
 }
@@ -1187,9 +1188,10 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         // planes per chunk, so they get longer chunks (measured on 512^3)
         const int want_chunk = p->radius >= 3 ? 64 : 32;
         int chunk = p->chunk_z > 0 ? p->chunk_z : (p->nz >= 2 * want_chunk ? want_chunk : p->nz);
-        if (p->chunk_z <= 0 && p->radius >= 4) {
+        if (p->chunk_z <= 0 && (p->radius >= 4 || (p->shape == STENCIL_BOX && p->radius >= 2))) {
             // The radius-4 star is no longer bound by memory alone (25 DFMA and 15 shared-memory
-            // loads per pair of points): every SM should get the same number of planes and as
+            // loads per pair of points) and the 125-point box is bound by the FP64 pipe: every SM
+            // should get the same number of planes and as
             // few re-read halo planes as possible, so z is cut into the number of chunks whose
             // CTAs fill whole waves of the two-per-SM slots at the least cost (512^3: one chunk,
             // 296 CTAs, 356 against 313 GPoints/s with 64-plane chunks).

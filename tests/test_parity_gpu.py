@@ -550,7 +550,8 @@ def check_f64(dims, R, shape, w, boundary, a, steps=1, **kw):
     return used
 
 
-@pytest.mark.parametrize("R,box", [(1, False), (2, False), (3, False), (4, False), (1, True), (2, True), (3, True)])
+@pytest.mark.parametrize("R,box", [(1, False), (2, False), (3, False), (4, False), (1, True), (2, True), (3, True),
+                                   (4, True)])
 @pytest.mark.parametrize("dims,chunk,stages", [
     ((67, 66), 0, 0),            # two 64-column strips, the second 2 columns wide
     ((200, 258), 37, 2),         # several chunks of rows, chunk not a multiple of the batch
@@ -565,7 +566,7 @@ def test_f64_rows2d_kernel_matches_oracle(R, box, dims, chunk, stages):
     assert used == "stream"
 
 
-@pytest.mark.parametrize("R,box", [(1, False), (2, False), (3, False), (4, False), (1, True)])
+@pytest.mark.parametrize("R,box", [(1, False), (2, False), (3, False), (4, False), (1, True), (2, True)])
 @pytest.mark.parametrize("dims,chunk_z,stages", [
     ((37, 45, 66), 10, 3),       # two 64-column tiles, ragged in x, y and z
     ((8, 16, 64), 0, 0),         # exactly one tile
