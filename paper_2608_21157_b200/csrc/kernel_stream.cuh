@@ -324,15 +324,20 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
     } else {
         // M = 2R+1 accumulators per row; the accumulator of output plane z lives in slot
         // z mod M, so nothing is shifted: M planes per trip, slots known at compile time.
+        // From 125 taps on, M copies of the plane body (M x 500 FFMA per row) no longer fit the
+        // instruction cache (measured: 4 fetch stalls per issued instruction); there the body
+        // exists once and the M accumulators rotate by register moves after every plane
+        // (M moves against (2R+1)^3 FMAs).
         constexpr int M = 2 * R + 1;
+        constexpr int UNR = R >= 2 ? 1 : M;              // copies of the plane body
         float4 T[K][M];
 #pragma unroll
         for (int k = 0; k < K; ++k)
 #pragma unroll
             for (int d = 0; d < M; ++d) T[k][d] = make_float4(0.f, 0.f, 0.f, 0.f);
 
-        for (int i0 = 0; i0 < nplanes; i0 += M) {
-            const bool ok = static_for<M>([&](auto uc) -> bool {
+        for (int i0 = 0; i0 < nplanes; i0 += UNR) {
+            const bool ok = static_for<UNR>([&](auto uc) -> bool {
                 constexpr int u = decltype(uc)::value;
                 const int i = i0 + u;
                 if (i >= nplanes) return true;
@@ -384,6 +389,15 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                             if (row_ok[k]) store_f4(op + (size_t)k * g.nx, T[k][(u + R + 1) % M], streaming);
                     }
                     op += plane_stride;
+                }
+                if constexpr (UNR == 1) {                 // next plane finds every accumulator one slot down
+#pragma unroll
+                    for (int k = 0; k < K; ++k) {
+                        const float4 first = T[k][0];
+#pragma unroll
+                        for (int j = 0; j + 1 < M; ++j) T[k][j] = T[k][j + 1];
+                        T[k][M - 1] = first;
+                    }
                 }
                 return true;
             });
