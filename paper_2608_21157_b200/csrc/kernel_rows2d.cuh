@@ -49,6 +49,7 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
     using S = Rows2DShape<YB>;
     constexpr int PX = kStreamPX;
     constexpr int M = 2 * R + 1;
+    constexpr int kRowCopies = (BOX && R >= 3) ? 1 : YB;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     unsigned char* base = smem_raw + ((128u - (smem_addr(smem_raw) & 127u)) & 127u);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -108,7 +109,9 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
             return;
         }
         const float* bp = ring + (size_t)s * S::BATCH_FLOATS;
-#pragma unroll
+        // the big boxes keep one copy of the row body: YB copies of (2R+1)^2 FMAs per point would
+        // not fit the instruction cache
+#pragma unroll(kRowCopies)
         for (int r = 0; r < YB; ++r) {
             const int i = b * YB + r;                    // input row index inside the chunk
             if (i < nrows) {
