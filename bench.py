@@ -313,14 +313,33 @@ def run_gpu(args):
     algo_bytes = 2.0 * wk.itemsize * wk.npoints * steps_per_launch
     achieved = algo_bytes / (kernel_ms / 1e3) / 1e9
     fuse = plan.get(b.KEY_FUSE_STEPS) if wk.steps > 1 else 1
-    kernel_name = "stencil_generic_kernel" if plan.variant == "generic" else (
-        "stencil_fused_kernel" if fuse > 1 else "stencil_stream_kernel")
+    f64 = wk.itemsize == 8
+    if plan.variant == "generic":
+        kernel_name = "stencil_generic_kernel"
+    elif fuse > 1:
+        kernel_name = "stencil_fused_kernel"
+    elif len(wk.dims) == 2:
+        kernel_name = "stencil_rows2d_f64_kernel" if f64 else "stencil_rows2d_kernel"
+    else:
+        kernel_name = "stencil_stream_f64_kernel" if f64 else "stencil_stream_kernel"
     roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                 "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(wk.name),
                 "peak_kind": f"of {peak_kind} (copy bandwidth)", "kernel": kernel_name,
                 "kernel_ms": round(kernel_ms, 5), "algorithmic_bytes_per_launch": int(algo_bytes),
                 "time_steps_per_launch": steps_per_launch,
                 "frac_of_nominal_8tbs": round(achieved / NOMINAL_HBM_GBS, 4)}
+    # The sweeps with many taps are bound by plain FMA arithmetic, not by memory: report
+    # against whichever limit the kernel is closer to.  ALU peak = 148 SMs x 128 fp32 (64 FP64)
+    # FMA lanes x 2 flop x the maximum SM clock (1965 MHz).
+    taps = int(np.count_nonzero(wk.weights()))
+    alu_peak = 148 * (64 if f64 else 128) * 2 * 1.965e9 / 1e12
+    alu_achieved = 2.0 * taps * wk.npoints * steps_per_launch / (kernel_ms / 1e3) / 1e12
+    if alu_achieved / alu_peak > achieved / peak:
+        roofline.update({"bound": "alu", "achieved": round(alu_achieved, 2), "peak": round(alu_peak, 1),
+                         "unit": "TFLOP/s", "frac": round(alu_achieved / alu_peak, 4),
+                         "peak_kind": "148 SMs x %d FMA lanes x 2 flop x 1965 MHz (no measured peak for plain "
+                                      "FMA; the part runs 1.5-1.8 GHz under its power cap)" % (64 if f64 else 128),
+                         "hbm_frac_of_measured": round(achieved / peak, 4), "taps": taps})
     info = {"variant": plan.variant, "tile_y": plan.get(b.KEY_TILE_Y),
             "rows_per_thread": plan.get(b.KEY_ROWS_PER_THREAD), "fuse_steps": fuse}
     plan.destroy()

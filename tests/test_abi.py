@@ -168,3 +168,62 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(b, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         b.load()
+
+
+def test_fuse_knob_rules():
+    """Which iterated applies fuse time steps by default, and with which region (host logic only)."""
+    star = wl.star_weights(3, 1, 0.4, [0.1])
+    with b.Plan((64, 64, 1000), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 512      # two regions, 98 % of their lanes
+    with b.Plan((64, 64, 1024), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # would take three regions (two store 504 columns each): 67 %
+        p.set(b.KEY_FUSE_STEPS, 4)
+        assert p.get(b.KEY_FUSE_STEPS) == 4
+    with b.Plan((64, 64, 320), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # a 512-wide region would idle too many lanes
+    with b.Plan((64, 64, 512), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_FUSED_TILE_Y) == 16   # one 512-wide region per row
+    with b.Plan((64, 64, 448), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2
+    with b.Plan((64, 64, 64), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # half of a 128-wide region's lanes would idle
+    with b.Plan((64, 64, 200), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # 78 % of a 256-wide region
+    with b.Plan((64, 64, 128), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 128     # too few CTAs for three levels
+    with b.Plan((512, 512, 128), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 3 and p.get(b.KEY_TILE_X) == 128     # narrow regions: three levels fit
+        p.set(b.KEY_FUSE_STEPS, 2)
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 128
+    with b.Plan((64, 64, 256), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) >= 2         # iterated applies fuse by default
+        assert p.get(b.KEY_TILE_X) == 256 and p.get(b.KEY_FUSED_TILE_Y) == 16
+        p.set(b.KEY_FUSE_STEPS, 1)
+        assert p.get(b.KEY_FUSE_STEPS) == 1
+        with pytest.raises(b.StencilError):
+            p.set(b.KEY_FUSE_STEPS, 7)
+    with b.Plan((64, 64, 64), 1, b.BOX, wl.random_box_weights(3, 1, 3), b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # no fused kernel for box stencils
+        with pytest.raises(b.StencilError):
+            p.set(b.KEY_VARIANT, b.VARIANT_FUSED)
+
+
+def test_fp64_variant_selection_rules():
+    """Which FP64 requests the tiled kernels take (host logic only)."""
+    def plan(dims, R, box, boundary):
+        nd = len(dims)
+        w = (wl.random_box_weights if box else wl.random_star_weights)(nd, R, 3, np.float64)
+        return b.Plan(dims, R, b.BOX if box else b.STAR, w, boundary)
+    tiled = [((64, 64), 4, True, b.ZERO), ((64, 64), 4, False, b.PERIODIC), ((33, 65), 3, True, b.ZERO),
+             ((32, 32, 32), 2, True, b.ZERO), ((32, 32, 32), 4, False, b.PERIODIC), ((8, 9, 31), 1, True, b.ZERO)]
+    generic = [((64, 64), 5, True, b.ZERO), ((32, 32, 32), 3, True, b.ZERO), ((32, 32, 32), 5, False, b.ZERO),
+               ((32, 32, 31), 1, False, b.PERIODIC), ((64, 63), 1, False, b.PERIODIC)]
+    for args in tiled:
+        with plan(*args) as p:
+            assert p.f64 and p.variant == "stream", args
+    for args in generic:
+        with plan(*args) as p:
+            assert p.f64 and p.variant == "generic", args
+            with pytest.raises(b.StencilError) as e:
+                p.set(b.KEY_VARIANT, b.VARIANT_STREAM)
+            assert e.value.status == b.ERR_UNSUPPORTED

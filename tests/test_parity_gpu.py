@@ -391,43 +391,6 @@ def test_fused_equals_unfused_within_tolerance_and_keeps_zero_boundary():
     assert fused[0, 0, 0] < 0.5                     # the corner has lost heat to the zero exterior
 
 
-def test_fuse_knob_rules():
-    star = wl.star_weights(3, 1, 0.4, [0.1])
-    with b.Plan((64, 64, 1000), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 512      # two regions, 98 % of their lanes
-    with b.Plan((64, 64, 1024), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 1         # would take three regions (two store 504 columns each): 67 %
-        p.set(b.KEY_FUSE_STEPS, 4)
-        assert p.get(b.KEY_FUSE_STEPS) == 4
-    with b.Plan((64, 64, 320), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 1         # a 512-wide region would idle too many lanes
-    with b.Plan((64, 64, 512), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_FUSED_TILE_Y) == 16   # one 512-wide region per row
-    with b.Plan((64, 64, 448), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 2
-    with b.Plan((64, 64, 64), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 1         # half of a 128-wide region's lanes would idle
-    with b.Plan((64, 64, 200), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 1         # 78 % of a 256-wide region
-    with b.Plan((64, 64, 128), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 128     # too few CTAs for three levels
-    with b.Plan((512, 512, 128), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 3 and p.get(b.KEY_TILE_X) == 128     # narrow regions: three levels fit
-        p.set(b.KEY_FUSE_STEPS, 2)
-        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 128
-    with b.Plan((64, 64, 256), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) >= 2         # iterated applies fuse by default
-        assert p.get(b.KEY_TILE_X) == 256 and p.get(b.KEY_FUSED_TILE_Y) == 16
-        p.set(b.KEY_FUSE_STEPS, 1)
-        assert p.get(b.KEY_FUSE_STEPS) == 1
-        with pytest.raises(b.StencilError):
-            p.set(b.KEY_FUSE_STEPS, 7)
-    with b.Plan((64, 64, 64), 1, b.BOX, wl.random_box_weights(3, 1, 3), b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 1         # no fused kernel for box stencils
-        with pytest.raises(b.StencilError):
-            p.set(b.KEY_VARIANT, b.VARIANT_FUSED)
-
-
 # ------------------------------------------------------ sharded sweep, one rank --
 @pytest.mark.parametrize("halo_steps", [1, 2])
 def test_sharded_sweep_single_rank_on_gpu(halo_steps):
