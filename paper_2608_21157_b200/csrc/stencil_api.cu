@@ -21,6 +21,7 @@
 #include "kernel_stream.cuh"
 #include "kernel_fused.cuh"
 #include "kernel_rows2d.cuh"
+#include "kernel_rows2d_fused.cuh"
 #include "kernel_rows2d_f64.cuh"
 #include "kernel_stream_f64.cuh"
 
@@ -134,6 +135,20 @@ struct Rows2DConfig {
                           int grid, size_t smem, cudaStream_t);
 };
 
+// ---------------------------------------------------------------------------
+// ROWS2D FUSED kernel configurations (iterated 2D sweeps, T time steps per pass)
+// ---------------------------------------------------------------------------
+struct Rows2DFusedConfig {
+    int radius;
+    bool box;
+    int T, YB, NW, batch_bytes;
+    const void* kernel;
+    mutable size_t smem_allowed;
+    mutable int cache_device;
+    cudaError_t (*launch)(const struct stencil_plan_s*, const CUtensorMap&, float*, const Rows2DFusedGeom&,
+                          int grid, size_t smem, cudaStream_t);
+};
+
 }  // namespace
 
 struct Rows2D64Config {
@@ -201,6 +216,7 @@ struct stencil_plan_s {
     bool stream_cfg_tuned;         // the library has chosen it for this grid
     const FusedConfig* fused_cfg;  // non-null: iterated applies run fused passes
     const Rows2DConfig* rows2d_cfg; // non-null: 2D grid on the row-streaming kernel
+    const Rows2DFusedConfig* fused2d_cfg;  // non-null: iterated applies of a 2D grid run fused passes
     int tile_x;                    // requested region width for fused passes (0 = auto)
     int fused_tile_y;              // requested region height for fused passes (0 = any)
     // bookkeeping
@@ -387,6 +403,46 @@ const Rows2DConfig* find_rows2d_cfg(int radius, bool box) {
     return nullptr;
 }
 
+template <int R, bool BOX, int T, int YB, int NW>
+cudaError_t launch_rows2d_fused_t(const stencil_plan_s* p, const CUtensorMap& map, float* out,
+                                  const Rows2DFusedGeom& g, int grid, size_t smem, cudaStream_t st) {
+    Weights2D<R> wt;
+    for (int a = -R; a <= R; ++a)
+        for (int b = -R; b <= R; ++b) wt.w[a + R][b + R] = dense_w(p, 0, a, b);
+    return launch_kernel(&stencil_rows2d_fused_kernel<R, BOX, T, YB, NW>, grid, NW * 32, smem, st, p->chained, map,
+                         out, g, wt, p->d_status);
+}
+
+template <int R, bool BOX, int T, int YB, int NW>
+Rows2DFusedConfig make_rows2d_fused() {
+    Rows2DFusedConfig c;
+    c.radius = R; c.box = BOX; c.T = T; c.YB = YB; c.NW = NW; c.batch_bytes = Rows2DShape<YB>::BATCH_BYTES;
+    c.kernel = reinterpret_cast<const void*>(&stencil_rows2d_fused_kernel<R, BOX, T, YB, NW>);
+    c.smem_allowed = 0; c.cache_device = -1;
+    c.launch = &launch_rows2d_fused_t<R, BOX, T, YB, NW>;
+    return c;
+}
+
+// One depth per operator: the deepest with (T - 1) * R <= 4 (the columns a strip spoils must stay inside
+// its end lanes) that the operator's arithmetic leaves room for.
+const std::vector<Rows2DFusedConfig>& rows2d_fused_configs() {
+    static const std::vector<Rows2DFusedConfig> v = {
+        make_rows2d_fused<1, false, 4, 8, 8>(), make_rows2d_fused<1, true, 4, 8, 8>(),
+        make_rows2d_fused<2, false, 3, 8, 8>(), make_rows2d_fused<2, true, 2, 8, 8>(),
+        make_rows2d_fused<3, false, 2, 8, 8>(), make_rows2d_fused<4, false, 2, 8, 8>(),
+    };
+    return v;
+}
+
+// Temporal blocking of a 2D grid: zero boundary, 16-byte rows, the operators in the table above.
+const Rows2DFusedConfig* pick_fused2d(const stencil_plan_s* p) {
+    if (p->ndim != 2 || p->boundary != STENCIL_ZERO || p->nx % 4 != 0 || p->fuse_steps == 1) return nullptr;
+    for (const Rows2DFusedConfig& c : rows2d_fused_configs())
+        if (c.radius == p->radius && c.box == (p->shape == STENCIL_BOX) && (p->fuse_steps == 0 || p->fuse_steps == c.T))
+            return &c;
+    return nullptr;
+}
+
 // The tiled kernels need rows whose byte length is a multiple of 16 (a TMA stride rule).
 // The zero boundary comes from TMA's zero fill of out-of-grid cells; a periodic grid is first
 // copied into a padded grid with wrapped halos (kernel_pad.cuh) and swept from there.  A
@@ -450,12 +506,17 @@ const FusedConfig* pick_fused(const stencil_plan_s* p) {
 
 int resolve_variant(stencil_plan_s* p, int want) {
     if (want == STENCIL_VARIANT_AUTO) want = stream_supported(p) ? STENCIL_VARIANT_STREAM : STENCIL_VARIANT_GENERIC;
-    if (want == STENCIL_VARIANT_GENERIC) { p->variant = want; p->fused_cfg = nullptr; return STENCIL_OK; }
+    if (want == STENCIL_VARIANT_GENERIC) {
+        p->variant = want; p->fused_cfg = nullptr; p->fused2d_cfg = nullptr;
+        return STENCIL_OK;
+    }
     if (want == STENCIL_VARIANT_STREAM || want == STENCIL_VARIANT_FUSED) {
         if (!stream_supported(p)) return STENCIL_ERR_UNSUPPORTED;
         if (p->ndim == 2) {
-            if (want == STENCIL_VARIANT_FUSED) return STENCIL_ERR_UNSUPPORTED;
+            const Rows2DFusedConfig* f2 = pick_fused2d(p);
+            if (want == STENCIL_VARIANT_FUSED && !f2) return STENCIL_ERR_UNSUPPORTED;
             p->rows2d_cfg = find_rows2d_cfg(p->radius, p->shape == STENCIL_BOX);
+            p->fused2d_cfg = f2;
             p->stream_cfg = nullptr; p->fused_cfg = nullptr;
             p->variant = STENCIL_VARIANT_STREAM;
             return STENCIL_OK;
@@ -829,6 +890,59 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
 }
 
 // One fused pass: dst = S^nlev(src), nlev <= cfg->T.
+// One fused pass of a 2D grid: nlev time steps (1..T) from src to dst.
+int launch_rows2d_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cudaStream_t st) {
+    const Rows2DFusedConfig* cfg = p->fused2d_cfg;
+    const CUtensorMap* map = nullptr;
+    int rc = get_tensor_map(p, cfg, kStreamPX, cfg->YB, src, &map);
+    if (rc != STENCIL_OK) return rc;
+    const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
+    const size_t smem = (size_t)cfg->NW * stages * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8;
+    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    {
+        std::lock_guard<std::mutex> lock(g_config_mutex);
+        if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->cache_device = dev; }
+        if (smem > cfg->smem_allowed) {
+            if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess) {
+                cudaGetLastError();
+                return STENCIL_ERR_CUDA;
+            }
+            cfg->smem_allowed = smem;
+        }
+    }
+    Rows2DFusedGeom g;
+    g.ny = p->ny; g.nx = p->nx;
+    g.strips = (p->nx + kFused2DTile - 1) / kFused2DTile;
+    g.stages = stages;
+    g.nlev = nlev;
+    int chunk = p->chunk_z;                          // the streamed axis of a 2D grid is y
+    if (chunk <= 0) {
+        // A unit reads chunk + 2*nlev*R rows in batches of YB and recomputes the 2*nlev*R extra ones at
+        // every level, so chunks are long: 16 batches (6 % extra rows at a halo of 4), fewer only where the
+        // grid would otherwise not fill the machine's warp slots once.
+        const int H = nlev * p->radius;
+        const int slots = 2 * sm_count() * cfg->NW;
+        const int nch_max = std::max(1, slots / g.strips);
+        const int chunk_min = (p->ny + nch_max - 1) / nch_max;
+        int nbatch = std::max(1, (chunk_min + 2 * H + cfg->YB - 1) / cfg->YB);
+        nbatch = std::min(nbatch, 16);
+        while (nbatch * cfg->YB - 2 * H < 1) ++nbatch;
+        chunk = nbatch * cfg->YB - 2 * H;
+    }
+    chunk = std::max(1, std::min(chunk, p->ny));
+    g.chunk_y = chunk;
+    g.nchunks = (p->ny + chunk - 1) / chunk;
+    const int64_t units = (int64_t)g.strips * g.nchunks;
+    const int64_t grid64 = (units + cfg->NW - 1) / cfg->NW;
+    if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
+    if (cfg->launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
+    p->launches++;
+    return STENCIL_OK;
+}
+
 int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cudaStream_t st) {
     const FusedConfig* cfg = p->fused_cfg;
     const CUtensorMap* map = nullptr;
@@ -1444,7 +1558,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->copy_in = nullptr; p->copy_out = nullptr;
     p->variant = STENCIL_VARIANT_GENERIC;
     p->tile_y = 0; p->rows_per_thread = 0; p->chunk_z = 0; p->stages = 0; p->fuse_steps = 0; p->streaming_store = 0;
-    p->stream_cfg = nullptr; p->fused_cfg = nullptr; p->rows2d_cfg = nullptr; p->tile_x = 0; p->fused_tile_y = 0;
+    p->stream_cfg = nullptr; p->fused_cfg = nullptr; p->rows2d_cfg = nullptr; p->fused2d_cfg = nullptr; p->tile_x = 0; p->fused_tile_y = 0;
     p->stream_cfg_fixed = false; p->stream_cfg_tuned = false;
     p->wait_polls = kWaitPolls; p->drop_plane = -1;
     p->chain_launches = true; p->chained = false;
@@ -1566,8 +1680,10 @@ int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void
     // A pass advances the field by T time steps (T = 1 without temporal blocking).
     // Ping-pong between `out` and the scratch grid so that the last pass writes
     // `out` and `in` stays intact.
-    const bool fuse = p->variant == STENCIL_VARIANT_STREAM && p->fused_cfg != nullptr && steps > 1;
-    const int T = fuse ? p->fused_cfg->T : 1;
+    const bool fuse3d = p->variant == STENCIL_VARIANT_STREAM && p->fused_cfg != nullptr && steps > 1;
+    const bool fuse2d = p->variant == STENCIL_VARIANT_STREAM && p->fused2d_cfg != nullptr && steps > 1;
+    const bool fuse = fuse3d || fuse2d;
+    const int T = fuse3d ? p->fused_cfg->T : fuse2d ? p->fused2d_cfg->T : 1;
     const int passes = (steps + T - 1) / T;
     const float* src = in;
     int done = 0;
@@ -1576,7 +1692,9 @@ int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void
         float* dst = (remaining % 2 == 0) ? out : p->scratch;
         const int nlev = std::min(T, steps - done);
         p->chained = p->chain_launches && k > 0;
-        rc = (fuse && nlev > 1) ? launch_fused(p, src, dst, nlev, st) : launch_sweep(p, src, dst, st);
+        rc = !(fuse && nlev > 1) ? launch_sweep(p, src, dst, st)
+             : fuse3d           ? launch_fused(p, src, dst, nlev, st)
+                                : launch_rows2d_fused(p, src, dst, nlev, st);
         p->chained = false;
         if (rc != STENCIL_OK) return rc;
         done += nlev;
@@ -1849,7 +1967,15 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
             if (value < 0) return STENCIL_ERR_INVALID;
             const int old_fuse = p->fuse_steps, old_tx = p->tile_x;
             if (key == STENCIL_KEY_TILE_X) p->tile_x = (int)value; else p->fuse_steps = (int)value;
-            if (p->variant == STENCIL_VARIANT_STREAM) {
+            if (p->variant == STENCIL_VARIANT_STREAM && p->ndim == 2) {
+                // a 2D operator has one fused depth: 0 = use it, 1 = off, T = that depth
+                const Rows2DFusedConfig* f2 = pick_fused2d(p);
+                if ((!f2 && p->fuse_steps > 1) || (key == STENCIL_KEY_TILE_X && value != 0)) {
+                    p->fuse_steps = old_fuse; p->tile_x = old_tx;
+                    return STENCIL_ERR_UNSUPPORTED;
+                }
+                p->fused2d_cfg = f2;
+            } else if (p->variant == STENCIL_VARIANT_STREAM) {
                 const FusedConfig* f = pick_fused(p);
                 const bool wants_fusion = p->fuse_steps > 1 || (key == STENCIL_KEY_TILE_X && value != 0 && p->fuse_steps != 1);
                 if (!f && wants_fusion) { p->fuse_steps = old_fuse; p->tile_x = old_tx; return STENCIL_ERR_UNSUPPORTED; }
@@ -1935,7 +2061,10 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
             *value = (p->variant == STENCIL_VARIANT_STREAM && p->stream_cfg) ? p->stream_cfg->K : 0;
             return STENCIL_OK;
         case STENCIL_KEY_FUSE_STEPS:
-            *value = (p->variant == STENCIL_VARIANT_STREAM && p->fused_cfg) ? p->fused_cfg->T : 1;
+            *value = p->variant != STENCIL_VARIANT_STREAM ? 1
+                     : p->fused_cfg                           ? p->fused_cfg->T
+                     : p->fused2d_cfg                         ? p->fused2d_cfg->T
+                                                              : 1;
             return STENCIL_OK;
         case STENCIL_KEY_LAUNCHES: *value = p->launches; return STENCIL_OK;
         case STENCIL_KEY_SCRATCH_BYTES: {

@@ -256,6 +256,13 @@ def _build_table() -> Dict[str, Workload]:
         lambda: star_weights(3, 1, -6.0, [1.0]),
         _resizable(lambda d: uniform_field(d, -1.0, 1.0, 1), (512, 512, 512)))
 
+    # supplementary: the iterated 2D heat update (5 points) on the paper's grid size
+    t["heat2d"] = Workload(
+        "heat2d", "2D 5-point heat update u += 0.1*(sum nb - 4u), 10240^2, 16 steps, zero boundary",
+        (10240, 10240), 1, STAR, ZERO, 16,
+        lambda: star_weights(2, 1, 1.0 - 4 * 0.1, [0.1]),
+        _resizable(lambda d: uniform_field(d, 0.0, 1.0, 10), (10240, 10240)))
+
     # supplementary: the widest box the tiled 3D kernel covers (125 taps: bound by the FMA pipe)
     t["box3d_r2"] = Workload(
         "box3d_r2", "3D 125-point box R=2 512^3, random weights with sum|w|=1, zero boundary, 1 step",

@@ -227,3 +227,28 @@ def test_fp64_variant_selection_rules():
             with pytest.raises(b.StencilError) as e:
                 p.set(b.KEY_VARIANT, b.VARIANT_STREAM)
             assert e.value.status == b.ERR_UNSUPPORTED
+
+
+def test_fuse_rules_2d():
+    """Iterated 2D applies fuse T steps per pass for the operators with a fused kernel (host logic only)."""
+    for R, box, T in [(1, False, 4), (1, True, 4), (2, False, 3), (2, True, 2), (3, False, 2), (4, False, 2)]:
+        w = wl.random_box_weights(2, R, 3) if box else wl.random_star_weights(2, R, 3)
+        with b.Plan((64, 128), R, b.BOX if box else b.STAR, w, b.ZERO) as p:
+            assert p.get(b.KEY_FUSE_STEPS) == T
+            p.set(b.KEY_FUSE_STEPS, 1)
+            assert p.get(b.KEY_FUSE_STEPS) == 1
+            p.set(b.KEY_FUSE_STEPS, T)
+            assert p.get(b.KEY_FUSE_STEPS) == T
+            with pytest.raises(b.StencilError) as e:
+                p.set(b.KEY_FUSE_STEPS, T + 1)
+            assert e.value.status == b.ERR_UNSUPPORTED and p.get(b.KEY_FUSE_STEPS) == T
+            p.set(b.KEY_FUSE_STEPS, 0)
+            assert p.get(b.KEY_FUSE_STEPS) == T
+        with b.Plan((64, 128), R, b.BOX if box else b.STAR, w, b.PERIODIC) as p:
+            assert p.get(b.KEY_FUSE_STEPS) == 1         # no temporal blocking under a periodic boundary
+        with b.Plan((64, 126), R, b.BOX if box else b.STAR, w, b.ZERO) as p:
+            assert p.get(b.KEY_FUSE_STEPS) == 1         # rows that are not 16-byte multiples
+    with b.Plan((64, 128), 3, b.BOX, wl.random_box_weights(2, 3, 3), b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1             # the 49-point box is bound by the FMA pipe: not fused
+        with pytest.raises(b.StencilError):
+            p.set(b.KEY_VARIANT, b.VARIANT_FUSED)

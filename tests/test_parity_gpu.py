@@ -340,6 +340,49 @@ def test_paper_shaped_2d_box_radius3():
     assert np.max(np.abs(got - want)) <= wl.tolerance(w, float(np.abs(a).max()), wk.steps)
 
 
+# ------------------------------------------------------------ 2D temporal blocking --
+FUSED2D_OPS = [(1, False, 4), (1, True, 4), (2, False, 3), (2, True, 2), (3, False, 2), (4, False, 2)]   # R, box, T
+
+
+@pytest.mark.parametrize("R,box,T", FUSED2D_OPS)
+@pytest.mark.parametrize("dims,chunk,stages", [
+    ((67, 132), 0, 0),           # two strips (each stores 120 columns), ragged in both axes
+    ((200, 260), 37, 2),         # three strips, several chunks of rows, chunk not a multiple of the batch
+    ((3, 8), 0, 0),              # smaller than the reach of T steps
+    ((129, 512), 16, 4),         # five strips; chunks shorter than their halo of T*R rows on either side
+    ((300, 120), 0, 0),          # exactly one strip
+])
+def test_fused_2d_passes_match_oracle(R, box, T, dims, chunk, stages):
+    w = wl.random_box_weights(2, R, 71) if box else wl.random_star_weights(2, R, 71)    # sum|w| = 1
+    a = wl.normal_field(dims, 72)
+    for steps in (T, T + 1, 2 * T + 1, 2):
+        dev = torch.device("cuda:0")
+        src = torch.from_numpy(a).to(dev)
+        dst = torch.full_like(src, float("nan"))
+        with b.Plan(dims, R, b.BOX if box else b.STAR, w, b.ZERO, chunk_z=chunk or None, stages=stages or None) as p:
+            assert p.variant == "stream" and p.get(b.KEY_FUSE_STEPS) == T
+            p.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
+            assert p.query_status() == b.OK
+            assert p.launches == -(-steps // T)
+        got = dst.cpu().numpy()
+        want = oracle.apply(a, w, b.ZERO, steps)
+        tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+        err = float(np.max(np.abs(got - want)))
+        assert err <= tol, f"R={R} box={box} T={T} dims={dims} steps={steps}: {err:.3e} > {tol:.3e}"
+
+
+def test_fused_2d_equals_unfused_and_keeps_the_zero_boundary():
+    dims = (96, 384)
+    w = wl.star_weights(2, 1, 0.6, [0.1])                 # heat update: constant fields decay only at the edges
+    a = np.ones(dims, dtype=np.float32)
+    fused, _ = gpu_sweep(dims, 1, b.STAR, w, b.ZERO, a, steps=8)
+    plain, _ = gpu_sweep(dims, 1, b.STAR, w, b.ZERO, a, steps=8, fuse_steps=1)
+    want = oracle.apply(a, w, b.ZERO, 8)
+    tol = wl.tolerance(w, 1.0, 8)
+    assert np.max(np.abs(fused - want)) <= tol and np.max(np.abs(plain - want)) <= tol
+    assert fused[0, 0] < 0.5 and abs(fused[48, 192] - 1.0) < 1e-5
+
+
 # -------------------------------------------------------------------- fused --
 FUSED_CONFIGS = [   # (radius, fuse_steps, region width, region height)
     (1, 2, 256, 32), (1, 2, 256, 16), (1, 3, 256, 32), (1, 4, 128, 32), (1, 2, 128, 32), (1, 3, 128, 32),
