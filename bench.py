@@ -44,6 +44,7 @@ NCU_TRAFFIC_BYTES = {
     "cfg4": 995.7e6,    # stream kernel, star R=4
     "cfg5": 99.9e6,     # one fused pass (2 time steps of 256^3): 77.7 MB read + 22.2 MB written
     "cfg5L": 1035.1e6,  # one fused pass (2 time steps of 512^3): 545.4 MB read + 489.7 MB written
+    "heat2d": 756.3e6,  # one fused pass (4 time steps of 10240^2): 2.5 x (180.6 + 121.9 MB) captured on 4096 x 10240
 }
 
 
@@ -317,7 +318,7 @@ def run_gpu(args):
     if plan.variant == "generic":
         kernel_name = "stencil_generic_kernel"
     elif fuse > 1:
-        kernel_name = "stencil_fused_kernel"
+        kernel_name = "stencil_rows2d_fused_kernel" if len(wk.dims) == 2 else "stencil_fused_kernel"
     elif len(wk.dims) == 2:
         kernel_name = "stencil_rows2d_f64_kernel" if f64 else "stencil_rows2d_kernel"
     else:
@@ -540,7 +541,7 @@ def main():
     ap.add_argument("--stages", type=int, default=None)
     ap.add_argument("--fuse-steps", dest="fuse_steps", type=int, default=None)
     ap.add_argument("--streaming-store", dest="streaming_store", type=int, default=None)
-    ap.add_argument("--also", default="cfg1,cfg3,cfg4,cfg5,cfg5L,paper2d,paper2d_f64", help="other workloads summarised in all_configs")
+    ap.add_argument("--also", default="cfg1,cfg3,cfg4,cfg5,cfg5L,paper2d,paper2d_f64,heat2d", help="other workloads summarised in all_configs")
     ap.add_argument("--also-steps", dest="also_steps", type=int, default=20)
     ap.add_argument("--no-all-configs", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
