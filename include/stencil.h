@@ -156,8 +156,8 @@ STENCIL_API int stencil_apply(stencil_plan_t plan, const float* in, float* out, 
  * TMA-staged kernels cover 2D star and box radius <= 4, 3D star radius <= 4
  * and box radius <= 2, with a zero boundary (rows of an odd number of
  * doubles through grids with padded rows) or a periodic one (even nx);
- * everything else runs on the one-thread-per-point kernel.  No temporal
- * blocking in FP64.
+ * everything else runs on the one-thread-per-point kernel.  Temporal blocking
+ * in FP64 exists for 2D grids with radius <= 2 (zero boundary, even nx).
  */
 STENCIL_API int stencil_plan_f64(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radius,
                                  int shape, const double* weights, int boundary);

@@ -23,6 +23,7 @@
 #include "kernel_rows2d.cuh"
 #include "kernel_rows2d_fused.cuh"
 #include "kernel_rows2d_f64.cuh"
+#include "kernel_rows2d_fused_f64.cuh"
 #include "kernel_stream_f64.cuh"
 
 using namespace stencil;
@@ -153,6 +154,19 @@ struct Rows2DFusedConfig {
 
 }  // namespace
 
+struct Rows2DFused64Config {
+    int radius;
+    bool box;
+    int T, YB, NW, batch_bytes;
+    const void* kernel;
+    mutable size_t smem_allowed;
+    mutable size_t occ_smem;
+    mutable int occ;
+    mutable int cache_device;
+    cudaError_t (*launch)(const struct stencil_plan_s*, const CUtensorMap&, double*, const stencil::Rows2DFusedGeom&,
+                          int grid, size_t smem, cudaStream_t);
+};
+
 struct Rows2D64Config {
     int radius;
     bool box;
@@ -189,6 +203,7 @@ struct stencil_plan_s {
     TapT<double>* d_taps64;
     double* scratch64;             // N doubles, iteration ping-pong of FP64 plans
     const struct Rows2D64Config* rows2d64_cfg;
+    const struct Rows2DFused64Config* fused2d64_cfg;   // non-null: iterated applies of a 2D FP64 grid run fused passes
     const struct Stream64Config* stream64_cfg;
     // device state (created lazily, on the device current at first apply)
     int device;
@@ -1228,16 +1243,54 @@ const Stream64Config* find_stream64_cfg(const stencil_plan_s* p) {
     return nullptr;
 }
 
+template <int R, bool BOX, int T, int YB, int NW>
+cudaError_t launch_rows2d_fused64_t(const stencil_plan_s* p, const CUtensorMap& map, double* out,
+                                    const Rows2DFusedGeom& g, int grid, size_t smem, cudaStream_t st) {
+    Weights2D64<R> wt;
+    for (int a = -R; a <= R; ++a)
+        for (int b = -R; b <= R; ++b) wt.w[a + R][b + R] = dense_w64(p, a, b);
+    return launch_kernel(&stencil_rows2d_fused_f64_kernel<R, BOX, T, YB, NW>, grid, NW * 32, smem, st, p->chained,
+                         map, out, g, wt, p->d_status);
+}
+
+template <int R, bool BOX, int T, int YB, int NW>
+Rows2DFused64Config make_rows2d_fused64() {
+    Rows2DFused64Config c;
+    c.radius = R; c.box = BOX; c.T = T; c.YB = YB; c.NW = NW; c.batch_bytes = Rows2D64Shape<YB>::BATCH_BYTES;
+    c.kernel = reinterpret_cast<const void*>(&stencil_rows2d_fused_f64_kernel<R, BOX, T, YB, NW>);
+    c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
+    c.launch = &launch_rows2d_fused64_t<R, BOX, T, YB, NW>;
+    return c;
+}
+
+// FP64 twin of rows2d_fused_configs(): radius <= 2 (one neighbour lane per side in the register exchange).
+const std::vector<Rows2DFused64Config>& rows2d_fused64_configs() {
+    static const std::vector<Rows2DFused64Config> v = {
+        make_rows2d_fused64<1, false, 4, 8, 8>(), make_rows2d_fused64<1, true, 4, 8, 8>(),
+        make_rows2d_fused64<2, false, 3, 8, 8>(), make_rows2d_fused64<2, true, 2, 8, 8>(),
+    };
+    return v;
+}
+
+const Rows2DFused64Config* pick_fused2d64(const stencil_plan_s* p) {
+    if (p->ndim != 2 || p->boundary != STENCIL_ZERO || p->nx % 2 != 0 || p->fuse_steps == 1) return nullptr;
+    for (const Rows2DFused64Config& c : rows2d_fused64_configs())
+        if (c.radius == p->radius && c.box == (p->shape == STENCIL_BOX) && (p->fuse_steps == 0 || p->fuse_steps == c.T))
+            return &c;
+    return nullptr;
+}
+
 int resolve_variant_f64(stencil_plan_s* p, int want) {
     const Rows2D64Config* c2 = find_rows2d64_cfg(p);
     const Stream64Config* c3 = find_stream64_cfg(p);
     if (want == STENCIL_VARIANT_AUTO) want = (c2 || c3) ? STENCIL_VARIANT_STREAM : STENCIL_VARIANT_GENERIC;
     if (want == STENCIL_VARIANT_GENERIC) {
-        p->variant = want; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr;
+        p->variant = want; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr; p->fused2d64_cfg = nullptr;
         return STENCIL_OK;
     }
     if (want == STENCIL_VARIANT_STREAM && (c2 || c3)) {
         p->variant = want; p->rows2d64_cfg = c2; p->stream64_cfg = c3;
+        p->fused2d64_cfg = c2 ? pick_fused2d64(p) : nullptr;
         return STENCIL_OK;
     }
     return STENCIL_ERR_UNSUPPORTED;
@@ -1266,6 +1319,65 @@ int get_tensor_map_f64(stencil_plan_s* p, const void* cfg, int box_x, int box_y,
     if (p->maps.size() >= 8) p->maps.erase(p->maps.begin());
     p->maps.push_back(e);
     *out = &p->maps.back().map;
+    return STENCIL_OK;
+}
+
+// One fused pass of a 2D FP64 grid: nlev time steps (1..T) from src to dst.
+int launch_rows2d_fused64(stencil_plan_s* p, const double* src, double* dst, int nlev, cudaStream_t st) {
+    const Rows2DFused64Config* cfg = p->fused2d64_cfg;
+    const CUtensorMap* map = nullptr;
+    int rc = get_tensor_map_f64(p, cfg, kPX64, cfg->YB, src, &map);
+    if (rc != STENCIL_OK) return rc;
+    const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 2;
+    const size_t smem = (size_t)cfg->NW * stages * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8;
+    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
+    int dev = -1, occ = 1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    {
+        std::lock_guard<std::mutex> lock(g_config_mutex);
+        if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->occ_smem = 0; cfg->cache_device = dev; }
+        if (smem > cfg->smem_allowed) {
+            if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess) {
+                cudaGetLastError();
+                return STENCIL_ERR_CUDA;
+            }
+            cfg->smem_allowed = smem;
+        }
+        if (cfg->occ_smem != smem) {
+            int o = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, cfg->kernel, cfg->NW * 32, smem) != cudaSuccess) {
+                cudaGetLastError();
+                o = 0;
+            }
+            cfg->occ = std::max(o, 1);
+            cfg->occ_smem = smem;
+        }
+        occ = cfg->occ;
+    }
+    Rows2DFusedGeom g;
+    g.ny = p->ny; g.nx = p->nx;
+    g.strips = (p->nx + kFused2D64Tile - 1) / kFused2D64Tile;
+    g.stages = stages;
+    g.nlev = nlev;
+    int chunk = p->chunk_z;
+    if (chunk <= 0) {                                 // same sizing rule as the fp32 kernel
+        const int H = nlev * p->radius;
+        const int slots = occ * sm_count() * cfg->NW;
+        const int nch_max = std::max(1, slots / g.strips);
+        const int chunk_min = (p->ny + nch_max - 1) / nch_max;
+        int nbatch = std::max(1, (chunk_min + 2 * H + cfg->YB - 1) / cfg->YB);
+        while (nbatch * cfg->YB - 2 * H < 1) ++nbatch;
+        chunk = nbatch * cfg->YB - 2 * H;
+    }
+    chunk = std::max(1, std::min(chunk, p->ny));
+    g.chunk_y = chunk;
+    g.nchunks = (p->ny + chunk - 1) / chunk;
+    const int64_t units = (int64_t)g.strips * g.nchunks;
+    const int64_t grid64 = (units + cfg->NW - 1) / cfg->NW;
+    if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
+    if (cfg->launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
+    p->launches++;
     return STENCIL_OK;
 }
 
@@ -1567,7 +1679,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->radius = radius; p->shape = shape; p->boundary = boundary;
     p->device = -1;
     p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0; p->src_padded = false; p->periodic_route = 0;
-    p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr;
+    p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr; p->fused2d64_cfg = nullptr;
     p->host_in = nullptr; p->host_out = nullptr;
     p->copy_in = nullptr; p->copy_out = nullptr;
     p->variant = STENCIL_VARIANT_GENERIC;
@@ -1765,14 +1877,21 @@ int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps
         if (use_wrap_correction(p, steps)) return apply_periodic_corrected(p, in, out, p->scratch64, steps, st);
         if (steps > 1) return apply_periodic(p, in, out, steps, st);
     }
+    // A pass advances the field by T time steps (T = 1 without temporal blocking), as in stencil_apply.
+    const bool fuse = p->variant == STENCIL_VARIANT_STREAM && p->fused2d64_cfg != nullptr && steps > 1;
+    const int T = fuse ? p->fused2d64_cfg->T : 1;
+    const int passes = (steps + T - 1) / T;
     const double* src = in;
-    for (int k = 0; k < steps; ++k) {
-        const int remaining = steps - 1 - k;
+    int done = 0;
+    for (int k = 0; k < passes; ++k) {
+        const int remaining = passes - 1 - k;
         double* dst = (remaining % 2 == 0) ? out : p->scratch64;
+        const int nlev = std::min(T, steps - done);
         p->chained = p->chain_launches && k > 0;
-        rc = launch_sweep_f64(p, src, dst, st);
+        rc = (fuse && nlev > 1) ? launch_rows2d_fused64(p, src, dst, nlev, st) : launch_sweep_f64(p, src, dst, st);
         p->chained = false;
         if (rc != STENCIL_OK) return rc;
+        done += nlev;
         src = dst;
     }
     return STENCIL_OK;
@@ -1976,7 +2095,18 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
         }
         case STENCIL_KEY_TILE_X:
         case STENCIL_KEY_FUSE_STEPS: {
-            if (p->f64) return value <= 1 ? STENCIL_OK : STENCIL_ERR_UNSUPPORTED;
+            if (p->f64) {
+                // FP64: only the 2D register cascade exists; 0 = use it, 1 = off, T = its depth
+                if (key == STENCIL_KEY_TILE_X) return value == 0 ? STENCIL_OK : STENCIL_ERR_UNSUPPORTED;
+                if (value < 0) return STENCIL_ERR_INVALID;
+                const int old = p->fuse_steps;
+                p->fuse_steps = (int)value;
+                const Rows2DFused64Config* f2 =
+                    (p->variant == STENCIL_VARIANT_STREAM && p->rows2d64_cfg) ? pick_fused2d64(p) : nullptr;
+                if (!f2 && value > 1) { p->fuse_steps = old; return STENCIL_ERR_UNSUPPORTED; }
+                p->fused2d64_cfg = f2;
+                return STENCIL_OK;
+            }
             // region width (128, 256 or 512) and time steps per pass of the fused kernel
             if (value < 0) return STENCIL_ERR_INVALID;
             const int old_fuse = p->fuse_steps, old_tx = p->tile_x;
@@ -2078,6 +2208,7 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
             *value = p->variant != STENCIL_VARIANT_STREAM ? 1
                      : p->fused_cfg                           ? p->fused_cfg->T
                      : p->fused2d_cfg                         ? p->fused2d_cfg->T
+                     : p->fused2d64_cfg                       ? p->fused2d64_cfg->T
                                                               : 1;
             return STENCIL_OK;
         case STENCIL_KEY_LAUNCHES: *value = p->launches; return STENCIL_OK;

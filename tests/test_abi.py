@@ -252,3 +252,26 @@ def test_fuse_rules_2d():
         assert p.get(b.KEY_FUSE_STEPS) == 1             # the 49-point box is bound by the FMA pipe: not fused
         with pytest.raises(b.StencilError):
             p.set(b.KEY_VARIANT, b.VARIANT_FUSED)
+
+
+def test_fuse_rules_2d_fp64():
+    for R, box, T in [(1, False, 4), (1, True, 4), (2, False, 3), (2, True, 2)]:
+        w = (wl.random_box_weights if box else wl.random_star_weights)(2, R, 3, np.float64)
+        with b.Plan((64, 128), R, b.BOX if box else b.STAR, w, b.ZERO) as p:
+            assert p.f64 and p.get(b.KEY_FUSE_STEPS) == T
+            p.set(b.KEY_FUSE_STEPS, 1)
+            assert p.get(b.KEY_FUSE_STEPS) == 1
+            with pytest.raises(b.StencilError):
+                p.set(b.KEY_FUSE_STEPS, T + 1)
+            p.set(b.KEY_FUSE_STEPS, 0)
+            assert p.get(b.KEY_FUSE_STEPS) == T
+        with b.Plan((64, 127), R, b.BOX if box else b.STAR, w, b.ZERO) as p:
+            assert p.get(b.KEY_FUSE_STEPS) == 1         # odd rows run between padded-row grids, unfused
+    w = wl.random_star_weights(2, 3, 3, np.float64)
+    with b.Plan((64, 128), 3, b.STAR, w, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1             # radius 3 needs two neighbour lanes: no FP64 cascade
+    w = wl.random_star_weights(3, 1, 3, np.float64)
+    with b.Plan((32, 32, 64), 1, b.STAR, w, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1             # no FP64 temporal blocking in 3D
+        with pytest.raises(b.StencilError):
+            p.set(b.KEY_FUSE_STEPS, 2)

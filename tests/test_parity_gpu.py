@@ -383,6 +383,34 @@ def test_fused_2d_equals_unfused_and_keeps_the_zero_boundary():
     assert fused[0, 0] < 0.5 and abs(fused[48, 192] - 1.0) < 1e-5
 
 
+@pytest.mark.parametrize("R,box,T", [(1, False, 4), (1, True, 4), (2, False, 3), (2, True, 2)])
+@pytest.mark.parametrize("dims,chunk,stages", [
+    ((67, 66), 0, 0),            # two strips (each stores 56 columns), ragged in both axes
+    ((200, 130), 37, 2),         # three strips, several chunks of rows
+    ((3, 8), 0, 0),              # smaller than the reach of T steps
+    ((129, 256), 16, 4),         # five strips; chunks shorter than their halo
+    ((300, 56), 0, 0),           # exactly one strip
+])
+def test_f64_fused_2d_passes_match_oracle(R, box, T, dims, chunk, stages):
+    mk = wl.random_box_weights if box else wl.random_star_weights
+    w = mk(2, R, 73, np.float64)
+    a = wl.normal_field(dims, 74, np.float64)
+    for steps in (T, T + 1, 2 * T + 1, 2):
+        dev = torch.device("cuda:0")
+        src = torch.from_numpy(a).to(dev)
+        dst = torch.full_like(src, float("nan"))
+        with b.Plan(dims, R, b.BOX if box else b.STAR, w, b.ZERO, chunk_z=chunk or None, stages=stages or None) as p:
+            assert p.f64 and p.variant == "stream" and p.get(b.KEY_FUSE_STEPS) == T
+            p.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
+            assert p.query_status() == b.OK
+            assert p.launches == -(-steps // T)
+        got = dst.cpu().numpy()
+        want = oracle.apply(a, w, b.ZERO, steps)
+        tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+        err = float(np.max(np.abs(got - want)))
+        assert err <= tol, f"R={R} box={box} T={T} dims={dims} steps={steps}: {err:.3e} > {tol:.3e}"
+
+
 # -------------------------------------------------------------------- fused --
 FUSED_CONFIGS = [   # (radius, fuse_steps, region width, region height)
     (1, 2, 256, 32), (1, 2, 256, 16), (1, 3, 256, 32), (1, 4, 128, 32), (1, 2, 128, 32), (1, 3, 128, 32),
