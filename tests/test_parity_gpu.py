@@ -794,6 +794,20 @@ def test_2d_grid_with_more_than_2_to_the_31_points():
         want = oracle.apply(sub, w, b.ZERO, 1)[R]
         got = dst[yc].cpu().numpy()
         assert float(np.max(np.abs(got - want))) <= tol, f"row {yc}"
+    # two time steps in one fused pass on the same grid; the band of rows around a sampled row ends
+    # either at the grid's own edge or 2R rows away from the row, so the row itself is exact
+    with b.Plan((ny, nx), R, b.BOX, w, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2
+        p.apply(src, dst, 2, torch.cuda.current_stream().cuda_stream)
+        assert p.query_status() == b.OK and p.launches == 1
+    torch.cuda.synchronize()
+    tol = wl.tolerance(w, 1.0, 2)
+    for yc in (0, 3, 23111, ny - 1):
+        lo, hi = max(yc - 2 * R, 0), min(yc + 2 * R + 1, ny)
+        band = (field(lo, hi, np) / 8.0).astype(np.float32)
+        want = oracle.apply(band, w, b.ZERO, 2)[yc - lo]
+        got = dst[yc].cpu().numpy()
+        assert float(np.max(np.abs(got - want))) <= tol, f"row {yc}, two fused steps"
     del src, dst
     torch.cuda.empty_cache()
 
