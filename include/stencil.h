@@ -67,9 +67,12 @@ enum {
 /* Keys of stencil_plan_set / stencil_plan_get. */
 enum {
     STENCIL_KEY_VARIANT      = 0,  /* set/get: STENCIL_VARIANT_*                                 */
-    STENCIL_KEY_TILE_X       = 1,  /* set/get: region width of fused passes, 128, 256 or 512 (0 = auto) */
+    STENCIL_KEY_TILE_X       = 1,  /* set/get: region width of fused 3D passes, 128, 256 or 512 (0 = auto) */
     STENCIL_KEY_TILE_Y       = 2,  /* set/get: tile height in rows   (0 = default)               */
-    STENCIL_KEY_FUSE_STEPS   = 3,  /* set: time steps fused per pass (0 = auto, 1 = off);
+    STENCIL_KEY_FUSE_STEPS   = 3,  /* set: time steps fused per pass (0 = auto, 1 = off; 3D fp32
+                                      stars: 2-4; 2D grids: the one depth the operator's fused
+                                      kernel has: star and box R=1: 4, star R=2: 3, box R=2: 2,
+                                      fp32 stars R=3 and 4: 2);
                                       get: the number iterated applies will use (1 = none)       */
     STENCIL_KEY_LAUNCHES     = 4,  /* get: kernels launched by this plan so far                  */
     STENCIL_KEY_SCRATCH_BYTES= 5,  /* get: device bytes the plan currently owns as scratch       */
@@ -83,7 +86,7 @@ enum {
                                       programmatic dependent launches: each begins its preamble
                                       while its predecessor drains and waits for it before it
                                       touches global memory; 0 = ordinary launches             */
-    STENCIL_KEY_FUSED_TILE_Y = 13,   /* set/get: region height of fused passes, 16 or 32 (0 = auto) */
+    STENCIL_KEY_FUSED_TILE_Y = 13,   /* set/get: region height of fused 3D passes, 16 or 32 (0 = auto) */
     STENCIL_KEY_PERIODIC_ROUTE = 14, /* set/get: how the tiled kernels handle a periodic boundary.
                                       1 = sweep from a padded copy with wrapped halos; 2 = zero-
                                       boundary sweep plus a correction of the points within R of
