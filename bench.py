@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum +
 # dram__bytes_write.sum from an ncu capture; see profiles/).  None = not captured.
 NCU_TRAFFIC_BYTES = {
-    "cfg2": 1003.8e6,   # stream kernel, star R=1: 2 x (279.4 MB read + 222.5 MB written) on the half grid
+    "cfg2": 978.1e6,    # stream kernel, star R=1: 2 x (268.5 MB read + 220.5 MB written) on the half grid
     "cfg3": 1004.6e6,   # stream kernel, box R=1
     "cfg4": 995.7e6,    # stream kernel, star R=4
     "cfg5": 99.9e6,     # one fused pass (2 time steps of 256^3): 77.7 MB read + 22.2 MB written
