@@ -32,6 +32,15 @@ constexpr int kStreamPX = kStreamTX + 8;  // smem row pitch: 4-float halo each s
                                           // TMA x-coordinates and LDS.128 16-byte aligned
 constexpr int kMaxStages = 8;
 
+// Halo columns on either side of a tile row in shared memory: 4 floats reach radius 4; the
+// wider stars (radius 5..8) take 8.  Multiples of 4 keep TMA x-coordinates and LDS.128 aligned.
+template <int R>
+struct StreamHalo {
+    static_assert(R >= 1 && R <= 8, "radius 1..8");
+    static constexpr int HX = R <= 4 ? 4 : 8;
+    static constexpr int PX = kStreamTX + 2 * HX;      // smem row pitch
+};
+
 template <int R>
 struct StarWeights {            // taps of a star stencil, index d + R along each axis
     float c;
@@ -60,7 +69,7 @@ template <int R, int K, int NW>
 struct StreamShape {
     static constexpr int TY = NW * K;
     static constexpr int ROWS = TY + 2 * R;
-    static constexpr int PLANE_FLOATS = ROWS * kStreamPX;
+    static constexpr int PLANE_FLOATS = ROWS * StreamHalo<R>::PX;
     static constexpr int BOX_BYTES = PLANE_FLOATS * 4;
     static constexpr int PLANE_BYTES = (BOX_BYTES + 127) / 128 * 128;
     static constexpr int THREADS = (NW + 1) * 32;
@@ -103,7 +112,8 @@ __device__ __forceinline__ float lds_if(bool take, const float* p, float keep) {
 
 // Fills v[0 .. 4+2R) with the R values left of the lane's float4, the float4
 // itself, and the R values right of it, for one smem row.  `rowp` points at the
-// lane's float4 inside the row; `rowbase` at the row's first float (x = -4).
+// lane's float4 inside the row; `rowbase` at the row's first float (x = -4; the
+// R <= 2 path, the only one that uses it, always has a 4-float halo).
 template <int R>
 __device__ __forceinline__ void gather_row(const float* rowp, const float* rowbase, int lane,
                                            const float4& ctr, float (&v)[4 + 2 * R]) {
@@ -122,7 +132,7 @@ __device__ __forceinline__ void gather_row(const float* rowp, const float* rowba
             v[t] = lane == 0 ? hl : l;
             v[R + 4 + t] = lane == 31 ? hr : r;
         }
-    } else {
+    } else if constexpr (R <= 4) {
         const float4 l = *reinterpret_cast<const float4*>(rowp - 4);
         const float4 r = *reinterpret_cast<const float4*>(rowp + 4);
         const float l4[4] = {l.x, l.y, l.z, l.w};
@@ -131,6 +141,19 @@ __device__ __forceinline__ void gather_row(const float* rowp, const float* rowba
         for (int t = 0; t < R; ++t) {
             v[t] = l4[4 - R + t];
             v[R + 4 + t] = r4[t];
+        }
+    } else {
+        // radius 5..8: two float4 on either side (the row has an 8-float halo)
+        const float4 la = *reinterpret_cast<const float4*>(rowp - 8);
+        const float4 lb = *reinterpret_cast<const float4*>(rowp - 4);
+        const float4 ra = *reinterpret_cast<const float4*>(rowp + 4);
+        const float4 rb = *reinterpret_cast<const float4*>(rowp + 8);
+        const float l8[8] = {la.x, la.y, la.z, la.w, lb.x, lb.y, lb.z, lb.w};
+        const float r8[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+#pragma unroll
+        for (int t = 0; t < R; ++t) {
+            v[t] = l8[8 - R + t];
+            v[R + 4 + t] = r8[t];
         }
     }
 }
@@ -143,7 +166,8 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                       const __grid_constant__ BoxWeights<BOX ? R : 0> bw,
                       int* __restrict__ status) {
     using S = StreamShape<R, K, NW>;
-    constexpr int PX = kStreamPX;
+    constexpr int PX = StreamHalo<R>::PX;
+    constexpr int HX = StreamHalo<R>::HX;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     // ring of planes first (128-byte aligned slots), then the barriers.  The pointer is
     // formed by indexing the shared array (no integer round trip), so the compiler
@@ -194,7 +218,7 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                 if (i != g.drop_plane) {
                     mbar_arrive_expect_tx(full0 + 8 * s, S::BOX_BYTES);
                     tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_BYTES), &tmap_in, full0 + 8 * s,
-                                x0 - 4 + g.in_off_x, y0 - R + g.in_off_y, pstart + i + g.in_off_z);
+                                x0 - HX + g.in_off_x, y0 - R + g.in_off_y, pstart + i + g.in_off_z);
                 }
                 issued = i + 1;
                 if (++s == nstage) { s = 0; ph ^= 1; }
@@ -248,7 +272,7 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                 return;
             }
             const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
-            const float* colp = pl + row0 * PX + 4 + 4 * lane;
+            const float* colp = pl + row0 * PX + HX + 4 * lane;
             // Rows are visited once, top to bottom.  A row is a y-neighbour of up to 2R output
             // rows and the centre row of at most one; it is consumed at once, so only one
             // loaded row is live at a time.  acc[k] is the output whose centre plane this is:
@@ -343,7 +367,7 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                 if (i >= nplanes) return true;
                 if (!mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) return false;
                 const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
-                const float* colp = pl + row0 * PX + 4 + 4 * lane;
+                const float* colp = pl + row0 * PX + HX + 4 * lane;
                 float v[K + 2 * R][4 + 2 * R];
 #pragma unroll
                 for (int kk = 0; kk < K + 2 * R; ++kk) {

@@ -96,6 +96,7 @@ struct StreamConfig {
     int K, NW;            // rows per thread, consumer warps
     int tile_y;           // K * NW
     int plane_bytes, box_rows, threads;
+    int px;               // columns of the TMA box: the tile plus its halo on both sides
     mutable int occupancy[kMaxStages + 1];   // resident CTAs per SM by ring depth; 0 = not asked yet
     mutable size_t smem_allowed;             // dynamic shared memory the kernel is currently allowed
     mutable int cache_device;                // device the two caches above were filled on
@@ -289,6 +290,7 @@ StreamConfig make_cfg() {
     StreamConfig c;
     c.radius = R; c.box = BOX; c.K = K; c.NW = NW; c.tile_y = S::TY;
     c.plane_bytes = S::PLANE_BYTES; c.box_rows = S::ROWS; c.threads = S::THREADS;
+    c.px = StreamHalo<R>::PX;
     for (int& o : c.occupancy) o = 0;
     c.smem_allowed = 0;
     c.cache_device = -1;
@@ -311,6 +313,12 @@ const std::vector<StreamConfig>& stream_configs() {
         make_cfg<3, false, 4, 8, 1>(),  make_cfg<3, false, 2, 8, 2>(),  make_cfg<3, false, 2, 7, 2>(),
         make_cfg<4, false, 2, 8, 2>(),  make_cfg<4, false, 2, 7, 2>(),  make_cfg<4, false, 4, 8, 1>(),
         make_cfg<4, false, 2, 16, 1>(),
+        // radius 5..8 (8-float halo columns): one row per thread, the 2R accumulators per row leave no
+        // registers for more; 16-row tiles halve the share of the 2R halo rows
+        make_cfg<5, false, 1, 16, 1>(), make_cfg<5, false, 1, 8, 2>(),
+        make_cfg<6, false, 1, 16, 1>(), make_cfg<6, false, 1, 8, 2>(),
+        make_cfg<7, false, 1, 16, 1>(), make_cfg<7, false, 1, 8, 2>(),
+        make_cfg<8, false, 1, 16, 1>(), make_cfg<8, false, 1, 8, 2>(),
         make_cfg<1, true, 2, 8, 1>(),   make_cfg<1, true, 2, 7, 4>(),   make_cfg<1, true, 4, 8, 1>(),
         make_cfg<1, true, 4, 7, 1>(),   make_cfg<1, true, 1, 8, 1>(),
         // 125 taps: one row per thread (56 registers, twice the warps of two rows per thread)
@@ -467,8 +475,12 @@ const Rows2DFusedConfig* pick_fused2d(const stencil_plan_s* p) {
 // copied into a padded grid with wrapped halos (kernel_pad.cuh) and swept from there.  A
 // zero-boundary grid with other row lengths is swept between two grids with padded rows
 // (apply_row_padded).
+bool wrap_correction_fits(const stencil_plan_s* p);
+
 bool stream_supported(const stencil_plan_s* p) {
     if (p->nx % 4 != 0 && p->boundary != STENCIL_ZERO) return false;
+    // radius > 4: the padded periodic copy has only 4 halo columns, so the wrap correction must fit
+    if (p->radius > 4 && p->boundary == STENCIL_PERIODIC && !wrap_correction_fits(p)) return false;
     const bool box = p->shape == STENCIL_BOX;
     if (p->ndim == 2) return find_rows2d_cfg(p->radius, box) != nullptr;
     return find_stream_cfg(p->radius, box, 0, 0) != nullptr;
@@ -820,9 +832,9 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
         int pnx, pny, pnz;
         const float* padded = nullptr;
         if ((rc = pad_periodic(p, src, st, &padded, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
-        rc = get_tensor_map(p, cfg, kStreamPX, cfg->box_rows, padded, &map, pnx, pny, pnz);
+        rc = get_tensor_map(p, cfg, cfg->px, cfg->box_rows, padded, &map, pnx, pny, pnz);
     } else {
-        rc = get_tensor_map(p, cfg, kStreamPX, cfg->box_rows, src, &map);
+        rc = get_tensor_map(p, cfg, cfg->px, cfg->box_rows, src, &map);
     }
     if (rc != STENCIL_OK) return rc;
 
@@ -1624,6 +1636,7 @@ bool wrap_correction_fits(const stencil_plan_s* p) {
 // measured on 512^3, the correction wins except for the 125-tap box and, when the copy is
 // spread over several steps, for the wide 3D stars.
 bool use_wrap_correction(const stencil_plan_s* p, int steps) {
+    if (p->radius > 4) return true;                 // the only periodic route of the wide stars (see stream_supported)
     if (p->periodic_route == 1 || !wrap_correction_fits(p)) return false;
     if (p->periodic_route == 2) return true;
     if (p->ndim == 3 && p->shape == STENCIL_BOX && p->radius >= 2) return false;

@@ -110,7 +110,13 @@ def test_variant_selection_rules():
     with b.Plan((64, 64, 66), 1, b.STAR, star, b.ZERO) as p:       # nx % 4 != 0: swept between grids with padded rows
         assert p.variant == "stream"
         assert p.get(b.KEY_FUSE_STEPS) == 1         # no temporal blocking over padded rows
-    with b.Plan((64, 64, 66), 5, b.STAR, wl.star_weights(3, 5, -6.0, [1.0] * 5), b.ZERO) as p:
+    with b.Plan((64, 64, 64), 6, b.STAR, wl.star_weights(3, 6, -6.0, [1.0] * 6), b.ZERO) as p:
+        assert p.variant == "stream"                # the wide stars run on the tiled 3D kernel (8-column halos)
+    with b.Plan((64, 64), 6, b.STAR, wl.star_weights(2, 6, -6.0, [1.0] * 6), b.ZERO) as p:
+        assert p.variant == "generic"               # ... but not in 2D
+    with b.Plan((8, 64, 64), 6, b.STAR, wl.star_weights(3, 6, -6.0, [1.0] * 6), b.PERIODIC) as p:
+        assert p.variant == "generic"               # periodic wide star on a grid thinner than 2R
+    with b.Plan((64, 64, 66), 3, b.BOX, wl.random_box_weights(3, 3, 4), b.ZERO) as p:
         assert p.variant == "generic"               # radius beyond the tiled kernels
         with pytest.raises(b.StencilError) as e:
             p.set(b.KEY_VARIANT, b.VARIANT_STREAM)

@@ -209,6 +209,28 @@ def test_non_default_stream():
     assert np.max(np.abs(dst.cpu().numpy() - want)) <= wl.tolerance(w, float(np.abs(a).max()), 3)
 
 
+@pytest.mark.parametrize("R", [5, 6, 7, 8])
+@pytest.mark.parametrize("dims,chunk_z,stages", [
+    ((37, 45, 132), 10, 3),      # ragged in x, y and z; several chunks; 2 x-tiles
+    ((8, 16, 128), 0, 0),        # exactly one tile
+    ((3, 5, 4), 0, 2),           # much smaller than the stencil reach
+    ((40, 33, 260), 0, 0),       # three x-tiles, the last 4 points wide
+])
+def test_wide_star_stream_kernel_matches_oracle(R, dims, chunk_z, stages):
+    """Stars of radius 5..8 on the tiled 3D kernel (8-column halos, one row per thread)."""
+    w = wl.random_star_weights(3, R, 23)
+    a = wl.normal_field(dims, 24)
+    for knobs in (dict(), dict(tile_y=8)):
+        used = check(dims, R, b.STAR, w, b.ZERO, a, variant=b.VARIANT_STREAM, chunk_z=chunk_z or None,
+                     stages=stages or None, **knobs)
+        assert used == "stream"
+    used = check(dims, R, b.STAR, w, b.ZERO, a, steps=3)
+    assert used == "stream"
+    if min(dims) >= 2 * R:
+        used = check(dims, R, b.STAR, w, b.PERIODIC, a, steps=2)         # wrap correction is the only route here
+        assert used == "stream"
+
+
 # ------------------------------------------------- periodic boundary, tiled path --
 # periodic_route: None = chosen by the library, 2 = wrap correction after a zero-boundary sweep (extents >= 2R),
 # 1 = sweep from a padded copy with wrapped halos
