@@ -106,7 +106,10 @@ enum {
  *   plan_out  HOST, receives the handle; set to NULL on any error.
  *   ndim      2 or 3.
  *   dims      HOST, ndim entries, slowest axis first, each >= 1.
- *   radius    R >= 1; R <= 8 (larger: STENCIL_ERR_UNSUPPORTED).
+ *   radius    R >= 1; R <= 8 (larger: STENCIL_ERR_UNSUPPORTED).  The TMA-staged kernels
+ *             cover, in fp32, 3D stars up to radius 8 and 3D boxes up to radius 2,
+ *             2D stars and boxes up to radius 4; other requests run on the
+ *             one-thread-per-point kernel.
  *   shape     STENCIL_STAR or STENCIL_BOX.
  *   weights   HOST, dense (2R+1)^ndim floats in C order, same axis order as
  *             dims: entry [dz+R][dy+R][dx+R] multiplies in[p+(dz,dy,dx)]
