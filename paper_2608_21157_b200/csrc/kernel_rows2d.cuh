@@ -32,9 +32,9 @@ struct Rows2DGeom {
     int in_off_x, in_off_y;     // added to the TMA coordinates (padded input of a periodic grid), else 0
 };
 
-template <int YB>
+template <int YB, int PXV = kStreamPX>     // PXV: row pitch of a batch (the strip plus its halo columns)
 struct Rows2DShape {
-    static constexpr int BATCH_FLOATS = YB * kStreamPX;
+    static constexpr int BATCH_FLOATS = YB * PXV;
     static constexpr int BATCH_BYTES = BATCH_FLOATS * 4;          // multiple of 128 for even YB
     static size_t smem_bytes(int nwarps, int stages) {
         return (size_t)nwarps * stages * BATCH_BYTES + 128 + (size_t)nwarps * kMaxStages * 8;
@@ -46,8 +46,9 @@ __global__ void __launch_bounds__(NW * 32)
 stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restrict__ out,
                       const Rows2DGeom g, const __grid_constant__ Weights2D<R> wt,
                       int* __restrict__ status) {
-    using S = Rows2DShape<YB>;
-    constexpr int PX = kStreamPX;
+    constexpr int PX = StreamHalo<R>::PX;          // 4 halo columns per side up to radius 4, 8 beyond
+    constexpr int HX = StreamHalo<R>::HX;
+    using S = Rows2DShape<YB, PX>;
     constexpr int M = 2 * R + 1;
     constexpr int kRowCopies = (BOX && R >= 3) ? 1 : YB;
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -85,7 +86,7 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
         for (int b = 0; b < pre; ++b) {
             mbar_arrive_expect_tx(full0 + 8 * b, S::BATCH_BYTES);
             tma_load_3d(smem_addr(ring + (size_t)b * S::BATCH_FLOATS), &tmap_in, full0 + 8 * b,
-                        x0 - 4 + g.in_off_x, ystart + b * YB + g.in_off_y, 0);
+                        x0 - HX + g.in_off_x, ystart + b * YB + g.in_off_y, 0);
         }
     }
 
@@ -116,7 +117,7 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
             const int i = b * YB + r;                    // input row index inside the chunk
             if (i < nrows) {
                 const float* rowbase = bp + r * PX;
-                const float* rowp = rowbase + 4 + 4 * lane;
+                const float* rowp = rowbase + HX + 4 * lane;
                 const float4 c = *reinterpret_cast<const float4*>(rowp);
                 float v[4 + 2 * R];
                 gather_row<R>(rowp, rowbase, lane, c, v);
@@ -184,7 +185,7 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
         if (lane == 0 && b + nstage < nbatches) {
             mbar_arrive_expect_tx(full0 + 8 * s, S::BATCH_BYTES);
             tma_load_3d(smem_addr(ring + (size_t)s * S::BATCH_FLOATS), &tmap_in, full0 + 8 * s,
-                        x0 - 4 + g.in_off_x, ystart + (b + nstage) * YB + g.in_off_y, 0);
+                        x0 - HX + g.in_off_x, ystart + (b + nstage) * YB + g.in_off_y, 0);
             issued = b + nstage + 1;
         }
         if (++s == nstage) { s = 0; ph ^= 1; }

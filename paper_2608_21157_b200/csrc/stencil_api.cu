@@ -130,6 +130,7 @@ struct Rows2DConfig {
     int radius;
     bool box;
     int YB, NW, batch_bytes;
+    int px;                     // columns of the TMA box: the strip plus its halo on both sides
     const void* kernel;
     mutable size_t smem_allowed;
     mutable int cache_device;
@@ -404,7 +405,9 @@ cudaError_t launch_rows2d_t(const stencil_plan_s* p, const CUtensorMap& map, flo
 template <int R, bool BOX, int YB, int NW>
 Rows2DConfig make_rows2d() {
     Rows2DConfig c;
-    c.radius = R; c.box = BOX; c.YB = YB; c.NW = NW; c.batch_bytes = Rows2DShape<YB>::BATCH_BYTES;
+    c.radius = R; c.box = BOX; c.YB = YB; c.NW = NW;
+    c.px = StreamHalo<R>::PX;
+    c.batch_bytes = Rows2DShape<YB, StreamHalo<R>::PX>::BATCH_BYTES;
     c.kernel = reinterpret_cast<const void*>(&stencil_rows2d_kernel<R, BOX, YB, NW>);
     c.smem_allowed = 0; c.cache_device = -1;
     c.launch = &launch_rows2d_t<R, BOX, YB, NW>;
@@ -420,6 +423,9 @@ const std::vector<Rows2DConfig>& rows2d_configs() {
         // 81 taps: batches of 4 rows and 16 warps per CTA (twice the warps per SM) measured 329
         // against 286 GPoints/s on 10240^2; the smaller boxes gain nothing from it
         make_rows2d<4, true, 4, 16>(),
+        // stars of radius 5..8: batches with 8 halo columns per side
+        make_rows2d<5, false, 8, 8>(), make_rows2d<6, false, 8, 8>(), make_rows2d<7, false, 8, 8>(),
+        make_rows2d<8, false, 8, 8>(),
     };
     return v;
 }
@@ -887,9 +893,9 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
         int pnx, pny, pnz;
         const float* padded = nullptr;
         if ((rc = pad_periodic(p, src, st, &padded, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
-        rc = get_tensor_map(p, cfg, kStreamPX, cfg->YB, padded, &map, pnx, pny, pnz);
+        rc = get_tensor_map(p, cfg, cfg->px, cfg->YB, padded, &map, pnx, pny, pnz);
     } else {
-        rc = get_tensor_map(p, cfg, kStreamPX, cfg->YB, src, &map);
+        rc = get_tensor_map(p, cfg, cfg->px, cfg->YB, src, &map);
     }
     if (rc != STENCIL_OK) return rc;
     const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;

@@ -113,7 +113,9 @@ def test_variant_selection_rules():
     with b.Plan((64, 64, 64), 6, b.STAR, wl.star_weights(3, 6, -6.0, [1.0] * 6), b.ZERO) as p:
         assert p.variant == "stream"                # the wide stars run on the tiled 3D kernel (8-column halos)
     with b.Plan((64, 64), 6, b.STAR, wl.star_weights(2, 6, -6.0, [1.0] * 6), b.ZERO) as p:
-        assert p.variant == "generic"               # ... but not in 2D
+        assert p.variant == "stream" and p.get(b.KEY_FUSE_STEPS) == 1     # also in 2D; no fused kernel for them
+    with b.Plan((64, 64), 5, b.BOX, wl.random_box_weights(2, 5, 4), b.ZERO) as p:
+        assert p.variant == "generic"               # boxes beyond radius 4 are not tiled
     with b.Plan((8, 64, 64), 6, b.STAR, wl.star_weights(3, 6, -6.0, [1.0] * 6), b.PERIODIC) as p:
         assert p.variant == "generic"               # periodic wide star on a grid thinner than 2R
     with b.Plan((64, 64, 66), 3, b.BOX, wl.random_box_weights(3, 3, 4), b.ZERO) as p:

@@ -231,6 +231,21 @@ def test_wide_star_stream_kernel_matches_oracle(R, dims, chunk_z, stages):
         assert used == "stream"
 
 
+@pytest.mark.parametrize("R", [5, 6, 7, 8])
+@pytest.mark.parametrize("dims,chunk,stages", [((67, 132), 0, 0), ((200, 260), 37, 2), ((3, 8), 0, 0), ((129, 512), 16, 4)])
+def test_wide_star_rows2d_kernel_matches_oracle(R, dims, chunk, stages):
+    """Stars of radius 5..8 on the 2D row-streaming kernel (8-column halos)."""
+    w = wl.random_star_weights(2, R, 25)
+    a = wl.normal_field(dims, 26)
+    used = check(dims, R, b.STAR, w, b.ZERO, a, chunk_z=chunk or None, stages=stages or None)
+    assert used == "stream"
+    used = check(dims, R, b.STAR, w, b.ZERO, a, steps=3)
+    assert used == "stream"
+    if min(dims) >= 2 * R:
+        used = check(dims, R, b.STAR, w, b.PERIODIC, a, steps=2)
+        assert used == "stream"
+
+
 # ------------------------------------------------- periodic boundary, tiled path --
 # periodic_route: None = chosen by the library, 2 = wrap correction after a zero-boundary sweep (extents >= 2R),
 # 1 = sweep from a padded copy with wrapped halos
