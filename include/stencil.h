@@ -107,8 +107,8 @@ enum {
  *   ndim      2 or 3.
  *   dims      HOST, ndim entries, slowest axis first, each >= 1.
  *   radius    R >= 1; R <= 8 (larger: STENCIL_ERR_UNSUPPORTED).  The TMA-staged kernels
- *             cover, in fp32, 3D stars up to radius 8 and 3D boxes up to radius 2,
- *             2D stars and boxes up to radius 4; other requests run on the
+ *             cover, in fp32 and FP64, stars up to radius 8, 3D boxes up to radius 2
+ *             and 2D boxes up to radius 4; other requests run on the
  *             one-thread-per-point kernel.
  *   shape     STENCIL_STAR or STENCIL_BOX.
  *   weights   HOST, dense (2R+1)^ndim floats in C order, same axis order as

@@ -5,7 +5,7 @@
 // slide down one slot inside the FMA that updates them.
 //
 // Differences: a lane owns one double2 (two points), so a strip is 64 columns wide; the
-// x neighbourhood of a lane (R <= 4 values on each side) is read straight from shared
+// x neighbourhood of a lane (R values on each side) is read straight from shared
 // memory as aligned double2 loads.  The sweep is bound by the FP64 pipe (49 DFMA per
 // point at 64 DFMA per clock per SM) about as much as by HBM (16 B per point).
 #pragma once
@@ -23,10 +23,10 @@ struct Weights2D64 {                         // dense, [dy+R][dx+R]
     double w[2 * R + 1][2 * R + 1];
 };
 
-template <int YB>
+template <int YB, int PXV = kPX64>
 struct Rows2D64Shape {
-    static constexpr int BATCH_DOUBLES = YB * kPX64;
-    static constexpr int BATCH_BYTES = BATCH_DOUBLES * 8;        // 576 * YB: a multiple of 128 for even YB
+    static constexpr int BATCH_DOUBLES = YB * PXV;
+    static constexpr int BATCH_BYTES = BATCH_DOUBLES * 8;        // 576 * YB (640 * YB for the wide stars): a multiple of 128 for even YB
 };
 
 template <int R, bool BOX, int YB, int NW>
@@ -34,7 +34,9 @@ __global__ void __launch_bounds__(NW * 32)
 stencil_rows2d_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* __restrict__ out,
                           const Rows2DGeom g, const __grid_constant__ Weights2D64<R> wt,
                           int* __restrict__ status) {
-    using S = Rows2D64Shape<YB>;
+    constexpr int PX = StreamHalo64<R>::PX;
+    constexpr int HX = StreamHalo64<R>::HX;
+    using S = Rows2D64Shape<YB, PX>;
     constexpr int M = 2 * R + 1;
     constexpr int HW = (R + 1) / 2 * 2;          // halo doubles read per side, rounded up to a double2
     constexpr int NV = 2 * HW + 2;               // window of a lane: columns -HW .. 1+HW around its pair
@@ -73,7 +75,7 @@ stencil_rows2d_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
         for (int b = 0; b < pre; ++b) {
             mbar_arrive_expect_tx(full0 + 8 * b, S::BATCH_BYTES);
             tma_load_3d(smem_addr(ring + (size_t)b * S::BATCH_DOUBLES), &tmap_in, full0 + 8 * b,
-                        x0 - 4 + g.in_off_x, ystart + b * YB + g.in_off_y, 0);
+                        x0 - HX + g.in_off_x, ystart + b * YB + g.in_off_y, 0);
         }
     }
 
@@ -101,7 +103,7 @@ stencil_rows2d_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
             const int i = b * YB + r;
             if (i < nrows) {
                 // v[HW + m + dx] is the input at column (pair column m) + dx
-                const double* wp = bp + r * kPX64 + 4 + 2 * lane - HW;
+                const double* wp = bp + r * PX + HX + 2 * lane - HW;
                 double v[NV];
 #pragma unroll
                 for (int t = 0; t < NV / 2; ++t) {
@@ -166,7 +168,7 @@ stencil_rows2d_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
         if (lane == 0 && b + nstage < nbatches) {
             mbar_arrive_expect_tx(full0 + 8 * s, S::BATCH_BYTES);
             tma_load_3d(smem_addr(ring + (size_t)s * S::BATCH_DOUBLES), &tmap_in, full0 + 8 * s,
-                        x0 - 4 + g.in_off_x, ystart + (b + nstage) * YB + g.in_off_y, 0);
+                        x0 - HX + g.in_off_x, ystart + (b + nstage) * YB + g.in_off_y, 0);
             issued = b + nstage + 1;
         }
         if (++s == nstage) { s = 0; ph ^= 1; }

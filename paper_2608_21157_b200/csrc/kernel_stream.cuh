@@ -41,6 +41,14 @@ struct StreamHalo {
     static constexpr int PX = kStreamTX + 2 * HX;      // smem row pitch
 };
 
+// The same for the FP64 kernels, whose tile rows are 64 doubles wide.
+template <int R>
+struct StreamHalo64 {
+    static_assert(R >= 1 && R <= 8, "radius 1..8");
+    static constexpr int HX = R <= 4 ? 4 : 8;
+    static constexpr int PX = 64 + 2 * HX;
+};
+
 template <int R>
 struct StarWeights {            // taps of a star stencil, index d + R along each axis
     float c;

@@ -5,7 +5,7 @@
 // Differences: a lane owns one double2 (two points), so a tile is 64 columns wide; the x
 // neighbourhood of a lane is read from shared memory as aligned double2 loads instead of
 // being exchanged by shuffles.  At 16 B per point the sweep is bound by HBM for the stars
-// (radius <= 4: 25 DFMA per point at most) and the 27-point box, since the FP64 pipe
+// (25 DFMA per point at radius 4) and the 27-point box, since the FP64 pipe
 // sustains 64 DFMA per clock per SM; the 125-point box is bound by that pipe.
 #pragma once
 #include "common.cuh"
@@ -15,7 +15,7 @@
 namespace stencil {
 
 constexpr int kStream64TX = 64;                  // tile width in points
-constexpr int kStream64PX = kStream64TX + 8;     // + 4 doubles of halo on both sides
+constexpr int kStream64PX = kStream64TX + 8;     // + 4 doubles of halo on both sides (radius <= 4; see StreamHalo64)
 
 template <int R>
 struct StarWeights64 {
@@ -32,7 +32,8 @@ template <int R, int K, int NW>
 struct Stream64Shape {
     static constexpr int TY = NW * K;
     static constexpr int ROWS = TY + 2 * R;             // even, so a plane is a multiple of 128 bytes
-    static constexpr int PLANE_DOUBLES = ROWS * kStream64PX;
+    static constexpr int PLANE_DOUBLES = ROWS * StreamHalo64<R>::PX;   // 576 or 640 bytes per row
+
     static constexpr int PLANE_BYTES = PLANE_DOUBLES * 8;
     static constexpr int THREADS = (NW + 1) * 32;
 };
@@ -47,7 +48,8 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
                           const __grid_constant__ BoxWeights64<BOX ? R : 0> bw,
                           int* __restrict__ status) {
     using S = Stream64Shape<R, K, NW>;
-    constexpr int PX = kStream64PX;
+    constexpr int PX = StreamHalo64<R>::PX;
+    constexpr int HX = StreamHalo64<R>::HX;
     constexpr int HW = (R + 1) / 2 * 2;              // halo doubles read per side (a whole double2)
     constexpr int NV = 2 * HW + 2;                   // x window of a lane
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -94,7 +96,7 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
                 if (i >= nstage && !mbar_wait_bounded(empty0 + 8 * s, ph, g.wait_polls)) { ok = false; break; }
                 mbar_arrive_expect_tx(full0 + 8 * s, S::PLANE_BYTES);
                 tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_DOUBLES), &tmap_in, full0 + 8 * s,
-                            x0 - 4 + g.in_off_x, y0 - R + g.in_off_y, pstart + i + g.in_off_z);
+                            x0 - HX + g.in_off_x, y0 - R + g.in_off_y, pstart + i + g.in_off_z);
                 issued = i + 1;
                 if (++s == nstage) { s = 0; ph ^= 1; }
             }
@@ -131,7 +133,7 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
                 return;
             }
             const double* pl = ring + (size_t)s * S::PLANE_DOUBLES;
-            const double* colp = pl + row0 * PX + 4 + 2 * lane;
+            const double* colp = pl + row0 * PX + HX + 2 * lane;
             double acc[K][2];
 #pragma unroll
             for (int k = 0; k < K; ++k) { acc[k][0] = A[k][R].x; acc[k][1] = A[k][R].y; }
@@ -206,7 +208,7 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
                 if (i >= nplanes) return true;
                 if (!mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) return false;
                 const double* pl = ring + (size_t)s * S::PLANE_DOUBLES;
-                const double* colp = pl + row0 * PX + 4 + 2 * lane;
+                const double* colp = pl + row0 * PX + HX + 2 * lane;
                 double v[K + 2 * R][NV];
 #pragma unroll
                 for (int kk = 0; kk < K + 2 * R; ++kk)

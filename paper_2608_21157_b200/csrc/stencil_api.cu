@@ -172,7 +172,7 @@ struct Rows2DFused64Config {
 struct Rows2D64Config {
     int radius;
     bool box;
-    int YB, NW, batch_bytes;
+    int YB, NW, batch_bytes, px;
     const void* kernel;
     mutable size_t smem_allowed;
     mutable int cache_device;
@@ -183,7 +183,7 @@ struct Rows2D64Config {
 struct Stream64Config {
     int radius;
     bool box;
-    int tile_y, plane_bytes, box_rows, threads;
+    int tile_y, plane_bytes, box_rows, threads, px;
     const void* kernel;
     mutable size_t smem_allowed;
     mutable size_t occ_smem;                 // shared-memory size the occupancy below was asked for
@@ -1195,7 +1195,8 @@ cudaError_t launch_rows2d64_t(const stencil_plan_s* p, const CUtensorMap& map, d
 template <int R, bool BOX, int YB, int NW>
 Rows2D64Config make_rows2d64() {
     Rows2D64Config c;
-    c.radius = R; c.box = BOX; c.YB = YB; c.NW = NW; c.batch_bytes = Rows2D64Shape<YB>::BATCH_BYTES;
+    c.radius = R; c.box = BOX; c.YB = YB; c.NW = NW; c.px = StreamHalo64<R>::PX;
+    c.batch_bytes = Rows2D64Shape<YB, StreamHalo64<R>::PX>::BATCH_BYTES;
     c.kernel = reinterpret_cast<const void*>(&stencil_rows2d_f64_kernel<R, BOX, YB, NW>);
     c.smem_allowed = 0; c.cache_device = -1;
     c.launch = &launch_rows2d64_t<R, BOX, YB, NW>;
@@ -1205,7 +1206,8 @@ Rows2D64Config make_rows2d64() {
 const std::vector<Rows2D64Config>& rows2d64_configs() {
     static const std::vector<Rows2D64Config> v = {
         make_rows2d64<1, false, 8, 8>(), make_rows2d64<2, false, 8, 8>(), make_rows2d64<3, false, 8, 8>(),
-        make_rows2d64<4, false, 8, 8>(),
+        make_rows2d64<4, false, 8, 8>(), make_rows2d64<5, false, 8, 8>(), make_rows2d64<6, false, 8, 8>(),
+        make_rows2d64<7, false, 8, 8>(), make_rows2d64<8, false, 8, 8>(),
         // the FP64 boxes from 25 taps on are bound by the FP64 pipe and run better with twice the warps
         // per SM (batches of 4 rows, 16 warps per CTA): 10240^2, 49 taps 291 against 265 GPoints/s, 25
         // taps 337 against 318
@@ -1217,6 +1219,7 @@ const std::vector<Rows2D64Config>& rows2d64_configs() {
 
 const Rows2D64Config* find_rows2d64_cfg(const stencil_plan_s* p) {
     if (p->ndim != 2 || (p->boundary != STENCIL_ZERO && p->nx % 2 != 0)) return nullptr;   // odd rows: apply_row_padded_f64
+    if (p->radius > 4 && p->boundary == STENCIL_PERIODIC && !wrap_correction_fits(p)) return nullptr;
     for (const Rows2D64Config& c : rows2d64_configs())
         if (c.radius == p->radius && c.box == (p->shape == STENCIL_BOX)) return &c;
     return nullptr;
@@ -1257,7 +1260,7 @@ Stream64Config make_stream64() {
     using S = Stream64Shape<R, K, NW>;
     Stream64Config c;
     c.radius = R; c.box = BOX; c.tile_y = S::TY; c.plane_bytes = S::PLANE_BYTES; c.box_rows = S::ROWS;
-    c.threads = S::THREADS;
+    c.threads = S::THREADS; c.px = StreamHalo64<R>::PX;
     c.kernel = reinterpret_cast<const void*>(&stencil_stream_f64_kernel<R, BOX, K, NW, MINB>);
     c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
     c.launch = &launch_stream64_t<R, BOX, K, NW, MINB>;
@@ -1273,12 +1276,15 @@ const std::vector<Stream64Config>& stream64_configs() {
         // capped 313, 2 x 7 capped 323.
         make_stream64<1, false, 2, 8, 1>(), make_stream64<2, false, 2, 8, 1>(), make_stream64<3, false, 4, 4, 2>(),
         make_stream64<4, false, 2, 7, 2>(), make_stream64<1, true, 2, 8, 1>(), make_stream64<2, true, 1, 8, 1>(),
+        make_stream64<5, false, 1, 8, 2>(), make_stream64<6, false, 1, 8, 2>(), make_stream64<7, false, 1, 8, 2>(),
+        make_stream64<8, false, 1, 8, 2>(),
     };
     return v;
 }
 
 const Stream64Config* find_stream64_cfg(const stencil_plan_s* p) {
     if (p->ndim != 3 || (p->boundary != STENCIL_ZERO && p->nx % 2 != 0)) return nullptr;   // odd rows: apply_row_padded_f64
+    if (p->radius > 4 && p->boundary == STENCIL_PERIODIC && !wrap_correction_fits(p)) return nullptr;
     for (const Stream64Config& c : stream64_configs())
         if (c.radius == p->radius && c.box == (p->shape == STENCIL_BOX)) return &c;
     return nullptr;
@@ -1432,9 +1438,9 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
             int pnx, pny, pnz;
             const double* padded = nullptr;
             if ((rc = pad_periodic(p, src, st, &padded, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
-            rc = get_tensor_map_f64(p, cfg, kStream64PX, cfg->box_rows, padded, &map, pnx, pny, pnz);
+            rc = get_tensor_map_f64(p, cfg, cfg->px, cfg->box_rows, padded, &map, pnx, pny, pnz);
         } else {
-            rc = get_tensor_map_f64(p, cfg, kStream64PX, cfg->box_rows, src, &map);
+            rc = get_tensor_map_f64(p, cfg, cfg->px, cfg->box_rows, src, &map);
         }
         if (rc != STENCIL_OK) return rc;
         const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : (p->radius >= 3 ? 5 : 4);
@@ -1521,9 +1527,9 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
             int pnx, pny, pnz;
             const double* padded = nullptr;
             if ((rc = pad_periodic(p, src, st, &padded, &pnx, &pny, &pnz)) != STENCIL_OK) return rc;
-            rc = get_tensor_map_f64(p, cfg, kPX64, cfg->YB, padded, &map, pnx, pny, pnz);
+            rc = get_tensor_map_f64(p, cfg, cfg->px, cfg->YB, padded, &map, pnx, pny, pnz);
         } else {
-            rc = get_tensor_map_f64(p, cfg, kPX64, cfg->YB, src, &map);
+            rc = get_tensor_map_f64(p, cfg, cfg->px, cfg->YB, src, &map);
         }
         if (rc != STENCIL_OK) return rc;
         const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;

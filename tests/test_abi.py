@@ -223,8 +223,9 @@ def test_fp64_variant_selection_rules():
         w = (wl.random_box_weights if box else wl.random_star_weights)(nd, R, 3, np.float64)
         return b.Plan(dims, R, b.BOX if box else b.STAR, w, boundary)
     tiled = [((64, 64), 4, True, b.ZERO), ((64, 64), 4, False, b.PERIODIC), ((33, 65), 3, True, b.ZERO),
-             ((32, 32, 32), 2, True, b.ZERO), ((32, 32, 32), 4, False, b.PERIODIC), ((8, 9, 31), 1, True, b.ZERO)]
-    generic = [((64, 64), 5, True, b.ZERO), ((32, 32, 32), 3, True, b.ZERO), ((32, 32, 32), 5, False, b.ZERO),
+             ((32, 32, 32), 2, True, b.ZERO), ((32, 32, 32), 4, False, b.PERIODIC), ((8, 9, 31), 1, True, b.ZERO),
+             ((32, 32, 32), 5, False, b.ZERO), ((64, 64), 8, False, b.PERIODIC), ((16, 16, 16), 8, False, b.PERIODIC)]
+    generic = [((64, 64), 5, True, b.ZERO), ((32, 32, 32), 3, True, b.ZERO), ((32, 32, 12), 7, False, b.PERIODIC),
                ((32, 32, 31), 1, False, b.PERIODIC), ((64, 63), 1, False, b.PERIODIC)]
     for args in tiled:
         with plan(*args) as p:

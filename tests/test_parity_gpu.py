@@ -246,6 +246,26 @@ def test_wide_star_rows2d_kernel_matches_oracle(R, dims, chunk, stages):
         assert used == "stream"
 
 
+@pytest.mark.parametrize("R", [5, 6, 7, 8])
+@pytest.mark.parametrize("dims,chunk,stages", [((67, 66), 0, 0), ((200, 258), 37, 2), ((3, 8), 0, 0), ((40, 33, 130), 0, 0),
+                                               ((37, 29, 64), 9, 3), ((3, 5, 4), 0, 2)])
+def test_wide_star_fp64_kernels_match_oracle(R, dims, chunk, stages):
+    """FP64 stars of radius 5..8 on the tiled kernels (8 halo doubles per side)."""
+    nd = len(dims)
+    w = wl.random_star_weights(nd, R, 27, np.float64)
+    a = wl.normal_field(dims, 28, np.float64)
+    for steps in (1, 3):
+        got, used = gpu_sweep(dims, R, b.STAR, w, b.ZERO, a, steps, chunk_z=chunk or None, stages=stages or None)
+        assert used == "stream" and got.dtype == np.float64
+        want = oracle.apply(a, w, b.ZERO, steps)
+        assert float(np.max(np.abs(got - want))) <= wl.tolerance(w, float(np.abs(a).max()), steps)
+    if min(dims) >= 2 * R:
+        got, used = gpu_sweep(dims, R, b.STAR, w, b.PERIODIC, a, 2)
+        assert used == "stream"
+        want = oracle.apply(a, w, b.PERIODIC, 2)
+        assert float(np.max(np.abs(got - want))) <= wl.tolerance(w, float(np.abs(a).max()), 2)
+
+
 # ------------------------------------------------- periodic boundary, tiled path --
 # periodic_route: None = chosen by the library, 2 = wrap correction after a zero-boundary sweep (extents >= 2R),
 # 1 = sweep from a padded copy with wrapped halos
