@@ -43,9 +43,9 @@ struct FusedShape {
     static constexpr int TYE = NWY * K;
     static constexpr int THREADS = XW * NWY * 32;
     // A TMA box is at most 256 elements wide, so a wider plane lies in shared memory as NP parts
-    // of PW columns, each loaded by its own copy and each with its own pad rows:
+    // of PW columns (two of 256 for a 512-wide region, three of 128 for a 384-wide one), each loaded by its own copy and each with its own pad rows:
     // cell (row r, column x) of a plane is at  (x / PW) * PART_FLOATS + r * PW + x % PW.
-    static constexpr int PW = TXE > 256 ? 256 : TXE;
+    static constexpr int PW = TXE <= 256 ? TXE : (TXE % 256 == 0 ? 256 : 128);
     static constexpr int NP = TXE / PW;
     static constexpr int PART_FLOATS = (TYE + 2 * R) * PW;      // R pad rows above and below
     static constexpr int SLOT_FLOATS = NP * PART_FLOATS;

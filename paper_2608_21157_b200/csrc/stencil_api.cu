@@ -111,6 +111,7 @@ struct StreamConfig {
 struct FusedConfig {
     int radius, T, K, XW, NWY;
     int txe, tye, threads, slot_bytes;
+    int pw;                                  // width of the TMA boxes a plane is loaded as
     const void* kernel;
     const void* kernel_spec;                 // the instantiation for full passes over rows of exactly txe points
     mutable size_t smem_allowed;             // dynamic shared memory already granted to both kernels
@@ -365,7 +366,7 @@ FusedConfig make_fused() {
     using S = FusedShape<R, K, XW, NWY>;
     FusedConfig c;
     c.radius = R; c.T = T; c.K = K; c.XW = XW; c.NWY = NWY;
-    c.txe = S::TXE; c.tye = S::TYE; c.threads = S::THREADS; c.slot_bytes = S::SLOT_BYTES;
+    c.txe = S::TXE; c.tye = S::TYE; c.threads = S::THREADS; c.slot_bytes = S::SLOT_BYTES; c.pw = S::PW;
     c.kernel = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, false>);
     c.kernel_spec = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, true>);
     c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
@@ -378,7 +379,7 @@ FusedConfig make_fused() {
 const std::vector<FusedConfig>& fused_configs() {
     static const std::vector<FusedConfig> v = {
         make_fused<1, 2, 4, 2, 8>(),  make_fused<1, 3, 4, 2, 8>(),  make_fused<1, 2, 4, 2, 4>(),
-        make_fused<1, 2, 2, 2, 8>(),  make_fused<1, 2, 4, 4, 4>(),
+        make_fused<1, 2, 2, 2, 8>(),  make_fused<1, 2, 4, 4, 4>(),  make_fused<1, 2, 4, 3, 5>(),
         make_fused<1, 4, 2, 1, 16>(), make_fused<1, 2, 2, 1, 16>(), make_fused<1, 3, 2, 1, 16>(),
         make_fused<2, 2, 2, 1, 16>(),
     };
@@ -510,15 +511,26 @@ const FusedConfig* pick_fused(const stencil_plan_s* p) {
         // grids stay unfused unless the caller asks for fusion.  Measured (G updates/s, fused
         // vs unfused, 512 x 512 x nx): nx = 128: 1083 vs 644 (256-wide region: 499); 192: 744 vs
         // 709; 400: 761 vs 776; 448: 851 vs 788; 512: 1257 vs 781.
-        // Rows wider than 512 points take several 512-wide regions, each with 4 halo columns
-        // per side for every 2 levels of radius 1, under the same 80 % rule (256 x 512 x nx:
-        // nx = 1000, two regions: 977 vs 782; 1024, three regions: 629 vs 786; 2048, five: 812
-        // vs 775; 4096, nine: 848 vs 761).
+        // 384-wide regions are 20 rows high (15 warps, one CTA per SM; their planes are loaded as
+        // three boxes of 128 columns): 512 x 512 x 384 1359 vs 827, nx = 320: 1027 vs 773.
+        // Rows wider than 512 points take several 384- or 512-wide regions, each with 4 halo
+        // columns per side for every 2 levels of radius 1, under the same 80 % rule; per lane the
+        // 384-wide regions are a quarter faster there (256 x 512 x nx, 384-wide / 512-wide / unfused:
+        // nx = 1128: 1217 / 693 / 836; 1500: 1128 / 954 / 830; 256 x 1024 x 1024: 1126 / 687 / 808;
+        // nx = 768 fills neither to 80 %: 788 / 753 / 828).
         const FusedConfig* c = nullptr;
-        const int width = p->nx <= 128 ? 128 : p->nx <= 256 ? 256 : 512;
-        const int tile = width - 2 * ((2 * p->radius + 3) / 4 * 4);          // columns a region stores
-        const int64_t regions = p->nx <= width ? 1 : (p->nx + tile - 1) / tile;
-        if ((int64_t)p->nx * 5 >= regions * width * 4) {
+        const int halo = (2 * p->radius + 3) / 4 * 4;                         // per side, when a row takes several regions
+        auto lanes_used = [&](int w) {
+            const int64_t regions = p->nx <= w ? 1 : (p->nx + (w - 2 * halo) - 1) / (w - 2 * halo);
+            return (double)p->nx / (double)(regions * w);
+        };
+        int width = p->nx <= 128 ? 128 : p->nx <= 256 ? 256 : p->nx <= 384 ? 384 : 512;
+        if (p->nx > 512 && 1.25 * lanes_used(384) >= lanes_used(512)) width = 384;
+        const int height = width == 128 ? 0 : width == 384 ? 20 : 16;
+        // the 384-wide regions pay off from fewer used lanes: any row of 257..384 points (nx = 260:
+        // 838 vs 676), three quarters of the lanes with several regions per row (896: 983 vs 843)
+        const double need = width != 384 ? 0.8 : p->nx <= 384 ? 0.0 : 0.75;
+        if (lanes_used(width) >= need) {
             // 128-wide regions leave registers for a third level (512 x 512 x 128: 1224 G updates/s
             // with three steps per pass, 1083 with two, 1108 with four); at 256 columns three
             // levels spill (256^3: 820 against 1056)
@@ -533,7 +545,7 @@ const FusedConfig* pick_fused(const stencil_plan_s* p) {
                     if (ctas >= 148) c = c3;
                 }
             }
-            if (!c) c = find_fused_cfg(p->radius, 2, width, width == 128 ? 0 : 16);
+            if (!c) c = find_fused_cfg(p->radius, 2, width, height);
             if (!c && width == 256) c = find_fused_cfg(p->radius, 2, 256);
         }
         if (c || p->fuse_steps == 0) return c;
@@ -1016,7 +1028,7 @@ int launch_rows2d_fused(stencil_plan_s* p, const float* src, float* dst, int nle
 int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cudaStream_t st) {
     const FusedConfig* cfg = p->fused_cfg;
     const CUtensorMap* map = nullptr;
-    int rc = get_tensor_map(p, cfg, std::min(cfg->txe, 256), cfg->tye, src, &map);   // a box is at most 256 wide
+    int rc = get_tensor_map(p, cfg, cfg->pw, cfg->tye, src, &map);   // a box is at most 256 wide
     if (rc != STENCIL_OK) return rc;
     const int R = p->radius, T = cfg->T;
     FusedGeom g;

@@ -182,13 +182,22 @@ def test_fuse_knob_rules():
     """Which iterated applies fuse time steps by default, and with which region (host logic only)."""
     star = wl.star_weights(3, 1, 0.4, [0.1])
     with b.Plan((64, 64, 1000), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 512      # two regions, 98 % of their lanes
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 384      # three 384-wide regions: 87 % of their lanes
     with b.Plan((64, 64, 1024), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 1         # would take three regions (two store 504 columns each): 67 %
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 384      # three regions store 376 columns each: 89 %
+        assert p.get(b.KEY_FUSED_TILE_Y) == 20
         p.set(b.KEY_FUSE_STEPS, 4)
         assert p.get(b.KEY_FUSE_STEPS) == 4
+    with b.Plan((64, 64, 768), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # three 384-wide regions 67 %, two 512-wide ones 75 %
     with b.Plan((64, 64, 320), 1, b.STAR, star, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 1         # a 512-wide region would idle too many lanes
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 384      # 83 % of a 384-wide region
+    with b.Plan((64, 64, 260), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 384      # pays off from 257 points on
+    with b.Plan((64, 64, 400), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # 78 % of a 512-wide region
+    with b.Plan((64, 64, 896), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_TILE_X) == 384      # three regions, 78 %
     with b.Plan((64, 64, 512), 1, b.STAR, star, b.ZERO) as p:
         assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_FUSED_TILE_Y) == 16   # one 512-wide region per row
     with b.Plan((64, 64, 448), 1, b.STAR, star, b.ZERO) as p:

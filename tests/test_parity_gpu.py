@@ -471,7 +471,7 @@ def test_f64_fused_2d_passes_match_oracle(R, box, T, dims, chunk, stages):
 # -------------------------------------------------------------------- fused --
 FUSED_CONFIGS = [   # (radius, fuse_steps, region width, region height)
     (1, 2, 256, 32), (1, 2, 256, 16), (1, 3, 256, 32), (1, 4, 128, 32), (1, 2, 128, 32), (1, 3, 128, 32),
-    (2, 2, 128, 32), (1, 2, 512, 16),
+    (2, 2, 128, 32), (1, 2, 512, 16), (1, 2, 384, 20),
 ]
 
 
@@ -483,6 +483,7 @@ FUSED_CONFIGS = [   # (radius, fuse_steps, region width, region height)
     ((21, 37, 512), 8),         # ... and for the 512-wide region, which is loaded as two TMA boxes
     ((19, 30, 452), 0),         # a row that ends inside the second box of a 512-wide region
     ((9, 20, 1000), 0),         # two 512-wide regions per row
+    ((17, 41, 384), 6),         # a 384-wide region (three TMA boxes of 128) spans the row
     ((5, 9, 12), 0),            # much smaller than one region
 ])
 def test_fused_passes_match_oracle(R, T, width, height, dims, chunk_z):
