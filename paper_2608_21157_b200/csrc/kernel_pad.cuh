@@ -102,6 +102,37 @@ stencil_refresh_halo_kernel(T* __restrict__ pad, Grid g, int ry, int rz) {
 // of the grid to be at least 2R, so that the three parts are disjoint.
 constexpr int kWrapSmemTaps = 128;
 
+// Point number i of the shell of depth R (rz along z): first the 2*rz whole planes next to the
+// z faces, then the 2R whole rows next to the y faces of the other planes, then the first and
+// last R points of the other rows.
+__device__ __forceinline__ void shell_point(int64_t i, const Grid& g, int R, int rz, int64_t part1, int64_t part2,
+                                            int inner_y, int& z, int& y, int& x) {
+    if (i < part1) {
+        const int64_t plane = (int64_t)g.ny * g.nx;
+        const int zi = (int)(i / plane);
+        const int r = (int)(i % plane);
+        z = zi < rz ? zi : g.nz - 2 * rz + zi;
+        y = r / g.nx;
+        x = r % g.nx;
+    } else if (i < part1 + part2) {
+        const int64_t j = i - part1;
+        const int per_z = 2 * R * g.nx;
+        const int r = (int)(j % per_z);
+        const int yi = r / g.nx;
+        z = (int)(j / per_z) + rz;
+        y = yi < R ? yi : g.ny - 2 * R + yi;
+        x = r % g.nx;
+    } else {
+        const int64_t j = i - part1 - part2;
+        const int64_t per_z = (int64_t)inner_y * 2 * R;
+        const int r = (int)(j % per_z);
+        const int c = r % (2 * R);
+        z = (int)(j / per_z) + rz;
+        y = r / (2 * R) + R;
+        x = c < R ? c : g.nx - 2 * R + c;
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256)
 stencil_wrap_correction_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g, int R, int rz,
@@ -119,30 +150,7 @@ stencil_wrap_correction_kernel(const T* __restrict__ in, T* __restrict__ out, Gr
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
         int z, y, x;
-        if (i < part1) {
-            const int64_t plane = (int64_t)g.ny * g.nx;
-            const int zi = (int)(i / plane);
-            const int r = (int)(i % plane);
-            z = zi < rz ? zi : g.nz - 2 * rz + zi;
-            y = r / g.nx;
-            x = r % g.nx;
-        } else if (i < part1 + part2) {
-            const int64_t j = i - part1;
-            const int per_z = 2 * R * g.nx;
-            const int r = (int)(j % per_z);
-            const int yi = r / g.nx;
-            z = (int)(j / per_z) + rz;
-            y = yi < R ? yi : g.ny - 2 * R + yi;
-            x = r % g.nx;
-        } else {
-            const int64_t j = i - part1 - part2;
-            const int64_t per_z = (int64_t)inner_y * 2 * R;
-            const int r = (int)(j % per_z);
-            const int c = r % (2 * R);
-            z = (int)(j / per_z) + rz;
-            y = r / (2 * R) + R;
-            x = c < R ? c : g.nx - 2 * R + c;
-        }
+        shell_point(i, g, R, rz, part1, part2, inner_y, z, y, x);
         T acc = T(0);
         for (int t = 0; t < ntaps; ++t) {
             const TapT<T> tap = staged ? s_taps[t] : taps[t];
@@ -158,6 +166,210 @@ stencil_wrap_correction_kernel(const T* __restrict__ in, T* __restrict__ out, Gr
         }
         const int64_t self = ((int64_t)z * g.ny + y) * g.nx + x;
         out[self] += acc;
+    }
+}
+
+// Periodic boundary under temporal blocking.  A fused pass of L time steps with a zero boundary
+// is right wherever the L-step cone of dependence stays inside the grid: at every point at
+// least H = L*R cells from every face.  The sweep is linear and, on the torus, invariant under
+// shifts, so L periodic steps equal ONE sweep with the operator's L-fold self-convolution (radius
+// H).  This kernel walks the shell of depth H and overwrites each of its points with that
+// composite sweep of the pass's input, indices wrapped.  The composite taps are doubles and the
+// sum runs in double, rounded once: the shell points skip the rounding to T after every
+// intermediate step, a difference far below the rounding error of the steps themselves.
+// Needs every extent of the grid to be at least 2H.
+// The kernel is bound by integer instructions (decoding the point, wrapping and indexing each
+// tap), so the index type I is 32 bits wide where the grid has fewer than 2^31 points, an axis
+// is only wrapped for points within H of its faces, and the point decode divides 32-bit numbers.
+template <typename T, typename I>
+__global__ void __launch_bounds__(256)
+stencil_shell_compose_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g, int H, int hz,
+                             const TapT<double>* __restrict__ taps, int ntaps) {
+    __shared__ TapT<double> s_taps[kWrapSmemTaps];
+    __shared__ I s_off[kWrapSmemTaps];
+    const bool staged = ntaps <= kWrapSmemTaps;
+    const I row = (I)g.nx, plane = (I)g.ny * (I)g.nx;
+    if (staged)
+        for (int t = threadIdx.x; t < ntaps; t += blockDim.x) {
+            s_taps[t] = taps[t];
+            s_off[t] = (I)taps[t].dz * plane + (I)taps[t].dy * row + (I)taps[t].dx;
+        }
+    __syncthreads();
+    const int inner_z = g.nz - 2 * hz, inner_y = g.ny - 2 * H;
+    const I part1 = (I)2 * hz * plane;
+    const I per_z2 = (I)2 * H * row, part2 = (I)inner_z * per_z2;
+    const I per_z3 = (I)inner_y * 2 * H, part3 = (I)inner_z * per_z3;
+    const I total = part1 + part2 + part3;
+    const I stride = (I)gridDim.x * blockDim.x;
+    for (I i = (I)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        int z, y, x;
+        if (i < part1) {                            // whole planes next to the z faces
+            const int zi = (int)(i / plane);
+            const I r = i - (I)zi * plane;
+            z = zi < hz ? zi : g.nz - 2 * hz + zi;
+            y = (int)(r / row);
+            x = (int)(r - (I)y * row);
+        } else if (i < part1 + part2) {             // whole rows next to the y faces of the other planes
+            const I j = i - part1;
+            const int zi = (int)(j / per_z2);
+            const I r = j - (I)zi * per_z2;
+            const int yi = (int)(r / row);
+            z = zi + hz;
+            y = yi < H ? yi : g.ny - 2 * H + yi;
+            x = (int)(r - (I)yi * row);
+        } else {                                    // the first and last H points of the other rows
+            const I j = i - part1 - part2;
+            const int zi = (int)(j / per_z3);
+            const int r = (int)(j - (I)zi * per_z3);
+            const int yi = r / (2 * H);
+            const int c = r - yi * 2 * H;
+            z = zi + hz;
+            y = yi + H;
+            x = c < H ? c : g.nx - 2 * H + c;
+        }
+        const I self = (I)z * plane + (I)y * row + (I)x;
+        // An axis wraps only for points within H of its faces, and then in one direction only: a
+        // point near the low face wraps taps with d < -coordinate, one near the high face taps with
+        // d >= extent - coordinate.  (Every extent is at least 2H, so a point is near one face at most.)
+        const bool zlo = z < hz, zhi = z >= g.nz - hz;
+        const bool ylo = y < H, yhi = y >= g.ny - H;
+        const bool xlo = x < H, xhi = x >= g.nx - H;
+        const I zfix = zlo ? (I)g.nz * plane : -(I)g.nz * plane;
+        const I yfix = ylo ? plane : -plane;
+        const I xfix = xlo ? row : -row;
+        double acc = 0.0;
+#pragma unroll 4
+        for (int t = 0; t < ntaps; ++t) {
+            TapT<double> tap;
+            I idx;
+            if (staged) { tap = s_taps[t]; idx = self + s_off[t]; }
+            else { tap = taps[t]; idx = self + (I)tap.dz * plane + (I)tap.dy * row + (I)tap.dx; }
+            if (zlo || zhi) { if (zlo ? z + tap.dz < 0 : z + tap.dz >= g.nz) idx += zfix; }
+            if (ylo || yhi) { if (ylo ? y + tap.dy < 0 : y + tap.dy >= g.ny) idx += yfix; }
+            if (xlo || xhi) { if (xlo ? x + tap.dx < 0 : x + tap.dx >= g.nx) idx += xfix; }
+            acc = fma(tap.w, (double)in[idx], acc);
+        }
+        out[self] = (T)acc;
+    }
+}
+
+// The same job split in two for speed (the point-by-point walk above spends some 30 instructions
+// per tap on wrapping and indexing, and stays as the fallback for operators with more than
+// kShellTaps composite taps).  The sums run in T with the composite weights rounded to T.
+//
+// Whole rows (the planes next to the z faces, the rows next to the y faces of the other planes):
+// one CTA per kShellRowChunk points of a row.  The row's z and y are the CTA's, so the wrapped row every tap reads from is
+// resolved once per CTA into shared memory; a point between the row's ends then spends a shared
+// load, an add, a global load and an FMA per tap, and only the first and last H points wrap in x.
+constexpr int kShellTaps = 160;
+constexpr int kShellRowChunk = 512;
+
+template <typename T>
+struct ShellRowTap {
+    int64_t base;          // index of the cell the tap reads for x = 0 (dx included)
+    T w;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+stencil_shell_rows_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g, int H, int hz,
+                          const TapT<double>* __restrict__ taps, int ntaps, int xchunks) {
+    __shared__ ShellRowTap<T> s_tap[kShellTaps];
+    __shared__ int s_dx[kShellTaps];
+    const int r = blockIdx.x / xchunks;
+    const int xbegin = (int)(blockIdx.x % xchunks) * kShellRowChunk;
+    const int xend = min(xbegin + kShellRowChunk, g.nx);
+    int z, y;
+    if (r < 2 * hz * g.ny) {
+        const int zi = r / g.ny;
+        z = zi < hz ? zi : g.nz - 2 * hz + zi;
+        y = r - zi * g.ny;
+    } else {
+        const int q = r - 2 * hz * g.ny;
+        const int yi = q % (2 * H);
+        z = q / (2 * H) + hz;
+        y = yi < H ? yi : g.ny - 2 * H + yi;
+    }
+    for (int t = threadIdx.x; t < ntaps; t += blockDim.x) {
+        const TapT<double> tap = taps[t];
+        int qz = z + tap.dz, qy = y + tap.dy;
+        // every extent is at least 2H >= |offset|: one step brings the index back
+        qz = qz < 0 ? qz + g.nz : (qz >= g.nz ? qz - g.nz : qz);
+        qy = qy < 0 ? qy + g.ny : (qy >= g.ny ? qy - g.ny : qy);
+        s_tap[t].base = ((int64_t)qz * g.ny + qy) * g.nx + tap.dx;
+        s_tap[t].w = (T)tap.w;
+        s_dx[t] = tap.dx;
+    }
+    __syncthreads();
+    T* orow = out + ((int64_t)z * g.ny + y) * g.nx;
+    for (int x = xbegin + threadIdx.x; x < xend; x += blockDim.x) {
+        T acc = T(0);
+        if (x >= H && x < g.nx - H) {
+            const T* px = in + x;
+#pragma unroll 4
+            for (int t = 0; t < ntaps; ++t) acc = fma_t(s_tap[t].w, px[s_tap[t].base], acc);
+        } else {
+            for (int t = 0; t < ntaps; ++t) {
+                const int qx = x + s_dx[t];
+                const int fix = qx < 0 ? g.nx : (qx >= g.nx ? -g.nx : 0);
+                acc = fma_t(s_tap[t].w, in[s_tap[t].base + x + fix], acc);
+            }
+        }
+        orow[x] = acc;
+    }
+}
+
+// The first and last H points of all other rows.  Walked point by point, every tap of every
+// point costs a 32-byte sector of its own; here a CTA takes a tile of TZ planes x TY rows, first
+// gathers the two ends of every row the tile's taps reach into shared memory as one circular
+// segment of 4H cells ([nx - 2H, nx) followed by [0, 2H)), and sums from there: the tile's rows lie
+// at least H rows and planes inside the grid, so nothing wraps in y or z, and the x wrap is the
+// segment's own order.  seg is (TZ + 2hz) x (TY + 2H) x 4H cells of dynamic shared memory.
+constexpr int kShellTY = 32;
+__host__ __device__ constexpr int shell_tz(int H, int hz) { return hz == 0 ? 1 : (H <= 2 ? 8 : 4); }   // planes per tile
+
+template <typename T>
+struct ShellSegTap {
+    int off;               // offset of the tap's cell from the output's own cell inside seg
+    T w;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+stencil_shell_xfaces_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g, int H, int hz,
+                            const TapT<double>* __restrict__ taps, int ntaps) {
+    extern __shared__ __align__(16) unsigned char shell_smem[];
+    __shared__ ShellSegTap<T> s_tap[kShellTaps];
+    T* seg = reinterpret_cast<T*>(shell_smem);
+    const int tz = shell_tz(H, hz);
+    const int tiles_y = (g.ny - 2 * H + kShellTY - 1) / kShellTY;
+    const int y0 = H + (int)(blockIdx.x % tiles_y) * kShellTY;          // first output row and plane of the tile
+    const int z0 = hz + (int)(blockIdx.x / tiles_y) * tz;
+    const int sw = 4 * H, sy = kShellTY + 2 * H, sz = tz + 2 * hz;
+    for (int t = threadIdx.x; t < ntaps; t += blockDim.x) {
+        s_tap[t].off = (taps[t].dz * sy + taps[t].dy) * sw + taps[t].dx;
+        s_tap[t].w = (T)taps[t].w;
+    }
+    const int64_t plane = (int64_t)g.ny * g.nx;
+    // one thread per (row of the tile, cell of its segment); consecutive threads read consecutive cells
+    const int rows_per_round = blockDim.x / sw, k = threadIdx.x % sw;
+    for (int row = threadIdx.x / sw; row < sz * sy && (int)threadIdx.x < rows_per_round * sw; row += rows_per_round) {
+        const int lz = row / sy, ly = row - lz * sy;
+        const int gz = z0 - hz + lz, gy = y0 - H + ly;
+        const int gx = k < 2 * H ? g.nx - 2 * H + k : k - 2 * H;
+        seg[row * sw + k] = (gz < g.nz && gy < g.ny) ? in[(int64_t)gz * plane + (int64_t)gy * g.nx + gx] : T(0);
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < tz * kShellTY * 2 * H; e += blockDim.x) {
+        const int c = e % (2 * H), ly = (e / (2 * H)) % kShellTY, lz = e / (2 * H * kShellTY);
+        const int z = z0 + lz, y = y0 + ly;
+        if (z >= g.nz - hz || y >= g.ny - H) continue;
+        const T* ctr = seg + ((lz + hz) * sy + (ly + H)) * sw + H + c;          // this output's own cell
+        T acc = T(0);
+#pragma unroll 4
+        for (int t = 0; t < ntaps; ++t) acc = fma_t(s_tap[t].w, ctr[s_tap[t].off], acc);
+        const int x = c < H ? g.nx - H + c : c - H;                             // the cell at segment position H + c
+        out[(int64_t)z * plane + (int64_t)y * g.nx + x] = acc;
     }
 }
 

@@ -126,7 +126,11 @@ def test_variant_selection_rules():
         assert p.variant == "generic"
     with b.Plan((64, 64, 64), 1, b.STAR, star, b.PERIODIC) as p:
         assert p.variant == "stream"                # swept from a padded copy with wrapped halos
-        assert p.get(b.KEY_FUSE_STEPS) == 1         # no temporal blocking under a periodic boundary
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # rows of 64 points are too narrow for the fused regions
+    with b.Plan((64, 64, 256), 1, b.STAR, star, b.PERIODIC) as p:
+        assert p.variant == "stream" and p.get(b.KEY_FUSE_STEPS) == 2     # periodic grids fuse like zero-boundary ones
+    with b.Plan((3, 64, 256), 1, b.STAR, star, b.PERIODIC) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1         # ... when every extent holds both shells of depth T * R
     with b.Plan((64, 64, 62), 1, b.STAR, star, b.PERIODIC) as p:
         assert p.variant == "generic"
         with pytest.raises(b.StencilError) as e:
@@ -263,7 +267,9 @@ def test_fuse_rules_2d():
             p.set(b.KEY_FUSE_STEPS, 0)
             assert p.get(b.KEY_FUSE_STEPS) == T
         with b.Plan((64, 128), R, b.BOX if box else b.STAR, w, b.PERIODIC) as p:
-            assert p.get(b.KEY_FUSE_STEPS) == 1         # no temporal blocking under a periodic boundary
+            assert p.get(b.KEY_FUSE_STEPS) == T         # a periodic grid fuses too (its shell is rewritten after a pass) ...
+        with b.Plan((2 * T * R - 1, 128), R, b.BOX if box else b.STAR, w, b.PERIODIC) as p:
+            assert p.get(b.KEY_FUSE_STEPS) == 1         # ... when it holds both shells of depth T * R
         with b.Plan((64, 126), R, b.BOX if box else b.STAR, w, b.ZERO) as p:
             assert p.get(b.KEY_FUSE_STEPS) == 1         # rows that are not 16-byte multiples
     with b.Plan((64, 128), 3, b.BOX, wl.random_box_weights(2, 3, 3), b.ZERO) as p:

@@ -266,6 +266,82 @@ def test_wide_star_fp64_kernels_match_oracle(R, dims, chunk, stages):
         assert float(np.max(np.abs(got - want))) <= wl.tolerance(w, float(np.abs(a).max()), 2)
 
 
+# ------------------------------------------- periodic boundary under temporal blocking --
+@pytest.mark.parametrize("dims,R,knobs", [
+    ((21, 37, 256), 1, {}),                                         # one 256-wide region per row, T = 2
+    ((33, 50, 128), 1, {}),                                         # 128-wide region
+    ((16, 18, 128), 1, dict(fuse_steps=4, tile_x=128)),             # the deepest pass: shells of depth 4
+    ((12, 20, 1000), 1, {}),                                        # several regions per row
+    ((17, 30, 384), 1, dict(chunk_z=5)),                            # 384-wide region, several z chunks
+    ((16, 40, 128), 2, dict(fuse_steps=2, tile_x=128)),             # radius 2: shells of depth 4
+    ((4, 4, 128), 1, dict(fuse_steps=2, tile_x=128)),               # the two shells fill the grid in z and y
+])
+def test_periodic_fused_3d_matches_oracle(dims, R, knobs):
+    w = wl.random_star_weights(3, R, 71)
+    a = wl.normal_field(dims, 72)
+    T = knobs.get("fuse_steps", 0)
+    for steps in (2, 3, 5, 9):
+        dev = torch.device("cuda:0")
+        src = torch.from_numpy(a).to(dev)
+        dst = torch.full_like(src, float("nan"))
+        with b.Plan(dims, R, b.STAR, w, b.PERIODIC, **knobs) as p:
+            depth = p.get(b.KEY_FUSE_STEPS)
+            assert depth > 1 and (T == 0 or depth == T)
+            p.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
+            assert p.query_status() == b.OK
+            passes = -(-steps // depth)
+            assert 2 * passes <= p.launches <= 3 * passes           # a pass and its one or two shell kernels
+        got = dst.cpu().numpy()
+        want = oracle.apply(a, w, b.PERIODIC, steps)
+        tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+        err = float(np.max(np.abs(got - want)))
+        assert err <= tol, f"dims={dims} R={R} steps={steps}: {err:.3e} > {tol:.3e}"
+
+
+@pytest.mark.parametrize("R,box,T", [(1, False, 4), (1, True, 4), (2, False, 3), (2, True, 2), (3, False, 2), (4, False, 2)])
+@pytest.mark.parametrize("dims", [(67, 132), (200, 260), (16, 16)])
+@pytest.mark.parametrize("f64", [False, True])
+def test_periodic_fused_2d_matches_oracle(R, box, T, dims, f64):
+    if f64 and R > 2:
+        pytest.skip("no FP64 cascade beyond radius 2")
+    dt = np.float64 if f64 else np.float32
+    w = (wl.random_box_weights if box else wl.random_star_weights)(2, R, 73, dt)
+    a = wl.normal_field(dims, 74, dt)
+    fits = min(dims) >= 2 * T * R
+    for steps in (T, T + 1, 2 * T + 1):
+        got, used = gpu_sweep(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC, a, steps)
+        assert used == "stream"
+        want = oracle.apply(a, w, b.PERIODIC, steps)
+        tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+        err = float(np.max(np.abs(got.astype(np.float64) - want.astype(np.float64))))
+        assert err <= tol, f"R={R} box={box} dims={dims} steps={steps} f64={f64} fits={fits}: {err:.3e} > {tol:.3e}"
+    with b.Plan(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == (T if fits else 1)
+
+
+def test_periodic_fused_conserves_the_sum_on_a_large_grid():
+    """Heat weights sum to 1: under a periodic boundary the total is conserved through fused passes
+    (a grid too large for the element-wise oracle)."""
+    dims = (256, 256, 256)
+    w = wl.star_weights(3, 1, 0.4, [0.1])
+    a = wl.uniform_field(dims, 0.0, 1.0, 75)
+    src = torch.from_numpy(a).cuda()
+    dst = torch.empty_like(src)
+    with b.Plan(dims, 1, b.STAR, w, b.PERIODIC) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2
+        p.apply(src, dst, 16, torch.cuda.current_stream().cuda_stream)
+        assert p.query_status() == b.OK
+    total0 = float(src.double().sum())
+    total1 = float(dst.double().sum())
+    assert abs(total1 - total0) <= 2e-6 * abs(total0)
+    assert float(dst.min()) >= 0.0 and float(dst.max()) <= float(src.max())      # max principle
+    # the same apply through the unfused wrap-correction route
+    ref = torch.empty_like(src)
+    with b.Plan(dims, 1, b.STAR, w, b.PERIODIC, fuse_steps=1) as p:
+        p.apply(src, ref, 16, torch.cuda.current_stream().cuda_stream)
+    assert float((dst - ref).abs().max()) <= 16 * 1e-5 + 1e-6
+
+
 # ------------------------------------------------- periodic boundary, tiled path --
 # periodic_route: None = chosen by the library, 2 = wrap correction after a zero-boundary sweep (extents >= 2R),
 # 1 = sweep from a padded copy with wrapped halos
