@@ -67,7 +67,7 @@ enum {
 /* Keys of stencil_plan_set / stencil_plan_get. */
 enum {
     STENCIL_KEY_VARIANT      = 0,  /* set/get: STENCIL_VARIANT_*                                 */
-    STENCIL_KEY_TILE_X       = 1,  /* set/get: region width of fused 3D passes, 128, 256 or 512 (0 = auto) */
+    STENCIL_KEY_TILE_X       = 1,  /* set/get: region width of fused 3D passes, 128, 256, 384 or 512 (0 = auto) */
     STENCIL_KEY_TILE_Y       = 2,  /* set/get: tile height in rows   (0 = default)               */
     STENCIL_KEY_FUSE_STEPS   = 3,  /* set: time steps fused per pass (0 = auto, 1 = off; 3D fp32
                                       stars: 2-4; 2D grids: the one depth the operator's fused
@@ -86,12 +86,16 @@ enum {
                                       programmatic dependent launches: each begins its preamble
                                       while its predecessor drains and waits for it before it
                                       touches global memory; 0 = ordinary launches             */
-    STENCIL_KEY_FUSED_TILE_Y = 13,   /* set/get: region height of fused 3D passes, 16 or 32 (0 = auto) */
+    STENCIL_KEY_FUSED_TILE_Y = 13,   /* set/get: region height of fused 3D passes, 16, 20 or 32 (0 = auto) */
     STENCIL_KEY_PERIODIC_ROUTE = 14, /* set/get: how the tiled kernels handle a periodic boundary.
                                       1 = sweep from a padded copy with wrapped halos; 2 = zero-
                                       boundary sweep plus a correction of the points within R of
                                       a face (needs every extent >= 2R, else as 1); 0 (default)
-                                      = whichever of the two is cheaper for the operator          */
+                                      = whichever of the two is cheaper for the operator.
+                                      Iterated applies of an operator with a fused kernel run
+                                      fused zero-boundary passes of L steps and rewrite the points
+                                      within L*R of a face afterwards (every extent >= 2*L*R),
+                                      unless this key is 1 or STENCIL_KEY_FUSE_STEPS is 1         */
     STENCIL_KEY_TEST_DROP_PLANE = 11 /* set/get, test hook: every CTA of the 3D single-step kernel
                                       never loads its input plane of this index, so the bounded
                                       wait for it expires and stencil_query_status reports
