@@ -19,18 +19,20 @@ zero boundary): the sends and receives are started, the planes that read no
 ghost plane are swept meanwhile, and the R planes next to each neighbour follow
 once the ghost planes have arrived.
 
-The first rank has no ghost planes below and the last none above: their slabs
-end at the grid's own zero boundary, which the local plan imposes at every
-step.  There is no all-reduce or all-gather on the data path.
+Under the zero boundary the first rank has no ghost planes below and the last
+none above: their slabs end at the grid's own boundary, which the local plan
+imposes at every step.  Under the periodic boundary the ranks form a ring (the
+first rank's lower neighbour is the last rank), every rank keeps ghost planes on
+both sides, and the local plan is periodic: right along the two axes a rank holds
+completely, and wrong only at the ends of the extended slab along the split
+axis, where the ghost planes absorb it like the zero boundary's error.  There
+is no all-reduce or all-gather on the data path.
 
 The paper runs every task on a single GPU and leaves multi-GPU execution open;
 this module is the natural sharding of the sweep, kept outside the three-call C
 ABI.  It has been exercised with several ranks on CPU (gloo), with one rank on a
 GPU, and with the slabs of several ranks swept one after the other on one GPU
 (exchange by direct copies), never yet on several GPUs.
-
-Zero boundary only: a periodic grid would also wrap the first rank's planes
-around to the last rank.
 """
 from __future__ import annotations
 
@@ -41,6 +43,7 @@ import numpy as np
 from . import binding
 
 ZERO = binding.ZERO
+PERIODIC = binding.PERIODIC
 
 
 def slab_range(n: int, world: int, rank: int) -> Tuple[int, int]:
@@ -69,8 +72,8 @@ class ShardedSweep:
                  boundary: int = ZERO, *, rank: int, world: int, dist=None, group=None,
                  halo_steps: int = 1, local_apply: Optional[Callable] = None,
                  local_apply_planes: Optional[Callable] = None, overlap: bool = True):
-        if boundary != ZERO:
-            raise ValueError("sharded sweeps support the zero boundary only")
+        if boundary not in (ZERO, PERIODIC):
+            raise ValueError("boundary must be ZERO or PERIODIC")
         if halo_steps < 1:
             raise ValueError("halo_steps must be >= 1")
         self.dims = tuple(int(d) for d in dims)
@@ -85,8 +88,14 @@ class ShardedSweep:
             raise ValueError("every rank needs at least halo_steps * R planes of its own")
         if self.world > 1 and dist is None:
             raise ValueError("world > 1 needs torch.distributed")
-        self.lo = self.depth if self.rank > 0 else 0       # ghost planes below / above the own planes
-        self.hi = self.depth if self.rank < self.world - 1 else 0
+        # neighbours along the split axis: a chain under the zero boundary, a ring under the periodic one
+        ring = boundary == PERIODIC and self.world > 1
+        self.lower = (self.rank - 1) % self.world if (ring or self.rank > 0) else None
+        self.upper = (self.rank + 1) % self.world if (ring or self.rank < self.world - 1) else None
+        if self.world == 1:
+            self.lower = self.upper = None
+        self.lo = self.depth if self.lower is not None else 0       # ghost planes below / above the own planes
+        self.hi = self.depth if self.upper is not None else 0
         self.local_dims = (self.lo + self.nlocal + self.hi,) + self.dims[1:]
         self._plan = None
         if local_apply is None:
@@ -97,7 +106,7 @@ class ShardedSweep:
                 self._plan.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
 
             ranged = (len(self.dims) == 3 and self._plan.variant == "stream" and not self._plan.f64
-                      and self.dims[-1] % 4 == 0)
+                      and self.dims[-1] % 4 == 0 and boundary == ZERO)
             if ranged and local_apply_planes is None:
                 def local_apply_planes(src, dst, z_begin, z_end):
                     self._plan.apply_planes(src, dst, z_begin, z_end, torch.cuda.current_stream().cuda_stream)
@@ -127,13 +136,19 @@ class ShardedSweep:
         if self.world == 1:
             return []
         d, D, n, lo = self.dist, self.depth, self.nlocal, self.lo
+        # Messages travelling down the axis carry tag 1, those travelling up tag 0.  In a ring of two
+        # ranks both neighbours are the same peer: the receives are listed in the order of that
+        # peer's sends (its "down" arrives from above, its "up" from below) for backends that
+        # match the messages of a pair by order instead of by tag.
         ops = []
-        if self.rank > 0:                                    # my lowest planes <-> lower neighbour
-            ops.append(d.P2POp(d.isend, ext[lo:lo + D], self.rank - 1, self.group))
-            ops.append(d.P2POp(d.irecv, ext[:lo], self.rank - 1, self.group))
-        if self.rank < self.world - 1:                       # my highest planes <-> upper neighbour
-            ops.append(d.P2POp(d.isend, ext[lo + n - D:lo + n], self.rank + 1, self.group))
-            ops.append(d.P2POp(d.irecv, ext[lo + n:], self.rank + 1, self.group))
+        if self.lower is not None:                           # my lowest planes -> lower neighbour
+            ops.append(d.P2POp(d.isend, ext[lo:lo + D], self.lower, self.group, 1))
+        if self.upper is not None:                           # my highest planes -> upper neighbour
+            ops.append(d.P2POp(d.isend, ext[lo + n - D:lo + n], self.upper, self.group, 0))
+        if self.upper is not None:                           # upper ghost planes <- upper neighbour's lowest
+            ops.append(d.P2POp(d.irecv, ext[lo + n:], self.upper, self.group, 1))
+        if self.lower is not None:                           # lower ghost planes <- lower neighbour's highest
+            ops.append(d.P2POp(d.irecv, ext[:lo], self.lower, self.group, 0))
         return d.batch_isend_irecv(ops)
 
     @staticmethod
@@ -161,8 +176,8 @@ class ShardedSweep:
                 # planes travel, then the R planes next to each neighbour (an edge rank's outer
                 # side has no ghosts: its planes belong to the first range)
                 R, lo, n = self.R, self.lo, self.nlocal
-                inner0 = lo + (R if self.rank > 0 else 0)
-                inner1 = lo + n - (R if self.rank < self.world - 1 else 0)
+                inner0 = lo + (R if self.lower is not None else 0)
+                inner1 = lo + n - (R if self.upper is not None else 0)
                 reqs = self.start_exchange(cur)
                 self._local_apply_planes(cur, other, inner0, inner1)
                 self.finish_exchange(reqs)

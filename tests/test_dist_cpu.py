@@ -63,7 +63,7 @@ def test_slab_ranges_cover_the_axis_once():
         assert max(sizes) - min(sizes) <= 1
 
 
-def _sharded_worker(rank, world, port, dims, R, steps, halo_steps, overlap, out):
+def _sharded_worker(rank, world, port, dims, R, steps, halo_steps, overlap, periodic, out):
     import numpy as np
     import oracle
     from paper_2608_21157_b200 import workloads as wl
@@ -77,29 +77,31 @@ def _sharded_worker(rank, world, port, dims, R, steps, halo_steps, overlap, out)
         a = wl.normal_field(dims, 6)                    # every rank builds the same global field
 
         calls = []
+        boundary = oracle.PERIODIC if periodic else oracle.ZERO
 
         def local_apply(src, dst, nsteps):              # sweeps of the local slab, on the CPU
             calls.append(nsteps)
-            dst.copy_(torch.from_numpy(oracle.apply(src.numpy(), w, oracle.ZERO, nsteps)))
+            dst.copy_(torch.from_numpy(oracle.apply(src.numpy(), w, boundary, nsteps)))
 
         ranges = []
 
         def local_apply_planes(src, dst, z_begin, z_end):   # one sweep, output planes [z_begin, z_end) only
             ranges.append((z_begin, z_end))
-            full = torch.from_numpy(oracle.apply(src.numpy(), w, oracle.ZERO, 1))
+            full = torch.from_numpy(oracle.apply(src.numpy(), w, boundary, 1))
             dst[z_begin:z_end].copy_(full[z_begin:z_end])
 
-        sw = ShardedSweep(dims, R, 1, w, rank=rank, world=world, dist=dist, halo_steps=halo_steps,
-                          local_apply=local_apply, local_apply_planes=local_apply_planes if overlap else None)
+        sw = ShardedSweep(dims, R, 1, w, 1 if periodic else 0, rank=rank, world=world, dist=dist,
+                          halo_steps=halo_steps, local_apply=local_apply,
+                          local_apply_planes=local_apply_planes if overlap else None)
         assert sw.overlap == (overlap and halo_steps == 1)
-        expected_ghosts = halo_steps * R * ((rank > 0) + (rank < world - 1))
+        expected_ghosts = halo_steps * R * (2 if periodic else (rank > 0) + (rank < world - 1))
         assert sw.local_dims[0] == (sw.z1 - sw.z0) + expected_ghosts
         ext = sw.scatter(torch.from_numpy(a))
         res = sw.apply(ext, steps)
         if sw.overlap:
             # per step: the planes that read no ghost plane first, then R planes per neighbour; together
             # they cover the own planes exactly once
-            per_step = 1 + (rank > 0) + (rank < world - 1)
+            per_step = 3 if periodic else 1 + (rank > 0) + (rank < world - 1)
             assert len(ranges) == steps * per_step and not calls
             covered = sorted(ranges[:per_step])
             assert covered[0][0] == sw.lo and covered[-1][1] == sw.lo + sw.nlocal
@@ -112,16 +114,20 @@ def _sharded_worker(rank, world, port, dims, R, steps, halo_steps, overlap, out)
 
 
 @pytest.mark.timeout(180)
-@pytest.mark.parametrize("world,dims,R,steps,halo_steps,overlap", [
-    (2, (11, 9, 12), 1, 3, 1, False), (3, (13, 10), 2, 4, 1, False), (2, (4, 6, 8), 2, 2, 1, False),
-    (2, (11, 9, 12), 1, 5, 2, False),      # two steps per exchange, the last round one step
-    (3, (19, 10), 2, 6, 3, False),         # three ranks, ghost zones of 6 rows, two rounds
-    (2, (12, 6, 8), 1, 4, 4, False),       # one exchange for the whole run
-    (3, (17, 9, 12), 1, 3, 1, True),       # exchange overlapped with the sweep of the inner planes
-    (2, (14, 6, 8), 2, 2, 1, True),
-    (2, (11, 9, 12), 1, 4, 2, True),       # overlap asked for, but two steps per exchange: not used
+@pytest.mark.parametrize("world,dims,R,steps,halo_steps,overlap,periodic", [
+    (2, (11, 9, 12), 1, 3, 1, False, False), (3, (13, 10), 2, 4, 1, False, False), (2, (4, 6, 8), 2, 2, 1, False, False),
+    (2, (11, 9, 12), 1, 5, 2, False, False),      # two steps per exchange, the last round one step
+    (3, (19, 10), 2, 6, 3, False, False),         # three ranks, ghost zones of 6 rows, two rounds
+    (2, (12, 6, 8), 1, 4, 4, False, False),       # one exchange for the whole run
+    (3, (17, 9, 12), 1, 3, 1, True, False),       # exchange overlapped with the sweep of the inner planes
+    (2, (14, 6, 8), 2, 2, 1, True, False),
+    (2, (11, 9, 12), 1, 4, 2, True, False),       # overlap asked for, but two steps per exchange: not used
+    (3, (13, 9, 12), 1, 3, 1, False, True),       # periodic: the ranks form a ring, ghosts on both sides of every rank
+    (2, (11, 10), 2, 5, 2, False, True),          # a ring of two: both neighbours are the same peer
+    (2, (12, 6, 8), 1, 4, 4, False, True),
+    (3, (17, 9, 12), 1, 3, 1, True, True),        # ... with the exchange overlapped
 ])
-def test_sharded_sweep_equals_the_single_grid_sweep(world, dims, R, steps, halo_steps, overlap):
+def test_sharded_sweep_equals_the_single_grid_sweep(world, dims, R, steps, halo_steps, overlap, periodic):
     """Halo exchange + local sweeps on 2-3 gloo ranks reproduce the sweep of the whole grid
     bit for bit (every point sees the same neighbours in the same order), also when the
     ghost zones are deep enough for several steps between two exchanges."""
@@ -131,12 +137,12 @@ def test_sharded_sweep_equals_the_single_grid_sweep(world, dims, R, steps, halo_
     port = _free_port()
     with mp.Manager() as mgr:
         out = mgr.dict()
-        mp.spawn(_sharded_worker, args=(world, port, dims, R, steps, halo_steps, overlap, out), nprocs=world,
-                 join=True)
+        mp.spawn(_sharded_worker, args=(world, port, dims, R, steps, halo_steps, overlap, periodic, out),
+                 nprocs=world, join=True)
         parts = dict(out)
     w = wl.random_box_weights(len(dims), R, 5)
     a = wl.normal_field(dims, 6)
-    want = oracle.apply(a, w, oracle.ZERO, steps)
+    want = oracle.apply(a, w, oracle.PERIODIC if periodic else oracle.ZERO, steps)
     got = np.empty_like(want)
     for r in range(world):
         z0, z1, block, calls = parts[r]

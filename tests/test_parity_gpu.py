@@ -617,19 +617,20 @@ def test_sharded_sweep_single_rank_on_gpu(halo_steps):
     assert np.max(np.abs(got - want)) <= wl.tolerance(w, 1.0, 5)
 
 
+@pytest.mark.parametrize("boundary", [b.ZERO, b.PERIODIC])
 @pytest.mark.parametrize("world,halo_steps,steps", [(2, 1, 3), (3, 2, 5), (4, 2, 4), (2, 3, 6)])
-def test_sharded_slabs_with_real_kernels_ranks_emulated_in_one_process(world, halo_steps, steps):
+def test_sharded_slabs_with_real_kernels_ranks_emulated_in_one_process(world, halo_steps, steps, boundary):
     """The slabs of 2-4 ranks swept by the real kernels on one GPU, one after the other, with
     the halo exchange done by direct copies between the slabs (no process group, nothing
     waits on anything): ghost depth, edge ranks without outer ghosts and several steps per
-    exchange give the sweep of the whole grid."""
+    exchange give the sweep of the whole grid.  Under the periodic boundary the ranks form a ring."""
     from paper_2608_21157_b200.sharded import ShardedSweep
     dims = (45, 40, 128)
     R = 1
     w = wl.star_weights(3, R, 0.4, [0.1])
     a = wl.uniform_field(dims, 0.0, 1.0, 96)
     g = torch.from_numpy(a).cuda()
-    sws = [ShardedSweep(dims, R, b.STAR, w, rank=r, world=world, dist=object(), halo_steps=halo_steps)
+    sws = [ShardedSweep(dims, R, b.STAR, w, boundary, rank=r, world=world, dist=object(), halo_steps=halo_steps)
            for r in range(world)]
     try:
         cur = [sw.scatter(g) for sw in sws]
@@ -640,15 +641,17 @@ def test_sharded_slabs_with_real_kernels_ranks_emulated_in_one_process(world, ha
             n = min(halo_steps, steps - done)
             own = [sw.interior(c) for sw, c in zip(sws, cur)]
             for r, sw in enumerate(sws):
-                if r > 0:
-                    cur[r][:sw.lo].copy_(own[r - 1][-D:])
-                if r < world - 1:
-                    cur[r][sw.lo + sw.nlocal:].copy_(own[r + 1][:D])
+                assert (sw.lower is None) == (boundary == b.ZERO and r == 0)
+                assert (sw.upper is None) == (boundary == b.ZERO and r == world - 1)
+                if sw.lower is not None:
+                    cur[r][:sw.lo].copy_(own[sw.lower][-D:])
+                if sw.upper is not None:
+                    cur[r][sw.lo + sw.nlocal:].copy_(own[sw.upper][:D])
             for r, sw in enumerate(sws):
                 if sw.overlap:                          # one step per exchange: inner planes, then the edges
                     lo, nl = sw.lo, sw.nlocal
-                    inner0 = lo + (R if r > 0 else 0)
-                    inner1 = lo + nl - (R if r < world - 1 else 0)
+                    inner0 = lo + (R if sw.lower is not None else 0)
+                    inner1 = lo + nl - (R if sw.upper is not None else 0)
                     sw._local_apply_planes(cur[r], other[r], inner0, inner1)
                     if inner0 > lo:
                         sw._local_apply_planes(cur[r], other[r], lo, inner0)
@@ -663,7 +666,7 @@ def test_sharded_slabs_with_real_kernels_ranks_emulated_in_one_process(world, ha
     finally:
         for sw in sws:
             sw.close()
-    want = oracle.apply(a, w, b.ZERO, steps)
+    want = oracle.apply(a, w, boundary, steps)
     assert got.shape == want.shape
     assert np.max(np.abs(got - want)) <= wl.tolerance(w, 1.0, steps)
 
