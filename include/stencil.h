@@ -175,21 +175,25 @@ STENCIL_API int stencil_apply_f64(stencil_plan_t plan, const double* in, double*
                                   void* stream);
 
 /*
- * stencil_apply_planes — one sweep restricted to the output planes
- * [z_begin, z_end) of a 3D grid:  out[z] = S(in)[z] for those planes, the rest
- * of `out` is left untouched.  All of `in` the planes depend on (R planes on
- * either side, inside the grid) must be valid.  Lets a caller that owns a slab
- * of a larger grid sweep the planes that do not depend on its neighbours'
- * data while that data is still on its way, and the others afterwards.  The
- * paper has no counterpart (it runs on one GPU).
+ * stencil_apply_planes / stencil_apply_planes_f64 — one sweep restricted to the
+ * output planes [z_begin, z_end) of a 3D grid (rows [z_begin, z_end) of a 2D
+ * grid: the range always runs along the slowest axis):  out[z] = S(in)[z] for
+ * those planes, the rest of `out` is left untouched.  All of `in` the planes
+ * depend on (R planes on either side, inside the grid) must be valid.  Lets a
+ * caller that owns a slab of a larger grid sweep the planes that do not depend
+ * on its neighbours' data while that data is still on its way, and the others
+ * afterwards.  The paper has no counterpart (it runs on one GPU).
  *
- * fp32 plans on the tiled 3D kernel with a zero boundary and nx a multiple of 4
- * only; STENCIL_ERR_UNSUPPORTED otherwise (2D, FP64, periodic, generic
- * variant).  Pointers and errors as for stencil_apply; INVALID also for
- * z_begin < 0, z_end > nz or z_begin >= z_end.  Enqueue only.
+ * Plans on the tiled kernels with a zero boundary and rows that are a multiple
+ * of 16 bytes only; STENCIL_ERR_UNSUPPORTED otherwise (periodic, generic
+ * variant, other row lengths).  Pointers and errors as for stencil_apply
+ * (stencil_apply_f64); INVALID also for z_begin < 0, z_end beyond the slowest
+ * extent or z_begin >= z_end.  Enqueue only.
  */
 STENCIL_API int stencil_apply_planes(stencil_plan_t plan, const float* in, float* out, int64_t z_begin,
                                      int64_t z_end, void* stream);
+STENCIL_API int stencil_apply_planes_f64(stencil_plan_t plan, const double* in, double* out, int64_t z_begin,
+                                         int64_t z_end, void* stream);
 
 /*
  * stencil_apply_host — the same operation on HOST buffers: copies `in_host`

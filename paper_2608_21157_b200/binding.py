@@ -31,7 +31,8 @@ VARIANT_AUTO, VARIANT_GENERIC, VARIANT_STREAM, VARIANT_FUSED = 0, 1, 2, 3
 #: every symbol include/stencil.h declares
 EXPORTS = (
     "stencil_plan", "stencil_apply", "stencil_plan_f64", "stencil_apply_f64",
-    "stencil_apply_host", "stencil_apply_static", "stencil_apply_planes", "stencil_destroy",
+    "stencil_apply_host", "stencil_apply_static", "stencil_apply_planes", "stencil_apply_planes_f64",
+    "stencil_destroy",
     "stencil_status_string", "stencil_variant_name", "stencil_query_status",
     "stencil_plan_set", "stencil_plan_get",
 )
@@ -70,6 +71,8 @@ def load() -> ctypes.CDLL:
     lib.stencil_apply_host.argtypes = [vp, vp, vp, ctypes.c_int, vp]
     lib.stencil_apply_planes.restype = ctypes.c_int
     lib.stencil_apply_planes.argtypes = [vp, vp, vp, ctypes.c_int64, ctypes.c_int64, vp]
+    lib.stencil_apply_planes_f64.restype = ctypes.c_int
+    lib.stencil_apply_planes_f64.argtypes = [vp, vp, vp, ctypes.c_int64, ctypes.c_int64, vp]
     lib.stencil_apply_static.restype = ctypes.c_int
     lib.stencil_apply_static.argtypes = [vp, vp, vp, ctypes.c_int, vp]
     lib.stencil_destroy.restype = ctypes.c_int
@@ -140,9 +143,15 @@ def stencil_apply_host(plan, in_ptr: int, out_ptr: int, steps: int, stream: int 
 
 
 def stencil_apply_planes(plan, in_ptr: int, out_ptr: int, z_begin: int, z_end: int, stream: int = 0) -> int:
-    """One sweep restricted to the output planes [z_begin, z_end) of a 3D grid."""
+    """One sweep restricted to the output planes [z_begin, z_end) of a 3D grid (rows of a 2D grid)."""
     return load().stencil_apply_planes(plan, ctypes.c_void_p(in_ptr), ctypes.c_void_p(out_ptr), int(z_begin),
                                        int(z_end), ctypes.c_void_p(stream))
+
+
+def stencil_apply_planes_f64(plan, in_ptr: int, out_ptr: int, z_begin: int, z_end: int, stream: int = 0) -> int:
+    """The same for an FP64 plan."""
+    return load().stencil_apply_planes_f64(plan, ctypes.c_void_p(in_ptr), ctypes.c_void_p(out_ptr), int(z_begin),
+                                           int(z_end), ctypes.c_void_p(stream))
 
 
 def stencil_apply_static(plan, in_ptr: int, out_ptr: int, steps: int, stream: int = 0) -> int:
@@ -234,9 +243,10 @@ class Plan:
             raise StencilError(rc, "stencil_apply_f64" if self.f64 else "stencil_apply")
 
     def apply_planes(self, src, dst, z_begin: int, z_end: int, stream: int = 0) -> None:
-        rc = stencil_apply_planes(self._h, self._ptr(src), self._ptr(dst), z_begin, z_end, stream)
+        fn = stencil_apply_planes_f64 if self.f64 else stencil_apply_planes
+        rc = fn(self._h, self._ptr(src), self._ptr(dst), z_begin, z_end, stream)
         if rc != OK:
-            raise StencilError(rc, "stencil_apply_planes")
+            raise StencilError(rc, "stencil_apply_planes_f64" if self.f64 else "stencil_apply_planes")
 
     def apply_static(self, src, dst, steps: int = 1, stream: int = 0) -> None:
         rc = stencil_apply_static(self._h, self._ptr(src), self._ptr(dst), steps, stream)

@@ -30,6 +30,7 @@ struct Rows2DGeom {
     int nchunks;
     int stages;                 // batches in a warp's ring
     int in_off_x, in_off_y;     // added to the TMA coordinates (padded input of a periodic grid), else 0
+    int y_begin, y_end;         // output rows of this launch (the whole grid: 0, ny)
 };
 
 template <int YB, int PXV = kStreamPX>     // PXV: row pitch of a batch (the strip plus its halo columns)
@@ -72,8 +73,8 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
     const int strip = unit % g.strips;                   // neighbouring strips run side by side (shared halo in L2)
     const int chunk = unit / g.strips;
     const int x0 = strip * kStreamTX;
-    const int y0 = chunk * g.chunk_y;
-    const int y1 = min(y0 + g.chunk_y, g.ny);
+    const int y0 = g.y_begin + chunk * g.chunk_y;
+    const int y1 = min(y0 + g.chunk_y, g.y_end);
     const int nrows = (y1 - y0) + 2 * R;                 // input rows y0-R .. y1-1+R
     const int nbatches = (nrows + YB - 1) / YB;
     const int ystart = y0 - R;

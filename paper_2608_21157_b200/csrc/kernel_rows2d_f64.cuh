@@ -61,8 +61,8 @@ stencil_rows2d_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
     const int strip = unit % g.strips;
     const int chunk = unit / g.strips;
     const int x0 = strip * kStrip64;
-    const int y0 = chunk * g.chunk_y;
-    const int y1 = min(y0 + g.chunk_y, g.ny);
+    const int y0 = g.y_begin + chunk * g.chunk_y;
+    const int y1 = min(y0 + g.chunk_y, g.y_end);
     const int nrows = (y1 - y0) + 2 * R;
     const int nbatches = (nrows + YB - 1) / YB;
     const int ystart = y0 - R;

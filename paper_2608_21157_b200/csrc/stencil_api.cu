@@ -915,8 +915,11 @@ int short_chunk_2d(const stencil_plan_s* p, int YB) {
     return std::max(1, nbatch * YB - 2 * R);
 }
 
-// 2D grids: one warp per (128-column strip, chunk of rows).
-int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
+// 2D grids: one warp per (128-column strip, chunk of rows).  dst[y_begin, y_end) = one sweep of
+// src; the whole grid when y_end <= y_begin.
+int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st, int y_begin = 0, int y_end = 0) {
+    if (y_end <= y_begin) { y_begin = 0; y_end = p->ny; }
+    const int span = y_end - y_begin;
     const Rows2DConfig* cfg = p->rows2d_cfg;
     const CUtensorMap* map = nullptr;
     const bool periodic = p->boundary == STENCIL_PERIODIC;
@@ -962,15 +965,16 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
         const int R = p->radius;
         const int slots = 2 * sm_count() * cfg->NW;
         const int nch_max = std::max(1, slots / g.strips);
-        const int chunk_min = (p->ny + nch_max - 1) / nch_max;
+        const int chunk_min = (span + nch_max - 1) / nch_max;
         int nbatch = std::max(1, (chunk_min + 2 * R + cfg->YB - 1) / cfg->YB);
         while (nbatch * cfg->YB - 2 * R < 1) ++nbatch;
         chunk = nbatch * cfg->YB - 2 * R;
         chunk = std::min(chunk, short_chunk_2d(p, cfg->YB));
     }
-    chunk = std::max(1, std::min(chunk, p->ny));
+    chunk = std::max(1, std::min(chunk, span));
     g.chunk_y = chunk;
-    g.nchunks = (p->ny + chunk - 1) / chunk;
+    g.nchunks = (span + chunk - 1) / chunk;
+    g.y_begin = y_begin; g.y_end = y_end;
     const int64_t units = (int64_t)g.strips * g.nchunks;
     const int64_t grid64 = (units + cfg->NW - 1) / cfg->NW;
     if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
@@ -1460,7 +1464,11 @@ int launch_rows2d_fused64(stencil_plan_s* p, const double* src, double* dst, int
     return STENCIL_OK;
 }
 
-int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStream_t st) {
+// dst = one sweep of src; with begin < end only the output planes (3D) or rows (2D) [begin, end) on the tiled kernels.
+int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStream_t st, int begin = 0, int end = 0) {
+    const int slow = p->ndim == 3 ? p->nz : p->ny;              // extent of the streamed axis
+    if (end <= begin) { begin = 0; end = slow; }
+    const int span = end - begin;
     if (p->variant == STENCIL_VARIANT_STREAM && p->stream64_cfg) {
         const Stream64Config* cfg = p->stream64_cfg;
         const CUtensorMap* map = nullptr;
@@ -1498,7 +1506,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         g.tiles_y = (p->ny + cfg->tile_y - 1) / cfg->tile_y;
         g.stages = stages;
         g.streaming_store = 0;
-        g.z_begin = 0; g.z_end = p->nz;
+        g.z_begin = begin; g.z_end = end;
         g.in_off_x = periodic ? kPadX : 0;
         g.in_off_y = periodic ? p->radius : 0;
         g.in_off_z = periodic ? p->radius : 0;
@@ -1506,8 +1514,8 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         // many short CTAs, as for the bandwidth-bound fp32 sweeps; the wide stars re-read 2R halo
         // planes per chunk, so they get longer chunks (measured on 512^3)
         const int want_chunk = p->radius >= 3 ? 64 : 32;
-        int chunk = p->chunk_z > 0 ? p->chunk_z : (p->nz >= 2 * want_chunk ? want_chunk : p->nz);
-        if (p->chunk_z <= 0 && p->shape == STENCIL_STAR && p->radius == 1 && p->nz >= 16) {
+        int chunk = p->chunk_z > 0 ? p->chunk_z : (span >= 2 * want_chunk ? want_chunk : span);
+        if (p->chunk_z <= 0 && p->shape == STENCIL_STAR && p->radius == 1 && span >= 16) {
             int occ64 = 0;                            // the 7-point star: very short chunks, as in fp32
             {
                 std::lock_guard<std::mutex> lock(g_config_mutex);
@@ -1523,7 +1531,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
                 }
                 occ64 = cfg->occ;
             }
-            chunk = short_chunk_star1(p->nz, (int64_t)g.tiles_x * g.tiles_y, (int64_t)occ64 * sm_count());
+            chunk = short_chunk_star1(span, (int64_t)g.tiles_x * g.tiles_y, (int64_t)occ64 * sm_count());
         }
         if (p->chunk_z <= 0 && (p->radius >= 4 || (p->shape == STENCIL_BOX && p->radius >= 2))) {
             // The radius-4 star is no longer bound by memory alone (25 DFMA and 15 shared-memory
@@ -1535,16 +1543,16 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
             const int64_t tiles = (int64_t)g.tiles_x * g.tiles_y;
             const int64_t slots = 2 * (int64_t)sm_count();
             double best = 1e300;
-            for (int n = 1; n <= std::max(1, p->nz / (4 * p->radius)); ++n) {
-                const int c = (p->nz + n - 1) / n;
-                const int64_t ctas = tiles * ((p->nz + c - 1) / c);
+            for (int n = 1; n <= std::max(1, span / (4 * p->radius)); ++n) {
+                const int c = (span + n - 1) / n;
+                const int64_t ctas = tiles * ((span + c - 1) / c);
                 const double cost = (double)((ctas + slots - 1) / slots) * (c + 2 * p->radius + 4.0);
                 if (cost < best * 0.999) { best = cost; chunk = c; }
             }
         }
-        chunk = std::max(1, std::min(chunk, p->nz));
+        chunk = std::max(1, std::min(chunk, span));
         g.chunk_z = chunk;
-        const int64_t grid64 = (int64_t)g.tiles_x * g.tiles_y * ((p->nz + chunk - 1) / chunk);
+        const int64_t grid64 = (int64_t)g.tiles_x * g.tiles_y * ((span + chunk - 1) / chunk);
         if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
         if (cfg->launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
         p->launches++;
@@ -1592,15 +1600,16 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
             const int R = p->radius;
             const int slots = 2 * sm_count() * cfg->NW;
             const int nch_max = std::max(1, slots / g.strips);
-            const int chunk_min = (p->ny + nch_max - 1) / nch_max;
+            const int chunk_min = (span + nch_max - 1) / nch_max;
             int nbatch = std::max(1, (chunk_min + 2 * R + cfg->YB - 1) / cfg->YB);
             while (nbatch * cfg->YB - 2 * R < 1) ++nbatch;
             chunk = nbatch * cfg->YB - 2 * R;
             chunk = std::min(chunk, short_chunk_2d(p, cfg->YB));
         }
-        chunk = std::max(1, std::min(chunk, p->ny));
+        chunk = std::max(1, std::min(chunk, span));
         g.chunk_y = chunk;
-        g.nchunks = (p->ny + chunk - 1) / chunk;
+        g.nchunks = (span + chunk - 1) / chunk;
+        g.y_begin = begin; g.y_end = end;
         const int64_t units = (int64_t)g.strips * g.nchunks;
         const int64_t grid64 = (units + cfg->NW - 1) / cfg->NW;
         if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
@@ -2066,15 +2075,36 @@ int stencil_apply_planes(stencil_plan_t p, const float* in, float* out, int64_t 
     if ((a | b) & 15u) return STENCIL_ERR_INVALID;
     const uintptr_t bytes = (uintptr_t)p->npoints * sizeof(float);
     if (a < b + bytes && b < a + bytes) return STENCIL_ERR_INVALID;
-    if (z_begin < 0 || z_end > p->nz || z_begin >= z_end) return STENCIL_ERR_INVALID;
-    if (p->variant != STENCIL_VARIANT_STREAM || p->ndim != 3 || p->boundary != STENCIL_ZERO || p->nx % 4 != 0)
+    const int slow = p->ndim == 3 ? p->nz : p->ny;
+    if (z_begin < 0 || z_end > slow || z_begin >= z_end) return STENCIL_ERR_INVALID;
+    if (p->variant != STENCIL_VARIANT_STREAM || p->boundary != STENCIL_ZERO || p->nx % 4 != 0)
         return STENCIL_ERR_UNSUPPORTED;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const int rc = ensure_device_state(p);
     if (rc != STENCIL_OK) return rc;
     p->last_stream = st;
     p->used = true;
-    return launch_stream(p, in, out, st, (int)z_begin, (int)z_end);
+    return p->ndim == 3 ? launch_stream(p, in, out, st, (int)z_begin, (int)z_end)
+                        : launch_rows2d(p, in, out, st, (int)z_begin, (int)z_end);
+}
+
+int stencil_apply_planes_f64(stencil_plan_t p, const double* in, double* out, int64_t z_begin, int64_t z_end,
+                             void* stream) {
+    if (!valid_plan(p) || !p->f64 || !in || !out) return STENCIL_ERR_INVALID;
+    const uintptr_t a = reinterpret_cast<uintptr_t>(in), b = reinterpret_cast<uintptr_t>(out);
+    if ((a | b) & 15u) return STENCIL_ERR_INVALID;
+    const uintptr_t bytes = (uintptr_t)p->npoints * sizeof(double);
+    if (a < b + bytes && b < a + bytes) return STENCIL_ERR_INVALID;
+    const int slow = p->ndim == 3 ? p->nz : p->ny;
+    if (z_begin < 0 || z_end > slow || z_begin >= z_end) return STENCIL_ERR_INVALID;
+    if (p->variant != STENCIL_VARIANT_STREAM || p->boundary != STENCIL_ZERO || p->nx % 2 != 0)
+        return STENCIL_ERR_UNSUPPORTED;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int rc = ensure_device_state(p);
+    if (rc != STENCIL_OK) return rc;
+    p->last_stream = st;
+    p->used = true;
+    return launch_sweep_f64(p, in, out, st, (int)z_begin, (int)z_end);
 }
 
 int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps, void* stream) {

@@ -14,8 +14,8 @@ rank's own planes, which are exact.  ``G = 1`` exchanges before every step;
 run its two-step fused passes.
 
 With ``G = 1`` a round also overlaps the exchange with compute where the local
-sweep can be restricted to a range of planes (``stencil_apply_planes``: 3D fp32,
-zero boundary): the sends and receives are started, the planes that read no
+sweep can be restricted to a range of planes (``stencil_apply_planes``: tiled
+kernels, zero boundary, 16-byte rows): the sends and receives are started, the planes that read no
 ghost plane are swept meanwhile, and the R planes next to each neighbour follow
 once the ghost planes have arrived.
 
@@ -105,8 +105,8 @@ class ShardedSweep:
             def local_apply(src, dst, steps):
                 self._plan.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
 
-            ranged = (len(self.dims) == 3 and self._plan.variant == "stream" and not self._plan.f64
-                      and self.dims[-1] % 4 == 0 and boundary == ZERO)
+            ranged = (self._plan.variant == "stream" and boundary == ZERO
+                      and self.dims[-1] % (2 if self._plan.f64 else 4) == 0)
             if ranged and local_apply_planes is None:
                 def local_apply_planes(src, dst, z_begin, z_end):
                     self._plan.apply_planes(src, dst, z_begin, z_end, torch.cuda.current_stream().cuda_stream)

@@ -672,15 +672,20 @@ def test_sharded_slabs_with_real_kernels_ranks_emulated_in_one_process(world, ha
 
 
 @pytest.mark.parametrize("R,box", [(1, False), (4, False), (1, True), (2, True)])
-def test_apply_planes_sweeps_exactly_the_requested_planes(R, box):
-    dims = (37, 45, 132)
-    w = wl.random_box_weights(3, R, 97) if box else wl.random_star_weights(3, R, 97)
-    a = wl.normal_field(dims, 98)
+@pytest.mark.parametrize("dims", [(37, 45, 132), (37, 260)])
+@pytest.mark.parametrize("f64", [False, True])
+def test_apply_planes_sweeps_exactly_the_requested_planes(R, box, dims, f64):
+    """Ranges along the slowest axis: planes of a 3D grid, rows of a 2D grid, fp32 and FP64."""
+    nd = len(dims)
+    dt = np.float64 if f64 else np.float32
+    w = (wl.random_box_weights if box else wl.random_star_weights)(nd, R, 97, dt)
+    a = wl.normal_field(dims, 98, dt)
     want = oracle.apply(a, w, b.ZERO, 1)
     tol = wl.tolerance(w, float(np.abs(a).max()), 1)
     src = torch.from_numpy(a).cuda()
     st = torch.cuda.current_stream().cuda_stream
     with b.Plan(dims, R, b.BOX if box else b.STAR, w, b.ZERO) as p:
+        assert p.variant == "stream"
         dst = torch.full_like(src, float("nan"))
         p.apply_planes(src, dst, 5, 19, st)
         torch.cuda.synchronize()
@@ -700,13 +705,54 @@ def test_apply_planes_sweeps_exactly_the_requested_planes(R, box):
         with pytest.raises(b.StencilError) as e:
             p.apply_planes(src, torch.empty_like(src), 0, 4, st)
         assert e.value.status == b.ERR_UNSUPPORTED
-    a2 = wl.normal_field((40, 64), 99)
-    w2 = wl.random_star_weights(2, 1, 97)
-    with b.Plan((40, 64), 1, b.STAR, w2, b.ZERO) as p:
-        s2 = torch.from_numpy(a2).cuda()
+    with b.Plan(dims, R, b.BOX if box else b.STAR, w, b.ZERO, variant=b.VARIANT_GENERIC) as p:
         with pytest.raises(b.StencilError) as e:
-            p.apply_planes(s2, torch.empty_like(s2), 0, 1, st)
+            p.apply_planes(src, torch.empty_like(src), 0, 4, st)
         assert e.value.status == b.ERR_UNSUPPORTED
+    if f64:                                             # the fp32 entry point refuses an FP64 plan and vice versa
+        with b.Plan(dims, R, b.BOX if box else b.STAR, w, b.ZERO) as p:
+            assert b.stencil_apply_planes(p._h, src.data_ptr(), dst.data_ptr(), 0, 4, st) == b.ERR_INVALID
+
+
+@pytest.mark.parametrize("dims,f64", [((45, 260), False), ((45, 40, 64), True), ((45, 130), True)])
+def test_sharded_overlap_on_2d_and_fp64_slabs(dims, f64):
+    """The exchange/compute overlap of the slab decomposition (ranged sweeps) beyond 3D fp32: the slabs of
+    three emulated ranks, one step per exchange, exchange by direct copies."""
+    from paper_2608_21157_b200.sharded import ShardedSweep
+    world, steps, R = 3, 3, 1
+    dt = np.float64 if f64 else np.float32
+    w = wl.random_star_weights(len(dims), R, 101, dt)
+    a = wl.normal_field(dims, 102, dt)
+    g = torch.from_numpy(a).cuda()
+    sws = [ShardedSweep(dims, R, b.STAR, w, rank=r, world=world, dist=object()) for r in range(world)]
+    try:
+        assert all(sw.overlap for sw in sws)
+        cur = [sw.scatter(g) for sw in sws]
+        other = [torch.empty_like(c) for c in cur]
+        for _ in range(steps):
+            own = [sw.interior(c) for sw, c in zip(sws, cur)]
+            for r, sw in enumerate(sws):
+                if sw.lower is not None:
+                    cur[r][:sw.lo].copy_(own[sw.lower][-R:])
+                if sw.upper is not None:
+                    cur[r][sw.lo + sw.nlocal:].copy_(own[sw.upper][:R])
+            for r, sw in enumerate(sws):
+                lo, nl = sw.lo, sw.nlocal
+                inner0 = lo + (R if sw.lower is not None else 0)
+                inner1 = lo + nl - (R if sw.upper is not None else 0)
+                sw._local_apply_planes(cur[r], other[r], inner0, inner1)
+                if inner0 > lo:
+                    sw._local_apply_planes(cur[r], other[r], lo, inner0)
+                if inner1 < lo + nl:
+                    sw._local_apply_planes(cur[r], other[r], inner1, lo + nl)
+            cur, other = other, cur
+        torch.cuda.synchronize()
+        got = torch.cat([sw.interior(c) for sw, c in zip(sws, cur)]).cpu().numpy()
+    finally:
+        for sw in sws:
+            sw.close()
+    want = oracle.apply(a, w, b.ZERO, steps)
+    assert np.max(np.abs(got - want)) <= wl.tolerance(w, float(np.abs(a).max()), steps)
 
 
 # --------------------------------------------------------------------- FP64 --
