@@ -947,6 +947,45 @@ def test_grid_with_more_than_2_to_the_31_points():
     torch.cuda.empty_cache()
 
 
+def test_periodic_fused_pass_on_a_grid_with_more_than_2_to_the_31_points():
+    """The same grid under the periodic boundary, two steps in one fused pass (three 384-wide regions
+    per row) plus the two shell kernels: sampled output planes, among them the wrapped ones at both
+    ends, against the oracle run on the 5 input planes around each (the centre plane of such a block
+    does not depend on how the block ends in z)."""
+    nz, ny, nx = 2100, 1024, 1024
+    R, steps = 1, 2
+    w = wl.random_star_weights(3, R, 103)
+
+    def field(zs, xp):
+        z = zs.reshape(-1, 1, 1)
+        y = xp.arange(ny).reshape(1, -1, 1)
+        x = xp.arange(nx).reshape(1, 1, -1)
+        return (((x * 3 + y * 5 + z * 7) % 17) - 8)
+
+    dev = torch.device("cuda:0")
+    src = torch.empty((nz, ny, nx), dtype=torch.float32, device=dev)
+    for z0 in range(0, nz, 100):
+        z1 = min(z0 + 100, nz)
+        src[z0:z1] = field(torch.arange(z0, z1), torch).to(dev).float() / 8.0
+    dst = torch.empty_like(src)
+    with b.Plan((nz, ny, nx), R, b.STAR, w, b.PERIODIC) as p:
+        assert p.variant == "stream" and p.get(b.KEY_FUSE_STEPS) == 2
+        p.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
+        assert p.query_status() == b.OK
+        assert p.launches == 3
+    torch.cuda.synchronize()
+    tol = wl.tolerance(w, 1.0, steps)
+    H = steps * R
+    for zc in (0, 1, 1049, nz - 2, nz - 1):
+        zs = np.arange(zc - H, zc + H + 1) % nz
+        sub = (field(zs, np) / 8.0).astype(np.float32)
+        want = oracle.apply(sub, w, b.PERIODIC, steps)[H]
+        got = dst[zc].cpu().numpy()
+        assert float(np.max(np.abs(got - want))) <= tol, f"plane {zc}"
+    del src, dst
+    torch.cuda.empty_cache()
+
+
 def test_2d_grid_with_more_than_2_to_the_31_points():
     """The same for the 2D row-streaming kernel: 46400 x 46400 = 2.15e9 points."""
     ny = nx = 46400
