@@ -541,7 +541,7 @@ def main():
     ap.add_argument("--stages", type=int, default=None)
     ap.add_argument("--fuse-steps", dest="fuse_steps", type=int, default=None)
     ap.add_argument("--streaming-store", dest="streaming_store", type=int, default=None)
-    ap.add_argument("--also", default="cfg1,cfg3,cfg4,cfg5,cfg5L,paper2d,paper2d_f64,heat2d", help="other workloads summarised in all_configs")
+    ap.add_argument("--also", default="cfg1,cfg3,cfg4,cfg5,cfg5L,cfg5L_periodic,paper2d,paper2d_f64,heat2d", help="other workloads summarised in all_configs")
     ap.add_argument("--also-steps", dest="also_steps", type=int, default=20)
     ap.add_argument("--no-all-configs", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
