@@ -60,14 +60,20 @@ __device__ __forceinline__ void consumer_barrier(int nthreads) {
     asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
 }
 
-// SPEC: the launch advances exactly T levels and one region spans a whole row of exactly
+// MODE 1 (SPEC): the launch advances exactly T levels and one region spans a whole row of exactly
 // 128*XW points.  The level count, the row pitch and the x bounds are then compile-time
 // constants (the common case of the iterated apply on a 256-wide grid).
-template <int R, int T, int K, int XW, int NWY, bool SPEC = false>
+// MODE 2 (SPEC and WRAP): the same, on a grid that is periodic along x and z (the pass of a
+// periodic grid; its y faces are put right afterwards).  z wraps in the plane coordinate of the
+// TMA loads, since every plane is a load of its own, and no plane counts as outside the grid;
+// x wraps where the first and last warp of a row fetch the cells beyond the row's ends, at every
+// level, from the other end of the same row of the level's plane in shared memory.
+template <int R, int T, int K, int XW, int NWY, int MODE = 0>
 __global__ void __launch_bounds__(XW * NWY * 32, (XW * NWY * 32 <= 256 ? 2 : 1))
 stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restrict__ out,
                      const FusedGeom g, const __grid_constant__ StarWeights<R> sw,
                      int* __restrict__ status) {
+    constexpr bool SPEC = MODE >= 1, WRAP = MODE == 2;
     using S = FusedShape<R, K, XW, NWY>;
     constexpr int TXE = S::TXE;
     constexpr int PW = S::PW;
@@ -143,6 +149,12 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
     const int hl_off = wx > 0 ? ((wx * 128 - 1) / PW) * S::PART_FLOATS + (wx * 128 - R) - ((wx * 128 - 1) / PW) * PW : 0;
     const int hr_off = wx < XW - 1 ? (((wx + 1) * 128) / PW) * S::PART_FLOATS + (wx + 1) * 128 - (((wx + 1) * 128) / PW) * PW : 0;
 
+    // the plane a load fetches: wrapped into the grid under WRAP (nz >= 2*T*R, so one step is enough)
+    auto plane_coord = [&](int zc) { return !WRAP ? zc : (zc < 0 ? zc + g.nz : (zc >= g.nz ? zc - g.nz : zc)); };
+    // the cells beyond the two ends of a row under WRAP: the last R cells of the last part, the first R of the first
+    constexpr int wrap_l_off = (S::NP - 1) * S::PART_FLOATS + PW - R;
+    constexpr int wrap_r_off = 0;
+
     int issued = 0;                                // planes requested so far (thread 0 only)
     if (tid == 0) {
         prefetch_tensormap(&tmap_in);
@@ -153,7 +165,7 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
 #pragma unroll
             for (int part = 0; part < S::NP; ++part)
                 tma_load_3d(smem_addr(ring + (size_t)i * S::SLOT_FLOATS + part * S::PART_FLOATS + R * PW), &tmap_in,
-                            full0 + 8 * i, x0e + part * PW, y0e, pstart + i);
+                            full0 + 8 * i, x0e + part * PW, y0e, plane_coord(pstart + i));
         }
     }
 
@@ -210,6 +222,10 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                                         if (wx > 0) xl = rowb[hl_off + t];
                                         if (wx < XW - 1) xr = rowb[hr_off + t];
                                     }
+                                    if (WRAP) {
+                                        if (wx == 0) xl = rowb[wrap_l_off + t];
+                                        if (wx == XW - 1) xr = rowb[wrap_r_off + t];
+                                    }
                                     const float lft = __shfl_up_sync(0xffffffffu, c4[4 - R + t], 1);
                                     const float rgt = __shfl_down_sync(0xffffffffu, c4[t], 1);
                                     v[t] = lane == 0 ? xl : lft;
@@ -254,8 +270,8 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                         }
                         // the zero boundary holds at every time level: cells outside the grid go
                         // back to zero (nothing to do for regions and planes inside the grid)
-                        if (!warp_all_in || zl < 0 || zl >= g.nz) {
-                            const bool z_in = zl >= 0 && zl < g.nz;
+                        if (!warp_all_in || (!WRAP && (zl < 0 || zl >= g.nz))) {
+                            const bool z_in = WRAP || (zl >= 0 && zl < g.nz);
 #pragma unroll
                             for (int k = 0; k < K; ++k)
                                 if (!(z_in && ((in_mask >> k) & 1u))) e[k] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -292,7 +308,8 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
 #pragma unroll
                             for (int part = 0; part < S::NP; ++part)
                                 tma_load_3d(smem_addr(ring + (size_t)s * S::SLOT_FLOATS + part * S::PART_FLOATS + R * PW),
-                                            &tmap_in, full0 + 8 * s, x0e + part * PW, y0e, pstart + i + nstage);
+                                            &tmap_in, full0 + 8 * s, x0e + part * PW, y0e,
+                                            plane_coord(pstart + i + nstage));
                             issued = i + nstage + 1;
                         }
                     }

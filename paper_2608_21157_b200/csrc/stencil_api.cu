@@ -114,6 +114,7 @@ struct FusedConfig {
     int pw;                                  // width of the TMA boxes a plane is loaded as
     const void* kernel;
     const void* kernel_spec;                 // the instantiation for full passes over rows of exactly txe points
+    const void* kernel_wrap;                 // ... and the one of those that wraps x and z (passes of a periodic grid)
     mutable size_t smem_allowed;             // dynamic shared memory already granted to both kernels
     mutable size_t occ_smem;                 // ... and the occupancy measured at this size
     mutable int occ;
@@ -121,6 +122,8 @@ struct FusedConfig {
     cudaError_t (*launch)(const struct stencil_plan_s*, const CUtensorMap&, float*, const FusedGeom&,
                           int grid, size_t smem, cudaStream_t);
     cudaError_t (*launch_spec)(const struct stencil_plan_s*, const CUtensorMap&, float*, const FusedGeom&,
+                               int grid, size_t smem, cudaStream_t);
+    cudaError_t (*launch_wrap)(const struct stencil_plan_s*, const CUtensorMap&, float*, const FusedGeom&,
                                int grid, size_t smem, cudaStream_t);
 };
 
@@ -226,6 +229,7 @@ struct stencil_plan_s {
     float* pad2;                   // second padded-row grid
     int tmap_nx;                   // non-zero while a padded-row sweep runs: the true row length
     int periodic_route;            // knob: 0 = by measured cost, 1 = padded copy, 2 = wrap correction where it fits
+    bool fused_wrap;               // set for one launch_fused call: the pass wraps x and z in the kernel
     bool src_padded;               // set while an iterated periodic apply runs: the source of a sweep is
                                    // a padded grid with current halos
     float* host_in;                // N floats each, apply_host staging
@@ -358,12 +362,12 @@ void pack_star(const stencil_plan_s* p, StarWeights<R>& sw) {
     }
 }
 
-template <int R, int T, int K, int XW, int NWY, bool SPEC>
+template <int R, int T, int K, int XW, int NWY, int MODE>
 cudaError_t launch_fused_t(const stencil_plan_s* p, const CUtensorMap& map, float* out, const FusedGeom& g,
                            int grid, size_t smem, cudaStream_t st) {
     StarWeights<R> sw;
     pack_star<R>(p, sw);
-    return launch_kernel(&stencil_fused_kernel<R, T, K, XW, NWY, SPEC>, grid, FusedShape<R, K, XW, NWY>::THREADS,
+    return launch_kernel(&stencil_fused_kernel<R, T, K, XW, NWY, MODE>, grid, FusedShape<R, K, XW, NWY>::THREADS,
                          smem, st, p->chained, map, out, g, sw, p->d_status);
 }
 
@@ -373,11 +377,13 @@ FusedConfig make_fused() {
     FusedConfig c;
     c.radius = R; c.T = T; c.K = K; c.XW = XW; c.NWY = NWY;
     c.txe = S::TXE; c.tye = S::TYE; c.threads = S::THREADS; c.slot_bytes = S::SLOT_BYTES; c.pw = S::PW;
-    c.kernel = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, false>);
-    c.kernel_spec = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, true>);
+    c.kernel = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, 0>);
+    c.kernel_spec = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, 1>);
+    c.kernel_wrap = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, 2>);
     c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
-    c.launch = &launch_fused_t<R, T, K, XW, NWY, false>;
-    c.launch_spec = &launch_fused_t<R, T, K, XW, NWY, true>;
+    c.launch = &launch_fused_t<R, T, K, XW, NWY, 0>;
+    c.launch_spec = &launch_fused_t<R, T, K, XW, NWY, 1>;
+    c.launch_wrap = &launch_fused_t<R, T, K, XW, NWY, 2>;
     return c;
 }
 
@@ -1088,6 +1094,8 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
             if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
                     cudaSuccess ||
                 cudaFuncSetAttribute(cfg->kernel_spec, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                    cudaSuccess ||
+                cudaFuncSetAttribute(cfg->kernel_wrap, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
                     cudaSuccess) {
                 cudaGetLastError();
                 return STENCIL_ERR_CUDA;
@@ -1131,9 +1139,12 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
     const int64_t grid64 = (int64_t)tiles * ((p->nz + chunk - 1) / chunk);
     if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
     // full passes over rows of exactly one region take the instantiation with those facts compiled in
+    // ... and the one that also wraps x and z when the pass belongs to a periodic apply (fused_wrap_ok tells
+    // the caller beforehand that it will)
     const bool spec = nlev == T && p->nx == cfg->txe;
-    if ((spec ? cfg->launch_spec : cfg->launch)(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess)
-        return STENCIL_ERR_CUDA;
+    auto launch = !spec ? cfg->launch : (p->fused_wrap ? cfg->launch_wrap : cfg->launch_spec);
+    if (p->fused_wrap && !spec) return STENCIL_ERR_UNSUPPORTED;
+    if (launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
     p->launches++;
     return STENCIL_OK;
 }
@@ -1790,6 +1801,12 @@ int fused_any(stencil_plan_s* p, const double* src, double* dst, int nlev, cudaS
     return launch_rows2d_fused64(p, src, dst, nlev, st);
 }
 
+// A full 3D pass over rows of exactly one region can wrap x and z inside the fused kernel; only the
+// rows next to the y faces are then left to put right.
+bool fused_wrap_ok(const stencil_plan_s* p, int nlev) {
+    return !p->f64 && p->ndim == 3 && p->fused_cfg && nlev == p->fused_cfg->T && p->nx == p->fused_cfg->txe;
+}
+
 // Iterated periodic apply under temporal blocking: every pass is a fused zero-boundary pass of
 // L <= T steps, right everywhere but within L*R cells of a face, followed by
 // stencil_shell_compose_kernel, which rewrites that shell from the pass's input.
@@ -1806,12 +1823,32 @@ int apply_periodic_fused(stencil_plan_s* p, const T* in, T* out, T* other, int s
         const TapT<double>* taps = nullptr;
         int ntaps = 0, rc;
         if ((rc = composite_taps(p, L, &taps, &ntaps)) != STENCIL_OK) return rc;
+        const bool wrapped = L > 1 && fused_wrap_ok(p, L);
         {
             ScopedGridView view(p, p->nz, p->ny, p->nx, 0, STENCIL_ZERO);
+            p->fused_wrap = wrapped;
             rc = L > 1 ? fused_any(p, src, dst, L, st) : sweep_any(p, src, dst, st);
+            p->fused_wrap = false;
         }
         if (rc != STENCIL_OK) return rc;
-        const int H = L * R, hz = p->ndim == 3 ? H : 0;
+        const int H = L * R;
+        if (wrapped) {
+            // x and z are right already: the 2H rows next to the y faces of every plane remain (the row
+            // kernel with a z shell of depth 0 walks exactly those, wrapping the taps' planes itself)
+            const int xchunks = (g.nx + kShellRowChunk - 1) / kShellRowChunk;
+            const int64_t nrows = (int64_t)g.nz * 2 * H * xchunks;
+            if (ntaps <= kShellTaps && nrows <= 0x7fffffffLL) {
+                stencil_shell_rows_kernel<T><<<(int)nrows, 256, 0, st>>>(src, dst, g, H, 0, taps, ntaps, xchunks);
+                if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
+                p->launches++;
+                done += L;
+                src = dst;
+                continue;
+            }
+            // (an operator with too many composite taps for the row kernel: the whole shell below, which
+            // rewrites the x and z faces with the values they already have)
+        }
+        const int hz = p->ndim == 3 ? H : 0;
         // 3D: whole rows of the shell and the ends of the other rows go to their own kernels (512^3,
         // 7-point star, two steps per pass: 74 us against 124 us for the point-by-point walk).
         // Operators with very many composite taps, shells too deep for the tile, rows too short to
@@ -1913,7 +1950,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->npoints = n;
     p->radius = radius; p->shape = shape; p->boundary = boundary;
     p->device = -1;
-    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0; p->src_padded = false; p->periodic_route = 0;
+    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0; p->src_padded = false; p->fused_wrap = false; p->periodic_route = 0;
     for (int l = 0; l <= kMaxFuseLevels; ++l) p->d_ctaps[l] = nullptr;
     p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr; p->fused2d64_cfg = nullptr;
     p->host_in = nullptr; p->host_out = nullptr;
