@@ -58,6 +58,54 @@ def check(dims, R, shape, weights, boundary, a, steps=1, **kw):
     return used
 
 
+# ------------------------------------------------------- randomized requests --
+def _random_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < n:
+        ndim = int(rng.integers(2, 4))
+        R = int(rng.choice([1, 1, 1, 2, 2, 3, 4, 5, 6, 8]))
+        box = bool(rng.integers(0, 2))
+        if box and ndim == 3 and R > 2:
+            R = int(rng.integers(1, 3))                 # keep the oracle's tap count small
+        if box and R > 4:
+            R = 4
+        f64 = bool(rng.integers(0, 3) == 0)
+        periodic = bool(rng.integers(0, 2))
+        steps = int(rng.choice([1, 1, 2, 3, 5, 8]))
+        # the fastest axis: mostly 16-byte rows of the widths the tiled and fused kernels distinguish, some odd ones
+        nx = int(rng.choice([8, 64, 128, 132, 200, 256, 260, 384, 388, 512, 520, 1000, 61, 130, 255]))
+        if ndim == 2:
+            ny = int(rng.integers(1, 300))
+            dims = (ny, nx)
+        else:
+            budget = 400_000 // nx
+            ny = int(rng.integers(1, max(2, min(60, budget))))
+            nz = int(rng.integers(1, max(2, min(60, budget // ny + 1))))
+            dims = (nz, ny, nx)
+        taps = (2 * R + 1) ** ndim if box else 2 * ndim * R + 1
+        if int(np.prod(dims)) * taps * steps > 60_000_000:
+            continue
+        cases.append((dims, R, box, periodic, steps, f64))
+    return cases
+
+
+@pytest.mark.parametrize("dims,R,box,periodic,steps,f64", _random_cases(90, 20261125))
+def test_randomized_requests_match_oracle(dims, R, box, periodic, steps, f64):
+    """Seeded random requests through the default route of the library (whatever kernel, fusion
+    depth and periodic route it picks for them), every point against the oracle."""
+    dt = np.float64 if f64 else np.float32
+    nd = len(dims)
+    w = (wl.random_box_weights if box else wl.random_star_weights)(nd, R, 7 + R, dt)
+    a = wl.normal_field(dims, 11 + steps, dt)
+    boundary = b.PERIODIC if periodic else b.ZERO
+    got, used = gpu_sweep(dims, R, b.BOX if box else b.STAR, w, boundary, a, steps)
+    want = oracle.apply(a, w, boundary, steps)
+    tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+    err = float(np.max(np.abs(got.astype(np.float64) - want.astype(np.float64))))
+    assert err <= tol, f"{used}: {err:.3e} > {tol:.3e} dims={dims} R={R} box={box} periodic={periodic} steps={steps} f64={f64}"
+
+
 # ------------------------------------------------------------------ generic --
 GENERIC_CASES = [
     # dims, R, star?, boundary
