@@ -939,8 +939,10 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
         rc = get_tensor_map(p, cfg, cfg->px, cfg->YB, src, &map);
     }
     if (rc != STENCIL_OK) return rc;
-    const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
-    const size_t smem = (size_t)cfg->NW * stages * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8;
+    int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
+    auto smem_for = [&](int s_) { return (size_t)cfg->NW * s_ * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8; };
+    while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
+    const size_t smem = smem_for(stages);
     if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
@@ -998,8 +1000,10 @@ int launch_rows2d_fused(stencil_plan_s* p, const float* src, float* dst, int nle
     if (rc != STENCIL_OK) return rc;
     // two batches per warp: the small ring lets three CTAs share an SM (measured on 10240^2: 2082 G
     // updates/s against 1671 with three batches and 1214 with four)
-    const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 2;
-    const size_t smem = (size_t)cfg->NW * stages * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8;
+    int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 2;
+    auto smem_for = [&](int s_) { return (size_t)cfg->NW * s_ * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8; };
+    while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
+    const size_t smem = smem_for(stages);
     if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
     int dev = -1, occ = 1;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
@@ -1422,8 +1426,10 @@ int launch_rows2d_fused64(stencil_plan_s* p, const double* src, double* dst, int
     const CUtensorMap* map = nullptr;
     int rc = get_tensor_map_f64(p, cfg, kPX64, cfg->YB, src, &map);
     if (rc != STENCIL_OK) return rc;
-    const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 2;
-    const size_t smem = (size_t)cfg->NW * stages * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8;
+    int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 2;
+    auto smem_for = [&](int s_) { return (size_t)cfg->NW * s_ * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8; };
+    while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
+    const size_t smem = smem_for(stages);
     if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
     int dev = -1, occ = 1;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
@@ -1494,8 +1500,10 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
             rc = get_tensor_map_f64(p, cfg, cfg->px, cfg->box_rows, src, &map);
         }
         if (rc != STENCIL_OK) return rc;
-        const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : (p->radius >= 3 ? 5 : 4);
-        const size_t smem = (size_t)stages * cfg->plane_bytes + 128 + 2 * kMaxStages * sizeof(uint64_t);
+        int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : (p->radius >= 3 ? 5 : 4);
+        auto smem_for = [&](int s_) { return (size_t)s_ * cfg->plane_bytes + 128 + 2 * kMaxStages * sizeof(uint64_t); };
+        while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
+        const size_t smem = smem_for(stages);
         if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
         int dev = -1;
         if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
@@ -1583,8 +1591,10 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
             rc = get_tensor_map_f64(p, cfg, cfg->px, cfg->YB, src, &map);
         }
         if (rc != STENCIL_OK) return rc;
-        const int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
-        const size_t smem = (size_t)cfg->NW * stages * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8;
+        int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
+        auto smem_for = [&](int s_) { return (size_t)cfg->NW * s_ * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8; };
+        while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
+        const size_t smem = smem_for(stages);
         if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
         int dev = -1;
         if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
