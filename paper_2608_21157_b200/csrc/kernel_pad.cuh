@@ -5,6 +5,7 @@
 // write of the grid per sweep, which still beats gathering wrapped taps one by one.
 #pragma once
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace stencil {
 
@@ -301,6 +302,10 @@ stencil_shell_rows_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g,
         s_dx[t] = tap.dx;
     }
     __syncthreads();
+    // launched as a programmatic dependent of the pass whose shell it rewrites (and the next pass as
+    // a dependent of this kernel): everything above overlaps with the predecessor's tail
+    allow_dependents();
+    dependency_wait();
     T* orow = out + ((int64_t)z * g.ny + y) * g.nx;
     for (int x = xbegin + threadIdx.x; x < xend; x += blockDim.x) {
         T acc = T(0);

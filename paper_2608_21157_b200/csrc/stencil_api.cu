@@ -1837,6 +1837,9 @@ int apply_periodic_fused(stencil_plan_s* p, const T* in, T* out, T* other, int s
         {
             ScopedGridView view(p, p->nz, p->ny, p->nx, 0, STENCIL_ZERO);
             p->fused_wrap = wrapped;
+            // a programmatic dependent launch behind the previous pass's shell kernel: the preamble runs
+            // while that kernel drains, and the pass waits for all of it before it touches global memory
+            p->chained = p->chain_launches && k > 0;
             rc = L > 1 ? fused_any(p, src, dst, L, st) : sweep_any(p, src, dst, st);
             p->fused_wrap = false;
         }
@@ -1848,8 +1851,9 @@ int apply_periodic_fused(stencil_plan_s* p, const T* in, T* out, T* other, int s
             const int xchunks = (g.nx + kShellRowChunk - 1) / kShellRowChunk;
             const int64_t nrows = (int64_t)g.nz * 2 * H * xchunks;
             if (ntaps <= kShellTaps && nrows <= 0x7fffffffLL) {
-                stencil_shell_rows_kernel<T><<<(int)nrows, 256, 0, st>>>(src, dst, g, H, 0, taps, ntaps, xchunks);
-                if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
+                if (launch_kernel(&stencil_shell_rows_kernel<T>, (int)nrows, 256, 0, st, p->chain_launches, src, dst, g, H,
+                                  0, taps, ntaps, xchunks) != cudaSuccess)
+                    return STENCIL_ERR_CUDA;
                 p->launches++;
                 done += L;
                 src = dst;
