@@ -82,6 +82,12 @@ struct StreamShape {
     static constexpr int PLANE_BYTES = (BOX_BYTES + 127) / 128 * 128;
     static constexpr int THREADS = (NW + 1) * 32;
     static size_t smem_bytes(int stages) { return (size_t)stages * PLANE_BYTES + 128 + 128; }
+    // Periodic sweeps (WRAP): beside every plane of the ring, the cells the plane's halo would hold on a
+    // torus, each block loaded by a TMA copy of its own: the 4 columns beyond the left and the right end of
+    // the tile's rows (ROWS x 4 cells each) and the R rows above and below it (R x PX cells each).
+    static constexpr int XS_BYTES = (ROWS * 16 + 127) / 128 * 128;
+    static constexpr int YS_BYTES = (R * StreamHalo<R>::PX * 4 + 127) / 128 * 128;
+    static constexpr int STAGE_BYTES = 2 * XS_BYTES + 2 * YS_BYTES;
 };
 
 // Calls f(integral_constant<int, 0>) ... f(integral_constant<int, N-1>) in order and
@@ -166,22 +172,28 @@ __device__ __forceinline__ void gather_row(const float* rowp, const float* rowba
     }
 }
 
-template <int R, bool BOX, int K, int NW, int MINB>
-__global__ void __launch_bounds__((NW + 1) * 32, MINB)
-stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restrict__ out,
-                      const StreamGeom g,
-                      const __grid_constant__ StarWeights<R> sw,
-                      const __grid_constant__ BoxWeights<BOX ? R : 0> bw,
-                      int* __restrict__ status) {
+// WRAP: the sweep of a periodic grid (stars of radius <= 4, rows a whole number of tiles).  z wraps
+// in the plane coordinate of the TMA loads (every plane is a load of its own).  A tile at an x or y
+// face gets, beside each plane, the cells its halo would hold on a torus (see StreamShape), and
+// every consumer warp copies those of them that it is about to read over the zeros TMA filled in:
+// the 4 halo columns of its own centre rows, its own columns of the halo rows.  The corners of the
+// halo stay zero: a star does not read them.
+template <int R, bool BOX, int K, int NW, bool WRAP>
+__device__ __forceinline__ void
+stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtensorMap& tmap_ys,
+            float* __restrict__ out, const StreamGeom& g, const StarWeights<R>& sw,
+            const BoxWeights<BOX ? R : 0>& bw, int* __restrict__ status) {
+    static_assert(!WRAP || (!BOX && R <= 4), "WRAP: stars of radius <= 4");
     using S = StreamShape<R, K, NW>;
     constexpr int PX = StreamHalo<R>::PX;
     constexpr int HX = StreamHalo<R>::HX;
+    constexpr int SLOT_BYTES = S::PLANE_BYTES + (WRAP ? S::STAGE_BYTES : 0);
     extern __shared__ __align__(128) unsigned char smem_raw[];
     // ring of planes first (128-byte aligned slots), then the barriers.  The pointer is
     // formed by indexing the shared array (no integer round trip), so the compiler
     // keeps it in the shared address space and emits ld.shared for the plane reads.
     unsigned char* ring = smem_raw + ((128u - (smem_addr(smem_raw) & 127u)) & 127u);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)g.stages * S::PLANE_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)g.stages * SLOT_BYTES);
     const uint32_t full0 = smem_addr(bars);
     const uint32_t empty0 = smem_addr(bars + kMaxStages);
 
@@ -212,6 +224,11 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
     const int z1 = min(z0 + g.chunk_z, g.z_end);
     const int nplanes = (z1 - z0) + 2 * R;      // input planes z0-R .. z1-1+R
     const int pstart = z0 - R;
+    // WRAP: which faces the tile touches, and the plane row where the halo below the grid begins
+    const bool edge_l = WRAP && tile_x == 0, edge_r = WRAP && tile_x == g.tiles_x - 1;
+    // (a short last tile leaves the halo of the tile before it reaching below the grid as well)
+    const bool edge_t = WRAP && tile_y == 0, edge_b = WRAP && y0 + S::TY + R > g.ny;
+    const int row_b = R + g.ny - y0;
 
     if (warp == NW) {
         // ---------------- producer: one lane drives the TMA ring ----------------
@@ -224,9 +241,25 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
             for (int i = 0; i < nplanes; ++i) {
                 if (i >= nstage && !mbar_wait_bounded(empty0 + 8 * s, ph, g.wait_polls)) { ok = false; break; }
                 if (i != g.drop_plane) {
-                    mbar_arrive_expect_tx(full0 + 8 * s, S::BOX_BYTES);
-                    tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_BYTES), &tmap_in, full0 + 8 * s,
-                                x0 - HX + g.in_off_x, y0 - R + g.in_off_y, pstart + i + g.in_off_z);
+                    if constexpr (WRAP) {
+                        int zc = pstart + i;                       // nz >= 2R: one step brings it back
+                        zc = zc < 0 ? zc + g.nz : (zc >= g.nz ? zc - g.nz : zc);
+                        const uint32_t bar = full0 + 8 * s;
+                        unsigned char* slot = ring + (size_t)s * SLOT_BYTES;
+                        mbar_arrive_expect_tx(bar, S::BOX_BYTES + ((int)edge_l + (int)edge_r) * S::ROWS * 16 +
+                                                       ((int)edge_t + (int)edge_b) * R * PX * 4);
+                        tma_load_3d(smem_addr(slot), &tmap_in, bar, x0 - HX, y0 - R, zc);
+                        unsigned char* stage = slot + S::PLANE_BYTES;
+                        if (edge_l) tma_load_3d(smem_addr(stage), &tmap_xs, bar, g.nx - 4, y0 - R, zc);
+                        if (edge_r) tma_load_3d(smem_addr(stage + S::XS_BYTES), &tmap_xs, bar, 0, y0 - R, zc);
+                        if (edge_t) tma_load_3d(smem_addr(stage + 2 * S::XS_BYTES), &tmap_ys, bar, x0 - HX, g.ny - R, zc);
+                        if (edge_b)
+                            tma_load_3d(smem_addr(stage + 2 * S::XS_BYTES + S::YS_BYTES), &tmap_ys, bar, x0 - HX, 0, zc);
+                    } else {
+                        mbar_arrive_expect_tx(full0 + 8 * s, S::BOX_BYTES);
+                        tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_BYTES), &tmap_in, full0 + 8 * s,
+                                    x0 - HX + g.in_off_x, y0 - R + g.in_off_y, pstart + i + g.in_off_z);
+                    }
                 }
                 issued = i + 1;
                 if (++s == nstage) { s = 0; ph ^= 1; }
@@ -279,7 +312,34 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                 atomicExch(status, kStatusTimeout);
                 return;
             }
-            const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
+            const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * SLOT_BYTES);
+            if constexpr (WRAP) {
+                if (edge_l || edge_r || edge_t || edge_b) {            // uniform over the CTA
+                    float* plw = reinterpret_cast<float*>(ring + (size_t)s * SLOT_BYTES);
+                    const float* stage = pl + S::PLANE_BYTES / 4;
+                    const int rc = row0 + R + lane;                    // lane k < K takes the warp's centre row k
+                    if (edge_l && lane < K)
+                        *reinterpret_cast<float4*>(plw + rc * PX) = *reinterpret_cast<const float4*>(stage + rc * 4);
+                    if (edge_r && lane < K)
+                        *reinterpret_cast<float4*>(plw + rc * PX + HX + kStreamTX) =
+                            *reinterpret_cast<const float4*>(stage + S::XS_BYTES / 4 + rc * 4);
+#pragma unroll
+                    for (int rr = 0; rr < R; ++rr) {
+                        // the halo rows inside this warp's window of rows, the lane's own columns
+                        if (edge_t && rr >= row0 && rr < row0 + K + 2 * R)
+                            *reinterpret_cast<float4*>(plw + rr * PX + HX + 4 * lane) =
+                                *reinterpret_cast<const float4*>(stage + 2 * S::XS_BYTES / 4 + rr * PX + HX + 4 * lane);
+                        const int rb = row_b + rr;
+                        if (edge_b && rb < S::ROWS && rb >= row0 && rb < row0 + K + 2 * R)
+                            *reinterpret_cast<float4*>(plw + rb * PX + HX + 4 * lane) =
+                                *reinterpret_cast<const float4*>(stage + (2 * S::XS_BYTES + S::YS_BYTES) / 4 + rr * PX +
+                                                                 HX + 4 * lane);
+                    }
+                    // later TMA copies into this slot must not overtake these stores
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                }
+            }
             const float* colp = pl + row0 * PX + HX + 4 * lane;
             // Rows are visited once, top to bottom.  A row is a y-neighbour of up to 2R output
             // rows and the centre row of at most one; it is consumed at once, so only one
@@ -374,7 +434,7 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                 const int i = i0 + u;
                 if (i >= nplanes) return true;
                 if (!mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) return false;
-                const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * S::PLANE_BYTES);
+                const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * SLOT_BYTES);
                 const float* colp = pl + row0 * PX + HX + 4 * lane;
                 float v[K + 2 * R][4 + 2 * R];
 #pragma unroll
@@ -439,6 +499,27 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
             }
         }
     }
+}
+
+template <int R, bool BOX, int K, int NW, int MINB>
+__global__ void __launch_bounds__((NW + 1) * 32, MINB)
+stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restrict__ out,
+                      const StreamGeom g,
+                      const __grid_constant__ StarWeights<R> sw,
+                      const __grid_constant__ BoxWeights<BOX ? R : 0> bw,
+                      int* __restrict__ status) {
+    stream_body<R, BOX, K, NW, false>(tmap_in, tmap_in, tmap_in, out, g, sw, bw, status);
+}
+
+// The sweep of a periodic grid: tmap_xs has boxes of 4 columns x ROWS rows, tmap_ys of PX columns x R rows.
+template <int R, int K, int NW, int MINB>
+__global__ void __launch_bounds__((NW + 1) * 32, MINB)
+stencil_stream_wrap_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_xs,
+                           const __grid_constant__ CUtensorMap tmap_ys, float* __restrict__ out,
+                           const StreamGeom g, const __grid_constant__ StarWeights<R> sw,
+                           int* __restrict__ status) {
+    const BoxWeights<0> bw = {};
+    stream_body<R, false, K, NW, true>(tmap_in, tmap_xs, tmap_ys, out, g, sw, bw, status);
 }
 
 }  // namespace stencil

@@ -103,6 +103,12 @@ struct StreamConfig {
     const void* kernel;
     cudaError_t (*launch)(const struct stencil_plan_s*, const StreamConfig&, const CUtensorMap&,
                           float*, const StreamGeom&, int grid, size_t smem, cudaStream_t);
+    // the sweep of a periodic grid inside the kernel (stars of radius <= 4; null otherwise)
+    const void* kernel_wrap;
+    int stage_bytes;                         // per ring slot, beside the plane
+    mutable size_t smem_allowed_wrap;
+    cudaError_t (*launch_wrap)(const struct stencil_plan_s*, const CUtensorMap&, const CUtensorMap&,
+                               const CUtensorMap&, float*, const StreamGeom&, int grid, size_t smem, cudaStream_t);
 };
 
 // ---------------------------------------------------------------------------
@@ -230,6 +236,7 @@ struct stencil_plan_s {
     int tmap_nx;                   // non-zero while a padded-row sweep runs: the true row length
     int periodic_route;            // knob: 0 = by measured cost, 1 = padded copy, 2 = wrap correction where it fits
     bool fused_wrap;               // set for one launch_fused call: the pass wraps x and z in the kernel
+    bool stream_wrap;              // set while a periodic apply sweeps with the kernel that wraps all three axes
     bool src_padded;               // set while an iterated periodic apply runs: the source of a sweep is
                                    // a padded grid with current halos
     float* host_in;                // N floats each, apply_host staging
@@ -296,6 +303,23 @@ cudaError_t launch_stream_t(const stencil_plan_s* p, const StreamConfig&, const 
                          st, p->chained, map, out, g, sw, bw, p->d_status);
 }
 
+template <int R, int K, int NW, int MINB>
+cudaError_t launch_stream_wrap_t(const stencil_plan_s* p, const CUtensorMap& map, const CUtensorMap& map_xs,
+                                 const CUtensorMap& map_ys, float* out, const StreamGeom& g, int grid, size_t smem,
+                                 cudaStream_t st) {
+    StarWeights<R> sw;
+    std::memset(&sw, 0, sizeof(sw));
+    sw.c = dense_w(p, 0, 0, 0);
+    for (int d = -R; d <= R; ++d) {
+        if (d == 0) continue;
+        sw.x[d + R] = dense_w(p, 0, 0, d);
+        sw.y[d + R] = dense_w(p, 0, d, 0);
+        sw.z[d + R] = dense_w(p, d, 0, 0);
+    }
+    return launch_kernel(&stencil_stream_wrap_kernel<R, K, NW, MINB>, grid, StreamShape<R, K, NW>::THREADS, smem, st,
+                         p->chained, map, map_xs, map_ys, out, g, sw, p->d_status);
+}
+
 template <int R, bool BOX, int K, int NW, int MINB>
 StreamConfig make_cfg() {
     using S = StreamShape<R, K, NW>;
@@ -308,6 +332,12 @@ StreamConfig make_cfg() {
     c.cache_device = -1;
     c.kernel = reinterpret_cast<const void*>(&stencil_stream_kernel<R, BOX, K, NW, MINB>);
     c.launch = &launch_stream_t<R, BOX, K, NW, MINB>;
+    c.kernel_wrap = nullptr; c.launch_wrap = nullptr; c.stage_bytes = 0; c.smem_allowed_wrap = 0;
+    if constexpr (!BOX && R <= 4) {
+        c.kernel_wrap = reinterpret_cast<const void*>(&stencil_stream_wrap_kernel<R, K, NW, MINB>);
+        c.launch_wrap = &launch_stream_wrap_t<R, K, NW, MINB>;
+        c.stage_bytes = S::STAGE_BYTES;
+    }
     return c;
 }
 
@@ -725,6 +755,7 @@ int stream_occupancy(const StreamConfig* cfg, int stages) {
     if (dev != cfg->cache_device) {                // function attributes are per device
         for (int& o : cfg->occupancy) o = 0;
         cfg->smem_allowed = 0;
+        cfg->smem_allowed_wrap = 0;
         cfg->cache_device = dev;
     }
     if (smem > cfg->smem_allowed) {                // the limit only ever grows
@@ -836,6 +867,61 @@ int pad_periodic(stencil_plan_s* p, const T* src, cudaStream_t st, const T** pad
     return STENCIL_OK;
 }
 
+// One sweep of a periodic grid with the kernel that wraps all three axes itself (see stream_body).
+// Called under a zero-boundary view of the plan; the tensor maps are copied out of the plan's cache
+// at once, since a later entry may move the earlier ones.
+int launch_stream_wrap(stencil_plan_s* p, const StreamConfig* cfg, int stages, const float* src, float* dst,
+                       cudaStream_t st) {
+    if (!cfg->launch_wrap) return STENCIL_ERR_UNSUPPORTED;
+    const char* key = reinterpret_cast<const char*>(cfg);
+    const CUtensorMap* m = nullptr;
+    CUtensorMap map, map_xs, map_ys;
+    int rc;
+    if ((rc = get_tensor_map(p, key, cfg->px, cfg->box_rows, src, &m)) != STENCIL_OK) return rc;
+    map = *m;
+    if ((rc = get_tensor_map(p, key + 1, 4, cfg->box_rows, src, &m)) != STENCIL_OK) return rc;
+    map_xs = *m;
+    if ((rc = get_tensor_map(p, key + 2, cfg->px, p->radius, src, &m)) != STENCIL_OK) return rc;
+    map_ys = *m;
+    const size_t smem = (size_t)stages * (cfg->plane_bytes + cfg->stage_bytes) + 128 + 2 * kMaxStages * sizeof(uint64_t);
+    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    {
+        std::lock_guard<std::mutex> lock(g_config_mutex);
+        if (dev != cfg->cache_device) {
+            cfg->smem_allowed = 0; cfg->smem_allowed_wrap = 0; cfg->cache_device = dev;
+            for (int& o : cfg->occupancy) o = 0;
+        }
+        if (smem > cfg->smem_allowed_wrap) {
+            if (cudaFuncSetAttribute(cfg->kernel_wrap, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                cudaSuccess) {
+                cudaGetLastError();
+                return STENCIL_ERR_CUDA;
+            }
+            cfg->smem_allowed_wrap = smem;
+        }
+    }
+    StreamGeom g;
+    g.in_off_x = g.in_off_y = g.in_off_z = 0;
+    g.nz = p->nz; g.ny = p->ny; g.nx = p->nx;
+    g.tiles_x = (p->nx + kStreamTX - 1) / kStreamTX;
+    g.tiles_y = (p->ny + cfg->tile_y - 1) / cfg->tile_y;
+    g.stages = stages;
+    g.streaming_store = p->streaming_store;
+    if (stream_occupancy(cfg, stages) <= 0) return STENCIL_ERR_UNSUPPORTED;
+    int chunk = p->chunk_z > 0 ? p->chunk_z : choose_chunk(p, cfg, stages, nullptr, p->nz);
+    chunk = std::max(1, std::min(chunk, p->nz));
+    g.chunk_z = chunk;
+    g.z_begin = 0; g.z_end = p->nz;
+    g.wait_polls = p->wait_polls; g.drop_plane = -1;
+    const int64_t grid64 = (int64_t)g.tiles_x * g.tiles_y * ((p->nz + chunk - 1) / chunk);
+    if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
+    if (cfg->launch_wrap(p, map, map_xs, map_ys, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
+    p->launches++;
+    return STENCIL_OK;
+}
+
 // dst[z_begin, z_end) = one sweep of src; the whole grid when z_end <= z_begin.
 int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st, int z_begin = 0,
                   int z_end = 0) {
@@ -869,6 +955,7 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
         p->stream_cfg_tuned = true;
     }
     const StreamConfig* cfg = p->stream_cfg;
+    if (p->stream_wrap) return launch_stream_wrap(p, cfg, stages, src, dst, st);
     const CUtensorMap* map = nullptr;
     const bool periodic = p->boundary == STENCIL_PERIODIC;
     int rc;
@@ -1748,6 +1835,31 @@ int apply_periodic_corrected(stencil_plan_s* p, const T* in, T* out, T* other, i
     return STENCIL_OK;
 }
 
+// A periodic 3D star of radius <= 4 whose rows are a whole number of 128-column tiles is swept by the
+// kernel that wraps all three axes itself: no correction pass, no padded copy.
+bool stream_wrap_ok(const stencil_plan_s* p) {
+    return !p->f64 && p->ndim == 3 && p->shape == STENCIL_STAR && p->variant == STENCIL_VARIANT_STREAM &&
+           p->stream_cfg && p->stream_cfg->launch_wrap && p->nx % kStreamTX == 0 && wrap_correction_fits(p);
+}
+
+int apply_periodic_inkernel(stencil_plan_s* p, const float* in, float* out, int steps, cudaStream_t st) {
+    const float* src = in;
+    for (int k = 0; k < steps; ++k) {
+        float* dst = ((steps - 1 - k) % 2 == 0) ? out : p->scratch;
+        int rc;
+        {
+            ScopedGridView view(p, p->nz, p->ny, p->nx, 0, STENCIL_ZERO);
+            p->stream_wrap = true;
+            p->chained = p->chain_launches && k > 0;
+            rc = launch_stream(p, src, dst, st);
+            p->stream_wrap = false;
+        }
+        if (rc != STENCIL_OK) return rc;
+        src = dst;
+    }
+    return STENCIL_OK;
+}
+
 // Taps of the operator applied L times in a row (its L-fold self-convolution: the sweep is a
 // cross-correlation, and correlating with w twice is correlating with w * w), as doubles on the
 // device.  Built from the plan's own weights at first need.
@@ -1804,6 +1916,17 @@ int composite_taps(stencil_plan_s* p, int L, const TapT<double>** taps, int* nta
     return STENCIL_OK;
 }
 
+// One periodic step with the kernel that wraps all three axes, where it applies (fp32 3D stars).
+bool sweep_wrapped(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st, int* rc) {
+    if (!stream_wrap_ok(p)) return false;
+    ScopedGridView view(p, p->nz, p->ny, p->nx, 0, STENCIL_ZERO);
+    p->stream_wrap = true;
+    *rc = launch_stream(p, src, dst, st);
+    p->stream_wrap = false;
+    return true;
+}
+bool sweep_wrapped(stencil_plan_s*, const double*, double*, cudaStream_t, int*) { return false; }
+
 int fused_any(stencil_plan_s* p, const float* src, float* dst, int nlev, cudaStream_t st) {
     return p->ndim == 3 ? launch_fused(p, src, dst, nlev, st) : launch_rows2d_fused(p, src, dst, nlev, st);
 }
@@ -1833,6 +1956,12 @@ int apply_periodic_fused(stencil_plan_s* p, const T* in, T* out, T* other, int s
         const TapT<double>* taps = nullptr;
         int ntaps = 0, rc;
         if ((rc = composite_taps(p, L, &taps, &ntaps)) != STENCIL_OK) return rc;
+        if (L == 1 && sweep_wrapped(p, src, dst, st, &rc)) {       // a last single step needs no shell kernel
+            if (rc != STENCIL_OK) return rc;
+            done += L;
+            src = dst;
+            continue;
+        }
         const bool wrapped = L > 1 && fused_wrap_ok(p, L);
         {
             ScopedGridView view(p, p->nz, p->ny, p->nx, 0, STENCIL_ZERO);
@@ -1964,7 +2093,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->npoints = n;
     p->radius = radius; p->shape = shape; p->boundary = boundary;
     p->device = -1;
-    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0; p->src_padded = false; p->fused_wrap = false; p->periodic_route = 0;
+    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0; p->src_padded = false; p->fused_wrap = false; p->stream_wrap = false; p->periodic_route = 0;
     for (int l = 0; l <= kMaxFuseLevels; ++l) p->d_ctaps[l] = nullptr;
     p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr; p->fused2d64_cfg = nullptr;
     p->host_in = nullptr; p->host_out = nullptr;
@@ -2090,6 +2219,7 @@ int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void
         const int depth = p->fused_cfg ? p->fused_cfg->T : p->fused2d_cfg ? p->fused2d_cfg->T : 1;
         if (steps > 1 && depth > 1 && p->periodic_route != 1)
             return apply_periodic_fused(p, in, out, p->scratch, steps, depth, st);
+        if (p->periodic_route == 0 && stream_wrap_ok(p)) return apply_periodic_inkernel(p, in, out, steps, st);
         if (use_wrap_correction(p, steps)) return apply_periodic_corrected(p, in, out, p->scratch, steps, st);
         if (steps > 1) return apply_periodic(p, in, out, steps, st);
     }

@@ -314,6 +314,43 @@ def test_wide_star_fp64_kernels_match_oracle(R, dims, chunk, stages):
         assert float(np.max(np.abs(got - want))) <= wl.tolerance(w, float(np.abs(a).max()), 2)
 
 
+# ------------------------------------- periodic boundary wrapped inside the sweep --
+@pytest.mark.parametrize("R", [1, 2, 3, 4])
+@pytest.mark.parametrize("dims,chunk_z,knobs", [
+    ((19, 37, 128), 0, {}),                       # one tile per row: it touches both x faces
+    ((12, 50, 384), 5, {}),                       # three tiles per row, several z chunks, ragged last tile in y
+    ((9, 16, 256), 0, {}),                        # one tile in y at the default tile height: both y faces
+    ((8, 8, 128), 3, {}),                         # every extent exactly 2R for radius 4
+    ((21, 33, 256), 4, dict(tile_y=14)),          # the 7-warp tiles
+    ((10, 70, 128), 0, dict(rows_per_thread=4)),  # 32-row tiles
+])
+def test_periodic_3d_star_wrapped_inside_the_sweep(R, dims, chunk_z, knobs):
+    """Periodic 3D stars on rows of whole tiles: the sweep wraps x, y and z itself (one launch per step,
+    no correction kernel, no padded copy); fused passes are switched off to reach it for radius 1."""
+    if min(dims) < 2 * R:
+        pytest.skip("needs every extent >= 2R")
+    w = wl.random_star_weights(3, R, 81)
+    a = wl.normal_field(dims, 82)
+    for steps in (1, 3):
+        dev = torch.device("cuda:0")
+        src = torch.from_numpy(a).to(dev)
+        dst = torch.full_like(src, float("nan"))
+        try:
+            plan = b.Plan(dims, R, b.STAR, w, b.PERIODIC, fuse_steps=1, chunk_z=chunk_z or None, **knobs)
+        except b.StencilError as e:                    # a tile shape this radius does not have
+            assert e.status == b.ERR_UNSUPPORTED and knobs
+            return
+        with plan as p:
+            p.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
+            assert p.query_status() == b.OK
+            assert p.launches == steps and p.get(b.KEY_SCRATCH_BYTES) == (a.nbytes if steps > 1 else 0)
+        got = dst.cpu().numpy()
+        want = oracle.apply(a, w, b.PERIODIC, steps)
+        tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+        err = float(np.max(np.abs(got - want)))
+        assert err <= tol, f"R={R} dims={dims} steps={steps}: {err:.3e} > {tol:.3e}"
+
+
 # ------------------------------------------- periodic boundary under temporal blocking --
 @pytest.mark.parametrize("dims,R,knobs", [
     ((21, 37, 256), 1, {}),                                         # one 256-wide region per row, T = 2
@@ -338,7 +375,8 @@ def test_periodic_fused_3d_matches_oracle(dims, R, knobs):
             p.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
             assert p.query_status() == b.OK
             passes = -(-steps // depth)
-            assert 2 * passes <= p.launches <= 3 * passes           # a pass and its one or two shell kernels
+            # a fused pass and its one or two shell kernels; a last single step may wrap inside its sweep
+            assert 2 * passes - 1 <= p.launches <= 3 * passes
         got = dst.cpu().numpy()
         want = oracle.apply(a, w, b.PERIODIC, steps)
         tol = wl.tolerance(w, float(np.abs(a).max()), steps)
