@@ -172,12 +172,47 @@ __device__ __forceinline__ void gather_row(const float* rowp, const float* rowba
     }
 }
 
+// gather_row for a row whose halo columns may live elsewhere (radius <= 4).  Everything is an offset
+// from one pointer into shared memory, so that the loads stay shared-space loads whichever way the
+// selects go: `o_rowp` is the lane's float4, `o_lh` the 4 cells left of the row's first tile column,
+// `o_rh` the 4 cells right of its last one.
+template <int R>
+__device__ __forceinline__ void gather_row_split(const float* base, int o_rowp, int o_lh, int o_rh, int lane,
+                                                 const float4& ctr, float (&v)[4 + 2 * R]) {
+    static_assert(R <= 4, "4-column halos");
+    v[R + 0] = ctr.x; v[R + 1] = ctr.y; v[R + 2] = ctr.z; v[R + 3] = ctr.w;
+    if constexpr (R <= 2) {
+        const float c4[4] = {ctr.x, ctr.y, ctr.z, ctr.w};
+#pragma unroll
+        for (int t = 0; t < R; ++t) {
+            const float hl = base[o_lh + 4 - R + t];
+            const float hr = base[o_rh + t];
+            const float l = __shfl_up_sync(0xffffffffu, c4[4 - R + t], 1);
+            const float r = __shfl_down_sync(0xffffffffu, c4[t], 1);
+            v[t] = lane == 0 ? hl : l;
+            v[R + 4 + t] = lane == 31 ? hr : r;
+        }
+    } else {
+        const float4 l = *reinterpret_cast<const float4*>(base + (lane == 0 ? o_lh : o_rowp - 4));
+        const float4 r = *reinterpret_cast<const float4*>(base + (lane == 31 ? o_rh : o_rowp + 4));
+        const float l4[4] = {l.x, l.y, l.z, l.w};
+        const float r4[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int t = 0; t < R; ++t) {
+            v[t] = l4[4 - R + t];
+            v[R + 4 + t] = r4[t];
+        }
+    }
+}
+
 // WRAP: the sweep of a periodic grid (stars of radius <= 4, rows a whole number of tiles).  z wraps
 // in the plane coordinate of the TMA loads (every plane is a load of its own).  A tile at an x or y
 // face gets, beside each plane, the cells its halo would hold on a torus (see StreamShape), and
-// every consumer warp copies those of them that it is about to read over the zeros TMA filled in:
-// the 4 halo columns of its own centre rows, its own columns of the halo rows.  The corners of the
-// halo stay zero: a star does not read them.
+// its consumer warps read the halo columns of their centre rows straight from there (a tile in the
+// middle of a row reads them from the plane, as ever: one pointer select per row); the halo rows,
+// which only the few tiles at a y face need, are copied over the zeros TMA filled in, every warp
+// copying its own columns of the rows it is about to read.  The corners of the halo stay zero: a
+// star does not read them.
 template <int R, bool BOX, int K, int NW, bool WRAP>
 __device__ __forceinline__ void
 stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtensorMap& tmap_ys,
@@ -314,15 +349,9 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
             }
             const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * SLOT_BYTES);
             if constexpr (WRAP) {
-                if (edge_l || edge_r || edge_t || edge_b) {            // uniform over the CTA
+                if (edge_t || edge_b) {                                // uniform over the CTA
                     float* plw = reinterpret_cast<float*>(ring + (size_t)s * SLOT_BYTES);
                     const float* stage = pl + S::PLANE_BYTES / 4;
-                    const int rc = row0 + R + lane;                    // lane k < K takes the warp's centre row k
-                    if (edge_l && lane < K)
-                        *reinterpret_cast<float4*>(plw + rc * PX) = *reinterpret_cast<const float4*>(stage + rc * 4);
-                    if (edge_r && lane < K)
-                        *reinterpret_cast<float4*>(plw + rc * PX + HX + kStreamTX) =
-                            *reinterpret_cast<const float4*>(stage + S::XS_BYTES / 4 + rc * 4);
 #pragma unroll
                     for (int rr = 0; rr < R; ++rr) {
                         // the halo rows inside this warp's window of rows, the lane's own columns
@@ -365,7 +394,14 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
                 if (kk >= R && kk < K + R) {
                     const int k = kk - R;                  // centre row of output row k
                     float v[4 + 2 * R];
-                    gather_row<R>(colp + kk * PX, pl + (row0 + kk) * PX, lane, c, v);
+                    if constexpr (WRAP) {
+                        const int o_row = (row0 + kk) * PX;
+                        const int o_xs = S::PLANE_BYTES / 4 + (row0 + kk) * 4;
+                        gather_row_split<R>(pl, o_row + HX + 4 * lane, edge_l ? o_xs : o_row,
+                                            edge_r ? o_xs + S::XS_BYTES / 4 : o_row + HX + kStreamTX, lane, c, v);
+                    } else {
+                        gather_row<R>(colp + kk * PX, pl + (row0 + kk) * PX, lane, c, v);
+                    }
 #pragma unroll
                     for (int m = 0; m < 4; ++m) {
                         float a = fmaf(sw.c, v[R + m], acc[k][m]);
