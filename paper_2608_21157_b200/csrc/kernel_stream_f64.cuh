@@ -36,18 +36,27 @@ struct Stream64Shape {
 
     static constexpr int PLANE_BYTES = PLANE_DOUBLES * 8;
     static constexpr int THREADS = (NW + 1) * 32;
+    // periodic sweeps (WRAP): beside every plane the cells its halo would hold on a torus, as in the
+    // fp32 kernel: 4 columns x ROWS rows beyond either end of the rows, R rows x PX columns above and below
+    static constexpr int XS_BYTES = (ROWS * 32 + 127) / 128 * 128;
+    static constexpr int YS_BYTES = (R * StreamHalo64<R>::PX * 8 + 127) / 128 * 128;
+    static constexpr int STAGE_BYTES = 2 * XS_BYTES + 2 * YS_BYTES;
 };
 
 __device__ __forceinline__ double d2get(const double2& v, int m) { return m == 0 ? v.x : v.y; }
 
-template <int R, bool BOX, int K, int NW, int MINB>
-__global__ void __launch_bounds__((NW + 1) * 32, MINB)
-stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* __restrict__ out,
-                          const StreamGeom g,
-                          const __grid_constant__ StarWeights64<R> sw,
-                          const __grid_constant__ BoxWeights64<BOX ? R : 0> bw,
-                          int* __restrict__ status) {
+// WRAP: the sweep of a periodic grid, as in the fp32 kernel (stars of radius <= 4, rows a whole number
+// of 64-column tiles): z wraps in the plane coordinate of the TMA loads; a tile at an x face reads the
+// halo columns of its centre rows from blocks loaded beside the plane; a tile at a y face copies its
+// own columns of the halo rows over the zeros TMA filled in.
+template <int R, bool BOX, int K, int NW, bool WRAP>
+__device__ __forceinline__ void
+stream_f64_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtensorMap& tmap_ys,
+                double* __restrict__ out, const StreamGeom& g, const StarWeights64<R>& sw,
+                const BoxWeights64<BOX ? R : 0>& bw, int* __restrict__ status) {
+    static_assert(!WRAP || (!BOX && R <= 4), "WRAP: stars of radius <= 4");
     using S = Stream64Shape<R, K, NW>;
+    constexpr int SLOT_DOUBLES = (S::PLANE_BYTES + (WRAP ? S::STAGE_BYTES : 0)) / 8;
     constexpr int PX = StreamHalo64<R>::PX;
     constexpr int HX = StreamHalo64<R>::HX;
     constexpr int HW = (R + 1) / 2 * 2;              // halo doubles read per side (a whole double2)
@@ -55,7 +64,7 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
     extern __shared__ __align__(128) unsigned char smem_raw[];
     unsigned char* base = smem_raw + ((128u - (smem_addr(smem_raw) & 127u)) & 127u);
     double* ring = reinterpret_cast<double*>(base);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)g.stages * S::PLANE_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)g.stages * SLOT_DOUBLES * 8);
     const uint32_t full0 = smem_addr(bars);
     const uint32_t empty0 = smem_addr(bars + kMaxStages);
 
@@ -84,6 +93,10 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
     const int z1 = min(z0 + g.chunk_z, g.z_end);
     const int nplanes = (z1 - z0) + 2 * R;
     const int pstart = z0 - R;
+    // WRAP: which faces the tile's halo reaches across, and the plane row where the halo below the grid begins
+    const bool edge_l = WRAP && tile_x == 0, edge_r = WRAP && tile_x == g.tiles_x - 1;
+    const bool edge_t = WRAP && tile_y == 0, edge_b = WRAP && y0 + S::TY + R > g.ny;
+    const int row_b = R + g.ny - y0;
 
     if (warp == NW) {
         if (lane == 0) {
@@ -94,9 +107,25 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
             uint32_t ph = 1;
             for (int i = 0; i < nplanes; ++i) {
                 if (i >= nstage && !mbar_wait_bounded(empty0 + 8 * s, ph, g.wait_polls)) { ok = false; break; }
-                mbar_arrive_expect_tx(full0 + 8 * s, S::PLANE_BYTES);
-                tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_DOUBLES), &tmap_in, full0 + 8 * s,
-                            x0 - HX + g.in_off_x, y0 - R + g.in_off_y, pstart + i + g.in_off_z);
+                if constexpr (WRAP) {
+                    int zc = pstart + i;                           // nz >= 2R: one step brings it back
+                    zc = zc < 0 ? zc + g.nz : (zc >= g.nz ? zc - g.nz : zc);
+                    const uint32_t bar = full0 + 8 * s;
+                    double* slot = ring + (size_t)s * SLOT_DOUBLES;
+                    mbar_arrive_expect_tx(bar, S::PLANE_BYTES + ((int)edge_l + (int)edge_r) * S::ROWS * 32 +
+                                                   ((int)edge_t + (int)edge_b) * R * PX * 8);
+                    tma_load_3d(smem_addr(slot), &tmap_in, bar, x0 - HX, y0 - R, zc);
+                    double* stage = slot + S::PLANE_DOUBLES;
+                    if (edge_l) tma_load_3d(smem_addr(stage), &tmap_xs, bar, g.nx - 4, y0 - R, zc);
+                    if (edge_r) tma_load_3d(smem_addr(stage + S::XS_BYTES / 8), &tmap_xs, bar, 0, y0 - R, zc);
+                    if (edge_t) tma_load_3d(smem_addr(stage + 2 * S::XS_BYTES / 8), &tmap_ys, bar, x0 - HX, g.ny - R, zc);
+                    if (edge_b)
+                        tma_load_3d(smem_addr(stage + (2 * S::XS_BYTES + S::YS_BYTES) / 8), &tmap_ys, bar, x0 - HX, 0, zc);
+                } else {
+                    mbar_arrive_expect_tx(full0 + 8 * s, S::PLANE_BYTES);
+                    tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_DOUBLES), &tmap_in, full0 + 8 * s,
+                                x0 - HX + g.in_off_x, y0 - R + g.in_off_y, pstart + i + g.in_off_z);
+                }
                 issued = i + 1;
                 if (++s == nstage) { s = 0; ph ^= 1; }
             }
@@ -132,7 +161,28 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
                 atomicExch(status, kStatusTimeout);
                 return;
             }
-            const double* pl = ring + (size_t)s * S::PLANE_DOUBLES;
+            const double* pl = ring + (size_t)s * SLOT_DOUBLES;
+            if constexpr (WRAP) {
+                if (edge_t || edge_b) {                                // uniform over the CTA
+                    double* plw = ring + (size_t)s * SLOT_DOUBLES;
+                    const double* stage = pl + S::PLANE_DOUBLES;
+#pragma unroll
+                    for (int rr = 0; rr < R; ++rr) {
+                        // the halo rows inside this warp's window of rows, the lane's own columns
+                        if (edge_t && rr >= row0 && rr < row0 + K + 2 * R)
+                            *reinterpret_cast<double2*>(plw + rr * PX + HX + 2 * lane) =
+                                *reinterpret_cast<const double2*>(stage + 2 * S::XS_BYTES / 8 + rr * PX + HX + 2 * lane);
+                        const int rb = row_b + rr;
+                        if (edge_b && rb < S::ROWS && rb >= row0 && rb < row0 + K + 2 * R)
+                            *reinterpret_cast<double2*>(plw + rb * PX + HX + 2 * lane) =
+                                *reinterpret_cast<const double2*>(stage + (2 * S::XS_BYTES + S::YS_BYTES) / 8 + rr * PX +
+                                                                  HX + 2 * lane);
+                    }
+                    // later TMA copies into this slot must not overtake these stores
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                }
+            }
             const double* colp = pl + row0 * PX + HX + 2 * lane;
             double acc[K][2];
 #pragma unroll
@@ -154,7 +204,20 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
                     double v[NV];                     // v[HW + m + dx]: the input at column m + dx of the pair
 #pragma unroll
                     for (int t = 0; t < NV / 2; ++t) {
-                        const double2 dd = *reinterpret_cast<const double2*>(colp + kk * PX - HW + 2 * t);
+                        double2 dd;
+                        if constexpr (WRAP) {
+                            // the double2 that holds tile columns c, c+1.  The windows of the first (last) HW/2
+                            // lanes reach into the row's halo, c < 0 (c >= 64): at an x face that halo is the
+                            // staged block (4 columns per row), else the plane's own halo columns.
+                            const int c = 2 * lane - HW + 2 * t;
+                            int o = (row0 + kk) * PX + HX + c;
+                            const int o_xs = S::PLANE_DOUBLES + (row0 + kk) * 4;
+                            if (2 * t < HW && edge_l && c < 0) o = o_xs + 4 + c;
+                            if (2 * t >= HW + 2 && edge_r && c >= kStream64TX) o = o_xs + S::XS_BYTES / 8 + c - kStream64TX;
+                            dd = *reinterpret_cast<const double2*>(pl + o);
+                        } else {
+                            dd = *reinterpret_cast<const double2*>(colp + kk * PX - HW + 2 * t);
+                        }
                         v[2 * t] = dd.x;
                         v[2 * t + 1] = dd.y;
                     }
@@ -207,7 +270,7 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
                 const int i = i0 + u;
                 if (i >= nplanes) return true;
                 if (!mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) return false;
-                const double* pl = ring + (size_t)s * S::PLANE_DOUBLES;
+                const double* pl = ring + (size_t)s * SLOT_DOUBLES;
                 const double* colp = pl + row0 * PX + HX + 2 * lane;
                 double v[K + 2 * R][NV];
 #pragma unroll
@@ -260,6 +323,28 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
             }
         }
     }
+}
+
+template <int R, bool BOX, int K, int NW, int MINB>
+__global__ void __launch_bounds__((NW + 1) * 32, MINB)
+stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* __restrict__ out,
+                          const StreamGeom g,
+                          const __grid_constant__ StarWeights64<R> sw,
+                          const __grid_constant__ BoxWeights64<BOX ? R : 0> bw,
+                          int* __restrict__ status) {
+    stream_f64_body<R, BOX, K, NW, false>(tmap_in, tmap_in, tmap_in, out, g, sw, bw, status);
+}
+
+// The sweep of a periodic grid: tmap_xs has boxes of 4 columns x ROWS rows, tmap_ys of PX columns x R rows.
+template <int R, int K, int NW, int MINB>
+__global__ void __launch_bounds__((NW + 1) * 32, MINB)
+stencil_stream_f64_wrap_kernel(const __grid_constant__ CUtensorMap tmap_in,
+                               const __grid_constant__ CUtensorMap tmap_xs,
+                               const __grid_constant__ CUtensorMap tmap_ys, double* __restrict__ out,
+                               const StreamGeom g, const __grid_constant__ StarWeights64<R> sw,
+                               int* __restrict__ status) {
+    const BoxWeights64<0> bw = {};
+    stream_f64_body<R, false, K, NW, true>(tmap_in, tmap_xs, tmap_ys, out, g, sw, bw, status);
 }
 
 }  // namespace stencil

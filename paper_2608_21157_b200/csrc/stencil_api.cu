@@ -201,6 +201,12 @@ struct Stream64Config {
     mutable int cache_device;
     cudaError_t (*launch)(const struct stencil_plan_s*, const CUtensorMap&, double*, const StreamGeom&,
                           int grid, size_t smem, cudaStream_t);
+    // the sweep of a periodic grid inside the kernel (stars of radius <= 4; null otherwise)
+    const void* kernel_wrap;
+    int stage_bytes;                         // per ring slot, beside the plane
+    mutable size_t smem_allowed_wrap;
+    cudaError_t (*launch_wrap)(const struct stencil_plan_s*, const CUtensorMap&, const CUtensorMap&,
+                               const CUtensorMap&, double*, const StreamGeom&, int grid, size_t smem, cudaStream_t);
 };
 
 constexpr int kMaxFuseLevels = 4;          // deepest temporal blocking of any fused kernel
@@ -1393,6 +1399,23 @@ cudaError_t launch_stream64_t(const stencil_plan_s* p, const CUtensorMap& map, d
                          smem, st, p->chained, map, out, g, sw, bw, p->d_status);
 }
 
+template <int R, int K, int NW, int MINB>
+cudaError_t launch_stream64_wrap_t(const stencil_plan_s* p, const CUtensorMap& map, const CUtensorMap& map_xs,
+                                   const CUtensorMap& map_ys, double* out, const StreamGeom& g, int grid,
+                                   size_t smem, cudaStream_t st) {
+    StarWeights64<R> sw;
+    std::memset(&sw, 0, sizeof(sw));
+    sw.c = dense_w64_3d(p, 0, 0, 0);
+    for (int d = -R; d <= R; ++d) {
+        if (d == 0) continue;
+        sw.x[d + R] = dense_w64_3d(p, 0, 0, d);
+        sw.y[d + R] = dense_w64_3d(p, 0, d, 0);
+        sw.z[d + R] = dense_w64_3d(p, d, 0, 0);
+    }
+    return launch_kernel(&stencil_stream_f64_wrap_kernel<R, K, NW, MINB>, grid, Stream64Shape<R, K, NW>::THREADS,
+                         smem, st, p->chained, map, map_xs, map_ys, out, g, sw, p->d_status);
+}
+
 template <int R, bool BOX, int K, int NW, int MINB>
 Stream64Config make_stream64() {
     using S = Stream64Shape<R, K, NW>;
@@ -1402,6 +1425,12 @@ Stream64Config make_stream64() {
     c.kernel = reinterpret_cast<const void*>(&stencil_stream_f64_kernel<R, BOX, K, NW, MINB>);
     c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
     c.launch = &launch_stream64_t<R, BOX, K, NW, MINB>;
+    c.kernel_wrap = nullptr; c.launch_wrap = nullptr; c.stage_bytes = 0; c.smem_allowed_wrap = 0;
+    if constexpr (!BOX && R <= 4) {
+        c.kernel_wrap = reinterpret_cast<const void*>(&stencil_stream_f64_wrap_kernel<R, K, NW, MINB>);
+        c.launch_wrap = &launch_stream64_wrap_t<R, K, NW, MINB>;
+        c.stage_bytes = S::STAGE_BYTES;
+    }
     return c;
 }
 
@@ -1587,8 +1616,23 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
             rc = get_tensor_map_f64(p, cfg, cfg->px, cfg->box_rows, src, &map);
         }
         if (rc != STENCIL_OK) return rc;
+        // the sweep that wraps a periodic grid itself: three tensor maps, copied out of the plan's cache at
+        // once (a later entry may move the earlier ones), and the staged halo blocks beside every plane
+        const bool wrap = p->stream_wrap && cfg->launch_wrap;
+        if (p->stream_wrap && !wrap) return STENCIL_ERR_UNSUPPORTED;
+        CUtensorMap map0, map_xs, map_ys;
+        if (wrap) {
+            const char* key = reinterpret_cast<const char*>(cfg);
+            map0 = *map;
+            if ((rc = get_tensor_map_f64(p, key + 1, 4, cfg->box_rows, src, &map)) != STENCIL_OK) return rc;
+            map_xs = *map;
+            if ((rc = get_tensor_map_f64(p, key + 2, cfg->px, p->radius, src, &map)) != STENCIL_OK) return rc;
+            map_ys = *map;
+        }
         int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : (p->radius >= 3 ? 5 : 4);
-        auto smem_for = [&](int s_) { return (size_t)s_ * cfg->plane_bytes + 128 + 2 * kMaxStages * sizeof(uint64_t); };
+        auto smem_for = [&](int s_) {
+            return (size_t)s_ * (cfg->plane_bytes + (wrap ? cfg->stage_bytes : 0)) + 128 + 2 * kMaxStages * sizeof(uint64_t);
+        };
         while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
         const size_t smem = smem_for(stages);
         if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
@@ -1596,14 +1640,17 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
         {
             std::lock_guard<std::mutex> lock(g_config_mutex);
-            if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->occ_smem = 0; cfg->cache_device = dev; }
-            if (smem > cfg->smem_allowed) {
-                if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                    cudaSuccess) {
+            if (dev != cfg->cache_device) {
+                cfg->smem_allowed = 0; cfg->smem_allowed_wrap = 0; cfg->occ_smem = 0; cfg->cache_device = dev;
+            }
+            size_t& allowed = wrap ? cfg->smem_allowed_wrap : cfg->smem_allowed;
+            if (smem > allowed) {
+                if (cudaFuncSetAttribute(wrap ? cfg->kernel_wrap : cfg->kernel,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
                     cudaGetLastError();
                     return STENCIL_ERR_CUDA;
                 }
-                cfg->smem_allowed = smem;
+                allowed = smem;
             }
         }
         StreamGeom g;
@@ -1660,7 +1707,9 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         g.chunk_z = chunk;
         const int64_t grid64 = (int64_t)g.tiles_x * g.tiles_y * ((span + chunk - 1) / chunk);
         if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
-        if (cfg->launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
+        const cudaError_t err = wrap ? cfg->launch_wrap(p, map0, map_xs, map_ys, dst, g, (int)grid64, smem, st)
+                                     : cfg->launch(p, *map, dst, g, (int)grid64, smem, st);
+        if (err != cudaSuccess) return STENCIL_ERR_CUDA;
         p->launches++;
         return STENCIL_OK;
     }
@@ -1838,20 +1887,31 @@ int apply_periodic_corrected(stencil_plan_s* p, const T* in, T* out, T* other, i
 // A periodic 3D star of radius <= 4 whose rows are a whole number of 128-column tiles is swept by the
 // kernel that wraps all three axes itself: no correction pass, no padded copy.
 bool stream_wrap_ok(const stencil_plan_s* p) {
-    return !p->f64 && p->ndim == 3 && p->shape == STENCIL_STAR && p->variant == STENCIL_VARIANT_STREAM &&
-           p->stream_cfg && p->stream_cfg->launch_wrap && p->nx % kStreamTX == 0 && wrap_correction_fits(p);
+    if (p->ndim != 3 || p->shape != STENCIL_STAR || p->variant != STENCIL_VARIANT_STREAM || !wrap_correction_fits(p))
+        return false;
+    if (p->f64) return p->stream64_cfg && p->stream64_cfg->launch_wrap && p->nx % kStream64TX == 0;
+    return p->stream_cfg && p->stream_cfg->launch_wrap && p->nx % kStreamTX == 0;
 }
 
-int apply_periodic_inkernel(stencil_plan_s* p, const float* in, float* out, int steps, cudaStream_t st) {
-    const float* src = in;
+int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStream_t st, int begin, int end);
+inline int wrapped_sweep(stencil_plan_s* p, const float* src, float* dst, cudaStream_t st) {
+    return launch_stream(p, src, dst, st);
+}
+inline int wrapped_sweep(stencil_plan_s* p, const double* src, double* dst, cudaStream_t st) {
+    return launch_sweep_f64(p, src, dst, st, 0, 0);
+}
+
+template <typename T>
+int apply_periodic_inkernel(stencil_plan_s* p, const T* in, T* out, T* other, int steps, cudaStream_t st) {
+    const T* src = in;
     for (int k = 0; k < steps; ++k) {
-        float* dst = ((steps - 1 - k) % 2 == 0) ? out : p->scratch;
+        T* dst = ((steps - 1 - k) % 2 == 0) ? out : other;
         int rc;
         {
             ScopedGridView view(p, p->nz, p->ny, p->nx, 0, STENCIL_ZERO);
             p->stream_wrap = true;
             p->chained = p->chain_launches && k > 0;
-            rc = launch_stream(p, src, dst, st);
+            rc = wrapped_sweep(p, src, dst, st);
             p->stream_wrap = false;
         }
         if (rc != STENCIL_OK) return rc;
@@ -2219,7 +2279,7 @@ int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void
         const int depth = p->fused_cfg ? p->fused_cfg->T : p->fused2d_cfg ? p->fused2d_cfg->T : 1;
         if (steps > 1 && depth > 1 && p->periodic_route != 1)
             return apply_periodic_fused(p, in, out, p->scratch, steps, depth, st);
-        if (p->periodic_route == 0 && stream_wrap_ok(p)) return apply_periodic_inkernel(p, in, out, steps, st);
+        if (p->periodic_route == 0 && stream_wrap_ok(p)) return apply_periodic_inkernel(p, in, out, p->scratch, steps, st);
         if (use_wrap_correction(p, steps)) return apply_periodic_corrected(p, in, out, p->scratch, steps, st);
         if (steps > 1) return apply_periodic(p, in, out, steps, st);
     }
@@ -2318,6 +2378,8 @@ int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps
         const int depth = p->fused2d64_cfg ? p->fused2d64_cfg->T : 1;
         if (steps > 1 && depth > 1 && p->periodic_route != 1)
             return apply_periodic_fused(p, in, out, p->scratch64, steps, depth, st);
+        if (p->periodic_route == 0 && stream_wrap_ok(p))
+            return apply_periodic_inkernel(p, in, out, p->scratch64, steps, st);
         if (use_wrap_correction(p, steps)) return apply_periodic_corrected(p, in, out, p->scratch64, steps, st);
         if (steps > 1) return apply_periodic(p, in, out, steps, st);
     }
