@@ -314,6 +314,24 @@ def test_wide_star_fp64_kernels_match_oracle(R, dims, chunk, stages):
         assert float(np.max(np.abs(got - want))) <= wl.tolerance(w, float(np.abs(a).max()), 2)
 
 
+@pytest.mark.parametrize("dims,R,box,steps", [
+    ((32, 40, 128), 1, False, 1), ((32, 40, 128), 1, False, 4), ((20, 30, 256), 3, False, 2),
+    ((33, 50, 128), 1, True, 2), ((40, 260), 2, False, 3), ((64, 256), 1, True, 5),
+])
+def test_apply_host_on_periodic_plans(dims, R, box, steps):
+    """The host-buffer entry point takes the same periodic routes as the device one."""
+    nd = len(dims)
+    w = (wl.random_box_weights if box else wl.random_star_weights)(nd, R, 5)
+    a = wl.normal_field(dims, 6)
+    src = torch.from_numpy(a).pin_memory()
+    dst = torch.empty_like(src).pin_memory()
+    with b.Plan(dims, R, b.BOX if box else b.STAR, w, b.PERIODIC) as p:
+        p.apply_host(src, dst, steps, torch.cuda.current_stream().cuda_stream)
+        assert p.query_status() == b.OK
+    want = oracle.apply(a, w, b.PERIODIC, steps)
+    assert float(np.max(np.abs(dst.numpy() - want))) <= wl.tolerance(w, float(np.abs(a).max()), steps)
+
+
 # ------------------------------------- periodic boundary wrapped inside the sweep --
 @pytest.mark.parametrize("R", [1, 2, 3, 4])
 @pytest.mark.parametrize("dims,chunk_z,knobs", [
