@@ -87,7 +87,9 @@ struct StreamShape {
     // the tile's rows (ROWS x 4 cells each) and the R rows above and below it (R x PX cells each).
     static constexpr int XS_BYTES = (ROWS * 16 + 127) / 128 * 128;
     static constexpr int YS_BYTES = (R * StreamHalo<R>::PX * 4 + 127) / 128 * 128;
-    static constexpr int STAGE_BYTES = 2 * XS_BYTES + 2 * YS_BYTES;
+    // ... and, for boxes, the four corners of the halo (4 columns x R rows each)
+    static constexpr int CS_BYTES = (R * 16 + 127) / 128 * 128;
+    static constexpr int STAGE_BYTES = 2 * XS_BYTES + 2 * YS_BYTES + 4 * CS_BYTES;
 };
 
 // Calls f(integral_constant<int, 0>) ... f(integral_constant<int, N-1>) in order and
@@ -205,20 +207,21 @@ __device__ __forceinline__ void gather_row_split(const float* base, int o_rowp, 
     }
 }
 
-// WRAP: the sweep of a periodic grid (stars of radius <= 4, rows a whole number of tiles).  z wraps
+// WRAP: the sweep of a periodic grid (stars of radius <= 4, boxes of radius <= 2, rows a whole number of tiles).  z wraps
 // in the plane coordinate of the TMA loads (every plane is a load of its own).  A tile at an x or y
 // face gets, beside each plane, the cells its halo would hold on a torus (see StreamShape), and
 // its consumer warps read the halo columns of their centre rows straight from there (a tile in the
 // middle of a row reads them from the plane, as ever: one pointer select per row); the halo rows,
 // which only the few tiles at a y face need, are copied over the zeros TMA filled in, every warp
-// copying its own columns of the rows it is about to read.  The corners of the halo stay zero: a
-// star does not read them.
+// copying its own columns of the rows it is about to read.  A star does not read the corners of
+// the halo; a box does, so its tiles at an x and a y face get them as four more small blocks, which
+// go into the halo rows of the staged column blocks in the same step.
 template <int R, bool BOX, int K, int NW, bool WRAP>
 __device__ __forceinline__ void
 stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtensorMap& tmap_ys,
-            float* __restrict__ out, const StreamGeom& g, const StarWeights<R>& sw,
+            const CUtensorMap& tmap_cs, float* __restrict__ out, const StreamGeom& g, const StarWeights<R>& sw,
             const BoxWeights<BOX ? R : 0>& bw, int* __restrict__ status) {
-    static_assert(!WRAP || (!BOX && R <= 4), "WRAP: stars of radius <= 4");
+    static_assert(!WRAP || R <= 4, "WRAP: 4-column halos");
     using S = StreamShape<R, K, NW>;
     constexpr int PX = StreamHalo<R>::PX;
     constexpr int HX = StreamHalo<R>::HX;
@@ -281,8 +284,9 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
                         zc = zc < 0 ? zc + g.nz : (zc >= g.nz ? zc - g.nz : zc);
                         const uint32_t bar = full0 + 8 * s;
                         unsigned char* slot = ring + (size_t)s * SLOT_BYTES;
+                        const int ncorner = BOX ? ((int)edge_l + (int)edge_r) * ((int)edge_t + (int)edge_b) : 0;
                         mbar_arrive_expect_tx(bar, S::BOX_BYTES + ((int)edge_l + (int)edge_r) * S::ROWS * 16 +
-                                                       ((int)edge_t + (int)edge_b) * R * PX * 4);
+                                                       ((int)edge_t + (int)edge_b) * R * PX * 4 + ncorner * R * 16);
                         tma_load_3d(smem_addr(slot), &tmap_in, bar, x0 - HX, y0 - R, zc);
                         unsigned char* stage = slot + S::PLANE_BYTES;
                         if (edge_l) tma_load_3d(smem_addr(stage), &tmap_xs, bar, g.nx - 4, y0 - R, zc);
@@ -290,6 +294,13 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
                         if (edge_t) tma_load_3d(smem_addr(stage + 2 * S::XS_BYTES), &tmap_ys, bar, x0 - HX, g.ny - R, zc);
                         if (edge_b)
                             tma_load_3d(smem_addr(stage + 2 * S::XS_BYTES + S::YS_BYTES), &tmap_ys, bar, x0 - HX, 0, zc);
+                        if constexpr (BOX) {                       // corners: (left, right) x (top, bottom)
+                            unsigned char* cs = stage + 2 * S::XS_BYTES + 2 * S::YS_BYTES;
+                            if (edge_l && edge_t) tma_load_3d(smem_addr(cs), &tmap_cs, bar, g.nx - 4, g.ny - R, zc);
+                            if (edge_r && edge_t) tma_load_3d(smem_addr(cs + S::CS_BYTES), &tmap_cs, bar, 0, g.ny - R, zc);
+                            if (edge_l && edge_b) tma_load_3d(smem_addr(cs + 2 * S::CS_BYTES), &tmap_cs, bar, g.nx - 4, 0, zc);
+                            if (edge_r && edge_b) tma_load_3d(smem_addr(cs + 3 * S::CS_BYTES), &tmap_cs, bar, 0, 0, zc);
+                        }
                     } else {
                         mbar_arrive_expect_tx(full0 + 8 * s, S::BOX_BYTES);
                         tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_BYTES), &tmap_in, full0 + 8 * s,
@@ -471,12 +482,56 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
                 if (i >= nplanes) return true;
                 if (!mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) return false;
                 const float* pl = reinterpret_cast<const float*>(ring + (size_t)s * SLOT_BYTES);
+                if constexpr (WRAP) {
+                    if (edge_t || edge_b) {                            // uniform over the CTA
+                        // The halo rows inside this warp's window of rows: the lane's own columns, the row's own
+                        // halo columns (first and last lane; a tile in the middle of a row reads them) and,
+                        // at an x face, the corner cells, which go into the halo rows of the column blocks.
+                        float* plw = reinterpret_cast<float*>(ring + (size_t)s * SLOT_BYTES);
+                        float* stw = plw + S::PLANE_BYTES / 4;
+                        const float* ys = stw + 2 * S::XS_BYTES / 4;
+                        const float* cs = ys + 2 * S::YS_BYTES / 4;
+#pragma unroll
+                        for (int rr = 0; rr < R; ++rr) {
+#pragma unroll
+                            for (int side = 0; side < 2; ++side) {     // 0: rows above the grid, 1: rows below it
+                                const int r = side == 0 ? rr : row_b + rr;
+                                const bool mine = (side == 0 ? edge_t : edge_b) && r < S::ROWS && r >= row0 &&
+                                                  r < row0 + K + 2 * R;
+                                if (!mine) continue;
+                                const float* yrow = ys + side * (S::YS_BYTES / 4) + rr * PX;
+                                *reinterpret_cast<float4*>(plw + r * PX + HX + 4 * lane) =
+                                    *reinterpret_cast<const float4*>(yrow + HX + 4 * lane);
+                                if (lane == 0) *reinterpret_cast<float4*>(plw + r * PX) = *reinterpret_cast<const float4*>(yrow);
+                                if (lane == 31)
+                                    *reinterpret_cast<float4*>(plw + r * PX + HX + kStreamTX) =
+                                        *reinterpret_cast<const float4*>(yrow + HX + kStreamTX);
+                                if (edge_l && lane == 1)
+                                    *reinterpret_cast<float4*>(stw + r * 4) =
+                                        *reinterpret_cast<const float4*>(cs + (2 * side) * (S::CS_BYTES / 4) + rr * 4);
+                                if (edge_r && lane == 2)
+                                    *reinterpret_cast<float4*>(stw + S::XS_BYTES / 4 + r * 4) =
+                                        *reinterpret_cast<const float4*>(cs + (2 * side + 1) * (S::CS_BYTES / 4) + rr * 4);
+                            }
+                        }
+                        // later TMA copies into this slot must not overtake these stores
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                    }
+                }
                 const float* colp = pl + row0 * PX + HX + 4 * lane;
                 float v[K + 2 * R][4 + 2 * R];
 #pragma unroll
                 for (int kk = 0; kk < K + 2 * R; ++kk) {
                     const float4 ctr = *reinterpret_cast<const float4*>(colp + kk * PX);
-                    gather_row<R>(colp + kk * PX, pl + (row0 + kk) * PX, lane, ctr, v[kk]);
+                    if constexpr (WRAP) {
+                        const int o_row = (row0 + kk) * PX;
+                        const int o_xs = S::PLANE_BYTES / 4 + (row0 + kk) * 4;
+                        gather_row_split<R>(pl, o_row + HX + 4 * lane, edge_l ? o_xs : o_row,
+                                            edge_r ? o_xs + S::XS_BYTES / 4 : o_row + HX + kStreamTX, lane, ctr, v[kk]);
+                    } else {
+                        gather_row<R>(colp + kk * PX, pl + (row0 + kk) * PX, lane, ctr, v[kk]);
+                    }
                 }
                 __syncwarp();
                 mbar_arrive_if(lane == 0, empty0 + 8 * s);
@@ -544,18 +599,30 @@ stencil_stream_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                       const __grid_constant__ StarWeights<R> sw,
                       const __grid_constant__ BoxWeights<BOX ? R : 0> bw,
                       int* __restrict__ status) {
-    stream_body<R, BOX, K, NW, false>(tmap_in, tmap_in, tmap_in, out, g, sw, bw, status);
+    stream_body<R, BOX, K, NW, false>(tmap_in, tmap_in, tmap_in, tmap_in, out, g, sw, bw, status);
 }
 
-// The sweep of a periodic grid: tmap_xs has boxes of 4 columns x ROWS rows, tmap_ys of PX columns x R rows.
-template <int R, int K, int NW, int MINB>
-__global__ void __launch_bounds__((NW + 1) * 32, MINB)
+// The sweep of a periodic grid: tmap_xs has boxes of 4 columns x ROWS rows, tmap_ys of PX columns x R rows,
+// tmap_cs (boxes only) of 4 columns x R rows.
+// The boxes need their register count capped to keep the CTAs per SM of the zero-boundary kernels
+// (left alone the 27-point box takes 80 registers instead of 64 and the 125-point box 108 instead of 56).
+template <int R, bool BOX, int K, int NW, int MINB>
+constexpr int wrap_min_ctas() {
+    if (!BOX) return MINB;
+    const int threads = (NW + 1) * 32;
+    const int regs = R == 1 ? (K == 1 ? 48 : K == 2 ? 64 : 96) : (K == 1 ? 56 : 96);   // of the zero-boundary kernels
+    const int n = 65536 / (threads * regs);
+    return n < 1 ? 1 : (n > 4 ? 4 : n);
+}
+
+template <int R, bool BOX, int K, int NW, int MINB>
+__global__ void __launch_bounds__((NW + 1) * 32, wrap_min_ctas<R, BOX, K, NW, MINB>())
 stencil_stream_wrap_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_xs,
-                           const __grid_constant__ CUtensorMap tmap_ys, float* __restrict__ out,
-                           const StreamGeom g, const __grid_constant__ StarWeights<R> sw,
-                           int* __restrict__ status) {
-    const BoxWeights<0> bw = {};
-    stream_body<R, false, K, NW, true>(tmap_in, tmap_xs, tmap_ys, out, g, sw, bw, status);
+                           const __grid_constant__ CUtensorMap tmap_ys, const __grid_constant__ CUtensorMap tmap_cs,
+                           float* __restrict__ out, const StreamGeom g,
+                           const __grid_constant__ StarWeights<R> sw,
+                           const __grid_constant__ BoxWeights<BOX ? R : 0> bw, int* __restrict__ status) {
+    stream_body<R, BOX, K, NW, true>(tmap_in, tmap_xs, tmap_ys, tmap_cs, out, g, sw, bw, status);
 }
 
 }  // namespace stencil

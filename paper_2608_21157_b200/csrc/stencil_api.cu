@@ -103,12 +103,13 @@ struct StreamConfig {
     const void* kernel;
     cudaError_t (*launch)(const struct stencil_plan_s*, const StreamConfig&, const CUtensorMap&,
                           float*, const StreamGeom&, int grid, size_t smem, cudaStream_t);
-    // the sweep of a periodic grid inside the kernel (stars of radius <= 4; null otherwise)
+    // the sweep of a periodic grid inside the kernel (stars of radius <= 4 and the boxes; null otherwise)
     const void* kernel_wrap;
     int stage_bytes;                         // per ring slot, beside the plane
     mutable size_t smem_allowed_wrap;
     cudaError_t (*launch_wrap)(const struct stencil_plan_s*, const CUtensorMap&, const CUtensorMap&,
-                               const CUtensorMap&, float*, const StreamGeom&, int grid, size_t smem, cudaStream_t);
+                               const CUtensorMap&, const CUtensorMap&, float*, const StreamGeom&, int grid,
+                               size_t smem, cudaStream_t);
 };
 
 // ---------------------------------------------------------------------------
@@ -309,21 +310,30 @@ cudaError_t launch_stream_t(const stencil_plan_s* p, const StreamConfig&, const 
                          st, p->chained, map, out, g, sw, bw, p->d_status);
 }
 
-template <int R, int K, int NW, int MINB>
+template <int R, bool BOX, int K, int NW, int MINB>
 cudaError_t launch_stream_wrap_t(const stencil_plan_s* p, const CUtensorMap& map, const CUtensorMap& map_xs,
-                                 const CUtensorMap& map_ys, float* out, const StreamGeom& g, int grid, size_t smem,
-                                 cudaStream_t st) {
+                                 const CUtensorMap& map_ys, const CUtensorMap& map_cs, float* out,
+                                 const StreamGeom& g, int grid, size_t smem, cudaStream_t st) {
     StarWeights<R> sw;
+    BoxWeights<BOX ? R : 0> bw;
     std::memset(&sw, 0, sizeof(sw));
-    sw.c = dense_w(p, 0, 0, 0);
-    for (int d = -R; d <= R; ++d) {
-        if (d == 0) continue;
-        sw.x[d + R] = dense_w(p, 0, 0, d);
-        sw.y[d + R] = dense_w(p, 0, d, 0);
-        sw.z[d + R] = dense_w(p, d, 0, 0);
+    std::memset(&bw, 0, sizeof(bw));
+    if (!BOX) {
+        sw.c = dense_w(p, 0, 0, 0);
+        for (int d = -R; d <= R; ++d) {
+            if (d == 0) continue;
+            sw.x[d + R] = dense_w(p, 0, 0, d);
+            sw.y[d + R] = dense_w(p, 0, d, 0);
+            sw.z[d + R] = dense_w(p, d, 0, 0);
+        }
+    } else {
+        constexpr int RB = BOX ? R : 0;
+        for (int a = -RB; a <= RB; ++a)
+            for (int b = -RB; b <= RB; ++b)
+                for (int c = -RB; c <= RB; ++c) bw.w[a + RB][b + RB][c + RB] = dense_w(p, a, b, c);
     }
-    return launch_kernel(&stencil_stream_wrap_kernel<R, K, NW, MINB>, grid, StreamShape<R, K, NW>::THREADS, smem, st,
-                         p->chained, map, map_xs, map_ys, out, g, sw, p->d_status);
+    return launch_kernel(&stencil_stream_wrap_kernel<R, BOX, K, NW, MINB>, grid, StreamShape<R, K, NW>::THREADS, smem,
+                         st, p->chained, map, map_xs, map_ys, map_cs, out, g, sw, bw, p->d_status);
 }
 
 template <int R, bool BOX, int K, int NW, int MINB>
@@ -339,9 +349,9 @@ StreamConfig make_cfg() {
     c.kernel = reinterpret_cast<const void*>(&stencil_stream_kernel<R, BOX, K, NW, MINB>);
     c.launch = &launch_stream_t<R, BOX, K, NW, MINB>;
     c.kernel_wrap = nullptr; c.launch_wrap = nullptr; c.stage_bytes = 0; c.smem_allowed_wrap = 0;
-    if constexpr (!BOX && R <= 4) {
-        c.kernel_wrap = reinterpret_cast<const void*>(&stencil_stream_wrap_kernel<R, K, NW, MINB>);
-        c.launch_wrap = &launch_stream_wrap_t<R, K, NW, MINB>;
+    if constexpr (R <= 4) {
+        c.kernel_wrap = reinterpret_cast<const void*>(&stencil_stream_wrap_kernel<R, BOX, K, NW, MINB>);
+        c.launch_wrap = &launch_stream_wrap_t<R, BOX, K, NW, MINB>;
         c.stage_bytes = S::STAGE_BYTES;
     }
     return c;
@@ -729,7 +739,7 @@ int get_tensor_map(stencil_plan_s* p, const void* cfg, int box_x, int box_y, con
                      box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return STENCIL_ERR_CUDA;
-    if (p->maps.size() >= 8) p->maps.erase(p->maps.begin());
+    if (p->maps.size() >= 16) p->maps.erase(p->maps.begin());
     p->maps.push_back(e);
     *out = &p->maps.back().map;
     return STENCIL_OK;
@@ -881,7 +891,7 @@ int launch_stream_wrap(stencil_plan_s* p, const StreamConfig* cfg, int stages, c
     if (!cfg->launch_wrap) return STENCIL_ERR_UNSUPPORTED;
     const char* key = reinterpret_cast<const char*>(cfg);
     const CUtensorMap* m = nullptr;
-    CUtensorMap map, map_xs, map_ys;
+    CUtensorMap map, map_xs, map_ys, map_cs;
     int rc;
     if ((rc = get_tensor_map(p, key, cfg->px, cfg->box_rows, src, &m)) != STENCIL_OK) return rc;
     map = *m;
@@ -889,6 +899,11 @@ int launch_stream_wrap(stencil_plan_s* p, const StreamConfig* cfg, int stages, c
     map_xs = *m;
     if ((rc = get_tensor_map(p, key + 2, cfg->px, p->radius, src, &m)) != STENCIL_OK) return rc;
     map_ys = *m;
+    map_cs = map;                                   // the corner blocks: boxes only
+    if (cfg->box) {
+        if ((rc = get_tensor_map(p, key + 3, 4, p->radius, src, &m)) != STENCIL_OK) return rc;
+        map_cs = *m;
+    }
     const size_t smem = (size_t)stages * (cfg->plane_bytes + cfg->stage_bytes) + 128 + 2 * kMaxStages * sizeof(uint64_t);
     if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
     int dev = -1;
@@ -923,7 +938,8 @@ int launch_stream_wrap(stencil_plan_s* p, const StreamConfig* cfg, int stages, c
     g.wait_polls = p->wait_polls; g.drop_plane = -1;
     const int64_t grid64 = (int64_t)g.tiles_x * g.tiles_y * ((p->nz + chunk - 1) / chunk);
     if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
-    if (cfg->launch_wrap(p, map, map_xs, map_ys, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
+    if (cfg->launch_wrap(p, map, map_xs, map_ys, map_cs, dst, g, (int)grid64, smem, st) != cudaSuccess)
+        return STENCIL_ERR_CUDA;
     p->launches++;
     return STENCIL_OK;
 }
@@ -1530,7 +1546,7 @@ int get_tensor_map_f64(stencil_plan_s* p, const void* cfg, int box_x, int box_y,
                      estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return STENCIL_ERR_CUDA;
-    if (p->maps.size() >= 8) p->maps.erase(p->maps.begin());
+    if (p->maps.size() >= 16) p->maps.erase(p->maps.begin());
     p->maps.push_back(e);
     *out = &p->maps.back().map;
     return STENCIL_OK;
@@ -1884,12 +1900,12 @@ int apply_periodic_corrected(stencil_plan_s* p, const T* in, T* out, T* other, i
     return STENCIL_OK;
 }
 
-// A periodic 3D star of radius <= 4 whose rows are a whole number of 128-column tiles is swept by the
-// kernel that wraps all three axes itself: no correction pass, no padded copy.
+// A periodic 3D star of radius <= 4 or box (fp32) whose rows are a whole number of tiles is swept by
+// the kernel that wraps all three axes itself: no correction pass, no padded copy.
 bool stream_wrap_ok(const stencil_plan_s* p) {
-    if (p->ndim != 3 || p->shape != STENCIL_STAR || p->variant != STENCIL_VARIANT_STREAM || !wrap_correction_fits(p))
-        return false;
-    if (p->f64) return p->stream64_cfg && p->stream64_cfg->launch_wrap && p->nx % kStream64TX == 0;
+    if (p->ndim != 3 || p->variant != STENCIL_VARIANT_STREAM || !wrap_correction_fits(p)) return false;
+    if (p->f64)
+        return p->shape == STENCIL_STAR && p->stream64_cfg && p->stream64_cfg->launch_wrap && p->nx % kStream64TX == 0;
     return p->stream_cfg && p->stream_cfg->launch_wrap && p->nx % kStreamTX == 0;
 }
 

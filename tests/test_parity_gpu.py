@@ -376,6 +376,37 @@ def test_periodic_3d_star_wrapped_inside_the_sweep(R, dims, chunk_z, knobs, f64)
         assert err <= tol, f"R={R} dims={dims} steps={steps} f64={f64}: {err:.3e} > {tol:.3e}"
 
 
+@pytest.mark.parametrize("R", [1, 2])
+@pytest.mark.parametrize("dims,chunk_z,knobs", [
+    ((11, 23, 128), 0, {}),                       # one tile per row: all four corners in one tile
+    ((9, 40, 384), 4, {}),                        # three tiles per row, ragged last tile in y
+    ((6, 16, 256), 0, {}),                        # one tile in y
+    ((7, 30, 256), 3, dict(tile_y=14)),
+    ((5, 37, 128), 0, dict(rows_per_thread=1)),
+])
+def test_periodic_3d_box_wrapped_inside_the_sweep(R, dims, chunk_z, knobs):
+    """Periodic 3D boxes on rows of whole tiles: the sweep wraps x, y and z itself, corners of the halo included."""
+    w = wl.random_box_weights(3, R, 83)
+    a = wl.normal_field(dims, 84)
+    for steps in (1, 2):
+        src = torch.from_numpy(a).cuda()
+        dst = torch.full_like(src, float("nan"))
+        try:
+            plan = b.Plan(dims, R, b.BOX, w, b.PERIODIC, chunk_z=chunk_z or None, **knobs)
+        except b.StencilError as e:                    # a tile shape this radius does not have
+            assert e.status == b.ERR_UNSUPPORTED and knobs
+            return
+        with plan as p:
+            p.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
+            assert p.query_status() == b.OK
+            assert p.launches == steps
+        got = dst.cpu().numpy()
+        want = oracle.apply(a, w, b.PERIODIC, steps)
+        tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+        err = float(np.max(np.abs(got - want)))
+        assert err <= tol, f"R={R} dims={dims} steps={steps}: {err:.3e} > {tol:.3e}"
+
+
 # ------------------------------------------- periodic boundary under temporal blocking --
 @pytest.mark.parametrize("dims,R,knobs", [
     ((21, 37, 256), 1, {}),                                         # one 256-wide region per row, T = 2
