@@ -89,8 +89,8 @@ enum {
     STENCIL_KEY_FUSED_TILE_Y = 13,   /* set/get: region height of fused 3D passes, 16, 20 or 32 (0 = auto) */
     STENCIL_KEY_PERIODIC_ROUTE = 14, /* set/get: how the tiled kernels handle a periodic boundary
                                       where the sweep does not wrap by itself (it does for 3D
-                                      stars of radius <= 4 and fp32 3D boxes with nx a multiple
-                                      of 128, in FP64 of 64, unless this key is 1 or 2).
+                                      stars of radius <= 4 and 3D boxes with nx a multiple of
+                                      128, in FP64 of 64, unless this key is 1 or 2).
                                       1 = sweep from a padded copy with wrapped halos; 2 = zero-
                                       boundary sweep plus a correction of the points within R of
                                       a face (needs every extent >= 2R, else as 1); 0 (default)

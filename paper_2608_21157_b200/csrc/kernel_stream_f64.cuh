@@ -40,7 +40,8 @@ struct Stream64Shape {
     // fp32 kernel: 4 columns x ROWS rows beyond either end of the rows, R rows x PX columns above and below
     static constexpr int XS_BYTES = (ROWS * 32 + 127) / 128 * 128;
     static constexpr int YS_BYTES = (R * StreamHalo64<R>::PX * 8 + 127) / 128 * 128;
-    static constexpr int STAGE_BYTES = 2 * XS_BYTES + 2 * YS_BYTES;
+    static constexpr int CS_BYTES = (R * 32 + 127) / 128 * 128;      // boxes: a corner of the halo, 4 columns x R rows
+    static constexpr int STAGE_BYTES = 2 * XS_BYTES + 2 * YS_BYTES + 4 * CS_BYTES;
 };
 
 __device__ __forceinline__ double d2get(const double2& v, int m) { return m == 0 ? v.x : v.y; }
@@ -52,9 +53,9 @@ __device__ __forceinline__ double d2get(const double2& v, int m) { return m == 0
 template <int R, bool BOX, int K, int NW, bool WRAP>
 __device__ __forceinline__ void
 stream_f64_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtensorMap& tmap_ys,
-                double* __restrict__ out, const StreamGeom& g, const StarWeights64<R>& sw,
+                const CUtensorMap& tmap_cs, double* __restrict__ out, const StreamGeom& g, const StarWeights64<R>& sw,
                 const BoxWeights64<BOX ? R : 0>& bw, int* __restrict__ status) {
-    static_assert(!WRAP || (!BOX && R <= 4), "WRAP: stars of radius <= 4");
+    static_assert(!WRAP || R <= 4, "WRAP: 4-column halos");
     using S = Stream64Shape<R, K, NW>;
     constexpr int SLOT_DOUBLES = (S::PLANE_BYTES + (WRAP ? S::STAGE_BYTES : 0)) / 8;
     constexpr int PX = StreamHalo64<R>::PX;
@@ -112,8 +113,9 @@ stream_f64_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CU
                     zc = zc < 0 ? zc + g.nz : (zc >= g.nz ? zc - g.nz : zc);
                     const uint32_t bar = full0 + 8 * s;
                     double* slot = ring + (size_t)s * SLOT_DOUBLES;
+                    const int ncorner = BOX ? ((int)edge_l + (int)edge_r) * ((int)edge_t + (int)edge_b) : 0;
                     mbar_arrive_expect_tx(bar, S::PLANE_BYTES + ((int)edge_l + (int)edge_r) * S::ROWS * 32 +
-                                                   ((int)edge_t + (int)edge_b) * R * PX * 8);
+                                                   ((int)edge_t + (int)edge_b) * R * PX * 8 + ncorner * R * 32);
                     tma_load_3d(smem_addr(slot), &tmap_in, bar, x0 - HX, y0 - R, zc);
                     double* stage = slot + S::PLANE_DOUBLES;
                     if (edge_l) tma_load_3d(smem_addr(stage), &tmap_xs, bar, g.nx - 4, y0 - R, zc);
@@ -121,6 +123,13 @@ stream_f64_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CU
                     if (edge_t) tma_load_3d(smem_addr(stage + 2 * S::XS_BYTES / 8), &tmap_ys, bar, x0 - HX, g.ny - R, zc);
                     if (edge_b)
                         tma_load_3d(smem_addr(stage + (2 * S::XS_BYTES + S::YS_BYTES) / 8), &tmap_ys, bar, x0 - HX, 0, zc);
+                    if constexpr (BOX) {                           // corners: (left, right) x (top, bottom)
+                        double* cs = stage + (2 * S::XS_BYTES + 2 * S::YS_BYTES) / 8;
+                        if (edge_l && edge_t) tma_load_3d(smem_addr(cs), &tmap_cs, bar, g.nx - 4, g.ny - R, zc);
+                        if (edge_r && edge_t) tma_load_3d(smem_addr(cs + S::CS_BYTES / 8), &tmap_cs, bar, 0, g.ny - R, zc);
+                        if (edge_l && edge_b) tma_load_3d(smem_addr(cs + 2 * S::CS_BYTES / 8), &tmap_cs, bar, g.nx - 4, 0, zc);
+                        if (edge_r && edge_b) tma_load_3d(smem_addr(cs + 3 * S::CS_BYTES / 8), &tmap_cs, bar, 0, 0, zc);
+                    }
                 } else {
                     mbar_arrive_expect_tx(full0 + 8 * s, S::PLANE_BYTES);
                     tma_load_3d(smem_addr(ring + (size_t)s * S::PLANE_DOUBLES), &tmap_in, full0 + 8 * s,
@@ -271,13 +280,64 @@ stream_f64_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CU
                 if (i >= nplanes) return true;
                 if (!mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) return false;
                 const double* pl = ring + (size_t)s * SLOT_DOUBLES;
+                if constexpr (WRAP) {
+                    if (edge_t || edge_b) {                            // uniform over the CTA
+                        // the halo rows inside this warp's window of rows: the lane's own columns, the rows' own
+                        // halo columns (first and last two lanes) and, at an x face, the corner cells, which go
+                        // into the halo rows of the column blocks
+                        double* plw = ring + (size_t)s * SLOT_DOUBLES;
+                        double* stw = plw + S::PLANE_DOUBLES;
+                        const double* ys = stw + 2 * S::XS_BYTES / 8;
+                        const double* cs = ys + 2 * S::YS_BYTES / 8;
+#pragma unroll
+                        for (int rr = 0; rr < R; ++rr) {
+#pragma unroll
+                            for (int side = 0; side < 2; ++side) {     // 0: rows above the grid, 1: rows below it
+                                const int r = side == 0 ? rr : row_b + rr;
+                                const bool mine = (side == 0 ? edge_t : edge_b) && r < S::ROWS && r >= row0 &&
+                                                  r < row0 + K + 2 * R;
+                                if (!mine) continue;
+                                const double* yrow = ys + side * (S::YS_BYTES / 8) + rr * PX;
+                                *reinterpret_cast<double2*>(plw + r * PX + HX + 2 * lane) =
+                                    *reinterpret_cast<const double2*>(yrow + HX + 2 * lane);
+                                if (lane < 2)                          // the 4 halo columns left of the tile
+                                    *reinterpret_cast<double2*>(plw + r * PX + 2 * lane) =
+                                        *reinterpret_cast<const double2*>(yrow + 2 * lane);
+                                if (lane >= 30)                        // ... and right of it
+                                    *reinterpret_cast<double2*>(plw + r * PX + HX + kStream64TX + 2 * (lane - 30)) =
+                                        *reinterpret_cast<const double2*>(yrow + HX + kStream64TX + 2 * (lane - 30));
+                                if (edge_l && (lane == 2 || lane == 3))
+                                    *reinterpret_cast<double2*>(stw + r * 4 + 2 * (lane - 2)) =
+                                        *reinterpret_cast<const double2*>(cs + (2 * side) * (S::CS_BYTES / 8) + rr * 4 +
+                                                                          2 * (lane - 2));
+                                if (edge_r && (lane == 4 || lane == 5))
+                                    *reinterpret_cast<double2*>(stw + S::XS_BYTES / 8 + r * 4 + 2 * (lane - 4)) =
+                                        *reinterpret_cast<const double2*>(cs + (2 * side + 1) * (S::CS_BYTES / 8) + rr * 4 +
+                                                                          2 * (lane - 4));
+                            }
+                        }
+                        // later TMA copies into this slot must not overtake these stores
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                    }
+                }
                 const double* colp = pl + row0 * PX + HX + 2 * lane;
                 double v[K + 2 * R][NV];
 #pragma unroll
                 for (int kk = 0; kk < K + 2 * R; ++kk)
 #pragma unroll
                     for (int t = 0; t < NV / 2; ++t) {
-                        const double2 dd = *reinterpret_cast<const double2*>(colp + kk * PX - HW + 2 * t);
+                        double2 dd;
+                        if constexpr (WRAP) {
+                            const int c = 2 * lane - HW + 2 * t;       // first tile column of this double2
+                            int o = (row0 + kk) * PX + HX + c;
+                            const int o_xs = S::PLANE_DOUBLES + (row0 + kk) * 4;
+                            if (2 * t < HW && edge_l && c < 0) o = o_xs + 4 + c;
+                            if (2 * t >= HW + 2 && edge_r && c >= kStream64TX) o = o_xs + S::XS_BYTES / 8 + c - kStream64TX;
+                            dd = *reinterpret_cast<const double2*>(pl + o);
+                        } else {
+                            dd = *reinterpret_cast<const double2*>(colp + kk * PX - HW + 2 * t);
+                        }
                         v[kk][2 * t] = dd.x;
                         v[kk][2 * t + 1] = dd.y;
                     }
@@ -332,19 +392,21 @@ stencil_stream_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
                           const __grid_constant__ StarWeights64<R> sw,
                           const __grid_constant__ BoxWeights64<BOX ? R : 0> bw,
                           int* __restrict__ status) {
-    stream_f64_body<R, BOX, K, NW, false>(tmap_in, tmap_in, tmap_in, out, g, sw, bw, status);
+    stream_f64_body<R, BOX, K, NW, false>(tmap_in, tmap_in, tmap_in, tmap_in, out, g, sw, bw, status);
 }
 
 // The sweep of a periodic grid: tmap_xs has boxes of 4 columns x ROWS rows, tmap_ys of PX columns x R rows.
-template <int R, int K, int NW, int MINB>
-__global__ void __launch_bounds__((NW + 1) * 32, MINB)
+// (the 27-point box is held to two CTAs per SM like its zero-boundary kernel: left alone it takes 120 registers;
+// the 125-point box takes 84 instead of 68 and spills when it is held to the three CTAs those 68 allow)
+template <int R, bool BOX, int K, int NW, int MINB>
+__global__ void __launch_bounds__((NW + 1) * 32, (BOX && R == 1) ? 2 : MINB)
 stencil_stream_f64_wrap_kernel(const __grid_constant__ CUtensorMap tmap_in,
                                const __grid_constant__ CUtensorMap tmap_xs,
-                               const __grid_constant__ CUtensorMap tmap_ys, double* __restrict__ out,
+                               const __grid_constant__ CUtensorMap tmap_ys,
+                               const __grid_constant__ CUtensorMap tmap_cs, double* __restrict__ out,
                                const StreamGeom g, const __grid_constant__ StarWeights64<R> sw,
-                               int* __restrict__ status) {
-    const BoxWeights64<0> bw = {};
-    stream_f64_body<R, false, K, NW, true>(tmap_in, tmap_xs, tmap_ys, out, g, sw, bw, status);
+                               const __grid_constant__ BoxWeights64<BOX ? R : 0> bw, int* __restrict__ status) {
+    stream_f64_body<R, BOX, K, NW, true>(tmap_in, tmap_xs, tmap_ys, tmap_cs, out, g, sw, bw, status);
 }
 
 }  // namespace stencil

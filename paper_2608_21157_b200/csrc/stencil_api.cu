@@ -207,7 +207,8 @@ struct Stream64Config {
     int stage_bytes;                         // per ring slot, beside the plane
     mutable size_t smem_allowed_wrap;
     cudaError_t (*launch_wrap)(const struct stencil_plan_s*, const CUtensorMap&, const CUtensorMap&,
-                               const CUtensorMap&, double*, const StreamGeom&, int grid, size_t smem, cudaStream_t);
+                               const CUtensorMap&, const CUtensorMap&, double*, const StreamGeom&, int grid,
+                               size_t smem, cudaStream_t);
 };
 
 constexpr int kMaxFuseLevels = 4;          // deepest temporal blocking of any fused kernel
@@ -1415,21 +1416,30 @@ cudaError_t launch_stream64_t(const stencil_plan_s* p, const CUtensorMap& map, d
                          smem, st, p->chained, map, out, g, sw, bw, p->d_status);
 }
 
-template <int R, int K, int NW, int MINB>
+template <int R, bool BOX, int K, int NW, int MINB>
 cudaError_t launch_stream64_wrap_t(const stencil_plan_s* p, const CUtensorMap& map, const CUtensorMap& map_xs,
-                                   const CUtensorMap& map_ys, double* out, const StreamGeom& g, int grid,
-                                   size_t smem, cudaStream_t st) {
+                                   const CUtensorMap& map_ys, const CUtensorMap& map_cs, double* out,
+                                   const StreamGeom& g, int grid, size_t smem, cudaStream_t st) {
     StarWeights64<R> sw;
+    BoxWeights64<BOX ? R : 0> bw;
     std::memset(&sw, 0, sizeof(sw));
-    sw.c = dense_w64_3d(p, 0, 0, 0);
-    for (int d = -R; d <= R; ++d) {
-        if (d == 0) continue;
-        sw.x[d + R] = dense_w64_3d(p, 0, 0, d);
-        sw.y[d + R] = dense_w64_3d(p, 0, d, 0);
-        sw.z[d + R] = dense_w64_3d(p, d, 0, 0);
+    std::memset(&bw, 0, sizeof(bw));
+    if (!BOX) {
+        sw.c = dense_w64_3d(p, 0, 0, 0);
+        for (int d = -R; d <= R; ++d) {
+            if (d == 0) continue;
+            sw.x[d + R] = dense_w64_3d(p, 0, 0, d);
+            sw.y[d + R] = dense_w64_3d(p, 0, d, 0);
+            sw.z[d + R] = dense_w64_3d(p, d, 0, 0);
+        }
+    } else {
+        constexpr int RB = BOX ? R : 0;
+        for (int a = -RB; a <= RB; ++a)
+            for (int b = -RB; b <= RB; ++b)
+                for (int c = -RB; c <= RB; ++c) bw.w[a + RB][b + RB][c + RB] = dense_w64_3d(p, a, b, c);
     }
-    return launch_kernel(&stencil_stream_f64_wrap_kernel<R, K, NW, MINB>, grid, Stream64Shape<R, K, NW>::THREADS,
-                         smem, st, p->chained, map, map_xs, map_ys, out, g, sw, p->d_status);
+    return launch_kernel(&stencil_stream_f64_wrap_kernel<R, BOX, K, NW, MINB>, grid, Stream64Shape<R, K, NW>::THREADS,
+                         smem, st, p->chained, map, map_xs, map_ys, map_cs, out, g, sw, bw, p->d_status);
 }
 
 template <int R, bool BOX, int K, int NW, int MINB>
@@ -1442,9 +1452,9 @@ Stream64Config make_stream64() {
     c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
     c.launch = &launch_stream64_t<R, BOX, K, NW, MINB>;
     c.kernel_wrap = nullptr; c.launch_wrap = nullptr; c.stage_bytes = 0; c.smem_allowed_wrap = 0;
-    if constexpr (!BOX && R <= 4) {
-        c.kernel_wrap = reinterpret_cast<const void*>(&stencil_stream_f64_wrap_kernel<R, K, NW, MINB>);
-        c.launch_wrap = &launch_stream64_wrap_t<R, K, NW, MINB>;
+    if constexpr (R <= 4) {
+        c.kernel_wrap = reinterpret_cast<const void*>(&stencil_stream_f64_wrap_kernel<R, BOX, K, NW, MINB>);
+        c.launch_wrap = &launch_stream64_wrap_t<R, BOX, K, NW, MINB>;
         c.stage_bytes = S::STAGE_BYTES;
     }
     return c;
@@ -1636,7 +1646,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         // once (a later entry may move the earlier ones), and the staged halo blocks beside every plane
         const bool wrap = p->stream_wrap && cfg->launch_wrap;
         if (p->stream_wrap && !wrap) return STENCIL_ERR_UNSUPPORTED;
-        CUtensorMap map0, map_xs, map_ys;
+        CUtensorMap map0, map_xs, map_ys, map_cs;
         if (wrap) {
             const char* key = reinterpret_cast<const char*>(cfg);
             map0 = *map;
@@ -1644,6 +1654,11 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
             map_xs = *map;
             if ((rc = get_tensor_map_f64(p, key + 2, cfg->px, p->radius, src, &map)) != STENCIL_OK) return rc;
             map_ys = *map;
+            map_cs = map0;                                // the corner blocks: boxes only
+            if (cfg->box) {
+                if ((rc = get_tensor_map_f64(p, key + 3, 4, p->radius, src, &map)) != STENCIL_OK) return rc;
+                map_cs = *map;
+            }
         }
         int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : (p->radius >= 3 ? 5 : 4);
         auto smem_for = [&](int s_) {
@@ -1723,7 +1738,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         g.chunk_z = chunk;
         const int64_t grid64 = (int64_t)g.tiles_x * g.tiles_y * ((span + chunk - 1) / chunk);
         if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
-        const cudaError_t err = wrap ? cfg->launch_wrap(p, map0, map_xs, map_ys, dst, g, (int)grid64, smem, st)
+        const cudaError_t err = wrap ? cfg->launch_wrap(p, map0, map_xs, map_ys, map_cs, dst, g, (int)grid64, smem, st)
                                      : cfg->launch(p, *map, dst, g, (int)grid64, smem, st);
         if (err != cudaSuccess) return STENCIL_ERR_CUDA;
         p->launches++;
@@ -1900,12 +1915,11 @@ int apply_periodic_corrected(stencil_plan_s* p, const T* in, T* out, T* other, i
     return STENCIL_OK;
 }
 
-// A periodic 3D star of radius <= 4 or box (fp32) whose rows are a whole number of tiles is swept by
+// A periodic 3D star of radius <= 4 or box whose rows are a whole number of tiles is swept by
 // the kernel that wraps all three axes itself: no correction pass, no padded copy.
 bool stream_wrap_ok(const stencil_plan_s* p) {
     if (p->ndim != 3 || p->variant != STENCIL_VARIANT_STREAM || !wrap_correction_fits(p)) return false;
-    if (p->f64)
-        return p->shape == STENCIL_STAR && p->stream64_cfg && p->stream64_cfg->launch_wrap && p->nx % kStream64TX == 0;
+    if (p->f64) return p->stream64_cfg && p->stream64_cfg->launch_wrap && p->nx % kStream64TX == 0;
     return p->stream_cfg && p->stream_cfg->launch_wrap && p->nx % kStreamTX == 0;
 }
 
