@@ -322,6 +322,7 @@ stream_f64_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CU
                     }
                 }
                 const double* colp = pl + row0 * PX + HX + 2 * lane;
+                (void)colp;                                        // the WRAP instantiation indexes from pl
                 double v[K + 2 * R][NV];
 #pragma unroll
                 for (int kk = 0; kk < K + 2 * R; ++kk)
