@@ -16,6 +16,26 @@ using Tap = TapT<float>;
 __device__ __forceinline__ float fma_t(float a, float b, float c) { return fmaf(a, b, c); }
 __device__ __forceinline__ double fma_t(double a, double b, double c) { return fma(a, b, c); }
 
+// Packed fp32 arithmetic: one instruction does two IEEE operations, each rounded exactly like
+// fmaf / * on its own half (round to nearest even, denormals kept), so results are bit-identical to
+// the scalar forms.  It halves the issue slots of FMA chains whose operands sit in aligned
+// register pairs (the two halves of a float4).  All three operands are register pairs, the
+// weight (w, w) included: it pays where a few weights serve many FMAs (the stars), not where every
+// FMA has a weight of its own (the boxes).
+__device__ __forceinline__ float2 fma2(float w, float2 v, float2 a) { return __ffma2_rn(make_float2(w, w), v, a); }
+__device__ __forceinline__ float2 mul2(float w, float2 v) { return __fmul2_rn(make_float2(w, w), v); }
+__device__ __forceinline__ float2 lo2(const float4& v) { return make_float2(v.x, v.y); }
+__device__ __forceinline__ float2 hi2(const float4& v) { return make_float2(v.z, v.w); }
+__device__ __forceinline__ float4 join4(float2 lo, float2 hi) { return make_float4(lo.x, lo.y, hi.x, hi.y); }
+// a = w * v + a on all four lanes of a float4
+__device__ __forceinline__ void fma4(float4& a, float w, const float4& v) {
+    a = join4(fma2(w, lo2(v), lo2(a)), fma2(w, hi2(v), hi2(a)));
+}
+__device__ __forceinline__ float4 fma4r(float w, const float4& v, const float4& a) {
+    return join4(fma2(w, lo2(v), lo2(a)), fma2(w, hi2(v), hi2(a)));
+}
+__device__ __forceinline__ float4 mul4(float w, const float4& v) { return join4(mul2(w, lo2(v)), mul2(w, hi2(v))); }
+
 // Grid extents as the kernels see them; 2D grids have nz == 1.
 struct Grid {
     int nz, ny, nx;

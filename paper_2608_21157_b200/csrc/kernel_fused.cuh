@@ -182,13 +182,12 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
     bool dead = false;
     int s = 0;                                     // input ring slot and its phase parity
     uint32_t ph = 0;
-    // two planes per trip, so that the parity of the level buffers is a compile-time
-    // constant in each copy of the body
-    for (int i0 = 0; i0 < nsteps; i0 += 2) {
-        static_for<2>([&](auto uc) -> bool {
-            constexpr int par = decltype(uc)::value & 1;
-            const int i = i0 + decltype(uc)::value;
-            if (i >= nsteps) return true;
+    // One plane step.  `par` is the parity of the level buffers; FAST marks a step in the steady
+    // state whose planes lie inside the grid along z at every level: nothing needs its z range
+    // checked and the last level always stores.
+    auto step = [&](auto par_c, auto fast_c, const int i) {
+            constexpr int par = decltype(par_c)::value & 1;
+            constexpr bool FAST = decltype(fast_c)::value != 0;
             if (!dead && !mbar_wait_bounded(full0 + 8 * s, ph)) {
                 dead = true;
                 atomicExch(status, kStatusTimeout);
@@ -233,45 +232,39 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                                 }
                             }
                             float4 (&Al)[2 * R] = A[l - 1][k];
-                            // the output whose centre plane this is continues from Al[R]
-                            float acc[4] = {Al[R].x, Al[R].y, Al[R].z, Al[R].w};
+                            // the output whose centre plane this is continues from Al[R]; the centre and
+                            // y taps work on aligned pairs (packed FMAs), the x taps on single lanes
+                            float4 a4 = fma4r(sw.c, ctr, Al[R]);
+#pragma unroll
+                            for (int d = 1; d <= R; ++d) {
+                                fma4(a4, sw.y[R - d], cin[k + R - d]);
+                                fma4(a4, sw.y[R + d], cin[k + R + d]);
+                            }
+                            float acc[4] = {a4.x, a4.y, a4.z, a4.w};
 #pragma unroll
                             for (int m = 0; m < 4; ++m) {
-                                float a = fmaf(sw.c, v[R + m], acc[m]);
+                                float a = acc[m];
 #pragma unroll
                                 for (int d = 1; d <= R; ++d) {
                                     a = fmaf(sw.x[R - d], v[R + m - d], a);
                                     a = fmaf(sw.x[R + d], v[R + m + d], a);
                                 }
-#pragma unroll
-                                for (int d = 1; d <= R; ++d) {
-                                    a = fmaf(sw.y[R - d], f4get(cin[k + R - d], m), a);
-                                    a = fmaf(sw.y[R + d], f4get(cin[k + R + d], m), a);
-                                }
                                 acc[m] = a;
                             }
                             // z taps: oldest output complete; the others slide down inside their FMA
-                            e[k].x = fmaf(sw.z[2 * R], ctr.x, Al[0].x);
-                            e[k].y = fmaf(sw.z[2 * R], ctr.y, Al[0].y);
-                            e[k].z = fmaf(sw.z[2 * R], ctr.z, Al[0].z);
-                            e[k].w = fmaf(sw.z[2 * R], ctr.w, Al[0].w);
+                            e[k] = fma4r(sw.z[2 * R], ctr, Al[0]);
 #pragma unroll
                             for (int j = 0; j < 2 * R - 1; ++j) {
                                 if (j == R - 1) continue;
-                                const float wz = sw.z[2 * R - 1 - j];
-                                Al[j].x = fmaf(wz, ctr.x, Al[j + 1].x);
-                                Al[j].y = fmaf(wz, ctr.y, Al[j + 1].y);
-                                Al[j].z = fmaf(wz, ctr.z, Al[j + 1].z);
-                                Al[j].w = fmaf(wz, ctr.w, Al[j + 1].w);
+                                Al[j] = fma4r(sw.z[2 * R - 1 - j], ctr, Al[j + 1]);
                             }
-                            Al[2 * R - 1] = make_float4(sw.z[0] * ctr.x, sw.z[0] * ctr.y, sw.z[0] * ctr.z,
-                                                        sw.z[0] * ctr.w);
+                            Al[2 * R - 1] = mul4(sw.z[0], ctr);
                             Al[R - 1] = make_float4(acc[0], acc[1], acc[2], acc[3]);
                         }
                         // the zero boundary holds at every time level: cells outside the grid go
                         // back to zero (nothing to do for regions and planes inside the grid)
-                        if (!warp_all_in || (!WRAP && (zl < 0 || zl >= g.nz))) {
-                            const bool z_in = WRAP || (zl >= 0 && zl < g.nz);
+                        if (!warp_all_in || (!WRAP && !FAST && (zl < 0 || zl >= g.nz))) {
+                            const bool z_in = WRAP || FAST || (zl >= 0 && zl < g.nz);
 #pragma unroll
                             for (int k = 0; k < K; ++k)
                                 if (!(z_in && ((in_mask >> k) & 1u))) e[k] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -279,7 +272,7 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
 
                         if (l == nlev) {
                             // last level of this pass: interior of the tile goes to global memory
-                            if (!dead && zl >= z0 && zl < z1) {
+                            if (!dead && (FAST || (zl >= z0 && zl < z1))) {
                                 float* op = out_col + (size_t)zl * plane_stride;
                                 if (warp_all_store) {
 #pragma unroll
@@ -327,8 +320,20 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                 }
             }
             if (++s == nstage) { s = 0; ph ^= 1; }
-            return true;
-        });
+    };
+    // two planes per trip, so that the parity of the level buffers is a compile-time constant in
+    // each copy of the step; the first 2*nlev*R steps fill the pipeline and store nothing
+    using std::integral_constant;
+    for (int i0 = 0; i0 < nsteps; i0 += 2) {
+        const bool fast = SPEC && i0 >= 2 * nlev * R && i0 + 1 < nsteps &&
+                          (WRAP || (pstart + i0 - nlev * R >= 0 && pstart + i0 + 1 - R < g.nz));
+        if (fast) {
+            step(integral_constant<int, 0>{}, integral_constant<int, 1>{}, i0);
+            step(integral_constant<int, 1>{}, integral_constant<int, 1>{}, i0 + 1);
+        } else {
+            step(integral_constant<int, 0>{}, integral_constant<int, 0>{}, i0);
+            if (i0 + 1 < nsteps) step(integral_constant<int, 1>{}, integral_constant<int, 0>{}, i0 + 1);
+        }
     }
     if (dead && tid == 0) {
         // let copies that may still be in flight land before shared memory is released

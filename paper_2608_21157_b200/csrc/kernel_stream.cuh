@@ -385,11 +385,12 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
             // rows and the centre row of at most one; it is consumed at once, so only one
             // loaded row is live at a time.  acc[k] is the output whose centre plane this is:
             // it continues from the partial sum A[k][R] that the planes below have built.
-            float acc[K][4];
+            // The y, centre and z taps work on aligned pairs of the lane's float4 (packed FMAs), and so
+            // do the x taps at even distances; the x taps at odd distances straddle the pairs and stay
+            // single FMAs.
+            float4 acc[K];
 #pragma unroll
-            for (int k = 0; k < K; ++k) {
-                acc[k][0] = A[k][R].x; acc[k][1] = A[k][R].y; acc[k][2] = A[k][R].z; acc[k][3] = A[k][R].w;
-            }
+            for (int k = 0; k < K; ++k) acc[k] = A[k][R];
             float4 done[K];
 #pragma unroll
             for (int kk = 0; kk < K + 2 * R; ++kk) {
@@ -397,10 +398,7 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
 #pragma unroll
                 for (int k = 0; k < K; ++k) {
                     const int d = kk - k - R;              // row kk is tap dy = d of output row k
-                    if (d != 0 && d >= -R && d <= R) {
-#pragma unroll
-                        for (int m = 0; m < 4; ++m) acc[k][m] = fmaf(sw.y[d + R], f4get(c, m), acc[k][m]);
-                    }
+                    if (d != 0 && d >= -R && d <= R) fma4(acc[k], sw.y[d + R], c);
                 }
                 if (kk >= R && kk < K + R) {
                     const int k = kk - R;                  // centre row of output row k
@@ -413,37 +411,44 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
                     } else {
                         gather_row<R>(colp + kk * PX, pl + (row0 + kk) * PX, lane, c, v);
                     }
+                    float4 a4 = fma4r(sw.c, c, acc[k]);
+                    // v[R + m + d] is tap dx = d of the lane's point m: for even d the operands of points
+                    // (0, 1) and (2, 3) are the register pairs the row was loaded as (R >= 3: the row's
+                    // left and right float4; the shuffled neighbours of R <= 2 have no such pairs)
+                    float2 alo = lo2(a4), ahi = hi2(a4);
+#pragma unroll
+                    for (int d = 2; d <= R; d += 2) {
+                        if constexpr (R >= 3) {
+                            alo = fma2(sw.x[R - d], make_float2(v[R - d], v[R + 1 - d]), alo);
+                            ahi = fma2(sw.x[R - d], make_float2(v[R + 2 - d], v[R + 3 - d]), ahi);
+                            alo = fma2(sw.x[R + d], make_float2(v[R + d], v[R + 1 + d]), alo);
+                            ahi = fma2(sw.x[R + d], make_float2(v[R + 2 + d], v[R + 3 + d]), ahi);
+                        }
+                    }
+                    float a[4] = {alo.x, alo.y, ahi.x, ahi.y};
 #pragma unroll
                     for (int m = 0; m < 4; ++m) {
-                        float a = fmaf(sw.c, v[R + m], acc[k][m]);
 #pragma unroll
                         for (int d = 1; d <= R; ++d) {
-                            a = fmaf(sw.x[R - d], v[R + m - d], a);
-                            a = fmaf(sw.x[R + d], v[R + m + d], a);
+                            if (R >= 3 && d % 2 == 0) continue;     // done above
+                            a[m] = fmaf(sw.x[R - d], v[R + m - d], a[m]);
+                            a[m] = fmaf(sw.x[R + d], v[R + m + d], a[m]);
                         }
-                        acc[k][m] = a;
                     }
+                    acc[k] = make_float4(a[0], a[1], a[2], a[3]);
                     // z taps: this plane is tap dz = +R of the oldest output (now complete),
                     // dz = R-1-j of the one moving into slot j, dz = -R of the new one
-                    done[k].x = fmaf(sw.z[2 * R], c.x, A[k][0].x);
-                    done[k].y = fmaf(sw.z[2 * R], c.y, A[k][0].y);
-                    done[k].z = fmaf(sw.z[2 * R], c.z, A[k][0].z);
-                    done[k].w = fmaf(sw.z[2 * R], c.w, A[k][0].w);
+                    done[k] = fma4r(sw.z[2 * R], c, A[k][0]);
 #pragma unroll
                     for (int j = 0; j < 2 * R - 1; ++j) {
                         if (j == R - 1) continue;          // that slot receives acc[k] below
-                        const float wz = sw.z[2 * R - 1 - j];
-                        A[k][j].x = fmaf(wz, c.x, A[k][j + 1].x);
-                        A[k][j].y = fmaf(wz, c.y, A[k][j + 1].y);
-                        A[k][j].z = fmaf(wz, c.z, A[k][j + 1].z);
-                        A[k][j].w = fmaf(wz, c.w, A[k][j + 1].w);
+                        A[k][j] = fma4r(sw.z[2 * R - 1 - j], c, A[k][j + 1]);
                     }
-                    A[k][2 * R - 1] = make_float4(sw.z[0] * c.x, sw.z[0] * c.y, sw.z[0] * c.z, sw.z[0] * c.w);
+                    A[k][2 * R - 1] = mul4(sw.z[0], c);
                 }
             }
 #pragma unroll
-            for (int k = 0; k < K; ++k)
-                A[k][R - 1] = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
+            for (int k = 0; k < K; ++k) A[k][R - 1] = acc[k];
             __syncwarp();
             mbar_arrive_if(lane == 0, empty0 + 8 * s);
             if (++s == nstage) { s = 0; ph ^= 1; }
@@ -537,6 +542,9 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
                 mbar_arrive_if(lane == 0, empty0 + 8 * s);
                 if (++s == nstage) { s = 0; ph ^= 1; }
 
+                // (Packed FMAs do not pay here: their three operands are register pairs, so each of the
+                // (2R+1)^3 weights would have to sit in two registers or be moved there before use; measured
+                // on 512^3, 27 taps: 703 against 755 GPoints/s.)
 #pragma unroll
                 for (int k = 0; k < K; ++k) {
 #pragma unroll
