@@ -3,19 +3,29 @@
     python -m paper_2608_21157_b200.build [--force] [--verbose]
 
 The result, ``paper_2608_21157_b200/libstencil_b200.so``, is what the Python
-binding loads.  nvcc cross-compiles, so no GPU is needed to build.
+binding loads.  nvcc cross-compiles, so no GPU is needed to build.  The host
+side is split by kernel family (``csrc/host_*.cu`` and ``csrc/abi.cu``); the
+units compile in parallel into ``paper_2608_21157_b200/build/`` and only those
+whose sources changed are recompiled.
 """
 from __future__ import annotations
 
 import os
+import re
 import shutil
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libstencil_b200.so")
-SOURCES = ["stencil_api.cu"]
+HEADER = os.path.join(os.path.dirname(HERE), "include", "stencil.h")
+SOURCES = ["abi.cu", "host_common.cu", "host_stream.cu", "host_fused.cu", "host_rows2d.cu", "host_f64.cu",
+           "host_periodic.cu"]
+FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
+         "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]
 
 
 def _nvcc() -> str:
@@ -25,27 +35,52 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found; the CUDA library cannot be built")
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _includes(path: str, seen: set) -> set:
+    """Files under csrc/ that `path` includes, directly or not."""
+    if path in seen:
+        return seen
+    seen.add(path)
+    with open(path) as f:
+        for name in re.findall(r'^#include "([^"]+)"', f.read(), flags=re.M):
+            dep = os.path.normpath(os.path.join(os.path.dirname(path), name))
+            if os.path.exists(dep):
+                _includes(dep, seen)
+    return seen
+
+
+def _stale(target: str, deps) -> bool:
+    if not os.path.exists(target):
         return True
-    t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
-    deps.append(os.path.join(os.path.dirname(HERE), "include", "stencil.h"))
+    t = os.path.getmtime(target)
     return any(os.path.getmtime(d) > t for d in deps)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    if not (force or _stale()):
-        return LIB
-    tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
-           "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
-           "--expt-relaxed-constexpr", "-cudart", "static"]
-    if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
-    subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
+    os.makedirs(OBJ, exist_ok=True)
+    nvcc = _nvcc()
+    jobs = []
+    for s in SOURCES:
+        src = os.path.join(CSRC, s)
+        obj = os.path.join(OBJ, s[:-3] + ".o")
+        if force or _stale(obj, _includes(src, set()) | {HEADER}):
+            jobs.append((src, obj))
+
+    def compile_one(job):
+        src, obj = job
+        tmp = obj + f".tmp{os.getpid()}"
+        cmd = [nvcc] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", "-o", tmp, src]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, obj)
+
+    if jobs:
+        with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 1)) as pool:
+            list(pool.map(compile_one, jobs))
+    objs = [os.path.join(OBJ, s[:-3] + ".o") for s in SOURCES]
+    if force or jobs or _stale(LIB, objs):
+        tmp = LIB + f".tmp{os.getpid()}"
+        subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-cudart", "static",
+                        "-o", tmp] + objs, check=True)
+        os.replace(tmp, LIB)
     return LIB
 
 

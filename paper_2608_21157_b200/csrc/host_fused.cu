@@ -1,0 +1,223 @@
+// Host side of 3D temporal blocking (fp32): configurations, the default fusion rule, launches.
+#include "host.h"
+#include "kernel_fused.cuh"
+
+namespace stencil_host {
+
+template <int R>
+void pack_star(const stencil_plan_s* p, StarWeights<R>& sw) {
+    std::memset(&sw, 0, sizeof(sw));
+    sw.c = dense_w(p, 0, 0, 0);
+    for (int d = -R; d <= R; ++d) {
+        if (d == 0) continue;
+        sw.x[d + R] = dense_w(p, 0, 0, d);
+        sw.y[d + R] = dense_w(p, 0, d, 0);
+        sw.z[d + R] = dense_w(p, d, 0, 0);
+    }
+}
+
+template <int R, int T, int K, int XW, int NWY, int MODE>
+cudaError_t launch_fused_t(const stencil_plan_s* p, const CUtensorMap& map, float* out, const FusedGeom& g,
+                           int grid, size_t smem, cudaStream_t st) {
+    StarWeights<R> sw;
+    pack_star<R>(p, sw);
+    return launch_kernel(&stencil_fused_kernel<R, T, K, XW, NWY, MODE>, grid, FusedShape<R, K, XW, NWY>::THREADS,
+                         smem, st, p->chained, map, out, g, sw, p->d_status);
+}
+
+template <int R, int T, int K, int XW, int NWY>
+FusedConfig make_fused() {
+    using S = FusedShape<R, K, XW, NWY>;
+    FusedConfig c;
+    c.radius = R; c.T = T; c.K = K; c.XW = XW; c.NWY = NWY; c.box = false;
+    c.txe = S::TXE; c.tye = S::TYE; c.threads = S::THREADS; c.slot_bytes = S::SLOT_BYTES; c.pw = S::PW;
+    c.kernel = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, 0>);
+    c.kernel_spec = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, 1>);
+    c.kernel_wrap = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, 2>);
+    c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
+    c.launch = &launch_fused_t<R, T, K, XW, NWY, 0>;
+    c.launch_spec = &launch_fused_t<R, T, K, XW, NWY, 1>;
+    c.launch_wrap = &launch_fused_t<R, T, K, XW, NWY, 2>;
+    return c;
+}
+
+// First match of (radius, T, region width) wins; T == 0 / width == 0 match anything.
+const std::vector<FusedConfig>& fused_configs() {
+    static const std::vector<FusedConfig> v = {
+        make_fused<1, 2, 4, 2, 8>(),  make_fused<1, 3, 4, 2, 8>(),  make_fused<1, 2, 4, 2, 4>(),
+        make_fused<1, 2, 2, 2, 8>(),  make_fused<1, 2, 4, 4, 4>(),  make_fused<1, 2, 4, 3, 5>(),
+        make_fused<1, 4, 2, 1, 16>(), make_fused<1, 2, 2, 1, 16>(), make_fused<1, 3, 2, 1, 16>(),
+        make_fused<2, 2, 2, 1, 16>(),
+    };
+    return v;
+}
+
+const FusedConfig* find_fused_cfg(int radius, int T, int txe, int tye = 0) {
+    for (const FusedConfig& c : fused_configs())
+        if (c.radius == radius && (T == 0 || c.T == T) && (txe == 0 || c.txe == txe) && (tye == 0 || c.tye == tye))
+            return &c;
+    return nullptr;
+}
+
+// Temporal blocking covers what the STREAM kernels cover, restricted to star stencils.
+const FusedConfig* pick_fused_region(const stencil_plan_s* p);
+
+const FusedConfig* pick_fused(const stencil_plan_s* p) {
+    const FusedConfig* c = pick_fused_region(p);
+    if (c && p->boundary == STENCIL_PERIODIC && !shell_fits(p, c->T * p->radius)) c = nullptr;
+    return c;
+}
+
+const FusedConfig* pick_fused_region(const stencil_plan_s* p) {
+    if (!stream_supported(p) || p->shape != STENCIL_STAR || p->ndim != 3) return nullptr;
+    if (p->nx % 4 != 0) return nullptr;                   // ... over the row pitch, which padded rows exceed
+    if (p->fuse_steps == 1) return nullptr;
+    int txe = p->tile_x;
+    // no preference for the region: the default below, also when the caller asks for its step count
+    if ((p->fuse_steps == 0 || p->fuse_steps == 2) && txe == 0 && p->fused_tile_y == 0) {
+        // Default: fuse two steps per pass when one region spans a whole row (no redundant
+        // columns) and the row fills at least 80 % of the region's lanes.  Regions are 128, 256
+        // (two CTAs per SM, which cover each other's barrier stalls: 16-row regions beat 32-row
+        // ones, 922 vs 846 G updates/s on 256^3) or 512 columns wide (one CTA per SM, each plane
+        // loaded as two TMA boxes).  With several regions per row the halo recomputation costs
+        // more than the saved traffic, and idle lanes cost what they would compute, so other
+        // grids stay unfused unless the caller asks for fusion.  Measured (G updates/s, fused
+        // vs unfused, 512 x 512 x nx): nx = 128: 1083 vs 644 (256-wide region: 499); 192: 744 vs
+        // 709; 400: 761 vs 776; 448: 851 vs 788; 512: 1257 vs 781.
+        // 384-wide regions are 20 rows high (15 warps, one CTA per SM; their planes are loaded as
+        // three boxes of 128 columns): 512 x 512 x 384 1359 vs 827, nx = 320: 1027 vs 773.
+        // Rows wider than 512 points take several 384- or 512-wide regions, each with 4 halo
+        // columns per side for every 2 levels of radius 1, under the same 80 % rule; per lane the
+        // 384-wide regions are a quarter faster there (256 x 512 x nx, 384-wide / 512-wide / unfused:
+        // nx = 1128: 1217 / 693 / 836; 1500: 1128 / 954 / 830; 256 x 1024 x 1024: 1126 / 687 / 808;
+        // nx = 768 fills neither to 80 %: 788 / 753 / 828).
+        const FusedConfig* c = nullptr;
+        const int halo = (2 * p->radius + 3) / 4 * 4;                         // per side, when a row takes several regions
+        auto lanes_used = [&](int w) {
+            const int64_t regions = p->nx <= w ? 1 : (p->nx + (w - 2 * halo) - 1) / (w - 2 * halo);
+            return (double)p->nx / (double)(regions * w);
+        };
+        int width = p->nx <= 128 ? 128 : p->nx <= 256 ? 256 : p->nx <= 384 ? 384 : 512;
+        if (p->nx > 512 && 1.25 * lanes_used(384) >= lanes_used(512)) width = 384;
+        const int height = width == 128 ? 0 : width == 384 ? 20 : 16;
+        // the 384-wide regions pay off from fewer used lanes: any row of 257..384 points (nx = 260:
+        // 838 vs 676), three quarters of the lanes with several regions per row (896: 983 vs 843)
+        const double need = width != 384 ? 0.8 : p->nx <= 384 ? 0.0 : 0.75;
+        if (lanes_used(width) >= need) {
+            // 128-wide regions leave registers for a third level (512 x 512 x 128: 1224 G updates/s
+            // with three steps per pass, 1083 with two, 1108 with four); at 256 columns three
+            // levels spill (256^3: 820 against 1056)
+            // ... provided the grid still cuts into a machine's worth of CTAs (a B200 has 148
+            // SMs; 128^3 x 64 steps: 302 with three levels, 393 with two)
+            if (width == 128 && p->fuse_steps == 0) {
+                const FusedConfig* c3 = find_fused_cfg(p->radius, 3, 128);
+                if (c3) {
+                    const int tile_y = c3->tye - 2 * 3 * p->radius;
+                    const int64_t ctas = tile_y < 1 ? 0 : (int64_t)((p->ny + tile_y - 1) / tile_y) *
+                                                              std::max(1, p->nz / (4 * 3 * p->radius));
+                    if (ctas >= 148) c = c3;
+                }
+            }
+            if (!c) c = find_fused_cfg(p->radius, 2, width, height);
+            if (!c && width == 256) c = find_fused_cfg(p->radius, 2, 256);
+        }
+        if (c || p->fuse_steps == 0) return c;
+    }
+    return find_fused_cfg(p->radius, p->fuse_steps, txe, p->fused_tile_y);
+}
+
+int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cudaStream_t st) {
+    const FusedConfig* cfg = p->fused_cfg;
+    const CUtensorMap* map = nullptr;
+    int rc = get_tensor_map(p, cfg, cfg->pw, cfg->tye, src, &map);   // a box is at most 256 wide
+    if (rc != STENCIL_OK) return rc;
+    const int R = p->radius, T = cfg->T;
+    FusedGeom g;
+    g.nz = p->nz; g.ny = p->ny; g.nx = p->nx;
+    g.nlev = nlev;
+    if (p->nx <= cfg->txe) {                     // one region spans the row: the x halo is the zero boundary
+        g.halo_x = 0; g.tile_x = cfg->txe; g.tiles_x = 1;
+    } else {
+        g.halo_x = (T * R + 3) / 4 * 4;
+        g.tile_x = cfg->txe - 2 * g.halo_x;
+        g.tiles_x = (p->nx + g.tile_x - 1) / g.tile_x;
+    }
+    g.halo_y = T * R;
+    g.tile_y = cfg->tye - 2 * g.halo_y;
+    if (g.tile_x < 4 || g.tile_y < 1) return STENCIL_ERR_UNSUPPORTED;
+    g.tiles_y = (p->ny + g.tile_y - 1) / g.tile_y;
+    // shared memory: input ring + two planes per intermediate level
+    int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 2;   // measured: 2 beats 3 and 4
+    auto smem_for = [&](int s) { return (size_t)(s + 2 * (T - 1)) * cfg->slot_bytes + 128 + kMaxStages * sizeof(uint64_t); };
+    while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;
+    const size_t smem = smem_for(stages);
+    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
+    g.stages = stages;
+    const int tiles = g.tiles_x * g.tiles_y;
+    int occ = 1;
+    {
+        // shared-memory limit and occupancy of the kernel, asked once per device and size
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+        std::lock_guard<std::mutex> lock(g_config_mutex);
+        if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->occ_smem = 0; cfg->cache_device = dev; }
+        if (smem > cfg->smem_allowed) {
+            if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                    cudaSuccess ||
+                cudaFuncSetAttribute(cfg->kernel_spec, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                    cudaSuccess ||
+                cudaFuncSetAttribute(cfg->kernel_wrap, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                    cudaSuccess) {
+                cudaGetLastError();
+                return STENCIL_ERR_CUDA;
+            }
+            cfg->smem_allowed = smem;
+        }
+        if (cfg->occ_smem != smem) {
+            int o = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, cfg->kernel, cfg->threads, smem) != cudaSuccess) {
+                cudaGetLastError();
+                o = 0;
+            }
+            cfg->occ = std::max(o, 1);
+            cfg->occ_smem = smem;
+        }
+        occ = cfg->occ;
+    }
+    int chunk = p->chunk_z;
+    if (chunk <= 0) {
+        // The kernel is bound by instruction issue, so every SM should get the same number of
+        // planes: cut z into the number of chunks whose CTAs fill whole waves of the machine's
+        // resident-CTA slots at the least total cost, a chunk costing its planes plus the
+        // 2*T*R extra input planes and the start-up of its pipeline.
+        const int slots = occ * sm_count();
+        const int max_chunks = std::max(1, p->nz / (4 * T * R));
+        const double fill = 4.0;
+        double best = 1e300;
+        int best_n = 1;
+        for (int n = 1; n <= max_chunks; ++n) {
+            const int c = (p->nz + n - 1) / n;
+            const int real_n = (p->nz + c - 1) / c;
+            const int64_t ctas = (int64_t)tiles * real_n;
+            const double waves = (double)((ctas + slots - 1) / slots);
+            const double cost = waves * (c + 2 * T * R + fill);
+            if (cost < best * 0.999) { best = cost; best_n = real_n; }
+        }
+        chunk = (p->nz + best_n - 1) / best_n;
+    }
+    chunk = std::max(1, std::min(chunk, p->nz));
+    g.chunk_z = chunk;
+    const int64_t grid64 = (int64_t)tiles * ((p->nz + chunk - 1) / chunk);
+    if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
+    // full passes over rows of exactly one region take the instantiation with those facts compiled in
+    // ... and the one that also wraps x and z when the pass belongs to a periodic apply (fused_wrap_ok tells
+    // the caller beforehand that it will)
+    const bool spec = nlev == T && p->nx == cfg->txe;
+    auto launch = !spec ? cfg->launch : (p->fused_wrap ? cfg->launch_wrap : cfg->launch_spec);
+    if (p->fused_wrap && !spec) return STENCIL_ERR_UNSUPPORTED;
+    if (launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
+    p->launches++;
+    return STENCIL_OK;
+}
+
+}  // namespace stencil_host

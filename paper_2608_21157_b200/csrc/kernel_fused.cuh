@@ -27,15 +27,6 @@
 
 namespace stencil {
 
-struct FusedGeom {
-    int nz, ny, nx;
-    int tiles_x, tiles_y;
-    int tile_x, tile_y;        // output tile (interior) size
-    int halo_x, halo_y;        // region = tile + 2*halo; halo_x is a multiple of 4
-    int chunk_z;
-    int stages;
-    int nlev;                  // time steps advanced by this pass, 1..T
-};
 
 template <int R, int K, int XW, int NWY>
 struct FusedShape {

@@ -5,11 +5,11 @@
 // write of the grid per sweep, which still beats gathering wrapped taps one by one.
 #pragma once
 #include "common.cuh"
+#include "geom.cuh"
 #include "ptx.cuh"
 
 namespace stencil {
 
-constexpr int kPadX = 4;            // halo columns per side of the padded copy
 
 template <typename T> struct Vec16;                          // the 16-byte vector of a grid's value type
 template <> struct Vec16<float>  { using type = float4;  static constexpr int n = 4; };

@@ -23,15 +23,6 @@ struct Weights2D {              // dense, [dy+R][dx+R]; a star has zeros off the
     float w[2 * R + 1][2 * R + 1];
 };
 
-struct Rows2DGeom {
-    int ny, nx;
-    int strips;                 // ceil(nx / 128)
-    int chunk_y;                // output rows per warp
-    int nchunks;
-    int stages;                 // batches in a warp's ring
-    int in_off_x, in_off_y;     // added to the TMA coordinates (padded input of a periodic grid), else 0
-    int y_begin, y_end;         // output rows of this launch (the whole grid: 0, ny)
-};
 
 template <int YB, int PXV = kStreamPX>     // PXV: row pitch of a batch (the strip plus its halo columns)
 struct Rows2DShape {

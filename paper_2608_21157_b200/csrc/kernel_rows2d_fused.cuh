@@ -30,14 +30,6 @@ namespace stencil {
 constexpr int kFused2DHalo = 4;                         // columns per side of a strip that are not stored
 constexpr int kFused2DTile = kStreamTX - 2 * kFused2DHalo;
 
-struct Rows2DFusedGeom {
-    int ny, nx;
-    int strips;                 // ceil(nx / kFused2DTile)
-    int chunk_y;                // output rows per warp
-    int nchunks;
-    int stages;                 // batches in a warp's ring
-    int nlev;                   // time steps advanced by this pass, 1..T
-};
 
 // x neighbourhood of a row held in registers: the lane's float4 plus R values on either
 // side from the neighbour lanes; zero where the warp ends.

@@ -23,14 +23,13 @@
 #include <utility>
 
 #include "common.cuh"
+#include "geom.cuh"
 #include "ptx.cuh"
 
 namespace stencil {
 
-constexpr int kStreamTX = 128;            // tile width (points); one warp spans a row
 constexpr int kStreamPX = kStreamTX + 8;  // smem row pitch: 4-float halo each side keeps
                                           // TMA x-coordinates and LDS.128 16-byte aligned
-constexpr int kMaxStages = 8;
 
 // Halo columns on either side of a tile row in shared memory: 4 floats reach radius 4; the
 // wider stars (radius 5..8) take 8.  Multiples of 4 keep TMA x-coordinates and LDS.128 aligned.
@@ -60,18 +59,6 @@ struct BoxWeights {             // dense cube, [dz+R][dy+R][dx+R]
     float w[2 * R + 1][2 * R + 1][2 * R + 1];
 };
 
-struct StreamGeom {
-    int nz, ny, nx;
-    int tiles_x, tiles_y;
-    int z_begin, z_end;         // output planes of this launch: [z_begin, z_end), normally [0, nz)
-    int chunk_z;                // planes of output per CTA
-    int stages;                 // depth of the plane ring
-    int streaming_store;        // 1: st.global.cs
-    int in_off_x, in_off_y, in_off_z;   // added to every TMA coordinate: non-zero when the input is a
-                                // padded copy of the grid (periodic boundary), else 0
-    unsigned wait_polls;        // cap of every bounded wait
-    int drop_plane;             // test hook: the producer never loads this plane of a CTA (-1: none)
-};
 
 template <int R, int K, int NW>
 struct StreamShape {
