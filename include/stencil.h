@@ -9,7 +9,9 @@
  *
  * applied once or iterated over time steps (the protocol repeats the sweep and
  * reports the amortised per-step latency).  This library generalises the
- * paper's 2D box to 2D/3D, star or box neighbourhoods, fp32 grids.
+ * paper's 2D box to 2D/3D, star or box neighbourhoods, on fp32 grids
+ * (stencil_plan / stencil_apply) and on FP64 grids, the paper's own precision
+ * (stencil_plan_f64 / stencil_apply_f64).
  *
  * Conventions for every call
  *   - returns a status (STENCIL_OK or a negative STENCIL_ERR_*); never throws,
@@ -80,8 +82,8 @@ enum {
     STENCIL_KEY_STAGES       = 7,  /* set/get: depth of the shared-memory plane ring (0 = auto)  */
     STENCIL_KEY_STREAMING_STORE = 8, /* set/get: 1 = write results with evict-first stores       */
     STENCIL_KEY_ROWS_PER_THREAD = 9, /* set/get: tile rows each thread computes (0 = default)    */
-    STENCIL_KEY_WAIT_POLLS   = 10, /* set/get: polls after which a device-side wait of the 3D
-                                      single-step kernel gives up (each poll sleeps <= 20 us)    */
+    STENCIL_KEY_WAIT_POLLS   = 10, /* set/get: polls after which a device-side wait of the tiled
+                                      kernels gives up (each poll sleeps <= 20 us)               */
     STENCIL_KEY_CHAIN_LAUNCHES = 12, /* set/get: 1 (default) = launches 2..n of an iterated apply are
                                       programmatic dependent launches: each begins its preamble
                                       while its predecessor drains and waits for it before it
@@ -99,10 +101,15 @@ enum {
                                       fused zero-boundary passes of L steps and rewrite the points
                                       within L*R of a face afterwards (every extent >= 2*L*R),
                                       unless this key is 1 or STENCIL_KEY_FUSE_STEPS is 1         */
-    STENCIL_KEY_TEST_DROP_PLANE = 11 /* set/get, test hook: every CTA of the 3D single-step kernel
-                                      never loads its input plane of this index, so the bounded
-                                      wait for it expires and stencil_query_status reports
-                                      STENCIL_ERR_TIMEOUT (-1 = off, the default)                */
+    STENCIL_KEY_TEST_DROP_PLANE = 11, /* set/get, test hook: every CTA (2D kernels: every warp) of the
+                                      tiled kernels never loads its input plane (2D: batch of
+                                      rows) of this index, so the bounded wait for it expires and
+                                      stencil_query_status reports STENCIL_ERR_TIMEOUT; nothing
+                                      faults (-1 = off, the default)                             */
+    STENCIL_KEY_DEVICE       = 15    /* get: the CUDA device the plan's device state lives on
+                                      (the one current at its first apply; -1 before that).
+                                      Later applies must run with that device current
+                                      (STENCIL_ERR_INVALID otherwise)                            */
 };
 
 /*
@@ -166,11 +173,11 @@ STENCIL_API int stencil_apply(stencil_plan_t plan, const float* in, float* out, 
  * stencil_apply with double in place of float.  A plan made by one of the two
  * plan calls is only accepted by the matching apply call (STENCIL_ERR_INVALID
  * otherwise); stencil_destroy, stencil_query_status and the knobs serve both.
- * TMA-staged kernels cover 2D star and box radius <= 4, 3D star radius <= 4
- * and box radius <= 2, with a zero boundary (rows of an odd number of
- * doubles through grids with padded rows) or a periodic one (even nx);
- * everything else runs on the one-thread-per-point kernel.  Temporal blocking
- * in FP64 exists for 2D grids with radius <= 2 (zero boundary, even nx).
+ * TMA-staged kernels cover stars up to radius 8 (2D and 3D), 2D boxes up to
+ * radius 4 and 3D boxes up to radius 2, with a zero boundary (rows of an odd
+ * number of doubles through grids with padded rows) or a periodic one (even
+ * nx); everything else runs on the one-thread-per-point kernel.  Temporal
+ * blocking in FP64 exists for 2D grids with radius <= 2 (even nx).
  */
 STENCIL_API int stencil_plan_f64(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radius,
                                  int shape, const double* weights, int boundary);
@@ -199,7 +206,9 @@ STENCIL_API int stencil_apply_planes_f64(stencil_plan_t plan, const double* in, 
                                          int64_t z_end, void* stream);
 
 /*
- * stencil_apply_host — the same operation on HOST buffers: copies `in_host`
+ * stencil_apply_host — the same operation on HOST buffers (an addition of this
+ * library for end-to-end use; the paper's protocol times device-resident
+ * grids and has no counterpart): copies `in_host`
  * to a plan-owned device grid, runs stencil_apply, copies the result back to
  * `out_host` and waits for it.  Pinned host memory makes the copies
  * asynchronous up to the final wait; pageable memory works but is slower.
@@ -223,9 +232,9 @@ STENCIL_API int stencil_apply_host(stencil_plan_t plan, const float* in_host, fl
  * cudaFree bring.  stencil_apply allocates on first use (a status word, the tap
  * list, and for steps > 1 a scratch grid).  This entry point allocates nothing,
  * neither through the CUDA runtime nor through any library: its ping-pong grid
- * and tap list sit in one fixed array inside the library, 8 MiB + 79 KiB of
- * device memory that every GPU which loads the library holds until the process
- * ends.
+ * and tap list sit in one fixed array inside the library, 8 MiB + 77 KiB
+ * (8,467,456 bytes) of device memory that every GPU which loads the library
+ * holds until the process ends.
  *
  *   in, out, steps, stream   exactly as for stencil_apply; the result is the
  *                            same up to fp32 summation order (it runs the
@@ -236,16 +245,26 @@ STENCIL_API int stencil_apply_host(stencil_plan_t plan, const float* in_host, fl
  *
  * The first call on each device also looks up the array's device address (the
  * name of the array is not an address on the host); make that first call with
- * the device current and before starting any stream capture.  All calls, from
- * all plans, share the one array: two calls whose GPU work overlaps (different
- * streams, or different host threads) race on it and on the tap list, so
- * serialise them.  Nothing has to be cleared between calls: each call rewrites
- * the taps and writes every scratch cell before reading it.
+ * the device current and before starting any stream capture.  A call whose
+ * plan's taps are not in the array (the plan's first call, or after a call of
+ * another plan) uploads them with an asynchronous copy from the plan's own,
+ * pageable host memory: that copy may make the host wait for earlier work on
+ * `stream`, and it does not belong inside a stream capture either; a plan that
+ * calls again straight after itself uploads nothing.  All calls, from all plans,
+ * share the one array: two calls whose GPU work overlaps (different streams, or
+ * different host threads) race on it and on the tap list, so serialise them.
+ * Nothing has to be cleared between calls: every scratch cell is written before
+ * it is read, and the taps are replaced whenever another plan's are in place.
  */
 STENCIL_API int stencil_apply_static(stencil_plan_t plan, const float* in, float* out, int steps,
                                      void* stream);
 
-/* stencil_destroy — free the plan and everything it owns.  NULL is a no-op. */
+/*
+ * stencil_destroy — free the plan and everything it owns (its device memory on
+ * the device it lives on, after waiting for the stream of its last apply).
+ * NULL is a no-op.  Housekeeping of this library: no passage of the paper
+ * defines it.
+ */
 STENCIL_API int stencil_destroy(stencil_plan_t plan);
 
 /* Static, NUL-terminated description of a status code. */

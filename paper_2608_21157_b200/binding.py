@@ -26,7 +26,7 @@ VARIANT_AUTO, VARIANT_GENERIC, VARIANT_STREAM, VARIANT_FUSED = 0, 1, 2, 3
 
 (KEY_VARIANT, KEY_TILE_X, KEY_TILE_Y, KEY_FUSE_STEPS, KEY_LAUNCHES, KEY_SCRATCH_BYTES,
  KEY_CHUNK_Z, KEY_STAGES, KEY_STREAMING_STORE, KEY_ROWS_PER_THREAD, KEY_WAIT_POLLS,
- KEY_TEST_DROP_PLANE, KEY_CHAIN_LAUNCHES, KEY_FUSED_TILE_Y, KEY_PERIODIC_ROUTE) = range(15)
+ KEY_TEST_DROP_PLANE, KEY_CHAIN_LAUNCHES, KEY_FUSED_TILE_Y, KEY_PERIODIC_ROUTE, KEY_DEVICE) = range(16)
 
 #: every symbol include/stencil.h declares
 EXPORTS = (

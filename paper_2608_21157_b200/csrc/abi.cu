@@ -54,6 +54,13 @@ int launch_sweep(stencil_plan_s* p, const float* src, float* dst, cudaStream_t s
 // ---------------------------------------------------------------------------
 // plan construction, shared by the fp32 and the FP64 entry point
 // ---------------------------------------------------------------------------
+uint64_t next_plan_serial() {
+    static std::mutex m;
+    static uint64_t n = 0;
+    std::lock_guard<std::mutex> lock(m);
+    return ++n;
+}
+
 template <typename T>
 int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radius, int shape,
               const T* weights, int boundary) {
@@ -76,6 +83,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     stencil_plan_s* p = new (std::nothrow) stencil_plan_s();
     if (!p) return STENCIL_ERR_ALLOC;
     p->magic = kPlanMagic;
+    p->serial = next_plan_serial();
     p->f64 = kF64;
     p->ndim = ndim;
     p->nz = ndim == 3 ? (int)dims[0] : 1;
@@ -151,8 +159,12 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticGridBytes
 // asked for, once per device, while that device is current.
 std::mutex g_static_mutex;
 unsigned char* g_static_ptr[kStaticMaxDevices] = {nullptr};
+// serial number of the plan whose taps were last uploaded into the array, per device (0: none)
+uint64_t g_static_tap_owner[kStaticMaxDevices] = {0};
 
-int static_scratch_address(unsigned char** out) {
+// `upload` comes back true when the array does not hold the taps of plan `serial` yet; the caller
+// then uploads them (the array is marked as that plan's at once: calls do not overlap, by contract).
+int static_scratch_address(unsigned char** out, uint64_t serial, bool* upload) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
     if (dev < 0 || dev >= kStaticMaxDevices) return STENCIL_ERR_UNSUPPORTED;
@@ -166,6 +178,8 @@ int static_scratch_address(unsigned char** out) {
         g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
     }
     *out = g_static_ptr[dev];
+    *upload = g_static_tap_owner[dev] != serial;
+    g_static_tap_owner[dev] = serial;
     return STENCIL_OK;
 }
 
@@ -195,6 +209,7 @@ int stencil_apply(stencil_plan_t p, const float* in, float* out, int steps, void
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 
     int rc = ensure_device_state(p);
+    if (rc == STENCIL_OK) rc = check_device(p);
     if (rc != STENCIL_OK) return rc;
     p->last_stream = st;
     p->used = true;
@@ -257,7 +272,8 @@ int stencil_apply_planes(stencil_plan_t p, const float* in, float* out, int64_t 
     if (p->variant != STENCIL_VARIANT_STREAM || p->boundary != STENCIL_ZERO || p->nx % 4 != 0)
         return STENCIL_ERR_UNSUPPORTED;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    const int rc = ensure_device_state(p);
+    int rc = ensure_device_state(p);
+    if (rc == STENCIL_OK) rc = check_device(p);
     if (rc != STENCIL_OK) return rc;
     p->last_stream = st;
     p->used = true;
@@ -277,7 +293,8 @@ int stencil_apply_planes_f64(stencil_plan_t p, const double* in, double* out, in
     if (p->variant != STENCIL_VARIANT_STREAM || p->boundary != STENCIL_ZERO || p->nx % 2 != 0)
         return STENCIL_ERR_UNSUPPORTED;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    const int rc = ensure_device_state(p);
+    int rc = ensure_device_state(p);
+    if (rc == STENCIL_OK) rc = check_device(p);
     if (rc != STENCIL_OK) return rc;
     p->last_stream = st;
     p->used = true;
@@ -292,6 +309,7 @@ int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps
     if (a < b + bytes && b < a + bytes) return STENCIL_ERR_INVALID;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     int rc = ensure_device_state(p);
+    if (rc == STENCIL_OK) rc = check_device(p);
     if (rc != STENCIL_OK) return rc;
     p->last_stream = st;
     p->used = true;
@@ -342,6 +360,7 @@ int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps
 int stencil_apply_host(stencil_plan_t p, const float* in_host, float* out_host, int steps, void* stream) {
     if (!valid_plan(p) || p->f64 || !in_host || !out_host || steps < 0) return STENCIL_ERR_INVALID;
     int rc = ensure_device_state(p);
+    if (rc == STENCIL_OK) rc = check_device(p);
     if (rc != STENCIL_OK) return rc;
     if ((rc = ensure_grid(&p->host_in, p->npoints)) != STENCIL_OK) return rc;
     if ((rc = ensure_grid(&p->host_out, p->npoints)) != STENCIL_OK) return rc;
@@ -423,12 +442,6 @@ int stencil_apply_static(stencil_plan_t p, const float* in, float* out, int step
     if (p->npoints > kStaticMaxPoints || (int64_t)p->taps.size() > kStaticMaxTaps) return STENCIL_ERR_TOO_LARGE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 
-    unsigned char* base = nullptr;                 // first call on a device also looks the array up
-    int rc = static_scratch_address(&base);
-    if (rc != STENCIL_OK) return rc;
-    float* grid = reinterpret_cast<float*>(base);
-    Tap* taps = reinterpret_cast<Tap*>(base + kStaticGridBytes);
-
     if (steps == 0) {
         if (cudaMemcpyAsync(out, in, bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
             cudaGetLastError();
@@ -436,9 +449,17 @@ int stencil_apply_static(stencil_plan_t p, const float* in, float* out, int step
         }
         return STENCIL_OK;
     }
+    unsigned char* base = nullptr;                 // first call on a device also looks the array up
+    bool upload = true;
+    int rc = static_scratch_address(&base, p->serial, &upload);
+    if (rc != STENCIL_OK) return rc;
+    float* grid = reinterpret_cast<float*>(base);
+    Tap* taps = reinterpret_cast<Tap*>(base + kStaticGridBytes);
     const int ntaps = (int)p->taps.size();
-    if (ntaps > 0 && cudaMemcpyAsync(taps, p->taps.data(), (size_t)ntaps * sizeof(Tap), cudaMemcpyHostToDevice,
-                                     st) != cudaSuccess) {
+    // The taps go up only when the array holds another plan's (or nothing yet): a plan that calls
+    // again finds them in place and enqueues nothing but its kernels.
+    if (upload && ntaps > 0 &&
+        cudaMemcpyAsync(taps, p->taps.data(), (size_t)ntaps * sizeof(Tap), cudaMemcpyHostToDevice, st) != cudaSuccess) {
         cudaGetLastError();
         return STENCIL_ERR_CUDA;
     }
@@ -674,6 +695,7 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
         case STENCIL_KEY_FUSED_TILE_Y:
             *value = (p->variant == STENCIL_VARIANT_STREAM && p->fused_cfg) ? p->fused_cfg->tye : 0;
             return STENCIL_OK;
+        case STENCIL_KEY_DEVICE: *value = p->device; return STENCIL_OK;
         case STENCIL_KEY_WAIT_POLLS: *value = p->wait_polls; return STENCIL_OK;
         case STENCIL_KEY_TEST_DROP_PLANE: *value = p->drop_plane; return STENCIL_OK;
         default: return STENCIL_ERR_INVALID;

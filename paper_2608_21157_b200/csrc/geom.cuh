@@ -29,6 +29,8 @@ struct FusedGeom {
     int chunk_z;
     int stages;
     int nlev;                  // time steps advanced by this pass, 1..T
+    unsigned wait_polls;       // cap of every bounded wait
+    int drop_plane;            // test hook: a CTA never loads its input plane of this index (-1: none)
 };
 
 struct Rows2DGeom {
@@ -39,6 +41,8 @@ struct Rows2DGeom {
     int stages;                 // batches in a warp's ring
     int in_off_x, in_off_y;     // added to the TMA coordinates (padded input of a periodic grid), else 0
     int y_begin, y_end;         // output rows of this launch (the whole grid: 0, ny)
+    unsigned wait_polls;        // cap of every bounded wait
+    int drop_batch;             // test hook: a warp never loads its input batch of this index (-1: none)
 };
 
 struct Rows2DFusedGeom {
@@ -48,6 +52,8 @@ struct Rows2DFusedGeom {
     int nchunks;
     int stages;                 // batches in a warp's ring
     int nlev;                   // time steps advanced by this pass, 1..T
+    unsigned wait_polls;        // cap of every bounded wait
+    int drop_batch;             // test hook: a warp never loads its input batch of this index (-1: none)
 };
 
 }  // namespace stencil

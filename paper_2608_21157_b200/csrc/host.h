@@ -203,6 +203,7 @@ struct Stream64Config {
 
 struct stencil_plan_s {
     uint32_t magic;
+    uint64_t serial;               // unique per plan of this process, never reused
     int ndim;
     int nz, ny, nx;
     int64_t npoints;
@@ -310,6 +311,7 @@ private:
 // ---- host_common.cu ---------------------------------------------------------
 int sm_count();
 int ensure_device_state(stencil_plan_s* p);
+int check_device(const stencil_plan_s* p);
 int ensure_grid(float** slot, int64_t npoints);
 int get_tensor_map(stencil_plan_s* p, const void* cfg, int box_x, int box_y, const float* src,
                    const CUtensorMap** out, int tnx = 0, int tny = 0, int tnz = 0);
@@ -320,10 +322,6 @@ int launch_generic_f64(stencil_plan_s* p, const double* src, double* dst, cudaSt
 // the one-thread-per-point kernel on caller-given taps (stencil_apply_static)
 int launch_generic_taps(stencil_plan_s* p, const float* src, float* dst, const Tap* d_taps, int ntaps,
                         cudaStream_t st);
-// Shared-memory limit and occupancy of a kernel at `smem` bytes, cached per device in the
-// configuration's fields; returns the resident CTAs per SM (>= 1) or -1 on a CUDA error.
-int kernel_limits(const void* kernel, int threads, size_t smem, size_t* smem_allowed, size_t* occ_smem, int* occ,
-                  int* cache_device);
 
 // ---- host_stream.cu ---------------------------------------------------------
 const StreamConfig* find_stream_cfg(int radius, bool box, int tile_y, int rows_per_thread);

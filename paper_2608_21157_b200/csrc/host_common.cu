@@ -78,16 +78,29 @@ int ensure_grid(float** slot, int64_t npoints) {
     return STENCIL_OK;
 }
 
+// Multiprocessors of the current device (asked once per device).
 int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-            n = v;
-        else { cudaGetLastError(); n = 148; }
+    constexpr int kMaxDevices = 64;
+    static int cache[kMaxDevices] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 148; }
+    if (dev >= 0 && dev < kMaxDevices && cache[dev] > 0) return cache[dev];
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+        cudaGetLastError();
+        return 148;
     }
-    return n;
+    if (dev >= 0 && dev < kMaxDevices) cache[dev] = v;      // a benign race: every writer stores the same value
+    return v;
+}
+
+// A plan's device state (status word, taps, scratch grids, tensor maps) belongs to the device
+// that was current at its first apply; later applies must run with the same device current.
+int check_device(const stencil_plan_s* p) {
+    if (p->device < 0) return STENCIL_OK;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    return dev == p->device ? STENCIL_OK : STENCIL_ERR_INVALID;
 }
 
 int get_tensor_map(stencil_plan_s* p, const void* cfg, int box_x, int box_y, const float* src,

@@ -249,6 +249,7 @@ int launch_rows2d_fused64(stencil_plan_s* p, const double* src, double* dst, int
     g.strips = (p->nx + kFused2D64Tile - 1) / kFused2D64Tile;
     g.stages = stages;
     g.nlev = nlev;
+    g.wait_polls = p->wait_polls; g.drop_batch = p->drop_plane;
     int chunk = p->chunk_z;
     if (chunk <= 0) {                                 // same sizing rule as the fp32 kernel
         const int H = nlev * p->radius;
@@ -341,7 +342,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         g.in_off_x = periodic ? kPadX : 0;
         g.in_off_y = periodic ? p->radius : 0;
         g.in_off_z = periodic ? p->radius : 0;
-        g.wait_polls = p->wait_polls; g.drop_plane = -1;
+        g.wait_polls = p->wait_polls; g.drop_plane = p->drop_plane;
         // many short CTAs, as for the bandwidth-bound fp32 sweeps; the wide stars re-read 2R halo
         // planes per chunk, so they get longer chunks (measured on 512^3)
         const int want_chunk = p->radius >= 3 ? 64 : 32;
@@ -445,6 +446,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         g.chunk_y = chunk;
         g.nchunks = (span + chunk - 1) / chunk;
         g.y_begin = begin; g.y_end = end;
+        g.wait_polls = p->wait_polls; g.drop_batch = p->drop_plane;
         const int64_t units = (int64_t)g.strips * g.nchunks;
         const int64_t grid64 = (units + cfg->NW - 1) / cfg->NW;
         if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;

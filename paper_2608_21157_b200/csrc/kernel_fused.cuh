@@ -152,6 +152,7 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
         const int pre = min(nstage, nsteps);
         issued = pre;
         for (int i = 0; i < pre; ++i) {
+            if (i == g.drop_plane) continue;
             mbar_arrive_expect_tx(full0 + 8 * i, S::BOX_BYTES);
 #pragma unroll
             for (int part = 0; part < S::NP; ++part)
@@ -179,7 +180,7 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
     auto step = [&](auto par_c, auto fast_c, const int i) {
             constexpr int par = decltype(par_c)::value & 1;
             constexpr bool FAST = decltype(fast_c)::value != 0;
-            if (!dead && !mbar_wait_bounded(full0 + 8 * s, ph)) {
+            if (!dead && !mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) {
                 dead = true;
                 atomicExch(status, kStatusTimeout);
             }
@@ -286,7 +287,7 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                     if (l < nlev || l == 1) {
                         // everyone has finished with level l-1's plane and has published level l
                         consumer_barrier(S::THREADS);
-                        if (l == 1 && tid == 0 && i + nstage < nsteps) {
+                        if (l == 1 && tid == 0 && i + nstage < nsteps && i + nstage != g.drop_plane) {
                             // the input slot is free: refill it with the plane nstage steps ahead
                             mbar_arrive_expect_tx(full0 + 8 * s, S::BOX_BYTES);
 #pragma unroll
@@ -329,7 +330,7 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
     if (dead && tid == 0) {
         // let copies that may still be in flight land before shared memory is released
         for (int i = max(0, issued - nstage); i < issued; ++i)
-            mbar_wait_bounded(full0 + 8 * (i % nstage), (i / nstage) & 1);
+            mbar_wait_bounded(full0 + 8 * (i % nstage), (i / nstage) & 1, g.wait_polls);
     }
 }
 

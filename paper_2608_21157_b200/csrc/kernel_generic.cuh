@@ -79,7 +79,9 @@ stencil_generic_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g,
             }
             __syncthreads();
             // Branch-free inner loop so that several loads are in flight per thread: a tap that
-            // leaves the grid reads the thread's own point with weight zero.
+            // leaves the grid loads the thread's own point (a safe address) and contributes an exact
+            // zero, value and weight both, so that a non-finite own point cannot leak into the sum
+            // (the tiled kernels read zero-filled halos there and give the same result).
 #pragma unroll 4
             for (int t = 0; t < nt; ++t) {
                 const ResolvedTap<T> r = s_tap[t];
@@ -91,7 +93,7 @@ stencil_generic_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g,
                     ok = ok && (unsigned)qx < (unsigned)g.nx;
                 }
                 const T v = __ldg(in + (ok ? r.row + qx : self));
-                acc = fma_t(ok ? r.w : T(0), v, acc);
+                acc = fma_t(ok ? r.w : T(0), ok ? v : T(0), acc);
             }
         }
         if (xb * kGenericThreads + (int)threadIdx.x < g.nx) out[self] = acc;

@@ -76,6 +76,7 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
         const int pre = min(nstage, nbatches);
         issued = pre;
         for (int b = 0; b < pre; ++b) {
+            if (b == g.drop_batch) continue;
             mbar_arrive_expect_tx(full0 + 8 * b, S::BATCH_BYTES);
             tma_load_3d(smem_addr(ring + (size_t)b * S::BATCH_FLOATS), &tmap_in, full0 + 8 * b,
                         x0 - HX + g.in_off_x, ystart + b * YB + g.in_off_y, 0);
@@ -93,12 +94,12 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
     int s = 0;
     uint32_t ph = 0;
     for (int b = 0; b < nbatches; ++b) {
-        if (!mbar_wait_bounded(full0 + 8 * s, ph)) {
+        if (!mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) {
             atomicExch(status, kStatusTimeout);
             // let copies that may still be in flight land before the warp leaves
             if (lane == 0)
                 for (int q = max(b + 1, issued - nstage); q < issued; ++q)
-                    mbar_wait_bounded(full0 + 8 * (q % nstage), (q / nstage) & 1);
+                    mbar_wait_bounded(full0 + 8 * (q % nstage), (q / nstage) & 1, g.wait_polls);
             return;
         }
         const float* bp = ring + (size_t)s * S::BATCH_FLOATS;
@@ -174,7 +175,7 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
         }
         // every lane is done with the batch: refill its slot with the batch nstage ahead
         __syncwarp();
-        if (lane == 0 && b + nstage < nbatches) {
+        if (lane == 0 && b + nstage < nbatches && b + nstage != g.drop_batch) {
             mbar_arrive_expect_tx(full0 + 8 * s, S::BATCH_BYTES);
             tma_load_3d(smem_addr(ring + (size_t)s * S::BATCH_FLOATS), &tmap_in, full0 + 8 * s,
                         x0 - HX + g.in_off_x, ystart + (b + nstage) * YB + g.in_off_y, 0);

@@ -73,6 +73,7 @@ stencil_rows2d_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
         const int pre = min(nstage, nbatches);
         issued = pre;
         for (int b = 0; b < pre; ++b) {
+            if (b == g.drop_batch) continue;
             mbar_arrive_expect_tx(full0 + 8 * b, S::BATCH_BYTES);
             tma_load_3d(smem_addr(ring + (size_t)b * S::BATCH_DOUBLES), &tmap_in, full0 + 8 * b,
                         x0 - HX + g.in_off_x, ystart + b * YB + g.in_off_y, 0);
@@ -90,11 +91,11 @@ stencil_rows2d_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
     int s = 0;
     uint32_t ph = 0;
     for (int b = 0; b < nbatches; ++b) {
-        if (!mbar_wait_bounded(full0 + 8 * s, ph)) {
+        if (!mbar_wait_bounded(full0 + 8 * s, ph, g.wait_polls)) {
             atomicExch(status, kStatusTimeout);
             if (lane == 0)
                 for (int q = max(b + 1, issued - nstage); q < issued; ++q)
-                    mbar_wait_bounded(full0 + 8 * (q % nstage), (q / nstage) & 1);
+                    mbar_wait_bounded(full0 + 8 * (q % nstage), (q / nstage) & 1, g.wait_polls);
             return;
         }
         const double* bp = ring + (size_t)s * S::BATCH_DOUBLES;
@@ -165,7 +166,7 @@ stencil_rows2d_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
             }
         }
         __syncwarp();
-        if (lane == 0 && b + nstage < nbatches) {
+        if (lane == 0 && b + nstage < nbatches && b + nstage != g.drop_batch) {
             mbar_arrive_expect_tx(full0 + 8 * s, S::BATCH_BYTES);
             tma_load_3d(smem_addr(ring + (size_t)s * S::BATCH_DOUBLES), &tmap_in, full0 + 8 * s,
                         x0 - HX + g.in_off_x, ystart + (b + nstage) * YB + g.in_off_y, 0);

@@ -108,7 +108,9 @@ stream_f64_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CU
             uint32_t ph = 1;
             for (int i = 0; i < nplanes; ++i) {
                 if (i >= nstage && !mbar_wait_bounded(empty0 + 8 * s, ph, g.wait_polls)) { ok = false; break; }
-                if constexpr (WRAP) {
+                if (i == g.drop_plane) {
+                    // test hook: this plane is never requested, so the consumers' wait for it runs out
+                } else if constexpr (WRAP) {
                     int zc = pstart + i;                           // nz >= 2R: one step brings it back
                     zc = zc < 0 ? zc + g.nz : (zc >= g.nz ? zc - g.nz : zc);
                     const uint32_t bar = full0 + 8 * s;

@@ -299,3 +299,33 @@ def test_fuse_rules_2d_fp64():
         assert p.get(b.KEY_FUSE_STEPS) == 1             # no FP64 temporal blocking in 3D
         with pytest.raises(b.StencilError):
             p.set(b.KEY_FUSE_STEPS, 2)
+
+
+def test_device_key_reads_minus_one_before_the_first_apply():
+    w = wl.star_weights(2, 1, -4.0, [1.0])
+    rc, h = b.stencil_plan((16, 16), 1, b.STAR, w, b.ZERO)
+    assert rc == b.OK
+    rc, dev = b.stencil_plan_get(h, b.KEY_DEVICE)
+    assert rc == b.OK and dev == -1
+    assert b.stencil_destroy(h) == b.OK
+
+
+@pytest.mark.gpu
+def test_a_plan_stays_on_the_device_of_its_first_apply():
+    """The plan's status word, taps, scratch grids and tensor maps live on the device that was
+    current at the first apply; an apply with another device current is refused."""
+    import torch
+    w = wl.star_weights(2, 1, -4.0, [1.0])
+    with b.Plan((64, 128), 1, b.STAR, w, b.ZERO) as p:
+        with torch.cuda.device(0):
+            src = torch.zeros((64, 128), dtype=torch.float32, device="cuda:0")
+            dst = torch.empty_like(src)
+            p.apply(src, dst, 1, 0)
+            assert p.get(b.KEY_DEVICE) == 0
+        if torch.cuda.device_count() < 2:
+            pytest.skip("needs two visible GPUs to make another device current")
+        with torch.cuda.device(1):
+            assert b.stencil_apply(p._h, src.data_ptr(), dst.data_ptr(), 1, 0) == b.ERR_INVALID
+        with torch.cuda.device(0):
+            p.apply(src, dst, 1, 0)
+            assert p.query_status() == b.OK

@@ -1001,30 +1001,57 @@ def test_f64_paper_shaped_box_iterated_and_type_checks():
 
 
 # ------------------------------------------------------------ bounded waits --
-def test_expired_device_wait_is_reported_and_the_context_stays_usable():
-    """Failure detection without a fault: the producer is told never to load one input
-    plane, so the consumers' bounded wait for it runs out (64 polls of at most 20 us), the
-    kernel returns early, and the host reads STENCIL_ERR_TIMEOUT from the status word.
-    Nothing traps or spins forever; the next apply on the same plan is correct again."""
-    dims = (8, 16, 128)                              # one CTA
-    w = wl.star_weights(3, 1, -6.0, [1.0])
-    a = wl.uniform_field(dims, -1.0, 1.0, 91)
+# (family, dims, radius, box, FP64, boundary, time steps, plan knobs, launches of the family's kernel per apply)
+_WAIT_CASES = [
+    ("stream", (8, 16, 128), 1, False, False, b.ZERO, 1, {}, 1),
+    ("stream box", (8, 16, 128), 1, True, False, b.ZERO, 1, {}, 1),
+    ("stream wrap", (8, 16, 128), 1, False, False, b.PERIODIC, 1, {}, 1),
+    ("fused 3d", (8, 16, 128), 1, False, False, b.ZERO, 2, {"fuse_steps": 2}, 1),
+    ("rows2d", (24, 128), 1, False, False, b.ZERO, 1, {}, 1),
+    ("rows2d box", (24, 128), 3, True, False, b.ZERO, 1, {}, 1),
+    ("rows2d fused", (40, 128), 1, False, False, b.ZERO, 4, {}, 1),
+    ("stream f64", (8, 16, 64), 1, False, True, b.ZERO, 1, {}, 1),
+    ("stream f64 wrap", (8, 16, 64), 1, False, True, b.PERIODIC, 1, {}, 1),
+    ("rows2d f64", (24, 64), 2, False, True, b.ZERO, 1, {}, 1),
+    ("rows2d fused f64", (40, 64), 1, False, True, b.ZERO, 4, {}, 1),
+]
+
+
+@pytest.mark.parametrize("family,dims,R,box,f64,boundary,steps,knobs,launches", _WAIT_CASES,
+                         ids=[c[0].replace(" ", "_") for c in _WAIT_CASES])
+def test_expired_device_wait_is_reported_and_the_context_stays_usable(family, dims, R, box, f64, boundary, steps,
+                                                                      knobs, launches):
+    """Failure detection without a fault, for every family of tiled kernels: the thread that
+    requests the input is told never to load one plane (3D) or batch of rows (2D), so the
+    bounded wait for it runs out (64 polls of at most 20 us), the kernel returns early, and the
+    host reads STENCIL_ERR_TIMEOUT from the status word.  Nothing traps or spins forever; the
+    next apply on the same plan is correct again."""
+    dt = np.float64 if f64 else np.float32
+    ndim = len(dims)
+    if steps > 1:                                    # iterated: non-negative weights that sum to one
+        w = wl.star_weights(ndim, 1, 1.0 - 0.2 * ndim, [0.1]).astype(dt)
+    else:
+        w = (wl.random_box_weights if box else wl.random_star_weights)(ndim, R, 5, dt)
+    a = wl.uniform_field(dims, -1.0, 1.0, 91, dt)
     src = torch.from_numpy(a).cuda()
     dst = torch.zeros_like(src)
     stream = torch.cuda.current_stream().cuda_stream
-    with b.Plan(dims, 1, b.STAR, w, b.ZERO, variant=b.VARIANT_STREAM) as p:
+    with b.Plan(dims, R, b.BOX if box else b.STAR, w, boundary, variant=b.VARIANT_STREAM, **knobs) as p:
         p.set(b.KEY_WAIT_POLLS, 64)
-        p.set(b.KEY_TEST_DROP_PLANE, 2)
-        p.apply(src, dst, 1, stream)
+        p.set(b.KEY_TEST_DROP_PLANE, 0)
+        l0 = p.launches
+        p.apply(src, dst, steps, stream)
+        assert p.launches - l0 == launches, f"{family}: the apply did not take the route under test"
         assert p.query_status() == b.ERR_TIMEOUT
         assert p.query_status() == b.OK              # the word is cleared by the query
         p.set(b.KEY_TEST_DROP_PLANE, -1)
         p.set(b.KEY_WAIT_POLLS, 1 << 20)
-        p.apply(src, dst, 1, stream)
+        p.apply(src, dst, steps, stream)
         assert p.query_status() == b.OK
     torch.cuda.synchronize()
-    want = oracle.apply(a, w, b.ZERO, 1)
-    assert np.max(np.abs(dst.cpu().numpy() - want)) <= wl.tolerance(w, 1.0, 1)
+    want = oracle.apply(a, w, boundary, steps)
+    err = np.max(np.abs(dst.cpu().numpy().astype(np.float64) - want.astype(np.float64)))
+    assert err <= wl.tolerance(w, 1.0, steps)        # the bound follows the dtype of the weights
 
 
 # ----------------------------------------------------- the five full configs --
@@ -1186,3 +1213,25 @@ def test_generic_kernel_on_a_full_3d_config():
     wk = wl.get("cfg2").scaled((128, 128, 128))
     a, w = wk.input(), wk.weights()
     check(wk.dims, wk.radius, wk.shape, w, wk.boundary, a, variant=b.VARIANT_GENERIC)
+
+
+# ------------------------------------------------- non-finite input at a face --
+@pytest.mark.parametrize("variant", [b.VARIANT_GENERIC, b.VARIANT_STREAM], ids=["generic", "stream"])
+@pytest.mark.parametrize("dims", [(24, 128), (6, 10, 128)], ids=["2d", "3d"])
+def test_infinity_at_a_face_does_not_leak_through_taps_that_leave_the_grid(dims, variant):
+    """A tap that leaves the grid contributes an exact zero whatever the grid holds next to the face.
+    With one +Inf at a corner point and a star whose taps are all non-zero, the result is infinite
+    exactly where a tap reaches the corner and finite (no NaN) everywhere else, on both kernel
+    families: the one-thread-per-point kernel once loaded the thread's own point for such a tap and
+    multiplied it by a zero weight, which turned the corner itself into NaN."""
+    ndim = len(dims)
+    a = wl.uniform_field(dims, -1.0, 1.0, 17)
+    a[(0,) * ndim] = np.inf
+    w = wl.random_star_weights(ndim, 1, 3)
+    assert np.count_nonzero(w) == 1 + 2 * ndim
+    got, used = gpu_sweep(dims, 1, b.STAR, w, b.ZERO, a, 1, variant=variant)
+    want = oracle.apply(a, w, b.ZERO, 1)
+    assert not np.isnan(want).any()
+    inf = np.isinf(want)
+    assert np.array_equal(np.isinf(got), inf) and np.array_equal(np.sign(got[inf]), np.sign(want[inf]))
+    assert np.max(np.abs(got[~inf] - want[~inf])) <= wl.tolerance(w, 1.0, 1)
