@@ -1,13 +1,18 @@
 #!/usr/bin/env python
 """Benchmark of the stencil sweep on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference] [--sharded]
 
 One "step" is one ``stencil_apply`` of the workload (all of its time steps)
-on a grid resident in HBM.  Rank 0 prints ONE JSON line.  With N > 1 (under
-torchrun) every rank runs its own replica of the workload: the sweep has no
-exchange step on one GPU, so there is no data-path collective; the timing is
-the max over ranks and the value is the sum of all ranks' points.
+on a grid resident in HBM.  Rank 0 prints ONE JSON line.
+
+With N > 1 (under torchrun) the default is replicas: every rank runs its own
+copy of the workload, there is no data-path collective, the time is the
+slowest rank's and the value the sum of all ranks' points ("weak").  With
+``--sharded`` the ranks instead share ONE grid, cut into slabs along the
+slowest axis (``paper_2608_21157_b200.sharded``): the boundary planes travel
+between neighbours by NCCL point-to-point sends, the value is the whole
+grid's point-updates over the slowest rank's time ("strong").
 
 ``--impl reference`` times the CPU oracle (the plain definition, as it
 stands) on a bounded slab of the same workload instead.
@@ -35,13 +40,15 @@ METRIC = "stencil_gpoints_per_s"
 UNIT = "GPoints/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+SM_COUNT, SM_MAX_MHZ = 148, 1965.0
 
-# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum +
-# dram__bytes_write.sum from an ncu capture; see profiles/).  None = not captured.
+# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of
+# one launch at the workload's full size, from the ncu captures summarised under profiles/).
+# None = not captured.
 NCU_TRAFFIC_BYTES = {
-    "cfg2": 978.1e6,    # stream kernel, star R=1: 2 x (268.5 MB read + 220.5 MB written) on the half grid
-    "cfg3": 1004.6e6,   # stream kernel, box R=1
-    "cfg4": 995.7e6,    # stream kernel, star R=4
+    "cfg2": 1023.6e6,   # stream kernel, star R=1, 512^3: 537.2 MB read + 486.4 MB written
+    "cfg3": 1047.0e6,   # stream kernel, box R=1, 512^3: 559.7 + 487.3
+    "cfg4": 1040.4e6,   # stream kernel, star R=4, 512^3: 553.3 + 487.1
     "cfg5": 99.9e6,     # one fused pass (2 time steps of 256^3): 77.7 MB read + 22.2 MB written
     "cfg5L": 1035.1e6,  # one fused pass (2 time steps of 512^3): 545.4 MB read + 489.7 MB written
     "heat2d": 756.3e6,  # one fused pass (4 time steps of 10240^2): 2.5 x (180.6 + 121.9 MB) captured on 4096 x 10240
@@ -66,7 +73,7 @@ class ClockSampler:
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_id: str, period_ms: int = 50):
+    def __init__(self, gpu_id: str, period_ms: int = 100):
         self.gpu_id, self.period_ms = gpu_id, period_ms
         self.rows, self.proc, self.thread = [], None, None
 
@@ -118,58 +125,124 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------
-# GPU arm
+# helpers of the GPU arm
 # ---------------------------------------------------------------------------
-def time_workload(torch, b, wk, steps, warmup, knobs, variant=None, per_launch_events=True):
-    """Times `steps` applies of workload `wk` with inputs resident in HBM.
-    Returns dict with batch ms/step, per-apply event ms, launches, plan info."""
-    dev = torch.device("cuda", torch.cuda.current_device())
-    a = wk.input()
-    src = torch.from_numpy(a).to(dev)
-    dst = torch.empty_like(src)
-    stream = torch.cuda.current_stream()
-    plan = b.Plan.for_workload(wk, variant=variant, **knobs)
-    for _ in range(max(warmup, 0)):
-        plan.apply(src, dst, wk.steps, stream.cuda_stream)
+def is_tiny(wk) -> bool:
+    """Launch-latency-bound: the host cannot issue applies as fast as the GPU retires them, so an
+    event after every apply would be what the loop measures."""
+    return wk.point_updates < (1 << 22)
+
+
+def host_warmup(torch, plan, src, dst, wk, stream, seconds=0.2):
+    """A launch-latency-bound workload measures the host's launch path, which takes some ten
+    thousand calls to reach its steady rate (7 us per apply at first, 4.1 us after): issue applies
+    for `seconds` before such a workload is timed."""
+    sp, dp, handle, t0 = src.data_ptr(), dst.data_ptr(), stream.cuda_stream, time.time()
+    while time.time() - t0 < seconds:
+        for _ in range(1000):
+            plan.apply(sp, dp, wk.steps, handle)
     torch.cuda.synchronize()
-    l0 = plan.launches
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+
+
+def time_applies(torch, plan, src, dst, wk, steps, stream, per_apply=True):
+    """`steps` applies, CUDA events on the launching stream.  Returns (total ms, per-apply ms or None)."""
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1 if per_apply else 2)]
+    sp, dp, handle, tsteps = src.data_ptr(), dst.data_ptr(), stream.cuda_stream, wk.steps
     evs[0].record(stream)
     for i in range(steps):
-        plan.apply(src, dst, wk.steps, stream.cuda_stream)
-        evs[i + 1].record(stream)
+        plan.apply(sp, dp, tsteps, handle)
+        if per_apply:
+            evs[i + 1].record(stream)
+    if not per_apply:
+        evs[1].record(stream)
     torch.cuda.synchronize()
     total_ms = evs[0].elapsed_time(evs[-1])
-    per = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
-    launches = plan.launches - l0
-    status = plan.query_status()
-    info = {"variant": plan.variant, "tile_y": plan.get(b.KEY_TILE_Y),
+    per = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)] if per_apply else None
+    return total_ms, per
+
+
+def graph_replay_ms(torch, plan, src, dst, wk, steps, stream):
+    """ms per apply of a CUDA graph that replays `steps` applies (the device-side rate of a
+    launch-latency-bound workload); None if capture fails."""
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(steps):
+                plan.apply(src, dst, wk.steps, torch.cuda.current_stream().cuda_stream)
+        graph.replay()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        graph.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        ms = g0.elapsed_time(g1) / steps
+        del graph
+        return ms
+    except Exception:
+        return None
+
+
+def plan_info(b, plan, wk):
+    return {"variant": plan.variant, "tile_y": plan.get(b.KEY_TILE_Y),
             "rows_per_thread": plan.get(b.KEY_ROWS_PER_THREAD),
             "fuse_steps": plan.get(b.KEY_FUSE_STEPS) if wk.steps > 1 else 1}
-    graph_ms = None
-    if wk.point_updates < (1 << 22):
-        # a launch-latency-bound workload: the host loop above cannot issue launches as fast
-        # as the GPU retires them, so also time a CUDA graph that replays `steps` applies
-        try:
-            side = torch.cuda.Stream()
-            side.wait_stream(stream)
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=side):
-                for _ in range(steps):
-                    plan.apply(src, dst, wk.steps, torch.cuda.current_stream().cuda_stream)
-            graph.replay()
-            torch.cuda.synchronize()
-            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            g0.record()
-            graph.replay()
-            g1.record()
-            torch.cuda.synchronize()
-            graph_ms = g0.elapsed_time(g1) / steps
-            del graph
-        except Exception:
-            graph_ms = None
-    return {"total_ms": total_ms, "per_apply_ms": per, "launches": launches, "status": status,
-            "plan": plan, "src": src, "dst": dst, "info": info, "input": a, "graph_ms_per_apply": graph_ms}
+
+
+def kernel_name(wk, info):
+    f64, fuse = wk.itemsize == 8, info["fuse_steps"]
+    if info["variant"] == "generic":
+        return "stencil_generic_kernel"
+    if fuse > 1:
+        if len(wk.dims) == 2:
+            return "stencil_rows2d_fused_f64_kernel" if f64 else "stencil_rows2d_fused_kernel"
+        return "stencil_fused_kernel"
+    if len(wk.dims) == 2:
+        return "stencil_rows2d_f64_kernel" if f64 else "stencil_rows2d_kernel"
+    if wk.boundary == wl.PERIODIC:
+        return "stencil_stream_f64_wrap_kernel" if f64 else "stencil_stream_wrap_kernel"
+    return "stencil_stream_f64_kernel" if f64 else "stencil_stream_kernel"
+
+
+def roofline_block(wk, info, ms_per_apply, launches_per_apply, peak, peak_kind, sm_mhz=None):
+    """Roofline of the dominant kernel: algorithmic bytes (one read + one write of the grid's
+    element type per point per time step) per launch over the launch's average duration, against
+    the measured copy bandwidth; sweeps with many taps are bound by plain FMA arithmetic instead
+    and report against 148 SMs x 128 fp32 (64 FP64) FMA lanes x 2 flop x the maximum SM clock."""
+    launches_per_apply = max(int(launches_per_apply), 1)
+    kernel_ms = ms_per_apply / launches_per_apply
+    steps_per_launch = max(wk.steps, 1) / launches_per_apply
+    algo_bytes = 2.0 * wk.itemsize * wk.npoints * steps_per_launch
+    achieved = algo_bytes / (kernel_ms / 1e3) / 1e9
+    f64 = wk.itemsize == 8
+    if is_tiny(wk):
+        return {"bound": "launch latency", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                "frac": round(achieved / peak, 4), "traffic": None, "kernel": kernel_name(wk, info),
+                "kernel_ms": round(kernel_ms, 5),
+                "note": "the grid fits L2 and one launch is shorter than its own latency: the fraction is not meaningful"}
+    r = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+         "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(wk.name),
+         "peak_kind": f"of {peak_kind} (copy bandwidth)", "kernel": kernel_name(wk, info),
+         "kernel_ms": round(kernel_ms, 5), "algorithmic_bytes_per_launch": int(algo_bytes),
+         "time_steps_per_launch": steps_per_launch,
+         "frac_of_nominal_8tbs": round(achieved / NOMINAL_HBM_GBS, 4)}
+    lanes = 64 if f64 else 128
+    taps = int(np.count_nonzero(wk.weights()))
+    alu_peak = SM_COUNT * lanes * 2 * SM_MAX_MHZ * 1e6 / 1e12
+    alu_achieved = 2.0 * taps * wk.npoints * steps_per_launch / (kernel_ms / 1e3) / 1e12
+    if alu_achieved / alu_peak > achieved / peak:
+        r.update({"bound": "alu", "achieved": round(alu_achieved, 2), "peak": round(alu_peak, 1),
+                  "unit": "TFLOP/s", "frac": round(alu_achieved / alu_peak, 4),
+                  "peak_kind": "148 SMs x %d FMA lanes x 2 flop x 1965 MHz (no measured peak for plain "
+                               "FMA; the part runs 1.5-1.8 GHz under its power cap)" % lanes,
+                  "hbm_frac_of_measured": round(achieved / peak, 4), "taps": taps})
+        if sm_mhz:
+            # the same fraction at the clock the part actually held while the kernel ran
+            r["frac_at_sampled_clock"] = round(alu_achieved / (alu_peak * sm_mhz / SM_MAX_MHZ), 4)
+            r["sampled_sm_mhz"] = sm_mhz
+    return r
 
 
 def config_summary(wk, total_ms, steps, peak):
@@ -200,6 +273,23 @@ def whole_job_gpoints(world, point_updates_per_apply, applies, total_ms):
     return world * point_updates_per_apply * applies / (total_ms / 1e3) / 1e9
 
 
+def sharded_job_summary(dims, radius, time_steps, halo_steps, applies, total_ms, world, itemsize):
+    """Sharded run: the ranks share ONE grid, so the job's point count is the grid's, whatever the
+    number of ranks, over the slowest rank's time.  Also the bytes a rank sends per time step: to
+    each neighbour `halo_steps * radius` planes once every `halo_steps` steps."""
+    npoints = 1
+    for d in dims:
+        npoints *= int(d)
+    plane_bytes = itemsize * npoints // int(dims[0])
+    neighbours = 0 if world == 1 else 2          # an inner rank's; the two end ranks of a chain have one
+    rounds = -(-int(time_steps) // int(halo_steps))
+    return {"value": npoints * int(time_steps) * applies / (total_ms / 1e3) / 1e9,
+            "exchange_bytes_per_rank_per_apply": neighbours * halo_steps * radius * plane_bytes * rounds,
+            "exchange_bytes_per_rank_per_time_step":
+                neighbours * halo_steps * radius * plane_bytes * rounds / max(int(time_steps), 1),
+            "messages_per_rank_per_apply": neighbours * rounds}
+
+
 def pick_workload(args):
     wk = wl.get(args.workload)
     if args.dims:
@@ -207,11 +297,7 @@ def pick_workload(args):
     return wk
 
 
-def run_gpu(args):
-    import torch
-    from paper_2608_21157_b200 import binding as b
-    from paper_2608_21157_b200 import build as build_mod
-
+def init_ranks(torch, sharded=False):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -223,6 +309,18 @@ def run_gpu(args):
         import torch.distributed as dist_mod
         dist = dist_mod
         dist.init_process_group("nccl", device_id=torch.device("cuda", torch.cuda.current_device()))
+    return rank, world, dist
+
+
+# ---------------------------------------------------------------------------
+# GPU arm: one grid per rank
+# ---------------------------------------------------------------------------
+def run_gpu(args):
+    import torch
+    from paper_2608_21157_b200 import binding as b
+    from paper_2608_21157_b200 import build as build_mod
+
+    rank, world, dist = init_ranks(torch)
     if rank == 0:
         build_mod.build()
     if dist is not None:
@@ -257,31 +355,47 @@ def run_gpu(args):
     plan = b.Plan.for_workload(wk, variant=variant, **knobs)
     for _ in range(args.warmup):
         plan.apply(src, dst, wk.steps, stream.cuda_stream)
+    if is_tiny(wk):
+        host_warmup(torch, plan, src, dst, wk, stream)
     barrier()
     l0 = plan.launches
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     t_wall0 = time.time()
-    evs[0].record(stream)
-    for i in range(args.steps):
-        plan.apply(src, dst, wk.steps, stream.cuda_stream)
-        evs[i + 1].record(stream)
+    total_ms, per_apply = time_applies(torch, plan, src, dst, wk, args.steps, stream, per_apply=not is_tiny(wk))
     barrier()
     t_wall1 = time.time()
-    total_ms = evs[0].elapsed_time(evs[-1])
-    per_apply = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)]
     launches = plan.launches - l0
     if plan.query_status() != b.OK:
         raise SystemExit("device status word reports a timeout; results are invalid")
-
-    # keep the same kernel running long enough for nvidia-smi to see clocks under load
-    t_load0 = time.time()
-    while time.time() - t_load0 < args.clock_seconds:
-        for _ in range(20):
-            plan.apply(src, dst, wk.steps, stream.cuda_stream)
-        torch.cuda.synchronize()
-    t_load1 = time.time()
-
     total_ms_max = max_over_ranks(total_ms, dist, dev)
+
+    # ---- sustained: the same applies back to back for >= clock_seconds, timed as one region; the
+    # clock samples of exactly this window go with it -----------------------------------------
+    sustained = None
+    t_load0 = t_load1 = time.time()
+    if args.clock_seconds > 0:
+        per = max(total_ms / max(args.steps, 1), 1e-3)
+        batch = max(1, min(2000, int(100.0 / per)))            # ~0.1 s of applies between host syncs
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_sus = 0
+        torch.cuda.synchronize()
+        t_load0 = time.time()
+        s0.record(stream)
+        while time.time() - t_load0 < args.clock_seconds:
+            for _ in range(batch):
+                plan.apply(src, dst, wk.steps, stream.cuda_stream)
+            n_sus += batch
+            torch.cuda.synchronize()
+        s1.record(stream)
+        torch.cuda.synchronize()
+        t_load1 = time.time()
+        sus_ms = s0.elapsed_time(s1)
+        sus_clocks = sampler.summary(t_load0, t_load1)
+        sustained = {"value": round(wk.point_updates * n_sus / (sus_ms / 1e3) / 1e9, 3), "unit": UNIT,
+                     "applies": n_sus, "seconds": round(sus_ms / 1e3, 3),
+                     "sm_mhz": sus_clocks.get("sm_mhz"), "reasons": sus_clocks.get("reasons"),
+                     "power_w_max": sus_clocks.get("power_w_max"),
+                     "what": "the same applies back to back, CUDA events around the whole window "
+                             "(host syncs every ~0.1 s included); this rank"}
 
     # ---- end to end: host buffers through the C ABI, copies inside the timing --
     e2e = None
@@ -305,82 +419,40 @@ def run_gpu(args):
                "api": "stencil_apply_host (pinned host buffers)"}
         del hsrc, hdst
 
+    clocks = sampler.summary(t_wall0, t_load1)
+    clocks["sampled_over"] = "timed region plus the %.1f s sustained window of the same applies" % (t_load1 - t_load0)
+
     # ---- roofline of the dominant kernel --------------------------------------
+    info = plan_info(b, plan, wk)
     launches_per_apply = max(launches // max(args.steps, 1), 1)
-    kernel_ms = statistics.mean(per_apply) / launches_per_apply
-    # algorithmic bytes: 8 B (one fp32 read + one write) per point per time step; a launch
-    # advances N points by (time steps per apply / launches per apply) steps
-    steps_per_launch = max(wk.steps, 1) / launches_per_apply
-    algo_bytes = 2.0 * wk.itemsize * wk.npoints * steps_per_launch
-    achieved = algo_bytes / (kernel_ms / 1e3) / 1e9
-    fuse = plan.get(b.KEY_FUSE_STEPS) if wk.steps > 1 else 1
-    f64 = wk.itemsize == 8
-    if plan.variant == "generic":
-        kernel_name = "stencil_generic_kernel"
-    elif fuse > 1:
-        kernel_name = "stencil_rows2d_fused_kernel" if len(wk.dims) == 2 else "stencil_fused_kernel"
-    elif len(wk.dims) == 2:
-        kernel_name = "stencil_rows2d_f64_kernel" if f64 else "stencil_rows2d_kernel"
-    else:
-        kernel_name = "stencil_stream_f64_kernel" if f64 else "stencil_stream_kernel"
-    roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
-                "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(wk.name),
-                "peak_kind": f"of {peak_kind} (copy bandwidth)", "kernel": kernel_name,
-                "kernel_ms": round(kernel_ms, 5), "algorithmic_bytes_per_launch": int(algo_bytes),
-                "time_steps_per_launch": steps_per_launch,
-                "frac_of_nominal_8tbs": round(achieved / NOMINAL_HBM_GBS, 4)}
-    # The sweeps with many taps are bound by plain FMA arithmetic, not by memory: report
-    # against whichever limit the kernel is closer to.  ALU peak = 148 SMs x 128 fp32 (64 FP64)
-    # FMA lanes x 2 flop x the maximum SM clock (1965 MHz).
-    taps = int(np.count_nonzero(wk.weights()))
-    alu_peak = 148 * (64 if f64 else 128) * 2 * 1.965e9 / 1e12
-    alu_achieved = 2.0 * taps * wk.npoints * steps_per_launch / (kernel_ms / 1e3) / 1e12
-    if alu_achieved / alu_peak > achieved / peak:
-        roofline.update({"bound": "alu", "achieved": round(alu_achieved, 2), "peak": round(alu_peak, 1),
-                         "unit": "TFLOP/s", "frac": round(alu_achieved / alu_peak, 4),
-                         "peak_kind": "148 SMs x %d FMA lanes x 2 flop x 1965 MHz (no measured peak for plain "
-                                      "FMA; the part runs 1.5-1.8 GHz under its power cap)" % (64 if f64 else 128),
-                         "hbm_frac_of_measured": round(achieved / peak, 4), "taps": taps})
-    info = {"variant": plan.variant, "tile_y": plan.get(b.KEY_TILE_Y),
-            "rows_per_thread": plan.get(b.KEY_ROWS_PER_THREAD), "fuse_steps": fuse}
+    mean_apply_ms = statistics.mean(per_apply) if per_apply else total_ms / args.steps
+    roofline = roofline_block(wk, info, mean_apply_ms, launches_per_apply, peak, peak_kind, clocks.get("sm_mhz"))
     plan.destroy()
     del src, dst
+    torch.cuda.empty_cache()
 
     # ---- the other configs, short runs, rank 0 only ----------------------------
     all_cfg = {}
+    headline = dict(config_summary(wk, total_ms_max, args.steps, peak), **info)
+    headline["launches_per_apply"] = launches_per_apply
+    headline["roofline"] = roofline
+    headline["input_sha256"] = wl.sha256(a_host)
+    if rank == 0 and args.cudnn:
+        headline["cudnn_reference"] = cudnn_reference(torch, wk, a_host)
     if rank == 0 and not args.no_all_configs:
         for name in args.also.split(","):
             if not name or name == wk.name:
                 continue
-            w2 = wl.get(name)
-            n2 = args.also_steps
-            r = time_workload(torch, b, w2, n2, 3, {}, None)
-            s = config_summary(w2, r["total_ms"], n2, peak)
-            s.update(r["info"])
-            if r.get("graph_ms_per_apply"):
-                s["ms_per_apply_cuda_graph"] = round(r["graph_ms_per_apply"], 5)
-                s["gpoints_per_s_cuda_graph"] = round(w2.point_updates / r["graph_ms_per_apply"] / 1e6, 2)
-                s["note"] = "launch-latency-bound: the graph replay figure is the device-side rate"
-            s["launches_per_apply"] = r["launches"] // n2
-            all_cfg[name] = s
-            r["plan"].destroy()
-            del r
-            torch.cuda.empty_cache()
-    all_cfg[wk.name] = dict(config_summary(wk, total_ms_max, args.steps, peak), **info)
-
-    # ---- cuDNN reference point (fp32 conv via PyTorch), rank 0 only ------------
-    cudnn = None
-    if rank == 0 and args.cudnn:
-        cudnn = cudnn_reference(torch, wk, a_host)
+            all_cfg[name] = one_config(torch, b, wl.get(name), args, peak, peak_kind, sampler)
+    all_cfg[wk.name] = headline
 
     sampler.stop()
-    clocks = sampler.summary(t_wall0, t_load1)
-    clocks["sampled_over"] = "timed region plus %.1f s of the same kernel" % (t_load1 - t_load0)
 
     # ---- CPU baseline: the oracle, on this machine's cores, rank 0 at N=1 only ------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(wk, a_host, budget_s=args.cpu_seconds)
+        all_cfg[wk.name]["cpu_baseline"] = cpu
 
     if rank == 0:
         pts = world * wk.point_updates * args.steps
@@ -396,15 +468,17 @@ def run_gpu(args):
                        "l2": "grid in + out = %.0f MiB, larger than the 126 MB L2; no flush" % (2 * a_host.nbytes / 2**20)
                              if 2 * a_host.nbytes > 126e6 else "working set fits L2; warm-L2 figure",
                        "parallelism": "replicas only (one full grid per GPU, no exchange)" if world > 1 else "1 GPU",
+                       "input_sha256": headline["input_sha256"], "numpy": np.__version__,
                        **info},
             "effective_gbs": round(2.0 * wk.itemsize * pts / (total_ms_max / 1e3) / 1e9 / world, 1),
             "gpu_launches": int(launches),
+            "sustained": sustained,
             "clocks": clocks,
             "e2e": e2e,
             "roofline": roofline,
             "cpu_baseline": cpu,
             "all_configs": all_cfg,
-            "cudnn_reference": cudnn,
+            "cudnn_reference": headline.get("cudnn_reference"),
             "paper_context": "paper: 1.53x over cuDNN on A100-PCIE-40GB, FP64, 2D box R=3 10240^2 (4.71 ms/step); other hardware and precision",
         }
         print(json.dumps(line))
@@ -413,8 +487,78 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def one_config(torch, b, wk, args, peak, peak_kind, sampler):
+    """A short run of one more workload with its own roofline block, cuDNN reference point, a
+    bounded oracle baseline and the hash of its input."""
+    n = args.also_steps
+    dev = torch.device("cuda", torch.cuda.current_device())
+    a = wk.input()
+    src = torch.from_numpy(a).to(dev)
+    dst = torch.empty_like(src)
+    stream = torch.cuda.current_stream()
+    plan = b.Plan.for_workload(wk)
+    for _ in range(3):
+        plan.apply(src, dst, wk.steps, stream.cuda_stream)
+    if is_tiny(wk):
+        host_warmup(torch, plan, src, dst, wk, stream)
+        n = max(n, 2000)                                 # ... and time enough calls to average over
+    torch.cuda.synchronize()
+    l0 = plan.launches
+    t0 = time.time()
+    total_ms, _ = time_applies(torch, plan, src, dst, wk, n, stream, per_apply=False)
+    t1 = time.time()
+    launches = plan.launches - l0
+    info = plan_info(b, plan, wk)
+    s = config_summary(wk, total_ms, n, peak)
+    s.update(info)
+    s["launches_per_apply"] = launches // n
+    s["status"] = plan.query_status()
+    clk = None
+    if not is_tiny(wk) and args.also_clock_seconds > 0:
+        # the same applies for a little longer, so that the clock sampler sees the part under this load
+        per = max(total_ms / n, 1e-3)
+        batch = max(1, min(500, int(50.0 / per)))
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        m = 0
+        torch.cuda.synchronize()
+        c0 = time.time()
+        s0.record(stream)
+        while time.time() - c0 < args.also_clock_seconds:
+            for _ in range(batch):
+                plan.apply(src, dst, wk.steps, stream.cuda_stream)
+            m += batch
+            torch.cuda.synchronize()
+        s1.record(stream)
+        torch.cuda.synchronize()
+        c1 = time.time()
+        window = sampler.summary(c0, c1)
+        clk = window.get("sm_mhz")
+        s["sustained"] = {"gpoints_per_s": round(wk.point_updates * m / (s0.elapsed_time(s1) / 1e3) / 1e9, 2),
+                          "seconds": round(s0.elapsed_time(s1) / 1e3, 3), "sm_mhz": clk,
+                          "reasons": window.get("reasons")}
+    s["roofline"] = roofline_block(wk, info, total_ms / n, s["launches_per_apply"], peak, peak_kind, clk)
+    if is_tiny(wk):
+        g = graph_replay_ms(torch, plan, src, dst, wk, min(n, 200), stream)
+        if g:
+            s["ms_per_apply_cuda_graph"] = round(g, 5)
+            s["gpoints_per_s_cuda_graph"] = round(wk.point_updates / g / 1e6, 2)
+            s["note"] = ("launch-latency-bound: gpoints_per_s is the host-driven rate (one C-ABI call per "
+                         "apply), the graph replay figure the device-side rate")
+    plan.destroy()
+    del src, dst
+    torch.cuda.empty_cache()
+    s["input_sha256"] = wl.sha256(a)
+    if args.cudnn:
+        s["cudnn_reference"] = cudnn_reference(torch, wk, a)
+        torch.cuda.empty_cache()
+    if not args.no_cpu_baseline and args.also_cpu_seconds > 0:
+        s["cpu_baseline"] = cpu_baseline(wk, a, budget_s=args.also_cpu_seconds)
+    return s
+
+
 def cudnn_reference(torch, wk, a_host, iters=5):
-    """fp32 conv2d/conv3d (TF32 off) on the same GPU: a reference point only."""
+    """conv2d/conv3d of PyTorch (cuDNN; TF32 off) with the dense (2R+1)^d kernel on the same GPU, in
+    the workload's own dtype, iterated workloads as chained calls: a reference point only."""
     try:
         import torch.nn.functional as F
         if wk.boundary != wl.ZERO:
@@ -441,9 +585,103 @@ def cudnn_reference(torch, wk, a_host, iters=5):
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / iters
         return {"ms_per_apply": round(ms, 4), "gpoints_per_s": round(wk.point_updates / (ms / 1e3) / 1e9, 2),
-                "what": "torch.nn.functional.conv%dd fp32, TF32 off, dense (2R+1)^d kernel" % wk.ndim}
+                "what": "torch.nn.functional.conv%dd %s, TF32 off, dense (2R+1)^d kernel of %d entries, %d chained call(s)"
+                        % (wk.ndim, "fp64" if wk.itemsize == 8 else "fp32", (2 * wk.radius + 1) ** wk.ndim,
+                           max(wk.steps, 1))}
     except Exception as e:  # a reference point must never sink the benchmark
         return {"unavailable": f"{type(e).__name__}: {str(e)[:120]}"}
+
+
+# ---------------------------------------------------------------------------
+# GPU arm: one grid shared by all ranks (slab decomposition, halo exchange over NCCL)
+# ---------------------------------------------------------------------------
+def run_sharded(args):
+    import torch
+    from paper_2608_21157_b200 import binding as b
+    from paper_2608_21157_b200 import build as build_mod
+    from paper_2608_21157_b200.sharded import ShardedSweep
+
+    os.environ.setdefault("NCCL_DEBUG", "INFO")         # the communicator log stays on: it shows the transport
+    rank, world, dist = init_ranks(torch, sharded=True)
+    if rank == 0:
+        build_mod.build()
+    if dist is not None:
+        dist.barrier()
+    b.load()
+    wk = pick_workload(args)
+    if wk.itemsize == 8 and wk.dims[-1] % 2 or wk.itemsize == 4 and wk.dims[-1] % 4:
+        raise SystemExit("--sharded needs rows that are a multiple of 16 bytes")
+    dev = torch.device("cuda", torch.cuda.current_device())
+    stream = torch.cuda.current_stream()
+    G = max(1, int(args.halo_steps))
+    sw = ShardedSweep(wk.dims, wk.radius, wk.shape, wk.weights(), wk.boundary, rank=rank, world=world, dist=dist,
+                      halo_steps=G, overlap=not args.no_overlap)
+    a_host = wk.input()                                  # every rank draws the same seeded field and keeps its slab
+    ext = torch.zeros(sw.local_dims, dtype=torch.from_numpy(a_host[:1]).dtype, device=dev)
+    sw.interior(ext).copy_(torch.from_numpy(a_host[sw.z0:sw.z1]))
+    start = ext.clone()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    props = torch.cuda.get_device_properties(torch.cuda.current_device())
+    sampler = ClockSampler(f"GPU-{props.uuid}" if hasattr(props, "uuid") else str(torch.cuda.current_device()))
+    sampler.start()
+    for _ in range(args.warmup):
+        ext.copy_(start)
+        sw.apply(ext, wk.steps)
+    barrier()
+    launches0 = sw._plan.launches
+    total = 0.0
+    t_wall0 = time.time()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(args.steps):                          # the restore of the start field stays outside the timing
+        ext.copy_(start)
+        barrier()
+        e0.record(stream)
+        sw.apply(ext, wk.steps)
+        e1.record(stream)
+        barrier()
+        total += max_over_ranks(e0.elapsed_time(e1), dist, dev)
+    t_wall1 = time.time()
+    sampler.stop()
+    clocks = sampler.summary(t_wall0, t_wall1)
+    clocks["sampled_over"] = "the timed applies of rank 0 (restores of the start field and barriers included)"
+    launches = sw._plan.launches - launches0
+    status = sw._plan.query_status()
+    info = {"variant": sw._plan.variant, "fuse_steps": sw._plan.get(b.KEY_FUSE_STEPS) if wk.steps > 1 else 1}
+    sw.close()
+    if rank == 0:
+        if status != b.OK:
+            raise SystemExit("device status word reports a timeout; results are invalid")
+        s = sharded_job_summary(wk.dims, wk.radius, wk.steps, G, args.steps, total, world, wk.itemsize)
+        peak, peak_kind = measured_hbm_peak()
+        line = {
+            "metric": METRIC, "value": round(s["value"], 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(total / args.steps, 5), "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "f64" if wk.itemsize == 8 else "f32",
+            "data": "synthetic (seeded numpy default_rng fields; see config.workload)",
+            "config": {"workload": f"{wk.name}: {wk.description}", "dims": list(wk.dims), "radius": wk.radius,
+                       "taps": wk.taps(), "time_steps_per_apply": wk.steps,
+                       "parallelism": "one grid in %d slab(s) along the slowest axis, %d plane(s) per rank; halo "
+                                      "exchange by NCCL point-to-point sends into the receiver's ghost planes"
+                                      % (world, wk.dims[0] // world),
+                       "halo_steps": G, "overlap_exchange_with_inner_planes": bool(sw.overlap),
+                       "exchange_bytes_per_rank_per_time_step": int(s["exchange_bytes_per_rank_per_time_step"]),
+                       "messages_per_rank_per_apply": s["messages_per_rank_per_apply"],
+                       "timing": "each apply between barriers, CUDA events on the launching stream, max over ranks",
+                       **info},
+            "effective_gbs": round(2.0 * wk.itemsize * s["value"], 1),
+            "frac_of_measured_hbm_times_n_gpus": round(2.0 * wk.itemsize * s["value"] / (peak * world), 4),
+            "gpu_launches": int(launches), "clocks": clocks,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
 
 
 # ---------------------------------------------------------------------------
@@ -517,7 +755,8 @@ def run_reference(args):
         "ms_per_step": round(dt / args.steps * 1e3, 3), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64 accumulate, f32 store", "data": "synthetic (same seeded fields)",
         "config": {"workload": f"{wk.name}: {wk.description}", "dims": list(wk.dims), "radius": wk.radius,
-                   "taps": wk.taps(), "sample": sample_desc},
+                   "taps": wk.taps(), "time_steps_per_apply": wk.steps, "sample": sample_desc,
+                   "input_sha256": wl.sha256(a_host)},
         "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": sample_desc},
         "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -532,7 +771,7 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--workload", default=None, choices=sorted(wl.WORKLOADS))
     ap.add_argument("--dims", default=None, help="override the grid, e.g. 256,512,512 (profiling on smaller cases)")
     ap.add_argument("--variant", default="auto", choices=["auto", "generic", "stream", "fused"])
     ap.add_argument("--tile-y", dest="tile_y", type=int, default=None)
@@ -543,6 +782,10 @@ def main():
     ap.add_argument("--streaming-store", dest="streaming_store", type=int, default=None)
     ap.add_argument("--also", default="cfg1,cfg3,cfg4,cfg5,cfg5L,cfg5L_periodic,paper2d,paper2d_f64,heat2d", help="other workloads summarised in all_configs")
     ap.add_argument("--also-steps", dest="also_steps", type=int, default=20)
+    ap.add_argument("--also-cpu-seconds", dest="also_cpu_seconds", type=float, default=2.0,
+                    help="oracle baseline beside every entry of all_configs (0 = off)")
+    ap.add_argument("--also-clock-seconds", dest="also_clock_seconds", type=float, default=0.5,
+                    help="sustained window (and clock samples) of every entry of all_configs (0 = off)")
     ap.add_argument("--no-all-configs", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", dest="e2e_steps", type=int, default=10)
@@ -551,11 +794,20 @@ def main():
     ap.add_argument("--reference-seconds", dest="reference_seconds", type=float, default=90.0)
     ap.add_argument("--clock-seconds", dest="clock_seconds", type=float, default=1.5)
     ap.add_argument("--cudnn", type=int, default=1)
+    ap.add_argument("--sharded", action="store_true",
+                    help="all ranks share one grid (slabs along the slowest axis, halo exchange over NCCL)")
+    ap.add_argument("--halo-steps", dest="halo_steps", type=int, default=2,
+                    help="--sharded: time steps between two halo exchanges (1 overlaps the exchange with the inner planes)")
+    ap.add_argument("--no-overlap", action="store_true", help="--sharded, halo-steps 1: exchange first, then sweep")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.workload is None:
+        args.workload = "cfg5L" if args.sharded else "cfg2"
     if args.impl == "reference":
         run_reference(args)
+    elif args.sharded:
+        run_sharded(args)
     else:
         run_gpu(args)
 

@@ -91,7 +91,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->nx = ndim == 3 ? (int)dims[2] : (int)dims[1];
     p->npoints = n;
     p->radius = radius; p->shape = shape; p->boundary = boundary;
-    p->device = -1;
+    p->device = -1; p->sms = 0;
     p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0; p->src_padded = false; p->fused_wrap = false; p->stream_wrap = false; p->periodic_route = 0;
     for (int l = 0; l <= kMaxFuseLevels; ++l) p->d_ctaps[l] = nullptr;
     p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr; p->fused2d64_cfg = nullptr;

@@ -224,6 +224,7 @@ struct stencil_plan_s {
     const stencil_host::Stream64Config* stream64_cfg;
     // device state (created lazily, on the device current at first apply)
     int device;
+    int sms;                       // multiprocessors of that device
     stencil::Tap* d_taps;
     int* d_status;
     float* scratch;                // N floats, iteration ping-pong
@@ -309,7 +310,8 @@ private:
 };
 
 // ---- host_common.cu ---------------------------------------------------------
-int sm_count();
+int sm_count();                    // multiprocessors of the current device
+inline int plan_sms(const stencil_plan_s* p) { return p->sms > 0 ? p->sms : sm_count(); }
 int ensure_device_state(stencil_plan_s* p);
 int check_device(const stencil_plan_s* p);
 int ensure_grid(float** slot, int64_t npoints);

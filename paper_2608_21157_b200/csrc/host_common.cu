@@ -62,6 +62,7 @@ int ensure_device_state(stencil_plan_s* p) {
         return rc;
     }
     p->device = dev;
+    p->sms = sm_count();
     p->d_status = status;
     p->d_taps = taps;
     p->d_taps64 = taps64;
@@ -160,7 +161,7 @@ int launch_generic(stencil_plan_s* p, const float* src, float* dst, cudaStream_t
 
 int launch_generic_f64(stencil_plan_s* p, const double* src, double* dst, cudaStream_t st) {
     Grid g{p->nz, p->ny, p->nx};
-    const int grid = generic_grid_size(g, sm_count());
+    const int grid = generic_grid_size(g, plan_sms(p));
     const int ntaps = (int)p->taps64.size();
     if (p->boundary == STENCIL_PERIODIC)
         stencil_generic_kernel<true, double><<<grid, kGenericThreads, 0, st>>>(src, dst, g, p->d_taps64, ntaps);
@@ -174,7 +175,7 @@ int launch_generic_f64(stencil_plan_s* p, const double* src, double* dst, cudaSt
 int launch_generic_taps(stencil_plan_s* p, const float* src, float* dst, const Tap* d_taps, int ntaps,
                         cudaStream_t st) {
     Grid g{p->nz, p->ny, p->nx};
-    const int grid = generic_grid_size(g, sm_count());
+    const int grid = generic_grid_size(g, plan_sms(p));
     if (p->boundary == STENCIL_PERIODIC)
         stencil_generic_kernel<true><<<grid, kGenericThreads, 0, st>>>(src, dst, g, d_taps, ntaps);
     else

@@ -220,8 +220,8 @@ int launch_rows2d_fused64(stencil_plan_s* p, const double* src, double* dst, int
     while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
     const size_t smem = smem_for(stages);
     if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-    int dev = -1, occ = 1;
-    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    const int dev = p->device;                       // current: the apply entry points have checked it
+    int occ = 1;
     {
         std::lock_guard<std::mutex> lock(g_config_mutex);
         if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->occ_smem = 0; cfg->cache_device = dev; }
@@ -253,7 +253,7 @@ int launch_rows2d_fused64(stencil_plan_s* p, const double* src, double* dst, int
     int chunk = p->chunk_z;
     if (chunk <= 0) {                                 // same sizing rule as the fp32 kernel
         const int H = nlev * p->radius;
-        const int slots = occ * sm_count() * cfg->NW;
+        const int slots = occ * plan_sms(p) * cfg->NW;
         const int nch_max = std::max(1, slots / g.strips);
         const int chunk_min = (p->ny + nch_max - 1) / nch_max;
         int nbatch = std::max(1, (chunk_min + 2 * H + cfg->YB - 1) / cfg->YB);
@@ -315,8 +315,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
         const size_t smem = smem_for(stages);
         if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-        int dev = -1;
-        if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+        const int dev = p->device;                   // current: the apply entry points have checked it
         {
             std::lock_guard<std::mutex> lock(g_config_mutex);
             if (dev != cfg->cache_device) {
@@ -363,7 +362,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
                 }
                 occ64 = cfg->occ;
             }
-            chunk = short_chunk_star1(span, (int64_t)g.tiles_x * g.tiles_y, (int64_t)occ64 * sm_count());
+            chunk = short_chunk_star1(span, (int64_t)g.tiles_x * g.tiles_y, (int64_t)occ64 * plan_sms(p));
         }
         if (p->chunk_z <= 0 && (p->radius >= 4 || (p->shape == STENCIL_BOX && p->radius >= 2))) {
             // The radius-4 star is no longer bound by memory alone (25 DFMA and 15 shared-memory
@@ -373,7 +372,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
             // CTAs fill whole waves of the two-per-SM slots at the least cost (512^3: one chunk,
             // 296 CTAs, 356 against 313 GPoints/s with 64-plane chunks).
             const int64_t tiles = (int64_t)g.tiles_x * g.tiles_y;
-            const int64_t slots = 2 * (int64_t)sm_count();
+            const int64_t slots = 2 * (int64_t)plan_sms(p);
             double best = 1e300;
             for (int n = 1; n <= std::max(1, span / (4 * p->radius)); ++n) {
                 const int c = (span + n - 1) / n;
@@ -411,8 +410,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
         const size_t smem = smem_for(stages);
         if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-        int dev = -1;
-        if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+        const int dev = p->device;                   // current: the apply entry points have checked it
         {
             std::lock_guard<std::mutex> lock(g_config_mutex);
             if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->cache_device = dev; }
@@ -434,7 +432,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         int chunk = p->chunk_z;
         if (chunk <= 0) {                             // same sizing rule as the fp32 kernel
             const int R = p->radius;
-            const int slots = 2 * sm_count() * cfg->NW;
+            const int slots = 2 * plan_sms(p) * cfg->NW;
             const int nch_max = std::max(1, slots / g.strips);
             const int chunk_min = (span + nch_max - 1) / nch_max;
             int nbatch = std::max(1, (chunk_min + 2 * R + cfg->YB - 1) / cfg->YB);

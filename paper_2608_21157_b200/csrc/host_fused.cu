@@ -158,8 +158,7 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
     int occ = 1;
     {
         // shared-memory limit and occupancy of the kernel, asked once per device and size
-        int dev = -1;
-        if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+        const int dev = p->device;                   // current: the apply entry points have checked it
         std::lock_guard<std::mutex> lock(g_config_mutex);
         if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->occ_smem = 0; cfg->cache_device = dev; }
         if (smem > cfg->smem_allowed) {
@@ -191,7 +190,7 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
         // planes: cut z into the number of chunks whose CTAs fill whole waves of the machine's
         // resident-CTA slots at the least total cost, a chunk costing its planes plus the
         // 2*T*R extra input planes and the start-up of its pipeline.
-        const int slots = occ * sm_count();
+        const int slots = occ * plan_sms(p);
         const int max_chunks = std::max(1, p->nz / (4 * T * R));
         const double fill = 4.0;
         double best = 1e300;

@@ -27,7 +27,7 @@ int pad_periodic(stencil_plan_s* p, const T* src, cudaStream_t st, const T** pad
     }
     Grid g{p->nz, p->ny, p->nx};
     const int64_t cells = (int64_t)(*pnx / Vec16<T>::n) * *pny * *pnz;
-    const int grid = (int)std::min<int64_t>((cells + 255) / 256, (int64_t)sm_count() * 32);
+    const int grid = (int)std::min<int64_t>((cells + 255) / 256, (int64_t)plan_sms(p) * 32);
     stencil_pad_periodic_kernel<T><<<grid, 256, 0, st>>>(src, reinterpret_cast<T*>(p->pad), g, R, rz);
     if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
     p->launches++;
@@ -43,7 +43,7 @@ int repitch_rows(stencil_plan_s* p, const T* src, T* dst, int nx, int src_pitch,
     while ((1 << lanes_log2) < nx && lanes_log2 < 8) ++lanes_log2;
     const int rows_per_cta = 256 >> lanes_log2;
     const int64_t ctas = (rows + 4 * rows_per_cta - 1) / (4 * rows_per_cta);      // a thread takes 4 rows per round
-    const int grid = (int)std::min<int64_t>(ctas, (int64_t)sm_count() * 16);
+    const int grid = (int)std::min<int64_t>(ctas, (int64_t)plan_sms(p) * 16);
     stencil_repitch_rows_kernel<T><<<grid, 256, 0, st>>>(src, dst, rows, nx, src_pitch, dst_pitch, lanes_log2);
     if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
     p->launches++;
@@ -101,7 +101,7 @@ int apply_periodic(stencil_plan_s* p, const T* in, T* out, int steps, cudaStream
     const Grid g{p->nz, p->ny, p->nx};
     const int nz = p->nz, ny = p->ny, nx = p->nx;
     const int64_t shell = cells / Vec16<T>::n - (int64_t)nz * ny * (nx / Vec16<T>::n);
-    const int shell_grid = (int)std::max<int64_t>(1, std::min<int64_t>((shell + 255) / 256, (int64_t)sm_count() * 16));
+    const int shell_grid = (int)std::max<int64_t>(1, std::min<int64_t>((shell + 255) / 256, (int64_t)plan_sms(p) * 16));
     for (int k = 0; k + 1 < steps && rc == STENCIL_OK; ++k) {
         {
             ScopedGridView view(p, pnz, pny, pnx, 0, STENCIL_ZERO);
@@ -151,7 +151,7 @@ int apply_periodic_corrected(stencil_plan_s* p, const T* in, T* out, T* other, i
     const Grid g{p->nz, p->ny, p->nx};
     const int64_t shell = (int64_t)2 * rz * g.ny * g.nx + (int64_t)(g.nz - 2 * rz) * 2 * R * g.nx +
                           (int64_t)(g.nz - 2 * rz) * (g.ny - 2 * R) * 2 * R;
-    const int shell_grid = (int)std::max<int64_t>(1, std::min<int64_t>((shell + 255) / 256, (int64_t)sm_count() * 16));
+    const int shell_grid = (int)std::max<int64_t>(1, std::min<int64_t>((shell + 255) / 256, (int64_t)plan_sms(p) * 16));
     const T* src = in;
     for (int k = 0; k < steps; ++k) {
         T* dst = ((steps - 1 - k) % 2 == 0) ? out : other;
@@ -368,7 +368,7 @@ int apply_periodic_fused(stencil_plan_s* p, const T* in, T* out, T* other, int s
         } else {
             const int64_t shell = (int64_t)2 * hz * g.ny * g.nx + (int64_t)inner_z * 2 * H * g.nx +
                                   (int64_t)inner_z * inner_y * 2 * H;
-            const int shell_grid = (int)std::max<int64_t>(1, std::min<int64_t>((shell + 255) / 256, (int64_t)sm_count() * 16));
+            const int shell_grid = (int)std::max<int64_t>(1, std::min<int64_t>((shell + 255) / 256, (int64_t)plan_sms(p) * 16));
             // 32-bit indices where the grid leaves room for the grid-stride loop's last increment
             if (p->npoints < ((int64_t)1 << 31) - ((int64_t)1 << 24))
                 stencil_shell_compose_kernel<T, int><<<shell_grid, 256, 0, st>>>(src, dst, g, H, hz, taps, ntaps);

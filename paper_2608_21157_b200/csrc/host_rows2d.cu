@@ -125,8 +125,7 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
     const size_t smem = smem_for(stages);
     if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    const int dev = p->device;                       // current: the apply entry points have checked it
     {
         std::lock_guard<std::mutex> lock(g_config_mutex);
         if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->cache_device = dev; }
@@ -152,7 +151,7 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
         // reads chunk + 2R rows in batches of YB, so chunk + 2R is made a whole number of
         // batches; small grids end up with one batch per warp and as many warps as rows allow.
         const int R = p->radius;
-        const int slots = 2 * sm_count() * cfg->NW;
+        const int slots = 2 * plan_sms(p) * cfg->NW;
         const int nch_max = std::max(1, slots / g.strips);
         const int chunk_min = (span + nch_max - 1) / nch_max;
         int nbatch = std::max(1, (chunk_min + 2 * R + cfg->YB - 1) / cfg->YB);
@@ -187,8 +186,8 @@ int launch_rows2d_fused(stencil_plan_s* p, const float* src, float* dst, int nle
     while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
     const size_t smem = smem_for(stages);
     if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-    int dev = -1, occ = 1;
-    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    const int dev = p->device;                       // current: the apply entry points have checked it
+    int occ = 1;
     {
         std::lock_guard<std::mutex> lock(g_config_mutex);
         if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->occ_smem = 0; cfg->cache_device = dev; }
@@ -224,7 +223,7 @@ int launch_rows2d_fused(stencil_plan_s* p, const float* src, float* dst, int nle
         // resident warp slots once, never more (10240^2: 248-row chunks 2082 G updates/s, 504-row
         // chunks, half a wave, 1479; 120-row chunks 1843).
         const int H = nlev * p->radius;
-        const int slots = occ * sm_count() * cfg->NW;
+        const int slots = occ * plan_sms(p) * cfg->NW;
         const int nch_max = std::max(1, slots / g.strips);
         const int chunk_min = (p->ny + nch_max - 1) / nch_max;
         int nbatch = std::max(1, (chunk_min + 2 * H + cfg->YB - 1) / cfg->YB);

@@ -184,7 +184,7 @@ int choose_chunk(const stencil_plan_s* p, const StreamConfig* cfg, int stages, d
     const int nz = span > 0 ? span : p->nz;      // planes this launch covers
     const int tiles = ((p->nx + kStreamTX - 1) / kStreamTX) * ((p->ny + cfg->tile_y - 1) / cfg->tile_y);
     const int occ = std::max(1, stream_occupancy(cfg, stages));
-    const int slots = occ * sm_count();
+    const int slots = occ * plan_sms(p);
     if (!issue_bound(p)) {
         // measured on 512^3: 32-plane chunks (several thousand short CTAs) beat every longer chunk
         int chunk = nz >= 64 ? 32 : nz;
@@ -235,8 +235,7 @@ int launch_stream_wrap(stencil_plan_s* p, const StreamConfig* cfg, int stages, c
     }
     const size_t smem = (size_t)stages * (cfg->plane_bytes + cfg->stage_bytes) + 128 + 2 * kMaxStages * sizeof(uint64_t);
     if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return STENCIL_ERR_CUDA; }
+    const int dev = p->device;                       // current: the apply entry points have checked it
     {
         std::lock_guard<std::mutex> lock(g_config_mutex);
         if (dev != cfg->cache_device) {
@@ -288,7 +287,7 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
         // two rows per thread (GPoints/s, four rows vs two: 512^3 797 vs 667; 300^3 440 vs 511; 128^3 91 vs
         // 140; 64 x 1024^2 697 vs 716).
         const int64_t big_tiles = (int64_t)((p->nx + kStreamTX - 1) / kStreamTX) * ((p->ny + 31) / 32);
-        const bool plentiful = big_tiles * (span / 64) >= 2 * (int64_t)sm_count();
+        const bool plentiful = big_tiles * (span / 64) >= 2 * (int64_t)plan_sms(p);
         if (const StreamConfig* c = find_stream_cfg(3, false, 0, plentiful ? 4 : 2)) p->stream_cfg = c;
     }
     if (!p->stream_cfg_fixed && !p->stream_cfg_tuned) {
