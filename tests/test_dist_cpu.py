@@ -149,3 +149,45 @@ def test_sharded_sweep_equals_the_single_grid_sweep(world, dims, R, steps, halo_
         got[z0:z1] = block
         assert sum(calls) == steps and len(calls) == -(-steps // halo_steps) and max(calls) <= halo_steps
     assert np.array_equal(got, want)
+
+
+# ------------------------------------------------------ the benchmark's sharded arm --
+def _sharded_bench_worker(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        total = 0.0
+        for my_ms in ([4.0, 6.0] if rank == 0 else [5.0, 5.5]):     # two timed applies: the slower rank differs
+            dist.barrier()
+            total += bench.max_over_ranks(my_ms, dist, torch.device("cpu"))
+        out[rank] = (total, bench.sharded_job_summary((512, 512, 512), 1, 16, 2, 2, total, world, 4))
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.timeout(120)
+def test_sharded_arm_counts_the_grid_once_over_the_slowest_rank():
+    """`bench.py --sharded`: all ranks share ONE grid, so the job's value is the grid's
+    point-updates over the sum of the slowest rank's times, not world x that (the replicas rule)."""
+    world = 2
+    port = _free_port()
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_sharded_bench_worker, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    assert res[0] == res[1]
+    total, s = res[0]
+    assert total == 5.0 + 6.0
+    assert s["value"] == pytest.approx(512 ** 3 * 16 * 2 / 11e-3 / 1e9)
+    # two steps between exchanges: 8 rounds, each 2 planes of 512 x 512 floats to either neighbour
+    assert s["messages_per_rank_per_apply"] == 2 * 8
+    assert s["exchange_bytes_per_rank_per_apply"] == 2 * 8 * 2 * 512 * 512 * 4
+    assert s["exchange_bytes_per_rank_per_time_step"] == pytest.approx(2 * 512 * 512 * 4)
+
+
+def test_sharded_arm_on_one_rank_sends_nothing():
+    s = bench.sharded_job_summary((64, 32, 128), 2, 5, 2, 3, 10.0, 1, 4)
+    assert s["exchange_bytes_per_rank_per_apply"] == 0 and s["messages_per_rank_per_apply"] == 0
+    assert s["value"] == pytest.approx(64 * 32 * 128 * 5 * 3 / 10e-3 / 1e9)
