@@ -116,12 +116,13 @@ __device__ __forceinline__ float lds_if(bool take, const float* p, float keep) {
 // Fills v[0 .. 4+2R) with the R values left of the lane's float4, the float4
 // itself, and the R values right of it, for one smem row.  `rowp` points at the
 // lane's float4 inside the row; `rowbase` at the row's first float (x = -4; the
-// R <= 2 path, the only one that uses it, always has a 4-float halo).
-template <int R>
+// R <= 2 path, the only one that uses it, always has a 4-float halo).  FROM_SMEM
+// makes radius 1 and 2 read their neighbours from the row as well, like the wider radii.
+template <int R, bool FROM_SMEM = false>
 __device__ __forceinline__ void gather_row(const float* rowp, const float* rowbase, int lane,
                                            const float4& ctr, float (&v)[4 + 2 * R]) {
     v[R + 0] = ctr.x; v[R + 1] = ctr.y; v[R + 2] = ctr.z; v[R + 3] = ctr.w;
-    if constexpr (R <= 2) {
+    if constexpr (R <= 2 && !FROM_SMEM) {
         // neighbours' registers through shuffles; the row's two end lanes read the smem halo
         const float c4[4] = {ctr.x, ctr.y, ctr.z, ctr.w};
 #pragma unroll
@@ -461,6 +462,11 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
         // (M moves against (2R+1)^3 FMAs).
         constexpr int M = 2 * R + 1;
         constexpr int UNR = R >= 2 ? 1 : M;              // copies of the plane body
+        // The 125-point box takes a row's x neighbours as two more 128-bit loads from the plane instead
+        // of shuffles plus halo words (fewer instructions and registers: 512^3 218 against 201 GPoints/s);
+        // the 27-point box keeps the shuffles (769 against 752 in a short run; in a seconds-long run
+        // under the power cap the loads are ahead, 676 against 654).
+        constexpr bool kBoxRowsFromSmem = R >= 2;
         float4 T[K][M];
 #pragma unroll
         for (int k = 0; k < K; ++k)
@@ -522,7 +528,7 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
                         gather_row_split<R>(pl, o_row + HX + 4 * lane, edge_l ? o_xs : o_row,
                                             edge_r ? o_xs + S::XS_BYTES / 4 : o_row + HX + kStreamTX, lane, ctr, v[kk]);
                     } else {
-                        gather_row<R>(colp + kk * PX, pl + (row0 + kk) * PX, lane, ctr, v[kk]);
+                        gather_row<R, kBoxRowsFromSmem>(colp + kk * PX, pl + (row0 + kk) * PX, lane, ctr, v[kk]);
                     }
                 }
                 __syncwarp();
