@@ -780,7 +780,7 @@ def main():
     ap.add_argument("--stages", type=int, default=None)
     ap.add_argument("--fuse-steps", dest="fuse_steps", type=int, default=None)
     ap.add_argument("--streaming-store", dest="streaming_store", type=int, default=None)
-    ap.add_argument("--also", default="cfg1,cfg3,cfg4,cfg5,cfg5L,cfg5L_periodic,paper2d,paper2d_f64,heat2d", help="other workloads summarised in all_configs")
+    ap.add_argument("--also", default="cfg1,cfg3,cfg4,cfg5,cfg5L,cfg5L_periodic,cfg5L_f64,box27_iterated,paper2d,paper2d_f64,heat2d", help="other workloads summarised in all_configs")
     ap.add_argument("--also-steps", dest="also_steps", type=int, default=20)
     ap.add_argument("--also-cpu-seconds", dest="also_cpu_seconds", type=float, default=2.0,
                     help="oracle baseline beside every entry of all_configs (0 = off)")

@@ -94,7 +94,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->device = -1; p->sms = 0;
     p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0; p->src_padded = false; p->fused_wrap = false; p->stream_wrap = false; p->periodic_route = 0;
     for (int l = 0; l <= kMaxFuseLevels; ++l) p->d_ctaps[l] = nullptr;
-    p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr; p->fused2d64_cfg = nullptr;
+    p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr; p->fused2d64_cfg = nullptr; p->fused64_cfg = nullptr;
     p->host_in = nullptr; p->host_out = nullptr;
     p->copy_in = nullptr; p->copy_out = nullptr;
     p->variant = STENCIL_VARIANT_GENERIC;
@@ -338,8 +338,9 @@ int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps
         if (steps > 1) return apply_periodic(p, in, out, steps, st);
     }
     // A pass advances the field by T time steps (T = 1 without temporal blocking), as in stencil_apply.
-    const bool fuse = p->variant == STENCIL_VARIANT_STREAM && p->fused2d64_cfg != nullptr && steps > 1;
-    const int T = fuse ? p->fused2d64_cfg->T : 1;
+    const bool fuse3d = p->variant == STENCIL_VARIANT_STREAM && p->fused64_cfg != nullptr && steps > 1;
+    const bool fuse = fuse3d || (p->variant == STENCIL_VARIANT_STREAM && p->fused2d64_cfg != nullptr && steps > 1);
+    const int T = fuse3d ? p->fused64_cfg->T : fuse ? p->fused2d64_cfg->T : 1;
     const int passes = (steps + T - 1) / T;
     const double* src = in;
     int done = 0;
@@ -348,7 +349,9 @@ int stencil_apply_f64(stencil_plan_t p, const double* in, double* out, int steps
         double* dst = (remaining % 2 == 0) ? out : p->scratch64;
         const int nlev = std::min(T, steps - done);
         p->chained = p->chain_launches && k > 0;
-        rc = (fuse && nlev > 1) ? launch_rows2d_fused64(p, src, dst, nlev, st) : launch_sweep_f64(p, src, dst, st);
+        rc = !(fuse && nlev > 1) ? launch_sweep_f64(p, src, dst, st)
+             : fuse3d           ? launch_fused(p, src, dst, nlev, st)
+                                : launch_rows2d_fused64(p, src, dst, nlev, st);
         p->chained = false;
         if (rc != STENCIL_OK) return rc;
         done += nlev;
@@ -557,9 +560,20 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
         case STENCIL_KEY_TILE_X:
         case STENCIL_KEY_FUSE_STEPS: {
             if (p->f64) {
-                // FP64: only the 2D register cascade exists; 0 = use it, 1 = off, T = its depth
-                if (key == STENCIL_KEY_TILE_X) return value == 0 ? STENCIL_OK : STENCIL_ERR_UNSUPPORTED;
                 if (value < 0) return STENCIL_ERR_INVALID;
+                if (p->ndim == 3) {
+                    // FP64 3D stars of radius 1: region width 128 or 256, two or three steps per pass
+                    const int old_fuse = p->fuse_steps, old_tx = p->tile_x;
+                    if (key == STENCIL_KEY_TILE_X) p->tile_x = (int)value; else p->fuse_steps = (int)value;
+                    const FusedConfig* f3 =
+                        (p->variant == STENCIL_VARIANT_STREAM && p->stream64_cfg) ? pick_fused64(p) : nullptr;
+                    const bool wants = p->fuse_steps > 1 || (key == STENCIL_KEY_TILE_X && value != 0 && p->fuse_steps != 1);
+                    if (!f3 && wants) { p->fuse_steps = old_fuse; p->tile_x = old_tx; return STENCIL_ERR_UNSUPPORTED; }
+                    p->fused64_cfg = f3;
+                    return STENCIL_OK;
+                }
+                // FP64 2D: only the register cascade exists; 0 = use it, 1 = off, T = its depth
+                if (key == STENCIL_KEY_TILE_X) return value == 0 ? STENCIL_OK : STENCIL_ERR_UNSUPPORTED;
                 const int old = p->fuse_steps;
                 p->fuse_steps = (int)value;
                 const Rows2DFused64Config* f2 =
@@ -670,6 +684,7 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
                      : p->fused_cfg                           ? p->fused_cfg->T
                      : p->fused2d_cfg                         ? p->fused2d_cfg->T
                      : p->fused2d64_cfg                       ? p->fused2d64_cfg->T
+                     : p->fused64_cfg                         ? p->fused64_cfg->T
                                                               : 1;
             return STENCIL_OK;
         case STENCIL_KEY_LAUNCHES: *value = p->launches; return STENCIL_OK;

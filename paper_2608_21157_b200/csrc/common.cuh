@@ -36,6 +36,24 @@ __device__ __forceinline__ float4 fma4r(float w, const float4& v, const float4& 
 }
 __device__ __forceinline__ float4 mul4(float w, const float4& v) { return join4(mul2(w, lo2(v)), mul2(w, hi2(v))); }
 
+// The same operations on a double2 (two plain FP64 FMAs), so that kernels written for either
+// 16-byte vector share their arithmetic.
+__device__ __forceinline__ void fma4(double2& a, double w, const double2& v) {
+    a.x = fma(w, v.x, a.x); a.y = fma(w, v.y, a.y);
+}
+__device__ __forceinline__ double2 fma4r(double w, const double2& v, const double2& a) {
+    return make_double2(fma(w, v.x, a.x), fma(w, v.y, a.y));
+}
+__device__ __forceinline__ double2 mul4(double w, const double2& v) { return make_double2(w * v.x, w * v.y); }
+
+template <typename V> __device__ __forceinline__ V vzero();
+template <> __device__ __forceinline__ float4 vzero<float4>() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+template <> __device__ __forceinline__ double2 vzero<double2>() { return make_double2(0.0, 0.0); }
+__device__ __forceinline__ void vunpack(const float4& v, float (&a)[4]) { a[0] = v.x; a[1] = v.y; a[2] = v.z; a[3] = v.w; }
+__device__ __forceinline__ void vunpack(const double2& v, double (&a)[2]) { a[0] = v.x; a[1] = v.y; }
+template <typename V> __device__ __forceinline__ V vpack(const float (&a)[4]) { return make_float4(a[0], a[1], a[2], a[3]); }
+template <typename V> __device__ __forceinline__ V vpack(const double (&a)[2]) { return make_double2(a[0], a[1]); }
+
 // Grid extents as the kernels see them; 2D grids have nz == 1.
 struct Grid {
     int nz, ny, nx;

@@ -104,6 +104,7 @@ struct StreamConfig {
 struct FusedConfig {
     int radius, T, K, XW, NWY;
     bool box;
+    bool f64;                                // FP64 instantiation (two doubles per lane: 64 columns per warp)
     int txe, tye, threads, slot_bytes;
     int pw;                                  // width of the TMA boxes a plane is loaded as
     const void* kernel;
@@ -113,11 +114,12 @@ struct FusedConfig {
     mutable size_t occ_smem;                 // ... and the occupancy measured at this size
     mutable int occ;
     mutable int cache_device;
-    cudaError_t (*launch)(const stencil_plan_s*, const CUtensorMap&, float*, const FusedGeom&,
+    // `out` is a float* or double* as the configuration's element type says
+    cudaError_t (*launch)(const stencil_plan_s*, const CUtensorMap&, void* out, const FusedGeom&,
                           int grid, size_t smem, cudaStream_t);
-    cudaError_t (*launch_spec)(const stencil_plan_s*, const CUtensorMap&, float*, const FusedGeom&,
+    cudaError_t (*launch_spec)(const stencil_plan_s*, const CUtensorMap&, void* out, const FusedGeom&,
                                int grid, size_t smem, cudaStream_t);
-    cudaError_t (*launch_wrap)(const stencil_plan_s*, const CUtensorMap&, float*, const FusedGeom&,
+    cudaError_t (*launch_wrap)(const stencil_plan_s*, const CUtensorMap&, void* out, const FusedGeom&,
                                int grid, size_t smem, cudaStream_t);
 };
 
@@ -222,6 +224,7 @@ struct stencil_plan_s {
     const stencil_host::Rows2D64Config* rows2d64_cfg;
     const stencil_host::Rows2DFused64Config* fused2d64_cfg;   // non-null: iterated applies of a 2D FP64 grid run fused passes
     const stencil_host::Stream64Config* stream64_cfg;
+    const stencil_host::FusedConfig* fused64_cfg;      // non-null: iterated applies of a 3D FP64 grid run fused passes
     // device state (created lazily, on the device current at first apply)
     int device;
     int sms;                       // multiprocessors of that device
@@ -333,8 +336,9 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
 
 // ---- host_fused.cu ----------------------------------------------------------
 const FusedConfig* pick_fused(const stencil_plan_s* p);
-// one fused pass: dst = S^nlev(src), nlev <= the configuration's T
-int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cudaStream_t st);
+const FusedConfig* pick_fused64(const stencil_plan_s* p);
+// one fused pass: dst = S^nlev(src), nlev <= the configuration's T (grids of the plan's element type)
+int launch_fused(stencil_plan_s* p, const void* src, void* dst, int nlev, cudaStream_t st);
 
 // ---- host_rows2d.cu ---------------------------------------------------------
 const Rows2DConfig* find_rows2d_cfg(int radius, bool box);

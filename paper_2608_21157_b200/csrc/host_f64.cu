@@ -199,11 +199,13 @@ int resolve_variant_f64(stencil_plan_s* p, int want) {
     if (want == STENCIL_VARIANT_AUTO) want = (c2 || c3) ? STENCIL_VARIANT_STREAM : STENCIL_VARIANT_GENERIC;
     if (want == STENCIL_VARIANT_GENERIC) {
         p->variant = want; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr; p->fused2d64_cfg = nullptr;
+        p->fused64_cfg = nullptr;
         return STENCIL_OK;
     }
     if (want == STENCIL_VARIANT_STREAM && (c2 || c3)) {
         p->variant = want; p->rows2d64_cfg = c2; p->stream64_cfg = c3;
         p->fused2d64_cfg = c2 ? pick_fused2d64(p) : nullptr;
+        p->fused64_cfg = c3 ? pick_fused64(p) : nullptr;
         return STENCIL_OK;
     }
     return STENCIL_ERR_UNSUPPORTED;

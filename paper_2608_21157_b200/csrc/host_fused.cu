@@ -1,45 +1,60 @@
-// Host side of 3D temporal blocking (fp32): configurations, the default fusion rule, launches.
+// Host side of 3D temporal blocking (fp32 and FP64): configurations, the default fusion rule, launches.
 #include "host.h"
 #include "kernel_fused.cuh"
 
 namespace stencil_host {
 
-template <int R>
-void pack_star(const stencil_plan_s* p, StarWeights<R>& sw) {
+template <typename E>
+inline E dense_tap(const stencil_plan_s* p, int dz, int dy, int dx) {
+    const int R = p->radius, side = 2 * R + 1;
+    const size_t f = ((size_t)(dz + R) * side + (dy + R)) * side + (dx + R);
+    if constexpr (sizeof(E) == 8) return p->w64[f];
+    else return p->w[f];
+}
+
+template <typename E, int R>
+void pack_star(const stencil_plan_s* p, StarTaps<E, R>& sw) {
     std::memset(&sw, 0, sizeof(sw));
-    sw.c = dense_w(p, 0, 0, 0);
+    sw.c = dense_tap<E>(p, 0, 0, 0);
     for (int d = -R; d <= R; ++d) {
         if (d == 0) continue;
-        sw.x[d + R] = dense_w(p, 0, 0, d);
-        sw.y[d + R] = dense_w(p, 0, d, 0);
-        sw.z[d + R] = dense_w(p, d, 0, 0);
+        sw.x[d + R] = dense_tap<E>(p, 0, 0, d);
+        sw.y[d + R] = dense_tap<E>(p, 0, d, 0);
+        sw.z[d + R] = dense_tap<E>(p, d, 0, 0);
     }
 }
 
-template <int R, int T, int K, int XW, int NWY, int MODE>
-cudaError_t launch_fused_t(const stencil_plan_s* p, const CUtensorMap& map, float* out, const FusedGeom& g,
+template <typename E, int R, int T, int K, int XW, int NWY, int MODE>
+cudaError_t launch_fused_t(const stencil_plan_s* p, const CUtensorMap& map, void* out, const FusedGeom& g,
                            int grid, size_t smem, cudaStream_t st) {
-    StarWeights<R> sw;
-    pack_star<R>(p, sw);
-    return launch_kernel(&stencil_fused_kernel<R, T, K, XW, NWY, MODE>, grid, FusedShape<R, K, XW, NWY>::THREADS,
-                         smem, st, p->chained, map, out, g, sw, p->d_status);
+    StarTaps<E, R> sw;
+    pack_star<E, R>(p, sw);
+    return launch_kernel(&stencil_fused_kernel<E, R, T, K, XW, NWY, MODE>, grid,
+                         FusedShape<R, K, XW, NWY, E>::THREADS, smem, st, p->chained, map, static_cast<E*>(out), g,
+                         sw, p->d_status);
+}
+
+template <typename E, int R, int T, int K, int XW, int NWY>
+FusedConfig make_fused_e() {
+    using S = FusedShape<R, K, XW, NWY, E>;
+    FusedConfig c;
+    c.radius = R; c.T = T; c.K = K; c.XW = XW; c.NWY = NWY; c.box = false; c.f64 = sizeof(E) == 8;
+    c.txe = S::TXE; c.tye = S::TYE; c.threads = S::THREADS; c.slot_bytes = S::SLOT_BYTES; c.pw = S::PW;
+    c.kernel = reinterpret_cast<const void*>(&stencil_fused_kernel<E, R, T, K, XW, NWY, 0>);
+    c.kernel_spec = reinterpret_cast<const void*>(&stencil_fused_kernel<E, R, T, K, XW, NWY, 1>);
+    c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
+    c.launch = &launch_fused_t<E, R, T, K, XW, NWY, 0>;
+    c.launch_spec = &launch_fused_t<E, R, T, K, XW, NWY, 1>;
+    c.kernel_wrap = nullptr; c.launch_wrap = nullptr;
+    if constexpr (sizeof(E) == 4) {            // the pass of a periodic grid that wraps x and z itself: fp32 only
+        c.kernel_wrap = reinterpret_cast<const void*>(&stencil_fused_kernel<E, R, T, K, XW, NWY, 2>);
+        c.launch_wrap = &launch_fused_t<E, R, T, K, XW, NWY, 2>;
+    }
+    return c;
 }
 
 template <int R, int T, int K, int XW, int NWY>
-FusedConfig make_fused() {
-    using S = FusedShape<R, K, XW, NWY>;
-    FusedConfig c;
-    c.radius = R; c.T = T; c.K = K; c.XW = XW; c.NWY = NWY; c.box = false;
-    c.txe = S::TXE; c.tye = S::TYE; c.threads = S::THREADS; c.slot_bytes = S::SLOT_BYTES; c.pw = S::PW;
-    c.kernel = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, 0>);
-    c.kernel_spec = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, 1>);
-    c.kernel_wrap = reinterpret_cast<const void*>(&stencil_fused_kernel<R, T, K, XW, NWY, 2>);
-    c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
-    c.launch = &launch_fused_t<R, T, K, XW, NWY, 0>;
-    c.launch_spec = &launch_fused_t<R, T, K, XW, NWY, 1>;
-    c.launch_wrap = &launch_fused_t<R, T, K, XW, NWY, 2>;
-    return c;
-}
+FusedConfig make_fused() { return make_fused_e<float, R, T, K, XW, NWY>(); }
 
 // First match of (radius, T, region width) wins; T == 0 / width == 0 match anything.
 const std::vector<FusedConfig>& fused_configs() {
@@ -56,6 +71,44 @@ const FusedConfig* find_fused_cfg(int radius, int T, int txe, int tye = 0) {
     for (const FusedConfig& c : fused_configs())
         if (c.radius == radius && (T == 0 || c.T == T) && (txe == 0 || c.txe == txe) && (tye == 0 || c.tye == tye))
             return &c;
+    return nullptr;
+}
+
+// FP64: a lane holds two doubles, so a warp spans 64 columns and the regions are 128 (two CTAs per SM) or 256
+// columns wide (XW = 4: 512 threads, one CTA per SM); 512 columns would take 1024 threads of 64 registers, which
+// the two accumulators per row and level do not fit.
+const std::vector<FusedConfig>& fused64_configs() {
+    static const std::vector<FusedConfig> v = {
+        make_fused_e<double, 1, 2, 4, 4, 4>(), make_fused_e<double, 1, 2, 4, 2, 4>(),
+        make_fused_e<double, 1, 2, 2, 2, 8>(), make_fused_e<double, 1, 3, 2, 2, 8>(),
+    };
+    return v;
+}
+
+// Temporal blocking of an FP64 3D grid: the 7-point-like stars (radius 1), zero boundary, even rows.  Default:
+// two steps per pass where the rows fill 80 % of the lanes of their regions: one 128- or 256-wide region per row,
+// or, on wider rows, several 128-wide regions with 4 halo columns per side (two CTAs per SM, which the
+// 256-wide regions do not allow).  Measured, G updates/s, fused against one launch per step: 256^3 461 / 381,
+// 512 x 512 x 256 516 / 421, 512 x 512 x 128 620 / 408, 512^3 484 / 422 (five 128-wide regions per row; three
+// 256-wide ones: 275); three steps per pass on 128-wide regions lose to two (445 against 620).
+const FusedConfig* pick_fused64(const stencil_plan_s* p) {
+    if (!p->f64 || p->ndim != 3 || p->shape != STENCIL_STAR || p->boundary != STENCIL_ZERO) return nullptr;
+    if (p->nx % 2 != 0 || p->fuse_steps == 1) return nullptr;
+    const bool forced = p->fuse_steps > 2 || p->tile_x != 0 || p->fused_tile_y != 0;
+    const int width = p->nx <= 128 ? 128 : p->nx <= 256 ? 256 : 128;
+    const int64_t regions = p->nx <= width ? 1 : (p->nx + (width - 8) - 1) / (width - 8);
+    const double lanes_used = (double)p->nx / (double)(regions * width);
+    for (const FusedConfig& c : fused64_configs()) {
+        if (c.radius != p->radius) continue;
+        if (forced) {
+            if ((p->fuse_steps <= 1 || c.T == p->fuse_steps) && (p->tile_x == 0 || c.txe == p->tile_x) &&
+                (p->fused_tile_y == 0 || c.tye == p->fused_tile_y))
+                return &c;
+            continue;
+        }
+        // (a caller that asks for two steps per pass gets them on the default width whatever the rows fill)
+        if (c.T == 2 && c.txe == width && (lanes_used >= 0.8 || p->fuse_steps == 2)) return &c;
+    }
     return nullptr;
 }
 
@@ -126,10 +179,11 @@ const FusedConfig* pick_fused_region(const stencil_plan_s* p) {
     return find_fused_cfg(p->radius, p->fuse_steps, txe, p->fused_tile_y);
 }
 
-int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cudaStream_t st) {
-    const FusedConfig* cfg = p->fused_cfg;
+int launch_fused(stencil_plan_s* p, const void* src, void* dst, int nlev, cudaStream_t st) {
+    const FusedConfig* cfg = p->f64 ? p->fused64_cfg : p->fused_cfg;
     const CUtensorMap* map = nullptr;
-    int rc = get_tensor_map(p, cfg, cfg->pw, cfg->tye, src, &map);   // a box is at most 256 wide
+    int rc = p->f64 ? get_tensor_map_f64(p, cfg, cfg->pw, cfg->tye, static_cast<const double*>(src), &map)
+                    : get_tensor_map(p, cfg, cfg->pw, cfg->tye, static_cast<const float*>(src), &map);   // a box is at most 256 wide
     if (rc != STENCIL_OK) return rc;
     const int R = p->radius, T = cfg->T;
     FusedGeom g;
@@ -166,8 +220,9 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
                     cudaSuccess ||
                 cudaFuncSetAttribute(cfg->kernel_spec, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
                     cudaSuccess ||
-                cudaFuncSetAttribute(cfg->kernel_wrap, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                    cudaSuccess) {
+                (cfg->kernel_wrap &&
+                 cudaFuncSetAttribute(cfg->kernel_wrap, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+                     cudaSuccess)) {
                 cudaGetLastError();
                 return STENCIL_ERR_CUDA;
             }
@@ -214,7 +269,7 @@ int launch_fused(stencil_plan_s* p, const float* src, float* dst, int nlev, cuda
     // the caller beforehand that it will)
     const bool spec = nlev == T && p->nx == cfg->txe;
     auto launch = !spec ? cfg->launch : (p->fused_wrap ? cfg->launch_wrap : cfg->launch_spec);
-    if (p->fused_wrap && !spec) return STENCIL_ERR_UNSUPPORTED;
+    if (p->fused_wrap && (!spec || !cfg->launch_wrap)) return STENCIL_ERR_UNSUPPORTED;
     if (launch(p, *map, dst, g, (int)grid64, smem, st) != cudaSuccess) return STENCIL_ERR_CUDA;
     p->launches++;
     return STENCIL_OK;

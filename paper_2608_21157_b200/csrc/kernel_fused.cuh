@@ -1,5 +1,6 @@
 // FUSED kernel: temporal blocking for the iterated 3D star sweep with a zero
-// boundary.  One pass over the grid advances it by up to T time steps while
+// boundary, on fp32 or FP64 grids (element type E; a lane holds one 16-byte
+// vector of a row, four floats or two doubles).  One pass over the grid advances it by up to T time steps while
 // reading the input once and writing the result once.
 //
 // A CTA owns a TXE x TYE region of the x-y plane (its output tile plus a halo
@@ -7,7 +8,7 @@
 // arrive through a TMA ring exactly as in the single-step kernel.  Time level
 // l (1..T) is computed from level l-1 one plane at a time:
 //
-//   - each thread owns the same K rows x one float4 column at every level, so
+//   - each thread owns the same K rows x one 16-byte column at every level, so
 //     the centre values of level l-1 are already in its registers;
 //   - the rows above/below its block and the cells left/right of a warp come
 //     from the level's plane in shared memory (double-buffered; one CTA
@@ -17,8 +18,8 @@
 //
 // Level l lags level l-1 by R planes.  Cells outside the grid are forced back
 // to zero at every level (the zero boundary holds at every time step), and
-// every intermediate level is an fp32 value, so the result equals T separate
-// sweeps up to summation order.  The last level goes straight to global
+// every intermediate level is a value of the grid's own type, so the result equals
+// T separate sweeps up to summation order.  The last level goes straight to global
 // memory; only the tile interior is stored.
 #pragma once
 #include "common.cuh"
@@ -28,9 +29,22 @@
 namespace stencil {
 
 
-template <int R, int K, int XW, int NWY>
+// The 16-byte vector of a row that one lane holds, and the taps of a star in the grid's type.
+template <typename E> struct FusedVec;
+template <> struct FusedVec<float>  { using V = float4;  static constexpr int N = 4; };
+template <> struct FusedVec<double> { using V = double2; static constexpr int N = 2; };
+
+template <typename E, int R>
+struct StarTaps {               // index d + R along each axis, entry [R] unused
+    E c;
+    E x[2 * R + 1], y[2 * R + 1], z[2 * R + 1];
+};
+
+template <int R, int K, int XW, int NWY, typename E = float>
 struct FusedShape {
-    static constexpr int TXE = 128 * XW;
+    static constexpr int NV = FusedVec<E>::N;                   // points of a row per lane
+    static constexpr int WX = 32 * NV;                          // columns one warp spans
+    static constexpr int TXE = WX * XW;
     static constexpr int TYE = NWY * K;
     static constexpr int THREADS = XW * NWY * 32;
     // A TMA box is at most 256 elements wide, so a wider plane lies in shared memory as NP parts
@@ -40,8 +54,8 @@ struct FusedShape {
     static constexpr int NP = TXE / PW;
     static constexpr int PART_FLOATS = (TYE + 2 * R) * PW;      // R pad rows above and below
     static constexpr int SLOT_FLOATS = NP * PART_FLOATS;
-    static constexpr int SLOT_BYTES = SLOT_FLOATS * 4;          // multiple of 512
-    static constexpr int BOX_BYTES = TYE * TXE * 4;             // bytes of all parts of one plane
+    static constexpr int SLOT_BYTES = SLOT_FLOATS * (int)sizeof(E);   // multiple of 512
+    static constexpr int BOX_BYTES = TYE * TXE * (int)sizeof(E);      // bytes of all parts of one plane
     static size_t smem_bytes(int stages, int T) {
         return (size_t)(stages + 2 * (T - 1)) * SLOT_BYTES + 128 + kMaxStages * 8;
     }
@@ -52,46 +66,48 @@ __device__ __forceinline__ void consumer_barrier(int nthreads) {
 }
 
 // MODE 1 (SPEC): the launch advances exactly T levels and one region spans a whole row of exactly
-// 128*XW points.  The level count, the row pitch and the x bounds are then compile-time
+// 128*XW points (64*XW in FP64).  The level count, the row pitch and the x bounds are then compile-time
 // constants (the common case of the iterated apply on a 256-wide grid).
 // MODE 2 (SPEC and WRAP): the same, on a grid that is periodic along x and z (the pass of a
 // periodic grid; its y faces are put right afterwards).  z wraps in the plane coordinate of the
 // TMA loads, since every plane is a load of its own, and no plane counts as outside the grid;
 // x wraps where the first and last warp of a row fetch the cells beyond the row's ends, at every
 // level, from the other end of the same row of the level's plane in shared memory.
-template <int R, int T, int K, int XW, int NWY, int MODE = 0>
+template <typename E, int R, int T, int K, int XW, int NWY, int MODE = 0>
 __global__ void __launch_bounds__(XW * NWY * 32, (XW * NWY * 32 <= 256 ? 2 : 1))
-stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restrict__ out,
-                     const FusedGeom g, const __grid_constant__ StarWeights<R> sw,
+stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, E* __restrict__ out,
+                     const FusedGeom g, const __grid_constant__ StarTaps<E, R> sw,
                      int* __restrict__ status) {
     constexpr bool SPEC = MODE >= 1, WRAP = MODE == 2;
-    using S = FusedShape<R, K, XW, NWY>;
+    using S = FusedShape<R, K, XW, NWY, E>;
+    using V = typename FusedVec<E>::V;
+    constexpr int NV = S::NV;
     constexpr int TXE = S::TXE;
     constexpr int PW = S::PW;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     // indexing the shared array keeps every derived pointer in the shared address space
     unsigned char* base = smem_raw + ((128u - (smem_addr(smem_raw) & 127u)) & 127u);
     const int nstage = g.stages;
-    float* ring = reinterpret_cast<float*>(base);                                   // nstage slots
-    float* lvl = ring + (size_t)nstage * S::SLOT_FLOATS;                            // (T-1) x 2 slots
+    E* ring = reinterpret_cast<E*>(base);                                           // nstage slots
+    E* lvl = ring + (size_t)nstage * S::SLOT_FLOATS;                                // (T-1) x 2 slots
     uint64_t* bars = reinterpret_cast<uint64_t*>(lvl + (size_t)2 * (T - 1) * S::SLOT_FLOATS);
     const uint32_t full0 = smem_addr(bars);
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int wx = warp % XW, wy = warp / XW;
-    const int col = 4 * (wx * 32 + lane);          // x offset inside the region
+    const int col = NV * (wx * 32 + lane);         // x offset inside the region
     const int row0 = wy * K;                       // first region row of this thread
 
     // zero the pad rows of every slot once; TMA and the level stores never touch them
     {
         const int nslots = nstage + 2 * (T - 1);
         for (int s = 0; s < nslots; ++s) {
-            float* slot = ring + (size_t)s * S::SLOT_FLOATS;
+            E* slot = ring + (size_t)s * S::SLOT_FLOATS;
             for (int e = tid; e < R * TXE; e += S::THREADS) {
-                float* part = slot + (e / (R * PW)) * S::PART_FLOATS;
-                part[e % (R * PW)] = 0.0f;
-                part[(S::TYE + R) * PW + e % (R * PW)] = 0.0f;
+                E* part = slot + (e / (R * PW)) * S::PART_FLOATS;
+                part[e % (R * PW)] = E(0);
+                part[(S::TYE + R) * PW + e % (R * PW)] = E(0);
             }
         }
     }
@@ -134,11 +150,12 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
     const bool warp_all_in = __all_sync(0xffffffffu, in_mask == kAllRows);
     const bool warp_all_store = __all_sync(0xffffffffu, store_mask == kAllRows);
     const size_t plane_stride = (size_t)g.ny * nx;
-    float* const out_col = out + (size_t)(y0e + row0) * nx + xg;       // this thread's column of rows
+    E* const out_col = out + (size_t)(y0e + row0) * nx + xg;           // this thread's column of rows
     const int toff = (col / PW) * S::PART_FLOATS + row0 * PW + col % PW;   // its offset inside a plane
-    // the cells just left and right of the warp's 128 columns (they may lie in another part)
-    const int hl_off = wx > 0 ? ((wx * 128 - 1) / PW) * S::PART_FLOATS + (wx * 128 - R) - ((wx * 128 - 1) / PW) * PW : 0;
-    const int hr_off = wx < XW - 1 ? (((wx + 1) * 128) / PW) * S::PART_FLOATS + (wx + 1) * 128 - (((wx + 1) * 128) / PW) * PW : 0;
+    // the cells just left and right of the warp's columns (they may lie in another part)
+    constexpr int WX = S::WX;
+    const int hl_off = wx > 0 ? ((wx * WX - 1) / PW) * S::PART_FLOATS + (wx * WX - R) - ((wx * WX - 1) / PW) * PW : 0;
+    const int hr_off = wx < XW - 1 ? (((wx + 1) * WX) / PW) * S::PART_FLOATS + (wx + 1) * WX - (((wx + 1) * WX) / PW) * PW : 0;
 
     // the plane a load fetches: wrapped into the grid under WRAP (nz >= 2*T*R, so one step is enough)
     auto plane_coord = [&](int zc) { return !WRAP ? zc : (zc < 0 ? zc + g.nz : (zc >= g.nz ? zc - g.nz : zc)); };
@@ -163,13 +180,13 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
 
     // A[l][k][j]: level l+1's partial sums, oldest incomplete output plane first (see the
     // single-step kernel: arriving planes update them in place, nothing is copied)
-    float4 A[T][K][2 * R];
+    V A[T][K][2 * R];
 #pragma unroll
     for (int l = 0; l < T; ++l)
 #pragma unroll
         for (int k = 0; k < K; ++k)
 #pragma unroll
-            for (int j = 0; j < 2 * R; ++j) A[l][k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int j = 0; j < 2 * R; ++j) A[l][k][j] = vzero<V>();
 
     bool dead = false;
     int s = 0;                                     // input ring slot and its phase parity
@@ -184,31 +201,33 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                 dead = true;
                 atomicExch(status, kStatusTimeout);
             }
-            const float* src = ring + (size_t)s * S::SLOT_FLOATS + R * PW;      // region row 0 (of part 0)
-            float4 cin[K + 2 * R];
+            const E* src = ring + (size_t)s * S::SLOT_FLOATS + R * PW;          // region row 0 (of part 0)
+            V cin[K + 2 * R];
 #pragma unroll
             for (int kk = 0; kk < K + 2 * R; ++kk)
-                cin[kk] = *reinterpret_cast<const float4*>(src + toff + (kk - R) * PW);
+                cin[kk] = *reinterpret_cast<const V*>(src + toff + (kk - R) * PW);
 
 #pragma unroll
             for (int l = 1; l <= T; ++l) {
                 if (l <= nlev) {
                     const int zl = pstart + i - l * R;          // plane this level completes now
-                    float4 e[K];
+                    V e[K];
                     {
 #pragma unroll
                         for (int k = 0; k < K; ++k) {
-                            const float4 ctr = cin[k + R];
-                            float v[4 + 2 * R];
-                            v[R + 0] = ctr.x; v[R + 1] = ctr.y; v[R + 2] = ctr.z; v[R + 3] = ctr.w;
+                            const V ctr = cin[k + R];
+                            E v[NV + 2 * R];
+                            E c4[NV];
+                            vunpack(ctr, c4);
+#pragma unroll
+                            for (int m = 0; m < NV; ++m) v[R + m] = c4[m];
                             {
-                                const float c4[4] = {ctr.x, ctr.y, ctr.z, ctr.w};
-                                const float* rowb = src + (row0 + k) * PW;    // first cell of the region row (part 0)
+                                const E* rowb = src + (row0 + k) * PW;        // first cell of the region row (part 0)
 #pragma unroll
                                 for (int t = 0; t < R; ++t) {
                                     // cells across the warp boundary: one broadcast read per side from the
                                     // level's plane (wx is warp-uniform); zero at the region's edge
-                                    float xl = 0.0f, xr = 0.0f;
+                                    E xl = E(0), xr = E(0);
                                     if (XW > 1) {
                                         if (wx > 0) xl = rowb[hl_off + t];
                                         if (wx < XW - 1) xr = rowb[hr_off + t];
@@ -217,29 +236,30 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                                         if (wx == 0) xl = rowb[wrap_l_off + t];
                                         if (wx == XW - 1) xr = rowb[wrap_r_off + t];
                                     }
-                                    const float lft = __shfl_up_sync(0xffffffffu, c4[4 - R + t], 1);
-                                    const float rgt = __shfl_down_sync(0xffffffffu, c4[t], 1);
+                                    const E lft = __shfl_up_sync(0xffffffffu, c4[NV - R + t], 1);
+                                    const E rgt = __shfl_down_sync(0xffffffffu, c4[t], 1);
                                     v[t] = lane == 0 ? xl : lft;
-                                    v[R + 4 + t] = lane == 31 ? xr : rgt;
+                                    v[R + NV + t] = lane == 31 ? xr : rgt;
                                 }
                             }
-                            float4 (&Al)[2 * R] = A[l - 1][k];
+                            V (&Al)[2 * R] = A[l - 1][k];
                             // the output whose centre plane this is continues from Al[R]; the centre and
                             // y taps work on aligned pairs (packed FMAs), the x taps on single lanes
-                            float4 a4 = fma4r(sw.c, ctr, Al[R]);
+                            V a4 = fma4r(sw.c, ctr, Al[R]);
 #pragma unroll
                             for (int d = 1; d <= R; ++d) {
                                 fma4(a4, sw.y[R - d], cin[k + R - d]);
                                 fma4(a4, sw.y[R + d], cin[k + R + d]);
                             }
-                            float acc[4] = {a4.x, a4.y, a4.z, a4.w};
+                            E acc[NV];
+                            vunpack(a4, acc);
 #pragma unroll
-                            for (int m = 0; m < 4; ++m) {
-                                float a = acc[m];
+                            for (int m = 0; m < NV; ++m) {
+                                E a = acc[m];
 #pragma unroll
                                 for (int d = 1; d <= R; ++d) {
-                                    a = fmaf(sw.x[R - d], v[R + m - d], a);
-                                    a = fmaf(sw.x[R + d], v[R + m + d], a);
+                                    a = fma_t(sw.x[R - d], v[R + m - d], a);
+                                    a = fma_t(sw.x[R + d], v[R + m + d], a);
                                 }
                                 acc[m] = a;
                             }
@@ -251,7 +271,7 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                                 Al[j] = fma4r(sw.z[2 * R - 1 - j], ctr, Al[j + 1]);
                             }
                             Al[2 * R - 1] = mul4(sw.z[0], ctr);
-                            Al[R - 1] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                            Al[R - 1] = vpack<V>(acc);
                         }
                         // the zero boundary holds at every time level: cells outside the grid go
                         // back to zero (nothing to do for regions and planes inside the grid)
@@ -259,29 +279,29 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                             const bool z_in = WRAP || FAST || (zl >= 0 && zl < g.nz);
 #pragma unroll
                             for (int k = 0; k < K; ++k)
-                                if (!(z_in && ((in_mask >> k) & 1u))) e[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                if (!(z_in && ((in_mask >> k) & 1u))) e[k] = vzero<V>();
                         }
 
                         if (l == nlev) {
                             // last level of this pass: interior of the tile goes to global memory
                             if (!dead && (FAST || (zl >= z0 && zl < z1))) {
-                                float* op = out_col + (size_t)zl * plane_stride;
+                                E* op = out_col + (size_t)zl * plane_stride;
                                 if (warp_all_store) {
 #pragma unroll
                                     for (int k = 0; k < K; ++k)
-                                        *reinterpret_cast<float4*>(op + (size_t)k * nx) = e[k];
+                                        *reinterpret_cast<V*>(op + (size_t)k * nx) = e[k];
                                 } else {
 #pragma unroll
                                     for (int k = 0; k < K; ++k)
                                         if ((store_mask >> k) & 1u)
-                                            *reinterpret_cast<float4*>(op + (size_t)k * nx) = e[k];
+                                            *reinterpret_cast<V*>(op + (size_t)k * nx) = e[k];
                                 }
                             }
                         } else {
-                            float* buf = lvl + (size_t)(2 * (l - 1) + par) * S::SLOT_FLOATS + R * PW;
+                            E* buf = lvl + (size_t)(2 * (l - 1) + par) * S::SLOT_FLOATS + R * PW;
 #pragma unroll
                             for (int k = 0; k < K; ++k)
-                                *reinterpret_cast<float4*>(buf + toff + k * PW) = e[k];
+                                *reinterpret_cast<V*>(buf + toff + k * PW) = e[k];
                         }
                     }
                     if (l < nlev || l == 1) {
@@ -299,14 +319,14 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __restr
                         }
                     }
                     if (l < nlev) {
-                        const float* buf = lvl + (size_t)(2 * (l - 1) + par) * S::SLOT_FLOATS + R * PW;
+                        const E* buf = lvl + (size_t)(2 * (l - 1) + par) * S::SLOT_FLOATS + R * PW;
                         src = buf;
 #pragma unroll
                         for (int k = 0; k < K; ++k) cin[k + R] = e[k];
 #pragma unroll
                         for (int kk = 0; kk < R; ++kk) {
-                            cin[kk] = *reinterpret_cast<const float4*>(buf + toff + (kk - R) * PW);
-                            cin[K + R + kk] = *reinterpret_cast<const float4*>(buf + toff + (K + kk) * PW);
+                            cin[kk] = *reinterpret_cast<const V*>(buf + toff + (kk - R) * PW);
+                            cin[K + R + kk] = *reinterpret_cast<const V*>(buf + toff + (K + kk) * PW);
                         }
                     }
                 }

@@ -291,6 +291,19 @@ def _build_table() -> Dict[str, Workload]:
         _resizable(lambda d: uniform_field(d, -1.0, 1.0, 4, np.float64), (512, 512, 512)),
         dtype=np.float64)
 
+    # supplementary: the iterated heat update in FP64 (1 GiB per grid) and an iterated 27-point box
+    t["cfg5L_f64"] = Workload(
+        "cfg5L_f64", "3D 7-point heat diffusion 512^3 in FP64, 16 steps, zero boundary",
+        (512, 512, 512), 1, STAR, ZERO, 16,
+        lambda: star_weights(3, 1, 1.0 - 6 * 0.1, [0.1]).astype(np.float64),
+        _resizable(lambda d: uniform_field(d, 0.0, 1.0, 5, np.float64), (512, 512, 512)),
+        dtype=np.float64)
+    t["box27_iterated"] = Workload(
+        "box27_iterated", "3D 27-point box R=1 512^3, random weights with sum|w|=1, zero boundary, 16 steps",
+        (512, 512, 512), 1, BOX, ZERO, 16,
+        lambda: random_box_weights(3, 1, 2),
+        _resizable(lambda d: normal_field(d, 3), (512, 512, 512)))
+
     # supplementary: the iterated heat operator on a grid that does not fit L2
     t["cfg5L"] = Workload(
         "cfg5L", "3D 7-point heat diffusion 512^3, 16 steps (working set exceeds L2)",

@@ -730,6 +730,57 @@ def test_fused_passes_match_oracle(R, T, width, height, dims, chunk_z):
         assert err <= tol, f"R={R} T={T} width={width} dims={dims} steps={steps}: {err:.3e} > {tol:.3e}"
 
 
+FUSED64_CONFIGS = [   # (fuse_steps, region width in doubles): FP64 3D stars of radius 1
+    (2, 256), (2, 128), (3, 128),
+]
+
+
+@pytest.mark.parametrize("T,width", FUSED64_CONFIGS)
+@pytest.mark.parametrize("dims,chunk_z", [
+    ((29, 70, 300), 11),        # several regions in x and y, ragged everywhere, several z chunks
+    ((40, 64, 256), 0),         # a 256-wide region spans the whole row (the specialised instantiation)
+    ((33, 50, 128), 9),         # the same for the 128-wide regions; ragged in y, several z chunks
+    ((19, 30, 230), 0),         # a row that ends inside a 256-wide region
+    ((5, 9, 12), 0),            # much smaller than one region
+])
+def test_f64_fused_3d_passes_match_oracle(T, width, dims, chunk_z):
+    """Temporal blocking of FP64 3D grids: the fused kernel with two doubles per lane."""
+    w = wl.random_star_weights(3, 1, 61, np.float64)
+    a = wl.normal_field(dims, 62, np.float64)
+    for steps in (T, T + 1, 2 * T + 1):
+        src = torch.from_numpy(a).cuda()
+        dst = torch.full_like(src, float("nan"))
+        with b.Plan(dims, 1, b.STAR, w, b.ZERO, fuse_steps=T, tile_x=width, chunk_z=chunk_z or None) as p:
+            assert p.f64 and p.get(b.KEY_FUSE_STEPS) == T
+            p.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
+            assert p.query_status() == b.OK
+            assert p.launches == -(-steps // T)
+        got = dst.cpu().numpy()
+        want = oracle.apply(a, w, b.ZERO, steps)
+        tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+        err = float(np.max(np.abs(got - want)))
+        assert err <= tol, f"T={T} width={width} dims={dims} steps={steps}: {err:.3e} > {tol:.3e}"
+
+
+def test_f64_fused_3d_is_the_default_where_a_region_spans_the_row():
+    """Iterated FP64 applies fuse two steps per pass by default on rows that fill 80 % of the lanes of
+    their regions (one region of 128 or 256 doubles, or several 128-wide ones on wider rows); other rows,
+    other radii and periodic grids keep one launch per step."""
+    w = wl.star_weights(3, 1, 0.4, [0.1]).astype(np.float64)
+    for dims, want in [((16, 24, 256), 2), ((16, 24, 128), 2), ((16, 24, 210), 2), ((16, 24, 160), 1),
+                       ((16, 24, 512), 2), ((16, 24, 300), 1)]:
+        with b.Plan(dims, 1, b.STAR, w, b.ZERO) as p:
+            assert p.get(b.KEY_FUSE_STEPS) == want, dims
+    with b.Plan((16, 24, 256), 1, b.STAR, w, b.PERIODIC) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1
+    with b.Plan((16, 24, 256), 2, b.STAR, wl.random_star_weights(3, 2, 3, np.float64), b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1
+    a = wl.uniform_field((16, 24, 256), 0.0, 1.0, 3, np.float64)
+    check((16, 24, 256), 1, b.STAR, w, b.ZERO, a, steps=5)
+    a = wl.uniform_field((12, 20, 512), 0.0, 1.0, 4, np.float64)
+    check((12, 20, 512), 1, b.STAR, w, b.ZERO, a, steps=5)
+
+
 def test_fused_equals_unfused_within_tolerance_and_keeps_zero_boundary():
     """A field that would leak through the boundary if out-of-grid cells were
     allowed to evolve inside a fused pass: constant ones, heat weights."""
