@@ -296,7 +296,18 @@ def test_fuse_rules_2d_fp64():
         assert p.get(b.KEY_FUSE_STEPS) == 1             # radius 3 needs two neighbour lanes: no FP64 cascade
     w = wl.random_star_weights(3, 1, 3, np.float64)
     with b.Plan((32, 32, 64), 1, b.STAR, w, b.ZERO) as p:
-        assert p.get(b.KEY_FUSE_STEPS) == 1             # no FP64 temporal blocking in 3D
+        assert p.get(b.KEY_FUSE_STEPS) == 1             # FP64 3D: a 64-wide row fills half a 128-wide region
+        p.set(b.KEY_FUSE_STEPS, 2)                      # ... but the caller may ask for fused passes
+        assert p.get(b.KEY_FUSE_STEPS) == 2
+        with pytest.raises(b.StencilError):
+            p.set(b.KEY_FUSE_STEPS, 4)                  # FP64 3D passes fuse two or three steps
+        p.set(b.KEY_FUSE_STEPS, 0)
+        assert p.get(b.KEY_FUSE_STEPS) == 1
+    with b.Plan((32, 32, 256), 1, b.STAR, w, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2             # one 256-wide region spans the row
+    w2 = wl.random_star_weights(3, 2, 3, np.float64)
+    with b.Plan((32, 32, 256), 2, b.STAR, w2, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 1             # radius 1 only
         with pytest.raises(b.StencilError):
             p.set(b.KEY_FUSE_STEPS, 2)
 
