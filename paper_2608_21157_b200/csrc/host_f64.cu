@@ -348,23 +348,33 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         // planes per chunk, so they get longer chunks (measured on 512^3)
         const int want_chunk = p->radius >= 3 ? 64 : 32;
         int chunk = p->chunk_z > 0 ? p->chunk_z : (span >= 2 * want_chunk ? want_chunk : span);
-        if (p->chunk_z <= 0 && p->shape == STENCIL_STAR && p->radius == 1 && span >= 16) {
-            int occ64 = 0;                            // the 7-point star: very short chunks, as in fp32
-            {
-                std::lock_guard<std::mutex> lock(g_config_mutex);
-                if (cfg->occ_smem != smem) {          // asked once per device and size
-                    int o = 0;
-                    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, cfg->kernel, cfg->threads, smem) !=
-                        cudaSuccess) {
-                        cudaGetLastError();
-                        o = 0;
-                    }
-                    cfg->occ = std::max(o, 1);
-                    cfg->occ_smem = smem;
+        int occ64 = 1;                                // resident CTAs per SM, asked once per device and size
+        {
+            std::lock_guard<std::mutex> lock(g_config_mutex);
+            if (cfg->occ_smem != smem) {
+                int o = 0;
+                if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, cfg->kernel, cfg->threads, smem) != cudaSuccess) {
+                    cudaGetLastError();
+                    o = 0;
                 }
-                occ64 = cfg->occ;
+                cfg->occ = std::max(o, 1);
+                cfg->occ_smem = smem;
             }
-            chunk = short_chunk_star1(span, (int64_t)g.tiles_x * g.tiles_y, (int64_t)occ64 * plan_sms(p));
+            occ64 = cfg->occ;
+        }
+        const int64_t tiles64 = (int64_t)g.tiles_x * g.tiles_y, slots64 = (int64_t)occ64 * plan_sms(p);
+        if (p->chunk_z <= 0 && p->shape == STENCIL_STAR && p->radius == 1 && span >= 16) {
+            chunk = short_chunk_star1(span, tiles64, slots64);      // the 7-point star: very short chunks, as in fp32
+        } else if (p->chunk_z <= 0 && span >= 16 && tiles64 * ((span + want_chunk - 1) / want_chunk) < 4 * slots64) {
+            // a grid that does not cut into several machines' worth of CTAs: whole waves of chunks of 8 planes
+            // or more, none longer than the usual length (the same rule as the fp32 sweeps)
+            double best = 1e300;
+            for (int n = (span + want_chunk - 1) / want_chunk; n <= std::max(1, span / 8); ++n) {
+                const int c = (span + n - 1) / n;
+                const int64_t ctas = tiles64 * ((span + c - 1) / c);
+                const double cost = (double)((ctas + slots64 - 1) / slots64) * (c + 2 * p->radius + 4.0);
+                if (cost < best * 0.999) { best = cost; chunk = c; }
+            }
         }
         if (p->chunk_z <= 0 && (p->radius >= 4 || (p->shape == STENCIL_BOX && p->radius >= 2))) {
             // The radius-4 star is no longer bound by memory alone (25 DFMA and 15 shared-memory
