@@ -46,12 +46,13 @@ SM_COUNT, SM_MAX_MHZ = 148, 1965.0
 # one launch at the workload's full size, from the ncu captures summarised under profiles/).
 # None = not captured.
 NCU_TRAFFIC_BYTES = {
-    "cfg2": 1023.6e6,   # stream kernel, star R=1, 512^3: 537.2 MB read + 486.4 MB written
-    "cfg3": 1047.0e6,   # stream kernel, box R=1, 512^3: 559.7 + 487.3
-    "cfg4": 1040.4e6,   # stream kernel, star R=4, 512^3: 553.3 + 487.1
-    "cfg5": 99.9e6,     # one fused pass (2 time steps of 256^3): 77.7 MB read + 22.2 MB written
-    "cfg5L": 1035.1e6,  # one fused pass (2 time steps of 512^3): 545.4 MB read + 489.7 MB written
-    "heat2d": 756.3e6,  # one fused pass (4 time steps of 10240^2): 2.5 x (180.6 + 121.9 MB) captured on 4096 x 10240
+    "cfg2": 1026.4e6,       # stream kernel, star R=1, 512^3: 536.9 MB read + 489.5 MB written
+    "cfg3": 1055.0e6,       # stream kernel, box R=1, 512^3: 564.3 + 490.7
+    "cfg4": 1049.1e6,       # stream kernel, star R=4, 512^3: 557.4 + 491.7
+    "cfg5": 99.2e6,         # one fused pass (2 time steps of 256^3): 77.4 + 21.8 (both grids largely stay in L2)
+    "cfg5L": 1034.9e6,      # one fused pass (2 time steps of 512^3): 545.5 + 489.3
+    "cfg5L_f64": 2169.1e6,  # one fused pass (2 time steps of 512^3 in FP64): 1136.2 + 1032.8
+    "heat2d": 805.9e6,      # one fused pass (4 time steps of 10240^2): 432.9 + 373.0
 }
 
 
