@@ -144,27 +144,23 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                         A[2 * R - 1] = make_float4(a[0], a[1], a[2], a[3]);
                     }
                 } else {
-                    // star: only the output whose own row this is takes the x taps
-                    done.x = fmaf(wt.w[2 * R][R], c.x, A[0].x);
-                    done.y = fmaf(wt.w[2 * R][R], c.y, A[0].y);
-                    done.z = fmaf(wt.w[2 * R][R], c.z, A[0].z);
-                    done.w = fmaf(wt.w[2 * R][R], c.w, A[0].w);
-                    float acc[4] = {A[R].x, A[R].y, A[R].z, A[R].w};
+                    // star: only the output whose own row this is takes the x taps.  The y taps and the
+                    // centre tap work on the two halves of the lane's float4 (packed FMAs).
+                    done = fma4r(wt.w[2 * R][R], c, A[0]);
+                    const float4 ctr = fma4r(wt.w[R][R], c, A[R]);
+                    float acc[4] = {ctr.x, ctr.y, ctr.z, ctr.w};
 #pragma unroll
-                    for (int dx = 0; dx < M; ++dx)
+                    for (int dx = 0; dx < M; ++dx) {
+                        if (dx == R) continue;         // the centre tap is in `ctr` already (v[m + R] is c)
 #pragma unroll
                         for (int m = 0; m < 4; ++m) acc[m] = fmaf(wt.w[R][dx], v[m + dx], acc[m]);
+                    }
 #pragma unroll
                     for (int j = 0; j < 2 * R - 1; ++j) {
                         if (j == R - 1) continue;
-                        const float wy = wt.w[2 * R - 1 - j][R];
-                        A[j].x = fmaf(wy, c.x, A[j + 1].x);
-                        A[j].y = fmaf(wy, c.y, A[j + 1].y);
-                        A[j].z = fmaf(wy, c.z, A[j + 1].z);
-                        A[j].w = fmaf(wy, c.w, A[j + 1].w);
+                        A[j] = fma4r(wt.w[2 * R - 1 - j][R], c, A[j + 1]);
                     }
-                    A[2 * R - 1] = make_float4(wt.w[0][R] * c.x, wt.w[0][R] * c.y, wt.w[0][R] * c.z,
-                                               wt.w[0][R] * c.w);
+                    A[2 * R - 1] = mul4(wt.w[0][R], c);
                     A[R - 1] = make_float4(acc[0], acc[1], acc[2], acc[3]);
                 }
                 if (i >= 2 * R) {
