@@ -332,7 +332,7 @@ def run_gpu(args):
     wk = pick_workload(args)
     knobs = dict(tile_y=args.tile_y, chunk_z=args.chunk_z, stages=args.stages,
                  rows_per_thread=args.rows_per_thread, streaming_store=args.streaming_store,
-                 fuse_steps=args.fuse_steps)
+                 fuse_steps=args.fuse_steps, tile_x=args.tile_x)
     variant = {"auto": None, "generic": b.VARIANT_GENERIC, "stream": b.VARIANT_STREAM,
                "fused": b.VARIANT_FUSED}[args.variant]
 
@@ -780,6 +780,7 @@ def main():
     ap.add_argument("--chunk-z", dest="chunk_z", type=int, default=None)
     ap.add_argument("--stages", type=int, default=None)
     ap.add_argument("--fuse-steps", dest="fuse_steps", type=int, default=None)
+    ap.add_argument("--tile-x", dest="tile_x", type=int, default=None, help="region width of fused 3D passes")
     ap.add_argument("--streaming-store", dest="streaming_store", type=int, default=None)
     ap.add_argument("--also", default="cfg1,cfg3,cfg4,cfg5,cfg5L,cfg5L_periodic,cfg5L_f64,box27_iterated,paper2d,paper2d_f64,heat2d", help="other workloads summarised in all_configs")
     ap.add_argument("--also-steps", dest="also_steps", type=int, default=20)
