@@ -69,10 +69,12 @@ enum {
 /* Keys of stencil_plan_set / stencil_plan_get. */
 enum {
     STENCIL_KEY_VARIANT      = 0,  /* set/get: STENCIL_VARIANT_*                                 */
-    STENCIL_KEY_TILE_X       = 1,  /* set/get: region width of fused 3D passes, 128, 256, 384 or 512 (0 = auto) */
+    STENCIL_KEY_TILE_X       = 1,  /* set/get: region width of fused 3D passes, 128, 256, 384 or 512
+                                      (FP64: 128 or 256; 0 = auto)                               */
     STENCIL_KEY_TILE_Y       = 2,  /* set/get: tile height in rows   (0 = default)               */
     STENCIL_KEY_FUSE_STEPS   = 3,  /* set: time steps fused per pass (0 = auto, 1 = off; 3D fp32
-                                      stars: 2-4; 2D grids: the one depth the operator's fused
+                                      stars: 2-4; 3D FP64 stars of radius 1 with a zero boundary:
+                                      2 or 3; 2D grids: the one depth the operator's fused
                                       kernel has: star and box R=1: 4, star R=2: 3, box R=2: 2,
                                       fp32 stars R=3 and 4: 2);
                                       get: the number iterated applies will use (1 = none)       */
@@ -177,7 +179,8 @@ STENCIL_API int stencil_apply(stencil_plan_t plan, const float* in, float* out, 
  * radius 4 and 3D boxes up to radius 2, with a zero boundary (rows of an odd
  * number of doubles through grids with padded rows) or a periodic one (even
  * nx); everything else runs on the one-thread-per-point kernel.  Temporal
- * blocking in FP64 exists for 2D grids with radius <= 2 (even nx).
+ * blocking in FP64 exists for 2D grids with radius <= 2 and for 3D stars of
+ * radius 1 with a zero boundary (even nx).
  */
 STENCIL_API int stencil_plan_f64(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radius,
                                  int shape, const double* weights, int boundary);
