@@ -340,3 +340,48 @@ def test_a_plan_stays_on_the_device_of_its_first_apply():
         with torch.cuda.device(0):
             p.apply(src, dst, 1, 0)
             assert p.query_status() == b.OK
+
+
+def test_header_is_plain_c_and_links_against_the_library(tmp_path):
+    """include/stencil.h compiles as C99 with a strict compiler, and a C program that uses only the header
+    links against the library and gets the documented statuses back (host-side checks only: no GPU needed)."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "use_abi.c"
+    src.write_text(r'''
+#include "stencil.h"
+#include <stdio.h>
+int main(void) {
+    stencil_plan_t p = (stencil_plan_t)0x1;
+    int64_t dims[3] = {8, 8, 8};
+    float w[27];
+    for (int i = 0; i < 27; ++i) w[i] = 0.0f;
+    w[13] = -6.0f; w[4] = w[10] = w[12] = w[14] = w[16] = w[22] = 1.0f;
+    if (stencil_plan(&p, 3, dims, 0, STENCIL_STAR, w, STENCIL_ZERO) != STENCIL_ERR_INVALID || p != 0) return 1;
+    if (stencil_plan(&p, 3, dims, 9, STENCIL_STAR, w, STENCIL_ZERO) != STENCIL_ERR_UNSUPPORTED) return 2;
+    w[0] = 1.0f;                                   /* an off-axis weight breaks the STAR promise */
+    if (stencil_plan(&p, 3, dims, 1, STENCIL_STAR, w, STENCIL_ZERO) != STENCIL_ERR_INVALID) return 3;
+    if (stencil_plan(&p, 3, dims, 1, STENCIL_BOX, w, STENCIL_ZERO) != STENCIL_OK || p == 0) return 4;
+    int64_t v = -1;
+    if (stencil_plan_get(p, STENCIL_KEY_LAUNCHES, &v) != STENCIL_OK || v != 0) return 5;
+    if (stencil_plan_get(p, STENCIL_KEY_DEVICE, &v) != STENCIL_OK || v != -1) return 6;
+    if (stencil_apply(p, 0, 0, 1, 0) != STENCIL_ERR_INVALID) return 7;
+    if (stencil_query_status(p) != STENCIL_OK) return 8;
+    if (stencil_destroy(p) != STENCIL_OK || stencil_destroy(0) != STENCIL_OK) return 9;
+    puts(stencil_status_string(STENCIL_ERR_TIMEOUT));
+    return 0;
+}
+''')
+    exe = tmp_path / "use_abi"
+    lib_dir = os.path.dirname(b.LIB_PATH)
+    cmd = [gcc, "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(root, "include"),
+           str(src), "-o", str(exe), "-L", lib_dir, "-l:libstencil_b200.so", f"-Wl,-rpath,{lib_dir}"]
+    r = subprocess.run(cmd, capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
+    r = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert r.returncode == 0, f"step {r.returncode} of the C program failed"
+    assert "wait" in r.stdout
