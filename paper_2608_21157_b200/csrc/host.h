@@ -272,11 +272,48 @@ namespace stencil_host {
 
 inline bool valid_plan(const stencil_plan_s* p) { return p && p->magic == kPlanMagic; }
 
-// entry [dz+R][dy+R][dx+R] of the plan's dense fp32 weights (2D plans: dz must be 0)
-inline float dense_w(const stencil_plan_s* p, int dz, int dy, int dx) {
+// entry [dz+R][dy+R][dx+R] of the plan's dense weights in the plan's own precision
+template <typename E>
+inline E dense_tap(const stencil_plan_s* p, int dz, int dy, int dx) {
     const int R = p->radius, side = 2 * R + 1;
-    if (p->ndim == 3) return p->w[((size_t)(dz + R) * side + (dy + R)) * side + (dx + R)];
-    return dz == 0 ? p->w[(size_t)(dy + R) * side + (dx + R)] : 0.0f;
+    const size_t f = p->ndim == 3 ? ((size_t)(dz + R) * side + (dy + R)) * side + (dx + R)
+                                  : (size_t)(dy + R) * side + (dx + R);
+    if constexpr (sizeof(E) == 8) return p->w64[f];
+    else return p->w[f];
+}
+
+// The taps of a 3D star (members c, x[], y[], z[], index d + R) or box (member w[][][]) as the kernels take them.
+template <typename E, int R, typename SW>
+inline void pack_star3d(const stencil_plan_s* p, SW& sw) {
+    std::memset(&sw, 0, sizeof(sw));
+    sw.c = dense_tap<E>(p, 0, 0, 0);
+    for (int d = -R; d <= R; ++d) {
+        if (d == 0) continue;
+        sw.x[d + R] = dense_tap<E>(p, 0, 0, d);
+        sw.y[d + R] = dense_tap<E>(p, 0, d, 0);
+        sw.z[d + R] = dense_tap<E>(p, d, 0, 0);
+    }
+}
+template <typename E, int R, typename BW>
+inline void pack_box3d(const stencil_plan_s* p, BW& bw) {
+    std::memset(&bw, 0, sizeof(bw));
+    for (int a = -R; a <= R; ++a)
+        for (int b = -R; b <= R; ++b)
+            for (int c = -R; c <= R; ++c) bw.w[a + R][b + R][c + R] = dense_tap<E>(p, a, b, c);
+}
+// star or box, whichever the kernel instantiation reads (the other stays zero)
+template <typename E, int R, bool BOX, typename SW, typename BW>
+inline void pack_taps3d(const stencil_plan_s* p, SW& sw, BW& bw) {
+    std::memset(&sw, 0, sizeof(sw));
+    std::memset(&bw, 0, sizeof(bw));
+    if constexpr (BOX) pack_box3d<E, R>(p, bw);
+    else pack_star3d<E, R>(p, sw);
+}
+// the dense (2R+1)^2 weights of a 2D operator (member w[][])
+template <typename E, int R, typename W2>
+inline void pack_taps2d(const stencil_plan_s* p, W2& wt) {
+    for (int a = -R; a <= R; ++a)
+        for (int b = -R; b <= R; ++b) wt.w[a + R][b + R] = dense_tap<E>(p, 0, a, b);
 }
 
 // A periodic grid takes fused passes of L steps as zero-boundary passes whose shell of depth

@@ -7,21 +7,11 @@
 
 namespace stencil_host {
 
-// ---------------------------------------------------------------------------
-// FP64 plans: the generic kernel for everything, the row-streaming kernel for
-// 2D grids with a zero boundary (the paper's own case)
-// ---------------------------------------------------------------------------
-inline double dense_w64(const stencil_plan_s* p, int dy, int dx) {
-    const int R = p->radius, side = 2 * R + 1;
-    return p->w64[(size_t)(dy + R) * side + (dx + R)];
-}
-
 template <int R, bool BOX, int YB, int NW>
 cudaError_t launch_rows2d64_t(const stencil_plan_s* p, const CUtensorMap& map, double* out, const Rows2DGeom& g,
                               int grid, size_t smem, cudaStream_t st) {
     Weights2D64<R> wt;
-    for (int a = -R; a <= R; ++a)
-        for (int b = -R; b <= R; ++b) wt.w[a + R][b + R] = dense_w64(p, a, b);
+    pack_taps2d<double, R>(p, wt);
     return launch_kernel(&stencil_rows2d_f64_kernel<R, BOX, YB, NW>, grid, NW * 32, smem, st, p->chained, map, out,
                          g, wt, p->d_status);
 }
@@ -59,32 +49,12 @@ const Rows2D64Config* find_rows2d64_cfg(const stencil_plan_s* p) {
     return nullptr;
 }
 
-inline double dense_w64_3d(const stencil_plan_s* p, int dz, int dy, int dx) {
-    const int R = p->radius, side = 2 * R + 1;
-    return p->w64[((size_t)(dz + R) * side + (dy + R)) * side + (dx + R)];
-}
-
 template <int R, bool BOX, int K, int NW, int MINB>
 cudaError_t launch_stream64_t(const stencil_plan_s* p, const CUtensorMap& map, double* out, const StreamGeom& g,
                               int grid, size_t smem, cudaStream_t st) {
     StarWeights64<R> sw;
     BoxWeights64<BOX ? R : 0> bw;
-    std::memset(&sw, 0, sizeof(sw));
-    std::memset(&bw, 0, sizeof(bw));
-    if (!BOX) {
-        sw.c = dense_w64_3d(p, 0, 0, 0);
-        for (int d = -R; d <= R; ++d) {
-            if (d == 0) continue;
-            sw.x[d + R] = dense_w64_3d(p, 0, 0, d);
-            sw.y[d + R] = dense_w64_3d(p, 0, d, 0);
-            sw.z[d + R] = dense_w64_3d(p, d, 0, 0);
-        }
-    } else {
-        constexpr int RB = BOX ? R : 0;
-        for (int a = -RB; a <= RB; ++a)
-            for (int b = -RB; b <= RB; ++b)
-                for (int c = -RB; c <= RB; ++c) bw.w[a + RB][b + RB][c + RB] = dense_w64_3d(p, a, b, c);
-    }
+    pack_taps3d<double, R, BOX>(p, sw, bw);
     return launch_kernel(&stencil_stream_f64_kernel<R, BOX, K, NW, MINB>, grid, Stream64Shape<R, K, NW>::THREADS,
                          smem, st, p->chained, map, out, g, sw, bw, p->d_status);
 }
@@ -95,22 +65,7 @@ cudaError_t launch_stream64_wrap_t(const stencil_plan_s* p, const CUtensorMap& m
                                    const StreamGeom& g, int grid, size_t smem, cudaStream_t st) {
     StarWeights64<R> sw;
     BoxWeights64<BOX ? R : 0> bw;
-    std::memset(&sw, 0, sizeof(sw));
-    std::memset(&bw, 0, sizeof(bw));
-    if (!BOX) {
-        sw.c = dense_w64_3d(p, 0, 0, 0);
-        for (int d = -R; d <= R; ++d) {
-            if (d == 0) continue;
-            sw.x[d + R] = dense_w64_3d(p, 0, 0, d);
-            sw.y[d + R] = dense_w64_3d(p, 0, d, 0);
-            sw.z[d + R] = dense_w64_3d(p, d, 0, 0);
-        }
-    } else {
-        constexpr int RB = BOX ? R : 0;
-        for (int a = -RB; a <= RB; ++a)
-            for (int b = -RB; b <= RB; ++b)
-                for (int c = -RB; c <= RB; ++c) bw.w[a + RB][b + RB][c + RB] = dense_w64_3d(p, a, b, c);
-    }
+    pack_taps3d<double, R, BOX>(p, sw, bw);
     return launch_kernel(&stencil_stream_f64_wrap_kernel<R, BOX, K, NW, MINB>, grid, Stream64Shape<R, K, NW>::THREADS,
                          smem, st, p->chained, map, map_xs, map_ys, map_cs, out, g, sw, bw, p->d_status);
 }
@@ -160,8 +115,7 @@ template <int R, bool BOX, int T, int YB, int NW>
 cudaError_t launch_rows2d_fused64_t(const stencil_plan_s* p, const CUtensorMap& map, double* out,
                                     const Rows2DFusedGeom& g, int grid, size_t smem, cudaStream_t st) {
     Weights2D64<R> wt;
-    for (int a = -R; a <= R; ++a)
-        for (int b = -R; b <= R; ++b) wt.w[a + R][b + R] = dense_w64(p, a, b);
+    pack_taps2d<double, R>(p, wt);
     return launch_kernel(&stencil_rows2d_fused_f64_kernel<R, BOX, T, YB, NW>, grid, NW * 32, smem, st, p->chained,
                          map, out, g, wt, p->d_status);
 }

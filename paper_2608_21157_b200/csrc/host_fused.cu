@@ -4,31 +4,11 @@
 
 namespace stencil_host {
 
-template <typename E>
-inline E dense_tap(const stencil_plan_s* p, int dz, int dy, int dx) {
-    const int R = p->radius, side = 2 * R + 1;
-    const size_t f = ((size_t)(dz + R) * side + (dy + R)) * side + (dx + R);
-    if constexpr (sizeof(E) == 8) return p->w64[f];
-    else return p->w[f];
-}
-
-template <typename E, int R>
-void pack_star(const stencil_plan_s* p, StarTaps<E, R>& sw) {
-    std::memset(&sw, 0, sizeof(sw));
-    sw.c = dense_tap<E>(p, 0, 0, 0);
-    for (int d = -R; d <= R; ++d) {
-        if (d == 0) continue;
-        sw.x[d + R] = dense_tap<E>(p, 0, 0, d);
-        sw.y[d + R] = dense_tap<E>(p, 0, d, 0);
-        sw.z[d + R] = dense_tap<E>(p, d, 0, 0);
-    }
-}
-
 template <typename E, int R, int T, int K, int XW, int NWY, int MODE>
 cudaError_t launch_fused_t(const stencil_plan_s* p, const CUtensorMap& map, void* out, const FusedGeom& g,
                            int grid, size_t smem, cudaStream_t st) {
     StarTaps<E, R> sw;
-    pack_star<E, R>(p, sw);
+    pack_star3d<E, R>(p, sw);
     return launch_kernel(&stencil_fused_kernel<E, R, T, K, XW, NWY, MODE>, grid,
                          FusedShape<R, K, XW, NWY, E>::THREADS, smem, st, p->chained, map, static_cast<E*>(out), g,
                          sw, p->d_status);

@@ -9,8 +9,7 @@ template <int R, bool BOX, int YB, int NW>
 cudaError_t launch_rows2d_t(const stencil_plan_s* p, const CUtensorMap& map, float* out, const Rows2DGeom& g,
                             int grid, size_t smem, cudaStream_t st) {
     Weights2D<R> wt;
-    for (int a = -R; a <= R; ++a)
-        for (int b = -R; b <= R; ++b) wt.w[a + R][b + R] = dense_w(p, 0, a, b);
+    pack_taps2d<float, R>(p, wt);
     return launch_kernel(&stencil_rows2d_kernel<R, BOX, YB, NW>, grid, NW * 32, smem, st, p->chained, map, out, g,
                          wt, p->d_status);
 }
@@ -53,8 +52,7 @@ template <int R, bool BOX, int T, int YB, int NW>
 cudaError_t launch_rows2d_fused_t(const stencil_plan_s* p, const CUtensorMap& map, float* out,
                                   const Rows2DFusedGeom& g, int grid, size_t smem, cudaStream_t st) {
     Weights2D<R> wt;
-    for (int a = -R; a <= R; ++a)
-        for (int b = -R; b <= R; ++b) wt.w[a + R][b + R] = dense_w(p, 0, a, b);
+    pack_taps2d<float, R>(p, wt);
     return launch_kernel(&stencil_rows2d_fused_kernel<R, BOX, T, YB, NW>, grid, NW * 32, smem, st, p->chained, map,
                          out, g, wt, p->d_status);
 }

@@ -9,22 +9,7 @@ cudaError_t launch_stream_t(const stencil_plan_s* p, const StreamConfig&, const 
                             float* out, const StreamGeom& g, int grid, size_t smem, cudaStream_t st) {
     StarWeights<R> sw;
     BoxWeights<BOX ? R : 0> bw;
-    std::memset(&sw, 0, sizeof(sw));
-    std::memset(&bw, 0, sizeof(bw));
-    if (!BOX) {
-        sw.c = dense_w(p, 0, 0, 0);
-        for (int d = -R; d <= R; ++d) {
-            if (d == 0) continue;
-            sw.x[d + R] = dense_w(p, 0, 0, d);
-            sw.y[d + R] = dense_w(p, 0, d, 0);
-            sw.z[d + R] = dense_w(p, d, 0, 0);
-        }
-    } else {
-        constexpr int RB = BOX ? R : 0;
-        for (int a = -RB; a <= RB; ++a)
-            for (int b = -RB; b <= RB; ++b)
-                for (int c = -RB; c <= RB; ++c) bw.w[a + RB][b + RB][c + RB] = dense_w(p, a, b, c);
-    }
+    pack_taps3d<float, R, BOX>(p, sw, bw);
     return launch_kernel(&stencil_stream_kernel<R, BOX, K, NW, MINB>, grid, StreamShape<R, K, NW>::THREADS, smem,
                          st, p->chained, map, out, g, sw, bw, p->d_status);
 }
@@ -35,22 +20,7 @@ cudaError_t launch_stream_wrap_t(const stencil_plan_s* p, const CUtensorMap& map
                                  const StreamGeom& g, int grid, size_t smem, cudaStream_t st) {
     StarWeights<R> sw;
     BoxWeights<BOX ? R : 0> bw;
-    std::memset(&sw, 0, sizeof(sw));
-    std::memset(&bw, 0, sizeof(bw));
-    if (!BOX) {
-        sw.c = dense_w(p, 0, 0, 0);
-        for (int d = -R; d <= R; ++d) {
-            if (d == 0) continue;
-            sw.x[d + R] = dense_w(p, 0, 0, d);
-            sw.y[d + R] = dense_w(p, 0, d, 0);
-            sw.z[d + R] = dense_w(p, d, 0, 0);
-        }
-    } else {
-        constexpr int RB = BOX ? R : 0;
-        for (int a = -RB; a <= RB; ++a)
-            for (int b = -RB; b <= RB; ++b)
-                for (int c = -RB; c <= RB; ++c) bw.w[a + RB][b + RB][c + RB] = dense_w(p, a, b, c);
-    }
+    pack_taps3d<float, R, BOX>(p, sw, bw);
     return launch_kernel(&stencil_stream_wrap_kernel<R, BOX, K, NW, MINB>, grid, StreamShape<R, K, NW>::THREADS, smem,
                          st, p->chained, map, map_xs, map_ys, map_cs, out, g, sw, bw, p->d_status);
 }
