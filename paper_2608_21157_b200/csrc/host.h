@@ -67,6 +67,18 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), int grid, int block, size_t 
 // caches safe when several host threads drive their own plans.
 extern std::mutex g_config_mutex;
 
+// Per-device facts of one kernel, cached in its configuration (guarded by g_config_mutex).
+struct KernelLimits {
+    size_t smem_allowed = 0;     // dynamic shared memory the kernel has been granted (it only ever grows)
+    size_t occ_smem = 0;         // the shared-memory size `occ` was measured at
+    int occ = 0;                 // resident CTAs per SM at that size
+    int device = -1;             // the device these facts belong to
+};
+// Makes sure `kernel` may use `smem` bytes of dynamic shared memory on device `dev` (the current one) and
+// returns its resident CTAs per SM at that size (>= 1; 1 without a query when `want_occ` is false), or -1
+// when a CUDA call fails.
+int kernel_limits(const void* kernel, int threads, size_t smem, int dev, KernelLimits& lim, bool want_occ);
+
 }  // namespace stencil_host
 
 struct stencil_plan_s;
@@ -83,16 +95,13 @@ struct StreamConfig {
     int tile_y;           // K * NW
     int plane_bytes, box_rows, threads;
     int px;               // columns of the TMA box: the tile plus its halo on both sides
-    mutable int occupancy[kMaxStages + 1];   // resident CTAs per SM by ring depth; 0 = not asked yet
-    mutable size_t smem_allowed;             // dynamic shared memory the kernel is currently allowed
-    mutable int cache_device;                // device the two caches above were filled on
+    mutable KernelLimits lim, lim_wrap;      // of `kernel` and `kernel_wrap`
     const void* kernel;
     cudaError_t (*launch)(const stencil_plan_s*, const StreamConfig&, const CUtensorMap&,
                           float*, const StreamGeom&, int grid, size_t smem, cudaStream_t);
     // the sweep of a periodic grid inside the kernel (stars of radius <= 4 and the boxes; null otherwise)
     const void* kernel_wrap;
     int stage_bytes;                         // per ring slot, beside the plane
-    mutable size_t smem_allowed_wrap;
     cudaError_t (*launch_wrap)(const stencil_plan_s*, const CUtensorMap&, const CUtensorMap&,
                                const CUtensorMap&, const CUtensorMap&, float*, const StreamGeom&, int grid,
                                size_t smem, cudaStream_t);
@@ -110,10 +119,7 @@ struct FusedConfig {
     const void* kernel;
     const void* kernel_spec;                 // the instantiation for full passes over rows of exactly txe points
     const void* kernel_wrap;                 // ... and the one of those that wraps x and z (passes of a periodic grid)
-    mutable size_t smem_allowed;             // dynamic shared memory already granted to both kernels
-    mutable size_t occ_smem;                 // ... and the occupancy measured at this size
-    mutable int occ;
-    mutable int cache_device;
+    mutable KernelLimits lim, lim_spec, lim_wrap;   // of the three kernels
     // `out` is a float* or double* as the configuration's element type says
     cudaError_t (*launch)(const stencil_plan_s*, const CUtensorMap&, void* out, const FusedGeom&,
                           int grid, size_t smem, cudaStream_t);
@@ -132,8 +138,7 @@ struct Rows2DConfig {
     int YB, NW, batch_bytes;
     int px;                     // columns of the TMA box: the strip plus its halo on both sides
     const void* kernel;
-    mutable size_t smem_allowed;
-    mutable int cache_device;
+    mutable KernelLimits lim;
     cudaError_t (*launch)(const stencil_plan_s*, const CUtensorMap&, float*, const Rows2DGeom&,
                           int grid, size_t smem, cudaStream_t);
 };
@@ -146,10 +151,7 @@ struct Rows2DFusedConfig {
     bool box;
     int T, YB, NW, batch_bytes;
     const void* kernel;
-    mutable size_t smem_allowed;
-    mutable size_t occ_smem;                 // shared-memory size the occupancy below was measured at
-    mutable int occ;                         // resident CTAs per SM
-    mutable int cache_device;
+    mutable KernelLimits lim;
     cudaError_t (*launch)(const stencil_plan_s*, const CUtensorMap&, float*, const Rows2DFusedGeom&,
                           int grid, size_t smem, cudaStream_t);
 };
@@ -162,10 +164,7 @@ struct Rows2DFused64Config {
     bool box;
     int T, YB, NW, batch_bytes;
     const void* kernel;
-    mutable size_t smem_allowed;
-    mutable size_t occ_smem;
-    mutable int occ;
-    mutable int cache_device;
+    mutable KernelLimits lim;
     cudaError_t (*launch)(const stencil_plan_s*, const CUtensorMap&, double*, const Rows2DFusedGeom&,
                           int grid, size_t smem, cudaStream_t);
 };
@@ -175,8 +174,7 @@ struct Rows2D64Config {
     bool box;
     int YB, NW, batch_bytes, px;
     const void* kernel;
-    mutable size_t smem_allowed;
-    mutable int cache_device;
+    mutable KernelLimits lim;
     cudaError_t (*launch)(const stencil_plan_s*, const CUtensorMap&, double*, const Rows2DGeom&,
                           int grid, size_t smem, cudaStream_t);
 };
@@ -186,16 +184,12 @@ struct Stream64Config {
     bool box;
     int tile_y, plane_bytes, box_rows, threads, px;
     const void* kernel;
-    mutable size_t smem_allowed;
-    mutable size_t occ_smem;                 // shared-memory size the occupancy below was asked for
-    mutable int occ;                         // resident CTAs per SM
-    mutable int cache_device;
+    mutable KernelLimits lim, lim_wrap;      // of `kernel` and `kernel_wrap`
     cudaError_t (*launch)(const stencil_plan_s*, const CUtensorMap&, double*, const StreamGeom&,
                           int grid, size_t smem, cudaStream_t);
     // the sweep of a periodic grid inside the kernel (stars of radius <= 4; null otherwise)
     const void* kernel_wrap;
     int stage_bytes;                         // per ring slot, beside the plane
-    mutable size_t smem_allowed_wrap;
     cudaError_t (*launch_wrap)(const stencil_plan_s*, const CUtensorMap&, const CUtensorMap&,
                                const CUtensorMap&, const CUtensorMap&, double*, const StreamGeom&, int grid,
                                size_t smem, cudaStream_t);

@@ -30,6 +30,32 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
+int kernel_limits(const void* kernel, int threads, size_t smem, int dev, KernelLimits& lim, bool want_occ) {
+    std::lock_guard<std::mutex> lock(g_config_mutex);
+    if (dev != lim.device) {                       // function attributes are per device
+        lim = KernelLimits{};
+        lim.device = dev;
+    }
+    if (smem > lim.smem_allowed) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+            cudaGetLastError();
+            return -1;
+        }
+        lim.smem_allowed = smem;
+    }
+    if (!want_occ) return 1;
+    if (lim.occ_smem != smem || lim.occ <= 0) {
+        int o = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kernel, threads, smem) != cudaSuccess) {
+            cudaGetLastError();
+            o = 0;
+        }
+        lim.occ = std::max(o, 1);
+        lim.occ_smem = smem;
+    }
+    return lim.occ;
+}
+
 // ---------------------------------------------------------------------------
 // device state
 // ---------------------------------------------------------------------------

@@ -22,7 +22,6 @@ Rows2D64Config make_rows2d64() {
     c.radius = R; c.box = BOX; c.YB = YB; c.NW = NW; c.px = StreamHalo64<R>::PX;
     c.batch_bytes = Rows2D64Shape<YB, StreamHalo64<R>::PX>::BATCH_BYTES;
     c.kernel = reinterpret_cast<const void*>(&stencil_rows2d_f64_kernel<R, BOX, YB, NW>);
-    c.smem_allowed = 0; c.cache_device = -1;
     c.launch = &launch_rows2d64_t<R, BOX, YB, NW>;
     return c;
 }
@@ -77,9 +76,8 @@ Stream64Config make_stream64() {
     c.radius = R; c.box = BOX; c.tile_y = S::TY; c.plane_bytes = S::PLANE_BYTES; c.box_rows = S::ROWS;
     c.threads = S::THREADS; c.px = StreamHalo64<R>::PX;
     c.kernel = reinterpret_cast<const void*>(&stencil_stream_f64_kernel<R, BOX, K, NW, MINB>);
-    c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
     c.launch = &launch_stream64_t<R, BOX, K, NW, MINB>;
-    c.kernel_wrap = nullptr; c.launch_wrap = nullptr; c.stage_bytes = 0; c.smem_allowed_wrap = 0;
+    c.kernel_wrap = nullptr; c.launch_wrap = nullptr; c.stage_bytes = 0;
     if constexpr (R <= 4) {
         c.kernel_wrap = reinterpret_cast<const void*>(&stencil_stream_f64_wrap_kernel<R, BOX, K, NW, MINB>);
         c.launch_wrap = &launch_stream64_wrap_t<R, BOX, K, NW, MINB>;
@@ -125,7 +123,6 @@ Rows2DFused64Config make_rows2d_fused64() {
     Rows2DFused64Config c;
     c.radius = R; c.box = BOX; c.T = T; c.YB = YB; c.NW = NW; c.batch_bytes = Rows2D64Shape<YB>::BATCH_BYTES;
     c.kernel = reinterpret_cast<const void*>(&stencil_rows2d_fused_f64_kernel<R, BOX, T, YB, NW>);
-    c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
     c.launch = &launch_rows2d_fused64_t<R, BOX, T, YB, NW>;
     return c;
 }
@@ -173,33 +170,11 @@ int launch_rows2d_fused64(stencil_plan_s* p, const double* src, double* dst, int
     if (rc != STENCIL_OK) return rc;
     int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 2;
     auto smem_for = [&](int s_) { return (size_t)cfg->NW * s_ * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8; };
-    while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
+    while (stages > 2 && smem_for(stages) > kMaxSmemBytes) --stages;      // a ring deeper than shared memory holds is cut back
     const size_t smem = smem_for(stages);
-    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-    const int dev = p->device;                       // current: the apply entry points have checked it
-    int occ = 1;
-    {
-        std::lock_guard<std::mutex> lock(g_config_mutex);
-        if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->occ_smem = 0; cfg->cache_device = dev; }
-        if (smem > cfg->smem_allowed) {
-            if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess) {
-                cudaGetLastError();
-                return STENCIL_ERR_CUDA;
-            }
-            cfg->smem_allowed = smem;
-        }
-        if (cfg->occ_smem != smem) {
-            int o = 0;
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, cfg->kernel, cfg->NW * 32, smem) != cudaSuccess) {
-                cudaGetLastError();
-                o = 0;
-            }
-            cfg->occ = std::max(o, 1);
-            cfg->occ_smem = smem;
-        }
-        occ = cfg->occ;
-    }
+    if (smem > kMaxSmemBytes) return STENCIL_ERR_UNSUPPORTED;
+    const int occ = kernel_limits(cfg->kernel, cfg->NW * 32, smem, p->device, cfg->lim, true);
+    if (occ < 0) return STENCIL_ERR_CUDA;
     Rows2DFusedGeom g;
     g.ny = p->ny; g.nx = p->nx;
     g.strips = (p->nx + kFused2D64Tile - 1) / kFused2D64Tile;
@@ -268,25 +243,13 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         auto smem_for = [&](int s_) {
             return (size_t)s_ * (cfg->plane_bytes + (wrap ? cfg->stage_bytes : 0)) + 128 + 2 * kMaxStages * sizeof(uint64_t);
         };
-        while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
+        while (stages > 2 && smem_for(stages) > kMaxSmemBytes) --stages;      // a ring deeper than shared memory holds is cut back
         const size_t smem = smem_for(stages);
-        if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-        const int dev = p->device;                   // current: the apply entry points have checked it
-        {
-            std::lock_guard<std::mutex> lock(g_config_mutex);
-            if (dev != cfg->cache_device) {
-                cfg->smem_allowed = 0; cfg->smem_allowed_wrap = 0; cfg->occ_smem = 0; cfg->cache_device = dev;
-            }
-            size_t& allowed = wrap ? cfg->smem_allowed_wrap : cfg->smem_allowed;
-            if (smem > allowed) {
-                if (cudaFuncSetAttribute(wrap ? cfg->kernel_wrap : cfg->kernel,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
-                    cudaGetLastError();
-                    return STENCIL_ERR_CUDA;
-                }
-                allowed = smem;
-            }
-        }
+        if (smem > kMaxSmemBytes) return STENCIL_ERR_UNSUPPORTED;
+        // resident CTAs per SM of the kernel this launch runs, asked once per device and size
+        const int occ64 = wrap ? kernel_limits(cfg->kernel_wrap, cfg->threads, smem, p->device, cfg->lim_wrap, true)
+                               : kernel_limits(cfg->kernel, cfg->threads, smem, p->device, cfg->lim, true);
+        if (occ64 < 0) return STENCIL_ERR_CUDA;
         StreamGeom g;
         g.nz = p->nz; g.ny = p->ny; g.nx = p->nx;
         g.tiles_x = (p->nx + kStream64TX - 1) / kStream64TX;
@@ -302,20 +265,6 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         // planes per chunk, so they get longer chunks (measured on 512^3)
         const int want_chunk = p->radius >= 3 ? 64 : 32;
         int chunk = p->chunk_z > 0 ? p->chunk_z : (span >= 2 * want_chunk ? want_chunk : span);
-        int occ64 = 1;                                // resident CTAs per SM, asked once per device and size
-        {
-            std::lock_guard<std::mutex> lock(g_config_mutex);
-            if (cfg->occ_smem != smem) {
-                int o = 0;
-                if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, cfg->kernel, cfg->threads, smem) != cudaSuccess) {
-                    cudaGetLastError();
-                    o = 0;
-                }
-                cfg->occ = std::max(o, 1);
-                cfg->occ_smem = smem;
-            }
-            occ64 = cfg->occ;
-        }
         const int64_t tiles64 = (int64_t)g.tiles_x * g.tiles_y, slots64 = (int64_t)occ64 * plan_sms(p);
         if (p->chunk_z <= 0 && p->shape == STENCIL_STAR && p->radius == 1 && span >= 16) {
             chunk = short_chunk_star1(span, tiles64, slots64);      // the 7-point star: very short chunks, as in fp32
@@ -373,22 +322,10 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         if (rc != STENCIL_OK) return rc;
         int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
         auto smem_for = [&](int s_) { return (size_t)cfg->NW * s_ * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8; };
-        while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
+        while (stages > 2 && smem_for(stages) > kMaxSmemBytes) --stages;      // a ring deeper than shared memory holds is cut back
         const size_t smem = smem_for(stages);
-        if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-        const int dev = p->device;                   // current: the apply entry points have checked it
-        {
-            std::lock_guard<std::mutex> lock(g_config_mutex);
-            if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->cache_device = dev; }
-            if (smem > cfg->smem_allowed) {
-                if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                    cudaSuccess) {
-                    cudaGetLastError();
-                    return STENCIL_ERR_CUDA;
-                }
-                cfg->smem_allowed = smem;
-            }
-        }
+        if (smem > kMaxSmemBytes) return STENCIL_ERR_UNSUPPORTED;
+        if (kernel_limits(cfg->kernel, cfg->NW * 32, smem, p->device, cfg->lim, false) < 0) return STENCIL_ERR_CUDA;
         Rows2DGeom g;
         g.ny = p->ny; g.nx = p->nx;
         g.strips = (p->nx + kStrip64 - 1) / kStrip64;

@@ -22,7 +22,6 @@ FusedConfig make_fused_e() {
     c.txe = S::TXE; c.tye = S::TYE; c.threads = S::THREADS; c.slot_bytes = S::SLOT_BYTES; c.pw = S::PW;
     c.kernel = reinterpret_cast<const void*>(&stencil_fused_kernel<E, R, T, K, XW, NWY, 0>);
     c.kernel_spec = reinterpret_cast<const void*>(&stencil_fused_kernel<E, R, T, K, XW, NWY, 1>);
-    c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
     c.launch = &launch_fused_t<E, R, T, K, XW, NWY, 0>;
     c.launch_spec = &launch_fused_t<E, R, T, K, XW, NWY, 1>;
     c.kernel_wrap = nullptr; c.launch_wrap = nullptr;
@@ -184,41 +183,16 @@ int launch_fused(stencil_plan_s* p, const void* src, void* dst, int nlev, cudaSt
     // shared memory: input ring + two planes per intermediate level
     int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 2;   // measured: 2 beats 3 and 4
     auto smem_for = [&](int s) { return (size_t)(s + 2 * (T - 1)) * cfg->slot_bytes + 128 + kMaxStages * sizeof(uint64_t); };
-    while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;
+    while (stages > 2 && smem_for(stages) > kMaxSmemBytes) --stages;
     const size_t smem = smem_for(stages);
-    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
+    if (smem > kMaxSmemBytes) return STENCIL_ERR_UNSUPPORTED;
     g.stages = stages;
     const int tiles = g.tiles_x * g.tiles_y;
-    int occ = 1;
-    {
-        // shared-memory limit and occupancy of the kernel, asked once per device and size
-        const int dev = p->device;                   // current: the apply entry points have checked it
-        std::lock_guard<std::mutex> lock(g_config_mutex);
-        if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->occ_smem = 0; cfg->cache_device = dev; }
-        if (smem > cfg->smem_allowed) {
-            if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                    cudaSuccess ||
-                cudaFuncSetAttribute(cfg->kernel_spec, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                    cudaSuccess ||
-                (cfg->kernel_wrap &&
-                 cudaFuncSetAttribute(cfg->kernel_wrap, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                     cudaSuccess)) {
-                cudaGetLastError();
-                return STENCIL_ERR_CUDA;
-            }
-            cfg->smem_allowed = smem;
-        }
-        if (cfg->occ_smem != smem) {
-            int o = 0;
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, cfg->kernel, cfg->threads, smem) != cudaSuccess) {
-                cudaGetLastError();
-                o = 0;
-            }
-            cfg->occ = std::max(o, 1);
-            cfg->occ_smem = smem;
-        }
-        occ = cfg->occ;
-    }
+    // shared-memory limit of the three instantiations and occupancy of the general one, asked once per device and size
+    const int occ = kernel_limits(cfg->kernel, cfg->threads, smem, p->device, cfg->lim, true);
+    if (occ < 0 || kernel_limits(cfg->kernel_spec, cfg->threads, smem, p->device, cfg->lim_spec, false) < 0 ||
+        (cfg->kernel_wrap && kernel_limits(cfg->kernel_wrap, cfg->threads, smem, p->device, cfg->lim_wrap, false) < 0))
+        return STENCIL_ERR_CUDA;
     int chunk = p->chunk_z;
     if (chunk <= 0) {
         // The kernel is bound by instruction issue, so every SM should get the same number of

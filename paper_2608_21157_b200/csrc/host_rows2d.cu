@@ -21,7 +21,6 @@ Rows2DConfig make_rows2d() {
     c.px = StreamHalo<R>::PX;
     c.batch_bytes = Rows2DShape<YB, StreamHalo<R>::PX>::BATCH_BYTES;
     c.kernel = reinterpret_cast<const void*>(&stencil_rows2d_kernel<R, BOX, YB, NW>);
-    c.smem_allowed = 0; c.cache_device = -1;
     c.launch = &launch_rows2d_t<R, BOX, YB, NW>;
     return c;
 }
@@ -62,7 +61,6 @@ Rows2DFusedConfig make_rows2d_fused() {
     Rows2DFusedConfig c;
     c.radius = R; c.box = BOX; c.T = T; c.YB = YB; c.NW = NW; c.batch_bytes = Rows2DShape<YB>::BATCH_BYTES;
     c.kernel = reinterpret_cast<const void*>(&stencil_rows2d_fused_kernel<R, BOX, T, YB, NW>);
-    c.smem_allowed = 0; c.occ_smem = 0; c.occ = 0; c.cache_device = -1;
     c.launch = &launch_rows2d_fused_t<R, BOX, T, YB, NW>;
     return c;
 }
@@ -120,22 +118,10 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     if (rc != STENCIL_OK) return rc;
     int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 3;
     auto smem_for = [&](int s_) { return (size_t)cfg->NW * s_ * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8; };
-    while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
+    while (stages > 2 && smem_for(stages) > kMaxSmemBytes) --stages;      // a ring deeper than shared memory holds is cut back
     const size_t smem = smem_for(stages);
-    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-    const int dev = p->device;                       // current: the apply entry points have checked it
-    {
-        std::lock_guard<std::mutex> lock(g_config_mutex);
-        if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->cache_device = dev; }
-        if (smem > cfg->smem_allowed) {
-            if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess) {
-                cudaGetLastError();
-                return STENCIL_ERR_CUDA;
-            }
-            cfg->smem_allowed = smem;
-        }
-    }
+    if (smem > kMaxSmemBytes) return STENCIL_ERR_UNSUPPORTED;
+    if (kernel_limits(cfg->kernel, cfg->NW * 32, smem, p->device, cfg->lim, false) < 0) return STENCIL_ERR_CUDA;
     Rows2DGeom g;
     g.ny = p->ny; g.nx = p->nx;
     g.strips = (p->nx + kStreamTX - 1) / kStreamTX;
@@ -181,33 +167,11 @@ int launch_rows2d_fused(stencil_plan_s* p, const float* src, float* dst, int nle
     // updates/s against 1671 with three batches and 1214 with four)
     int stages = p->stages > 0 ? std::min(p->stages, kMaxStages) : 2;
     auto smem_for = [&](int s_) { return (size_t)cfg->NW * s_ * cfg->batch_bytes + 128 + (size_t)cfg->NW * kMaxStages * 8; };
-    while (stages > 2 && smem_for(stages) > 227 * 1024) --stages;      // a ring deeper than shared memory holds is cut back
+    while (stages > 2 && smem_for(stages) > kMaxSmemBytes) --stages;      // a ring deeper than shared memory holds is cut back
     const size_t smem = smem_for(stages);
-    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-    const int dev = p->device;                       // current: the apply entry points have checked it
-    int occ = 1;
-    {
-        std::lock_guard<std::mutex> lock(g_config_mutex);
-        if (dev != cfg->cache_device) { cfg->smem_allowed = 0; cfg->occ_smem = 0; cfg->cache_device = dev; }
-        if (smem > cfg->smem_allowed) {
-            if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess) {
-                cudaGetLastError();
-                return STENCIL_ERR_CUDA;
-            }
-            cfg->smem_allowed = smem;
-        }
-        if (cfg->occ_smem != smem) {
-            int o = 0;
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, cfg->kernel, cfg->NW * 32, smem) != cudaSuccess) {
-                cudaGetLastError();
-                o = 0;
-            }
-            cfg->occ = std::max(o, 1);
-            cfg->occ_smem = smem;
-        }
-        occ = cfg->occ;
-    }
+    if (smem > kMaxSmemBytes) return STENCIL_ERR_UNSUPPORTED;
+    const int occ = kernel_limits(cfg->kernel, cfg->NW * 32, smem, p->device, cfg->lim, true);
+    if (occ < 0) return STENCIL_ERR_CUDA;
     Rows2DFusedGeom g;
     g.ny = p->ny; g.nx = p->nx;
     g.strips = (p->nx + kFused2DTile - 1) / kFused2DTile;

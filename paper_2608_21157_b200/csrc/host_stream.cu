@@ -32,12 +32,9 @@ StreamConfig make_cfg() {
     c.radius = R; c.box = BOX; c.K = K; c.NW = NW; c.tile_y = S::TY;
     c.plane_bytes = S::PLANE_BYTES; c.box_rows = S::ROWS; c.threads = S::THREADS;
     c.px = StreamHalo<R>::PX;
-    for (int& o : c.occupancy) o = 0;
-    c.smem_allowed = 0;
-    c.cache_device = -1;
     c.kernel = reinterpret_cast<const void*>(&stencil_stream_kernel<R, BOX, K, NW, MINB>);
     c.launch = &launch_stream_t<R, BOX, K, NW, MINB>;
-    c.kernel_wrap = nullptr; c.launch_wrap = nullptr; c.stage_bytes = 0; c.smem_allowed_wrap = 0;
+    c.kernel_wrap = nullptr; c.launch_wrap = nullptr; c.stage_bytes = 0;
     if constexpr (R <= 4) {
         c.kernel_wrap = reinterpret_cast<const void*>(&stencil_stream_wrap_kernel<R, BOX, K, NW, MINB>);
         c.launch_wrap = &launch_stream_wrap_t<R, BOX, K, NW, MINB>;
@@ -89,34 +86,12 @@ size_t stream_smem_bytes(const StreamConfig* cfg, int stages) {
     return (size_t)stages * cfg->plane_bytes + 128 + 2 * kMaxStages * sizeof(uint64_t);
 }
 
-// Resident CTAs per SM of a configuration at a given ring depth (asked once).
-int stream_occupancy(const StreamConfig* cfg, int stages) {
+// Resident CTAs per SM of a configuration at a given ring depth on the plan's device (asked once per size),
+// -1 if the ring does not fit shared memory.
+int stream_occupancy(const stencil_plan_s* p, const StreamConfig* cfg, int stages) {
     const size_t smem = stream_smem_bytes(cfg, stages);
-    if (smem > 227 * 1024) return -1;
-    std::lock_guard<std::mutex> lock(g_config_mutex);
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return -1; }
-    if (dev != cfg->cache_device) {                // function attributes are per device
-        for (int& o : cfg->occupancy) o = 0;
-        cfg->smem_allowed = 0;
-        cfg->smem_allowed_wrap = 0;
-        cfg->cache_device = dev;
-    }
-    if (smem > cfg->smem_allowed) {                // the limit only ever grows
-        if (cudaFuncSetAttribute(cfg->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
-            cudaGetLastError();
-            return -1;
-        }
-        cfg->smem_allowed = smem;
-    }
-    if (cfg->occupancy[stages] != 0) return cfg->occupancy[stages];
-    int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, cfg->kernel, cfg->threads, smem) != cudaSuccess) {
-        cudaGetLastError();
-        occ = 0;
-    }
-    cfg->occupancy[stages] = occ > 0 ? occ : -1;
-    return cfg->occupancy[stages];
+    if (smem > kMaxSmemBytes) return -1;
+    return kernel_limits(cfg->kernel, cfg->threads, smem, p->device, cfg->lim, true);
 }
 
 // The sweeps with few FMAs per point are bound by HBM: there many short CTAs work
@@ -153,7 +128,7 @@ int choose_chunk(const stencil_plan_s* p, const StreamConfig* cfg, int stages, d
     const int R = p->radius;
     const int nz = span > 0 ? span : p->nz;      // planes this launch covers
     const int tiles = ((p->nx + kStreamTX - 1) / kStreamTX) * ((p->ny + cfg->tile_y - 1) / cfg->tile_y);
-    const int occ = std::max(1, stream_occupancy(cfg, stages));
+    const int occ = std::max(1, stream_occupancy(p, cfg, stages));
     const int slots = occ * plan_sms(p);
     if (!issue_bound(p)) {
         // measured on 512^3: 32-plane chunks (several thousand short CTAs) beat every longer chunk
@@ -221,23 +196,8 @@ int launch_stream_wrap(stencil_plan_s* p, const StreamConfig* cfg, int stages, c
         map_cs = *m;
     }
     const size_t smem = (size_t)stages * (cfg->plane_bytes + cfg->stage_bytes) + 128 + 2 * kMaxStages * sizeof(uint64_t);
-    if (smem > 227 * 1024) return STENCIL_ERR_UNSUPPORTED;
-    const int dev = p->device;                       // current: the apply entry points have checked it
-    {
-        std::lock_guard<std::mutex> lock(g_config_mutex);
-        if (dev != cfg->cache_device) {
-            cfg->smem_allowed = 0; cfg->smem_allowed_wrap = 0; cfg->cache_device = dev;
-            for (int& o : cfg->occupancy) o = 0;
-        }
-        if (smem > cfg->smem_allowed_wrap) {
-            if (cudaFuncSetAttribute(cfg->kernel_wrap, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess) {
-                cudaGetLastError();
-                return STENCIL_ERR_CUDA;
-            }
-            cfg->smem_allowed_wrap = smem;
-        }
-    }
+    if (smem > kMaxSmemBytes) return STENCIL_ERR_UNSUPPORTED;
+    if (kernel_limits(cfg->kernel_wrap, cfg->threads, smem, p->device, cfg->lim_wrap, false) < 0) return STENCIL_ERR_CUDA;
     StreamGeom g;
     g.in_off_x = g.in_off_y = g.in_off_z = 0;
     g.nz = p->nz; g.ny = p->ny; g.nx = p->nx;
@@ -245,7 +205,7 @@ int launch_stream_wrap(stencil_plan_s* p, const StreamConfig* cfg, int stages, c
     g.tiles_y = (p->ny + cfg->tile_y - 1) / cfg->tile_y;
     g.stages = stages;
     g.streaming_store = p->streaming_store;
-    if (stream_occupancy(cfg, stages) <= 0) return STENCIL_ERR_UNSUPPORTED;
+    if (stream_occupancy(p, cfg, stages) <= 0) return STENCIL_ERR_UNSUPPORTED;
     int chunk = p->chunk_z > 0 ? p->chunk_z : choose_chunk(p, cfg, stages, nullptr, p->nz);
     chunk = std::max(1, std::min(chunk, p->nz));
     g.chunk_z = chunk;
@@ -283,7 +243,7 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
         double best = 1e300;
         for (const StreamConfig& c : stream_configs()) {
             if (c.radius != p->radius || c.box != (p->shape == STENCIL_BOX) || c.K != p->stream_cfg->K) continue;
-            if (stream_occupancy(&c, stages) <= 0) continue;
+            if (stream_occupancy(p, &c, stages) <= 0) continue;
             double cost = 0;
             choose_chunk(p, &c, stages, &cost);
             if (cost < best * 0.98) { best = cost; best_cfg = &c; }
@@ -316,7 +276,7 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     g.stages = stages;
     g.streaming_store = p->streaming_store;
     const int tiles = g.tiles_x * g.tiles_y;
-    if (stream_occupancy(cfg, stages) <= 0) return STENCIL_ERR_UNSUPPORTED;
+    if (stream_occupancy(p, cfg, stages) <= 0) return STENCIL_ERR_UNSUPPORTED;
     int chunk = p->chunk_z > 0 ? p->chunk_z : choose_chunk(p, cfg, stages, nullptr, span);
     chunk = std::max(1, std::min(chunk, span));
     g.chunk_z = chunk;
