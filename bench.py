@@ -602,7 +602,10 @@ def run_sharded(args):
     from paper_2608_21157_b200 import build as build_mod
     from paper_2608_21157_b200.sharded import ShardedSweep
 
-    os.environ.setdefault("NCCL_DEBUG", "INFO")         # the communicator log stays on: it shows the transport
+    # the communicator log stays on (it shows the transport each pair of ranks uses), on stderr so that stdout
+    # keeps the one JSON line
+    os.environ.setdefault("NCCL_DEBUG", "INFO")
+    os.environ.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
     rank, world, dist = init_ranks(torch, sharded=True)
     if rank == 0:
         build_mod.build()
