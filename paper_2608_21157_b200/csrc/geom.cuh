@@ -21,16 +21,20 @@ struct StreamGeom {
     int drop_plane;             // test hook: the producer never loads this plane of a CTA (-1: none)
 };
 
-struct FusedGeom {
+// (a multiple of 16 bytes, so that the kernel parameters behind it keep their 16-byte alignment: without it the
+// fused kernels take four more registers)
+struct alignas(16) FusedGeom {
     int nz, ny, nx;
     int tiles_x, tiles_y;
     int tile_x, tile_y;        // output tile (interior) size
     int halo_x, halo_y;        // region = tile + 2*halo; halo_x is a multiple of 4
-    int chunk_z;
+    int chunk_z;               // planes per CTA over planes [0, nz - rest_z) of every region: main_ctas CTAs
     int stages;
     int nlev;                  // time steps advanced by this pass, 1..T
     unsigned wait_polls;       // cap of every bounded wait
     int drop_plane;            // test hook: a CTA never loads its input plane of this index (-1: none)
+    int rest_z, rest_chunk;    // the last rest_z planes of every region go to further CTAs, rest_chunk planes each
+    int main_ctas;             // (rest_z > 0 only for the kernels of more than 256 threads: one CTA per SM)
 };
 
 struct Rows2DGeom {

@@ -22,6 +22,7 @@
 #include <cstdint>
 #include <cstdlib>
 #include <cstring>
+#include <functional>
 #include <mutex>
 #include <new>
 #include <utility>
@@ -230,6 +231,9 @@ struct stencil_plan_s {
     float* pad2;                   // second padded-row grid
     int tmap_nx;                   // non-zero while a padded-row sweep runs: the true row length
     int periodic_route;            // knob: 0 = by measured cost, 1 = padded copy, 2 = wrap correction where it fits
+    // the z cut of the fused passes, found once per configuration and view of the grid
+    struct FusedSchedule { const void* cfg = nullptr; int nz = 0, tiles = 0, slots = 0, chunk = 0, rest = 0, rest_chunk = 1; };
+    FusedSchedule fused_schedule;
     bool fused_wrap;               // set for one launch_fused call: the pass wraps x and z in the kernel
     bool stream_wrap;              // set while a periodic apply sweeps with the kernel that wraps all three axes
     bool src_padded;               // set while an iterated periodic apply runs: the source of a sweep is

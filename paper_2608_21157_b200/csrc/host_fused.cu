@@ -193,30 +193,77 @@ int launch_fused(stencil_plan_s* p, const void* src, void* dst, int nlev, cudaSt
     if (occ < 0 || kernel_limits(cfg->kernel_spec, cfg->threads, smem, p->device, cfg->lim_spec, false) < 0 ||
         (cfg->kernel_wrap && kernel_limits(cfg->kernel_wrap, cfg->threads, smem, p->device, cfg->lim_wrap, false) < 0))
         return STENCIL_ERR_CUDA;
-    int chunk = p->chunk_z;
-    if (chunk <= 0) {
-        // The kernel is bound by instruction issue, so every SM should get the same number of
-        // planes: cut z into the number of chunks whose CTAs fill whole waves of the machine's
-        // resident-CTA slots at the least total cost, a chunk costing its planes plus the
-        // 2*T*R extra input planes and the start-up of its pipeline.
-        const int slots = occ * plan_sms(p);
+    int chunk = p->chunk_z, rest = 0, rest_chunk = 1;
+    const int slots = occ * plan_sms(p);
+    stencil_plan_s::FusedSchedule& memo = p->fused_schedule;
+    if (chunk <= 0 && memo.cfg == cfg && memo.nz == p->nz && memo.tiles == tiles && memo.slots == slots) {
+        chunk = memo.chunk; rest = memo.rest; rest_chunk = memo.rest_chunk;
+    } else if (chunk <= 0) {
+        // The kernel is bound by instruction issue, so every SM should be busy to the end: cut z into the chunks
+        // whose CTAs keep the machine's resident-CTA slots busy at the least total cost, a chunk costing its
+        // planes plus the 2*T*R extra input planes and the start-up of its pipeline.  Equal chunks fill whole
+        // waves of the slots only where the regions divide them (512^3 in 43 regions of 512 x 16: three chunks per
+        // region occupy 129 of 148 SMs).  Otherwise the last `rest` planes of every region are cut into shorter
+        // chunks, whose CTAs come last in the grid: the hardware hands them to the SMs that the main chunks
+        // leave idle, and to the others as they finish.  The cost of a candidate is the makespan of that order.
+        const double ovh = 2 * T * R + 4.0;
         const int max_chunks = std::max(1, p->nz / (4 * T * R));
-        const double fill = 4.0;
+        std::vector<double> free_at;
+        auto makespan = [&](int64_t n_main, double a, int64_t n_tail, double b) {
+            const int64_t w = n_main / slots, q = n_main % slots;
+            if (n_tail == 0) return (double)(w + (q ? 1 : 0)) * a;
+            free_at.assign((size_t)slots, (double)w * a);
+            for (int64_t i = 0; i < q; ++i) free_at[(size_t)i] += a;
+            std::make_heap(free_at.begin(), free_at.end(), std::greater<double>());
+            double end = 0;
+            for (int64_t i = 0; i < n_tail; ++i) {
+                std::pop_heap(free_at.begin(), free_at.end(), std::greater<double>());
+                free_at.back() += b;
+                end = std::max(end, free_at.back());
+                std::push_heap(free_at.begin(), free_at.end(), std::greater<double>());
+            }
+            for (double t : free_at) end = std::max(end, t);
+            return end;
+        };
         double best = 1e300;
         int best_n = 1;
         for (int n = 1; n <= max_chunks; ++n) {
             const int c = (p->nz + n - 1) / n;
             const int real_n = (p->nz + c - 1) / c;
-            const int64_t ctas = (int64_t)tiles * real_n;
-            const double waves = (double)((ctas + slots - 1) / slots);
-            const double cost = waves * (c + 2 * T * R + fill);
+            const double cost = makespan((int64_t)tiles * real_n, c + ovh, 0, 0);
             if (cost < best * 0.999) { best = cost; best_n = real_n; }
         }
         chunk = (p->nz + best_n - 1) / best_n;
+        // (grids of many waves are balanced already, and the search below is per candidate linear in the CTAs)
+        // ... and with two CTAs per SM the slots are not independent: a CTA alone on its SM runs faster, which
+        // evens out a ragged last wave by itself (256^3: every such cut measured slower than equal chunks)
+        if ((int64_t)tiles * best_n <= 8 * (int64_t)slots && occ == 1 && cfg->threads > 256) {
+            double best_tail = 1e300;
+            int t_chunk = 0, t_rest = 0, t_rc = 1;
+            for (int k = 1; k <= 4; ++k) {
+                const int n = (int)std::min<int64_t>((int64_t)k * slots / tiles, max_chunks);    // main chunks per region
+                if (n < 1) continue;
+                for (int r = 8; r <= p->nz / 2 && p->nz - r >= n * 4 * T * R; r += 2)
+                    for (int m = 1; m <= 2; ++m) {
+                        const int c = (p->nz - r + n - 1) / n, rc = (r + m - 1) / m;
+                        const int64_t n_main = (int64_t)tiles * ((p->nz - r + c - 1) / c);
+                        const int64_t n_tail = (int64_t)tiles * ((r + rc - 1) / rc);
+                        const double cost = makespan(n_main, c + ovh, n_tail, rc + ovh);
+                        if (cost < best_tail) { best_tail = cost; t_chunk = c; t_rest = r; t_rc = rc; }
+                    }
+            }
+            if (best_tail < best * 0.97) { chunk = t_chunk; rest = t_rest; rest_chunk = t_rc; }
+        }
+        memo.cfg = cfg; memo.nz = p->nz; memo.tiles = tiles; memo.slots = slots;
+        memo.chunk = chunk; memo.rest = rest; memo.rest_chunk = rest_chunk;
     }
-    chunk = std::max(1, std::min(chunk, p->nz));
+    chunk = std::max(1, std::min(chunk, p->nz - rest));
     g.chunk_z = chunk;
-    const int64_t grid64 = (int64_t)tiles * ((p->nz + chunk - 1) / chunk);
+    g.rest_z = rest;
+    g.rest_chunk = rest_chunk;
+    const int64_t main_ctas = (int64_t)tiles * ((p->nz - rest + chunk - 1) / chunk);
+    const int64_t grid64 = main_ctas + (int64_t)tiles * ((rest + rest_chunk - 1) / rest_chunk);
+    g.main_ctas = (int)std::min<int64_t>(main_ctas, 0x7fffffffLL);
     if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
     // full passes over rows of exactly one region take the instantiation with those facts compiled in
     // ... and the one that also wraps x and z when the pass belongs to a periodic apply (fused_wrap_ok tells

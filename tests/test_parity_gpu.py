@@ -1123,6 +1123,22 @@ def test_baseline_config_full_size(name):
         assert got.min() >= 0.0 and got.max() <= a.max()
 
 
+@pytest.mark.parametrize("boundary", [b.ZERO, b.PERIODIC])
+def test_fused_passes_whose_last_planes_go_to_short_chunks(boundary):
+    """256 x 512 x 512, two steps per pass in 43 regions of 512 x 16, one CTA per SM: three equal chunks
+    per region would occupy 129 of a B200's 148 SMs, so the launcher cuts the last planes of every region
+    into shorter chunks whose CTAs come last in the grid.  Every point of two passes against the oracle;
+    the output starts as NaN, so a plane that no chunk covers shows."""
+    dims, R, steps = (256, 512, 512), 1, 4
+    w = wl.random_star_weights(3, R, 311)
+    a = wl.normal_field(dims, 312)
+    got, used = gpu_sweep(dims, R, b.STAR, w, boundary, a, steps)
+    want = oracle.apply(a, w, boundary, steps)
+    tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+    err = float(np.max(np.abs(got - want)))
+    assert err <= tol, f"{used}: max err {err:.3e} > tol {tol:.3e}"
+
+
 def test_paper_workload_full_grid_one_step():
     """The paper's grid at full size (10240 x 10240, 49-point box), one time step, every
     point against the oracle, in the launch configuration the benchmark times."""
