@@ -109,8 +109,8 @@ const FusedConfig* pick_fused_region(const stencil_plan_s* p) {
     if ((p->fuse_steps == 0 || p->fuse_steps == 2) && txe == 0 && p->fused_tile_y == 0) {
         // Default: fuse two steps per pass when one region spans a whole row (no redundant
         // columns) and the row fills at least 80 % of the region's lanes.  Regions are 128, 256
-        // (two CTAs per SM, which cover each other's barrier stalls: 16-row regions beat 32-row
-        // ones, 922 vs 846 G updates/s on 256^3) or 512 columns wide (one CTA per SM, each plane
+        // (16 rows high with two CTAs per SM, which cover each other's barrier stalls, or 32 rows
+        // high: see `height` below) or 512 columns wide (one CTA per SM, each plane
         // loaded as two TMA boxes).  With several regions per row the halo recomputation costs
         // more than the saved traffic, and idle lanes cost what they would compute, so other
         // grids stay unfused unless the caller asks for fusion.  Measured (G updates/s, fused
@@ -131,7 +131,12 @@ const FusedConfig* pick_fused_region(const stencil_plan_s* p) {
         };
         int width = p->nx <= 128 ? 128 : p->nx <= 256 ? 256 : p->nx <= 384 ? 384 : 512;
         if (p->nx > 512 && 1.25 * lanes_used(384) >= lanes_used(512)) width = 384;
-        const int height = width == 128 ? 0 : width == 384 ? 20 : 16;
+        // 256-wide regions are 16 rows high (two CTAs per SM) on grids of fewer than 448 rows and 32 rows high (one
+        // CTA per SM, 28 of 32 rows stored instead of 12 of 16) from there on, where the taller regions' fewer
+        // CTAs still cut evenly (G updates/s, 16 / 32 rows, nz x ny x 256: 256 x 256: 1163 / 1093, 256 x 384:
+        // 1270 / 1245, 256 x 448: 1224 / 1302, 256 x 512: 1235 / 1300, 256 x 1024: 1330 / 1477, 512 x 512: 1329 /
+        // 1413, 512 x 256: 1300 / 1258)
+        const int height = width == 128 ? 0 : width == 384 ? 20 : (width == 256 && p->ny >= 448) ? 32 : 16;
         // the 384-wide regions pay off from fewer used lanes: any row of 257..384 points (nx = 260:
         // 838 vs 676), three quarters of the lanes with several regions per row (896: 983 vs 843)
         const double need = width != 384 ? 0.8 : p->nx <= 384 ? 0.0 : 0.75;

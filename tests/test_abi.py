@@ -223,6 +223,13 @@ def test_fuse_knob_rules():
         assert p.get(b.KEY_FUSE_STEPS) == 1
         with pytest.raises(b.StencilError):
             p.set(b.KEY_FUSE_STEPS, 7)
+    with b.Plan((64, 448, 256), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2         # from 448 rows on the 256-wide regions are 32 rows high
+        assert p.get(b.KEY_TILE_X) == 256 and p.get(b.KEY_FUSED_TILE_Y) == 32
+        p.set(b.KEY_FUSED_TILE_Y, 16)
+        assert p.get(b.KEY_FUSED_TILE_Y) == 16
+    with b.Plan((64, 444, 256), 1, b.STAR, star, b.ZERO) as p:
+        assert p.get(b.KEY_FUSED_TILE_Y) == 16
     with b.Plan((64, 64, 64), 1, b.BOX, wl.random_box_weights(3, 1, 3), b.ZERO) as p:
         assert p.get(b.KEY_FUSE_STEPS) == 1         # no fused kernel for box stencils
         with pytest.raises(b.StencilError):

@@ -1124,6 +1124,22 @@ def test_baseline_config_full_size(name):
 
 
 @pytest.mark.parametrize("boundary", [b.ZERO, b.PERIODIC])
+def test_default_fused_passes_of_a_tall_256_wide_grid(boundary):
+    """From 448 rows on a 256-wide grid takes 256 x 32 regions by default (one CTA per SM): an odd number
+    of steps, so that a single step follows the fused passes, against the oracle."""
+    dims, R, steps = (24, 452, 256), 1, 5
+    w = wl.random_star_weights(3, R, 321)
+    a = wl.normal_field(dims, 322)
+    with b.Plan(dims, R, b.STAR, w, boundary) as p:
+        assert p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_FUSED_TILE_Y) == 32
+    got, used = gpu_sweep(dims, R, b.STAR, w, boundary, a, steps)
+    want = oracle.apply(a, w, boundary, steps)
+    tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+    err = float(np.max(np.abs(got - want)))
+    assert err <= tol, f"{used}: max err {err:.3e} > tol {tol:.3e}"
+
+
+@pytest.mark.parametrize("boundary", [b.ZERO, b.PERIODIC])
 def test_fused_passes_whose_last_planes_go_to_short_chunks(boundary):
     """256 x 512 x 512, two steps per pass in 43 regions of 512 x 16, one CTA per SM: three equal chunks
     per region would occupy 129 of a B200's 148 SMs, so the launcher cuts the last planes of every region
