@@ -329,8 +329,11 @@ int apply_periodic_fused(stencil_plan_s* p, const T* in, T* out, T* other, int s
             const int xchunks = (g.nx + kShellRowChunk - 1) / kShellRowChunk;
             const int64_t nrows = (int64_t)g.nz * 2 * H * xchunks;
             if (ntaps <= kShellTaps && nrows <= 0x7fffffffLL) {
-                if (launch_kernel(&stencil_shell_rows_kernel<T>, (int)nrows, 256, 0, st, p->chain_launches, src, dst, g, H,
-                                  0, taps, ntaps, xchunks) != cudaSuccess)
+                const bool small = p->npoints + 2 * (int64_t)p->nx < 0x7fffffffLL;    // room for an index before its wrap
+                if ((small ? launch_kernel(&stencil_shell_rows_kernel<T, int>, (int)nrows, 256, 0, st, p->chain_launches,
+                                           src, dst, g, H, 0, taps, ntaps, xchunks)
+                           : launch_kernel(&stencil_shell_rows_kernel<T, int64_t>, (int)nrows, 256, 0, st,
+                                           p->chain_launches, src, dst, g, H, 0, taps, ntaps, xchunks)) != cudaSuccess)
                     return STENCIL_ERR_CUDA;
                 p->launches++;
                 done += L;
@@ -356,7 +359,10 @@ int apply_periodic_fused(stencil_plan_s* p, const T* in, T* out, T* other, int s
         if (p->ndim == 3 && ntaps <= kShellTaps && seg_bytes <= 40 * 1024 && g.nx >= 64 && nrows <= 0x7fffffffLL &&
             xtiles <= 0x7fffffffLL) {
             if (nrows > 0) {
-                stencil_shell_rows_kernel<T><<<(int)nrows, 256, 0, st>>>(src, dst, g, H, hz, taps, ntaps, xchunks);
+                if (p->npoints + 2 * (int64_t)p->nx < 0x7fffffffLL)
+                    stencil_shell_rows_kernel<T, int><<<(int)nrows, 256, 0, st>>>(src, dst, g, H, hz, taps, ntaps, xchunks);
+                else
+                    stencil_shell_rows_kernel<T, int64_t><<<(int)nrows, 256, 0, st>>>(src, dst, g, H, hz, taps, ntaps, xchunks);
                 if (cudaGetLastError() != cudaSuccess) return STENCIL_ERR_CUDA;
                 p->launches++;
             }

@@ -265,17 +265,19 @@ stencil_shell_compose_kernel(const T* __restrict__ in, T* __restrict__ out, Grid
 constexpr int kShellTaps = 160;
 constexpr int kShellRowChunk = 512;
 
-template <typename T>
+template <typename T, typename I>
 struct ShellRowTap {
-    int64_t base;          // index of the cell the tap reads for x = 0 (dx included)
+    I base;                // index of the cell the tap reads for x = 0 (dx included)
     T w;
 };
 
-template <typename T>
+// I: int where every index of the grid fits (a tap then costs a shared load, one address and a load and an FMA per
+// point), int64_t beyond.
+template <typename T, typename I>
 __global__ void __launch_bounds__(256)
 stencil_shell_rows_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g, int H, int hz,
                           const TapT<double>* __restrict__ taps, int ntaps, int xchunks) {
-    __shared__ ShellRowTap<T> s_tap[kShellTaps];
+    __shared__ ShellRowTap<T, I> s_tap[kShellTaps];
     __shared__ int s_dx[kShellTaps];
     const int r = blockIdx.x / xchunks;
     const int xbegin = (int)(blockIdx.x % xchunks) * kShellRowChunk;
@@ -297,7 +299,7 @@ stencil_shell_rows_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g,
         // every extent is at least 2H >= |offset|: one step brings the index back
         qz = qz < 0 ? qz + g.nz : (qz >= g.nz ? qz - g.nz : qz);
         qy = qy < 0 ? qy + g.ny : (qy >= g.ny ? qy - g.ny : qy);
-        s_tap[t].base = ((int64_t)qz * g.ny + qy) * g.nx + tap.dx;
+        s_tap[t].base = (I)(((int64_t)qz * g.ny + qy) * g.nx + tap.dx);
         s_tap[t].w = (T)tap.w;
         s_dx[t] = tap.dx;
     }
@@ -307,7 +309,22 @@ stencil_shell_rows_kernel(const T* __restrict__ in, T* __restrict__ out, Grid g,
     allow_dependents();
     dependency_wait();
     T* orow = out + ((int64_t)z * g.ny + y) * g.nx;
-    for (int x = xbegin + threadIdx.x; x < xend; x += blockDim.x) {
+    int x = xbegin + threadIdx.x;
+    // two points of the row per trip where both lie between the row's ends: they share the tap's shared load
+    for (; x >= H && x + (int)blockDim.x < min(xend, g.nx - H); x += 2 * blockDim.x) {
+        const T* px = in + x;
+        const T* py = px + blockDim.x;
+        T a0 = T(0), a1 = T(0);
+#pragma unroll 4
+        for (int t = 0; t < ntaps; ++t) {
+            const ShellRowTap<T, I> tap = s_tap[t];
+            a0 = fma_t(tap.w, px[tap.base], a0);
+            a1 = fma_t(tap.w, py[tap.base], a1);
+        }
+        orow[x] = a0;
+        orow[x + blockDim.x] = a1;
+    }
+    for (; x < xend; x += blockDim.x) {
         T acc = T(0);
         if (x >= H && x < g.nx - H) {
             const T* px = in + x;
