@@ -50,7 +50,8 @@ enum {
     STENCIL_ERR_CUDA        = -3,  /* a CUDA runtime/driver call failed (or no device)           */
     STENCIL_ERR_ALLOC       = -4,  /* host or device allocation failed                           */
     STENCIL_ERR_TIMEOUT     = -5,  /* a bounded device-side wait gave up (see query_status)      */
-    STENCIL_ERR_TOO_LARGE   = -6   /* grid larger than stencil_apply_static's fixed scratch      */
+    STENCIL_ERR_TOO_LARGE   = -6,  /* grid larger than stencil_apply_static's fixed scratch      */
+    STENCIL_ERR_BOUNDS      = -7   /* debug build only: a kernel's store fell outside the output  */
 };
 
 /* Largest grid, in points, that stencil_apply_static accepts (8 MiB of fp32). */
@@ -108,10 +109,20 @@ enum {
                                       rows) of this index, so the bounded wait for it expires and
                                       stencil_query_status reports STENCIL_ERR_TIMEOUT; nothing
                                       faults (-1 = off, the default)                             */
-    STENCIL_KEY_DEVICE       = 15    /* get: the CUDA device the plan's device state lives on
+    STENCIL_KEY_DEVICE       = 15,   /* get: the CUDA device the plan's device state lives on
                                       (the one current at its first apply; -1 before that).
                                       Later applies must run with that device current
                                       (STENCIL_ERR_INVALID otherwise)                            */
+    STENCIL_KEY_DEBUG_SHRINK = 16    /* set/get, debug builds of the library only (compiled with
+                                      -DSTENCIL_DEBUG; STENCIL_ERR_UNSUPPORTED otherwise, which
+                                      is also how a caller tells the two builds apart).  A debug
+                                      build checks every global store of the tiled kernels
+                                      against the extent of the output grid; a store outside it
+                                      is skipped and stencil_query_status reports
+                                      STENCIL_ERR_BOUNDS.  This test hook makes the checks take
+                                      the grid to be `value` points shorter than it is (0, the
+                                      default: its true extent), so that the stores to its last
+                                      points trip them; nothing faults                           */
 };
 
 /*
@@ -280,7 +291,9 @@ STENCIL_API const char* stencil_variant_name(int variant);
  * stencil_query_status — wait for the stream of the plan's last apply and
  * return the device status word: STENCIL_OK, or STENCIL_ERR_TIMEOUT if a
  * bounded wait inside a kernel expired (the kernel then returned early and
- * `out` is not valid).  The word is cleared by the query.
+ * `out` is not valid), or, from a debug build of the library,
+ * STENCIL_ERR_BOUNDS if a kernel skipped a store that fell outside the output
+ * grid (see STENCIL_KEY_DEBUG_SHRINK).  The word is cleared by the query.
  */
 STENCIL_API int stencil_query_status(stencil_plan_t plan);
 

@@ -4,6 +4,10 @@ Argument marshalling only: every sweep runs in the CUDA kernels of
 ``libstencil_b200.so``.  There is no CPU fallback; if the library has not been
 built, loading raises.  Device memory and streams come from the caller
 (PyTorch in the tests and the benchmark).
+
+With ``STENCIL_B200_DEBUG=1`` in the environment the binding loads the debug
+build, ``libstencil_b200_debug.so`` (``python -m paper_2608_21157_b200.build
+--debug``), whose kernels check every store against the output grid.
 """
 from __future__ import annotations
 
@@ -14,19 +18,21 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libstencil_b200.so")
+DEBUG_BUILD = os.environ.get("STENCIL_B200_DEBUG", "0") == "1"
+LIB_PATH = os.path.join(_HERE, "libstencil_b200_debug.so" if DEBUG_BUILD else "libstencil_b200.so")
 
 STAR, BOX = 0, 1
 ZERO, PERIODIC = 0, 1
 
-OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_ALLOC, ERR_TIMEOUT, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6
+OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_ALLOC, ERR_TIMEOUT, ERR_TOO_LARGE, ERR_BOUNDS = 0, -1, -2, -3, -4, -5, -6, -7
 STATIC_MAX_POINTS = 1 << 21
 
 VARIANT_AUTO, VARIANT_GENERIC, VARIANT_STREAM, VARIANT_FUSED = 0, 1, 2, 3
 
 (KEY_VARIANT, KEY_TILE_X, KEY_TILE_Y, KEY_FUSE_STEPS, KEY_LAUNCHES, KEY_SCRATCH_BYTES,
  KEY_CHUNK_Z, KEY_STAGES, KEY_STREAMING_STORE, KEY_ROWS_PER_THREAD, KEY_WAIT_POLLS,
- KEY_TEST_DROP_PLANE, KEY_CHAIN_LAUNCHES, KEY_FUSED_TILE_Y, KEY_PERIODIC_ROUTE, KEY_DEVICE) = range(16)
+ KEY_TEST_DROP_PLANE, KEY_CHAIN_LAUNCHES, KEY_FUSED_TILE_Y, KEY_PERIODIC_ROUTE, KEY_DEVICE,
+ KEY_DEBUG_SHRINK) = range(17)
 
 #: every symbol include/stencil.h declares
 EXPORTS = (
@@ -53,7 +59,8 @@ def load() -> ctypes.CDLL:
         return _lib
     if not os.path.exists(LIB_PATH):
         raise RuntimeError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2608_21157_b200.build` "
+            f"{LIB_PATH} is missing: build it with `python -m paper_2608_21157_b200.build"
+            f"{' --debug' if DEBUG_BUILD else ''}` "
             "(there is no CPU fallback)")
     lib = ctypes.CDLL(LIB_PATH)
     vp, i64p, f32p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_float)

@@ -92,7 +92,7 @@ int make_plan(stencil_plan_t* plan_out, int ndim, const int64_t* dims, int radiu
     p->npoints = n;
     p->radius = radius; p->shape = shape; p->boundary = boundary;
     p->device = -1; p->sms = 0;
-    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0; p->src_padded = false; p->fused_wrap = false; p->stream_wrap = false; p->periodic_route = 0;
+    p->d_taps = nullptr; p->d_status = nullptr; p->scratch = nullptr; p->pad = nullptr; p->pad2 = nullptr; p->tmap_nx = 0; p->src_padded = false; p->fused_wrap = false; p->stream_wrap = false; p->debug_shrink = 0; p->periodic_route = 0;
     for (int l = 0; l <= kMaxFuseLevels; ++l) p->d_ctaps[l] = nullptr;
     p->d_taps64 = nullptr; p->scratch64 = nullptr; p->rows2d64_cfg = nullptr; p->stream64_cfg = nullptr; p->fused2d64_cfg = nullptr; p->fused64_cfg = nullptr;
     p->host_in = nullptr; p->host_out = nullptr;
@@ -518,6 +518,7 @@ const char* stencil_status_string(int status) {
         case STENCIL_ERR_ALLOC: return "allocation failed";
         case STENCIL_ERR_TIMEOUT: return "bounded device wait expired";
         case STENCIL_ERR_TOO_LARGE: return "grid exceeds the fixed scratch of stencil_apply_static";
+        case STENCIL_ERR_BOUNDS: return "a store outside the output grid was skipped (debug build)";
         default: return "unknown status";
     }
 }
@@ -542,7 +543,7 @@ int stencil_query_status(stencil_plan_t p) {
         cudaGetLastError();
         return STENCIL_ERR_CUDA;
     }
-    return word == 0 ? STENCIL_OK : STENCIL_ERR_TIMEOUT;
+    return word == 0 ? STENCIL_OK : word == stencil::kStatusBounds ? STENCIL_ERR_BOUNDS : STENCIL_ERR_TIMEOUT;
 }
 
 int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
@@ -660,6 +661,14 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
             if (value < -1 || value > 0x7fffffff) return STENCIL_ERR_INVALID;
             p->drop_plane = (int)value;
             return STENCIL_OK;
+        case STENCIL_KEY_DEBUG_SHRINK:
+#ifdef STENCIL_DEBUG
+            if (value < 0 || value > p->npoints) return STENCIL_ERR_INVALID;
+            p->debug_shrink = value;
+            return STENCIL_OK;
+#else
+            return STENCIL_ERR_UNSUPPORTED;
+#endif
         default:
             return STENCIL_ERR_INVALID;
     }
@@ -713,6 +722,13 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
         case STENCIL_KEY_DEVICE: *value = p->device; return STENCIL_OK;
         case STENCIL_KEY_WAIT_POLLS: *value = p->wait_polls; return STENCIL_OK;
         case STENCIL_KEY_TEST_DROP_PLANE: *value = p->drop_plane; return STENCIL_OK;
+        case STENCIL_KEY_DEBUG_SHRINK:
+#ifdef STENCIL_DEBUG
+            *value = p->debug_shrink;
+            return STENCIL_OK;
+#else
+            return STENCIL_ERR_UNSUPPORTED;
+#endif
         default: return STENCIL_ERR_INVALID;
     }
 }

@@ -61,5 +61,24 @@ struct Grid {
 
 // Value of the plan's device status word once a bounded wait has given up.
 constexpr int kStatusTimeout = -5;
+constexpr int kStatusBounds = -7;
+
+// Debug builds (compiled with -DSTENCIL_DEBUG) check every global store of the tiled kernels against the extent
+// of the output grid: a store of n elements at p that would not lie inside [out, out + g.out_points) is skipped
+// and recorded in the status word (STENCIL_ERR_BOUNDS at the next stencil_query_status).  Release builds compile
+// the check away.
+template <typename E, typename G>
+__device__ __forceinline__ bool store_in_grid(const E* p, int n, const E* out, const G& g, int* status) {
+#ifdef STENCIL_DEBUG
+    const long long i = p - out;
+    if (i < 0 || i + n > g.out_points) {
+        atomicExch(status, kStatusBounds);
+        return false;
+    }
+#else
+    (void)p; (void)n; (void)out; (void)g; (void)status;
+#endif
+    return true;
+}
 
 }  // namespace stencil

@@ -19,6 +19,9 @@ struct StreamGeom {
                                 // padded copy of the grid (periodic boundary), else 0
     unsigned wait_polls;        // cap of every bounded wait
     int drop_plane;             // test hook: the producer never loads this plane of a CTA (-1: none)
+#ifdef STENCIL_DEBUG
+    long long out_points;       // debug build: the extent of the output grid that every store is checked against
+#endif
 };
 
 // (a multiple of 16 bytes, so that the kernel parameters behind it keep their 16-byte alignment: without it the
@@ -35,6 +38,9 @@ struct alignas(16) FusedGeom {
     int drop_plane;            // test hook: a CTA never loads its input plane of this index (-1: none)
     int rest_z, rest_chunk;    // the last rest_z planes of every region go to further CTAs, rest_chunk planes each
     int main_ctas;             // (rest_z > 0 only for the kernels of more than 256 threads: one CTA per SM)
+#ifdef STENCIL_DEBUG
+    long long out_points;       // debug build: the extent of the output grid that every store is checked against
+#endif
 };
 
 struct Rows2DGeom {
@@ -47,6 +53,9 @@ struct Rows2DGeom {
     int y_begin, y_end;         // output rows of this launch (the whole grid: 0, ny)
     unsigned wait_polls;        // cap of every bounded wait
     int drop_batch;             // test hook: a warp never loads its input batch of this index (-1: none)
+#ifdef STENCIL_DEBUG
+    long long out_points;       // debug build: the extent of the output grid that every store is checked against
+#endif
 };
 
 struct Rows2DFusedGeom {
@@ -58,6 +67,9 @@ struct Rows2DFusedGeom {
     int nlev;                   // time steps advanced by this pass, 1..T
     unsigned wait_polls;        // cap of every bounded wait
     int drop_batch;             // test hook: a warp never loads its input batch of this index (-1: none)
+#ifdef STENCIL_DEBUG
+    long long out_points;       // debug build: the extent of the output grid that every store is checked against
+#endif
 };
 
 }  // namespace stencil

@@ -249,6 +249,8 @@ struct stencil_plan_s {
     bool chained;                  // set by the apply loop for those launches
     unsigned wait_polls;           // cap of the bounded device waits
     int drop_plane;                // test hook, -1 = off
+    int64_t debug_shrink;          // debug builds, test hook: the store checks take the output grid to be this many
+                                   // points shorter than it is
     const stencil_host::StreamConfig* stream_cfg;
     bool stream_cfg_fixed;         // the caller chose the tile shape
     bool stream_cfg_tuned;         // the library has chosen it for this grid
@@ -267,6 +269,14 @@ struct stencil_plan_s {
 };
 
 namespace stencil_host {
+
+// Debug builds: the extent that a launch's stores are checked against (the grid as the plan sees it now).
+#ifdef STENCIL_DEBUG
+#define STENCIL_SET_OUT_POINTS(g, p) \
+    ((g).out_points = (long long)(p)->nz * (p)->ny * (p)->nx - (long long)(p)->debug_shrink)
+#else
+#define STENCIL_SET_OUT_POINTS(g, p) ((void)0)
+#endif
 
 inline bool valid_plan(const stencil_plan_s* p) { return p && p->magic == kPlanMagic; }
 

@@ -181,6 +181,7 @@ int launch_rows2d_fused64(stencil_plan_s* p, const double* src, double* dst, int
     g.stages = stages;
     g.nlev = nlev;
     g.wait_polls = p->wait_polls; g.drop_batch = p->drop_plane;
+    STENCIL_SET_OUT_POINTS(g, p);
     int chunk = p->chunk_z;
     if (chunk <= 0) {                                 // same sizing rule as the fp32 kernel
         const int H = nlev * p->radius;
@@ -261,6 +262,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         g.in_off_y = periodic ? p->radius : 0;
         g.in_off_z = periodic ? p->radius : 0;
         g.wait_polls = p->wait_polls; g.drop_plane = p->drop_plane;
+        STENCIL_SET_OUT_POINTS(g, p);
         // many short CTAs, as for the bandwidth-bound fp32 sweeps; the wide stars re-read 2R halo
         // planes per chunk, so they get longer chunks (measured on 512^3)
         const int want_chunk = p->radius >= 3 ? 64 : 32;
@@ -348,6 +350,7 @@ int launch_sweep_f64(stencil_plan_s* p, const double* src, double* dst, cudaStre
         g.nchunks = (span + chunk - 1) / chunk;
         g.y_begin = begin; g.y_end = end;
         g.wait_polls = p->wait_polls; g.drop_batch = p->drop_plane;
+        STENCIL_SET_OUT_POINTS(g, p);
         const int64_t units = (int64_t)g.strips * g.nchunks;
         const int64_t grid64 = (units + cfg->NW - 1) / cfg->NW;
         if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;

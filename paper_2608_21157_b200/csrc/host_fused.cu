@@ -174,6 +174,7 @@ int launch_fused(stencil_plan_s* p, const void* src, void* dst, int nlev, cudaSt
     g.nz = p->nz; g.ny = p->ny; g.nx = p->nx;
     g.nlev = nlev;
     g.wait_polls = p->wait_polls; g.drop_plane = p->drop_plane;
+    STENCIL_SET_OUT_POINTS(g, p);
     if (p->nx <= cfg->txe) {                     // one region spans the row: the x halo is the zero boundary
         g.halo_x = 0; g.tile_x = cfg->txe; g.tiles_x = 1;
     } else {

@@ -148,6 +148,7 @@ int launch_rows2d(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     g.nchunks = (span + chunk - 1) / chunk;
     g.y_begin = y_begin; g.y_end = y_end;
     g.wait_polls = p->wait_polls; g.drop_batch = p->drop_plane;
+    STENCIL_SET_OUT_POINTS(g, p);
     const int64_t units = (int64_t)g.strips * g.nchunks;
     const int64_t grid64 = (units + cfg->NW - 1) / cfg->NW;
     if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
@@ -178,6 +179,7 @@ int launch_rows2d_fused(stencil_plan_s* p, const float* src, float* dst, int nle
     g.stages = stages;
     g.nlev = nlev;
     g.wait_polls = p->wait_polls; g.drop_batch = p->drop_plane;
+    STENCIL_SET_OUT_POINTS(g, p);
     int chunk = p->chunk_z;                          // the streamed axis of a 2D grid is y
     if (chunk <= 0) {
         // A unit reads chunk + 2*nlev*R rows in batches of YB and recomputes the 2*nlev*R extra ones at

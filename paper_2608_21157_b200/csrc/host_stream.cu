@@ -211,6 +211,7 @@ int launch_stream_wrap(stencil_plan_s* p, const StreamConfig* cfg, int stages, c
     g.chunk_z = chunk;
     g.z_begin = 0; g.z_end = p->nz;
     g.wait_polls = p->wait_polls; g.drop_plane = p->drop_plane;
+    STENCIL_SET_OUT_POINTS(g, p);
     const int64_t grid64 = (int64_t)g.tiles_x * g.tiles_y * ((p->nz + chunk - 1) / chunk);
     if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;
     if (cfg->launch_wrap(p, map, map_xs, map_ys, map_cs, dst, g, (int)grid64, smem, st) != cudaSuccess)
@@ -282,6 +283,7 @@ int launch_stream(stencil_plan_s* p, const float* src, float* dst, cudaStream_t 
     g.chunk_z = chunk;
     g.z_begin = z_begin; g.z_end = z_end;
     g.wait_polls = p->wait_polls; g.drop_plane = p->drop_plane;
+    STENCIL_SET_OUT_POINTS(g, p);
     const int nchunks = (span + chunk - 1) / chunk;
     const int64_t grid64 = (int64_t)tiles * nchunks;
     if (grid64 > 0x7fffffffLL) return STENCIL_ERR_UNSUPPORTED;

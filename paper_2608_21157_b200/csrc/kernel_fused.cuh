@@ -296,11 +296,12 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, E* __restrict_
                                 if (warp_all_store) {
 #pragma unroll
                                     for (int k = 0; k < K; ++k)
-                                        *reinterpret_cast<V*>(op + (size_t)k * nx) = e[k];
+                                        if (store_in_grid(op + (size_t)k * nx, NV, out, g, status))
+                                            *reinterpret_cast<V*>(op + (size_t)k * nx) = e[k];
                                 } else {
 #pragma unroll
                                     for (int k = 0; k < K; ++k)
-                                        if ((store_mask >> k) & 1u)
+                                        if (((store_mask >> k) & 1u) && store_in_grid(op + (size_t)k * nx, NV, out, g, status))
                                             *reinterpret_cast<V*>(op + (size_t)k * nx) = e[k];
                                 }
                             }

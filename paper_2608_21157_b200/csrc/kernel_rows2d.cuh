@@ -164,7 +164,7 @@ stencil_rows2d_kernel(const __grid_constant__ CUtensorMap tmap_in, float* __rest
                     A[R - 1] = make_float4(acc[0], acc[1], acc[2], acc[3]);
                 }
                 if (i >= 2 * R) {
-                    if (x_in) *reinterpret_cast<float4*>(op) = done;
+                    if (x_in && store_in_grid(op, 4, out, g, status)) *reinterpret_cast<float4*>(op) = done;
                     op += g.nx;
                 }
             }

@@ -160,7 +160,7 @@ stencil_rows2d_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, double* _
                     A[R - 1] = make_double2(acc[0], acc[1]);
                 }
                 if (i >= 2 * R) {
-                    if (x_in) *reinterpret_cast<double2*>(op) = done;
+                    if (x_in && store_in_grid(op, 2, out, g, status)) *reinterpret_cast<double2*>(op) = done;
                     op += g.nx;
                 }
             }

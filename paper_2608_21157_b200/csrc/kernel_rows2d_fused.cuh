@@ -191,7 +191,7 @@ stencil_rows2d_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, float* 
                     if (!(x_in && yl >= 0 && yl < g.ny)) done = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (l == nlev) {
                         if (yl >= y0 && yl < y1) {
-                            if (x_store) *reinterpret_cast<float4*>(op) = done;
+                            if (x_store && store_in_grid(op, 4, out, g, status)) *reinterpret_cast<float4*>(op) = done;
                             op += g.nx;
                         }
                     } else {

@@ -185,7 +185,7 @@ stencil_rows2d_fused_f64_kernel(const __grid_constant__ CUtensorMap tmap_in, dou
                     if (!(x_in && yl >= 0 && yl < g.ny)) done = make_double2(0.0, 0.0);
                     if (l == nlev) {
                         if (yl >= y0 && yl < y1) {
-                            if (x_store) *reinterpret_cast<double2*>(op) = done;
+                            if (x_store && store_in_grid(op, 2, out, g, status)) *reinterpret_cast<double2*>(op) = done;
                             op += g.nx;
                         }
                     } else {

@@ -444,11 +444,13 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
             if (i >= 2 * R) {
                 if (all_ok) {
 #pragma unroll
-                    for (int k = 0; k < K; ++k) store_f4(op + (size_t)k * g.nx, done[k], streaming);
+                    for (int k = 0; k < K; ++k)
+                        if (store_in_grid(op + (size_t)k * g.nx, 4, out, g, status)) store_f4(op + (size_t)k * g.nx, done[k], streaming);
                 } else {
 #pragma unroll
                     for (int k = 0; k < K; ++k)
-                        if (row_ok[k]) store_f4(op + (size_t)k * g.nx, done[k], streaming);
+                        if (row_ok[k] && store_in_grid(op + (size_t)k * g.nx, 4, out, g, status))
+                            store_f4(op + (size_t)k * g.nx, done[k], streaming);
                 }
                 op += plane_stride;
             }
@@ -566,11 +568,13 @@ stream_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CUtens
                     if (all_ok) {
 #pragma unroll
                         for (int k = 0; k < K; ++k)
-                            store_f4(op + (size_t)k * g.nx, T[k][(u + R + 1) % M], streaming);
+                            if (store_in_grid(op + (size_t)k * g.nx, 4, out, g, status))
+                                store_f4(op + (size_t)k * g.nx, T[k][(u + R + 1) % M], streaming);
                     } else {
 #pragma unroll
                         for (int k = 0; k < K; ++k)
-                            if (row_ok[k]) store_f4(op + (size_t)k * g.nx, T[k][(u + R + 1) % M], streaming);
+                            if (row_ok[k] && store_in_grid(op + (size_t)k * g.nx, 4, out, g, status))
+                                store_f4(op + (size_t)k * g.nx, T[k][(u + R + 1) % M], streaming);
                     }
                     op += plane_stride;
                 }

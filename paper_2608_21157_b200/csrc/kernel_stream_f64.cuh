@@ -263,7 +263,8 @@ stream_f64_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CU
             if (i >= 2 * R) {
 #pragma unroll
                 for (int k = 0; k < K; ++k)
-                    if (row_ok[k]) *reinterpret_cast<double2*>(op + (size_t)k * g.nx) = done[k];
+                    if (row_ok[k] && store_in_grid(op + (size_t)k * g.nx, 2, out, g, status))
+                        *reinterpret_cast<double2*>(op + (size_t)k * g.nx) = done[k];
                 op += plane_stride;
             }
         }
@@ -375,7 +376,8 @@ stream_f64_body(const CUtensorMap& tmap_in, const CUtensorMap& tmap_xs, const CU
                 if (i >= 2 * R) {
 #pragma unroll
                     for (int k = 0; k < K; ++k)
-                        if (row_ok[k]) *reinterpret_cast<double2*>(op + (size_t)k * g.nx) = T[k][(u + R + 1) % M];
+                        if (row_ok[k] && store_in_grid(op + (size_t)k * g.nx, 2, out, g, status))
+                            *reinterpret_cast<double2*>(op + (size_t)k * g.nx) = T[k][(u + R + 1) % M];
                     op += plane_stride;
                 }
                 return true;
