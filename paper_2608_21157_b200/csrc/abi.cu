@@ -650,6 +650,10 @@ int stencil_plan_set(stencil_plan_t p, int key, int64_t value) {
                 const FusedConfig* f = pick_fused(p);
                 if (!f && value != 0) { p->fused_tile_y = old; return STENCIL_ERR_UNSUPPORTED; }
                 p->fused_cfg = f;
+            } else if (p->variant == STENCIL_VARIANT_STREAM && p->f64 && p->ndim == 3 && p->stream64_cfg) {
+                const FusedConfig* f = pick_fused64(p);
+                if (!f && value != 0) { p->fused_tile_y = old; return STENCIL_ERR_UNSUPPORTED; }
+                p->fused64_cfg = f;
             }
             return STENCIL_OK;
         }
@@ -717,7 +721,8 @@ int stencil_plan_get(stencil_plan_t p, int key, int64_t* value) {
         case STENCIL_KEY_CHAIN_LAUNCHES: *value = p->chain_launches ? 1 : 0; return STENCIL_OK;
         case STENCIL_KEY_PERIODIC_ROUTE: *value = p->periodic_route; return STENCIL_OK;
         case STENCIL_KEY_FUSED_TILE_Y:
-            *value = (p->variant == STENCIL_VARIANT_STREAM && p->fused_cfg) ? p->fused_cfg->tye : 0;
+            *value = p->variant != STENCIL_VARIANT_STREAM ? 0
+                     : p->f64 ? (p->fused64_cfg ? p->fused64_cfg->tye : 0) : (p->fused_cfg ? p->fused_cfg->tye : 0);
             return STENCIL_OK;
         case STENCIL_KEY_DEVICE: *value = p->device; return STENCIL_OK;
         case STENCIL_KEY_WAIT_POLLS: *value = p->wait_polls; return STENCIL_OK;

@@ -53,13 +53,15 @@ const FusedConfig* find_fused_cfg(int radius, int T, int txe, int tye = 0) {
     return nullptr;
 }
 
-// FP64: a lane holds two doubles, so a warp spans 64 columns and the regions are 128 (two CTAs per SM) or 256
+// FP64: a lane holds two doubles, so a warp spans 64 columns and the regions are 128 (two CTAs per SM, or one of
+// twice the height) or 256
 // columns wide (XW = 4: 512 threads, one CTA per SM); 512 columns would take 1024 threads of 64 registers, which
 // the two accumulators per row and level do not fit.
 const std::vector<FusedConfig>& fused64_configs() {
     static const std::vector<FusedConfig> v = {
         make_fused_e<double, 1, 2, 4, 4, 4>(), make_fused_e<double, 1, 2, 4, 2, 4>(),
         make_fused_e<double, 1, 2, 2, 2, 8>(), make_fused_e<double, 1, 3, 2, 2, 8>(),
+        make_fused_e<double, 1, 2, 4, 2, 8>(),
     };
     return v;
 }
@@ -77,6 +79,10 @@ const FusedConfig* pick_fused64(const stencil_plan_s* p) {
     const int width = p->nx <= 128 ? 128 : p->nx <= 256 ? 256 : 128;
     const int64_t regions = p->nx <= width ? 1 : (p->nx + (width - 8) - 1) / (width - 8);
     const double lanes_used = (double)p->nx / (double)(regions * width);
+    // as in fp32, the 128-wide regions are 32 rows high (one CTA per SM) from 448 rows on: G updates/s, 16 / 32 rows,
+    // nz x ny x nx: 512 x 512 x 128 619 / 666, 256 x 1024 x 128 622 / 708, 256 x 448 x 128 565 / 615, 256 x 384 x 128
+    // 598 / 580, 256 x 256 x 128 530 / 491, 128 x 640 x 640 469 / 501, 512^3 488 / 490
+    const int height = (width == 128 && p->ny >= 448) ? 32 : 16;
     for (const FusedConfig& c : fused64_configs()) {
         if (c.radius != p->radius) continue;
         if (forced) {
@@ -86,7 +92,7 @@ const FusedConfig* pick_fused64(const stencil_plan_s* p) {
             continue;
         }
         // (a caller that asks for two steps per pass gets them on the default width whatever the rows fill)
-        if (c.T == 2 && c.txe == width && (lanes_used >= 0.8 || p->fuse_steps == 2)) return &c;
+        if (c.T == 2 && c.txe == width && c.tye == height && (lanes_used >= 0.8 || p->fuse_steps == 2)) return &c;
     }
     return nullptr;
 }

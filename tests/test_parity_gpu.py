@@ -762,6 +762,27 @@ def test_f64_fused_3d_passes_match_oracle(T, width, dims, chunk_z):
         assert err <= tol, f"T={T} width={width} dims={dims} steps={steps}: {err:.3e} > {tol:.3e}"
 
 
+@pytest.mark.parametrize("dims", [(20, 452, 128), (12, 450, 480)])
+def test_f64_fused_3d_tall_grids_take_32_row_regions(dims):
+    """From 448 rows on the 128-wide FP64 regions are 32 rows high by default (one CTA per SM)."""
+    w = wl.random_star_weights(3, 1, 63, np.float64)
+    a = wl.normal_field(dims, 64, np.float64)
+    steps = 5
+    src = torch.from_numpy(a).cuda()
+    dst = torch.full_like(src, float("nan"))
+    with b.Plan(dims, 1, b.STAR, w, b.ZERO) as p:
+        assert p.f64 and p.get(b.KEY_FUSE_STEPS) == 2 and p.get(b.KEY_FUSED_TILE_Y) == 32
+        p.apply(src, dst, steps, torch.cuda.current_stream().cuda_stream)
+        assert p.query_status() == b.OK and p.launches == 3
+        p.set(b.KEY_FUSED_TILE_Y, 16)
+        assert p.get(b.KEY_FUSED_TILE_Y) == 16
+    got = dst.cpu().numpy()
+    want = oracle.apply(a, w, b.ZERO, steps)
+    tol = wl.tolerance(w, float(np.abs(a).max()), steps)
+    err = float(np.max(np.abs(got - want)))
+    assert err <= tol, f"dims={dims}: {err:.3e} > {tol:.3e}"
+
+
 def test_f64_fused_3d_is_the_default_where_a_region_spans_the_row():
     """Iterated FP64 applies fuse two steps per pass by default on rows that fill 80 % of the lanes of
     their regions (one region of 128 or 256 doubles, or several 128-wide ones on wider rows); other rows,
