@@ -91,7 +91,8 @@ enum {
                                       programmatic dependent launches: each begins its preamble
                                       while its predecessor drains and waits for it before it
                                       touches global memory; 0 = ordinary launches             */
-    STENCIL_KEY_FUSED_TILE_Y = 13,   /* set/get: region height of fused 3D passes, 16, 20 or 32 (0 = auto) */
+    STENCIL_KEY_FUSED_TILE_Y = 13,   /* set/get: region height of fused 3D passes, 16, 20 or 32 (FP64: 16
+                                      or 32); 0 = auto                                           */
     STENCIL_KEY_PERIODIC_ROUTE = 14, /* set/get: how the tiled kernels handle a periodic boundary
                                       where the sweep does not wrap by itself (it does for 3D
                                       stars of radius <= 4 and 3D boxes with nx a multiple of
