@@ -51,7 +51,7 @@ NCU_TRAFFIC_BYTES = {
     "cfg4": 1049.1e6,       # stream kernel, star R=4, 512^3: 557.4 + 491.7
     "cfg5": 99.2e6,         # one fused pass (2 time steps of 256^3): 77.4 + 21.8 (both grids largely stay in L2)
     "cfg5L": 1044.7e6,      # one fused pass (2 time steps of 512^3): 554.7 + 490.0
-    "cfg5L_f64": 2169.1e6,  # one fused pass (2 time steps of 512^3 in FP64): 1136.2 + 1032.8
+    "cfg5L_f64": 2121.4e6,  # one fused pass (2 time steps of 512^3 in FP64): 1093.7 + 1027.7
     "heat2d": 805.9e6,      # one fused pass (4 time steps of 10240^2): 432.9 + 373.0
 }
 
