@@ -37,7 +37,7 @@ struct alignas(16) FusedGeom {
     unsigned wait_polls;       // cap of every bounded wait
     int drop_plane;            // test hook: a CTA never loads its input plane of this index (-1: none)
     int rest_z, rest_chunk;    // the last rest_z planes of every region go to further CTAs, rest_chunk planes each
-    int main_ctas;             // (rest_z > 0 only for the kernels of more than 256 threads: one CTA per SM)
+    int main_ctas;
 #ifdef STENCIL_DEBUG
     long long out_points;       // debug build: the extent of the output grid that every store is checked against
 #endif

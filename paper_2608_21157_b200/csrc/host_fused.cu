@@ -247,9 +247,10 @@ int launch_fused(stencil_plan_s* p, const void* src, void* dst, int nlev, cudaSt
         }
         chunk = (p->nz + best_n - 1) / best_n;
         // (grids of many waves are balanced already, and the search below is per candidate linear in the CTAs)
-        // ... and with two CTAs per SM the slots are not independent: a CTA alone on its SM runs faster, which
-        // evens out a ragged last wave by itself (256^3: every such cut measured slower than equal chunks)
-        if ((int64_t)tiles * best_n <= 8 * (int64_t)slots && occ == 1 && cfg->threads > 256) {
+        // (with two CTAs per SM the slots are not independent, since a CTA alone on its SM runs faster, and the
+        // model rarely finds such a cut 3 % ahead: 256^3 keeps equal chunks, whose hand-picked alternatives all
+        // measured slower; FP64 256 x 320 x 512 takes one, 446 against 423 G updates/s)
+        if ((int64_t)tiles * best_n <= 8 * (int64_t)slots) {
             double best_tail = 1e300;
             int t_chunk = 0, t_rest = 0, t_rc = 1;
             for (int k = 1; k <= 4; ++k) {

@@ -120,18 +120,17 @@ stencil_fused_kernel(const __grid_constant__ CUtensorMap tmap_in, E* __restrict_
     dependency_wait();           // the input is the output of the previous pass
 
     // CTAs are numbered region-fastest.  The first g.main_ctas of them cut planes [0, nz - rest_z) of every
-    // region into chunks of chunk_z planes.  The kernels with one CTA per SM may be given more: those cut the
-    // last rest_z planes into chunks of rest_chunk planes; they are short and come last in the grid, so that
-    // they fill the SMs which the long chunks leave idle in their last wave.
-    constexpr bool TAILS = S::THREADS > 256;
-    const bool tail = TAILS && (int)blockIdx.x >= g.main_ctas;
+    // region into chunks of chunk_z planes.  The launcher may add more: those cut the last rest_z planes into
+    // chunks of rest_chunk planes; they are short and come last in the grid, so that they fill the SMs which
+    // the long chunks leave idle in their last wave.
+    const bool tail = (int)blockIdx.x >= g.main_ctas;
     const int bid = tail ? blockIdx.x - g.main_ctas : blockIdx.x;
     const int tix = bid % g.tiles_x;
     const int tiy = (bid / g.tiles_x) % g.tiles_y;
     const int chunk = bid / (g.tiles_x * g.tiles_y);
     const int x0e = SPEC ? 0 : tix * g.tile_x - g.halo_x;     // region origin (may be negative)
     const int y0e = tiy * g.tile_y - g.halo_y;
-    const int main_z = TAILS ? g.nz - g.rest_z : g.nz;
+    const int main_z = g.nz - g.rest_z;
     const int z0 = tail ? main_z + chunk * g.rest_chunk : chunk * g.chunk_z;
     const int z1 = tail ? min(z0 + g.rest_chunk, g.nz) : min(z0 + g.chunk_z, main_z);
     const int nlev = SPEC ? T : g.nlev;
