@@ -169,6 +169,67 @@ const FusedConfig* pick_fused_region(const stencil_plan_s* p) {
     return find_fused_cfg(p->radius, p->fuse_steps, txe, p->fused_tile_y);
 }
 
+// The z cut of a fused pass: every region (a strip of rows) is cut along z into chunks, one CTA each, handed to
+// the machine's `slots` resident-CTA slots in index order.  The kernel is bound by instruction issue, so every SM
+// should be busy to the end: a chunk costs its planes plus the `halo` (2*T*R) extra input planes and the start-up
+// of its pipeline, and the cut with the least makespan wins.  Equal chunks fill whole waves of the slots only where
+// the regions divide them (512^3 in 43 regions of 512 x 16: three chunks per region occupy 129 of 148 SMs).  So
+// the search also tries cuts whose last `rest` planes per region go to shorter chunks that come last in the grid:
+// the hardware hands those to the SMs that the long chunks leave idle, and to the others as they finish.  Such a
+// cut is taken where it models 3 % ahead of the best equal chunks.  (With two CTAs per SM the slots are not
+// independent, since a CTA alone on its SM runs faster, and the model rarely finds such a cut 3 % ahead: 256^3
+// keeps equal chunks, whose hand-picked alternatives all measured slower; FP64 256 x 320 x 512 takes one, 446
+// against 423 G updates/s.)
+void fused_z_cut(int nz, int tiles, int slots, int halo, int* chunk_out, int* rest_out, int* rest_chunk_out) {
+    const double ovh = halo + 4.0;
+    const int max_chunks = std::max(1, nz / (2 * halo));
+    std::vector<double> free_at;
+    // makespan of n_main CTAs of cost a followed by n_tail CTAs of cost b, each going to the slot that frees first
+    auto makespan = [&](int64_t n_main, double a, int64_t n_tail, double b) {
+        const int64_t w = n_main / slots, q = n_main % slots;
+        if (n_tail == 0) return (double)(w + (q ? 1 : 0)) * a;
+        free_at.assign((size_t)slots, (double)w * a);
+        for (int64_t i = 0; i < q; ++i) free_at[(size_t)i] += a;
+        std::make_heap(free_at.begin(), free_at.end(), std::greater<double>());
+        for (int64_t i = 0; i < n_tail; ++i) {
+            std::pop_heap(free_at.begin(), free_at.end(), std::greater<double>());
+            free_at.back() += b;
+            std::push_heap(free_at.begin(), free_at.end(), std::greater<double>());
+        }
+        return *std::max_element(free_at.begin(), free_at.end());
+    };
+    double best = 1e300;
+    int best_n = 1;
+    for (int n = 1; n <= max_chunks; ++n) {
+        const int c = (nz + n - 1) / n;
+        const int real_n = (nz + c - 1) / c;
+        const double cost = makespan((int64_t)tiles * real_n, c + ovh, 0, 0);
+        if (cost < best * 0.999) { best = cost; best_n = real_n; }
+    }
+    int chunk = (nz + best_n - 1) / best_n, rest = 0, rest_chunk = 1;
+    // (grids of many waves are balanced already, and a candidate costs time linear in its CTAs: the search stays
+    // within about a thousand candidates of a few thousand CTAs)
+    if ((int64_t)tiles * best_n <= 8 * (int64_t)slots) {
+        double best_tail = 1e300;
+        int t_chunk = 0, t_rest = 0, t_rc = 1;
+        const int step = std::max(2, nz / 256);
+        for (int k = 1; k <= 4; ++k) {
+            const int n = (int)std::min<int64_t>((int64_t)k * slots / tiles, max_chunks);    // long chunks per region
+            if (n < 1) continue;
+            for (int r = 8; r <= nz / 2 && nz - r >= n * 2 * halo; r += step)
+                for (int m = 1; m <= 2; ++m) {
+                    const int c = (nz - r + n - 1) / n, rc = (r + m - 1) / m;
+                    const int64_t n_main = (int64_t)tiles * ((nz - r + c - 1) / c);
+                    const int64_t n_tail = (int64_t)tiles * ((r + rc - 1) / rc);
+                    const double cost = makespan(n_main, c + ovh, n_tail, rc + ovh);
+                    if (cost < best_tail) { best_tail = cost; t_chunk = c; t_rest = r; t_rc = rc; }
+                }
+        }
+        if (best_tail < best * 0.97) { chunk = t_chunk; rest = t_rest; rest_chunk = t_rc; }
+    }
+    *chunk_out = chunk; *rest_out = rest; *rest_chunk_out = rest_chunk;
+}
+
 int launch_fused(stencil_plan_s* p, const void* src, void* dst, int nlev, cudaStream_t st) {
     const FusedConfig* cfg = p->f64 ? p->fused64_cfg : p->fused_cfg;
     const CUtensorMap* map = nullptr;
@@ -208,67 +269,12 @@ int launch_fused(stencil_plan_s* p, const void* src, void* dst, int nlev, cudaSt
     int chunk = p->chunk_z, rest = 0, rest_chunk = 1;
     const int slots = occ * plan_sms(p);
     stencil_plan_s::FusedSchedule& memo = p->fused_schedule;
-    if (chunk <= 0 && memo.cfg == cfg && memo.nz == p->nz && memo.tiles == tiles && memo.slots == slots) {
+    if (chunk <= 0) {
+        if (!(memo.cfg == cfg && memo.nz == p->nz && memo.tiles == tiles && memo.slots == slots)) {
+            memo.cfg = cfg; memo.nz = p->nz; memo.tiles = tiles; memo.slots = slots;
+            fused_z_cut(p->nz, tiles, slots, 2 * T * R, &memo.chunk, &memo.rest, &memo.rest_chunk);
+        }
         chunk = memo.chunk; rest = memo.rest; rest_chunk = memo.rest_chunk;
-    } else if (chunk <= 0) {
-        // The kernel is bound by instruction issue, so every SM should be busy to the end: cut z into the chunks
-        // whose CTAs keep the machine's resident-CTA slots busy at the least total cost, a chunk costing its
-        // planes plus the 2*T*R extra input planes and the start-up of its pipeline.  Equal chunks fill whole
-        // waves of the slots only where the regions divide them (512^3 in 43 regions of 512 x 16: three chunks per
-        // region occupy 129 of 148 SMs).  Otherwise the last `rest` planes of every region are cut into shorter
-        // chunks, whose CTAs come last in the grid: the hardware hands them to the SMs that the main chunks
-        // leave idle, and to the others as they finish.  The cost of a candidate is the makespan of that order.
-        const double ovh = 2 * T * R + 4.0;
-        const int max_chunks = std::max(1, p->nz / (4 * T * R));
-        std::vector<double> free_at;
-        auto makespan = [&](int64_t n_main, double a, int64_t n_tail, double b) {
-            const int64_t w = n_main / slots, q = n_main % slots;
-            if (n_tail == 0) return (double)(w + (q ? 1 : 0)) * a;
-            free_at.assign((size_t)slots, (double)w * a);
-            for (int64_t i = 0; i < q; ++i) free_at[(size_t)i] += a;
-            std::make_heap(free_at.begin(), free_at.end(), std::greater<double>());
-            double end = 0;
-            for (int64_t i = 0; i < n_tail; ++i) {
-                std::pop_heap(free_at.begin(), free_at.end(), std::greater<double>());
-                free_at.back() += b;
-                end = std::max(end, free_at.back());
-                std::push_heap(free_at.begin(), free_at.end(), std::greater<double>());
-            }
-            for (double t : free_at) end = std::max(end, t);
-            return end;
-        };
-        double best = 1e300;
-        int best_n = 1;
-        for (int n = 1; n <= max_chunks; ++n) {
-            const int c = (p->nz + n - 1) / n;
-            const int real_n = (p->nz + c - 1) / c;
-            const double cost = makespan((int64_t)tiles * real_n, c + ovh, 0, 0);
-            if (cost < best * 0.999) { best = cost; best_n = real_n; }
-        }
-        chunk = (p->nz + best_n - 1) / best_n;
-        // (grids of many waves are balanced already, and the search below is per candidate linear in the CTAs)
-        // (with two CTAs per SM the slots are not independent, since a CTA alone on its SM runs faster, and the
-        // model rarely finds such a cut 3 % ahead: 256^3 keeps equal chunks, whose hand-picked alternatives all
-        // measured slower; FP64 256 x 320 x 512 takes one, 446 against 423 G updates/s)
-        if ((int64_t)tiles * best_n <= 8 * (int64_t)slots) {
-            double best_tail = 1e300;
-            int t_chunk = 0, t_rest = 0, t_rc = 1;
-            for (int k = 1; k <= 4; ++k) {
-                const int n = (int)std::min<int64_t>((int64_t)k * slots / tiles, max_chunks);    // main chunks per region
-                if (n < 1) continue;
-                for (int r = 8; r <= p->nz / 2 && p->nz - r >= n * 4 * T * R; r += 2)
-                    for (int m = 1; m <= 2; ++m) {
-                        const int c = (p->nz - r + n - 1) / n, rc = (r + m - 1) / m;
-                        const int64_t n_main = (int64_t)tiles * ((p->nz - r + c - 1) / c);
-                        const int64_t n_tail = (int64_t)tiles * ((r + rc - 1) / rc);
-                        const double cost = makespan(n_main, c + ovh, n_tail, rc + ovh);
-                        if (cost < best_tail) { best_tail = cost; t_chunk = c; t_rest = r; t_rc = rc; }
-                    }
-            }
-            if (best_tail < best * 0.97) { chunk = t_chunk; rest = t_rest; rest_chunk = t_rc; }
-        }
-        memo.cfg = cfg; memo.nz = p->nz; memo.tiles = tiles; memo.slots = slots;
-        memo.chunk = chunk; memo.rest = rest; memo.rest_chunk = rest_chunk;
     }
     chunk = std::max(1, std::min(chunk, p->nz - rest));
     g.chunk_z = chunk;
